@@ -1,0 +1,165 @@
+"""Pins for the oracle's element formats, encoder and block scale (no GPU).
+
+Each check compares the oracle with something other than itself: the closed-form grids of the
+OCP element formats, PyTorch's float8 casts (a library), explicit rounding thresholds, and the
+closed form 2^(floor(log2 amax) - emax) of the E8M0 block scale.
+"""
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from oracle import E2M1, E4M3, E5M2
+
+GOLD = os.path.join(os.path.dirname(__file__), "golden")
+FMT = {"E4M3": E4M3, "E5M2": E5M2, "E2M1": E2M1}
+
+
+def test_e2m1_decode_grid():
+    grid = [0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0]
+    for c in range(8):
+        assert oracle.decode_elem(E2M1, c) == grid[c]
+        assert oracle.decode_elem(E2M1, c | 8) == -grid[c]
+    assert math.copysign(1.0, oracle.decode_elem(E2M1, 8)) == -1.0  # 0x8 is -0
+
+
+@pytest.mark.parametrize("fmt,tdtype", [(E4M3, torch.float8_e4m3fn), (E5M2, torch.float8_e5m2)])
+def test_fp8_decode_matches_library_view(fmt, tdtype):
+    codes = torch.arange(256, dtype=torch.uint8)
+    lib = codes.view(tdtype).to(torch.float64).numpy()
+    for c in range(256):
+        v = oracle.decode_elem(fmt, c)
+        if math.isnan(lib[c]):
+            assert math.isnan(v)
+        else:
+            assert v == lib[c], (c, v, lib[c])
+
+
+def test_fp8_landmarks():
+    assert oracle.decode_elem(E4M3, 0x7E) == 448.0
+    assert oracle.decode_elem(E4M3, 0x01) == 2.0 ** -9
+    assert oracle.decode_elem(E4M3, 0x08) == 2.0 ** -6
+    assert oracle.decode_elem(E5M2, 0x7B) == 57344.0
+    assert oracle.decode_elem(E5M2, 0x01) == 2.0 ** -16
+    assert oracle.decode_elem(E5M2, 0x04) == 2.0 ** -14
+    assert math.isinf(oracle.decode_elem(E5M2, 0x7C))
+
+
+@pytest.mark.parametrize("fmt,ncodes,maxc", [(E2M1, 16, 0x7), (E4M3, 256, 0x7E), (E5M2, 256, 0x7B)])
+def test_encode_roundtrip_midpoints_saturation(fmt, ncodes, maxc):
+    half = ncodes // 2
+    for m in range(maxc + 1):
+        for s in (0, half):
+            assert oracle.encode_elem(fmt, oracle.decode_elem(fmt, m | s)) == (m | s)
+    for m in range(maxc):
+        lo, hi = oracle.decode_elem(fmt, m), oracle.decode_elem(fmt, m + 1)
+        assert hi > lo  # monotone in code
+        mid = (lo + hi) / 2
+        even = m if m % 2 == 0 else m + 1
+        assert oracle.encode_elem(fmt, mid) == even
+        assert oracle.encode_elem(fmt, -mid) == (even | half)
+        assert oracle.encode_elem(fmt, np.nextafter(mid, 0.0)) == m
+        assert oracle.encode_elem(fmt, np.nextafter(mid, np.inf)) == m + 1
+    top = oracle.decode_elem(fmt, maxc)
+    for v in (top * 1.0001, top * 1.2, top * 2, 1e30):
+        assert oracle.encode_elem(fmt, v) == maxc
+        assert oracle.encode_elem(fmt, -v) == (maxc | half)
+    assert oracle.encode_elem(fmt, 0.0) == 0
+    assert oracle.encode_elem(fmt, -0.0) == half
+    assert oracle.encode_elem(fmt, -1e-30) == half  # negative underflow keeps the sign
+
+
+def test_e2m1_encode_explicit_thresholds():
+    # (upper bound, inclusive?) -> code ; ties go to the code with an even low bit
+    cases = [(0.2, 0), (0.25, 0), (0.26, 1), (0.74, 1), (0.75, 2), (1.2, 2), (1.25, 2), (1.3, 3), (1.74, 3),
+             (1.75, 4), (2.4, 4), (2.5, 4), (2.6, 5), (3.4, 5), (3.5, 6), (4.9, 6), (5.0, 6), (5.1, 7), (100.0, 7)]
+    for v, code in cases:
+        assert oracle.encode_elem(E2M1, v) == code, v
+        assert oracle.encode_elem(E2M1, -v) == code | 8, v
+
+
+@pytest.mark.parametrize("fmt,tdtype,top", [(E4M3, torch.float8_e4m3fn, 448.0), (E5M2, torch.float8_e5m2, 57344.0)])
+def test_fp8_encode_matches_library_cast(fmt, tdtype, top):
+    rng = np.random.default_rng(7)
+    v = np.concatenate([
+        rng.standard_normal(4000) * rng.choice([1e-4, 1e-2, 1.0, 30.0, 400.0, 5e4], 4000),
+        np.ldexp(rng.uniform(1, 2, 2000), rng.integers(-20, 17, 2000)) * rng.choice([-1, 1], 2000),
+        [0.0, -0.0, top, -top, top * 1.5, -top * 3],
+    ]).astype(np.float32)
+    lib = torch.from_numpy(v).clamp(-top, top).to(tdtype).view(torch.uint8).numpy()
+    for x, c in zip(v, lib):
+        assert oracle.encode_elem(fmt, float(x)) == int(c), (x, c)
+
+
+@pytest.mark.parametrize("fmt,emax", [(E2M1, 2), (E4M3, 8), (E5M2, 15)])
+def test_scale_closed_form(fmt, emax):
+    assert oracle.scale_code(fmt, 0.0) == 0
+    for k in range(-140, 128):
+        for amax in (2.0 ** k, 2.0 ** k * (1 + 2.0 ** -23), 2.0 ** k * (2 - 2.0 ** -22), 2.0 ** k * 1.5):
+            want = min(max(k - emax + 127, 0), 254)
+            assert oracle.scale_code(fmt, amax) == want, (k, amax)
+    # the same through an independent route: integer exponent field of the fp32 encoding
+    rng = np.random.default_rng(3)
+    a = np.abs(rng.standard_normal(2000) * rng.choice([1e-30, 1e-6, 1.0, 1e5, 1e30], 2000)).astype(np.float32)
+    a = a[a >= np.finfo(np.float32).tiny]
+    expo = ((a.view(np.uint32) >> 23) & 0xFF).astype(np.int64)
+    for x, e in zip(a, expo):
+        assert oracle.scale_code(fmt, float(x)) == min(max(int(e) - emax, 0), 254)
+
+
+def _golden_rows():
+    rows = []
+    with open(os.path.join(GOLD, "mx_block_vectors.txt")) as f:
+        for line in f:
+            line = line.strip()
+            if not line or line.startswith("#"):
+                continue
+            fmt, vals, scale, codes, deq = [t.strip() for t in line.split(";")]
+            rows.append((fmt, [float(t) for t in vals.split()], int(scale), [int(t, 16) for t in codes.split()],
+                         [float(t) for t in deq.split()]))
+    return rows
+
+
+@pytest.mark.parametrize("row", _golden_rows(), ids=lambda r: f"{r[0]}-{r[1][0]}")
+@pytest.mark.parametrize("block", [(1, 32), (32, 32)])
+def test_hand_derived_block_vectors(row, block):
+    fname, vals, scale, codes, deq = row
+    fmt = FMT[fname]
+    d = oracle.ConvDesc(1, 32, 1, 1, 32, 1, 1, 1, 1, 0, 0)
+    x = np.zeros((1, 32, 1, 1), np.float32)
+    x[0, : len(vals), 0, 0] = vals
+    c, s = oracle.quantize(d, oracle.ROLE_X, fmt, x, block)
+    assert s.tolist() == [scale]
+    if fmt == E2M1:
+        got = [(c[i // 2] >> (4 * (i % 2))) & 0xF for i in range(len(vals))]
+        assert not c[2:].any()
+    else:
+        got = c[: len(vals)].tolist()
+        assert not c[len(vals):].any()
+    assert got == codes
+    back = oracle.dequant(d, oracle.ROLE_X, fmt, c, s, block)[0, : len(vals), 0, 0]
+    np.testing.assert_allclose(back, deq, rtol=1e-11, atol=0)
+
+
+def test_paper_format_arithmetic():
+    gold = {}
+    with open(os.path.join(GOLD, "paper_format_arithmetic.txt")) as f:
+        for line in f:
+            if line.strip() and not line.startswith("#"):
+                k, v, _ = [t.strip() for t in line.split(";", 2)]
+                gold[k] = float(v)
+    d = oracle.ConvDesc(32, 64, 16, 16, 64, 3, 3, 1, 1, 1, 1)
+    fp32_bytes = 32 * 64 * 16 * 16 * 4
+    cb, sb = oracle.qtensor_sizes(d, oracle.ROLE_X, E2M1, (1, 32))  # 4-bit + one 8-bit scale per 32
+    assert round(fp32_bytes / (cb + sb), 2) == gold["backward_mem_move_fp32_over_4bit"]
+    cb, sb = oracle.qtensor_sizes(d, oracle.ROLE_X, E2M1, (8, 8))  # the paper's 8x8 block
+    elems = 32 * 64 * 16 * 16
+    assert (cb * 8 - elems) / elems + sb * 8 / elems == gold["bits_per_unsigned_fp4_pixel_B64"]  # 3 + 8/64
+    cb8, sb8 = oracle.qtensor_sizes(d, oracle.ROLE_X, E4M3, (8, 8))
+    assert abs(fp32_bytes / (cb8 + sb8) - gold["fp8_gain_over_fp32_B64"]) < 0.01
+    # storing the quantized im2col-expanded tensor instead costs Kh*Kw times more (stride 1, same-size output)
+    icb, isb = oracle.im2col_sizes(d, E2M1, (8, 8))
+    assert icb / cb == gold["act_quantizations_im2col_k3"] and isb / sb == gold["act_quantizations_im2col_k3"]
