@@ -1,0 +1,146 @@
+/* mq.h -- C ABI of the MicroQonv hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, on one GPU, the three parts of a microscaling-quantized convolution
+ * layer's training step as the paper lays them out:
+ *   1. a single-pass MX quantizer applied once each to X, W and G_Y (Sec. III-A, Eq. 5-6; the
+ *      square blocks and per-tensor directions of Sec. IV-B),
+ *   2. the channel-batch-first im2col of the already-quantized activation (Sec. IV-A),
+ *   3. the three block-scaled GEMMs Y, G_X, G_W (Sec. II-C, Sec. IV-B, Eq. 7).
+ *
+ * Conventions common to every call
+ *   - All tensor pointers are DEVICE pointers unless a parameter says "host".  The caller owns
+ *     every buffer, including workspace; the library allocates no device memory.
+ *   - Calls enqueue work on `stream` (a cudaStream_t passed as void*, NULL = default stream) and
+ *     return without synchronising.  Argument errors are detected on the host before anything is
+ *     launched; on error nothing is enqueued and outputs are untouched.
+ *   - Every device buffer must be 16-byte aligned.
+ *   - Problem statement (Sec. II-A): X is N x C_in x H x W, W is C_out x C_in x Kh x Kw, G_Y and Y
+ *     are N x C_out x Ho x Wo with Ho = floor((H + 2 pad_h - Kh) / stride_h) + 1 (likewise Wo).
+ *     Cross-correlation, zero padding, dilation 1, groups 1, no bias.
+ *
+ * Stored MX tensors (the "channel-batch-first" layouts of Sec. IV-A / IV-B; Cp = C rounded up to 32)
+ *   role X : codes [H][W][N][C_in_p],            scales [H][W][ceil(N/32)][C_in_p/32]
+ *   role W : codes [C_out][Kh][Kw][C_in_p],      scales [ceil(C_out/32)][Kh][Kw][C_in_p/32]
+ *   role DY: codes [Ho][Wo][N][C_out_p],         scales [Ho][Wo][ceil(N/32)][C_out_p/32]
+ *   The channel axis is fastest.  E4M3 / E5M2 codes take one byte; E2M1 codes are packed two per
+ *   byte, the lower channel index in bits 3:0.  Padded channels hold code 0.  A scale is one E8M0
+ *   byte (value 2^(code-127)) shared by a 32 x 32 tile: 32 channels x 32 samples (X, DY) or
+ *   32 input x 32 output channels (W) at one spatial / tap position, so that every 32-element
+ *   line of a tile, in either contraction direction, is a standard MX block (Sec. IV-B).
+ */
+#ifndef MQ_H_
+#define MQ_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  MQ_OK = 0,
+  MQ_ERR_INVALID_ARG = 1,      /* null pointer, non-positive dimension, unknown enum value        */
+  MQ_ERR_UNSUPPORTED = 2,      /* a valid request this build does not implement                   */
+  MQ_ERR_ALIGNMENT = 3,        /* a device pointer is not 16-byte aligned                         */
+  MQ_ERR_BUFFER_TOO_SMALL = 4, /* a declared buffer size is smaller than the call needs           */
+  MQ_ERR_CUDA = 5,             /* a CUDA runtime / driver call failed (launch, descriptor encode) */
+  MQ_ERR_TIMEOUT = 6           /* a bounded device-side wait gave up (see mq_last_device_status)  */
+} mq_status;
+
+typedef enum { MQ_E4M3 = 0, MQ_E5M2 = 1, MQ_E2M1 = 2 } mq_elem;        /* element format, Sec. II-D */
+typedef enum { MQ_ROLE_X = 0, MQ_ROLE_W = 1, MQ_ROLE_DY = 2 } mq_role; /* which tensor, Sec. IV-B   */
+typedef enum { MQ_NCHW = 0, MQ_HWNC = 1 } mq_layout;                   /* fp32 tensor layout        */
+typedef enum { MQ_OP_FWD = 0, MQ_OP_BWD_DATA = 1, MQ_OP_BWD_WEIGHT = 2 } mq_op;
+
+/* One convolution layer (Sec. II-A).  block_size must be 32 (the E8M0 block length). */
+typedef struct {
+  int N, C_in, H, W, C_out, Kh, Kw;
+  int stride_h, stride_w, pad_h, pad_w;
+  int block_size;
+} mq_conv_desc;
+
+/* A stored MX tensor: a view of caller-owned device memory, never freed by the library. */
+typedef struct {
+  void* codes;         /* element codes, layout above                 */
+  uint8_t* scales;     /* E8M0 tile scales, layout above              */
+  size_t codes_bytes;  /* size of the codes buffer                    */
+  size_t scales_bytes; /* size of the scales buffer                   */
+  int fmt;             /* mq_elem                                     */
+  int role;            /* mq_role                                     */
+} mq_qtensor;
+
+/* Size queries (host only, no GPU needed). */
+
+/* Bytes of codes and scales of the stored MX tensor of `role` (layouts above). */
+mq_status mq_qtensor_sizes(const mq_conv_desc* desc, int role, int fmt, size_t* codes_bytes, size_t* scales_bytes);
+
+/* Bytes of X'_{Cin,N} (Sec. IV-A): codes [Ho][Wo][N][Kh][Kw][C_in_p], scales [Ho][Wo][ceil(N/32)][Kh][Kw][C_in_p/32]. */
+mq_status mq_im2col_sizes(const mq_conv_desc* desc, int fmt, size_t* codes_bytes, size_t* scales_bytes);
+
+/* Bytes of scratch `op` (mq_op) needs for operand formats fmt_a, fmt_b (in the order of the call's
+ * two mq_qtensor arguments).  May be 0. */
+mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt_b, size_t* bytes);
+
+/* mq_quantize -- Sec. III-A (Eq. 5-6) in the E8M0 form of the original MX format (Sec. II-D), on the
+ * square blocks and in the directions of Sec. IV-B; also re-lays the tensor into its stored order
+ * (Sec. IV-A), so the tensor is read once and quantized once.
+ *   per tile: amax = max |x| over the valid elements; scale code = clamp(floor(log2 amax) - emax
+ *   + 127, 0, 254) (0 if amax = 0); element = round-to-nearest-even(x * 2^(127 - code)) on the
+ *   element format's grid, saturating at its largest finite magnitude, sign kept.
+ * src: fp32, `src_layout` = MQ_NCHW (X: NCHW, W: OIHW, G_Y: N.C_out.Ho.Wo); MQ_HWNC is not
+ * implemented (MQ_ERR_UNSUPPORTED).  dst->codes / dst->scales receive the stored tensor; dst->fmt and
+ * dst->role select format and role; the *_bytes fields must be at least mq_qtensor_sizes().
+ * Non-finite inputs are outside the contract (result unspecified, no fault). */
+mq_status mq_quantize(const mq_conv_desc* desc, const void* src, int src_layout, mq_qtensor* dst, void* stream);
+
+/* mq_cbf_im2col -- channel-batch-first im2col (Sec. IV-A) of the quantized activation `xq` (role X):
+ * row (kh,kw,c), column (ho,wo,n) of X' is the stored code at pixel (ho*stride+kh-pad,
+ * wo*stride+kw-pad); tile scales are gathered alongside; out-of-image taps are zero bytes (codes
+ * and scale).  No arithmetic on values: an element keeps its single quantized value everywhere.
+ * cols_codes / cols_scales: sizes from mq_im2col_sizes(). */
+mq_status mq_cbf_im2col(const mq_conv_desc* desc, const mq_qtensor* xq, void* cols_codes, uint8_t* cols_scales, void* stream);
+
+/* mq_conv_fwd -- Y_{f Cout,N} = W_{f Cout,Cin} . X'_{Cin,N} (Sec. II-C, IV-B; Eq. 1), block-scaled as
+ * Eq. 7 with K-blocks of 32 input channels at one tap; X' is formed on the fly from `xq`.
+ * y: fp32, `y_layout` MQ_NCHW ([N][C_out][Ho][Wo]) or MQ_HWNC ([Ho][Wo][N][C_out]); fp32 accumulation.
+ * workspace: ws_bytes >= mq_workspace_size(desc, MQ_OP_FWD, xq->fmt, wq->fmt) (may be NULL if 0). */
+mq_status mq_conv_fwd(const mq_conv_desc* desc, const mq_qtensor* xq, const mq_qtensor* wq, void* y, int y_layout,
+                      void* workspace, size_t ws_bytes, void* stream);
+
+/* mq_conv_bwd_data -- G_X' = W_f^T . G_Yf followed by the col2im reordering (Sec. II-C, IV-B; Eq. 2):
+ * the exact adjoint of mq_conv_fwd in X, K-blocks of 32 output channels at one tap.
+ * dx: fp32, MQ_NCHW ([N][C_in][H][W]) or MQ_HWNC ([H][W][N][C_in]). */
+mq_status mq_conv_bwd_data(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, void* dx, int dx_layout,
+                           void* workspace, size_t ws_bytes, void* stream);
+
+/* mq_conv_bwd_weight -- G_Wf = G_Yf . X'^T (Sec. II-C, IV-B; Eq. 3), K-blocks of 32 samples at one
+ * output pixel: the stored X and G_Y are read along N, the other direction of their square blocks.
+ * dw: fp32 OIHW ([C_out][C_in][Kh][Kw]) for MQ_NCHW, or [C_out][Kh][Kw][C_in] for MQ_HWNC.
+ * The reduction over (ho,wo,n) is split across thread blocks through `workspace` and summed in a
+ * fixed order (deterministic). */
+mq_status mq_conv_bwd_weight(const mq_conv_desc* desc, const mq_qtensor* xq, const mq_qtensor* dyq, void* dw, int dw_layout,
+                             void* workspace, size_t ws_bytes, void* stream);
+
+/* mq_conv_layer_host -- one whole pass of the path for a layer whose tensors live in HOST memory:
+ * copies X, W, G_Y (fp32; NCHW / OIHW / N.C_out.Ho.Wo; pinned memory makes the copies asynchronous)
+ * into `arena`, runs mq_quantize on each once, mq_cbf_im2col, mq_conv_fwd, mq_conv_bwd_data and
+ * mq_conv_bwd_weight, and copies Y, G_X, G_W (fp32, MQ_NCHW layouts) back to the host buffers.
+ * Everything is enqueued on `stream`; the host results are valid after the stream is synchronised.
+ * arena: device memory, arena_bytes >= mq_conv_layer_host_arena_size(); contents are scratch. */
+mq_status mq_conv_layer_host_arena_size(const mq_conv_desc* desc, int fmt_x, int fmt_w, int fmt_dy, size_t* bytes);
+mq_status mq_conv_layer_host(const mq_conv_desc* desc, int fmt_x, int fmt_w, int fmt_dy, const float* x_host, const float* w_host,
+                             const float* dy_host, float* y_host, float* dx_host, float* dw_host, void* arena, size_t arena_bytes,
+                             void* stream);
+
+/* Human-readable name of a status code (static storage). */
+const char* mq_status_string(int status);
+
+/* Synchronises `stream`, then reads and clears the device-side status word that kernels set when a
+ * bounded wait gives up.  Returns MQ_OK, MQ_ERR_TIMEOUT or MQ_ERR_CUDA. */
+mq_status mq_last_device_status(void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MQ_H_ */

@@ -1,0 +1,301 @@
+// CUDA-core implicit-GEMM kernels for the three block-scaled convolution GEMMs (Sec. II-C, IV-B,
+// Eq. 7).  They accept every shape and every element-format pair and serve the shapes the
+// tensor-core kernels do not cover (thin channel counts, odd geometry).  Operands are decoded
+// exactly (code -> fp16 -> fp32, times the tile's power-of-two scale) into shared memory, one
+// 32-element MX block of K per step, and accumulated in fp32.
+//
+//   fwd        : M = (ho,wo,n)   N = co           K = (kh,kw | ci)   A = X gathered, B = W     both K-contiguous
+//   bwd_data   : M = (h,w,n)     N = ci           K = (kh,kw | co)   A = G_Y gathered (K-contiguous), B = W (N-contiguous)
+//   bwd_weight : M = co          N = (kh,kw,ci)   K = (ho,wo | n)    A = G_Y, B = X gathered   both MN-contiguous
+#include "mq_internal.cuh"
+
+namespace mq {
+namespace {
+
+constexpr int TM = 64, TN = 64, TK = 32, GT = 256, PADF = 4;
+
+struct Tiles {
+  alignas(16) float As[TK][TM + PADF];
+  alignas(16) float Bs[TK][TN + PADF];
+};
+
+__device__ __forceinline__ void store_kmajor(float (*S)[TM + PADF], int row, int kq, const float* v) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) S[kq * 8 + j][row] = v[j];
+}
+__device__ __forceinline__ void store_mnmajor(float (*S)[TM + PADF], int k, int mq, const float* v) {
+  *reinterpret_cast<float4*>(&S[k][mq * 8]) = make_float4(v[0], v[1], v[2], v[3]);
+  *reinterpret_cast<float4*>(&S[k][mq * 8 + 4]) = make_float4(v[4], v[5], v[6], v[7]);
+}
+__device__ __forceinline__ void zero8(float* v) {
+#pragma unroll
+  for (int j = 0; j < 8; ++j) v[j] = 0.f;
+}
+
+__device__ __forceinline__ void mma_tile(const Tiles& sm, int ty, int tx, float acc[4][4]) {
+#pragma unroll
+  for (int k = 0; k < TK; ++k) {
+    float4 a = *reinterpret_cast<const float4*>(&sm.As[k][ty * 4]);
+    float4 b = *reinterpret_cast<const float4*>(&sm.Bs[k][tx * 4]);
+    float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) acc[i][j] = fmaf(av[i], bv[j], acc[i][j]);
+  }
+}
+
+// ------------------------------------------------------------------------------------ forward
+template <int FX, int FW>
+__global__ void __launch_bounds__(GT) fwd_generic(ConvArgs a) {
+  __shared__ Tiles sm;
+  const Geom& g = a.g;
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  const int row_l = tid >> 2, kq = tid & 3;
+  const long long M = (long long)g.Ho * g.Wo * g.N;
+  const long long m0 = (long long)blockIdx.x * TM;
+  const int n0 = blockIdx.y * TN;
+  const int taps = g.Kh * g.Kw;
+
+  const long long m = m0 + row_l;
+  const bool m_ok = m < M;
+  int n = 0, wo = 0, ho = 0;
+  if (m_ok) { n = (int)(m % g.N); long long q = m / g.N; wo = (int)(q % g.Wo); ho = (int)(q / g.Wo); }
+  const int co = n0 + row_l;
+  const bool co_ok = co < g.Cout;
+
+  float acc[4][4] = {};
+  for (int tap = 0; tap < taps; ++tap) {
+    const int kh = tap / g.Kw, kw = tap - kh * g.Kw;
+    const int h = ho * g.sh + kh - g.ph, w = wo * g.sw + kw - g.pw;
+    const bool pix_ok = m_ok && h >= 0 && h < g.H && w >= 0 && w < g.W;
+    const long long pix = (long long)h * g.W + w;
+    for (int kb = 0; kb < g.Ct; ++kb) {
+      float va[8], vb[8];
+      if (pix_ok) {
+        float s = e8m0_to_float(a.a_scales[(pix * g.Nt + (n >> 5)) * g.Ct + kb]);
+        decode8<FX>(a.a_codes, (pix * g.N + n) * g.Cp + kb * 32 + kq * 8, s, va);
+      } else zero8(va);
+      if (co_ok) {
+        float s = e8m0_to_float(a.b_scales[((long long)(co >> 5) * taps + tap) * g.Ct + kb]);
+        decode8<FW>(a.b_codes, ((long long)co * taps + tap) * g.Cp + kb * 32 + kq * 8, s, vb);
+      } else zero8(vb);
+      __syncthreads();
+      store_kmajor(sm.As, row_l, kq, va);
+      store_kmajor(sm.Bs, row_l, kq, vb);
+      __syncthreads();
+      mma_tile(sm, ty, tx, acc);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const long long mm = m0 + ty * 4 + i;
+    if (mm >= M) continue;
+    const int nn = (int)(mm % g.N); const long long q = mm / g.N;
+    const int wwo = (int)(q % g.Wo), hho = (int)(q / g.Wo);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int c = n0 + tx * 4 + j;
+      if (c >= g.Cout) continue;
+      if (a.out_layout == MQ_NCHW) a.out[(((long long)nn * g.Cout + c) * g.Ho + hho) * g.Wo + wwo] = acc[i][j];
+      else a.out[mm * g.Cout + c] = acc[i][j];
+    }
+  }
+}
+
+// --------------------------------------------------------------------------------- input gradient
+template <int FW, int FG>
+__global__ void __launch_bounds__(GT) bwd_data_generic(ConvArgs a) {
+  __shared__ Tiles sm;
+  const Geom& g = a.g;
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  const int row_l = tid >> 2, kq = tid & 3;   // A units: (row, 8 consecutive k)
+  const int k_l = tid >> 3, nq = tid & 7;     // B units: (k, 8 consecutive ci)
+  const long long M = (long long)g.H * g.W * g.N;
+  const long long m0 = (long long)blockIdx.x * TM;
+  const int n0 = blockIdx.y * TN;
+  const int taps = g.Kh * g.Kw;
+
+  const long long m = m0 + row_l;
+  const bool m_ok = m < M;
+  int n = 0, w = 0, h = 0;
+  if (m_ok) { n = (int)(m % g.N); long long q = m / g.N; w = (int)(q % g.W); h = (int)(q / g.W); }
+  const int ci0 = n0 + nq * 8;
+  const bool ci_ok = ci0 < g.Cp;
+
+  float acc[4][4] = {};
+  for (int tap = 0; tap < taps; ++tap) {
+    const int kh = tap / g.Kw, kw = tap - kh * g.Kw;
+    const int hn = h + g.ph - kh, wn = w + g.pw - kw;
+    bool pix_ok = m_ok && hn >= 0 && wn >= 0 && (hn % g.sh) == 0 && (wn % g.sw) == 0;
+    const int ho = hn / g.sh, wo = wn / g.sw;
+    pix_ok = pix_ok && ho < g.Ho && wo < g.Wo;
+    const long long pix = (long long)ho * g.Wo + wo;
+    for (int kb = 0; kb < g.Cot; ++kb) {
+      float va[8], vb[8];
+      if (pix_ok) {
+        float s = e8m0_to_float(a.b_scales[(pix * g.Nt + (n >> 5)) * g.Cot + kb]);
+        decode8<FG>(a.b_codes, (pix * g.N + n) * g.Cop + kb * 32 + kq * 8, s, va);
+      } else zero8(va);
+      const int co = kb * 32 + k_l;
+      if (ci_ok && co < g.Cout) {
+        float s = e8m0_to_float(a.a_scales[((long long)kb * taps + tap) * g.Ct + (ci0 >> 5)]);
+        decode8<FW>(a.a_codes, ((long long)co * taps + tap) * g.Cp + ci0, s, vb);
+      } else zero8(vb);
+      __syncthreads();
+      store_kmajor(sm.As, row_l, kq, va);
+      store_mnmajor(sm.Bs, k_l, nq, vb);
+      __syncthreads();
+      mma_tile(sm, ty, tx, acc);
+    }
+  }
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const long long mm = m0 + ty * 4 + i;
+    if (mm >= M) continue;
+    const int nn = (int)(mm % g.N); const long long q = mm / g.N;
+    const int ww = (int)(q % g.W), hh = (int)(q / g.W);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int c = n0 + tx * 4 + j;
+      if (c >= g.Cin) continue;
+      if (a.out_layout == MQ_NCHW) a.out[(((long long)nn * g.Cin + c) * g.H + hh) * g.W + ww] = acc[i][j];
+      else a.out[mm * g.Cin + c] = acc[i][j];
+    }
+  }
+}
+
+// -------------------------------------------------------------------------------- weight gradient
+// Partial sums over a slice of output pixels go to workspace [split][C_out][taps*Cp]; a second
+// kernel adds the slices in a fixed order and writes G_W in its final layout.
+template <int FX, int FG>
+__global__ void __launch_bounds__(GT) bwd_weight_generic(ConvArgs a, int splits) {
+  __shared__ Tiles sm;
+  const Geom& g = a.g;
+  const int tid = threadIdx.x, ty = tid >> 4, tx = tid & 15;
+  const int k_l = tid >> 3, q8 = tid & 7;
+  const int m0 = blockIdx.x * TM, n0 = blockIdx.y * TN;
+  const int taps = g.Kh * g.Kw;
+  const int J = taps * g.Cp;
+  const int npix = g.Ho * g.Wo;
+  const int split = blockIdx.z;
+  const int pix_begin = (int)((long long)npix * split / splits), pix_end = (int)((long long)npix * (split + 1) / splits);
+
+  const int co0 = m0 + q8 * 8;
+  const bool co_ok = co0 < g.Cop;
+  const int j0 = n0 + q8 * 8;
+  const bool j_ok = j0 < J;
+  const int tap = j_ok ? j0 / g.Cp : 0, ci0 = j_ok ? j0 - tap * g.Cp : 0;
+  const int kh = tap / g.Kw, kw = tap - kh * g.Kw;
+
+  float acc[4][4] = {};
+  for (int pix = pix_begin; pix < pix_end; ++pix) {
+    const int ho = pix / g.Wo, wo = pix - ho * g.Wo;
+    const int h = ho * g.sh + kh - g.ph, w = wo * g.sw + kw - g.pw;
+    const bool x_ok = j_ok && h >= 0 && h < g.H && w >= 0 && w < g.W;
+    const long long xpix = (long long)h * g.W + w;
+    for (int kb = 0; kb < g.Nt; ++kb) {
+      const int n = kb * 32 + k_l;
+      float va[8], vb[8];
+      if (co_ok && n < g.N) {
+        float s = e8m0_to_float(a.b_scales[((long long)pix * g.Nt + kb) * g.Cot + (co0 >> 5)]);
+        decode8<FG>(a.b_codes, ((long long)pix * g.N + n) * g.Cop + co0, s, va);
+      } else zero8(va);
+      if (x_ok && n < g.N) {
+        float s = e8m0_to_float(a.a_scales[(xpix * g.Nt + kb) * g.Ct + (ci0 >> 5)]);
+        decode8<FX>(a.a_codes, (xpix * g.N + n) * g.Cp + ci0, s, vb);
+      } else zero8(vb);
+      __syncthreads();
+      store_mnmajor(sm.As, k_l, q8, va);
+      store_mnmajor(sm.Bs, k_l, q8, vb);
+      __syncthreads();
+      mma_tile(sm, ty, tx, acc);
+    }
+  }
+  float* part = reinterpret_cast<float*>(a.workspace) + (long long)split * g.Cout * J;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    const int co = m0 + ty * 4 + i;
+    if (co >= g.Cout) continue;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int jj = n0 + tx * 4 + j;
+      if (jj < J) part[(long long)co * J + jj] = acc[i][j];
+    }
+  }
+}
+
+__global__ void bwd_weight_reduce(const float* __restrict__ part, float* __restrict__ out, Geom g, int splits, int layout) {
+  const int taps = g.Kh * g.Kw;
+  const long long total = (long long)g.Cout * taps * g.Cin;
+  const long long J = (long long)taps * g.Cp;
+  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
+    // i enumerates the output in its own layout so that writes are coalesced
+    int co, ci, tap;
+    if (layout == MQ_NCHW) { tap = (int)(i % taps); long long q = i / taps; ci = (int)(q % g.Cin); co = (int)(q / g.Cin); }
+    else { ci = (int)(i % g.Cin); long long q = i / g.Cin; tap = (int)(q % taps); co = (int)(q / taps); }
+    const float* p = part + (long long)co * J + (long long)tap * g.Cp + ci;
+    float s = 0.f;
+    for (int k = 0; k < splits; ++k) s += p[(long long)k * g.Cout * J];
+    out[i] = s;
+  }
+}
+
+}  // namespace
+
+int conv_generic_bwd_weight_splits(const Geom& g) {
+  const int taps = g.Kh * g.Kw;
+  const long long tiles = (long long)((g.Cop + TM - 1) / TM) * ((taps * g.Cp + TN - 1) / TN);
+  long long splits = (148LL * 4 + tiles - 1) / tiles;
+  const long long npix = (long long)g.Ho * g.Wo;
+  if (splits > npix) splits = npix;
+  if (splits > 256) splits = 256;
+  if (splits < 1) splits = 1;
+  return (int)splits;
+}
+
+size_t conv_generic_workspace(int op, const Geom& g) {
+  if (op != MQ_OP_BWD_WEIGHT) return 0;
+  return (size_t)conv_generic_bwd_weight_splits(g) * g.Cout * g.Kh * g.Kw * g.Cp * sizeof(float);
+}
+
+#define MQ_DISPATCH2(FA, FB, CALL)                                                         \
+  switch ((FA) * 3 + (FB)) {                                                               \
+    case 0: { constexpr int A_ = 0, B_ = 0; CALL; } break;                                 \
+    case 1: { constexpr int A_ = 0, B_ = 1; CALL; } break;                                 \
+    case 2: { constexpr int A_ = 0, B_ = 2; CALL; } break;                                 \
+    case 3: { constexpr int A_ = 1, B_ = 0; CALL; } break;                                 \
+    case 4: { constexpr int A_ = 1, B_ = 1; CALL; } break;                                 \
+    case 5: { constexpr int A_ = 1, B_ = 2; CALL; } break;                                 \
+    case 6: { constexpr int A_ = 2, B_ = 0; CALL; } break;                                 \
+    case 7: { constexpr int A_ = 2, B_ = 1; CALL; } break;                                 \
+    case 8: { constexpr int A_ = 2, B_ = 2; CALL; } break;                                 \
+    default: return cudaErrorInvalidValue;                                                 \
+  }
+
+cudaError_t launch_conv_generic(int op, const ConvArgs& a, cudaStream_t s) {
+  const Geom& g = a.g;
+  if (op == MQ_OP_FWD) {
+    const long long M = (long long)g.Ho * g.Wo * g.N;
+    dim3 grid((unsigned)((M + TM - 1) / TM), (unsigned)((g.Cout + TN - 1) / TN));
+    MQ_DISPATCH2(a.fmt_a, a.fmt_b, (fwd_generic<A_, B_><<<grid, GT, 0, s>>>(a)));
+  } else if (op == MQ_OP_BWD_DATA) {
+    const long long M = (long long)g.H * g.W * g.N;
+    dim3 grid((unsigned)((M + TM - 1) / TM), (unsigned)((g.Cin + TN - 1) / TN));
+    MQ_DISPATCH2(a.fmt_a, a.fmt_b, (bwd_data_generic<A_, B_><<<grid, GT, 0, s>>>(a)));
+  } else {
+    const int splits = conv_generic_bwd_weight_splits(g);
+    const int J = g.Kh * g.Kw * g.Cp;
+    dim3 grid((unsigned)((g.Cop + TM - 1) / TM), (unsigned)((J + TN - 1) / TN), (unsigned)splits);
+    MQ_DISPATCH2(a.fmt_a, a.fmt_b, (bwd_weight_generic<A_, B_><<<grid, GT, 0, s>>>(a, splits)));
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return e;
+    const long long total = (long long)g.Cout * g.Kh * g.Kw * g.Cin;
+    unsigned blocks = (unsigned)((total + 255) / 256);
+    if (blocks > 148u * 16) blocks = 148u * 16;
+    bwd_weight_reduce<<<blocks, 256, 0, s>>>(reinterpret_cast<const float*>(a.workspace), a.out, g, splits, a.out_layout);
+  }
+  return cudaGetLastError();
+}
+
+}  // namespace mq

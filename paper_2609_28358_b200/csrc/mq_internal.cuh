@@ -1,0 +1,115 @@
+// Internal declarations shared by the library's translation units (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_fp16.h>
+#include <cuda_fp8.h>
+#include <cuda_fp4.h>
+#include <stdint.h>
+
+#include "mq.h"
+
+namespace mq {
+
+// Derived geometry of one layer (Sec. II-A) and of its stored tensors (Sec. IV-A/B).
+struct Geom {
+  int N, Cin, H, W, Cout, Kh, Kw, sh, sw, ph, pw;
+  int Ho, Wo;
+  int Cp, Cop;  // channels rounded up to 32
+  int Nt;       // ceil(N / 32)
+  int Ct, Cot;  // Cp / 32, Cop / 32
+};
+
+inline Geom make_geom(const mq_conv_desc& d) {
+  Geom g;
+  g.N = d.N; g.Cin = d.C_in; g.H = d.H; g.W = d.W; g.Cout = d.C_out; g.Kh = d.Kh; g.Kw = d.Kw;
+  g.sh = d.stride_h; g.sw = d.stride_w; g.ph = d.pad_h; g.pw = d.pad_w;
+  g.Ho = (d.H + 2 * d.pad_h - d.Kh) / d.stride_h + 1;
+  g.Wo = (d.W + 2 * d.pad_w - d.Kw) / d.stride_w + 1;
+  g.Cp = (d.C_in + 31) / 32 * 32;
+  g.Cop = (d.C_out + 31) / 32 * 32;
+  g.Nt = (d.N + 31) / 32;
+  g.Ct = g.Cp / 32;
+  g.Cot = g.Cop / 32;
+  return g;
+}
+
+__host__ __device__ inline int fmt_bits(int fmt) { return fmt == MQ_E2M1 ? 4 : 8; }
+__host__ __device__ inline int fmt_emax(int fmt) { return fmt == MQ_E4M3 ? 8 : (fmt == MQ_E5M2 ? 15 : 2); }
+
+// ---- launchers (defined in the .cu files) ---------------------------------------------------
+struct QuantArgs {
+  const float* src;
+  uint8_t* codes;
+  uint8_t* scales;
+  int P, R, C, Cp;                 // positions, rows of the 2-D view, channels, padded channels
+  long long out_stride_p, out_stride_r;  // in elements of the codes tensor
+  long long sc_stride_p, sc_stride_r;    // in scale bytes
+  int fmt;
+};
+cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s);
+
+struct Im2colArgs {
+  const uint8_t* codes;
+  const uint8_t* scales;
+  uint8_t* out_codes;
+  uint8_t* out_scales;
+  Geom g;
+  int fmt;
+};
+cudaError_t launch_im2col(const Im2colArgs& a, cudaStream_t s);
+
+struct ConvArgs {
+  Geom g;
+  const uint8_t* a_codes;  // first operand of the call (fwd: X, bwd_data: W, bwd_weight: X)
+  const uint8_t* a_scales;
+  const uint8_t* b_codes;  // second operand (fwd: W, bwd_data: G_Y, bwd_weight: G_Y)
+  const uint8_t* b_scales;
+  int fmt_a, fmt_b;
+  float* out;
+  int out_layout;
+  void* workspace;
+  size_t ws_bytes;
+};
+// CUDA-core implicit-GEMM kernels: every shape, every format pair.
+cudaError_t launch_conv_generic(int op, const ConvArgs& a, cudaStream_t s);
+size_t conv_generic_workspace(int op, const Geom& g);
+int conv_generic_bwd_weight_splits(const Geom& g);
+
+// ---- device helpers --------------------------------------------------------------------------
+#ifdef __CUDACC__
+
+// 2^(code-127) as fp32 (code 0 gives the subnormal 2^-127)
+__device__ __forceinline__ float e8m0_to_float(unsigned code) {
+  return code == 0 ? __uint_as_float(0x00400000u) : __uint_as_float(code << 23);
+}
+
+// Exact decode of 8 consecutive codes (K- or MN-contiguous in memory) to fp32, times `scale`.
+template <int FMT>
+__device__ __forceinline__ void decode8(const uint8_t* codes_base, long long elem_off, float scale, float* out) {
+  if (FMT == MQ_E2M1) {
+    uint32_t v = *reinterpret_cast<const uint32_t*>(codes_base + (elem_off >> 1));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      __half2_raw h = __nv_cvt_fp4x2_to_halfraw2((__nv_fp4x2_storage_t)((v >> (8 * i)) & 0xFF), __NV_E2M1);
+      float2 f = __half22float2(*reinterpret_cast<__half2*>(&h));
+      out[2 * i] = f.x * scale;
+      out[2 * i + 1] = f.y * scale;
+    }
+  } else {
+    uint2 v = *reinterpret_cast<const uint2*>(codes_base + elem_off);
+    uint32_t w[2] = {v.x, v.y};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      unsigned short pair = (unsigned short)((w[i >> 1] >> (16 * (i & 1))) & 0xFFFF);
+      __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)pair, FMT == MQ_E4M3 ? __NV_E4M3 : __NV_E5M2);
+      float2 f = __half22float2(*reinterpret_cast<__half2*>(&h));
+      out[2 * i] = f.x * scale;
+      out[2 * i + 1] = f.y * scale;
+    }
+  }
+}
+
+#endif  // __CUDACC__
+
+}  // namespace mq

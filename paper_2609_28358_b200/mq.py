@@ -1,0 +1,184 @@
+"""Python binding of ``libmq.so``: the same names as the C ABI (``include/mq.h``), argument
+marshalling only.  PyTorch supplies device memory and the current CUDA stream; every step of the
+path runs in the library's kernels.  There is no fallback: if the library is missing or a call
+fails, an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from collections import namedtuple
+
+import torch
+
+ConvDesc = namedtuple("ConvDesc", "N C_in H W C_out Kh Kw stride_h stride_w pad_h pad_w")
+
+E4M3, E5M2, E2M1 = 0, 1, 2
+ROLE_X, ROLE_W, ROLE_DY = 0, 1, 2
+NCHW, HWNC = 0, 1
+OP_FWD, OP_BWD_DATA, OP_BWD_WEIGHT = 0, 1, 2
+OK = 0
+
+_LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmq.so")
+_lib = None
+
+
+class MqError(RuntimeError):
+    def __init__(self, call, status):
+        self.status = status
+        super().__init__(f"{call} failed: {status_string(status)} ({status})")
+
+
+class _Desc(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int) for n in
+                ("N", "C_in", "H", "W", "C_out", "Kh", "Kw", "stride_h", "stride_w", "pad_h", "pad_w", "block_size")]
+
+
+class _QTensor(ctypes.Structure):
+    _fields_ = [("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("codes_bytes", ctypes.c_size_t),
+                ("scales_bytes", ctypes.c_size_t), ("fmt", ctypes.c_int), ("role", ctypes.c_int)]
+
+
+def lib():
+    """The loaded C-ABI library.  Raises if it has not been built (python -m paper_2609_28358_b200.build)."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise RuntimeError(f"{_LIB_PATH} is missing: build it with `python -m paper_2609_28358_b200.build`; "
+                               "there is no fallback path")
+        _lib = ctypes.CDLL(_LIB_PATH)
+        _lib.mq_status_string.restype = ctypes.c_char_p
+    return _lib
+
+
+def status_string(status):
+    return lib().mq_status_string(int(status)).decode()
+
+
+def _d(desc, block_size=32):
+    return _Desc(*[int(v) for v in desc], block_size)
+
+
+def _check(call, st):
+    if st != OK:
+        raise MqError(call, st)
+
+
+def _stream(stream):
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return ctypes.c_void_p(stream.cuda_stream)
+
+
+class QTensor:
+    """A stored MX tensor: device uint8 buffers for codes and tile scales."""
+
+    def __init__(self, codes, scales, fmt, role):
+        self.codes, self.scales, self.fmt, self.role = codes, scales, fmt, role
+
+    def _c(self):
+        return _QTensor(self.codes.data_ptr(), self.scales.data_ptr(), self.codes.numel(), self.scales.numel(), self.fmt, self.role)
+
+
+def qtensor_sizes(desc, role, fmt):
+    cb, sb = ctypes.c_size_t(), ctypes.c_size_t()
+    _check("mq_qtensor_sizes", lib().mq_qtensor_sizes(ctypes.byref(_d(desc)), role, fmt, ctypes.byref(cb), ctypes.byref(sb)))
+    return cb.value, sb.value
+
+
+def im2col_sizes(desc, fmt):
+    cb, sb = ctypes.c_size_t(), ctypes.c_size_t()
+    _check("mq_im2col_sizes", lib().mq_im2col_sizes(ctypes.byref(_d(desc)), fmt, ctypes.byref(cb), ctypes.byref(sb)))
+    return cb.value, sb.value
+
+
+def workspace_size(desc, op, fmt_a, fmt_b):
+    b = ctypes.c_size_t()
+    _check("mq_workspace_size", lib().mq_workspace_size(ctypes.byref(_d(desc)), op, fmt_a, fmt_b, ctypes.byref(b)))
+    return b.value
+
+
+def empty_qtensor(desc, role, fmt, device="cuda"):
+    cb, sb = qtensor_sizes(desc, role, fmt)
+    return QTensor(torch.empty(cb, dtype=torch.uint8, device=device), torch.empty(sb, dtype=torch.uint8, device=device), fmt, role)
+
+
+def quantize(desc, role, fmt, src, out=None, src_layout=NCHW, stream=None):
+    """mq_quantize: fp32 device tensor (NCHW / OIHW) -> stored MX tensor."""
+    assert src.is_cuda and src.dtype == torch.float32 and src.is_contiguous()
+    if out is None:
+        out = empty_qtensor(desc, role, fmt, src.device)
+    q = out._c()
+    _check("mq_quantize", lib().mq_quantize(ctypes.byref(_d(desc)), ctypes.c_void_p(src.data_ptr()), src_layout, ctypes.byref(q), _stream(stream)))
+    return out
+
+
+def cbf_im2col(desc, xq, out_codes=None, out_scales=None, stream=None):
+    """mq_cbf_im2col: stored quantized activation -> (codes, scales) of X'."""
+    cb, sb = im2col_sizes(desc, xq.fmt)
+    if out_codes is None:
+        out_codes = torch.empty(cb, dtype=torch.uint8, device=xq.codes.device)
+    if out_scales is None:
+        out_scales = torch.empty(sb, dtype=torch.uint8, device=xq.codes.device)
+    q = xq._c()
+    _check("mq_cbf_im2col", lib().mq_cbf_im2col(ctypes.byref(_d(desc)), ctypes.byref(q), ctypes.c_void_p(out_codes.data_ptr()),
+                                               ctypes.c_void_p(out_scales.data_ptr()), _stream(stream)))
+    return out_codes, out_scales
+
+
+def _out_hw(desc):
+    d = ConvDesc(*desc)
+    return ((d.H + 2 * d.pad_h - d.Kh) // d.stride_h + 1, (d.W + 2 * d.pad_w - d.Kw) // d.stride_w + 1)
+
+
+def _conv(name, op, desc, qa, qb, out, shape_nchw, shape_hwnc, layout, workspace, stream):
+    dev = qa.codes.device
+    if out is None:
+        out = torch.empty(shape_nchw if layout == NCHW else shape_hwnc, dtype=torch.float32, device=dev)
+    need = workspace_size(desc, op, qa.fmt, qb.fmt)
+    if workspace is None and need > 0:
+        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+    wp = ctypes.c_void_p(workspace.data_ptr()) if workspace is not None else None
+    wn = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    a, b = qa._c(), qb._c()
+    fn = getattr(lib(), name)
+    _check(name, fn(ctypes.byref(_d(desc)), ctypes.byref(a), ctypes.byref(b), ctypes.c_void_p(out.data_ptr()), layout, wp,
+                    ctypes.c_size_t(wn), _stream(stream)))
+    return out
+
+
+def conv_fwd(desc, xq, wq, y=None, layout=NCHW, workspace=None, stream=None):
+    d = ConvDesc(*desc)
+    ho, wo = _out_hw(d)
+    return _conv("mq_conv_fwd", OP_FWD, desc, xq, wq, y, (d.N, d.C_out, ho, wo), (ho, wo, d.N, d.C_out), layout, workspace, stream)
+
+
+def conv_bwd_data(desc, wq, dyq, dx=None, layout=NCHW, workspace=None, stream=None):
+    d = ConvDesc(*desc)
+    return _conv("mq_conv_bwd_data", OP_BWD_DATA, desc, wq, dyq, dx, (d.N, d.C_in, d.H, d.W), (d.H, d.W, d.N, d.C_in), layout, workspace, stream)
+
+
+def conv_bwd_weight(desc, xq, dyq, dw=None, layout=NCHW, workspace=None, stream=None):
+    d = ConvDesc(*desc)
+    return _conv("mq_conv_bwd_weight", OP_BWD_WEIGHT, desc, xq, dyq, dw, (d.C_out, d.C_in, d.Kh, d.Kw), (d.C_out, d.Kh, d.Kw, d.C_in), layout, workspace, stream)
+
+
+def last_device_status(stream=None):
+    return int(lib().mq_last_device_status(_stream(stream)))
+
+
+def conv_layer_host_arena_size(desc, fmt_x, fmt_w, fmt_dy):
+    b = ctypes.c_size_t()
+    _check("mq_conv_layer_host_arena_size", lib().mq_conv_layer_host_arena_size(ctypes.byref(_d(desc)), fmt_x, fmt_w, fmt_dy, ctypes.byref(b)))
+    return b.value
+
+
+def conv_layer_host(desc, fmts, x, w, dy, y, dx, dw, arena, stream=None):
+    """mq_conv_layer_host: host fp32 tensors in (pinned for asynchronous copies), host fp32 results out."""
+    for t in (x, w, dy, y, dx, dw):
+        assert not t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()
+    assert arena.is_cuda
+    _check("mq_conv_layer_host", lib().mq_conv_layer_host(
+        ctypes.byref(_d(desc)), fmts[0], fmts[1], fmts[2], ctypes.c_void_p(x.data_ptr()), ctypes.c_void_p(w.data_ptr()),
+        ctypes.c_void_p(dy.data_ptr()), ctypes.c_void_p(y.data_ptr()), ctypes.c_void_p(dx.data_ptr()), ctypes.c_void_p(dw.data_ptr()),
+        ctypes.c_void_p(arena.data_ptr()), ctypes.c_size_t(arena.numel() * arena.element_size()), _stream(stream)))

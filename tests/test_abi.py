@@ -1,0 +1,87 @@
+"""Host-side checks of the C-ABI library (no GPU, no compute calls): it loads, exports every
+symbol the header declares, answers size queries like the oracle, and rejects bad arguments on
+the host before touching the device."""
+import ctypes
+import os
+import re
+
+import pytest
+
+import oracle
+from paper_2609_28358_b200 import inputs
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module")
+def mq():
+    from paper_2609_28358_b200 import build, mq as _mq
+
+    build.build()
+    return _mq
+
+
+def declared_symbols():
+    names = set()
+    for fn in os.listdir(os.path.join(ROOT, "include")):
+        if fn.endswith(".h"):
+            text = open(os.path.join(ROOT, "include", fn)).read()
+            text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+            names |= set(re.findall(r"\b(mq_[a-z0-9_]+)\s*\(", text))
+    return sorted(names)
+
+
+def test_library_exports_every_declared_symbol(mq):
+    syms = declared_symbols()
+    assert {"mq_quantize", "mq_cbf_im2col", "mq_conv_fwd", "mq_conv_bwd_data", "mq_conv_bwd_weight"} <= set(syms)
+    for s in syms:
+        assert hasattr(mq.lib(), s), s
+
+
+def test_status_strings(mq):
+    assert mq.status_string(0) == "MQ_OK"
+    assert mq.status_string(6) == "MQ_ERR_TIMEOUT"
+    assert len({mq.status_string(i) for i in range(7)}) == 7
+
+
+@pytest.mark.parametrize("desc", [inputs.conv_desc(8, 32, 32, 32, 64, 3), inputs.conv_desc(37, 48, 9, 7, 70, 3, 2),
+                                  inputs.conv_desc(256, 512, 14, 14, 512, 1, 1, 0)])
+def test_size_queries_match_oracle(mq, desc):
+    for fmt in (mq.E4M3, mq.E5M2, mq.E2M1):
+        for role in (mq.ROLE_X, mq.ROLE_W, mq.ROLE_DY):
+            assert mq.qtensor_sizes(desc, role, fmt) == oracle.qtensor_sizes(desc, role, fmt)
+        assert mq.im2col_sizes(desc, fmt) == oracle.im2col_sizes(desc, fmt)
+        for op in (mq.OP_FWD, mq.OP_BWD_DATA, mq.OP_BWD_WEIGHT):
+            assert mq.workspace_size(desc, op, fmt, fmt) >= 0
+
+
+def test_bad_arguments_are_rejected_on_the_host(mq):
+    L = mq.lib()
+    good = mq._d(inputs.conv_desc(8, 32, 8, 8, 32, 3))
+    cb, sb = ctypes.c_size_t(), ctypes.c_size_t()
+    assert L.mq_qtensor_sizes(None, 0, 0, ctypes.byref(cb), ctypes.byref(sb)) == 1
+    assert L.mq_qtensor_sizes(ctypes.byref(good), 7, 0, ctypes.byref(cb), ctypes.byref(sb)) == 1
+    assert L.mq_qtensor_sizes(ctypes.byref(good), 0, 9, ctypes.byref(cb), ctypes.byref(sb)) == 1
+    bad = mq._d(inputs.conv_desc(8, 32, 8, 8, 32, 3), block_size=16)
+    assert L.mq_qtensor_sizes(ctypes.byref(bad), 0, 0, ctypes.byref(cb), ctypes.byref(sb)) == 2  # unsupported block
+    neg = mq._d(inputs.conv_desc(0, 32, 8, 8, 32, 3))
+    assert L.mq_qtensor_sizes(ctypes.byref(neg), 0, 0, ctypes.byref(cb), ctypes.byref(sb)) == 1
+    big_k = mq._d(inputs.conv_desc(1, 32, 2, 2, 32, 7, 1, 0))
+    assert L.mq_qtensor_sizes(ctypes.byref(big_k), 0, 0, ctypes.byref(cb), ctypes.byref(sb)) == 1
+    # entry points: null / misaligned / undersized buffers never reach a launch
+    q = mq._QTensor(None, None, 0, 0, 0, 0)
+    assert L.mq_quantize(ctypes.byref(good), None, 0, ctypes.byref(q), None) == 1
+    q = mq._QTensor(0x1000, 0x2000, 16, 16, 0, 0)
+    assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), 0, ctypes.byref(q), None) == 4  # too small
+    q = mq._QTensor(0x1008, 0x2000, 1 << 30, 1 << 30, 0, 0)
+    assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), 0, ctypes.byref(q), None) == 3  # alignment
+    q = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 0)
+    assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), 1, ctypes.byref(q), None) == 2  # HWNC source
+    assert L.mq_cbf_im2col(ctypes.byref(good), ctypes.byref(q), None, None, None) == 1
+    qw = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 1)
+    assert L.mq_conv_fwd(ctypes.byref(good), ctypes.byref(qw), ctypes.byref(qw), ctypes.c_void_p(0x4000), 0, None, 0, None) == 1  # wrong role
+    assert L.mq_conv_fwd(ctypes.byref(good), ctypes.byref(q), ctypes.byref(qw), ctypes.c_void_p(0x4000), 5, None, 0, None) == 1  # layout
+    need = mq.workspace_size(inputs.conv_desc(8, 32, 8, 8, 32, 3), mq.OP_BWD_WEIGHT, 0, 0)
+    qg = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 2)
+    if need:
+        assert L.mq_conv_bwd_weight(ctypes.byref(good), ctypes.byref(q), ctypes.byref(qg), ctypes.c_void_p(0x4000), 0, None, 0, None) == 4

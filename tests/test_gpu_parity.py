@@ -1,0 +1,141 @@
+"""Parity of the CUDA path with the CPU oracle, through the C ABI (needs a B200).
+
+Small cases span several tiles and ragged tails in every dimension; the workload cases run the
+benchmark's configurations at full size and compare every quantized byte and sampled GEMM
+outputs (all outputs where the oracle finishes in seconds)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2609_28358_b200 import inputs, mq
+from parity_util import (OracleLayer, assert_same_bytes, check_convs, check_im2col, check_quantize, dev,
+                         gpu_quantize_layer)
+
+pytestmark = pytest.mark.gpu
+
+E4M3, E5M2, E2M1 = mq.E4M3, mq.E5M2, mq.E2M1
+FMT_SETS = [(E4M3, E4M3, E5M2), (E2M1, E2M1, E2M1), (E5M2, E4M3, E4M3), (E2M1, E4M3, E5M2)]
+
+
+def make_layer(name, desc, fmts, seed, kinds=("relu", "kaiming", "small")):
+    return inputs.Layer(name, desc, fmts[0], fmts[1], fmts[2], kinds[0], kinds[1], kinds[2], seed)
+
+
+SMALL_SHAPES = [
+    # N, C_in, H, W, C_out, K, stride, pad
+    ("ragged", (40, 48, 5, 6, 70, 3, 1, 1)),       # P = 30 (scalar loads), ragged N, C_in, C_out
+    ("aligned", (64, 96, 8, 8, 64, 3, 1, 1)),      # vector loads, whole tiles
+    ("stride2", (33, 64, 9, 11, 40, 3, 2, 1)),     # odd image, stride 2
+    ("k1", (36, 40, 6, 6, 72, 1, 1, 0)),           # 1x1
+    ("k1s2", (32, 32, 8, 8, 32, 1, 2, 0)),         # 1x1 stride 2
+    ("k5", (8, 16, 12, 12, 24, 5, 2, 2)),          # 5x5, C < 32
+    ("nopad", (16, 32, 7, 7, 32, 3, 1, 0)),        # no padding
+    ("rect", (4, 35, 6, 10, 33, 3, 1, 1)),
+]
+
+
+@pytest.mark.parametrize("fmts", FMT_SETS, ids=lambda f: "-".join(map(str, f)))
+@pytest.mark.parametrize("name,shape", SMALL_SHAPES, ids=[s[0] for s in SMALL_SHAPES])
+def test_small_layers_all_steps(name, shape, fmts):
+    d = inputs.conv_desc(*shape)
+    ol = OracleLayer(make_layer(name, d, fmts, seed=100 + len(name), kinds=("relu", "kaiming", "gauss")))
+    qs = check_quantize(ol)
+    check_im2col(ol, qs[0])
+    check_convs(ol, qs, samples=None, layouts=(mq.NCHW, mq.HWNC))
+
+
+@pytest.mark.parametrize("fmt", [E4M3, E5M2, E2M1])
+def test_quantize_edge_values(fmt):
+    """Zero tiles, -0, ties, saturation, huge and tiny magnitudes, fp32 subnormals."""
+    d = inputs.conv_desc(64, 64, 4, 4, 32, 1, 1, 0)
+    rng = np.random.default_rng(5)
+    x = rng.standard_normal((64, 64, 4, 4)).astype(np.float32)
+    x[:32, :32, 0, 0] = 0.0
+    x[0, 0, 0, 0] = -0.0
+    x[:32, 32:, 0, 1] = np.float32(1.5) * rng.choice([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0, 7.0, -7.9], (32, 32)).astype(np.float32)
+    x[32:, :32, 0, 2] *= np.float32(1e30)
+    x[32:, 32:, 0, 3] *= np.float32(1e-30)
+    x[:32, :32, 1, 0] = rng.standard_normal((32, 32)).astype(np.float32) * np.float32(1e-41)  # subnormal inputs
+    x[:32, :32, 1, 1] = np.ldexp(rng.standard_normal((32, 32)), rng.integers(-20, 20, (32, 32))).astype(np.float32)
+    x[:32, :32, 1, 2] = np.float32(3.4e38)
+    x[:32, 32:, 1, 3] = np.float32(448.0)
+    oc, osc = oracle.quantize(d, oracle.ROLE_X, fmt, x)
+    q = mq.quantize(d, mq.ROLE_X, fmt, dev(x))
+    assert_same_bytes(q.scales, osc, "scales")
+    assert_same_bytes(q.codes, oc, "codes")
+
+
+@pytest.mark.parametrize("fmts", [(E4M3, E4M3, E5M2), (E2M1, E2M1, E2M1)], ids=["fp8", "fp4"])
+def test_small_integer_inputs_are_exact_on_gpu(fmts):
+    """Integers in {-2..2} are exact in every format: the GPU GEMMs must equal the oracle exactly,
+    which isolates indexing and scale routing from rounding."""
+    d = inputs.conv_desc(33, 35, 6, 7, 34, 3, 2, 1)
+    ol = OracleLayer(make_layer("smallint", d, fmts, 23, ("smallint",) * 3))
+    qs = check_quantize(ol)
+    xh, wh, gh = ol.hat
+    y, _ = oracle.conv_fwd(d, xh, wh)
+    gx, _ = oracle.conv_bwd_data(d, wh, gh)
+    gw, _ = oracle.conv_bwd_weight(d, gh, xh)
+    assert np.array_equal(mq.conv_fwd(d, qs[0], qs[1]).cpu().numpy().astype(np.float64), y)
+    assert np.array_equal(mq.conv_bwd_data(d, qs[1], qs[2]).cpu().numpy().astype(np.float64), gx)
+    assert np.array_equal(mq.conv_bwd_weight(d, qs[0], qs[2]).cpu().numpy().astype(np.float64), gw)
+
+
+def test_config1_full_parity():
+    (layer,) = inputs.config1()
+    ol = OracleLayer(layer)
+    qs = check_quantize(ol)
+    check_im2col(ol, qs[0])
+    check_convs(ol, qs, samples=None)
+
+
+def test_config2_full_size():
+    """The benchmark's workload: every quantized byte, the whole im2col, sampled GEMM outputs."""
+    (layer,) = inputs.config2()
+    ol = OracleLayer(layer)
+    qs = check_quantize(ol)
+    # what the square-tile reading does to this workload: most tiles hold an outlier, so most
+    # ordinary activations round to zero -- the fraction must be what the oracle predicts
+    codes = ol.q[0][0]
+    nz_oracle = np.count_nonzero(codes & 0x7) + np.count_nonzero((codes >> 4) & 0x7)
+    g = qs[0].codes
+    nz_gpu = int(torch.count_nonzero(g & 0x7)) + int(torch.count_nonzero((g >> 4) & 0x7))
+    assert nz_gpu == nz_oracle
+    check_im2col(ol, qs[0])
+    check_convs(ol, qs, samples=20000)
+
+
+@pytest.mark.parametrize("idx", [0, 1], ids=["3x3", "1x1"])
+def test_config4_full_size(idx):
+    layer = inputs.config4()[idx]
+    ol = OracleLayer(layer)
+    qs = check_quantize(ol)
+    check_im2col(ol, qs[0])
+    check_convs(ol, qs, samples=8000)
+
+
+def _cfg3_layers():
+    return inputs.config3()
+
+
+@pytest.mark.parametrize("li", [0, 1, 2, 5, 11, 17, 18, 23])
+def test_config3_layers_full_size(li):
+    layer = _cfg3_layers()[li]
+    ol = OracleLayer(layer)
+    qs = check_quantize(ol)
+    check_im2col(ol, qs[0])
+    check_convs(ol, qs, samples=6000)
+
+
+CFG5_POINTS = ["cfg5_e4m3_k3s1_c64_hw14", "cfg5_e4m3_k3s2_c128_hw28", "cfg5_e4m3_k1s1_c256_hw14", "cfg5_e2m1_k3s1_c128_hw14",
+               "cfg5_e2m1_k1s2_c64_hw28", "cfg5_e2m1_k3s2_c256_hw14", "cfg5_e4m3_k3s1_c512_hw14", "cfg5_e4m3_k3s1_c64_hw56"]
+
+
+@pytest.mark.parametrize("name", CFG5_POINTS)
+def test_config5_points_full_size(name):
+    layer = {l.name: l for l in inputs.config5()}[name]
+    ol = OracleLayer(layer)
+    qs = check_quantize(ol)
+    check_im2col(ol, qs[0])
+    check_convs(ol, qs, samples=4000)
