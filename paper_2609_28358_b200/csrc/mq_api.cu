@@ -1,5 +1,8 @@
 // extern "C" entry points: argument validation, size arithmetic, kernel selection.
+#include <cstdlib>
+
 #include "mq_internal.cuh"
+#include "mq_conv_tc.cuh"
 
 namespace mq {
 
@@ -45,6 +48,134 @@ mq_status check_qtensor(const Geom& g, const mq_qtensor* q, int role) {
   return MQ_OK;
 }
 
+
+// ---- tensor-core path: eligibility, tile shape, tensor maps ------------------------------------
+int env_int(const char* name, int dflt) {
+  const char* v = std::getenv(name);
+  return v ? std::atoi(v) : dflt;
+}
+
+// fwd / bwd_data run on the tcgen05 kernel when both operands are 8-bit formats or both are E2M1 and a
+// tap's channel row is a whole number of 32-byte MMA K-atoms.
+bool conv_tc_eligible(int op, const Geom& g, int fmt_x_like, int fmt_w) {
+  if (op != MQ_OP_FWD && op != MQ_OP_BWD_DATA) return false;
+  if (env_int("MQ_DISABLE_TC", 0)) return false;
+  const bool fp4 = fmt_x_like == MQ_E2M1 && fmt_w == MQ_E2M1;
+  const bool fp8 = fmt_x_like != MQ_E2M1 && fmt_w != MQ_E2M1;
+  if (!fp4 && !fp8) return false;
+  const int Kp = op == MQ_OP_FWD ? g.Cp : g.Cop;
+  const int rowbytes = Kp * (fp4 ? 4 : 8) / 8;
+  return rowbytes % 32 == 0;
+}
+
+size_t conv_tc_workspace(int op, const Geom& g, int fmt_w) {
+  if (op != MQ_OP_BWD_DATA) return 0;
+  return (size_t)g.Cp * g.Kh * g.Kw * g.Cop * fmt_bits(fmt_w) / 8;  // W re-laid as [C_in_p][taps][C_out_p]
+}
+
+// Output columns per tile.  Rows of a tile are TW consecutive output columns x TN = 128/TW samples with
+// the column index fastest, so an NCHW store writes runs of TW floats; TW >= 8 fills 32-byte sectors.
+int choose_tw(int w_eff, int N, int layout) {
+  const int forced = env_int("MQ_TC_TW", 0);
+  if (forced > 0) return forced;
+  int best = 1;
+  double best_cost = 1e30;
+  for (int tw = 1; tw <= 32; tw *= 2) {
+    const int tn = 128 / tw;
+    const double waste = (double)((w_eff + tw - 1) / tw * tw) / w_eff * (double)((N + tn - 1) / tn * tn) / N;
+    double pen = 1.0;
+    if (layout == MQ_NCHW) pen = tw >= 8 ? 1.0 : (tw == 4 ? 1.25 : (tw == 2 ? 1.8 : 2.5));
+    const double cost = waste * pen;
+    if (cost < best_cost - 1e-9) { best_cost = cost; best = tw; }
+  }
+  return best;
+}
+
+mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq_qtensor* qw, float* out, int layout, void* ws,
+                      unsigned int* status, cudaStream_t stream) {
+  const bool fp4 = qw->fmt == MQ_E2M1;
+  const int bits = fp4 ? 4 : 8;
+  const int taps = g.Kh * g.Kw;
+  ConvTcParams p{};
+  p.mode = op;
+  p.kind_fp4 = fp4 ? 1 : 0;
+  p.N = g.N; p.Nt = g.Nt;
+  p.Kh = g.Kh; p.Kw = g.Kw; p.sh = g.sh; p.sw = g.sw; p.ph = g.ph; p.pw = g.pw;
+  int Kp, rows_b;
+  const uint8_t* b_codes;
+  if (op == MQ_OP_FWD) {
+    Kp = g.Cp; p.Hs = g.H; p.Ws = g.W; p.Hd = g.Ho; p.Wd = g.Wo; p.Cd = g.Cout; rows_b = g.Cout;
+    p.sb_row = taps * g.Ct; p.sb_tap = g.Ct; p.sb_k = 1;
+    b_codes = static_cast<const uint8_t*>(qw->codes);
+    p.tiles_h = g.Ho; p.classes = 1;
+  } else {
+    Kp = g.Cop; p.Hs = g.Ho; p.Ws = g.Wo; p.Hd = g.H; p.Wd = g.W; p.Cd = g.Cin; rows_b = g.Cp;
+    p.sb_row = 1; p.sb_tap = g.Ct; p.sb_k = taps * g.Ct;
+    if (launch_weight_transpose(static_cast<const uint8_t*>(qw->codes), static_cast<uint8_t*>(ws), g, qw->fmt, stream) != cudaSuccess) return MQ_ERR_CUDA;
+    b_codes = static_cast<const uint8_t*>(ws);
+    p.tiles_h = (g.H + g.sh - 1) / g.sh; p.classes = g.sh * g.sw;
+  }
+  p.Kblocks = Kp / 32;
+  const int rowbytes = Kp * bits / 8;
+  p.KB = rowbytes % 128 == 0 ? 128 : (rowbytes % 64 == 0 ? 64 : 32);
+  p.G = 128 / p.KB;
+  p.cpt = rowbytes / p.KB;
+  const int w_eff = op == MQ_OP_FWD ? g.Wo : (g.W + g.sw - 1) / g.sw;
+  p.TW = choose_tw(w_eff, g.N, layout);
+  if (p.TW < 1 || p.TW > 32 || (p.TW & (p.TW - 1))) return MQ_ERR_INVALID_ARG;
+  p.TN = 128 / p.TW;
+  p.lgTW = 0;
+  while ((1 << p.lgTW) < p.TW) ++p.lgTW;
+  const int cd16 = (p.Cd + 15) / 16 * 16;
+  p.BN = cd16 <= 128 ? cd16 : 128;
+  const int forced_bn = env_int("MQ_TC_BN", 0);
+  if (forced_bn >= 32 && forced_bn <= 256 && forced_bn % 32 == 0) p.BN = forced_bn < cd16 ? forced_bn : cd16;
+  p.tiles_c = (p.Cd + p.BN - 1) / p.BN;
+  p.tiles_w = (w_eff + p.TW - 1) / p.TW;
+  p.tiles_n = (g.N + p.TN - 1) / p.TN;
+  p.total_tiles = (long long)p.tiles_c * p.tiles_w * p.tiles_n * p.tiles_h * p.classes;
+  p.n_acc = (2 * p.BN + 48 <= 512) ? 2 : 1;
+  const size_t stage_bytes = 128 * 128 + (size_t)p.BN * 128 + 3072;
+  int stages = (int)((227 * 1024 - 2048) / stage_bytes);
+  if (stages > 8) stages = 8;
+  if (stages < 2) return MQ_ERR_UNSUPPORTED;
+  p.stages = stages;
+  const uint32_t fa = fp4 ? 1u : (qx_like->fmt == MQ_E5M2 ? 1u : 0u);
+  const uint32_t fb = fp4 ? 1u : (qw->fmt == MQ_E5M2 ? 1u : 0u);
+  p.idesc = (fa << 7) | (fb << 10) | ((uint32_t)(p.BN >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
+  p.a_scales = qx_like->scales;
+  p.b_scales = qw->scales;
+  p.out = out; p.out_layout = layout; p.status = status;
+
+  CUtensorMap map_a, map_b;
+  {
+    const uint64_t rb = (uint64_t)rowbytes;
+    const uint64_t dims[4] = {rb, (uint64_t)p.Ws, (uint64_t)g.N, (uint64_t)p.Hs};
+    const uint64_t strides[3] = {(uint64_t)g.N * rb, rb, (uint64_t)p.Ws * g.N * rb};
+    const uint32_t wst = op == MQ_OP_FWD ? (uint32_t)g.sw : 1u;
+    const uint32_t box[4] = {(uint32_t)p.KB, (uint32_t)((p.TW - 1) * wst + 1), (uint32_t)p.TN, 1u};
+    const uint32_t es[4] = {1u, wst, 1u, 1u};
+    if (!encode_tensor_map_u8(&map_a, qx_like->codes, 4, dims, strides, box, es, p.KB)) return MQ_ERR_CUDA;
+  }
+  {
+    const uint64_t rb = (uint64_t)rowbytes;
+    const uint64_t dims[3] = {rb, (uint64_t)taps, (uint64_t)rows_b};
+    const uint64_t strides[2] = {rb, (uint64_t)taps * rb};
+    const uint32_t box[3] = {(uint32_t)p.KB, 1u, (uint32_t)p.BN};
+    if (!encode_tensor_map_u8(&map_b, b_codes, 3, dims, strides, box, nullptr, p.KB)) return MQ_ERR_CUDA;
+  }
+  return launch_conv_tc(p, map_a, map_b, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
+}
+
+unsigned int* device_status_ptr() {
+  static unsigned int* ptr = nullptr;
+  if (!ptr) {
+    void* q = nullptr;
+    if (cudaGetSymbolAddress(&q, g_device_status) == cudaSuccess) ptr = static_cast<unsigned int*>(q);
+  }
+  return ptr;
+}
+
 mq_status run_conv(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int role_a, const mq_qtensor* qb, int role_b,
                    void* out, int layout, void* ws, size_t ws_bytes, void* stream) {
   mq_status st = check_desc(desc);
@@ -58,6 +189,10 @@ mq_status run_conv(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int r
   size_t need = 0;
   mq_workspace_size(desc, op, qa->fmt, qb->fmt, &need);
   if (need > 0 && (!ws || ws_bytes < need)) return MQ_ERR_BUFFER_TOO_SMALL;
+  if (op == MQ_OP_FWD && conv_tc_eligible(op, g, qa->fmt, qb->fmt))
+    return run_conv_tc(op, g, qa, qb, static_cast<float*>(out), layout, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
+  if (op == MQ_OP_BWD_DATA && conv_tc_eligible(op, g, qb->fmt, qa->fmt))
+    return run_conv_tc(op, g, qb, qa, static_cast<float*>(out), layout, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
   ConvArgs a;
   a.g = g;
   a.a_codes = static_cast<const uint8_t*>(qa->codes); a.a_scales = qa->scales; a.fmt_a = qa->fmt;
@@ -97,7 +232,9 @@ mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt
   if (st != MQ_OK) return st;
   if (!valid_fmt(fmt_a) || !valid_fmt(fmt_b) || !bytes) return MQ_ERR_INVALID_ARG;
   if (op != MQ_OP_FWD && op != MQ_OP_BWD_DATA && op != MQ_OP_BWD_WEIGHT) return MQ_ERR_INVALID_ARG;
-  *bytes = conv_generic_workspace(op, make_geom(*desc));
+  const Geom g = make_geom(*desc);
+  *bytes = conv_generic_workspace(op, g);
+  if (op == MQ_OP_BWD_DATA && conv_tc_eligible(op, g, fmt_b, fmt_a)) *bytes = conv_tc_workspace(op, g, fmt_a);
   return MQ_OK;
 }
 

@@ -1,0 +1,57 @@
+// Declarations shared by the tensor-core (tcgen05) convolution GEMM kernels and their host side.
+#pragma once
+
+#include <cuda.h>  // CUtensorMap (types only; the encoder is fetched through the runtime)
+
+#include "mq_internal.cuh"
+
+namespace mq {
+
+// Parameters of the persistent implicit-GEMM kernel that serves mq_conv_fwd and mq_conv_bwd_data.
+//
+// GEMM view: D[(y, x, n)][c] = sum over taps and K-blocks of A[(y', x', n)][k] * B[c][tap][k], where
+// A is a stored activation-like tensor ([Hs][Ws][N][Kp] codes, fwd: X, bwd_data: G_Y) gathered at a
+// tap-dependent pixel, and B is a stored weight-like tensor ([rows][taps][Kp] codes, fwd: W,
+// bwd_data: W re-laid as [C_in_p][taps][C_out_p]).
+struct ConvTcParams {
+  int mode;             // MQ_OP_FWD or MQ_OP_BWD_DATA
+  int kind_fp4;         // 1: both operands E2M1 (kind::mxf4), 0: 8-bit formats (kind::mxf8f6f4)
+  uint32_t idesc;       // instruction descriptor without scale ids
+  int KB;               // bytes of K per row per TMA box: 128, 64 or 32 (= swizzle span)
+  int G;                // boxes (chunks) per pipeline stage = 128 / KB
+  int cpt;              // chunks per tap = row bytes / KB
+  int BN;               // output channels per tile (multiple of 16, <= 256)
+  int stages;
+  int n_acc;            // accumulator buffers in TMEM (1 or 2)
+  int TW, TN, lgTW;     // tile = TW output columns x TN samples (TW * TN = 128), TW fastest among rows
+  // geometry
+  int N, Nt;
+  int Hs, Ws;           // spatial extent of the gathered source (fwd: H, W; bwd_data: Ho, Wo)
+  int Kblocks;          // 32-element K-blocks per tap (source channels / 32)
+  int Hd, Wd;           // spatial extent of the output (fwd: Ho, Wo; bwd_data: H, W)
+  int Cd;               // output channels (fwd: C_out; bwd_data: C_in)
+  int Kh, Kw, sh, sw, ph, pw;
+  // tiles
+  int tiles_c, tiles_w, tiles_n, tiles_h, classes;  // classes = sh*sw parity classes (bwd_data), else 1
+  long long total_tiles;
+  // scales
+  const uint8_t* a_scales;  // [Hs][Ws][Nt][Kblocks]
+  const uint8_t* b_scales;  // index = rowblock * sb_row + tap * sb_tap + kblock * sb_k
+  int sb_row, sb_tap, sb_k;
+  // output
+  float* out;
+  int out_layout;
+  unsigned int* status;
+};
+
+cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s);
+size_t conv_tc_smem_bytes(const ConvTcParams& p);
+
+// Re-lays the stored weight codes [C_out][taps][C_in_p] as [C_in_p][taps][C_out_p] (bwd_data's B operand).
+cudaError_t launch_weight_transpose(const uint8_t* w_codes, uint8_t* wt_codes, const Geom& g, int fmt, cudaStream_t s);
+
+// Host: encode a tiled tensor map over bytes.  dims / strides in bytes (stride[0] implied 1), fastest first.
+bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
+                          const uint32_t* box, const uint32_t* elem_strides, int swizzle_bytes);
+
+}  // namespace mq
