@@ -68,9 +68,14 @@ bool conv_tc_eligible(int op, const Geom& g, int fmt_x_like, int fmt_w) {
   return rowbytes % 32 == 0;
 }
 
+size_t wt_codes_bytes(const Geom& g, int fmt_w) {
+  return ((size_t)g.Cp * g.Kh * g.Kw * g.Cop * fmt_bits(fmt_w) / 8 + 255) / 256 * 256;
+}
+
 size_t conv_tc_workspace(int op, const Geom& g, int fmt_w) {
   if (op != MQ_OP_BWD_DATA) return 0;
-  return (size_t)g.Cp * g.Kh * g.Kw * g.Cop * fmt_bits(fmt_w) / 8;  // W re-laid as [C_in_p][taps][C_out_p]
+  // W re-laid as [C_in_p][taps][C_out_p] codes (rounded up to 256 bytes) + [C_in_p/32][taps][C_out_p/32] scales
+  return wt_codes_bytes(g, fmt_w) + (size_t)g.Ct * g.Kh * g.Kw * g.Cot;
 }
 
 // Output columns per tile.  Rows of a tile are TW consecutive output columns x TN = 128/TW samples with
@@ -105,14 +110,17 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
   const uint8_t* b_codes;
   if (op == MQ_OP_FWD) {
     Kp = g.Cp; p.Hs = g.H; p.Ws = g.W; p.Hd = g.Ho; p.Wd = g.Wo; p.Cd = g.Cout; rows_b = g.Cout;
-    p.sb_row = taps * g.Ct; p.sb_tap = g.Ct; p.sb_k = 1;
     b_codes = static_cast<const uint8_t*>(qw->codes);
+    p.b_scales = qw->scales;
     p.tiles_h = g.Ho; p.classes = 1;
   } else {
     Kp = g.Cop; p.Hs = g.Ho; p.Ws = g.Wo; p.Hd = g.H; p.Wd = g.W; p.Cd = g.Cin; rows_b = g.Cp;
-    p.sb_row = 1; p.sb_tap = g.Ct; p.sb_k = taps * g.Ct;
-    if (launch_weight_transpose(static_cast<const uint8_t*>(qw->codes), static_cast<uint8_t*>(ws), g, qw->fmt, stream) != cudaSuccess) return MQ_ERR_CUDA;
+    uint8_t* wt_scales = static_cast<uint8_t*>(ws) + wt_codes_bytes(g, qw->fmt);
+    if (launch_weight_transpose(static_cast<const uint8_t*>(qw->codes), qw->scales, static_cast<uint8_t*>(ws), wt_scales, g, qw->fmt, stream) !=
+        cudaSuccess)
+      return MQ_ERR_CUDA;
     b_codes = static_cast<const uint8_t*>(ws);
+    p.b_scales = wt_scales;
     p.tiles_h = (g.H + g.sh - 1) / g.sh; p.classes = g.sh * g.sw;
   }
   p.Kblocks = Kp / 32;
@@ -144,7 +152,6 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
   const uint32_t fb = fp4 ? 1u : (qw->fmt == MQ_E5M2 ? 1u : 0u);
   p.idesc = (fa << 7) | (fb << 10) | ((uint32_t)(p.BN >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
   p.a_scales = qx_like->scales;
-  p.b_scales = qw->scales;
   p.out = out; p.out_layout = layout; p.status = status;
 
   CUtensorMap map_a, map_b;

@@ -36,8 +36,7 @@ struct ConvTcParams {
   long long total_tiles;
   // scales
   const uint8_t* a_scales;  // [Hs][Ws][Nt][Kblocks]
-  const uint8_t* b_scales;  // index = rowblock * sb_row + tap * sb_tap + kblock * sb_k
-  int sb_row, sb_tap, sb_k;
+  const uint8_t* b_scales;  // [row blocks of 32][taps][Kblocks]
   // output
   float* out;
   int out_layout;
@@ -47,8 +46,10 @@ struct ConvTcParams {
 cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s);
 size_t conv_tc_smem_bytes(const ConvTcParams& p);
 
-// Re-lays the stored weight codes [C_out][taps][C_in_p] as [C_in_p][taps][C_out_p] (bwd_data's B operand).
-cudaError_t launch_weight_transpose(const uint8_t* w_codes, uint8_t* wt_codes, const Geom& g, int fmt, cudaStream_t s);
+// Re-lays the stored weight codes [C_out][taps][C_in_p] as [C_in_p][taps][C_out_p] and the tile scales
+// [C_out/32][taps][C_in_p/32] as [C_in_p/32][taps][C_out_p/32] (bwd_data's B operand).  No requantization.
+cudaError_t launch_weight_transpose(const uint8_t* w_codes, const uint8_t* w_scales, uint8_t* wt_codes, uint8_t* wt_scales, const Geom& g, int fmt,
+                                    cudaStream_t s);
 
 // Host: encode a tiled tensor map over bytes.  dims / strides in bytes (stride[0] implied 1), fastest first.
 bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
