@@ -7,7 +7,7 @@
 //   fwd        : M = (ho,wo,n)   N = co           K = (kh,kw | ci)   A = X gathered, B = W     both K-contiguous
 //   bwd_data   : M = (h,w,n)     N = ci           K = (kh,kw | co)   A = G_Y gathered (K-contiguous), B = W (N-contiguous)
 //   bwd_weight : M = co          N = (kh,kw,ci)   K = (ho,wo | n)    A = G_Y, B = X gathered   both MN-contiguous
-#include "mq_internal.cuh"
+#include "mq_conv_tc.cuh"
 
 namespace mq {
 namespace {
@@ -257,6 +257,14 @@ int conv_generic_bwd_weight_splits(const Geom& g) {
 size_t conv_generic_workspace(int op, const Geom& g) {
   if (op != MQ_OP_BWD_WEIGHT) return 0;
   return (size_t)conv_generic_bwd_weight_splits(g) * g.Cout * g.Kh * g.Kw * g.Cp * sizeof(float);
+}
+
+cudaError_t launch_bwd_weight_reduce(const float* partial, float* out, const Geom& g, int splits, int layout, cudaStream_t s) {
+  const long long total = (long long)g.Cout * g.Kh * g.Kw * g.Cin;
+  unsigned blocks = (unsigned)((total + 255) / 256);
+  if (blocks > 148u * 16) blocks = 148u * 16;
+  bwd_weight_reduce<<<blocks, 256, 0, s>>>(partial, out, g, splits, layout);
+  return cudaGetLastError();
 }
 
 #define MQ_DISPATCH2(FA, FB, CALL)                                                         \

@@ -51,6 +51,30 @@ size_t conv_tc_smem_bytes(const ConvTcParams& p);
 cudaError_t launch_weight_transpose(const uint8_t* w_codes, const uint8_t* w_scales, uint8_t* wt_codes, uint8_t* wt_scales, const Geom& g, int fmt,
                                     cudaStream_t s);
 
+// Parameters of the tensor-core weight-gradient kernel (see mq_wgrad_tc.cu).
+struct WgradTcParams {
+  int fp4;              // 1: E2M1 operands re-laid n-fastest (K-major, kind::mxf4); 0: 8-bit operands as stored (MN-major)
+  uint32_t idesc;
+  int stages;
+  int N, Nt, Ho, Wo, H, W, Cout, Cp, Ct, Cot, Kh, Kw, sh, sw, ph, pw;
+  int BPP;              // K-blocks (32 samples) taken per pixel per stage
+  int KPX;              // pixels per stage
+  int KBn;              // E2M1: bytes of n per pixel per stage (= 16 * BPP)
+  int nchunks;          // stages per pixel group
+  int groups_w;         // ceil(Wo / KPX)
+  int stages_total;     // Ho * groups_w * nchunks
+  int m_tiles, j_tiles, cb_tiles, splits;
+  const uint8_t* g_scales;  // [Ho][Wo][Nt][Cot]
+  const uint8_t* x_scales;  // [H][W][Nt][Ct]
+  float* partial;           // [splits][Cout][taps * Cp]
+  unsigned int* status;
+};
+cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s);
+// E2M1 codes [P][N][Cp] -> [P][Cp][Npad] (n fastest, zero-padded): a permutation of nibbles, no requantization.
+cudaError_t launch_fp4_to_n_major(const uint8_t* in, uint8_t* out, int P, int N, int Cp, int Npad, cudaStream_t s);
+// Adds the split partial sums in a fixed order and writes G_W in its final layout.
+cudaError_t launch_bwd_weight_reduce(const float* partial, float* out, const Geom& g, int splits, int layout, cudaStream_t s);
+
 // Host: encode a tiled tensor map over bytes.  dims / strides in bytes (stride[0] implied 1), fastest first.
 bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
                           const uint32_t* box, const uint32_t* elem_strides, int swizzle_bytes);
