@@ -45,7 +45,8 @@ typedef enum {
   MQ_ERR_ALIGNMENT = 3,        /* a device pointer is not 16-byte aligned                         */
   MQ_ERR_BUFFER_TOO_SMALL = 4, /* a declared buffer size is smaller than the call needs           */
   MQ_ERR_CUDA = 5,             /* a CUDA runtime / driver call failed (launch, descriptor encode) */
-  MQ_ERR_TIMEOUT = 6           /* a bounded device-side wait gave up (see mq_last_device_status)  */
+  MQ_ERR_TIMEOUT = 6,          /* a bounded device-side wait gave up (see mq_last_device_status)  */
+  MQ_ERR_STATIC_SCRATCH = 7    /* the layer needs more scratch than the built-in static array holds */
 } mq_status;
 
 typedef enum { MQ_E4M3 = 0, MQ_E5M2 = 1, MQ_E2M1 = 2 } mq_elem;        /* element format, Sec. II-D */
@@ -113,6 +114,29 @@ mq_status mq_conv_fwd(const mq_conv_desc* desc, const mq_qtensor* xq, const mq_q
  * dx: fp32, MQ_NCHW ([N][C_in][H][W]) or MQ_HWNC ([H][W][N][C_in]). */
 mq_status mq_conv_bwd_data(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, void* dx, int dx_layout,
                            void* workspace, size_t ws_bytes, void* stream);
+
+/* mq_conv_bwd_data_static -- the same computation as mq_conv_bwd_data for callers that cannot hand the
+ * library a scratch buffer because they cannot allocate device memory at all.  (The paper has no
+ * counterpart for this call; it exists for integration reasons only.)  Typical cases: a plug-in that runs
+ * inside a host application which owns the allocator and forbids cudaMalloc on its streams, code running
+ * while a memory pool is frozen, or a tiny embedding that links the library without any allocator.  Such
+ * a caller still supplies the inputs (wq, dyq) and the output (dx); only the scratch is taken care of.
+ *
+ * The scratch that mq_conv_bwd_data takes as `workspace` (the weight codes and tile scales re-laid for the
+ * input-gradient GEMM) lives here in a static array inside the library's device image,
+ * MQ_STATIC_SCRATCH_BYTES (4 MiB) long; every GPU that loads the library keeps that much memory reserved
+ * until the process exits.  A layer whose mq_workspace_size(desc, MQ_OP_BWD_DATA, ...) exceeds it is
+ * rejected with MQ_ERR_STATIC_SCRATCH and nothing is launched (512 x 512 x 3 x 3 FP8 weights need 2.4 MB).
+ * The call performs no cudaMalloc / cudaFree and calls no allocating library routine.
+ *
+ * First use on a device: the first call made while a given device is current looks up the array's device
+ * address (once per device, kept for later calls).  Make that first call outside of any stream capture.
+ * Sharing: all calls on a device use the same array and it keeps whatever the previous call left in it;
+ * each call overwrites every byte it later reads, so nothing needs clearing, but two calls whose kernels
+ * overlap on the GPU (different streams, no ordering between them) race on the array -- order them. */
+#define MQ_STATIC_SCRATCH_BYTES (4u << 20)
+mq_status mq_conv_bwd_data_static(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, void* dx, int dx_layout,
+                                  void* stream);
 
 /* mq_conv_bwd_weight -- G_Wf = G_Yf . X'^T (Sec. II-C, IV-B; Eq. 3), K-blocks of 32 samples at one
  * output pixel: the stored X and G_Y are read along N, the other direction of their square blocks.

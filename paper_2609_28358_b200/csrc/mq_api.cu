@@ -409,6 +409,33 @@ mq_status mq_conv_bwd_weight(const mq_conv_desc* desc, const mq_qtensor* xq, con
   return run_conv(MQ_OP_BWD_WEIGHT, desc, xq, MQ_ROLE_X, dyq, MQ_ROLE_DY, dw, dw_layout, workspace, ws_bytes, stream);
 }
 
+// ---- allocation-free variant of mq_conv_bwd_data ---------------------------------------------------
+// Scratch for callers that cannot allocate: a static array in the device image.  In host code the name
+// below is only a handle for the runtime, not a device address; the address is looked up once per device
+// with cudaGetSymbolAddress (with that device current) and that pointer is what the kernels receive.
+static __device__ __align__(256) unsigned char g_static_scratch[MQ_STATIC_SCRATCH_BYTES];
+static void* g_static_scratch_addr[64] = {};
+
+mq_status mq_conv_bwd_data_static(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, void* dx, int dx_layout,
+                                  void* stream) {
+  mq_status st = check_desc(desc);
+  if (st != MQ_OK) return st;
+  if (!wq || !dyq) return MQ_ERR_INVALID_ARG;
+  if (!valid_fmt(wq->fmt) || !valid_fmt(dyq->fmt)) return MQ_ERR_INVALID_ARG;
+  size_t need = 0;
+  if ((st = mq_workspace_size(desc, MQ_OP_BWD_DATA, wq->fmt, dyq->fmt, &need)) != MQ_OK) return st;
+  if (need > MQ_STATIC_SCRATCH_BYTES) return MQ_ERR_STATIC_SCRATCH;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return MQ_ERR_CUDA;
+  if (dev < 0 || dev >= 64) return MQ_ERR_UNSUPPORTED;
+  if (!g_static_scratch_addr[dev]) {
+    void* addr = nullptr;
+    if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || !addr) return MQ_ERR_CUDA;
+    g_static_scratch_addr[dev] = addr;
+  }
+  return run_conv(MQ_OP_BWD_DATA, desc, wq, MQ_ROLE_W, dyq, MQ_ROLE_DY, dx, dx_layout, g_static_scratch_addr[dev], MQ_STATIC_SCRATCH_BYTES, stream);
+}
+
 namespace {
 struct LayerArena {
   size_t off_x, off_w, off_g, off_y, off_dx, off_dw, off_ws, off_ic, off_is, total;
@@ -494,6 +521,7 @@ const char* mq_status_string(int status) {
     case MQ_ERR_BUFFER_TOO_SMALL: return "MQ_ERR_BUFFER_TOO_SMALL";
     case MQ_ERR_CUDA: return "MQ_ERR_CUDA";
     case MQ_ERR_TIMEOUT: return "MQ_ERR_TIMEOUT";
+    case MQ_ERR_STATIC_SCRATCH: return "MQ_ERR_STATIC_SCRATCH";
     default: return "MQ_ERR_UNKNOWN";
   }
 }

@@ -158,6 +158,23 @@ def conv_bwd_data(desc, wq, dyq, dx=None, layout=NCHW, workspace=None, stream=No
     return _conv("mq_conv_bwd_data", OP_BWD_DATA, desc, wq, dyq, dx, (d.N, d.C_in, d.H, d.W), (d.H, d.W, d.N, d.C_in), layout, workspace, stream)
 
 
+STATIC_SCRATCH_BYTES = 4 << 20
+
+
+def conv_bwd_data_static(desc, wq, dyq, dx=None, layout=NCHW, stream=None):
+    """mq_conv_bwd_data_static: the input gradient for callers that cannot allocate device memory (a plug-in
+    inside an application that owns the allocator, a frozen memory pool).  The library's own static device
+    array serves as scratch; layers needing more than STATIC_SCRATCH_BYTES raise MqError(MQ_ERR_STATIC_SCRATCH).
+    `dx` should be passed in by such callers; it is only created here for convenience when omitted."""
+    d = ConvDesc(*desc)
+    if dx is None:
+        dx = torch.empty((d.N, d.C_in, d.H, d.W) if layout == NCHW else (d.H, d.W, d.N, d.C_in), dtype=torch.float32, device=wq.codes.device)
+    a, b = wq._c(), dyq._c()
+    _check("mq_conv_bwd_data_static", lib().mq_conv_bwd_data_static(ctypes.byref(_d(desc)), ctypes.byref(a), ctypes.byref(b),
+                                                                  ctypes.c_void_p(dx.data_ptr()), layout, _stream(stream)))
+    return dx
+
+
 def conv_bwd_weight(desc, xq, dyq, dw=None, layout=NCHW, workspace=None, stream=None):
     d = ConvDesc(*desc)
     return _conv("mq_conv_bwd_weight", OP_BWD_WEIGHT, desc, xq, dyq, dw, (d.C_out, d.C_in, d.Kh, d.Kw), (d.C_out, d.Kh, d.Kw, d.C_in), layout, workspace, stream)
