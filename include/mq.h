@@ -157,6 +157,9 @@ mq_status mq_conv_layer_host(const mq_conv_desc* desc, int fmt_x, int fmt_w, int
                              const float* dy_host, float* y_host, float* dx_host, float* dw_host, void* arena, size_t arena_bytes,
                              void* stream);
 
+/* Diagnostic: how many kernels this library has launched so far in this process (all entry points). */
+unsigned long long mq_kernel_launch_count(void);
+
 /* Human-readable name of a status code (static storage). */
 const char* mq_status_string(int status);
 

@@ -1,4 +1,5 @@
 // extern "C" entry points: argument validation, size arithmetic, kernel selection.
+#include <atomic>
 #include <cstdlib>
 
 #include "mq_internal.cuh"
@@ -7,6 +8,9 @@
 namespace mq {
 
 __device__ unsigned int g_device_status = 0;  // set by kernels when a bounded wait gives up
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 
 namespace {
 
@@ -71,12 +75,7 @@ bool conv_tc_eligible(int op, const Geom& g, int fmt_x_like, int fmt_w) {
 size_t wt_codes_bytes(const Geom& g, int fmt_w) {
   return ((size_t)g.Cp * g.Kh * g.Kw * g.Cop * fmt_bits(fmt_w) / 8 + 255) / 256 * 256;
 }
-
-size_t conv_tc_workspace(int op, const Geom& g, int fmt_w) {
-  if (op != MQ_OP_BWD_DATA) return 0;
-  // W re-laid as [C_in_p][taps][C_out_p] codes (rounded up to 256 bytes) + [C_in_p/32][taps][C_out_p/32] scales
-  return wt_codes_bytes(g, fmt_w) + (size_t)g.Ct * g.Kh * g.Kw * g.Cot;
-}
+size_t up256(size_t v) { return (v + 255) / 256 * 256; }
 
 // Output columns per tile.  Rows of a tile are TW consecutive output columns x TN = 128/TW samples with
 // the column index fastest, so an NCHW store writes runs of TW floats; TW >= 8 fills 32-byte sectors.
@@ -96,9 +95,16 @@ int choose_tw(int w_eff, int N, int layout) {
   return best;
 }
 
-mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq_qtensor* qw, float* out, int layout, void* ws,
-                      unsigned int* status, cudaStream_t stream) {
-  const bool fp4 = qw->fmt == MQ_E2M1;
+// Geometry of a tensor-core fwd / bwd_data call and the layout of its scratch:
+//   [W re-laid codes | W re-laid scales]  (bwd_data only)  [A-side scale chunks][B-side scale chunks]
+struct ConvTcPlan {
+  ConvTcParams p;
+  int rowbytes, rows_b;
+  size_t off_wt_scales, off_sfa, off_sfb, total;
+};
+
+bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, ConvTcPlan* out) {
+  const bool fp4 = fmt_w == MQ_E2M1;
   const int bits = fp4 ? 4 : 8;
   const int taps = g.Kh * g.Kw;
   ConvTcParams p{};
@@ -106,31 +112,23 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
   p.kind_fp4 = fp4 ? 1 : 0;
   p.N = g.N; p.Nt = g.Nt;
   p.Kh = g.Kh; p.Kw = g.Kw; p.sh = g.sh; p.sw = g.sw; p.ph = g.ph; p.pw = g.pw;
-  int Kp, rows_b;
-  const uint8_t* b_codes;
+  int Kp;
   if (op == MQ_OP_FWD) {
-    Kp = g.Cp; p.Hs = g.H; p.Ws = g.W; p.Hd = g.Ho; p.Wd = g.Wo; p.Cd = g.Cout; rows_b = g.Cout;
-    b_codes = static_cast<const uint8_t*>(qw->codes);
-    p.b_scales = qw->scales;
+    Kp = g.Cp; p.Hs = g.H; p.Ws = g.W; p.Hd = g.Ho; p.Wd = g.Wo; p.Cd = g.Cout; out->rows_b = g.Cout;
     p.tiles_h = g.Ho; p.classes = 1;
   } else {
-    Kp = g.Cop; p.Hs = g.Ho; p.Ws = g.Wo; p.Hd = g.H; p.Wd = g.W; p.Cd = g.Cin; rows_b = g.Cp;
-    uint8_t* wt_scales = static_cast<uint8_t*>(ws) + wt_codes_bytes(g, qw->fmt);
-    if (launch_weight_transpose(static_cast<const uint8_t*>(qw->codes), qw->scales, static_cast<uint8_t*>(ws), wt_scales, g, qw->fmt, stream) !=
-        cudaSuccess)
-      return MQ_ERR_CUDA;
-    b_codes = static_cast<const uint8_t*>(ws);
-    p.b_scales = wt_scales;
+    Kp = g.Cop; p.Hs = g.Ho; p.Ws = g.Wo; p.Hd = g.H; p.Wd = g.W; p.Cd = g.Cin; out->rows_b = g.Cp;
     p.tiles_h = (g.H + g.sh - 1) / g.sh; p.classes = g.sh * g.sw;
   }
   p.Kblocks = Kp / 32;
   const int rowbytes = Kp * bits / 8;
+  out->rowbytes = rowbytes;
   p.KB = rowbytes % 128 == 0 ? 128 : (rowbytes % 64 == 0 ? 64 : 32);
   p.G = 128 / p.KB;
   p.cpt = rowbytes / p.KB;
   const int w_eff = op == MQ_OP_FWD ? g.Wo : (g.W + g.sw - 1) / g.sw;
   p.TW = choose_tw(w_eff, g.N, layout);
-  if (p.TW < 1 || p.TW > 32 || (p.TW & (p.TW - 1))) return MQ_ERR_INVALID_ARG;
+  if (p.TW < 1 || p.TW > 32 || (p.TW & (p.TW - 1))) return false;
   p.TN = 128 / p.TW;
   p.lgTW = 0;
   while ((1 << p.lgTW) < p.TW) ++p.lgTW;
@@ -142,21 +140,66 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
   p.tiles_w = (w_eff + p.TW - 1) / p.TW;
   p.tiles_n = (g.N + p.TN - 1) / p.TN;
   p.total_tiles = (long long)p.tiles_c * p.tiles_w * p.tiles_n * p.tiles_h * p.classes;
-  p.n_acc = (2 * p.BN + 48 <= 512) ? 2 : 1;
+  if (p.total_tiles > 0x7fffffffLL) return false;
   const size_t stage_bytes = 128 * 128 + (size_t)p.BN * 128 + 3072;
   int stages = (int)((227 * 1024 - 2048) / stage_bytes);
   if (stages > 8) stages = 8;
-  if (stages < 2) return MQ_ERR_UNSUPPORTED;
+  if (stages < 2) return false;
   p.stages = stages;
-  const uint32_t fa = fp4 ? 1u : (qx_like->fmt == MQ_E5M2 ? 1u : 0u);
-  const uint32_t fb = fp4 ? 1u : (qw->fmt == MQ_E5M2 ? 1u : 0u);
+  // TMEM (512 columns): accumulators (BN columns each) + one 24-column scale buffer per pipeline stage
+  p.n_acc = (2 * p.BN + 24 * stages <= 512) ? 2 : 1;
+  if (p.n_acc * p.BN + 24 * stages > 512) return false;
+  const int nkh = op == MQ_OP_FWD ? g.Kh : (g.Kh + g.sh - 1) / g.sh, nkw = op == MQ_OP_FWD ? g.Kw : (g.Kw + g.sw - 1) / g.sw;
+  p.max_stages = (nkh * nkw * p.cpt + p.G - 1) / p.G;
+  const uint32_t fa = fp4 ? 1u : (fmt_x_like == MQ_E5M2 ? 1u : 0u);
+  const uint32_t fb = fp4 ? 1u : (fmt_w == MQ_E5M2 ? 1u : 0u);
   p.idesc = (fa << 7) | (fb << 10) | ((uint32_t)(p.BN >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
+  out->p = p;
+  size_t o = 0;
+  out->off_wt_scales = 0;
+  if (op == MQ_OP_BWD_DATA) { o = wt_codes_bytes(g, fmt_w); out->off_wt_scales = o; o += up256((size_t)g.Ct * taps * g.Cot); }
+  out->off_sfa = o; o += up256(conv_tc_sfa_bytes(p));
+  out->off_sfb = o; o += up256(conv_tc_sfb_bytes(p));
+  out->total = o;
+  return true;
+}
+
+size_t conv_tc_workspace(int op, const Geom& g, int fmt_x_like, int fmt_w) {
+  size_t need = 0;
+  for (int layout = 0; layout < 2; ++layout) {   // the tile shape, hence the scratch, depends on the output layout
+    ConvTcPlan pl;
+    if (conv_tc_plan(op, g, fmt_x_like, fmt_w, layout, &pl) && pl.total > need) need = pl.total;
+  }
+  return need;
+}
+
+mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq_qtensor* qw, float* out, int layout, void* ws,
+                      unsigned int* status, cudaStream_t stream) {
+  ConvTcPlan pl;
+  if (!conv_tc_plan(op, g, qx_like->fmt, qw->fmt, layout, &pl)) return MQ_ERR_UNSUPPORTED;
+  ConvTcParams& p = pl.p;
+  const int taps = g.Kh * g.Kw;
+  uint8_t* base = static_cast<uint8_t*>(ws);
+  const uint8_t* b_codes;
+  if (op == MQ_OP_FWD) {
+    b_codes = static_cast<const uint8_t*>(qw->codes);
+    p.b_scales = qw->scales;
+  } else {
+    uint8_t* wt_scales = base + pl.off_wt_scales;
+    if (launch_weight_transpose(static_cast<const uint8_t*>(qw->codes), qw->scales, base, wt_scales, g, qw->fmt, stream) != cudaSuccess)
+      return MQ_ERR_CUDA;
+    b_codes = base;
+    p.b_scales = wt_scales;
+  }
   p.a_scales = qx_like->scales;
+  p.sfa_img = base + pl.off_sfa;
+  p.sfb_img = base + pl.off_sfb;
   p.out = out; p.out_layout = layout; p.status = status;
+  if (launch_expand_conv_scales(p, stream) != cudaSuccess) return MQ_ERR_CUDA;
 
   CUtensorMap map_a, map_b;
   {
-    const uint64_t rb = (uint64_t)rowbytes;
+    const uint64_t rb = (uint64_t)pl.rowbytes;
     const uint64_t dims[4] = {rb, (uint64_t)p.Ws, (uint64_t)g.N, (uint64_t)p.Hs};
     const uint64_t strides[3] = {(uint64_t)g.N * rb, rb, (uint64_t)p.Ws * g.N * rb};
     const uint32_t wst = op == MQ_OP_FWD ? (uint32_t)g.sw : 1u;
@@ -165,8 +208,8 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
     if (!encode_tensor_map_u8(&map_a, qx_like->codes, 4, dims, strides, box, es, p.KB)) return MQ_ERR_CUDA;
   }
   {
-    const uint64_t rb = (uint64_t)rowbytes;
-    const uint64_t dims[3] = {rb, (uint64_t)taps, (uint64_t)rows_b};
+    const uint64_t rb = (uint64_t)pl.rowbytes;
+    const uint64_t dims[3] = {rb, (uint64_t)taps, (uint64_t)pl.rows_b};
     const uint64_t strides[2] = {rb, (uint64_t)taps * rb};
     const uint32_t box[3] = {(uint32_t)p.KB, 1u, (uint32_t)p.BN};
     if (!encode_tensor_map_u8(&map_b, b_codes, 3, dims, strides, box, nullptr, p.KB)) return MQ_ERR_CUDA;
@@ -340,7 +383,8 @@ mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt
   if (op != MQ_OP_FWD && op != MQ_OP_BWD_DATA && op != MQ_OP_BWD_WEIGHT) return MQ_ERR_INVALID_ARG;
   const Geom g = make_geom(*desc);
   *bytes = conv_generic_workspace(op, g);
-  if (op == MQ_OP_BWD_DATA && conv_tc_eligible(op, g, fmt_b, fmt_a)) *bytes = conv_tc_workspace(op, g, fmt_a);
+  if (op == MQ_OP_FWD && conv_tc_eligible(op, g, fmt_a, fmt_b)) *bytes = conv_tc_workspace(op, g, fmt_a, fmt_b);
+  if (op == MQ_OP_BWD_DATA && conv_tc_eligible(op, g, fmt_b, fmt_a)) *bytes = conv_tc_workspace(op, g, fmt_b, fmt_a);
   if (op == MQ_OP_BWD_WEIGHT) {
     const WgradPlan w = wgrad_plan(g, fmt_a, fmt_b);
     if (w.ok) *bytes = w.total_bytes;
@@ -511,6 +555,8 @@ mq_status mq_conv_layer_host(const mq_conv_desc* desc, int fmt_x, int fmt_w, int
   if (cudaMemcpyAsync(dw_host, base + L.off_dw, L.nw, cudaMemcpyDeviceToHost, s) != cudaSuccess) return MQ_ERR_CUDA;
   return MQ_OK;
 }
+
+unsigned long long mq_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 const char* mq_status_string(int status) {
   switch (status) {

@@ -264,6 +264,7 @@ cudaError_t launch_bwd_weight_reduce(const float* partial, float* out, const Geo
   unsigned blocks = (unsigned)((total + 255) / 256);
   if (blocks > 148u * 16) blocks = 148u * 16;
   bwd_weight_reduce<<<blocks, 256, 0, s>>>(partial, out, g, splits, layout);
+  count_launches(1);
   return cudaGetLastError();
 }
 
@@ -302,7 +303,9 @@ cudaError_t launch_conv_generic(int op, const ConvArgs& a, cudaStream_t s) {
     unsigned blocks = (unsigned)((total + 255) / 256);
     if (blocks > 148u * 16) blocks = 148u * 16;
     bwd_weight_reduce<<<blocks, 256, 0, s>>>(reinterpret_cast<const float*>(a.workspace), a.out, g, splits, a.out_layout);
+    count_launches(1);
   }
+  count_launches(1);
   return cudaGetLastError();
 }
 

@@ -4,11 +4,15 @@
 // (the im2col of Sec. IV-A is implicit: every tap is a shifted TMA box, out-of-image taps are the
 // TMA zero fill).
 //
+// A small kernel first expands the compact tile scales (one E8M0 byte per 32x32 tile) into the per-row
+// scale-vector chunks the MMA reads, one chunk per (tile, pipeline stage), in scratch.
+//
 // One persistent thread block per SM, 12 warps:
-//   warp 0   TMA producer        one lane issues the A (gathered activation) and B (weight) boxes
-//   warp 1   MMA issuer          one lane copies the stage's scale vectors smem -> TMEM and issues the MMAs
-//   warps 2-3 scale expanders    (alternating stages) turn the compact tile scales (one E8M0 byte per 32x32 tile) into the
-//                                per-row scale vectors the MMA reads, for the tap / K-block of each stage
+//   warp 0   TMA producer        one lane issues the A (gathered activation) and B (weight) boxes and the
+//                                bulk copies of the stage's two scale chunks
+//   warp 1   MMA issuer          one lane issues the stage's MMAs
+//   warp 2   scale copier        one lane copies the stage's scale chunks smem -> TMEM (tcgen05.cp), one stage
+//                                ahead of the MMA issuer and from its own thread so the copies overlap the MMAs
 //   warps 4-11 epilogue          TMEM -> registers -> global (fp32), overlapped with the next tile's main loop;
 //                                two warps per TMEM lane quadrant, each taking half of the tile's columns
 // A pipeline stage holds 128 bytes of K per row (four MMAs): one 128-byte box, or 128/KB boxes of KB
@@ -109,7 +113,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const int stage_bytes = A_STAGE_BYTES + b_stage_bytes + SFA_BYTES + SFB_BYTES;
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * stage_bytes);
   uint64_t* empty = full + p.stages;
-  uint64_t* tfull = empty + p.stages;
+  uint64_t* sffull = empty + p.stages;     // scale vectors of the stage have landed in TMEM
+  uint64_t* tfull = sffull + p.stages;
   uint64_t* tempty = tfull + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -119,7 +124,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const unsigned total = (unsigned)p.total_tiles;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 2); mbar_init(&empty[s], 1); }
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 8); }
     *abort_flag = 0;
     mbar_fence_init();
@@ -144,12 +149,19 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int Q = tw.chunks(p);
         ChunkPos pos;
         pos.reset();
+        const unsigned tm = t / (unsigned)p.tiles_c;    // tile index without the channel tile
+        const uint8_t* sfa_src = p.sfa_img + (size_t)tm * p.max_stages * (512 * SPA);
+        const uint8_t* sfb_src = p.sfb_img + ((size_t)tile.cls * p.tiles_c + (t - tm * p.tiles_c)) * p.max_stages * (512 * SPA * atoms_b);
         for (int q0 = 0; q0 < Q; q0 += G) {
           if (!PROF_WAIT(mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
           const int nch = min(G, Q - q0);
           uint8_t* sa = smem + (size_t)s * stage_bytes;
           uint8_t* sb = sa + A_STAGE_BYTES;
-          mbar_arrive_expect_tx(&full[s], (uint32_t)nch * (128 + p.BN) * KB);
+          mbar_arrive_expect_tx(&full[s], (uint32_t)nch * (128 + p.BN) * KB + 512 * SPA * (1 + atoms_b));
+          bulk_load(sb + b_stage_bytes, sfa_src, 512 * SPA, &full[s]);
+          bulk_load(sb + b_stage_bytes + SFA_BYTES, sfb_src, 512 * SPA * atoms_b, &full[s]);
+          sfa_src += 512 * SPA;
+          sfb_src += 512 * SPA * atoms_b;
 #pragma unroll
           for (int c = 0; c < G; ++c) {
             if (c < nch) {
@@ -167,18 +179,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       const uint64_t op_desc = smem_desc_base(16, 8 * KB, LAYOUT);
-      const uint64_t sf_desc = smem_desc_base(0, 128, 0);
       const uint32_t sf_base = tmem + p.n_acc * p.BN;
       const uint32_t stage16 = (uint32_t)stage_bytes >> 4;
       const uint64_t a_desc0 = smem_desc(op_desc, smem_u32(smem));
       const uint64_t b_desc0 = smem_desc(op_desc, smem_u32(smem + A_STAGE_BYTES));
-      const uint64_t sfa_desc0 = smem_desc(sf_desc, smem_u32(smem + A_STAGE_BYTES + b_stage_bytes));
-      const uint64_t sfb_desc0 = smem_desc(sf_desc, smem_u32(smem + A_STAGE_BYTES + b_stage_bytes + SFA_BYTES));
       const uint32_t b_chunk16 = (uint32_t)(p.BN * KB) >> 4;
       uint32_t idesc_id[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) idesc_id[i] = idesc_with_sf_ids(p.idesc, i, i);
-      uint32_t s = 0, phase = 0, sfbuf = 0, tcount = 0;
+      uint32_t s = 0, phase = 0, tcount = 0;
       PROF_BEGIN();
       for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
         const Tile tile = decode_tile(p, t);
@@ -191,20 +200,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const uint32_t d_tmem = tmem + acc * p.BN;
         uint32_t accumulate = 0;
         for (int q0 = 0; q0 < Q; q0 += G) {
-          if (!PROF_WAIT(mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+          // the scale copier signals sffull[s] once the stage's operands are in smem and its scale vectors in TMEM
+          if (!PROF_WAIT(mbar_wait(&sffull[s], phase, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
           tc_fence_after_sync();
           const uint32_t so = s * stage16;
-          const uint32_t sfa_t = sf_base + sfbuf * SF_COLS, sfb_t = sfa_t + 8;
-#pragma unroll
-          for (int g = 0; g < SPA; ++g) {
-            tmem_cp_32x128b_warpx4(sfa_t + 4 * g, sfa_desc0 + so + g * 32);
-            for (int a = 0; a < atoms_b; ++a) tmem_cp_32x128b_warpx4(sfb_t + 4 * (g * atoms_b + a), sfb_desc0 + so + (g * atoms_b + a) * 32);
-          }
+          const uint32_t sfa_t = sf_base + s * SF_COLS, sfb_t = sfa_t + 8;
           const int natoms = min(G, Q - q0) * APC;
 #pragma unroll
           for (int a = 0; a < 4; ++a) {
             if (a < natoms) {
-              constexpr int dummy = 0; (void)dummy;
               const int c = a / APC, ja = a % APC;
               const uint64_t ad = a_desc0 + so + c * ((128 * KB) >> 4) + ja * 2;
               const uint64_t bd = b_desc0 + so + c * b_chunk16 + ja * 2;
@@ -215,150 +219,45 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             }
           }
           tc_commit(&empty[s]);
-          sfbuf ^= 1;
           if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
         }
         if (Q > 0) tc_commit(&tfull[acc]); else mbar_arrive(&tfull[acc]);
       }
       PROF_END(1);
     }
-  } else if (warp == 2 || warp == 3) {
-    // ------------------------------------------------------------------ scale expanders (two warps, alternate stages)
-    // The scale bytes of a chunk (one tap, KB bytes of channels) are contiguous in the stored scale
-    // tensor, so a lane fetches them with one naturally aligned load.  Loads are issued RING stages
-    // ahead of the stage being assembled and stay untouched in registers until then, which hides
-    // their latency behind the pipeline.
-    constexpr int RING = 4;
-    const int NTL = p.TN >= 32 ? p.TN / 32 : 1;
-    const int ncombos = p.TW * NTL;
-    const int wstep = MODE == MQ_OP_FWD ? p.sw : 1;
-    const int taps_all = p.Kh * p.Kw;
-    const int ctw = lane / NTL, cnl = lane - ctw * NTL;   // this lane's A combo: column offset, 32-sample block
-    // source lanes of the four rows 32j + lane this lane writes (row = tn * TW + tw)
-    int src_lane[4];
+  } else if (warp == 2) {
+    // ------------------------------------------------------------------ scale copier
+    // Copies the stage's scale chunks smem -> TMEM (one TMEM scale buffer per pipeline stage) from its own
+    // thread, so these copies overlap the MMA issuer's work on earlier stages.  The buffer of stage s is free
+    // whenever full[s] completes: the producer refilled the stage only after the MMAs that read it committed.
+    if (lane == 0) {
+      const uint64_t sf_desc = smem_desc_base(0, 128, 0);
+      const uint32_t sf_base = tmem + p.n_acc * p.BN;
+      const uint32_t stage16 = (uint32_t)stage_bytes >> 4;
+      const uint64_t sfa_desc0 = smem_desc(sf_desc, smem_u32(smem + A_STAGE_BYTES + b_stage_bytes));
+      const uint64_t sfb_desc0 = smem_desc(sf_desc, smem_u32(smem + A_STAGE_BYTES + b_stage_bytes + SFA_BYTES));
+      uint32_t s = 0, phase = 0;
+      bool alive = true;
+      for (unsigned t = blockIdx.x; t < total && alive && !*abort_flag; t += gridDim.x) {
+        const Tile tile = decode_tile(p, t);
+        TapWalk<MODE> tw;
+        tw.init(p, tile);
+        const int Q = tw.chunks(p);
+        for (int q0 = 0; q0 < Q; q0 += G) {
+          if (!mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; alive = false; break; }
+          tc_fence_after_sync();
+          const uint32_t so = s * stage16;
+          const uint32_t sfa_t = sf_base + s * SF_COLS, sfb_t = sfa_t + 8;
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      const int r = 32 * j + lane;
-      src_lane[j] = (r & (p.TW - 1)) * NTL + ((r >> p.lgTW) >> 5);
-    }
-    struct Walk {
-      unsigned t; Tile tile; TapWalk<MODE> tw; ChunkPos pos; int Q, q0; bool done;
-      bool a_ok, b_ok; int a_nt; long long b_row;
-    };
-    auto load_tile = [&](Walk& w) {
-      while (w.t < total) {
-        w.tile = decode_tile(p, w.t);
-        w.tw.init(p, w.tile);
-        w.Q = w.tw.chunks(p);
-        if (w.Q > 0) {
-          w.q0 = 0; w.pos.reset();
-          w.a_ok = lane < ncombos && (w.tile.n0 + cnl * 32) < p.N;
-          w.a_nt = (w.tile.n0 + cnl * 32) >> 5;
-          w.b_ok = lane < (p.BN + 31) / 32 && (w.tile.c0 + lane * 32) < p.Cd;
-          w.b_row = (long long)((w.tile.c0 >> 5) + lane) * taps_all;
-          return;
-        }
-        w.t += gridDim.x;
-      }
-      w.done = true;
-    };
-    // raw loads of one stage: up to G chunks x (A, B), 32 bits each (two words when a chunk has 8 bytes)
-    struct Raw { uint32_t a[G == 1 ? 2 : G]; uint32_t b[G == 1 ? 2 : G]; };
-    auto ld = [&](const uint8_t* ptr, uint32_t* dst) {
-      if (BPC == 1) dst[0] = __ldg(ptr);
-      else if (BPC == 2) dst[0] = __ldg(reinterpret_cast<const unsigned short*>(ptr));
-      else if (BPC == 4) dst[0] = __ldg(reinterpret_cast<const unsigned int*>(ptr));
-      else { const uint2 v = __ldg(reinterpret_cast<const uint2*>(ptr)); dst[0] = v.x; dst[1] = v.y; }
-    };
-    auto sf_load = [&](Walk& w, Raw& r) {
-#pragma unroll
-      for (int i = 0; i < (G == 1 ? 2 : G); ++i) { r.a[i] = 0u; r.b[i] = 0u; }
-#pragma unroll
-      for (int c = 0; c < G; ++c) {
-        if (w.q0 + c < w.Q) {
-          const int hs = src_h(w.tw, w.pos), ws = src_w0(w.tw, w.pos) + ctw * wstep;
-          if (w.a_ok && hs >= 0 && hs < p.Hs && ws >= 0 && ws < p.Ws)
-            ld(p.a_scales + (((long long)hs * p.Ws + ws) * p.Nt + w.a_nt) * p.Kblocks + w.pos.cc * BPC, &r.a[c]);
-          if (w.b_ok) ld(p.b_scales + (w.b_row + tap_index(w.tw, w.pos)) * p.Kblocks + w.pos.cc * BPC, &r.b[c]);
-          w.pos.advance(w.tw, p.cpt);
-        }
-      }
-      w.q0 += G;
-      if (w.q0 >= w.Q) { w.t += gridDim.x; load_tile(w); }
-    };
-    // stage scale words (4 bytes per group) from the raw chunk loads
-    auto word = [&](const uint32_t* raw, int g) -> uint32_t {
-      if (BPC == 8) return raw[g];                                   // G == 1: word g of the 8 bytes
-      if (BPC == 4) return raw[g];                                   // FP8 KB=128 (G=1, g=0) or FP4 KB=64 (G=2: chunk g)
-      if (BPC == 2) return G == 2 ? (raw[0] | (raw[1] << 16))        // FP8 KB=64: two chunks of 2 bytes, one group
-                                  : (raw[2 * g] | (raw[2 * g + 1] << 16));  // FP4 KB=32: four chunks of 2 bytes, two groups
-      return raw[0] | (raw[1] << 8) | (raw[2] << 16) | (raw[3] << 24);      // FP8 KB=32: four chunks of 1 byte
-    };
-    // advance a walk by one stage without loading (the other scale warp's stage)
-    auto sf_skip = [&](Walk& w) {
-#pragma unroll
-      for (int c = 0; c < G; ++c)
-        if (w.q0 + c < w.Q) w.pos.advance(w.tw, p.cpt);
-      w.q0 += G;
-      if (w.q0 >= w.Q) { w.t += gridDim.x; load_tile(w); }
-    };
-    Walk pre;
-    pre.t = blockIdx.x; pre.done = false; load_tile(pre);
-    if (warp == 3 && !pre.done) sf_skip(pre);
-    unsigned n_stages_left = 0;   // stages this block will run: count by walking the tiles once
-    for (unsigned t = blockIdx.x; t < total; t += gridDim.x) {
-      const Tile tile = decode_tile(p, t);
-      TapWalk<MODE> tw;
-      tw.init(p, tile);
-      n_stages_left += (tw.chunks(p) + G - 1) / G;
-    }
-    Raw ring[RING];
-#pragma unroll
-    for (int d = 0; d < RING; ++d) {
-#pragma unroll
-      for (int i = 0; i < (G == 1 ? 2 : G); ++i) { ring[d].a[i] = 0u; ring[d].b[i] = 0u; }
-      if (!pre.done) sf_load(pre, ring[d]);
-      if (!pre.done) sf_skip(pre);
-    }
-    uint32_t s = 0, phase = 0;
-    auto advance_stage = [&]() { if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; } };
-    if (warp == 3 && n_stages_left > 0) { advance_stage(); --n_stages_left; }
-    bool alive = true;
-    PROF_BEGIN();
-    while (alive && n_stages_left > 0) {
-#pragma unroll
-      for (int d = 0; d < RING; ++d) {
-        if (n_stages_left == 0 || !alive) break;
-        bool ok = true;
-        if (lane == 0) ok = !*abort_flag && PROF_WAIT(mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT));
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (!ok) { *abort_flag = 1; alive = false; break; }
-        uint8_t* sfa = smem + (size_t)s * stage_bytes + A_STAGE_BYTES + b_stage_bytes;
-        uint8_t* sfb = sfa + SFA_BYTES;
-#pragma unroll
-        for (int g = 0; g < SPA; ++g) {
-          const uint32_t aw = word(ring[d].a, g), bw = word(ring[d].b, g);
-          uint32_t w4[4];
-#pragma unroll
-          for (int j = 0; j < 4; ++j) w4[j] = __shfl_sync(0xffffffffu, aw, src_lane[j]);
-          *reinterpret_cast<uint4*>(sfa + g * 512 + lane * 16) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
-          for (int a = 0; a < atoms_b; ++a) {
-#pragma unroll
-            for (int j = 0; j < 4; ++j) w4[j] = __shfl_sync(0xffffffffu, bw, 4 * a + j);
-            *reinterpret_cast<uint4*>(sfb + (g * atoms_b + a) * 512 + lane * 16) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+          for (int g = 0; g < SPA; ++g) {
+            tmem_cp_32x128b_warpx4(sfa_t + 4 * g, sfa_desc0 + so + g * 32);
+            for (int a = 0; a < atoms_b; ++a) tmem_cp_32x128b_warpx4(sfb_t + 4 * (g * atoms_b + a), sfb_desc0 + so + (g * atoms_b + a) * 32);
           }
+          tc_commit(&sffull[s]);
+          if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
         }
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&full[s]);
-        advance_stage();
-        --n_stages_left;
-        if (n_stages_left > 0) { advance_stage(); --n_stages_left; }   // the other scale warp's stage
-        if (!pre.done) sf_load(pre, ring[d]);
-        if (!pre.done) sf_skip(pre);
       }
     }
-    if (lane == 0 && warp == 2) PROF_END(2);
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ epilogue
     const int quad = warp & 3;           // TMEM lane quadrant this warp may read
@@ -432,6 +331,103 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem, 512);
+}
+
+// ---- scale expansion --------------------------------------------------------------------------------
+// One warp per (tile, stage): writes the 512-byte scale-vector chunk(s) the MMA of that stage reads --
+// row r of the tile at byte (r % 32) * 16 + (r / 32) * 4, four consecutive K-blocks per 32-bit word --
+// from the compact tile scales.  A-side chunks exist per tile (without its channel index), B-side
+// chunks per (stride class, channel tile).
+template <int BPC>
+__device__ __forceinline__ unsigned long long load_scale_bytes(const uint8_t* ptr) {
+  if (BPC == 1) return __ldg(ptr);
+  if (BPC == 2) return __ldg(reinterpret_cast<const unsigned short*>(ptr));
+  if (BPC == 4) return __ldg(reinterpret_cast<const unsigned int*>(ptr));
+  return __ldg(reinterpret_cast<const unsigned long long*>(ptr));
+}
+
+template <int MODE, int KB, bool FP4>
+__global__ void __launch_bounds__(256) expand_conv_scales_kernel(const ConvTcParams p, unsigned n_tile_m) {
+  constexpr int G = 128 / KB, APC = KB / 32, SPA = FP4 ? 2 : 1, BPC = APC * SPA;
+  const int lane = threadIdx.x & 31;
+  const unsigned wid = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const unsigned nA = n_tile_m * (unsigned)p.max_stages;
+  const unsigned nB = (unsigned)(p.classes * p.tiles_c * p.max_stages);
+  const int atoms_b = (p.BN + 127) / 128;
+  if (wid < nA) {
+    const unsigned tm = wid / (unsigned)p.max_stages;
+    const int st = (int)(wid - tm * p.max_stages);
+    const Tile tile = decode_tile(p, tm * (unsigned)p.tiles_c);
+    TapWalk<MODE> tw;
+    tw.init(p, tile);
+    const int Q = tw.chunks(p);
+    if (st * G >= Q) return;
+    const int wstep = MODE == MQ_OP_FWD ? p.sw : 1;
+    unsigned long long acc[4] = {0ull, 0ull, 0ull, 0ull};
+#pragma unroll
+    for (int c = 0; c < G; ++c) {
+      const int q = st * G + c;
+      if (q < Q) {
+        ChunkPos pos;
+        const int per_row = tw.nkw * p.cpt;
+        pos.ia = q / per_row;
+        const int rem = q - pos.ia * per_row;
+        pos.ib = rem / p.cpt;
+        pos.cc = rem - pos.ib * p.cpt;
+        const int hs = src_h(tw, pos), ws0 = src_w0(tw, pos);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int r = 32 * j + lane;
+          const int tw_ = r & (p.TW - 1), tn = r >> p.lgTW;
+          const int n = tile.n0 + tn, ws = ws0 + tw_ * wstep;
+          if (n < p.N && hs >= 0 && hs < p.Hs && ws >= 0 && ws < p.Ws)
+            acc[j] |= load_scale_bytes<BPC>(p.a_scales + (((long long)hs * p.Ws + ws) * p.Nt + (n >> 5)) * p.Kblocks + pos.cc * BPC) << (8 * c * BPC);
+        }
+      }
+    }
+    uint8_t* dst = p.sfa_img + (size_t)wid * (512 * SPA) + lane * 16;
+#pragma unroll
+    for (int g = 0; g < SPA; ++g)
+      *reinterpret_cast<uint4*>(dst + g * 512) = make_uint4((uint32_t)(acc[0] >> (32 * g)), (uint32_t)(acc[1] >> (32 * g)), (uint32_t)(acc[2] >> (32 * g)),
+                                                          (uint32_t)(acc[3] >> (32 * g)));
+  } else if (wid < nA + nB) {
+    unsigned idx = wid - nA;
+    const int st = (int)(idx % (unsigned)p.max_stages); idx /= (unsigned)p.max_stages;
+    const int ct = (int)(idx % (unsigned)p.tiles_c);
+    Tile tile;
+    tile.cls = (int)(idx / (unsigned)p.tiles_c); tile.c0 = ct * p.BN; tile.w0 = 0; tile.n0 = 0; tile.h = 0;
+    TapWalk<MODE> tw;
+    tw.init(p, tile);
+    const int Q = tw.chunks(p);
+    if (st * G >= Q) return;
+    const int taps_all = p.Kh * p.Kw;
+    unsigned long long acc[8] = {0ull, 0ull, 0ull, 0ull, 0ull, 0ull, 0ull, 0ull};
+#pragma unroll
+    for (int c = 0; c < G; ++c) {
+      const int q = st * G + c;
+      if (q < Q) {
+        ChunkPos pos;
+        const int per_row = tw.nkw * p.cpt;
+        pos.ia = q / per_row;
+        const int rem = q - pos.ia * per_row;
+        pos.ib = rem / p.cpt;
+        pos.cc = rem - pos.ib * p.cpt;
+        const int tap = tap_index(tw, pos);
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (j < 4 * atoms_b && 32 * j < p.BN && tile.c0 + 32 * j < p.Cd)
+            acc[j] |= load_scale_bytes<BPC>(p.b_scales + ((long long)((tile.c0 >> 5) + j) * taps_all + tap) * p.Kblocks + pos.cc * BPC) << (8 * c * BPC);
+        }
+      }
+    }
+    uint8_t* dst = p.sfb_img + (size_t)(wid - nA) * (512 * SPA * atoms_b) + lane * 16;
+#pragma unroll
+    for (int g = 0; g < SPA; ++g)
+      for (int a = 0; a < atoms_b; ++a)
+        *reinterpret_cast<uint4*>(dst + (g * atoms_b + a) * 512) =
+            make_uint4((uint32_t)(acc[4 * a] >> (32 * g)), (uint32_t)(acc[4 * a + 1] >> (32 * g)), (uint32_t)(acc[4 * a + 2] >> (32 * g)),
+                       (uint32_t)(acc[4 * a + 3] >> (32 * g)));
+  }
 }
 
 // ---- W -> W^T re-layout (codes only; scales are indexed in place) ------------------------------
@@ -515,7 +511,7 @@ bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const ui
 
 size_t conv_tc_smem_bytes(const ConvTcParams& p) {
   const size_t stage = A_STAGE_BYTES + (size_t)p.BN * 128 + SFA_BYTES + SFB_BYTES;
-  return 1024 + (size_t)p.stages * stage + (2 * (size_t)p.stages + 4) * 8 + 64;
+  return 1024 + (size_t)p.stages * stage + (3 * (size_t)p.stages + 4) * 8 + 64;
 }
 
 template <int MODE, int KB, bool FP4>
@@ -532,7 +528,35 @@ cudaError_t launch_conv_tc_inst(const ConvTcParams& p, const CUtensorMap& map_a,
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const unsigned grid = (unsigned)(p.total_tiles < sms ? p.total_tiles : sms);
   conv_tc_kernel<MODE, KB, FP4><<<grid, TC_THREADS, smem, s>>>(map_a, map_b, p);
+  count_launches(1);
   return cudaGetLastError();
+}
+
+size_t conv_tc_sfa_bytes(const ConvTcParams& p) {
+  return (size_t)(p.total_tiles / p.tiles_c) * p.max_stages * 512 * (p.kind_fp4 ? 2 : 1);
+}
+size_t conv_tc_sfb_bytes(const ConvTcParams& p) {
+  return (size_t)p.classes * p.tiles_c * p.max_stages * 512 * (p.kind_fp4 ? 2 : 1) * ((p.BN + 127) / 128);
+}
+
+template <int MODE, int KB, bool FP4>
+cudaError_t launch_expand_inst(const ConvTcParams& p, cudaStream_t s) {
+  const unsigned n_tile_m = (unsigned)(p.total_tiles / p.tiles_c);
+  const unsigned long long warps = (unsigned long long)n_tile_m * p.max_stages + (unsigned long long)p.classes * p.tiles_c * p.max_stages;
+  const unsigned blocks = (unsigned)((warps + 7) / 8);
+  expand_conv_scales_kernel<MODE, KB, FP4><<<blocks, 256, 0, s>>>(p, n_tile_m);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_expand_conv_scales(const ConvTcParams& p, cudaStream_t s) {
+#define MQ_TC_CASE(M, K, F) if (p.mode == M && p.KB == K && (p.kind_fp4 != 0) == F) return launch_expand_inst<M, K, F>(p, s)
+  MQ_TC_CASE(MQ_OP_FWD, 128, false); MQ_TC_CASE(MQ_OP_FWD, 64, false); MQ_TC_CASE(MQ_OP_FWD, 32, false);
+  MQ_TC_CASE(MQ_OP_FWD, 128, true);  MQ_TC_CASE(MQ_OP_FWD, 64, true);  MQ_TC_CASE(MQ_OP_FWD, 32, true);
+  MQ_TC_CASE(MQ_OP_BWD_DATA, 128, false); MQ_TC_CASE(MQ_OP_BWD_DATA, 64, false); MQ_TC_CASE(MQ_OP_BWD_DATA, 32, false);
+  MQ_TC_CASE(MQ_OP_BWD_DATA, 128, true);  MQ_TC_CASE(MQ_OP_BWD_DATA, 64, true);  MQ_TC_CASE(MQ_OP_BWD_DATA, 32, true);
+#undef MQ_TC_CASE
+  return cudaErrorInvalidValue;
 }
 
 cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s) {
@@ -550,6 +574,7 @@ cudaError_t launch_weight_transpose(const uint8_t* w_codes, const uint8_t* w_sca
                                     cudaStream_t s) {
   dim3 grid(g.Cp / 32, g.Cop / 32, g.Kh * g.Kw), block(32, 8);
   weight_transpose_kernel<<<grid, block, 0, s>>>(w_codes, wt_codes, w_scales, wt_scales, g.Cout, g.Cop, g.Cp, g.Kh * g.Kw, fmt == MQ_E2M1 ? 1 : 0);
+  count_launches(1);
   return cudaGetLastError();
 }
 

@@ -37,6 +37,10 @@ struct ConvTcParams {
   // scales
   const uint8_t* a_scales;  // [Hs][Ws][Nt][Kblocks]
   const uint8_t* b_scales;  // [row blocks of 32][taps][Kblocks]
+  // per-stage scale-vector chunks expanded by expand_conv_scales (scratch)
+  uint8_t* sfa_img;         // [tile without the channel index][max_stages][512 * SPA]
+  uint8_t* sfb_img;         // [class][channel tile][max_stages][512 * SPA * atoms_b]
+  int max_stages;           // stages of the longest tile
   // output
   float* out;
   int out_layout;
@@ -44,6 +48,10 @@ struct ConvTcParams {
 };
 
 cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s);
+// Expands the compact tile scales into the per-stage scale-vector chunks the MMA reads (p.sfa_img, p.sfb_img).
+cudaError_t launch_expand_conv_scales(const ConvTcParams& p, cudaStream_t s);
+size_t conv_tc_sfa_bytes(const ConvTcParams& p);
+size_t conv_tc_sfb_bytes(const ConvTcParams& p);
 size_t conv_tc_smem_bytes(const ConvTcParams& p);
 
 // Re-lays the stored weight codes [C_out][taps][C_in_p] as [C_in_p][taps][C_out_p] and the tile scales

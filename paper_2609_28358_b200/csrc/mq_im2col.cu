@@ -61,6 +61,7 @@ cudaError_t launch_im2col(const Im2colArgs& a, cudaStream_t s) {
   if (blocks > cap) blocks = cap;
   if (blocks <= 0) return cudaErrorInvalidValue;
   im2col_kernel<<<(unsigned)blocks, IC_THREADS, 0, s>>>(a, row_chunks, code_chunks, n_scales);
+  count_launches(1);
   return cudaGetLastError();
 }
 

@@ -37,6 +37,9 @@ inline Geom make_geom(const mq_conv_desc& d) {
 __host__ __device__ inline int fmt_bits(int fmt) { return fmt == MQ_E2M1 ? 4 : 8; }
 __host__ __device__ inline int fmt_emax(int fmt) { return fmt == MQ_E4M3 ? 8 : (fmt == MQ_E5M2 ? 15 : 2); }
 
+// Number of kernels the library has launched in this process (diagnostic; see mq_kernel_launch_count).
+void count_launches(int n);
+
 // ---- launchers (defined in the .cu files) ---------------------------------------------------
 struct QuantArgs {
   const float* src;

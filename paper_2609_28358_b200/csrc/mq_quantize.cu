@@ -8,6 +8,8 @@
 // (per-thread max, warp shuffles, one shared-memory exchange), derives the E8M0 code from the
 // exponent field of the maximum, converts with the hardware RNE+saturate conversions and stages
 // the codes in shared memory so the [n][c] slab of each position leaves as 16-byte stores.
+#include <cstdlib>
+
 #include "mq_internal.cuh"
 
 namespace mq {
@@ -26,18 +28,32 @@ __device__ __forceinline__ unsigned encode2(float lo, float hi) {
   }
 }
 
+// 128-bit read-only load that asks L2 to bring in the whole 128-byte line (the other sectors of the
+// line are read next, by this block's following sub-strips)
+__device__ __forceinline__ float4 ldg128_l2_128(const float* p) {
+  float4 v;
+  asm volatile("ld.global.nc.L2::128B.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
+  return v;
+}
+
 template <int FMT, bool VEC>
-__global__ void __launch_bounds__(QT_THREADS) quantize_kernel(QuantArgs a, int n_pstrips, int Rt, int Ct) {
+__global__ void __launch_bounds__(QT_THREADS) quantize_kernel(QuantArgs a, int n_pstrips, int Rt, int Ct, int loops, int hint) {
   __shared__ __align__(16) unsigned red[8][2][4];          // per-warp, per-quad partial maxima
   __shared__ __align__(16) uint8_t stage[PS][32][32];       // codes, one byte each, [p][r][c]
 
   const int t = threadIdx.x;
   const int lane = t & 31, warp = t >> 5;
   long long bid = blockIdx.x;
-  const int ps = (int)(bid % n_pstrips); bid /= n_pstrips;
+  const int n_groups = (n_pstrips + loops - 1) / loops;
+  const int psg = (int)(bid % n_groups); bid /= n_groups;
   const int ct = (int)(bid % Ct);
   const int rt = (int)(bid / Ct);
-  const int p0 = ps * PS, r0 = rt * 32, c0 = ct * 32;
+  const int r0 = rt * 32, c0 = ct * 32;
+  for (int sub = 0; sub < loops; ++sub) {
+  const int ps = psg * loops + sub;
+  if (ps >= n_pstrips) break;
+  const int p0 = ps * PS;
+  if (sub > 0) __syncthreads();   // previous sub-strip's copy-out has finished reading `stage` / `red`
 
   // thread -> (channel, position quad); 8 rows of the tile: r = 4*i + t/64
   const int quad = t & 1;
@@ -54,7 +70,7 @@ __global__ void __launch_bounds__(QT_THREADS) quantize_kernel(QuantArgs a, int n
     const float* row = a.src + ((long long)r * a.C + (c0 + c)) * a.P;
     if (VEC) {
       float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (ok && pq < a.P) f = __ldg(reinterpret_cast<const float4*>(row + pq));  // P % 4 == 0: whole quad valid
+      if (ok && pq < a.P) f = hint ? ldg128_l2_128(row + pq) : __ldg(reinterpret_cast<const float4*>(row + pq));  // P % 4 == 0: whole quad valid
       v[i][0] = f.x; v[i][1] = f.y; v[i][2] = f.z; v[i][3] = f.w;
     } else {
 #pragma unroll
@@ -147,6 +163,7 @@ __global__ void __launch_bounds__(QT_THREADS) quantize_kernel(QuantArgs a, int n
       }
     }
   }
+  }  // sub-strips
 }
 
 }  // namespace
@@ -154,13 +171,18 @@ __global__ void __launch_bounds__(QT_THREADS) quantize_kernel(QuantArgs a, int n
 cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s) {
   const int n_pstrips = (a.P + PS - 1) / PS;
   const int Rt = (a.R + 31) / 32, Ct = a.Cp / 32;
-  const long long blocks = (long long)n_pstrips * Rt * Ct;
+  static int variant = -1;
+  if (variant < 0) { const char* v = std::getenv("MQ_QUANT_VARIANT"); variant = v ? std::atoi(v) : 0; }
+  const int hint = variant >= 1 ? 1 : 0;
+  int loops = variant >= 2 ? 4 : 1;
+  if (variant == 3) loops = 2;
+  const long long blocks = (long long)((n_pstrips + loops - 1) / loops) * Rt * Ct;
   if (blocks <= 0 || blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
   const bool vec = (a.P % 4 == 0) && ((reinterpret_cast<uintptr_t>(a.src) & 15) == 0);
 #define MQ_LAUNCH_Q(F)                                                                                  \
   do {                                                                                                  \
-    if (vec) quantize_kernel<F, true><<<(unsigned)blocks, QT_THREADS, 0, s>>>(a, n_pstrips, Rt, Ct);    \
-    else     quantize_kernel<F, false><<<(unsigned)blocks, QT_THREADS, 0, s>>>(a, n_pstrips, Rt, Ct);   \
+    if (vec) quantize_kernel<F, true><<<(unsigned)blocks, QT_THREADS, 0, s>>>(a, n_pstrips, Rt, Ct, loops, hint);    \
+    else     quantize_kernel<F, false><<<(unsigned)blocks, QT_THREADS, 0, s>>>(a, n_pstrips, Rt, Ct, loops, hint);   \
   } while (0)
   switch (a.fmt) {
     case MQ_E4M3: MQ_LAUNCH_Q(MQ_E4M3); break;
@@ -169,6 +191,7 @@ cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s) {
     default: return cudaErrorInvalidValue;
   }
 #undef MQ_LAUNCH_Q
+  count_launches(1);
   return cudaGetLastError();
 }
 

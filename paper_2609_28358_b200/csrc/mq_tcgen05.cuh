@@ -77,6 +77,13 @@ __device__ __forceinline__ void tma_load_4d(void* dst, const void* map, uint64_t
                : "memory");
 }
 
+// plain (untiled) bulk copy global -> shared; both addresses 16-byte aligned, size a multiple of 16 bytes
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(dst)),
+               "l"(reinterpret_cast<uint64_t>(src)), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+
 // ---- tensor memory ----------------------------------------------------------------------------------
 // ncols: power of two in [32, 512].  Whole-warp (sync.aligned) instructions.
 __device__ __forceinline__ void tmem_alloc(uint32_t* dst_smem, uint32_t ncols) {

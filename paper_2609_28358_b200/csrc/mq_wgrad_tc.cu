@@ -319,12 +319,14 @@ cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, co
   const unsigned grid = (unsigned)(p.m_tiles * p.j_tiles * p.splits);
   if (f) wgrad_tc_kernel<true><<<grid, WG_THREADS, smem, s>>>(map_a, map_b, p);
   else wgrad_tc_kernel<false><<<grid, WG_THREADS, smem, s>>>(map_a, map_b, p);
+  count_launches(1);
   return cudaGetLastError();
 }
 
 cudaError_t launch_fp4_to_n_major(const uint8_t* in, uint8_t* out, int P, int N, int Cp, int Npad, cudaStream_t s) {
   dim3 grid((P + 7) / 8, Npad / 32, (Cp + 63) / 64);
   fp4_to_n_major_kernel<<<grid, 256, 0, s>>>(in, out, P, N, Cp, Npad);
+  count_launches(1);
   return cudaGetLastError();
 }
 

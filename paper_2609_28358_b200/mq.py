@@ -48,6 +48,7 @@ def lib():
                                "there is no fallback path")
         _lib = ctypes.CDLL(_LIB_PATH)
         _lib.mq_status_string.restype = ctypes.c_char_p
+        _lib.mq_kernel_launch_count.restype = ctypes.c_ulonglong
     return _lib
 
 
@@ -178,6 +179,10 @@ def conv_bwd_data_static(desc, wq, dyq, dx=None, layout=NCHW, stream=None):
 def conv_bwd_weight(desc, xq, dyq, dw=None, layout=NCHW, workspace=None, stream=None):
     d = ConvDesc(*desc)
     return _conv("mq_conv_bwd_weight", OP_BWD_WEIGHT, desc, xq, dyq, dw, (d.C_out, d.C_in, d.Kh, d.Kw), (d.C_out, d.Kh, d.Kw, d.C_in), layout, workspace, stream)
+
+
+def kernel_launch_count():
+    return int(lib().mq_kernel_launch_count())
 
 
 def last_device_status(stream=None):
