@@ -123,10 +123,11 @@ mq_status mq_conv_bwd_data(const mq_conv_desc* desc, const mq_qtensor* wq, const
  * a caller still supplies the inputs (wq, dyq) and the output (dx); only the scratch is taken care of.
  *
  * The scratch that mq_conv_bwd_data takes as `workspace` (the weight codes and tile scales re-laid for the
- * input-gradient GEMM) lives here in a static array inside the library's device image,
- * MQ_STATIC_SCRATCH_BYTES (4 MiB) long; every GPU that loads the library keeps that much memory reserved
- * until the process exits.  A layer whose mq_workspace_size(desc, MQ_OP_BWD_DATA, ...) exceeds it is
- * rejected with MQ_ERR_STATIC_SCRATCH and nothing is launched (512 x 512 x 3 x 3 FP8 weights need 2.4 MB).
+ * input-gradient GEMM, and the per-stage scale-vector chunks expanded from the tile scales) lives here in a
+ * static array inside the library's device image, MQ_STATIC_SCRATCH_BYTES (16 MiB) long; every GPU that
+ * loads the library keeps that much memory reserved until the process exits.  A layer whose
+ * mq_workspace_size(desc, MQ_OP_BWD_DATA, ...) exceeds it is rejected with MQ_ERR_STATIC_SCRATCH and nothing
+ * is launched (for scale: N=32, 128->64 channels, 80x80, 3x3 needs about 6 MB).
  * The call performs no cudaMalloc / cudaFree and calls no allocating library routine.
  *
  * First use on a device: the first call made while a given device is current looks up the array's device
@@ -134,7 +135,7 @@ mq_status mq_conv_bwd_data(const mq_conv_desc* desc, const mq_qtensor* wq, const
  * Sharing: all calls on a device use the same array and it keeps whatever the previous call left in it;
  * each call overwrites every byte it later reads, so nothing needs clearing, but two calls whose kernels
  * overlap on the GPU (different streams, no ordering between them) race on the array -- order them. */
-#define MQ_STATIC_SCRATCH_BYTES (4u << 20)
+#define MQ_STATIC_SCRATCH_BYTES (16u << 20)
 mq_status mq_conv_bwd_data_static(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, void* dx, int dx_layout,
                                   void* stream);
 

@@ -159,7 +159,7 @@ def conv_bwd_data(desc, wq, dyq, dx=None, layout=NCHW, workspace=None, stream=No
     return _conv("mq_conv_bwd_data", OP_BWD_DATA, desc, wq, dyq, dx, (d.N, d.C_in, d.H, d.W), (d.H, d.W, d.N, d.C_in), layout, workspace, stream)
 
 
-STATIC_SCRATCH_BYTES = 4 << 20
+STATIC_SCRATCH_BYTES = 16 << 20
 
 
 def conv_bwd_data_static(desc, wq, dyq, dx=None, layout=NCHW, stream=None):

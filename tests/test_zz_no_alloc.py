@@ -49,11 +49,11 @@ def test_static_scratch_variant_matches_workspace_variant_on_two_calls_in_a_row(
 
 
 def test_static_scratch_variant_rejects_layers_beyond_its_limit():
-    d = inputs.conv_desc(32, 1024, 8, 8, 1024, 3)      # 1024 x 1024 x 9 FP8 weights re-laid: 9.4 MB > 4 MiB
+    d = inputs.conv_desc(32, 2048, 8, 8, 1024, 3)      # 2048 x 1024 x 9 FP8 weights re-laid: 18.9 MB > 16 MiB
     assert mq.workspace_size(d, mq.OP_BWD_DATA, mq.E4M3, mq.E5M2) > mq.STATIC_SCRATCH_BYTES
     wq = mq.empty_qtensor(d, mq.ROLE_W, mq.E4M3)
     gq = mq.empty_qtensor(d, mq.ROLE_DY, mq.E5M2)
-    dx = torch.zeros((32, 1024, 8, 8), dtype=torch.float32, device="cuda")
+    dx = torch.zeros((32, 2048, 8, 8), dtype=torch.float32, device="cuda")
     with pytest.raises(mq.MqError) as e:
         mq.conv_bwd_data_static(d, wq, gq, dx=dx)
     assert e.value.status == 7 and "STATIC_SCRATCH" in str(e.value)
