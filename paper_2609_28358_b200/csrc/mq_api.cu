@@ -218,75 +218,93 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
 }
 
 // ---- weight gradient on tensor cores ---------------------------------------------------------------
+// Scratch: [split-K partials][A-side scale chunks][B-side scale chunks][E2M1: re-laid X][E2M1: re-laid G_Y]
 struct WgradPlan {
-  bool ok, fp4;
-  int BPP, KPX, KBn, nchunks, Npad, groups_w, stages_total, m_tiles, cb_tiles, j_tiles, splits;
-  size_t partial_bytes, xt_bytes, gt_bytes, total_bytes;
+  bool ok;
+  WgradTcParams p;
+  int Npad, P_a, P_b;
+  size_t off_sfa, off_sfb, off_xt, off_gt, total;
 };
 
 WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   WgradPlan w{};
   if (env_int("MQ_DISABLE_TC", 0) || env_int("MQ_DISABLE_TC_WGRAD", 0)) return w;
-  w.fp4 = fmt_x == MQ_E2M1 && fmt_g == MQ_E2M1;
+  const bool fp4 = fmt_x == MQ_E2M1 && fmt_g == MQ_E2M1;
   const bool fp8 = fmt_x != MQ_E2M1 && fmt_g != MQ_E2M1;
-  if (!w.fp4 && !fp8) return w;
-  if (w.fp4) w.BPP = g.Nt >= 5 ? 8 : (g.Nt >= 3 ? 4 : g.Nt);
-  else w.BPP = g.Nt >= 3 ? 4 : g.Nt;
-  w.KPX = (w.fp4 ? 8 : 4) / w.BPP;
-  w.KBn = 16 * w.BPP;
-  w.nchunks = (g.Nt + w.BPP - 1) / w.BPP;
-  w.Npad = 32 * w.BPP * w.nchunks;
-  w.groups_w = (g.Wo + w.KPX - 1) / w.KPX;
-  w.stages_total = g.Ho * w.groups_w * w.nchunks;
-  w.m_tiles = (g.Cout + 127) / 128;
-  w.cb_tiles = (g.Cp + 127) / 128;
-  w.j_tiles = g.Kh * g.Kw * w.cb_tiles;
-  const int items = w.m_tiles * w.j_tiles;
+  if (!fp4 && !fp8) return w;
+  WgradTcParams& p = w.p;
+  p.N = g.N; p.Nt = g.Nt; p.Ho = g.Ho; p.Wo = g.Wo; p.H = g.H; p.W = g.W; p.Cout = g.Cout; p.Cp = g.Cp; p.Ct = g.Ct; p.Cot = g.Cot;
+  p.Kh = g.Kh; p.Kw = g.Kw; p.sh = g.sh; p.sw = g.sw; p.ph = g.ph; p.pw = g.pw;
+  const bool flat = fp4 && g.sh == 1 && g.sw == 1 && (g.Nt == 1 || g.Nt == 2 || g.Nt == 4 || g.Nt == 8) && !env_int("MQ_WGRAD_NO_FLAT", 0);
+  p.mode = fp8 ? MQ_WG_FP8 : (flat ? MQ_WG_FP4_FLAT : MQ_WG_FP4_PIXEL);
+  if (fp4) p.BPP = flat ? g.Nt : (g.Nt >= 5 ? 8 : (g.Nt >= 3 ? 4 : g.Nt));
+  else p.BPP = g.Nt >= 3 ? 4 : g.Nt;
+  p.KPX = (fp4 ? 8 : 4) / p.BPP;
+  p.KBn = 16 * p.BPP;
+  p.nchunks = (g.Nt + p.BPP - 1) / p.BPP;
+  w.Npad = 32 * p.BPP * p.nchunks;
+  p.groups_w = (g.Wo + p.KPX - 1) / p.KPX;
+  p.Wp = g.W + 2 * g.pw;
+  p.stages_total = flat ? (g.Ho * p.Wp + p.KPX - 1) / p.KPX : g.Ho * p.groups_w * p.nchunks;
+  p.b_rows = flat ? (g.Cp < 128 ? g.Cp : 128) : 128;
+  p.m_tiles = (g.Cout + 127) / 128;
+  p.cb_tiles = (g.Cp + p.b_rows - 1) / p.b_rows;
+  p.j_tiles = g.Kh * g.Kw * p.cb_tiles;
+  const int items = p.m_tiles * p.j_tiles;
   int splits = env_int("MQ_WGRAD_SPLITS", 0);
   if (splits <= 0) splits = items >= 148 ? 1 : 148 / items;
-  if (splits > w.stages_total) splits = w.stages_total;
+  if (splits > p.stages_total) splits = p.stages_total;
   if (splits < 1) splits = 1;
-  w.splits = splits;
-  auto up = [](size_t v) { return (v + 255) / 256 * 256; };
-  w.partial_bytes = up((size_t)splits * g.Cout * g.Kh * g.Kw * g.Cp * sizeof(float));
-  w.xt_bytes = w.fp4 ? up((size_t)g.Cp * g.H * g.W * w.Npad / 2) : 0;
-  w.gt_bytes = w.fp4 ? up((size_t)g.Cop * g.Ho * g.Wo * w.Npad / 2) : 0;
-  w.total_bytes = w.partial_bytes + w.xt_bytes + w.gt_bytes;
+  p.splits = splits;
+  p.stages = 6;
+  const int spa = fp4 ? 2 : 1;
+  w.P_a = p.stages_total * p.KPX;
+  w.P_b = (w.P_a + (g.Kh - 1) * p.Wp + g.Kw - 1 + 7) / 8 * 8;
+  size_t o = up256((size_t)splits * g.Cout * g.Kh * g.Kw * g.Cp * sizeof(float));
+  w.off_sfa = o; o += up256((size_t)p.m_tiles * p.stages_total * 512 * spa);
+  w.off_sfb = o; o += up256((size_t)p.cb_tiles * g.Kh * g.Kw * p.stages_total * 512 * spa);
+  w.off_xt = o;
+  if (flat) { p.xt_block_bytes = (long long)w.P_b * p.b_rows * p.KBn; o += up256((size_t)p.cb_tiles * p.xt_block_bytes); }
+  else if (fp4) o += up256((size_t)g.Cp * g.H * g.W * w.Npad / 2);
+  w.off_gt = o;
+  if (flat) { p.gt_block_bytes = (long long)w.P_a * 128 * p.KBn; o += up256((size_t)p.m_tiles * p.gt_block_bytes); }
+  else if (fp4) o += up256((size_t)g.Cop * g.Ho * g.Wo * w.Npad / 2);
+  w.total = o;
   w.ok = true;
   return w;
 }
 
-mq_status run_wgrad_tc(const Geom& g, const WgradPlan& w, const mq_qtensor* qx, const mq_qtensor* qg, float* out, int layout, void* ws,
+mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const mq_qtensor* qg, float* out, int layout, void* ws,
                        unsigned int* status, cudaStream_t stream) {
   uint8_t* base = static_cast<uint8_t*>(ws);
   float* partial = reinterpret_cast<float*>(base);
-  WgradTcParams p{};
-  p.fp4 = w.fp4 ? 1 : 0;
-  p.N = g.N; p.Nt = g.Nt; p.Ho = g.Ho; p.Wo = g.Wo; p.H = g.H; p.W = g.W; p.Cout = g.Cout; p.Cp = g.Cp; p.Ct = g.Ct; p.Cot = g.Cot;
-  p.Kh = g.Kh; p.Kw = g.Kw; p.sh = g.sh; p.sw = g.sw; p.ph = g.ph; p.pw = g.pw;
-  p.BPP = w.BPP; p.KPX = w.KPX; p.KBn = w.KBn; p.nchunks = w.nchunks; p.groups_w = w.groups_w; p.stages_total = w.stages_total;
-  p.m_tiles = w.m_tiles; p.j_tiles = w.j_tiles; p.cb_tiles = w.cb_tiles; p.splits = w.splits;
+  WgradTcParams& p = w.p;
   p.g_scales = qg->scales; p.x_scales = qx->scales; p.partial = partial; p.status = status;
-  p.stages = 6;
-  CUtensorMap map_a, map_b;
-  if (w.fp4) {
-    uint8_t* xt = base + w.partial_bytes;
-    uint8_t* gt = xt + w.xt_bytes;
+  p.sfa_img = base + w.off_sfa; p.sfb_img = base + w.off_sfb;
+  uint8_t* xt = base + w.off_xt;
+  uint8_t* gt = base + w.off_gt;
+  CUtensorMap map_a{}, map_b{};
+  if (p.mode == MQ_WG_FP4_FLAT) {
+    if (launch_fp4_to_flat(static_cast<const uint8_t*>(qx->codes), xt, g.H, g.W, g.N, g.Cp, w.P_b, p.Wp, g.ph, g.pw, p.b_rows, p.cb_tiles, p.KBn, stream) != cudaSuccess) return MQ_ERR_CUDA;
+    if (launch_fp4_to_flat(static_cast<const uint8_t*>(qg->codes), gt, g.Ho, g.Wo, g.N, g.Cop, w.P_a, p.Wp, 0, 0, 128, p.m_tiles, p.KBn, stream) != cudaSuccess) return MQ_ERR_CUDA;
+    p.xt = xt; p.gt = gt;
+    p.idesc = (1u << 7) | (1u << 10) | ((uint32_t)(p.b_rows >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
+  } else if (p.mode == MQ_WG_FP4_PIXEL) {
     if (launch_fp4_to_n_major(static_cast<const uint8_t*>(qx->codes), xt, g.H * g.W, g.N, g.Cp, w.Npad, stream) != cudaSuccess) return MQ_ERR_CUDA;
     if (launch_fp4_to_n_major(static_cast<const uint8_t*>(qg->codes), gt, g.Ho * g.Wo, g.N, g.Cop, w.Npad, stream) != cudaSuccess) return MQ_ERR_CUDA;
     p.idesc = (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
     const uint64_t nb = (uint64_t)w.Npad / 2;
-    const int swz = w.KBn >= 32 ? w.KBn : 0;
+    const int swz = p.KBn >= 32 ? p.KBn : 0;
     {
       const uint64_t dims[4] = {nb, (uint64_t)g.Cop, (uint64_t)g.Wo, (uint64_t)g.Ho};
       const uint64_t strides[3] = {nb, (uint64_t)g.Cop * nb, (uint64_t)g.Wo * g.Cop * nb};
-      const uint32_t box[4] = {(uint32_t)w.KBn, 128u, 1u, 1u};
+      const uint32_t box[4] = {(uint32_t)p.KBn, 128u, 1u, 1u};
       if (!encode_tensor_map_u8(&map_a, gt, 4, dims, strides, box, nullptr, swz)) return MQ_ERR_CUDA;
     }
     {
       const uint64_t dims[4] = {nb, (uint64_t)g.Cp, (uint64_t)g.W, (uint64_t)g.H};
       const uint64_t strides[3] = {nb, (uint64_t)g.Cp * nb, (uint64_t)g.W * g.Cp * nb};
-      const uint32_t box[4] = {(uint32_t)w.KBn, 128u, 1u, 1u};
+      const uint32_t box[4] = {(uint32_t)p.KBn, 128u, 1u, 1u};
       if (!encode_tensor_map_u8(&map_b, xt, 4, dims, strides, box, nullptr, swz)) return MQ_ERR_CUDA;
     }
   } else {
@@ -296,20 +314,21 @@ mq_status run_wgrad_tc(const Geom& g, const WgradPlan& w, const mq_qtensor* qx, 
       const uint64_t rb = (uint64_t)g.Cop;
       const uint64_t dims[4] = {rb, (uint64_t)g.N, (uint64_t)g.Wo, (uint64_t)g.Ho};
       const uint64_t strides[3] = {rb, (uint64_t)g.N * rb, (uint64_t)g.Wo * g.N * rb};
-      const uint32_t box[4] = {128u, (uint32_t)(w.BPP * 32), (uint32_t)w.KPX, 1u};
+      const uint32_t box[4] = {128u, (uint32_t)(p.BPP * 32), (uint32_t)p.KPX, 1u};
       if (!encode_tensor_map_u8(&map_a, qg->codes, 4, dims, strides, box, nullptr, 128)) return MQ_ERR_CUDA;
     }
     {
       const uint64_t rb = (uint64_t)g.Cp;
       const uint64_t dims[4] = {rb, (uint64_t)g.N, (uint64_t)g.W, (uint64_t)g.H};
       const uint64_t strides[3] = {rb, (uint64_t)g.N * rb, (uint64_t)g.W * g.N * rb};
-      const uint32_t box[4] = {128u, (uint32_t)(w.BPP * 32), (uint32_t)((w.KPX - 1) * g.sw + 1), 1u};
+      const uint32_t box[4] = {128u, (uint32_t)(p.BPP * 32), (uint32_t)((p.KPX - 1) * g.sw + 1), 1u};
       const uint32_t es[4] = {1u, 1u, (uint32_t)g.sw, 1u};
       if (!encode_tensor_map_u8(&map_b, qx->codes, 4, dims, strides, box, es, 128)) return MQ_ERR_CUDA;
     }
   }
+  if (launch_expand_wgrad_scales(p, stream) != cudaSuccess) return MQ_ERR_CUDA;
   if (launch_wgrad_tc(p, map_a, map_b, stream) != cudaSuccess) return MQ_ERR_CUDA;
-  return launch_bwd_weight_reduce(partial, out, g, w.splits, layout, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
+  return launch_bwd_weight_reduce(partial, out, g, p.splits, layout, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }
 
 unsigned int* device_status_ptr() {
@@ -339,7 +358,7 @@ mq_status run_conv(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int r
   if (op == MQ_OP_BWD_DATA && conv_tc_eligible(op, g, qb->fmt, qa->fmt))
     return run_conv_tc(op, g, qb, qa, static_cast<float*>(out), layout, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
   if (op == MQ_OP_BWD_WEIGHT) {
-    const WgradPlan w = wgrad_plan(g, qa->fmt, qb->fmt);
+    WgradPlan w = wgrad_plan(g, qa->fmt, qb->fmt);
     if (w.ok) return run_wgrad_tc(g, w, qa, qb, static_cast<float*>(out), layout, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
   }
   ConvArgs a;
@@ -387,7 +406,7 @@ mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt
   if (op == MQ_OP_BWD_DATA && conv_tc_eligible(op, g, fmt_b, fmt_a)) *bytes = conv_tc_workspace(op, g, fmt_b, fmt_a);
   if (op == MQ_OP_BWD_WEIGHT) {
     const WgradPlan w = wgrad_plan(g, fmt_a, fmt_b);
-    if (w.ok) *bytes = w.total_bytes;
+    if (w.ok) *bytes = w.total;
   }
   return MQ_OK;
 }

@@ -60,8 +60,11 @@ cudaError_t launch_weight_transpose(const uint8_t* w_codes, const uint8_t* w_sca
                                     cudaStream_t s);
 
 // Parameters of the tensor-core weight-gradient kernel (see mq_wgrad_tc.cu).
+enum { MQ_WG_FP8 = 0, MQ_WG_FP4_PIXEL = 1, MQ_WG_FP4_FLAT = 2 };
 struct WgradTcParams {
-  int fp4;              // 1: E2M1 operands re-laid n-fastest (K-major, kind::mxf4); 0: 8-bit operands as stored (MN-major)
+  int mode;             // MQ_WG_FP8: 8-bit operands as stored (MN-major TMA boxes); MQ_WG_FP4_PIXEL: E2M1 re-laid
+                        // [pixel][c][n], one TMA box per pixel; MQ_WG_FP4_FLAT: stride 1, E2M1 re-laid as contiguous
+                        // pre-swizzled pieces over the zero-padded, flattened pixel axis (bulk copies)
   uint32_t idesc;
   int stages;
   int N, Nt, Ho, Wo, H, W, Cout, Cp, Ct, Cot, Kh, Kw, sh, sw, ph, pw;
@@ -70,16 +73,29 @@ struct WgradTcParams {
   int KBn;              // E2M1: bytes of n per pixel per stage (= 16 * BPP)
   int nchunks;          // stages per pixel group
   int groups_w;         // ceil(Wo / KPX)
-  int stages_total;     // Ho * groups_w * nchunks
+  int stages_total;     // pixel: Ho * groups_w * nchunks; flat: ceil(Ho * Wp / KPX)
+  int Wp;               // flat: padded width W + 2 * pw
+  int b_rows;           // rows (input channels) of a B tile: 128, or min(128, Cp) in flat mode
   int m_tiles, j_tiles, cb_tiles, splits;
   const uint8_t* g_scales;  // [Ho][Wo][Nt][Cot]
   const uint8_t* x_scales;  // [H][W][Nt][Ct]
+  const uint8_t* gt;        // flat: [co block][padded pixel][128][KBn]
+  const uint8_t* xt;        // flat: [ci block][padded pixel][b_rows][KBn]
+  long long gt_block_bytes, xt_block_bytes;
+  uint8_t* sfa_img;         // [m tile][stage][512 * SPA]
+  uint8_t* sfb_img;         // [ci block][tap][stage][512 * SPA]
   float* partial;           // [splits][Cout][taps * Cp]
   unsigned int* status;
 };
 cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s);
+cudaError_t launch_expand_wgrad_scales(const WgradTcParams& p, cudaStream_t s);
 // E2M1 codes [P][N][Cp] -> [P][Cp][Npad] (n fastest, zero-padded): a permutation of nibbles, no requantization.
 cudaError_t launch_fp4_to_n_major(const uint8_t* in, uint8_t* out, int P, int N, int Cp, int Npad, cudaStream_t s);
+// E2M1 codes [Hs][Ws][N][Cs_p] -> [channel block][q][rows][KBn] over q = hq * Wp + wq in [0, P_out), source pixel
+// (hq - off_h, wq - off_w), zero outside the image / beyond the channels, each [rows][KBn] piece stored with the
+// shared-memory swizzle of span KBn already applied.
+cudaError_t launch_fp4_to_flat(const uint8_t* in, uint8_t* out, int Hs, int Ws, int N, int Cs_p, int P_out, int Wp, int off_h, int off_w,
+                               int rows, int nblocks, int KBn, cudaStream_t s);
 // Adds the split partial sums in a fixed order and writes G_W in its final layout.
 cudaError_t launch_bwd_weight_reduce(const float* partial, float* out, const Geom& g, int splits, int layout, cudaStream_t s);
 

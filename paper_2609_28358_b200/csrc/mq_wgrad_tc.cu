@@ -4,16 +4,20 @@
 //
 //   D[co][(tap, ci)] = sum over (ho, wo, n) of G[ho, wo, n, co] * X[ho*s + kh - p, wo*s + kw - p, n, ci]
 //
-// 8-bit formats: both operands are read exactly as stored ([pixel][n][c], c fastest) and handed to the
-// MMA as MN-major tiles (K = n runs across rows of 128 channel bytes); no re-layout, no requantization.
-// E2M1: tcgen05 accepts 4-bit operands only K-major, so mq_conv_bwd_weight first transposes the codes of X
-// and G_Y inside every pixel in scratch ([pixel][c][n], a pure permutation of nibbles, scales untouched);
-// this kernel then loads, per pixel, a [128 channels][n bytes] K-major box whose row length equals its
-// swizzle span (16 bytes: unswizzled core matrices, two boxes side by side per MMA).
+// 8-bit formats (MQ_WG_FP8): both operands are read exactly as stored ([pixel][n][c], c fastest) and handed
+// to the MMA as MN-major tiles (K = n runs across rows of 128 channel bytes); no re-layout.
+// E2M1: tcgen05 accepts 4-bit operands only K-major, so mq_conv_bwd_weight first permutes the nibbles of X
+// and G_Y in scratch (scales untouched, nothing requantized):
+//   MQ_WG_FP4_PIXEL  [pixel][c][n]; per pixel a [128 channels][n bytes] TMA box whose row length equals its
+//                    swizzle span (16 bytes: unswizzled core matrices, two boxes side by side per MMA);
+//   MQ_WG_FP4_FLAT   (stride 1) channel-blocked pieces over the zero-padded, flattened pixel axis q = h*Wp + w:
+//                    the input pixel of output pixel q at tap (kh, kw) is q + kh*Wp + kw, so a stage of
+//                    consecutive pixels is ONE contiguous, already swizzled run for each operand (bulk copy).
 //
-// One thread block per work item (128 output channels x 128 (tap, ci) columns x a slice of the
-// pixel range); partial sums go to scratch and are added in a fixed order by bwd_weight_reduce.
-// Warps: 0 TMA producer, 1 MMA issuer, 2-3 scale expanders (alternating stages), 4-7 epilogue.
+// A small kernel first expands the compact tile scales into the per-stage scale-vector chunks in scratch.
+// One thread block per work item (128 output channels x one tap's block of input channels x a slice of
+// the K range); partial sums go to scratch and are added in a fixed order by bwd_weight_reduce.
+// Warps: 0 producer (TMA / bulk copies), 1 MMA issuer, 2 scale copier (smem -> TMEM), 4-7 epilogue.
 #include "mq_conv_tc.cuh"
 #include "mq_tcgen05.cuh"
 
@@ -23,29 +27,83 @@ using namespace tc;
 
 constexpr int WG_THREADS = 256;
 constexpr int WG_STAGE_BYTES = 2 * 128 * 128 + 4 * 512;  // A 16 KB + B 16 KB + scale chunks (2 groups each)
+constexpr int WG_SF_COLS = 16;                           // TMEM columns of one stage's scale vectors (A 8 + B 8)
 
-// stage index -> (ho, wo group, n chunk), walked incrementally
-struct KPos {
-  int ho, wg, nc;
-  __device__ __forceinline__ void set(const WgradTcParams& p, int st) {
-    nc = st % p.nchunks; st /= p.nchunks;
-    wg = st % p.groups_w; ho = st / p.groups_w;
+// K-block b of stage st: output pixel and 32-sample block
+__device__ __forceinline__ void stage_block(const WgradTcParams& p, int st, int b, int& ho, int& wo, int& nb) {
+  const int px = b / p.BPP, sub = b - px * p.BPP;
+  if (p.mode == MQ_WG_FP4_FLAT) {
+    const int a = st * p.KPX + px;
+    ho = a / p.Wp; wo = a - ho * p.Wp; nb = sub;
+  } else {
+    const int nc = st % p.nchunks; const int t = st / p.nchunks;
+    const int wg = t % p.groups_w; ho = t / p.groups_w;
+    wo = wg * p.KPX + px; nb = nc * p.BPP + sub;
   }
-  __device__ __forceinline__ void next(const WgradTcParams& p) {
-    if (++nc == p.nchunks) { nc = 0; if (++wg == p.groups_w) { wg = 0; ++ho; } }
+}
+
+// ---- scale expansion: one warp per 512*SPA-byte chunk ----------------------------------------------------
+template <bool FP4>
+__global__ void __launch_bounds__(256) expand_wgrad_scales_kernel(const WgradTcParams p) {
+  constexpr int SPA = FP4 ? 2 : 1, NBS = 4 * SPA;
+  const int lane = threadIdx.x & 31;
+  const long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int taps = p.Kh * p.Kw;
+  const long long nA = (long long)p.m_tiles * p.stages_total;
+  const long long nB = (long long)p.cb_tiles * taps * p.stages_total;
+  if (wid >= nA + nB) return;
+  // this lane's byte: channel block j of the tile (row group), K-block b of the stage
+  const int j = lane >> 3, b = lane & 7;
+  uint32_t v = 0;
+  uint8_t* dst;
+  if (wid < nA) {
+    const int mt = (int)(wid / p.stages_total), st = (int)(wid - (long long)mt * p.stages_total);
+    const int cob = mt * 4 + j;
+    if (b < NBS && cob < p.Cot) {
+      int ho, wo, nb;
+      stage_block(p, st, b, ho, wo, nb);
+      if (ho < p.Ho && wo < p.Wo && nb < p.Nt) v = __ldg(p.g_scales + (((long long)ho * p.Wo + wo) * p.Nt + nb) * p.Cot + cob);
+    }
+    dst = p.sfa_img + wid * (512 * SPA);
+  } else {
+    long long idx = wid - nA;
+    const int st = (int)(idx % p.stages_total); idx /= p.stages_total;
+    const int tap = (int)(idx % taps); const int cb = (int)(idx / taps);
+    const int kh = tap / p.Kw, kw = tap - kh * p.Kw;
+    const int cib = (cb * p.b_rows) / 32 + j;
+    if (b < NBS && 32 * j < p.b_rows && cib < p.Ct) {
+      int ho, wo, nb;
+      stage_block(p, st, b, ho, wo, nb);
+      const int h = ho * p.sh + kh - p.ph, w = wo * p.sw + kw - p.pw;
+      if (ho < p.Ho && wo < p.Wo && nb < p.Nt && h >= 0 && h < p.H && w >= 0 && w < p.W)
+        v = __ldg(p.x_scales + (((long long)h * p.W + w) * p.Nt + nb) * p.Ct + cib);
+    }
+    dst = p.sfb_img + (wid - nA) * (512 * SPA);
   }
-};
+#pragma unroll
+  for (int g = 0; g < SPA; ++g) {
+    uint32_t w4[4];
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      uint32_t word = 0;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) word |= __shfl_sync(0xffffffffu, v, jj * 8 + 4 * g + k) << (8 * k);
+      w4[jj] = word;
+    }
+    *reinterpret_cast<uint4*>(dst + g * 512 + lane * 16) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+  }
+}
 
 template <bool FP4>
 __global__ void __launch_bounds__(WG_THREADS, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const WgradTcParams p) {
   constexpr int SPA = FP4 ? 2 : 1;     // scale bytes per MMA per row
-  constexpr int NBS = 4 * SPA;         // K-blocks (scale bytes) per stage
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * WG_STAGE_BYTES);
   uint64_t* empty = full + p.stages;
-  uint64_t* tfull = empty + p.stages;
+  uint64_t* sffull = empty + p.stages;
+  uint64_t* tfull = sffull + p.stages;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tfull + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -57,18 +115,17 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   const int split = item / p.j_tiles;
   const int tap = jt / p.cb_tiles, cb = jt - tap * p.cb_tiles;
   const int kh = tap / p.Kw, kw = tap - kh * p.Kw;
-  const int co0 = mt * 128, ci0 = cb * 128;
+  const int co0 = mt * 128, ci0 = cb * p.b_rows;
   const int st_begin = (int)((long long)p.stages_total * split / p.splits);
   const int st_end = (int)((long long)p.stages_total * (split + 1) / p.splits);
   const int nst = st_end - st_begin;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 2); mbar_init(&empty[s], 1); }
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); }
     mbar_init(tfull, 1);
     *abort_flag = 0;
     mbar_fence_init();
-    prefetch_tensormap(&map_a);
-    prefetch_tensormap(&map_b);
+    if (p.mode != MQ_WG_FP4_FLAT) { prefetch_tensormap(&map_a); prefetch_tensormap(&map_b); }
   }
   if (warp == 1) { tmem_alloc(tmem_slot, 256); tmem_relinquish(); }
   tc_fence_before_sync();
@@ -77,29 +134,47 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   const uint32_t tmem = *tmem_slot;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
+    // ------------------------------------------------------------------ producer
     if (lane == 0) {
-      KPos k;
-      k.set(p, st_begin);
+      const int taps = p.Kh * p.Kw;
+      const uint8_t* sfa_src = p.sfa_img + ((size_t)mt * p.stages_total + st_begin) * (512 * SPA);
+      const uint8_t* sfb_src = p.sfb_img + (((size_t)cb * taps + tap) * p.stages_total + st_begin) * (512 * SPA);
+      const uint32_t a_bytes = 128 * 128, b_bytes = (uint32_t)p.b_rows * 128;
+      const uint8_t* ga = nullptr; const uint8_t* gb = nullptr;
+      if (p.mode == MQ_WG_FP4_FLAT) {
+        ga = p.gt + (size_t)mt * p.gt_block_bytes + (size_t)st_begin * a_bytes;
+        gb = p.xt + (size_t)cb * p.xt_block_bytes + ((size_t)st_begin * p.KPX + (size_t)kh * p.Wp + kw) * ((size_t)p.b_rows * p.KBn);
+      }
       uint32_t s = 0, phase = 0;
       for (int i = 0; i < nst && !*abort_flag; ++i) {
         if (!mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
         uint8_t* sa = smem + (size_t)s * WG_STAGE_BYTES;
         uint8_t* sb = sa + 128 * 128;
-        mbar_arrive_expect_tx(&full[s], 2 * 128 * 128);
-        const int wo0 = k.wg * p.KPX;
-        if (FP4) {
-          // [pixel][c][n] re-laid codes: one box (n bytes, 128 channels) per pixel of the stage
-          for (int px = 0; px < p.KPX; ++px) {
-            tma_load_4d(sa + px * 128 * p.KBn, &map_a, &full[s], k.nc * p.KBn, co0, wo0 + px, k.ho);
-            tma_load_4d(sb + px * 128 * p.KBn, &map_b, &full[s], k.nc * p.KBn, ci0, (wo0 + px) * p.sw + kw - p.pw, k.ho * p.sh + kh - p.ph);
-          }
+        mbar_arrive_expect_tx(&full[s], a_bytes + b_bytes + 2 * 512 * SPA);
+        bulk_load(sb + 128 * 128, sfa_src, 512 * SPA, &full[s]);
+        bulk_load(sb + 128 * 128 + 1024, sfb_src, 512 * SPA, &full[s]);
+        sfa_src += 512 * SPA; sfb_src += 512 * SPA;
+        if (p.mode == MQ_WG_FP4_FLAT) {
+          bulk_load(sa, ga, a_bytes, &full[s]);
+          bulk_load(sb, gb, b_bytes, &full[s]);
+          ga += a_bytes; gb += b_bytes;
         } else {
-          // stored [ho][wo][n][c] codes: box (128 channel bytes, n rows, pixels, 1)
-          tma_load_4d(sa, &map_a, &full[s], co0, k.nc * p.BPP * 32, wo0, k.ho);
-          tma_load_4d(sb, &map_b, &full[s], ci0, k.nc * p.BPP * 32, wo0 * p.sw + kw - p.pw, k.ho * p.sh + kh - p.ph);
+          const int st = st_begin + i;
+          const int nc = st % p.nchunks; const int t = st / p.nchunks;
+          const int wg = t % p.groups_w, ho = t / p.groups_w;
+          const int wo0 = wg * p.KPX;
+          if (p.mode == MQ_WG_FP4_PIXEL) {
+            // [pixel][c][n] re-laid codes: one box (n bytes, 128 channels) per pixel of the stage
+            for (int px = 0; px < p.KPX; ++px) {
+              tma_load_4d(sa + px * 128 * p.KBn, &map_a, &full[s], nc * p.KBn, co0, wo0 + px, ho);
+              tma_load_4d(sb + px * 128 * p.KBn, &map_b, &full[s], nc * p.KBn, ci0, (wo0 + px) * p.sw + kw - p.pw, ho * p.sh + kh - p.ph);
+            }
+          } else {
+            // stored [ho][wo][n][c] codes: box (128 channel bytes, n rows, pixels, 1)
+            tma_load_4d(sa, &map_a, &full[s], co0, nc * p.BPP * 32, wo0, ho);
+            tma_load_4d(sb, &map_b, &full[s], ci0, nc * p.BPP * 32, wo0 * p.sw + kw - p.pw, ho * p.sh + kh - p.ph);
+          }
         }
-        k.next(p);
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
     }
@@ -107,130 +182,67 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       // 8-bit: MN-major tiles [K row][128 bytes], 128-byte swizzle, 8-row groups 1024 bytes apart; an MMA
-      // takes 32 K rows (4096 bytes).  E2M1: per-pixel K-major boxes [128 rows][KBn bytes], swizzle span
-      // = KBn (none for 16: 8x16-byte core matrices, the next 16 bytes of K one box further); an MMA takes
-      // 32 bytes of K.
+      // takes 32 K rows (4096 bytes).  E2M1: K-major pieces [rows][KBn bytes], swizzle span = KBn (none for
+      // 16: 8x16-byte core matrices, the next 16 bytes of K one piece further); an MMA takes 32 bytes of K.
       const uint32_t fp4_layout = p.KBn == 128 ? 2u : (p.KBn == 64 ? 4u : (p.KBn == 32 ? 6u : 0u));
-      const uint64_t op_desc = FP4 ? smem_desc_base(128 * 16, 8 * p.KBn, fp4_layout) : smem_desc_base(128 * 128, 1024, 2);
-      const uint64_t sf_desc = smem_desc_base(0, 128, 0);
+      const uint32_t a_piece = 128 * p.KBn, b_piece = (uint32_t)p.b_rows * p.KBn;
+      const uint64_t a_desc0 = smem_desc(FP4 ? smem_desc_base(a_piece, 8 * p.KBn, fp4_layout) : smem_desc_base(128 * 128, 1024, 2), smem_u32(smem));
+      const uint64_t b_desc0 = smem_desc(FP4 ? smem_desc_base(b_piece, 8 * p.KBn, fp4_layout) : smem_desc_base(128 * 128, 1024, 2), smem_u32(smem + 128 * 128));
       const uint32_t stage16 = WG_STAGE_BYTES >> 4;
-      const uint64_t a_desc0 = smem_desc(op_desc, smem_u32(smem));
-      const uint64_t b_desc0 = smem_desc(op_desc, smem_u32(smem + 128 * 128));
-      const uint64_t sfa_desc0 = smem_desc(sf_desc, smem_u32(smem + 2 * 128 * 128));
-      const uint64_t sfb_desc0 = smem_desc(sf_desc, smem_u32(smem + 2 * 128 * 128 + 1024));
-      uint32_t koff16[4];   // offset of MMA a's K slice inside the stage's operand tile, in 16-byte units
+      uint32_t ka16[4], kb16[4];   // offset of MMA a's K slice inside the stage's A / B tile, in 16-byte units
 #pragma unroll
       for (int a = 0; a < 4; ++a) {
-        if (FP4) { const int piece = (32 * a) / p.KBn, off = (32 * a) % p.KBn; koff16[a] = (uint32_t)(piece * 128 * p.KBn + off) >> 4; }
-        else koff16[a] = 256u * a;
+        if (FP4) {
+          const int piece = (32 * a) / p.KBn, off = (32 * a) % p.KBn;
+          ka16[a] = (piece * a_piece + off) >> 4; kb16[a] = (piece * b_piece + off) >> 4;
+        } else { ka16[a] = 256u * a; kb16[a] = 256u * a; }
       }
       uint32_t idesc_id[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) idesc_id[i] = idesc_with_sf_ids(p.idesc, i, i);
       const uint32_t sf_base = tmem + 128;
-      uint32_t s = 0, phase = 0, sfbuf = 0, accumulate = 0;
+      uint32_t s = 0, phase = 0, accumulate = 0;
+      for (int i = 0; i < nst && !*abort_flag; ++i) {
+        if (!mbar_wait(&sffull[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+        tc_fence_after_sync();
+        const uint32_t so = s * stage16;
+        const uint32_t sfa_t = sf_base + s * WG_SF_COLS, sfb_t = sfa_t + 8;
+#pragma unroll
+        for (int a = 0; a < 4; ++a) {
+          const int g = (a * SPA) >> 2, id = (a * SPA) & 3;
+          if (FP4) mma_mxf4(tmem, a_desc0 + so + ka16[a], b_desc0 + so + kb16[a], idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g, accumulate);
+          else mma_mxf8f6f4(tmem, a_desc0 + so + ka16[a], b_desc0 + so + kb16[a], idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g, accumulate);
+          accumulate = 1;
+        }
+        tc_commit(&empty[s]);
+        if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
+      }
+      if (nst > 0) tc_commit(tfull); else mbar_arrive(tfull);
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------------ scale copier (smem -> per-stage TMEM buffers)
+    if (lane == 0) {
+      const uint64_t sf_desc = smem_desc_base(0, 128, 0);
+      const uint64_t sfa_desc0 = smem_desc(sf_desc, smem_u32(smem + 2 * 128 * 128));
+      const uint64_t sfb_desc0 = smem_desc(sf_desc, smem_u32(smem + 2 * 128 * 128 + 1024));
+      const uint32_t stage16 = WG_STAGE_BYTES >> 4;
+      const uint32_t sf_base = tmem + 128;
+      uint32_t s = 0, phase = 0;
       for (int i = 0; i < nst && !*abort_flag; ++i) {
         if (!mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
         tc_fence_after_sync();
         const uint32_t so = s * stage16;
-        const uint32_t sfa_t = sf_base + sfbuf * 16, sfb_t = sfa_t + 8;
+        const uint32_t sfa_t = sf_base + s * WG_SF_COLS, sfb_t = sfa_t + 8;
 #pragma unroll
         for (int g = 0; g < SPA; ++g) {
           tmem_cp_32x128b_warpx4(sfa_t + 4 * g, sfa_desc0 + so + g * 32);
           tmem_cp_32x128b_warpx4(sfb_t + 4 * g, sfb_desc0 + so + g * 32);
         }
-#pragma unroll
-        for (int a = 0; a < 4; ++a) {
-          const int g = (a * SPA) >> 2, id = (a * SPA) & 3;
-          if (FP4) mma_mxf4(tmem, a_desc0 + so + koff16[a], b_desc0 + so + koff16[a], idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g, accumulate);
-          else mma_mxf8f6f4(tmem, a_desc0 + so + koff16[a], b_desc0 + so + koff16[a], idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g, accumulate);
-          accumulate = 1;
-        }
-        tc_commit(&empty[s]);
-        sfbuf ^= 1;
+        tc_commit(&sffull[s]);
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
-      if (nst > 0) tc_commit(tfull); else mbar_arrive(tfull);
     }
-  } else if (warp == 2 || warp == 3) {
-    // ------------------------------------------------------------------ scale expanders
-    // Lane l < 4*SPA computes the A word (row group j = l / SPA, byte group g = l % SPA); lanes
-    // 8..8+4*SPA the B words.  A word is the 4 scale bytes of 4 consecutive K-blocks (pixel, n block)
-    // for one block of 32 channels.  Loads are issued RING stages ahead and left raw until used.
-    constexpr int RING = 4;
-    const int wid = warp - 2;
-    const bool is_a = lane < 4 * SPA, is_b = lane >= 8 && lane < 8 + 4 * SPA;
-    const int wl = is_b ? lane - 8 : lane;
-    const int j = wl / SPA, g = wl - j * SPA;
-    const int cblk = is_b ? (ci0 >> 5) + j : (co0 >> 5) + j;
-    const bool lane_ok = (is_a && cblk < p.Cot) || (is_b && cblk < p.Ct);
-    const uint8_t* base = is_b ? p.x_scales : p.g_scales;
-    const int cstride = is_b ? p.Ct : p.Cot;
-    auto sf_load = [&](const KPos& k, uint32_t* raw) {
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        raw[i] = 0u;
-        const int b = 4 * g + i;                  // K-block of the stage
-        const int px = b / p.BPP, nb = k.nc * p.BPP + (b - px * p.BPP);
-        const int wo = k.wg * p.KPX + px;
-        if (lane_ok && nb < p.Nt && wo < p.Wo) {
-          int hh = k.ho, ww = wo, Wd = p.Wo;
-          bool ok = true;
-          if (is_b) {
-            hh = k.ho * p.sh + kh - p.ph; ww = wo * p.sw + kw - p.pw; Wd = p.W;
-            ok = hh >= 0 && hh < p.H && ww >= 0 && ww < p.W;
-          }
-          if (ok) raw[i] = __ldg(base + (((long long)hh * Wd + ww) * p.Nt + nb) * cstride + cblk);
-        }
-      }
-    };
-    KPos kpre;
-    kpre.set(p, st_begin);
-    int pre_left = nst;                       // stages not yet loaded (counting both warps' stages)
-    auto pre_advance = [&]() { kpre.next(p); --pre_left; };
-    if (wid == 1 && pre_left > 0) pre_advance();
-    uint32_t ring[RING][4];
-#pragma unroll
-    for (int d = 0; d < RING; ++d) {
-#pragma unroll
-      for (int i = 0; i < 4; ++i) ring[d][i] = 0u;
-      if (pre_left > 0) { sf_load(kpre, ring[d]); pre_advance(); if (pre_left > 0) pre_advance(); }
-    }
-    uint32_t s = 0, phase = 0;
-    auto advance_stage = [&]() { if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; } };
-    int left = nst;
-    if (wid == 1 && left > 0) { advance_stage(); --left; }
-    bool alive = true;
-    while (alive && left > 0) {
-#pragma unroll
-      for (int d = 0; d < RING; ++d) {
-        if (left == 0 || !alive) break;
-        bool ok = true;
-        if (lane == 0) ok = !*abort_flag && mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT);
-        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-        if (!ok) { *abort_flag = 1; alive = false; break; }
-        uint8_t* sfa = smem + (size_t)s * WG_STAGE_BYTES + 2 * 128 * 128;
-        uint8_t* sfb = sfa + 1024;
-        const uint32_t word = ring[d][0] | (ring[d][1] << 8) | (ring[d][2] << 16) | (ring[d][3] << 24);
-#pragma unroll
-        for (int gg = 0; gg < SPA; ++gg) {
-          uint32_t w4[4];
-#pragma unroll
-          for (int jj = 0; jj < 4; ++jj) w4[jj] = __shfl_sync(0xffffffffu, word, jj * SPA + gg);
-          *reinterpret_cast<uint4*>(sfa + gg * 512 + lane * 16) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
-#pragma unroll
-          for (int jj = 0; jj < 4; ++jj) w4[jj] = __shfl_sync(0xffffffffu, word, 8 + jj * SPA + gg);
-          *reinterpret_cast<uint4*>(sfb + gg * 512 + lane * 16) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
-        }
-        fence_proxy_async_smem();
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&full[s]);
-        advance_stage(); --left;
-        if (left > 0) { advance_stage(); --left; }
-        if (pre_left > 0) { sf_load(kpre, ring[d]); pre_advance(); if (pre_left > 0) pre_advance(); }
-      }
-    }
-  } else {
+  } else if (warp >= 4) {
     // ------------------------------------------------------------------ epilogue: partial sums to scratch
     const int quad = warp & 3;
     const int r = 32 * quad + lane;
@@ -242,7 +254,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const int co = co0 + r;
       const long long J = (long long)p.Kh * p.Kw * p.Cp;
       float* out = p.partial + ((long long)split * p.Cout + co) * J + (long long)tap * p.Cp + ci0;
-      const int ncols = min(128, p.Cp - ci0);
+      const int ncols = min(p.b_rows, p.Cp - ci0);
       const uint32_t taddr = tmem + ((uint32_t)(32 * quad) << 16);
       for (int c = 0; c < ncols; c += 16) {
         uint32_t v[16];
@@ -272,7 +284,6 @@ __global__ void __launch_bounds__(256) fp4_to_n_major_kernel(const uint8_t* __re
   __shared__ uint8_t t[8][32][65];  // [pixel][n][c] one code per byte
   const int p0 = blockIdx.x * 8, n0 = blockIdx.y * 32, c0 = blockIdx.z * 64;
   const int tid = threadIdx.x;
-  // load: 8 pixels x 32 rows x 32 bytes = 512 chunks of 16 bytes
   for (int i = tid; i < 512; i += 256) {
     const int px = i >> 6, n = (i >> 1) & 31, half = i & 1;
     uint4 v = make_uint4(0, 0, 0, 0);
@@ -285,7 +296,6 @@ __global__ void __launch_bounds__(256) fp4_to_n_major_kernel(const uint8_t* __re
       for (int b = 0; b < 8; ++b) t[px][n][32 * half + 8 * q + b] = (uint8_t)((w[q] >> (4 * b)) & 0xF);
   }
   __syncthreads();
-  // store: 64 channels x 8 pixels x 16 bytes (32 samples)
   for (int i = tid; i < 512; i += 256) {
     const int px = i >> 6, c = i & 63;
     if (c0 + c < Cp && p0 + px < P) {
@@ -302,14 +312,58 @@ __global__ void __launch_bounds__(256) fp4_to_n_major_kernel(const uint8_t* __re
   }
 }
 
+// ---- E2M1 re-layout for the flat mode (see launch_fp4_to_flat) -------------------------------------------------
+// One block: 8 output pixels x 32 samples x 64 channels.
+__global__ void __launch_bounds__(256) fp4_to_flat_kernel(const uint8_t* __restrict__ in, uint8_t* __restrict__ out, int Hs, int Ws, int N, int Cs_p,
+                                                           int P_out, int Wp, int off_h, int off_w, int rows, int nblocks, int KBn) {
+  __shared__ uint8_t t[8][32][65];
+  const int q0 = blockIdx.x * 8, n0 = blockIdx.y * 32, c0 = blockIdx.z * 64;
+  const int tid = threadIdx.x;
+  for (int i = tid; i < 512; i += 256) {
+    const int px = i >> 6, n = (i >> 1) & 31, half = i & 1;
+    const int q = q0 + px;
+    const int hq = q / Wp, wq = q - hq * Wp;
+    const int h = hq - off_h, w = wq - off_w;
+    uint4 v = make_uint4(0, 0, 0, 0);
+    if (q < P_out && h >= 0 && h < Hs && w >= 0 && w < Ws && n0 + n < N && c0 + 32 * half < Cs_p)
+      v = *reinterpret_cast<const uint4*>(in + ((((long long)h * Ws + w) * N + n0 + n) * Cs_p + c0 + 32 * half) / 2);
+    const uint32_t wd[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int k = 0; k < 4; ++k)
+#pragma unroll
+      for (int b = 0; b < 8; ++b) t[px][n][32 * half + 8 * k + b] = (uint8_t)((wd[k] >> (4 * b)) & 0xF);
+  }
+  __syncthreads();
+  const int cmax = nblocks * rows;
+  for (int i = tid; i < 512; i += 256) {
+    const int px = i >> 6, c = i & 63;
+    const int q = q0 + px, cc = c0 + c;
+    if (cc < cmax && q < P_out) {
+      uint32_t wd[4];
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        uint32_t acc = 0;
+#pragma unroll
+        for (int b = 0; b < 8; ++b) acc |= (uint32_t)t[px][8 * k + b][c] << (4 * b);
+        wd[k] = acc;
+      }
+      const int blk = cc / rows, r = cc - blk * rows;
+      const int chunk = n0 >> 5;   // 16-byte chunk of the row
+      const int sw = KBn == 128 ? (r & 7) : (KBn == 64 ? ((r >> 1) & 3) : (KBn == 32 ? ((r >> 2) & 1) : 0));
+      const long long off = (((long long)blk * P_out + q) * rows + r) * KBn + ((chunk ^ sw) << 4);
+      *reinterpret_cast<uint4*>(out + off) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+    }
+  }
+}
+
 }  // namespace
 
-size_t wgrad_tc_smem_bytes(const WgradTcParams& p) { return 1024 + (size_t)p.stages * WG_STAGE_BYTES + (2 * (size_t)p.stages + 2) * 8 + 64; }
+size_t wgrad_tc_smem_bytes(const WgradTcParams& p) { return 1024 + (size_t)p.stages * WG_STAGE_BYTES + (3 * (size_t)p.stages + 2) * 8 + 64; }
 
 cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s) {
   static bool attr_set[2] = {false, false};
   const size_t smem = wgrad_tc_smem_bytes(p);
-  const int f = p.fp4 ? 1 : 0;
+  const int f = p.mode == MQ_WG_FP8 ? 0 : 1;
   if (!attr_set[f]) {
     cudaError_t e = f ? cudaFuncSetAttribute(wgrad_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)
                       : cudaFuncSetAttribute(wgrad_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
@@ -323,9 +377,26 @@ cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, co
   return cudaGetLastError();
 }
 
+cudaError_t launch_expand_wgrad_scales(const WgradTcParams& p, cudaStream_t s) {
+  const long long warps = (long long)p.m_tiles * p.stages_total + (long long)p.cb_tiles * p.Kh * p.Kw * p.stages_total;
+  const unsigned blocks = (unsigned)((warps + 7) / 8);
+  if (p.mode == MQ_WG_FP8) expand_wgrad_scales_kernel<false><<<blocks, 256, 0, s>>>(p);
+  else expand_wgrad_scales_kernel<true><<<blocks, 256, 0, s>>>(p);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_fp4_to_n_major(const uint8_t* in, uint8_t* out, int P, int N, int Cp, int Npad, cudaStream_t s) {
   dim3 grid((P + 7) / 8, Npad / 32, (Cp + 63) / 64);
   fp4_to_n_major_kernel<<<grid, 256, 0, s>>>(in, out, P, N, Cp, Npad);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_fp4_to_flat(const uint8_t* in, uint8_t* out, int Hs, int Ws, int N, int Cs_p, int P_out, int Wp, int off_h, int off_w,
+                               int rows, int nblocks, int KBn, cudaStream_t s) {
+  dim3 grid((P_out + 7) / 8, KBn / 16, (nblocks * rows + 63) / 64);
+  fp4_to_flat_kernel<<<grid, 256, 0, s>>>(in, out, Hs, Ws, N, Cs_p, P_out, Wp, off_h, off_w, rows, nblocks, KBn);
   count_launches(1);
   return cudaGetLastError();
 }
