@@ -194,7 +194,7 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
   p.a_scales = qx_like->scales;
   p.sfa_img = base + pl.off_sfa;
   p.sfb_img = base + pl.off_sfb;
-  p.out = out; p.out_layout = layout; p.status = status;
+  p.out = out; p.out_layout = env_int("MQ_TC_SKIP_STORE", 0) ? 99 : layout; p.status = status;
   if (launch_expand_conv_scales(p, stream) != cudaSuccess) return MQ_ERR_CUDA;
 
   CUtensorMap map_a, map_b;

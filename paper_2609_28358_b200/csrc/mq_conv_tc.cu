@@ -45,14 +45,31 @@ __device__ unsigned long long g_prof[8][2];
 
 struct Tile { int c0, w0, n0, h, cls; };
 
+// Tile order: stride class fastest (the classes of an input gradient interleave inside the same 32-byte
+// sectors), then output column tile, output row, channel tile, sample tile.  Tiles that run at the same time
+// then complete whole (n, c) planes of an NCHW output quickly, so partially written lines do not linger in
+// L2, and they share input rows between neighbouring taps.
 __device__ __forceinline__ Tile decode_tile(const ConvTcParams& p, unsigned t) {
   Tile q;
-  unsigned u = t / (unsigned)p.tiles_c;
-  q.c0 = (int)(t - u * p.tiles_c) * p.BN; t = u;
+  unsigned u = t / (unsigned)p.classes;
+  q.cls = (int)(t - u * p.classes); t = u;
   u = t / (unsigned)p.tiles_w; q.w0 = (int)(t - u * p.tiles_w) * p.TW; t = u;
-  u = t / (unsigned)p.tiles_n; q.n0 = (int)(t - u * p.tiles_n) * p.TN; t = u;
-  u = t / (unsigned)p.tiles_h; q.h = (int)(t - u * p.tiles_h);
-  q.cls = (int)u;
+  u = t / (unsigned)p.tiles_h; q.h = (int)(t - u * p.tiles_h); t = u;
+  u = t / (unsigned)p.tiles_c; q.c0 = (int)(t - u * p.tiles_c) * p.BN;
+  q.n0 = (int)u * p.TN;
+  return q;
+}
+// index of a tile among the tiles that differ in anything but the channel tile (A-side scale chunks)
+__device__ __forceinline__ unsigned tile_m_index(const ConvTcParams& p, const Tile& q) {
+  return (((unsigned)(q.n0 / p.TN) * p.tiles_h + q.h) * p.tiles_w + q.w0 / p.TW) * p.classes + q.cls;
+}
+__device__ __forceinline__ Tile tile_of_m_index(const ConvTcParams& p, unsigned tm) {
+  Tile q;
+  unsigned u = tm / (unsigned)p.classes;
+  q.cls = (int)(tm - u * p.classes); tm = u;
+  u = tm / (unsigned)p.tiles_w; q.w0 = (int)(tm - u * p.tiles_w) * p.TW; tm = u;
+  u = tm / (unsigned)p.tiles_h; q.h = (int)(tm - u * p.tiles_h);
+  q.n0 = (int)u * p.TN; q.c0 = 0;
   return q;
 }
 
@@ -149,9 +166,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int Q = tw.chunks(p);
         ChunkPos pos;
         pos.reset();
-        const unsigned tm = t / (unsigned)p.tiles_c;    // tile index without the channel tile
-        const uint8_t* sfa_src = p.sfa_img + (size_t)tm * p.max_stages * (512 * SPA);
-        const uint8_t* sfb_src = p.sfb_img + ((size_t)tile.cls * p.tiles_c + (t - tm * p.tiles_c)) * p.max_stages * (512 * SPA * atoms_b);
+        const uint8_t* sfa_src = p.sfa_img + (size_t)tile_m_index(p, tile) * p.max_stages * (512 * SPA);
+        const uint8_t* sfb_src = p.sfb_img + ((size_t)tile.cls * p.tiles_c + tile.c0 / p.BN) * p.max_stages * (512 * SPA * atoms_b);
         for (int q0 = 0; q0 < Q; q0 += G) {
           if (!PROF_WAIT(mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
           const int nch = min(G, Q - q0);
@@ -298,7 +314,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 #pragma unroll
           for (int j = 0; j < 16; ++j) v[j] = 0u;
         }
-        if (row_ok) {
+        if (row_ok && p.out_layout != 99) {
           if (p.out_layout == MQ_NCHW) {
             if (full_cols) {
 #pragma unroll
@@ -357,7 +373,7 @@ __global__ void __launch_bounds__(256) expand_conv_scales_kernel(const ConvTcPar
   if (wid < nA) {
     const unsigned tm = wid / (unsigned)p.max_stages;
     const int st = (int)(wid - tm * p.max_stages);
-    const Tile tile = decode_tile(p, tm * (unsigned)p.tiles_c);
+    const Tile tile = tile_of_m_index(p, tm);
     TapWalk<MODE> tw;
     tw.init(p, tile);
     const int Q = tw.chunks(p);
