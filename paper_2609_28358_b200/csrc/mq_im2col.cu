@@ -1,22 +1,75 @@
 // Channel-batch-first im2col of the already-quantized activation (Sec. IV-A): a pure gather of MX
-// element bytes and of the tile scales that belong to them.  One thread moves one 16-byte chunk of
-// the output, so consecutive threads write consecutive bytes of X' (the write stream is Kh*Kw/s^2
-// times the read stream and sets the cost); the reads revisit each stored pixel Kh*Kw times and are
-// served by L2.  Out-of-image taps are written as zero bytes.
+// element bytes and of the tile scales that belong to them.  A thread block produces the X' rows of one
+// output pixel for 32 consecutive samples -- a contiguous run of 32 * Kh*Kw * row bytes -- so consecutive
+// threads write consecutive 16-byte chunks (the write stream is Kh*Kw/s^2 times the read stream and sets
+// the cost); the reads revisit each stored pixel Kh*Kw times and are served by L2.  Out-of-image taps are
+// written as zero bytes.  Index arithmetic is done once per block (a table of source offsets per chunk of
+// a row) and advanced incrementally, never per chunk.
 #include "mq_internal.cuh"
 
 namespace mq {
 namespace {
 
 constexpr int IC_THREADS = 256;
+constexpr int IC_MAX_J = 1024;   // chunks of 16 bytes per X' row held in the offset table
 
-__global__ void __launch_bounds__(IC_THREADS) im2col_kernel(Im2colArgs a, int row_chunks, long long code_chunks, long long n_scales) {
+__global__ void __launch_bounds__(IC_THREADS) im2col_kernel(Im2colArgs a, int rc, int J, unsigned n_main) {
+  const Geom& g = a.g;
+  __shared__ int soff[IC_MAX_J];   // source chunk offset of row chunk j relative to sample 0 of the source pixel, -1: zero
+  const int taps = g.Kh * g.Kw;
+  if (blockIdx.x < n_main) {
+    const unsigned pix = blockIdx.x / (unsigned)g.Nt;
+    const int nt = (int)(blockIdx.x - pix * (unsigned)g.Nt);
+    const int ho = (int)(pix / (unsigned)g.Wo), wo = (int)(pix - (unsigned)ho * (unsigned)g.Wo);
+    for (int j = threadIdx.x; j < J; j += IC_THREADS) {
+      const int tap = j / rc, ch = j - tap * rc;
+      const int kh = tap / g.Kw, kw = tap - kh * g.Kw;
+      const int h = ho * g.sh + kh - g.ph, w = wo * g.sw + kw - g.pw;
+      soff[j] = (h >= 0 && h < g.H && w >= 0 && w < g.W) ? ((h * g.W + w) * g.N) * rc + ch : -1;   // < 2^31 chunks checked on the host
+    }
+    __syncthreads();
+    const int n0 = nt * 32;
+    const int rows = min(32, g.N - n0);
+    const int total = rows * J;
+    const uint4* src = reinterpret_cast<const uint4*>(a.codes) + (long long)n0 * rc;
+    uint4* dst = reinterpret_cast<uint4*>(a.out_codes) + ((long long)pix * g.N + n0) * J;
+    // chunk i = n * J + j, advanced by IC_THREADS per step without divisions
+    int n = threadIdx.x / J, j = threadIdx.x - n * J;
+    const int dn = IC_THREADS / J, dj = IC_THREADS - dn * J;
+    for (int i = threadIdx.x; i < total; i += IC_THREADS) {
+      const int so = soff[j];
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (so >= 0) v = __ldg(src + so + n * rc);
+      __stcs(dst + i, v);
+      n += dn; j += dj;
+      if (j >= J) { j -= J; ++n; }
+    }
+  } else {
+    // scales [ho][wo][nt][kh][kw][ct]
+    const long long n_scales = (long long)g.Ho * g.Wo * g.Nt * taps * g.Ct;
+    for (long long id = (long long)(blockIdx.x - n_main) * IC_THREADS + threadIdx.x; id < n_scales; id += (long long)(gridDim.x - n_main) * IC_THREADS) {
+      long long q = id;
+      const int ct = (int)(q % g.Ct); q /= g.Ct;
+      const int tap = (int)(q % taps); q /= taps;
+      const int nt = (int)(q % g.Nt); q /= g.Nt;
+      const int wo = (int)(q % g.Wo);
+      const int ho = (int)(q / g.Wo);
+      const int kh = tap / g.Kw, kw = tap - kh * g.Kw;
+      const int h = ho * g.sh + kh - g.ph, w = wo * g.sw + kw - g.pw;
+      uint8_t sc = 0;
+      if (h >= 0 && h < g.H && w >= 0 && w < g.W) sc = a.scales[(((long long)h * g.W + w) * g.Nt + nt) * g.Ct + ct];
+      a.out_scales[id] = sc;
+    }
+  }
+}
+
+// General fallback (rows longer than the offset table, or tensors beyond 2^31 chunks): one thread per chunk.
+__global__ void __launch_bounds__(IC_THREADS) im2col_generic_kernel(Im2colArgs a, int row_chunks, long long code_chunks, long long n_scales) {
   const Geom& g = a.g;
   const long long stride = (long long)gridDim.x * IC_THREADS;
   const int taps = g.Kh * g.Kw;
   for (long long id = (long long)blockIdx.x * IC_THREADS + threadIdx.x; id < code_chunks + n_scales; id += stride) {
     if (id < code_chunks) {
-      // output order [ho][wo][n][kh][kw][chunk]
       long long q = id;
       const int ch = (int)(q % row_chunks); q /= row_chunks;
       const int tap = (int)(q % taps); q /= taps;
@@ -26,13 +79,9 @@ __global__ void __launch_bounds__(IC_THREADS) im2col_kernel(Im2colArgs a, int ro
       const int kh = tap / g.Kw, kw = tap - kh * g.Kw;
       const int h = ho * g.sh + kh - g.ph, w = wo * g.sw + kw - g.pw;
       uint4 v = make_uint4(0, 0, 0, 0);
-      if (h >= 0 && h < g.H && w >= 0 && w < g.W) {
-        const long long src = (((long long)h * g.W + w) * g.N + n) * row_chunks + ch;
-        v = __ldg(reinterpret_cast<const uint4*>(a.codes) + src);
-      }
+      if (h >= 0 && h < g.H && w >= 0 && w < g.W) v = __ldg(reinterpret_cast<const uint4*>(a.codes) + (((long long)h * g.W + w) * g.N + n) * row_chunks + ch);
       __stcs(reinterpret_cast<uint4*>(a.out_codes) + id, v);
     } else {
-      // scales [ho][wo][nt][kh][kw][ct]
       long long q = id - code_chunks;
       const int ct = (int)(q % g.Ct); q /= g.Ct;
       const int tap = (int)(q % taps); q /= taps;
@@ -52,16 +101,27 @@ __global__ void __launch_bounds__(IC_THREADS) im2col_kernel(Im2colArgs a, int ro
 
 cudaError_t launch_im2col(const Im2colArgs& a, cudaStream_t s) {
   const Geom& g = a.g;
-  const int row_chunks = g.Cp * fmt_bits(a.fmt) / 8 / 16;  // 16-byte chunks per (pixel, sample) row
-  const long long code_chunks = (long long)g.Ho * g.Wo * g.N * g.Kh * g.Kw * row_chunks;
-  const long long n_scales = (long long)g.Ho * g.Wo * g.Nt * g.Kh * g.Kw * g.Ct;
+  const int rc = g.Cp * fmt_bits(a.fmt) / 8 / 16;  // 16-byte chunks per (pixel, sample) row
+  const int taps = g.Kh * g.Kw;
+  const long long J = (long long)taps * rc;
+  const long long src_chunks = (long long)g.H * g.W * g.N * rc;
+  const long long n_main = (long long)g.Ho * g.Wo * g.Nt;
+  const long long n_scales = (long long)g.Ho * g.Wo * g.Nt * taps * g.Ct;
+  count_launches(1);
+  if (J <= IC_MAX_J && src_chunks < 0x7fffffffLL && n_main < 0x7fff0000LL) {
+    long long sc_blocks = (n_scales + IC_THREADS - 1) / IC_THREADS;
+    if (sc_blocks > 148 * 4) sc_blocks = 148 * 4;
+    if (sc_blocks < 1) sc_blocks = 1;
+    im2col_kernel<<<(unsigned)(n_main + sc_blocks), IC_THREADS, 0, s>>>(a, rc, (int)J, (unsigned)n_main);
+    return cudaGetLastError();
+  }
+  const long long code_chunks = (long long)g.Ho * g.Wo * g.N * J;
   const long long total = code_chunks + n_scales;
   long long blocks = (total + IC_THREADS - 1) / IC_THREADS;
   const long long cap = 148LL * 8 * 16;  // grid-stride beyond this
   if (blocks > cap) blocks = cap;
   if (blocks <= 0) return cudaErrorInvalidValue;
-  im2col_kernel<<<(unsigned)blocks, IC_THREADS, 0, s>>>(a, row_chunks, code_chunks, n_scales);
-  count_launches(1);
+  im2col_generic_kernel<<<(unsigned)blocks, IC_THREADS, 0, s>>>(a, rc, code_chunks, n_scales);
   return cudaGetLastError();
 }
 

@@ -2,12 +2,17 @@
 // also re-lays the tensor into its channel-batch-first stored order (Sec. IV-A).
 //
 // The logical source (NCHW / OIHW fp32) is seen as R x C matrices at P positions with the position
-// axis fastest in memory: element (p, r, c) lives at (r*C + c)*P + p.  One thread block owns one
+// axis fastest in memory: element (p, r, c) lives at (r*C + c)*P + p.  A work item is one
 // 32(r) x 32(c) tile at PS = 8 consecutive positions: 1024 source rows x 32 bytes, every 32-byte
-// sector read exactly once with 128-bit loads.  Per position it reduces |x| over the tile
-// (per-thread max, warp shuffles, one shared-memory exchange), derives the E8M0 code from the
-// exponent field of the maximum, converts with the hardware RNE+saturate conversions and stages
-// the codes in shared memory so the [n][c] slab of each position leaves as 16-byte stores.
+// sector read exactly once.
+//
+// Main kernel (P % 4 == 0): persistent thread blocks loop over work items; the next item's 32 KB stream
+// into shared memory with cp.async (16-byte copies, zero fill for out-of-range rows) while the current
+// item is reduced and converted, so the block always has bytes in flight.  Per position: amax over the
+// tile (per-thread max, one redux.sync per position, one shared-memory exchange), E8M0 code from the exponent field,
+// hardware RNE+saturate conversion; a thread owns 4 adjacent channels so codes leave as 32-bit (FP8) or
+// 16-bit (FP4) shared-memory stores, and each [n][c] slab is written with 16-byte global stores.
+// Fallback kernel (any P, e.g. the 3x3 = 9 positions of a weight tensor): scalar loads, same arithmetic.
 #include <cstdlib>
 
 #include "mq_internal.cuh"
@@ -15,8 +20,11 @@
 namespace mq {
 namespace {
 
-constexpr int PS = 8;           // positions per block
+constexpr int PS = 8;           // positions per work item
 constexpr int QT_THREADS = 256;
+// input buffer: 1024 rows of 32 bytes, plus 16 bytes of padding after every 4 rows so that the 8 lanes of
+// a quarter-warp (rows 4 apart) hit 8 different 16-byte bank groups
+constexpr int QBUF_BYTES = 1024 * 32 + 256 * 16;
 
 template <int FMT>
 __device__ __forceinline__ unsigned encode2(float lo, float hi) {
@@ -28,57 +36,188 @@ __device__ __forceinline__ unsigned encode2(float lo, float hi) {
   }
 }
 
-// 128-bit read-only load that asks L2 to bring in the whole 128-byte line (the other sectors of the
-// line are read next, by this block's following sub-strips)
-__device__ __forceinline__ float4 ldg128_l2_128(const float* p) {
-  float4 v;
-  asm volatile("ld.global.nc.L2::128B.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "l"(p));
-  return v;
+__device__ __forceinline__ int scale_code_of(unsigned amax_bits, int emax) {
+  // floor(log2 amax) = biased exponent - 127 for normal amax; subnormal / zero amax clamps to 0
+  const int e = (int)(amax_bits >> 23) - emax;
+  return min(max(e, 0), 254);
 }
 
-template <int FMT, bool VEC>
-__global__ void __launch_bounds__(QT_THREADS) quantize_kernel(QuantArgs a, int n_pstrips, int Rt, int Ct, int loops, int hint) {
-  __shared__ __align__(16) unsigned red[8][2][4];          // per-warp, per-quad partial maxima
-  __shared__ __align__(16) uint8_t stage[PS][32][32];       // codes, one byte each, [p][r][c]
+// 2^(127 - code) as a normal fp32 number: code = clamp(E - emax, 0, 254) with E <= 254 and emax >= 2, so
+// 127 - code lies in [-125, 127].  x * 2^(127 - code) is then exact (|result| < 2^(emax + 1)) except where it
+// underflows below 2^-126, far under half of the smallest element step, where it rounds to zero either way.
+__device__ __forceinline__ float scale_factor(int code) { return __uint_as_float((unsigned)(254 - code) << 23); }
 
-  const int t = threadIdx.x;
-  const int lane = t & 31, warp = t >> 5;
-  long long bid = blockIdx.x;
-  const int n_groups = (n_pstrips + loops - 1) / loops;
-  const int psg = (int)(bid % n_groups); bid /= n_groups;
-  const int ct = (int)(bid % Ct);
-  const int rt = (int)(bid / Ct);
-  const int r0 = rt * 32, c0 = ct * 32;
-  for (int sub = 0; sub < loops; ++sub) {
-  const int ps = psg * loops + sub;
-  if (ps >= n_pstrips) break;
-  const int p0 = ps * PS;
-  if (sub > 0) __syncthreads();   // previous sub-strip's copy-out has finished reading `stage` / `red`
+__device__ __forceinline__ void cp_async16(void* dst, const void* src, bool valid) {
+  const unsigned d = (unsigned)__cvta_generic_to_shared(dst);
+  const int bytes = valid ? 16 : 0;   // 0 source bytes: the 16 destination bytes are zero-filled
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(d), "l"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+template <int N>
+__device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
-  // thread -> (channel, position quad); 8 rows of the tile: r = 4*i + t/64
-  const int quad = t & 1;
-  const int c = (t >> 1) & 31;
-  const int rsub = t >> 6;
-  const int pq = p0 + 4 * quad;
+struct Item { int p0, r0, c0, rt, ct; };
+__device__ __forceinline__ Item item_of(unsigned it, int n_pstrips, int Ct) {
+  // channel tile fastest: the tiles that share an output line ([n][c] rows are c-contiguous) are produced
+  // together, so full 128-byte lines reach L2 at about the same time; then position strip, then row tile
+  Item q;
+  const unsigned u = it / (unsigned)Ct;
+  q.ct = (int)(it - u * (unsigned)Ct);
+  q.rt = (int)(u / (unsigned)n_pstrips);
+  const int ps = (int)(u - (unsigned)q.rt * (unsigned)n_pstrips);
+  q.p0 = ps * PS; q.r0 = q.rt * 32; q.c0 = q.ct * 32;
+  return q;
+}
 
-  float v[8][4];
-  const bool c_ok = (c0 + c) < a.C;
+template <int FMT, int NT>   // NT threads per block: 256 (two tile rows per thread) or 512 (one)
+__global__ void __launch_bounds__(NT) quantize_pipe_kernel(QuantArgs a, int n_pstrips, int Ct, unsigned n_items) {
+  constexpr int RI = 512 / NT;      // tile rows per thread
+  constexpr int NW = NT / 32;       // warps
+  constexpr int CPT = 2048 / NT;    // 16-byte input chunks per thread
+  extern __shared__ __align__(16) uint8_t qsmem[];
+  uint8_t* buf0 = qsmem;
+  uint8_t* buf1 = qsmem + QBUF_BYTES;
+  uint8_t* stage = qsmem + 2 * QBUF_BYTES;                              // codes [p][r][32 B (FP8) | 16 B (FP4)]
+  unsigned* red = reinterpret_cast<unsigned*>(stage + PS * 32 * 32);     // [warp][quad][4]
+
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  // compute mapping: 4 adjacent channels x 2 rows x 4 positions per thread
+  const int cq = t & 7, quad = (t >> 3) & 1, rs = t >> 4;
+  constexpr int RB = FMT == MQ_E2M1 ? 16 : 32;   // bytes of a staged row
+
+  // copy mapping: chunk (row, position quad) with row = (t >> 1) + (NT/2) m: channel (t >> 1) & 31, tile row
+  // (t >> 6) + (NT/64) m
+  constexpr int RSTEP = NT / 64;    // tile rows between a thread's consecutive chunks
+  const int ld_cc = (t >> 1) & 31, ld_rr = t >> 6, ld_qd = t & 1;
+  const int ld_row = t >> 1;
+  const unsigned ld_dst = (unsigned)(ld_row * 32 + (ld_row >> 2) * 16 + ld_qd * 16);   // + m * RSTEP * (32 * 32 + 8 * 16)
+  const long long row_step = (long long)RSTEP * a.C * a.P;   // floats between a thread's consecutive chunks
+  auto issue = [&](unsigned it, uint8_t* buf) -> Item {
+    const Item q = item_of(it, n_pstrips, Ct);
+    const int pq = q.p0 + 4 * ld_qd;
+    const bool col_ok = (q.c0 + ld_cc) < a.C && pq < a.P;
+    const float* src = a.src + ((long long)(q.r0 + ld_rr) * a.C + (q.c0 + ld_cc)) * a.P + pq;
+    const int rows_left = a.R - q.r0 - ld_rr;     // tile row 4 m is valid while 4 m < rows_left
 #pragma unroll
-  for (int i = 0; i < 8; ++i) {
-    const int r = r0 + 4 * i + rsub;
-    const bool ok = c_ok && r < a.R;
-    const float* row = a.src + ((long long)r * a.C + (c0 + c)) * a.P;
-    if (VEC) {
-      float4 f = make_float4(0.f, 0.f, 0.f, 0.f);
-      if (ok && pq < a.P) f = hint ? ldg128_l2_128(row + pq) : __ldg(reinterpret_cast<const float4*>(row + pq));  // P % 4 == 0: whole quad valid
-      v[i][0] = f.x; v[i][1] = f.y; v[i][2] = f.z; v[i][3] = f.w;
+    for (int m = 0; m < CPT; ++m) {
+      const bool ok = col_ok && RSTEP * m < rows_left;
+      cp_async16(buf + ld_dst + m * RSTEP * (32 * 32 + 8 * 16), ok ? src + m * row_step : a.src, ok);
+    }
+    cp_async_commit();
+    return q;
+  };
+
+  unsigned it = blockIdx.x;
+  const unsigned n_it = (unsigned)n_items;
+  Item q_next{};
+  if (it < n_it) q_next = issue(it, buf0);
+  int cur = 0;
+  const unsigned quad_mask = quad ? 0xFF00FF00u : 0x00FF00FFu;   // the 16 lanes that share this thread's position quad
+  for (; it < n_it; it += gridDim.x, cur ^= 1) {
+    uint8_t* buf = cur ? buf1 : buf0;
+    const unsigned nxt = it + gridDim.x;
+    const Item q = q_next;
+    if (nxt < n_it) { q_next = issue(nxt, cur ? buf0 : buf1); cp_async_wait<1>(); } else { cp_async_wait<0>(); }
+    __syncthreads();   // the current item's bytes are visible to every thread
+
+    float v[RI][4][4];   // [row i][channel k][position j]
+#pragma unroll
+    for (int i = 0; i < RI; ++i)
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int row = (rs + 16 * i) * 32 + 4 * cq + k;
+        const float4 f = *reinterpret_cast<const float4*>(buf + row * 32 + (row >> 2) * 16 + quad * 16);
+        v[i][k][0] = f.x; v[i][k][1] = f.y; v[i][k][2] = f.z; v[i][k][3] = f.w;
+      }
+    // amax per position on the bit patterns of |x| (order-preserving): thread, then the 16 lanes that share
+    // this position quad (lane bits 0,1,2,4), then the 8 warps
+    unsigned m4[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      float fm = 0.f;
+#pragma unroll
+      for (int i = 0; i < RI; ++i)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) fm = fmaxf(fm, fabsf(v[i][k][j]));
+      m4[j] = __reduce_max_sync(quad_mask, __float_as_uint(fm));
+    }
+    if ((lane & 23) == 0)   // lanes 0 (quad 0) and 8 (quad 1)
+      *reinterpret_cast<uint4*>(&red[(warp * 2 + quad) * 4]) = make_uint4(m4[0], m4[1], m4[2], m4[3]);
+    __syncthreads();
+    int code[4];
+    {
+      uint4 mx = make_uint4(0, 0, 0, 0);
+#pragma unroll
+      for (int w = 0; w < NW; ++w) {
+        const uint4 r4 = *reinterpret_cast<const uint4*>(&red[(w * 2 + quad) * 4]);
+        mx.x = max(mx.x, r4.x); mx.y = max(mx.y, r4.y); mx.z = max(mx.z, r4.z); mx.w = max(mx.w, r4.w);
+      }
+      code[0] = scale_code_of(mx.x, fmt_emax(FMT)); code[1] = scale_code_of(mx.y, fmt_emax(FMT));
+      code[2] = scale_code_of(mx.z, fmt_emax(FMT)); code[3] = scale_code_of(mx.w, fmt_emax(FMT));
+    }
+    if (t < PS) {
+      unsigned mm = 0;
+#pragma unroll
+      for (int w = 0; w < NW; ++w) mm = max(mm, red[(w * 2 + (t >> 2)) * 4 + (t & 3)]);
+      if (q.p0 + t < a.P)
+        a.scales[(long long)(q.p0 + t) * a.sc_stride_p + (long long)q.rt * a.sc_stride_r + q.ct] = (uint8_t)scale_code_of(mm, fmt_emax(FMT));
+    }
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float f = scale_factor(code[j]);
+#pragma unroll
+      for (int i = 0; i < RI; ++i) {
+        const unsigned lo = encode2<FMT>(v[i][0][j] * f, v[i][1][j] * f);
+        const unsigned hi = encode2<FMT>(v[i][2][j] * f, v[i][3][j] * f);
+        uint8_t* dst = stage + ((4 * quad + j) * 32 + rs + 16 * i) * RB;
+        if (FMT == MQ_E2M1) *reinterpret_cast<unsigned short*>(dst + 2 * cq) = (unsigned short)(lo | (hi << 8));
+        else *reinterpret_cast<unsigned*>(dst + 4 * cq) = lo | (hi << 16);
+      }
+    }
+    __syncthreads();
+    // copy out: per position a 32(r) x 32(c) slab; rows are contiguous runs of the stored tensor
+    if (FMT == MQ_E2M1) {
+      const int p = t >> 5, r = t & 31;   // 256 rows of 16 bytes
+      if (t < 256 && q.p0 + p < a.P && q.r0 + r < a.R) {
+        const uint4 val = *reinterpret_cast<const uint4*>(stage + (p * 32 + r) * 16);
+        const long long e = (long long)(q.p0 + p) * a.out_stride_p + (long long)(q.r0 + r) * a.out_stride_r + q.c0;
+        *reinterpret_cast<uint4*>(a.codes + (e >> 1)) = val;
+      }
     } else {
 #pragma unroll
-      for (int j = 0; j < 4; ++j) v[i][j] = (ok && pq + j < a.P) ? __ldg(row + pq + j) : 0.f;
+      for (int k = 0; k < 512 / NT; ++k) {
+        const int id = t + NT * k;  // 512 chunks of 16 bytes
+        const int p = id >> 6, r = (id >> 1) & 31, half = id & 1;
+        if (q.p0 + p < a.P && q.r0 + r < a.R) {
+          const uint4 val = *reinterpret_cast<const uint4*>(stage + (p * 32 + r) * 32 + 16 * half);
+          const long long e = (long long)(q.p0 + p) * a.out_stride_p + (long long)(q.r0 + r) * a.out_stride_r + q.c0 + 16 * half;
+          *reinterpret_cast<uint4*>(a.codes + e) = val;
+        }
+      }
     }
+    // the next iteration's __syncthreads (after its wait) orders these reads of `stage` / `red` before their reuse
   }
+}
 
-  // amax per position over the 32 x 32 tile, on the bit patterns of |x| (order-preserving)
+// Fallback for sources whose position axis is not a multiple of 4 elements (no 16-byte rows): one block per item.
+template <int FMT>
+__global__ void __launch_bounds__(QT_THREADS) quantize_simple_kernel(QuantArgs a, int n_pstrips, int Ct) {
+  __shared__ __align__(16) unsigned red[8][2][4];
+  __shared__ __align__(16) uint8_t stage[PS][32][32];   // one code per byte
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  const Item q = item_of(blockIdx.x, n_pstrips, Ct);
+  const int quad = t & 1, c = (t >> 1) & 31, rsub = t >> 6;
+  const int pq = q.p0 + 4 * quad;
+  float v[8][4];
+  const bool c_ok = (q.c0 + c) < a.C;
+#pragma unroll
+  for (int i = 0; i < 8; ++i) {
+    const int r = q.r0 + 4 * i + rsub;
+    const bool ok = c_ok && r < a.R;
+    const float* row = a.src + ((long long)r * a.C + (q.c0 + c)) * a.P;
+#pragma unroll
+    for (int j = 0; j < 4; ++j) v[i][j] = (ok && pq + j < a.P) ? __ldg(row + pq + j) : 0.f;
+  }
   unsigned m[4];
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
@@ -94,34 +233,27 @@ __global__ void __launch_bounds__(QT_THREADS) quantize_kernel(QuantArgs a, int n
     for (int j = 0; j < 4; ++j) red[warp][lane][j] = m[j];
   }
   __syncthreads();
-  unsigned code[4];
+  int code[4];
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
     unsigned mm = 0;
 #pragma unroll
     for (int w = 0; w < 8; ++w) mm = max(mm, red[w][quad][j]);
-    // floor(log2 amax) = biased exponent - 127 for normal amax; subnormal / zero amax clamps to 0
-    int e = (int)(mm >> 23) - fmt_emax(FMT);
-    code[j] = (unsigned)min(max(e, 0), 254);
+    code[j] = scale_code_of(mm, fmt_emax(FMT));
   }
-  if (t < PS) {  // thread t holds position p0 + t in quad t/4 only if its own quad matches: recompute
+  if (t < PS) {
     unsigned mm = 0;
 #pragma unroll
     for (int w = 0; w < 8; ++w) mm = max(mm, red[w][t >> 2][t & 3]);
-    int e = (int)(mm >> 23) - fmt_emax(FMT);
-    if (p0 + t < a.P) a.scales[(long long)(p0 + t) * a.sc_stride_p + (long long)rt * a.sc_stride_r + ct] = (uint8_t)min(max(e, 0), 254);
+    if (q.p0 + t < a.P)
+      a.scales[(long long)(q.p0 + t) * a.sc_stride_p + (long long)q.rt * a.sc_stride_r + q.ct] = (uint8_t)scale_code_of(mm, fmt_emax(FMT));
   }
-
-  // x * 2^(127 - code), exact: split the power of two so both factors are normal numbers
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    const int ex = 127 - (int)code[j];       // in [-127, 127]
-    const int e1 = ex / 2, e2 = ex - e1;      // |e1|, |e2| <= 64
-    const float f1 = __uint_as_float((unsigned)(e1 + 127) << 23);
-    const float f2 = __uint_as_float((unsigned)(e2 + 127) << 23);
+    const float f = scale_factor(code[j]);
 #pragma unroll
     for (int i = 0; i < 8; i += 2) {
-      unsigned two = encode2<FMT>(v[i][j] * f1 * f2, v[i + 1][j] * f1 * f2);
+      const unsigned two = encode2<FMT>(v[i][j] * f, v[i + 1][j] * f);
       unsigned lo, hi;
       if (FMT == MQ_E2M1) { lo = two & 0xF; hi = (two >> 4) & 0xF; }
       else { lo = two & 0xFF; hi = (two >> 8) & 0xFF; }
@@ -130,40 +262,68 @@ __global__ void __launch_bounds__(QT_THREADS) quantize_kernel(QuantArgs a, int n
     }
   }
   __syncthreads();
-
-  // copy out: per position a 32(r) x 32(c) slab; rows are contiguous runs of the stored tensor
   if (FMT == MQ_E2M1) {
-    // 256 rows (p, r), 16 bytes each after packing two codes per byte
     const int p = t >> 5, r = t & 31;
-    if (p0 + p < a.P && r0 + r < a.R) {
+    if (q.p0 + p < a.P && q.r0 + r < a.R) {
       const uint4* srcw = reinterpret_cast<const uint4*>(&stage[p][r][0]);
-      uint4 lo = srcw[0], hi = srcw[1];
-      uint32_t in[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
+      const uint4 lo = srcw[0], hi = srcw[1];
+      const uint32_t in[8] = {lo.x, lo.y, lo.z, lo.w, hi.x, hi.y, hi.z, hi.w};
       uint32_t outw[4];
 #pragma unroll
       for (int k = 0; k < 4; ++k) {
         // 8 one-byte codes (two words) -> one word of 8 nibbles, lower index in the lower nibble
-        uint32_t w0 = in[2 * k], w1 = in[2 * k + 1];
-        uint32_t b0 = (w0 & 0xF) | ((w0 >> 4) & 0xF0) | ((w0 >> 8) & 0xF00) | ((w0 >> 12) & 0xF000);
-        uint32_t b1 = (w1 & 0xF) | ((w1 >> 4) & 0xF0) | ((w1 >> 8) & 0xF00) | ((w1 >> 12) & 0xF000);
+        const uint32_t w0 = in[2 * k], w1 = in[2 * k + 1];
+        const uint32_t b0 = (w0 & 0xF) | ((w0 >> 4) & 0xF0) | ((w0 >> 8) & 0xF00) | ((w0 >> 12) & 0xF000);
+        const uint32_t b1 = (w1 & 0xF) | ((w1 >> 4) & 0xF0) | ((w1 >> 8) & 0xF00) | ((w1 >> 12) & 0xF000);
         outw[k] = b0 | (b1 << 16);
       }
-      long long e = (long long)(p0 + p) * a.out_stride_p + (long long)(r0 + r) * a.out_stride_r + c0;
+      const long long e = (long long)(q.p0 + p) * a.out_stride_p + (long long)(q.r0 + r) * a.out_stride_r + q.c0;
       *reinterpret_cast<uint4*>(a.codes + (e >> 1)) = make_uint4(outw[0], outw[1], outw[2], outw[3]);
     }
   } else {
 #pragma unroll
     for (int k = 0; k < 2; ++k) {
-      const int id = t + QT_THREADS * k;  // 512 chunks of 16 bytes
+      const int id = t + QT_THREADS * k;
       const int p = id >> 6, r = (id >> 1) & 31, half = id & 1;
-      if (p0 + p < a.P && r0 + r < a.R) {
-        uint4 val = *reinterpret_cast<const uint4*>(&stage[p][r][16 * half]);
-        long long e = (long long)(p0 + p) * a.out_stride_p + (long long)(r0 + r) * a.out_stride_r + c0 + 16 * half;
+      if (q.p0 + p < a.P && q.r0 + r < a.R) {
+        const uint4 val = *reinterpret_cast<const uint4*>(&stage[p][r][16 * half]);
+        const long long e = (long long)(q.p0 + p) * a.out_stride_p + (long long)(q.r0 + r) * a.out_stride_r + q.c0 + 16 * half;
         *reinterpret_cast<uint4*>(a.codes + e) = val;
       }
     }
   }
-  }  // sub-strips
+}
+
+constexpr size_t QPIPE_SMEM = 2 * QBUF_BYTES + PS * 32 * 32 + 16 * 2 * 4 * sizeof(unsigned);
+
+template <int FMT>
+cudaError_t launch_q(const QuantArgs& a, int n_pstrips, int Ct, long long n_items, bool vec, cudaStream_t s) {
+  if (!vec) {
+    quantize_simple_kernel<FMT><<<(unsigned)n_items, QT_THREADS, 0, s>>>(a, n_pstrips, Ct);
+    return cudaGetLastError();
+  }
+  static bool attr_set = false;
+  static int ctas_per_sm = 2;   // 80 KB of shared memory per block
+  static int nt = 256;   // 512-thread blocks measured slower: the kernel is bound by instruction issue
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(quantize_pipe_kernel<FMT, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QPIPE_SMEM);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(quantize_pipe_kernel<FMT, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QPIPE_SMEM);
+    if (e != cudaSuccess) return e;
+    const char* tv = std::getenv("MQ_QUANT_THREADS");
+    if (tv && std::atoi(tv) == 512) nt = 512;
+    const char* v = std::getenv("MQ_QUANT_CTAS");
+    if (v && std::atoi(v) > 0) ctas_per_sm = std::atoi(v);
+    attr_set = true;
+  }
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  long long grid = (long long)sms * ctas_per_sm;
+  if (grid > n_items) grid = n_items;
+  if (nt == 512) quantize_pipe_kernel<FMT, 512><<<(unsigned)grid, 512, QPIPE_SMEM, s>>>(a, n_pstrips, Ct, (unsigned)n_items);
+  else quantize_pipe_kernel<FMT, 256><<<(unsigned)grid, 256, QPIPE_SMEM, s>>>(a, n_pstrips, Ct, (unsigned)n_items);
+  return cudaGetLastError();
 }
 
 }  // namespace
@@ -171,28 +331,18 @@ __global__ void __launch_bounds__(QT_THREADS) quantize_kernel(QuantArgs a, int n
 cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s) {
   const int n_pstrips = (a.P + PS - 1) / PS;
   const int Rt = (a.R + 31) / 32, Ct = a.Cp / 32;
-  static int variant = -1;
-  if (variant < 0) { const char* v = std::getenv("MQ_QUANT_VARIANT"); variant = v ? std::atoi(v) : 0; }
-  const int hint = variant >= 1 ? 1 : 0;
-  int loops = variant >= 2 ? 4 : 1;
-  if (variant == 3) loops = 2;
-  const long long blocks = (long long)((n_pstrips + loops - 1) / loops) * Rt * Ct;
-  if (blocks <= 0 || blocks > 0x7fffffffLL) return cudaErrorInvalidValue;
+  const long long n_items = (long long)n_pstrips * Rt * Ct;
+  if (n_items <= 0 || n_items > 0x7fffffffLL) return cudaErrorInvalidValue;
   const bool vec = (a.P % 4 == 0) && ((reinterpret_cast<uintptr_t>(a.src) & 15) == 0);
-#define MQ_LAUNCH_Q(F)                                                                                  \
-  do {                                                                                                  \
-    if (vec) quantize_kernel<F, true><<<(unsigned)blocks, QT_THREADS, 0, s>>>(a, n_pstrips, Rt, Ct, loops, hint);    \
-    else     quantize_kernel<F, false><<<(unsigned)blocks, QT_THREADS, 0, s>>>(a, n_pstrips, Rt, Ct, loops, hint);   \
-  } while (0)
+  cudaError_t e;
   switch (a.fmt) {
-    case MQ_E4M3: MQ_LAUNCH_Q(MQ_E4M3); break;
-    case MQ_E5M2: MQ_LAUNCH_Q(MQ_E5M2); break;
-    case MQ_E2M1: MQ_LAUNCH_Q(MQ_E2M1); break;
+    case MQ_E4M3: e = launch_q<MQ_E4M3>(a, n_pstrips, Ct, n_items, vec, s); break;
+    case MQ_E5M2: e = launch_q<MQ_E5M2>(a, n_pstrips, Ct, n_items, vec, s); break;
+    case MQ_E2M1: e = launch_q<MQ_E2M1>(a, n_pstrips, Ct, n_items, vec, s); break;
     default: return cudaErrorInvalidValue;
   }
-#undef MQ_LAUNCH_Q
   count_launches(1);
-  return cudaGetLastError();
+  return e;
 }
 
 }  // namespace mq
