@@ -100,7 +100,7 @@ int choose_tw(int w_eff, int N, int layout) {
 struct ConvTcPlan {
   ConvTcParams p;
   int rowbytes, rows_b;
-  size_t off_wt_scales, off_sfa, off_sfb, total;
+  size_t off_wt_scales, off_sfa, off_sfb, off_bimg, total;
 };
 
 bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, ConvTcPlan* out) {
@@ -154,12 +154,31 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   const uint32_t fa = fp4 ? 1u : (fmt_x_like == MQ_E5M2 ? 1u : 0u);
   const uint32_t fb = fp4 ? 1u : (fmt_w == MQ_E5M2 ? 1u : 0u);
   p.idesc = (fa << 7) | (fb << 10) | ((uint32_t)(p.BN >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
+  // whole-tile-per-stage variant: stride 1, one chunk per tap (<= 64 bytes of channels), 8-column tiles
+  p.halo = 0;
+  if (g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && p.TW == 8 && taps <= 64 && !env_int("MQ_TC_NO_HALO", 0)) {
+    const int spa = fp4 ? 2 : 1, atoms_b = (p.BN + 127) / 128;
+    p.WH = p.TW + g.Kw - 1;
+    p.halo_a_bytes = (g.Kh * p.WH * p.TN * p.KB + 1023) / 1024 * 1024;
+    const int sf_bytes = p.max_stages * 512 * spa * (1 + atoms_b);
+    p.halo_stage_bytes = (p.halo_a_bytes + taps * p.BN * p.KB + sf_bytes + 1023) / 1024 * 1024;
+    int hst = (227 * 1024 - 2048) / p.halo_stage_bytes;
+    if (hst > 4) hst = 4;
+    while (hst >= 2 && p.BN + 24 * p.max_stages * hst > 512) --hst;   // TMEM: accumulator(s) + scale buffers of every stage
+    if (hst >= 2 && p.WH <= 256 && taps <= 256) {
+      p.halo = 1;
+      p.stages = hst;
+      p.n_acc = (2 * p.BN + 24 * p.max_stages * hst <= 512) ? 2 : 1;
+    }
+  }
   out->p = p;
   size_t o = 0;
   out->off_wt_scales = 0;
   if (op == MQ_OP_BWD_DATA) { o = wt_codes_bytes(g, fmt_w); out->off_wt_scales = o; o += up256((size_t)g.Ct * taps * g.Cot); }
   out->off_sfa = o; o += up256(conv_tc_sfa_bytes(p));
   out->off_sfb = o; o += up256(conv_tc_sfb_bytes(p));
+  out->off_bimg = o;
+  if (p.halo) o += up256((size_t)p.tiles_c * taps * p.BN * p.KB);
   out->total = o;
   return true;
 }
@@ -194,6 +213,7 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
   p.a_scales = qx_like->scales;
   p.sfa_img = base + pl.off_sfa;
   p.sfb_img = base + pl.off_sfb;
+  p.b_codes = b_codes; p.b_rows_total = pl.rows_b; p.b_rowbytes = pl.rowbytes; p.b_img = base + pl.off_bimg;
   p.out = out; p.out_layout = env_int("MQ_TC_SKIP_STORE", 0) ? 99 : layout; p.status = status;
   if (launch_expand_conv_scales(p, stream) != cudaSuccess) return MQ_ERR_CUDA;
 
@@ -203,11 +223,19 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
     const uint64_t dims[4] = {rb, (uint64_t)p.Ws, (uint64_t)g.N, (uint64_t)p.Hs};
     const uint64_t strides[3] = {(uint64_t)g.N * rb, rb, (uint64_t)p.Ws * g.N * rb};
     const uint32_t wst = op == MQ_OP_FWD ? (uint32_t)g.sw : 1u;
-    const uint32_t box[4] = {(uint32_t)p.KB, (uint32_t)((p.TW - 1) * wst + 1), (uint32_t)p.TN, 1u};
+    uint32_t box[4] = {(uint32_t)p.KB, (uint32_t)((p.TW - 1) * wst + 1), (uint32_t)p.TN, 1u};
+    if (p.halo) { box[1] = (uint32_t)p.WH; box[3] = (uint32_t)g.Kh; }   // the whole halo of a tile in one box
     const uint32_t es[4] = {1u, wst, 1u, 1u};
     if (!encode_tensor_map_u8(&map_a, qx_like->codes, 4, dims, strides, box, es, p.KB)) return MQ_ERR_CUDA;
   }
-  {
+  if (p.halo) {
+    // all taps of a weight tile in one box: dims ordered (channel bytes, rows, taps)
+    const uint64_t rb = (uint64_t)pl.rowbytes;
+    const uint64_t dims[3] = {rb, (uint64_t)pl.rows_b, (uint64_t)taps};
+    const uint64_t strides[2] = {(uint64_t)taps * rb, rb};
+    const uint32_t box[3] = {(uint32_t)p.KB, (uint32_t)p.BN, (uint32_t)taps};
+    if (!encode_tensor_map_u8(&map_b, b_codes, 3, dims, strides, box, nullptr, p.KB)) return MQ_ERR_CUDA;
+  } else {
     const uint64_t rb = (uint64_t)pl.rowbytes;
     const uint64_t dims[3] = {rb, (uint64_t)taps, (uint64_t)pl.rows_b};
     const uint64_t strides[2] = {rb, (uint64_t)taps * rb};

@@ -115,6 +115,79 @@ __device__ __forceinline__ int src_w0(const TapWalk<MODE>& w, const ChunkPos& c)
 template <int MODE>
 __device__ __forceinline__ int tap_index(const TapWalk<MODE>& w, const ChunkPos& c) { return w.tap0 + c.ia * w.tap_dh + c.ib * w.tap_dw; }
 
+// Epilogue role (warps 4-11): TMEM -> registers -> global (fp32), two warps per TMEM lane quadrant, each
+// taking half of the tile's columns.
+template <int MODE>
+__device__ __forceinline__ void epilogue_role(const ConvTcParams& p, uint32_t tmem, uint64_t* tfull, uint64_t* tempty, volatile int* abort_flag,
+                                              int warp, int lane, unsigned total) {
+    const int quad = warp & 3;           // TMEM lane quadrant this warp may read
+    const int half = (warp - 4) >> 2;    // warps 4-7 take the first half of the tile's columns, 8-11 the second
+    const int r = 32 * quad + lane;
+    const int tw_ = r & (p.TW - 1), tn = r >> p.lgTW;
+    const int cbeg = half == 0 ? 0 : ((p.BN / 2 + 15) & ~15);
+    const int cend = half == 0 ? ((p.BN / 2 + 15) & ~15) : p.BN;
+    const long long cs = (long long)p.Hd * p.Wd;
+    uint32_t tcount = 0;
+    PROF_BEGIN();
+    for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
+      const Tile tile = decode_tile(p, t);
+      TapWalk<MODE> tw;
+      tw.init(p, tile);
+      const int Q = tw.chunks(p);
+      const int acc = tcount % p.n_acc;
+      bool ok = true;
+      if (lane == 0) ok = PROF_WAIT(mbar_wait(&tfull[acc], (tcount / p.n_acc) & 1, p.status, MQ_ERR_TIMEOUT));
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) { *abort_flag = 1; break; }
+      tc_fence_after_sync();
+      int yo, xo;
+      if (MODE == MQ_OP_FWD) { yo = tile.h; xo = tile.w0 + tw_; }
+      else { yo = tile.cls / p.sw + p.sh * tile.h; xo = tile.cls % p.sw + p.sw * (tile.w0 + tw_); }
+      const int n = tile.n0 + tn;
+      const bool row_ok = yo < p.Hd && xo < p.Wd && n < p.N;
+      const uint32_t taddr = tmem + acc * p.BN + ((uint32_t)(32 * quad) << 16);
+      const bool full_cols = tile.c0 + p.BN <= p.Cd;
+      float* o_nchw = p.out + (((long long)n * p.Cd + tile.c0 + cbeg) * p.Hd + yo) * p.Wd + xo;
+      float* o_hwnc = p.out + (((long long)yo * p.Wd + xo) * p.N + n) * p.Cd + tile.c0 + cbeg;
+      for (int c = cbeg; c < cend; c += 16) {
+        uint32_t v[16];
+        if (Q > 0) {
+          tmem_ld_32x32b_x16(taddr + c, v);
+          tmem_ld_wait();
+        } else {
+#pragma unroll
+          for (int j = 0; j < 16; ++j) v[j] = 0u;
+        }
+        if (row_ok && p.out_layout != 99) {
+          if (p.out_layout == MQ_NCHW) {
+            if (full_cols) {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) { *o_nchw = __uint_as_float(v[j]); o_nchw += cs; }
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j) { if (tile.c0 + c + j < p.Cd) *o_nchw = __uint_as_float(v[j]); o_nchw += cs; }
+            }
+          } else {
+            if (full_cols && (p.Cd & 3) == 0) {
+#pragma unroll
+              for (int j = 0; j < 16; j += 4)
+                *reinterpret_cast<float4*>(o_hwnc + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+            } else {
+#pragma unroll
+              for (int j = 0; j < 16; ++j)
+                if (tile.c0 + c + j < p.Cd) o_hwnc[j] = __uint_as_float(v[j]);
+            }
+            o_hwnc += 16;
+          }
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty[acc]);
+    }
+    if (lane == 0 && warp == 4) PROF_END(3);
+}
+
 template <int MODE, int KB, bool FP4>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const ConvTcParams p) {
@@ -275,75 +348,161 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else if (warp >= 4) {
-    // ------------------------------------------------------------------ epilogue
-    const int quad = warp & 3;           // TMEM lane quadrant this warp may read
-    const int half = (warp - 4) >> 2;    // warps 4-7 take the first half of the tile's columns, 8-11 the second
-    const int r = 32 * quad + lane;
-    const int tw_ = r & (p.TW - 1), tn = r >> p.lgTW;
-    const int cbeg = half == 0 ? 0 : ((p.BN / 2 + 15) & ~15);
-    const int cend = half == 0 ? ((p.BN / 2 + 15) & ~15) : p.BN;
-    const long long cs = (long long)p.Hd * p.Wd;
-    uint32_t tcount = 0;
-    PROF_BEGIN();
-    for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
-      const Tile tile = decode_tile(p, t);
-      TapWalk<MODE> tw;
-      tw.init(p, tile);
-      const int Q = tw.chunks(p);
-      const int acc = tcount % p.n_acc;
-      bool ok = true;
-      if (lane == 0) ok = PROF_WAIT(mbar_wait(&tfull[acc], (tcount / p.n_acc) & 1, p.status, MQ_ERR_TIMEOUT));
-      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
-      if (!ok) { *abort_flag = 1; break; }
-      tc_fence_after_sync();
-      int yo, xo;
-      if (MODE == MQ_OP_FWD) { yo = tile.h; xo = tile.w0 + tw_; }
-      else { yo = tile.cls / p.sw + p.sh * tile.h; xo = tile.cls % p.sw + p.sw * (tile.w0 + tw_); }
-      const int n = tile.n0 + tn;
-      const bool row_ok = yo < p.Hd && xo < p.Wd && n < p.N;
-      const uint32_t taddr = tmem + acc * p.BN + ((uint32_t)(32 * quad) << 16);
-      const bool full_cols = tile.c0 + p.BN <= p.Cd;
-      float* o_nchw = p.out + (((long long)n * p.Cd + tile.c0 + cbeg) * p.Hd + yo) * p.Wd + xo;
-      float* o_hwnc = p.out + (((long long)yo * p.Wd + xo) * p.N + n) * p.Cd + tile.c0 + cbeg;
-      for (int c = cbeg; c < cend; c += 16) {
-        uint32_t v[16];
-        if (Q > 0) {
-          tmem_ld_32x32b_x16(taddr + c, v);
-          tmem_ld_wait();
-        } else {
-#pragma unroll
-          for (int j = 0; j < 16; ++j) v[j] = 0u;
-        }
-        if (row_ok && p.out_layout != 99) {
-          if (p.out_layout == MQ_NCHW) {
-            if (full_cols) {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) { *o_nchw = __uint_as_float(v[j]); o_nchw += cs; }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) { if (tile.c0 + c + j < p.Cd) *o_nchw = __uint_as_float(v[j]); o_nchw += cs; }
-            }
-          } else {
-            if (full_cols && (p.Cd & 3) == 0) {
-#pragma unroll
-              for (int j = 0; j < 16; j += 4)
-                *reinterpret_cast<float4*>(o_hwnc + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
-            } else {
-#pragma unroll
-              for (int j = 0; j < 16; ++j)
-                if (tile.c0 + c + j < p.Cd) o_hwnc[j] = __uint_as_float(v[j]);
-            }
-            o_hwnc += 16;
-          }
-        }
-      }
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&tempty[acc]);
-    }
-    if (lane == 0 && warp == 4) PROF_END(3);
+    epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
   }
   // teardown: everyone meets here (all loops are bounded), then the allocating warp frees TMEM
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) tmem_dealloc(tmem, 512);
+}
+
+// ---- whole-tile-per-stage variant -------------------------------------------------------------------
+// For stride-1 layers whose tap has at most 64 bytes of channels (one chunk per tap), the per-tap TMA boxes
+// of the kernel above are tiny and their issue rate is the limit.  Here a pipeline stage holds the whole K
+// range of a tile: ONE TMA box brings the activation halo ([Kh rows][TW + Kw - 1 columns][TN samples][KB]) --
+// every stored pixel once, the data reuse of Sec. IV-A -- and ONE bulk copy brings all taps of the weight tile
+// (a pre-swizzled image written by the expansion kernel; per-row TMA requests of 32 bytes were the limit);
+// each tap's A operand is a shifted view of the halo (start = (row * WH * TN + column shift) * KB, 8-row
+// groups WH * KB bytes apart: TW = 8 output columns are exactly one 8-row swizzle group).  Two bulk copies
+// bring the tile's scale chunks.  Roles and barriers are those of conv_tc_kernel.
+template <int MODE, int KB, bool FP4>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const ConvTcParams p) {
+  constexpr int G = 128 / KB, APC = KB / 32, SPA = FP4 ? 2 : 1;
+  constexpr int LAYOUT = KB == 128 ? 2 : (KB == 64 ? 4 : 6);
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  const int taps = p.Kh * p.Kw;
+  const int nsf = p.max_stages;                        // scale chunks (groups of 4 MMAs) per tile
+  const int atoms_b = (p.BN + 127) / 128;
+  const int b_bytes = taps * p.BN * KB;
+  const int sfa_bytes = nsf * 512 * SPA, sfb_bytes = nsf * 512 * SPA * atoms_b;
+  const int stage_bytes = p.halo_stage_bytes;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * stage_bytes);
+  uint64_t* empty = full + p.stages;
+  uint64_t* sffull = empty + p.stages;
+  uint64_t* tfull = sffull + p.stages;
+  uint64_t* tempty = tfull + 2;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned total = (unsigned)p.total_tiles;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 8); }
+    *abort_flag = 0;
+    mbar_fence_init();
+    prefetch_tensormap(&map_a);
+    prefetch_tensormap(&map_b);
+  }
+  if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem = *tmem_slot;
+  const uint32_t sf_cols_stage = (uint32_t)nsf * SF_COLS;
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ producer: 2 TMA boxes + 2 bulk copies per tile
+    if (lane == 0) {
+      uint32_t s = 0, phase = 0;
+      PROF_BEGIN();
+      for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x) {
+        const Tile tile = decode_tile(p, t);
+        if (!PROF_WAIT(mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+        uint8_t* sa = smem + (size_t)s * stage_bytes;
+        uint8_t* sb = sa + p.halo_a_bytes;
+        // first source pixel of the halo: forward (h - ph, w0 - pw); input gradient (h + ph - (Kh-1), w0 + pw - (Kw-1))
+        const int hs = MODE == MQ_OP_FWD ? tile.h - p.ph : tile.h + p.ph - (p.Kh - 1);
+        const int ws = MODE == MQ_OP_FWD ? tile.w0 - p.pw : tile.w0 + p.pw - (p.Kw - 1);
+        mbar_arrive_expect_tx(&full[s], (uint32_t)(p.Kh * p.WH * p.TN * KB + b_bytes + sfa_bytes + sfb_bytes));
+        tma_load_4d(sa, &map_a, &full[s], 0, ws, tile.n0, hs);
+        bulk_load(sb, p.b_img + (size_t)(tile.c0 / p.BN) * b_bytes, b_bytes, &full[s]);   // all taps, already swizzled
+        bulk_load(sb + b_bytes, p.sfa_img + (size_t)tile_m_index(p, tile) * sfa_bytes, sfa_bytes, &full[s]);
+        bulk_load(sb + b_bytes + sfa_bytes, p.sfb_img + ((size_t)tile.cls * p.tiles_c + tile.c0 / p.BN) * sfb_bytes, sfb_bytes, &full[s]);
+        if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
+      }
+      PROF_END(0);
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer: all taps of a tile per stage
+    if (lane == 0) {
+      const uint64_t a_desc_base = smem_desc_base(16, (uint32_t)(p.WH * KB), LAYOUT);   // 8-row groups WH pixels apart
+      const uint64_t b_desc_base = smem_desc_base(16, 8 * KB, LAYOUT);
+      const uint32_t sf_base = tmem + p.n_acc * p.BN;
+      uint32_t idesc_id[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) idesc_id[i] = idesc_with_sf_ids(p.idesc, i, i);
+      uint32_t s = 0, phase = 0, tcount = 0;
+      PROF_BEGIN();
+      for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
+        const int acc = tcount % p.n_acc;
+        if (!PROF_WAIT(mbar_wait(&tempty[acc], ((tcount / p.n_acc) & 1) ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+        if (!PROF_WAIT(mbar_wait(&sffull[s], phase, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+        tc_fence_after_sync();
+        const uint32_t d_tmem = tmem + acc * p.BN;
+        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
+        const uint32_t sb = sa + p.halo_a_bytes;
+        const uint32_t sf_t = sf_base + s * sf_cols_stage;
+        uint32_t accumulate = 0;
+        int q = 0;
+        for (int kh = 0; kh < p.Kh; ++kh)
+          for (int kw = 0; kw < p.Kw; ++kw, ++q) {
+            // tap q of the walk: forward reads halo row kh, column shift kw; the input gradient walks the taps in
+            // the same (kh, kw) order but its source pixel moves the other way
+            const int hrow = MODE == MQ_OP_FWD ? kh : p.Kh - 1 - kh, wsh = MODE == MQ_OP_FWD ? kw : p.Kw - 1 - kw;
+            const uint32_t a_addr = sa + (uint32_t)((hrow * p.WH * p.TN + wsh) * KB);
+            const uint32_t b_addr = sb + (uint32_t)((kh * p.Kw + kw) * p.BN * KB);
+            const int sfst = q / G;
+            const uint32_t sfa_t = sf_t + sfst * SF_COLS, sfb_t = sfa_t + 8;
+#pragma unroll
+            for (int ja = 0; ja < APC; ++ja) {
+              const int atom = (q % G) * APC + ja;
+              const int g = (atom * SPA) >> 2, id = (atom * SPA) & 3;
+              const uint64_t ad = smem_desc(a_desc_base, a_addr + ja * 32);
+              const uint64_t bd = smem_desc(b_desc_base, b_addr + ja * 32);
+              if (FP4) mma_mxf4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accumulate);
+              else mma_mxf8f6f4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accumulate);
+              accumulate = 1;
+            }
+          }
+        tc_commit(&empty[s]);
+        tc_commit(&tfull[acc]);
+        if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
+      }
+      PROF_END(1);
+    }
+  } else if (warp == 2) {
+    // ------------------------------------------------------------------ scale copier: the tile's chunks smem -> TMEM
+    if (lane == 0) {
+      const uint64_t sf_desc = smem_desc_base(0, 128, 0);
+      const uint32_t sf_base = tmem + p.n_acc * p.BN;
+      uint32_t s = 0, phase = 0;
+      PROF_BEGIN();
+      for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x) {
+        if (!PROF_WAIT(mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+        tc_fence_after_sync();
+        const uint32_t sfa_s = smem_u32(smem + (size_t)s * stage_bytes + p.halo_a_bytes + b_bytes);
+        const uint32_t sfb_s = sfa_s + sfa_bytes;
+        const uint32_t sf_t = sf_base + s * sf_cols_stage;
+        for (int st = 0; st < nsf; ++st) {
+          const uint32_t sfa_t = sf_t + st * SF_COLS, sfb_t = sfa_t + 8;
+#pragma unroll
+          for (int g = 0; g < SPA; ++g) {
+            tmem_cp_32x128b_warpx4(sfa_t + 4 * g, smem_desc(sf_desc, sfa_s + (st * SPA + g) * 512));
+            for (int a = 0; a < atoms_b; ++a)
+              tmem_cp_32x128b_warpx4(sfb_t + 4 * (g * atoms_b + a), smem_desc(sf_desc, sfb_s + ((st * SPA + g) * atoms_b + a) * 512));
+          }
+        }
+        tc_commit(&sffull[s]);
+        if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
+      }
+      PROF_END(2);
+    }
+  } else if (warp >= 4) {
+    epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
+  }
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem, 512);
@@ -370,6 +529,24 @@ __global__ void __launch_bounds__(256) expand_conv_scales_kernel(const ConvTcPar
   const unsigned nA = n_tile_m * (unsigned)p.max_stages;
   const unsigned nB = (unsigned)(p.classes * p.tiles_c * p.max_stages);
   const int atoms_b = (p.BN + 127) / 128;
+  if (p.halo && wid >= nA + nB) {
+    // weight tile images for the whole-tile variant: one 16-byte chunk per thread
+    const int taps_all = p.Kh * p.Kw;
+    constexpr int CPR = KB / 16;                       // chunks per row
+    const unsigned chunks = (unsigned)(p.tiles_c * taps_all * p.BN) * CPR;
+    const unsigned i = (wid - nA - nB) * 32u + (unsigned)lane;
+    if (i < chunks) {
+      const unsigned row_id = i / CPR; const int ch = (int)(i - row_id * CPR);
+      const unsigned tt = row_id / (unsigned)p.BN; const int r = (int)(row_id - tt * p.BN);
+      const int ct = (int)(tt / (unsigned)taps_all), tap = (int)(tt - (unsigned)ct * taps_all);
+      const int row = ct * p.BN + r;
+      uint4 v = make_uint4(0, 0, 0, 0);
+      if (row < p.b_rows_total) v = __ldg(reinterpret_cast<const uint4*>(p.b_codes + ((size_t)row * taps_all + tap) * p.b_rowbytes) + ch);
+      const int sw = KB == 128 ? (r & 7) : (KB == 64 ? ((r >> 1) & 3) : ((r >> 2) & 1));
+      *reinterpret_cast<uint4*>(p.b_img + (size_t)row_id * KB + ((ch ^ sw) << 4)) = v;
+    }
+    return;
+  }
   if (wid < nA) {
     const unsigned tm = wid / (unsigned)p.max_stages;
     const int st = (int)(wid - tm * p.max_stages);
@@ -558,7 +735,8 @@ size_t conv_tc_sfb_bytes(const ConvTcParams& p) {
 template <int MODE, int KB, bool FP4>
 cudaError_t launch_expand_inst(const ConvTcParams& p, cudaStream_t s) {
   const unsigned n_tile_m = (unsigned)(p.total_tiles / p.tiles_c);
-  const unsigned long long warps = (unsigned long long)n_tile_m * p.max_stages + (unsigned long long)p.classes * p.tiles_c * p.max_stages;
+  unsigned long long warps = (unsigned long long)n_tile_m * p.max_stages + (unsigned long long)p.classes * p.tiles_c * p.max_stages;
+  if (p.halo) warps += ((unsigned long long)p.tiles_c * p.Kh * p.Kw * p.BN * (KB / 16) + 31) / 32;
   const unsigned blocks = (unsigned)((warps + 7) / 8);
   expand_conv_scales_kernel<MODE, KB, FP4><<<blocks, 256, 0, s>>>(p, n_tile_m);
   count_launches(1);
@@ -575,8 +753,33 @@ cudaError_t launch_expand_conv_scales(const ConvTcParams& p, cudaStream_t s) {
   return cudaErrorInvalidValue;
 }
 
+template <int MODE, int KB, bool FP4>
+cudaError_t launch_conv_tc_halo_inst(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s) {
+  static bool attr_set = false;
+  const size_t smem = 1024 + (size_t)p.stages * p.halo_stage_bytes + (3 * (size_t)p.stages + 4) * 8 + 64;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(conv_tc_halo_kernel<MODE, KB, FP4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const unsigned grid = (unsigned)(p.total_tiles < sms ? p.total_tiles : sms);
+  conv_tc_halo_kernel<MODE, KB, FP4><<<grid, TC_THREADS, smem, s>>>(map_a, map_b, p);
+  count_launches(1);
+  return cudaGetLastError();
+}
+
 cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s) {
   if (p.total_tiles <= 0 || p.total_tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
+  if (p.halo) {
+#define MQ_TC_HCASE(M, K, F) if (p.mode == M && p.KB == K && (p.kind_fp4 != 0) == F) return launch_conv_tc_halo_inst<M, K, F>(p, map_a, map_b, s)
+    MQ_TC_HCASE(MQ_OP_FWD, 64, false); MQ_TC_HCASE(MQ_OP_FWD, 32, false); MQ_TC_HCASE(MQ_OP_FWD, 64, true); MQ_TC_HCASE(MQ_OP_FWD, 32, true);
+    MQ_TC_HCASE(MQ_OP_BWD_DATA, 64, false); MQ_TC_HCASE(MQ_OP_BWD_DATA, 32, false); MQ_TC_HCASE(MQ_OP_BWD_DATA, 64, true); MQ_TC_HCASE(MQ_OP_BWD_DATA, 32, true);
+#undef MQ_TC_HCASE
+    return cudaErrorInvalidValue;
+  }
 #define MQ_TC_CASE(M, K, F) if (p.mode == M && p.KB == K && (p.kind_fp4 != 0) == F) return launch_conv_tc_inst<M, K, F>(p, map_a, map_b, s)
   MQ_TC_CASE(MQ_OP_FWD, 128, false); MQ_TC_CASE(MQ_OP_FWD, 64, false); MQ_TC_CASE(MQ_OP_FWD, 32, false);
   MQ_TC_CASE(MQ_OP_FWD, 128, true);  MQ_TC_CASE(MQ_OP_FWD, 64, true);  MQ_TC_CASE(MQ_OP_FWD, 32, true);

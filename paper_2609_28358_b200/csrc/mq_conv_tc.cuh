@@ -41,6 +41,14 @@ struct ConvTcParams {
   uint8_t* sfa_img;         // [tile without the channel index][max_stages][512 * SPA]
   uint8_t* sfb_img;         // [class][channel tile][max_stages][512 * SPA * atoms_b]
   int max_stages;           // stages of the longest tile
+  // whole-tile-per-stage variant (small channel counts, stride 1): see conv_tc_halo_kernel
+  int halo;                 // 1: use it
+  int WH;                   // halo width in pixels = TW + Kw - 1
+  int halo_a_bytes;         // bytes of the activation halo of a tile (rounded up to 1024)
+  int halo_stage_bytes;     // bytes of one pipeline stage (halo + all taps of B + scale chunks)
+  const uint8_t* b_codes;   // weight-like codes [rows][taps][b_rowbytes] (source of the images below)
+  int b_rows_total, b_rowbytes;
+  uint8_t* b_img;           // [channel tile][tap][BN rows][KB], each row stored with the KB-byte swizzle applied
   // output
   float* out;
   int out_layout;
