@@ -79,7 +79,7 @@ size_t up256(size_t v) { return (v + 255) / 256 * 256; }
 
 // Output columns per tile.  Rows of a tile are TW consecutive output columns x TN = 128/TW samples with
 // the column index fastest, so an NCHW store writes runs of TW floats; TW >= 8 fills 32-byte sectors.
-int choose_tw(int w_eff, int N, int layout) {
+int choose_tw(int w_eff, int N, int layout, bool wide) {
   const int forced = env_int("MQ_TC_TW", 0);
   if (forced > 0) return forced;
   int best = 1;
@@ -89,6 +89,7 @@ int choose_tw(int w_eff, int N, int layout) {
     const double waste = (double)((w_eff + tw - 1) / tw * tw) / w_eff * (double)((N + tn - 1) / tn * tn) / N;
     double pen = 1.0;
     if (layout == MQ_NCHW) pen = tw >= 8 ? 1.0 : (tw == 4 ? 1.25 : (tw == 2 ? 1.8 : 2.5));
+    if (layout == MQ_NCHW && wide && env_int("MQ_TC_WIDE", 0)) pen = tw >= 32 ? 1.0 : (tw == 16 ? 1.05 : (tw == 8 ? 1.2 : pen * 1.2));
     const double cost = waste * pen;
     if (cost < best_cost - 1e-9) { best_cost = cost; best = tw; }
   }
@@ -127,7 +128,8 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   p.G = 128 / p.KB;
   p.cpt = rowbytes / p.KB;
   const int w_eff = op == MQ_OP_FWD ? g.Wo : (g.W + g.sw - 1) / g.sw;
-  p.TW = choose_tw(w_eff, g.N, layout);
+  const bool thin = g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && g.Kw > 1;
+  p.TW = choose_tw(w_eff, g.N, layout, thin && !env_int("MQ_TC_NO_HALO", 0));
   if (p.TW < 1 || p.TW > 32 || (p.TW & (p.TW - 1))) return false;
   p.TN = 128 / p.TW;
   p.lgTW = 0;
@@ -141,6 +143,19 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   p.tiles_n = (g.N + p.TN - 1) / p.TN;
   p.total_tiles = (long long)p.tiles_c * p.tiles_w * p.tiles_n * p.tiles_h * p.classes;
   if (p.total_tiles > 0x7fffffffLL) return false;
+  p.lgTN = 7 - p.lgTW;
+  {
+    // multiply-high reciprocals for the per-tile index arithmetic: exact while numerator * divisor < 2^32
+    bool exact = true;
+    auto magic = [&](int d) -> uint32_t {
+      if (d <= 1) return 0u;
+      if ((unsigned long long)p.total_tiles * (unsigned long long)d >= (1ull << 32)) { exact = false; return 0u; }
+      return (uint32_t)(((1ull << 32) + (unsigned long long)d - 1) / (unsigned long long)d);
+    };
+    p.m_classes = magic(p.classes); p.m_tiles_w = magic(p.tiles_w); p.m_tiles_h = magic(p.tiles_h); p.m_tiles_c = magic(p.tiles_c);
+    p.m_sh = magic(g.sh); p.m_sw = magic(g.sw);
+    if (!exact) return false;
+  }
   const size_t stage_bytes = 128 * 128 + (size_t)p.BN * 128 + 3072;
   int stages = (int)((227 * 1024 - 2048) / stage_bytes);
   if (stages > 8) stages = 8;
@@ -154,21 +169,32 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   const uint32_t fa = fp4 ? 1u : (fmt_x_like == MQ_E5M2 ? 1u : 0u);
   const uint32_t fb = fp4 ? 1u : (fmt_w == MQ_E5M2 ? 1u : 0u);
   p.idesc = (fa << 7) | (fb << 10) | ((uint32_t)(p.BN >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
-  // whole-tile-per-stage variant: stride 1, one chunk per tap (<= 64 bytes of channels), 8-column tiles
+  // whole-tile-per-stage variant: stride 1, one chunk per tap (<= 64 bytes of channels).  One box with the column
+  // halo needs 8-column tiles; one box per column shift takes 8, 16 or 32 columns (longer NCHW store runs).
   p.halo = 0;
-  if (g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && p.TW == 8 && taps <= 64 && !env_int("MQ_TC_NO_HALO", 0)) {
+  if (g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && taps <= 64 && !env_int("MQ_TC_NO_HALO", 0)) {
     const int spa = fp4 ? 2 : 1, atoms_b = (p.BN + 127) / 128;
-    p.WH = p.TW + g.Kw - 1;
-    p.halo_a_bytes = (g.Kh * p.WH * p.TN * p.KB + 1023) / 1024 * 1024;
-    const int sf_bytes = p.max_stages * 512 * spa * (1 + atoms_b);
-    p.halo_stage_bytes = (p.halo_a_bytes + taps * p.BN * p.KB + sf_bytes + 1023) / 1024 * 1024;
-    int hst = (227 * 1024 - 2048) / p.halo_stage_bytes;
-    if (hst > 4) hst = 4;
-    while (hst >= 2 && p.BN + 24 * p.max_stages * hst > 512) --hst;   // TMEM: accumulator(s) + scale buffers of every stage
-    if (hst >= 2 && p.WH <= 256 && taps <= 256) {
-      p.halo = 1;
-      p.stages = hst;
-      p.n_acc = (2 * p.BN + 24 * p.max_stages * hst <= 512) ? 2 : 1;
+    int nbox = env_int("MQ_TC_NBOX", 0);
+    if (nbox != 1 && nbox != g.Kw) nbox = (layout == MQ_NCHW && p.TW >= 16) ? g.Kw : 1;
+    if (g.Kw == 1) nbox = 1;
+    if ((nbox == 1 && p.TW == 8) || (nbox > 1 && p.TW >= 8)) {
+      p.nbox = nbox;
+      p.WH = nbox == 1 ? p.TW + g.Kw - 1 : p.TW;
+      p.halo_box_bytes = g.Kh * p.WH * p.TN * p.KB;
+      p.halo_a_bytes = (nbox * p.halo_box_bytes + 1023) / 1024 * 1024;
+      p.halo_stage_bytes = (p.halo_a_bytes + p.max_stages * 512 * spa + 1023) / 1024 * 1024;
+      p.halo_b_bytes = (taps * p.BN * p.KB + p.max_stages * 512 * spa * atoms_b + 1023) / 1024 * 1024;
+      // NCHW output through TMA stores: rows of the output must be 16-byte multiples
+      p.tma_store = layout == MQ_NCHW && p.Wd % 4 == 0 && p.TW >= 4 && p.TW <= 32 && !env_int("MQ_TC_NO_TMA_STORE", 0);
+      int hst = (227 * 1024 - 4096 - p.halo_b_bytes - (p.tma_store ? 65536 : 0)) / p.halo_stage_bytes;
+      if (hst > 4) hst = 4;
+      // TMEM: accumulator(s), 16 columns per chunk of resident weight scales, 8 per chunk per stage
+      while (hst >= 2 && p.BN + 16 * p.max_stages + 8 * p.max_stages * hst > 512) --hst;
+      if (hst >= 2 && p.WH <= 256 && (p.halo_box_bytes % 1024 == 0 || nbox == 1)) {
+        p.halo = 1;
+        p.stages = hst;
+        p.n_acc = (2 * p.BN + 16 * p.max_stages + 8 * p.max_stages * hst <= 512) ? 2 : 1;
+      }
     }
   }
   out->p = p;
@@ -229,12 +255,18 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
     if (!encode_tensor_map_u8(&map_a, qx_like->codes, 4, dims, strides, box, es, p.KB)) return MQ_ERR_CUDA;
   }
   if (p.halo) {
-    // all taps of a weight tile in one box: dims ordered (channel bytes, rows, taps)
-    const uint64_t rb = (uint64_t)pl.rowbytes;
-    const uint64_t dims[3] = {rb, (uint64_t)pl.rows_b, (uint64_t)taps};
-    const uint64_t strides[2] = {(uint64_t)taps * rb, rb};
-    const uint32_t box[3] = {(uint32_t)p.KB, (uint32_t)p.BN, (uint32_t)taps};
-    if (!encode_tensor_map_u8(&map_b, b_codes, 3, dims, strides, box, nullptr, p.KB)) return MQ_ERR_CUDA;
+    map_b = map_a;   // the weight tile comes as a pre-swizzled image by bulk copy; the second map is the output's
+    if (p.tma_store) {
+      if (reinterpret_cast<uintptr_t>(out) % 16 != 0) p.tma_store = 0;
+      else {
+        const uint64_t dims[4] = {(uint64_t)p.Wd, (uint64_t)g.N, (uint64_t)p.Cd, (uint64_t)p.Hd};
+        const uint64_t strides[3] = {(uint64_t)p.Cd * p.Hd * p.Wd * 4, (uint64_t)p.Hd * p.Wd * 4, (uint64_t)p.Wd * 4};
+        // one epilogue warp's 32 rows x the channels of a column half (at most 64)
+        const int half_cols = (p.BN / 2 + 15) & ~15;
+        const uint32_t box[4] = {(uint32_t)p.TW, (uint32_t)(32 / p.TW), (uint32_t)(half_cols < 64 ? half_cols : 64), 1u};
+        if (!encode_tensor_map_u8(&map_b, out, 4, dims, strides, box, nullptr, 0, true)) return MQ_ERR_CUDA;
+      }
+    }
   } else {
     const uint64_t rb = (uint64_t)pl.rowbytes;
     const uint64_t dims[3] = {rb, (uint64_t)taps, (uint64_t)pl.rows_b};

@@ -32,44 +32,55 @@ constexpr int SFB_BYTES = 2048;   // up to 2 groups x 2 atoms of 128 rows
 constexpr int SF_COLS = 24;       // TMEM columns of one scale buffer: 8 (A) + 16 (B)
 
 // Cycle counters of block 0's roles (debug aid): [role][0] = cycles in the role's loop, [role][1] = cycles waiting.
-__device__ unsigned long long g_prof[8][2];
 #ifdef MQ_TC_PROFILE
+__device__ unsigned long long g_prof[8][2];
+__device__ unsigned long long g_blk[160][4];   // per block: SM id, start, body start, end (ns)
+__device__ unsigned long long g_role[160][4][2];   // per block and role: cycles in the loop, cycles waiting
+#define PROF_CLK() clock64()
+#define PROF_ADD(slot, idx, v) do { if (blockIdx.x == 0) g_prof[slot][idx] += (unsigned long long)(v); } while (0)
 #define PROF_BEGIN() const long long prof_t0 = clock64(); long long prof_wait = 0
 #define PROF_WAIT(expr) ([&]() { const long long w0_ = clock64(); const bool r_ = (expr); prof_wait += clock64() - w0_; return r_; }())
-#define PROF_END(role) do { if (blockIdx.x == 0) { g_prof[role][0] = clock64() - prof_t0; g_prof[role][1] = prof_wait; } } while (0)
+#define PROF_END(role) do { if (blockIdx.x == 0) { g_prof[role][0] = clock64() - prof_t0; g_prof[role][1] = prof_wait; } \
+    if (blockIdx.x < 160) { g_role[blockIdx.x][role][0] = clock64() - prof_t0; g_role[blockIdx.x][role][1] = prof_wait; } } while (0)
 #else
+#define PROF_CLK() 0ll
+#define PROF_ADD(slot, idx, v) do { } while (0)
 #define PROF_BEGIN() do { } while (0)
 #define PROF_WAIT(expr) (expr)
 #define PROF_END(role) do { } while (0)
 #endif
 
-struct Tile { int c0, w0, n0, h, cls; };
+struct Tile { int c0, w0, n0, h, cls, ct; };
 
 // Tile order: stride class fastest (the classes of an input gradient interleave inside the same 32-byte
 // sectors), then output column tile, output row, channel tile, sample tile.  Tiles that run at the same time
 // then complete whole (n, c) planes of an NCHW output quickly, so partially written lines do not linger in
 // L2, and they share input rows between neighbouring taps.
+// Division by a launch constant: d == 1 costs nothing, otherwise one multiply-high with m = ceil(2^32 / d)
+// (exact while t * d < 2^32; the host refuses to plan a launch for which that does not hold).
+__device__ __forceinline__ unsigned fdiv(unsigned t, int d, uint32_t m) { return d == 1 ? t : __umulhi(t, m); }
+
 __device__ __forceinline__ Tile decode_tile(const ConvTcParams& p, unsigned t) {
   Tile q;
-  unsigned u = t / (unsigned)p.classes;
+  unsigned u = fdiv(t, p.classes, p.m_classes);
   q.cls = (int)(t - u * p.classes); t = u;
-  u = t / (unsigned)p.tiles_w; q.w0 = (int)(t - u * p.tiles_w) * p.TW; t = u;
-  u = t / (unsigned)p.tiles_h; q.h = (int)(t - u * p.tiles_h); t = u;
-  u = t / (unsigned)p.tiles_c; q.c0 = (int)(t - u * p.tiles_c) * p.BN;
+  u = fdiv(t, p.tiles_w, p.m_tiles_w); q.w0 = (int)(t - u * p.tiles_w) * p.TW; t = u;
+  u = fdiv(t, p.tiles_h, p.m_tiles_h); q.h = (int)(t - u * p.tiles_h); t = u;
+  u = fdiv(t, p.tiles_c, p.m_tiles_c); q.ct = (int)(t - u * p.tiles_c); q.c0 = q.ct * p.BN;
   q.n0 = (int)u * p.TN;
   return q;
 }
 // index of a tile among the tiles that differ in anything but the channel tile (A-side scale chunks)
 __device__ __forceinline__ unsigned tile_m_index(const ConvTcParams& p, const Tile& q) {
-  return (((unsigned)(q.n0 / p.TN) * p.tiles_h + q.h) * p.tiles_w + q.w0 / p.TW) * p.classes + q.cls;
+  return (((unsigned)(q.n0 >> p.lgTN) * p.tiles_h + q.h) * p.tiles_w + (q.w0 >> p.lgTW)) * p.classes + q.cls;
 }
 __device__ __forceinline__ Tile tile_of_m_index(const ConvTcParams& p, unsigned tm) {
   Tile q;
-  unsigned u = tm / (unsigned)p.classes;
+  unsigned u = fdiv(tm, p.classes, p.m_classes);
   q.cls = (int)(tm - u * p.classes); tm = u;
-  u = tm / (unsigned)p.tiles_w; q.w0 = (int)(tm - u * p.tiles_w) * p.TW; tm = u;
-  u = tm / (unsigned)p.tiles_h; q.h = (int)(tm - u * p.tiles_h);
-  q.n0 = (int)u * p.TN; q.c0 = 0;
+  u = fdiv(tm, p.tiles_w, p.m_tiles_w); q.w0 = (int)(tm - u * p.tiles_w) * p.TW; tm = u;
+  u = fdiv(tm, p.tiles_h, p.m_tiles_h); q.h = (int)(tm - u * p.tiles_h);
+  q.n0 = (int)u * p.TN; q.c0 = 0; q.ct = 0;
   return q;
 }
 
@@ -89,11 +100,12 @@ struct TapWalk {
       hs0 = t.h * p.sh - p.ph; ws0 = t.w0 * p.sw - p.pw;
       tap0 = 0; tap_dh = p.Kw; tap_dw = 1;
     } else {
-      const int ch = t.cls / p.sw, cw = t.cls - ch * p.sw;
-      const int kh0 = (ch + p.ph) % p.sh, kw0 = (cw + p.pw) % p.sw;
-      nkh = kh0 < p.Kh ? (p.Kh - kh0 + p.sh - 1) / p.sh : 0;
-      nkw = kw0 < p.Kw ? (p.Kw - kw0 + p.sw - 1) / p.sw : 0;
-      hs0 = t.h + (ch + p.ph - kh0) / p.sh; ws0 = t.w0 + (cw + p.pw - kw0) / p.sw;
+      const int ch = (int)fdiv((unsigned)t.cls, p.sw, p.m_sw), cw = t.cls - ch * p.sw;
+      const int kh0 = (ch + p.ph) - (int)fdiv((unsigned)(ch + p.ph), p.sh, p.m_sh) * p.sh;
+      const int kw0 = (cw + p.pw) - (int)fdiv((unsigned)(cw + p.pw), p.sw, p.m_sw) * p.sw;
+      nkh = kh0 < p.Kh ? (int)fdiv((unsigned)(p.Kh - kh0 + p.sh - 1), p.sh, p.m_sh) : 0;
+      nkw = kw0 < p.Kw ? (int)fdiv((unsigned)(p.Kw - kw0 + p.sw - 1), p.sw, p.m_sw) : 0;
+      hs0 = t.h + (int)fdiv((unsigned)(ch + p.ph - kh0), p.sh, p.m_sh); ws0 = t.w0 + (int)fdiv((unsigned)(cw + p.pw - kw0), p.sw, p.m_sw);
       tap0 = kh0 * p.Kw + kw0; tap_dh = p.sh * p.Kw; tap_dw = p.sw;
     }
   }
@@ -134,21 +146,27 @@ __device__ __forceinline__ void epilogue_role(const ConvTcParams& p, uint32_t tm
       TapWalk<MODE> tw;
       tw.init(p, tile);
       const int Q = tw.chunks(p);
-      const int acc = tcount % p.n_acc;
+      const int acc = (int)(tcount & (uint32_t)(p.n_acc - 1));
       bool ok = true;
-      if (lane == 0) ok = PROF_WAIT(mbar_wait(&tfull[acc], (tcount / p.n_acc) & 1, p.status, MQ_ERR_TIMEOUT));
+      if (lane == 0) ok = PROF_WAIT(mbar_wait(&tfull[acc], (tcount >> (p.n_acc - 1)) & 1, p.status, MQ_ERR_TIMEOUT));
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) { *abort_flag = 1; break; }
       tc_fence_after_sync();
       int yo, xo;
       if (MODE == MQ_OP_FWD) { yo = tile.h; xo = tile.w0 + tw_; }
-      else { yo = tile.cls / p.sw + p.sh * tile.h; xo = tile.cls % p.sw + p.sw * (tile.w0 + tw_); }
+      else {
+        const int ch = (int)fdiv((unsigned)tile.cls, p.sw, p.m_sw);
+        yo = ch + p.sh * tile.h; xo = tile.cls - ch * p.sw + p.sw * (tile.w0 + tw_);
+      }
       const int n = tile.n0 + tn;
       const bool row_ok = yo < p.Hd && xo < p.Wd && n < p.N;
       const uint32_t taddr = tmem + acc * p.BN + ((uint32_t)(32 * quad) << 16);
       const bool full_cols = tile.c0 + p.BN <= p.Cd;
       float* o_nchw = p.out + (((long long)n * p.Cd + tile.c0 + cbeg) * p.Hd + yo) * p.Wd + xo;
       float* o_hwnc = p.out + (((long long)yo * p.Wd + xo) * p.N + n) * p.Cd + tile.c0 + cbeg;
+      // one 16-column chunk at a time and no unrolling over chunks: this path serves the layouts the TMA-store
+      // epilogue cannot, and its code size matters more (instruction-cache misses stall every role) than its latency
+#pragma unroll 1
       for (int c = cbeg; c < cend; c += 16) {
         uint32_t v[16];
         if (Q > 0) {
@@ -160,13 +178,8 @@ __device__ __forceinline__ void epilogue_role(const ConvTcParams& p, uint32_t tm
         }
         if (row_ok && p.out_layout != 99) {
           if (p.out_layout == MQ_NCHW) {
-            if (full_cols) {
 #pragma unroll
-              for (int j = 0; j < 16; ++j) { *o_nchw = __uint_as_float(v[j]); o_nchw += cs; }
-            } else {
-#pragma unroll
-              for (int j = 0; j < 16; ++j) { if (tile.c0 + c + j < p.Cd) *o_nchw = __uint_as_float(v[j]); o_nchw += cs; }
-            }
+            for (int j = 0; j < 16; ++j) { if (full_cols || tile.c0 + c + j < p.Cd) *o_nchw = __uint_as_float(v[j]); o_nchw += cs; }
           } else {
             if (full_cols && (p.Cd & 3) == 0) {
 #pragma unroll
@@ -185,6 +198,79 @@ __device__ __forceinline__ void epilogue_role(const ConvTcParams& p, uint32_t tm
       __syncwarp();
       if (lane == 0) mbar_arrive(&tempty[acc]);
     }
+    if (lane == 0 && warp == 4) PROF_END(3);
+}
+
+// Epilogue role with TMA stores, NCHW output (warps 4-11).  Each warp moves its 32 rows x up to 64 channels on
+// its own: TMEM -> registers -> a private [channel][row] staging slice (row index fastest, so the writes are
+// conflict-free), then one lane stores the slice as a box of the output seen as (W, N, C, H): TW columns x
+// 32/TW samples x the channels.  The store engine clips the box at the tensor's edges and keeps the store
+// instructions out of the load/store pipe that the MMA issue shares.  The slice is reused only after the
+// previous tile's store has read it, which by then is long done.
+constexpr int EPI_STAGING_BYTES = 8 * 64 * 32 * 4;   // warps x [64 channels][32 rows] floats
+template <int MODE>
+__device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const CUtensorMap* map_out, float* staging, uint32_t tmem,
+                                                  uint64_t* tfull, uint64_t* tempty, volatile int* abort_flag, int warp, int lane, unsigned total) {
+    const int quad = warp & 3;
+    const int half = (warp - 4) >> 2;
+    const int cbeg = half == 0 ? 0 : ((p.BN / 2 + 15) & ~15);
+    const int cend = half == 0 ? ((p.BN / 2 + 15) & ~15) : p.BN;
+    float* buf = staging + (warp - 4) * (64 * 32);
+    const int n_off = quad * (32 >> p.lgTW);          // first sample of this warp's rows inside the tile
+    uint32_t tcount = 0;
+    PROF_BEGIN();
+    for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
+      const Tile tile = decode_tile(p, t);
+      TapWalk<MODE> tw;
+      tw.init(p, tile);
+      const int Q = tw.chunks(p);
+      const int acc = (int)(tcount & (uint32_t)(p.n_acc - 1));
+      bool ok = true;
+      if (lane == 0) ok = PROF_WAIT(mbar_wait(&tfull[acc], (tcount >> (p.n_acc - 1)) & 1, p.status, MQ_ERR_TIMEOUT));
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) { *abort_flag = 1; break; }
+      tc_fence_after_sync();
+      const int yo = MODE == MQ_OP_FWD ? tile.h : (int)fdiv((unsigned)tile.cls, p.sw, p.m_sw) + p.sh * tile.h;
+      const uint32_t taddr = tmem + acc * p.BN + ((uint32_t)(32 * quad) << 16);
+      if (cbeg >= cend) {      // a tile of 16 channels leaves the second half without columns
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tempty[acc]);
+      }
+#pragma unroll 1
+      for (int c0 = cbeg; c0 < cend; c0 += 64) {
+        const int nch = min(4, (cend - c0) >> 4);
+        if (lane == 0) bulk_wait_group_read<0>();      // the previous store has read the slice
+        __syncwarp();
+        // chunk by chunk, rolled: the hot loop stays small in the instruction cache
+#pragma unroll 1
+        for (int i = 0; i < nch; ++i) {
+          uint32_t v[16];
+          if (Q > 0) {
+            tmem_ld_32x32b_x16(taddr + c0 + 16 * i, v);
+            tmem_ld_wait();
+          } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) v[j] = 0u;
+          }
+          float* bi = buf + (16 * i) * 32 + lane;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) bi[j * 32] = __uint_as_float(v[j]);
+        }
+        if (c0 + 64 >= cend) {   // the accumulator has been read: hand it back before the store
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&tempty[acc]);
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0 && p.out_layout != 99) {
+          tma_store_4d(map_out, buf, tile.w0, tile.n0 + n_off, tile.c0 + c0, yo);
+          bulk_commit_group();
+        }
+      }
+    }
+    if (lane == 0) bulk_wait_group_all();
     if (lane == 0 && warp == 4) PROF_END(3);
 }
 
@@ -240,7 +326,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         ChunkPos pos;
         pos.reset();
         const uint8_t* sfa_src = p.sfa_img + (size_t)tile_m_index(p, tile) * p.max_stages * (512 * SPA);
-        const uint8_t* sfb_src = p.sfb_img + ((size_t)tile.cls * p.tiles_c + tile.c0 / p.BN) * p.max_stages * (512 * SPA * atoms_b);
+        const uint8_t* sfb_src = p.sfb_img + ((size_t)tile.cls * p.tiles_c + tile.ct) * p.max_stages * (512 * SPA * atoms_b);
         for (int q0 = 0; q0 < Q; q0 += G) {
           if (!PROF_WAIT(mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
           const int nch = min(G, Q - q0);
@@ -283,8 +369,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         TapWalk<MODE> tw;
         tw.init(p, tile);
         const int Q = tw.chunks(p);
-        const int acc = tcount % p.n_acc;
-        if (!PROF_WAIT(mbar_wait(&tempty[acc], ((tcount / p.n_acc) & 1) ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+        const int acc = (int)(tcount & (uint32_t)(p.n_acc - 1));
+        if (!PROF_WAIT(mbar_wait(&tempty[acc], ((tcount >> (p.n_acc - 1)) & 1) ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem + acc * p.BN;
         uint32_t accumulate = 0;
@@ -358,69 +444,113 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
 // ---- whole-tile-per-stage variant -------------------------------------------------------------------
 // For stride-1 layers whose tap has at most 64 bytes of channels (one chunk per tap), the per-tap TMA boxes
-// of the kernel above are tiny and their issue rate is the limit.  Here a pipeline stage holds the whole K
-// range of a tile: ONE TMA box brings the activation halo ([Kh rows][TW + Kw - 1 columns][TN samples][KB]) --
-// every stored pixel once, the data reuse of Sec. IV-A -- and ONE bulk copy brings all taps of the weight tile
-// (a pre-swizzled image written by the expansion kernel; per-row TMA requests of 32 bytes were the limit);
-// each tap's A operand is a shifted view of the halo (start = (row * WH * TN + column shift) * KB, 8-row
-// groups WH * KB bytes apart: TW = 8 output columns are exactly one 8-row swizzle group).  Two bulk copies
-// bring the tile's scale chunks.  Roles and barriers are those of conv_tc_kernel.
-template <int MODE, int KB, bool FP4>
+// of the kernel above are tiny and their issue rate is the limit.  Here
+//  * the weight tile (all taps, a pre-swizzled image written by the expansion kernel) and its scale chunks are
+//    RESIDENT: one bulk copy when the channel tile changes (never, when the layer has a single channel tile),
+//    its scale vectors copied to TMEM once;
+//  * a pipeline stage holds the whole K range of a tile's activations, every stored pixel once (the data reuse
+//    of Sec. IV-A), and each tap's A operand is a view into it.  Two shapes:
+//      nbox == 1  one TMA box [Kh rows][TN samples][TW + Kw - 1 columns][KB]; tap (kh, kw) starts at
+//                 (kh * TN * WH + kw) * KB with 8-row groups WH * KB bytes apart (TW = 8: one 8-row swizzle
+//                 group per sample);
+//      nbox == Kw one box [Kh][TN][TW][KB] per column shift (TW = 8, 16 or 32); tap (kh, kw) is the plain
+//                 128-row operand at ((kw * Kh + kh) * 128) * KB.  Longer runs of output columns per warp for
+//                 an NCHW store, at Kw times the shared-memory footprint.
+// Roles and barriers are those of conv_tc_kernel, plus bfull / bempty for the resident weight tile.
+// TAPS > 0 fixes the tap count at compile time (the MMA issue loop is then fully unrolled with the tap offsets in
+// registers: the single issuing thread is latency-bound, every instruction between two MMAs counts); 0 = any.
+template <int MODE, int KB, bool FP4, int TAPS>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const ConvTcParams p) {
+conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_out, const ConvTcParams p) {
   constexpr int G = 128 / KB, APC = KB / 32, SPA = FP4 ? 2 : 1;
   constexpr int LAYOUT = KB == 128 ? 2 : (KB == 64 ? 4 : 6);
+#ifdef MQ_TC_PROFILE
+  unsigned long long gt0 = 0;
+  if (threadIdx.x == 0) asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt0));
+#endif
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-  const int taps = p.Kh * p.Kw;
+  const int taps = TAPS > 0 ? TAPS : p.Kh * p.Kw;
   const int nsf = p.max_stages;                        // scale chunks (groups of 4 MMAs) per tile
   const int atoms_b = (p.BN + 127) / 128;
   const int b_bytes = taps * p.BN * KB;
   const int sfa_bytes = nsf * 512 * SPA, sfb_bytes = nsf * 512 * SPA * atoms_b;
   const int stage_bytes = p.halo_stage_bytes;
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * stage_bytes);
+  uint8_t* stage0 = smem + p.halo_b_bytes;             // [weight image | its scale chunks] then the stages
+  float* staging = reinterpret_cast<float*>(stage0 + (size_t)p.stages * stage_bytes);   // TMA-store epilogue only
+  uint64_t* full = reinterpret_cast<uint64_t*>(stage0 + (size_t)p.stages * stage_bytes + (p.tma_store ? EPI_STAGING_BYTES : 0));
   uint64_t* empty = full + p.stages;
   uint64_t* sffull = empty + p.stages;
   uint64_t* tfull = sffull + p.stages;
   uint64_t* tempty = tfull + 2;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
+  uint64_t* bfull = tempty + 2;
+  uint64_t* bempty = bfull + 1;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bempty + 1);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  uint32_t* tap_a = tmem_slot + 4;                     // per tap: offset of its A view / B rows, in 16-byte units
+  uint32_t* tap_b = tap_a + 64;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const unsigned total = (unsigned)p.total_tiles;
+  const unsigned tiles_per_c = (unsigned)(p.classes * p.tiles_w * p.tiles_h);   // tile order: (class, w, h) below the channel tile
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 8); }
+    mbar_init(bfull, 1); mbar_init(bempty, 1);
     *abort_flag = 0;
     mbar_fence_init();
     prefetch_tensormap(&map_a);
-    prefetch_tensormap(&map_b);
+    if (p.tma_store) prefetch_tensormap(&map_out);
+  }
+  if ((int)threadIdx.x < taps) {
+    const int kh = threadIdx.x / p.Kw, kw = threadIdx.x - kh * p.Kw;
+    // forward reads halo row kh, column shift kw; the input gradient walks the taps in the same order but its
+    // source pixel moves the other way
+    const int hrow = MODE == MQ_OP_FWD ? kh : p.Kh - 1 - kh, wsh = MODE == MQ_OP_FWD ? kw : p.Kw - 1 - kw;
+    const int aoff = p.nbox == 1 ? (hrow * p.TN * p.WH + wsh) * KB : (wsh * p.Kh + hrow) * 128 * KB;
+    tap_a[threadIdx.x] = (uint32_t)aoff >> 4;
+    tap_b[threadIdx.x] = (uint32_t)(threadIdx.x * p.BN * KB) >> 4;
   }
   if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
-  const uint32_t sf_cols_stage = (uint32_t)nsf * SF_COLS;
+#ifdef MQ_TC_PROFILE
+  unsigned long long gt1 = 0;
+  if (threadIdx.x == 0) asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt1));
+#endif
+  // TMEM columns: accumulators, the resident weight scale vectors (16 per chunk), then 8 per chunk per stage
+  const uint32_t sfb_base = tmem + p.n_acc * p.BN;
+  const uint32_t sfa_base = sfb_base + (uint32_t)nsf * 16;
+  const uint32_t sfa_cols_stage = (uint32_t)nsf * 8;
 
   if (warp == 0) {
-    // ------------------------------------------------------------------ producer: 2 TMA boxes + 2 bulk copies per tile
+    // ------------------------------------------------------------------ producer
     if (lane == 0) {
-      uint32_t s = 0, phase = 0;
+      uint32_t s = 0, phase = 0, bcount = 0;
+      int cur_ct = -1;
       PROF_BEGIN();
       for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x) {
         const Tile tile = decode_tile(p, t);
+        const int ct = tile.ct;
+        if (ct != cur_ct) {
+          // new weight tile: wait until the MMAs of the previous one have retired, then one copy of image + scales
+          if (bcount > 0 && !PROF_WAIT(mbar_wait(bempty, (bcount - 1) & 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+          mbar_arrive_expect_tx(bfull, (uint32_t)(b_bytes + sfb_bytes));
+          bulk_load(smem, p.b_img + (size_t)ct * b_bytes, b_bytes, bfull);
+          bulk_load(smem + b_bytes, p.sfb_img + ((size_t)tile.cls * p.tiles_c + ct) * sfb_bytes, sfb_bytes, bfull);
+          cur_ct = ct; ++bcount;
+        }
         if (!PROF_WAIT(mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
-        uint8_t* sa = smem + (size_t)s * stage_bytes;
-        uint8_t* sb = sa + p.halo_a_bytes;
+        uint8_t* sa = stage0 + (size_t)s * stage_bytes;
         // first source pixel of the halo: forward (h - ph, w0 - pw); input gradient (h + ph - (Kh-1), w0 + pw - (Kw-1))
         const int hs = MODE == MQ_OP_FWD ? tile.h - p.ph : tile.h + p.ph - (p.Kh - 1);
         const int ws = MODE == MQ_OP_FWD ? tile.w0 - p.pw : tile.w0 + p.pw - (p.Kw - 1);
-        mbar_arrive_expect_tx(&full[s], (uint32_t)(p.Kh * p.WH * p.TN * KB + b_bytes + sfa_bytes + sfb_bytes));
-        tma_load_4d(sa, &map_a, &full[s], 0, ws, tile.n0, hs);
-        bulk_load(sb, p.b_img + (size_t)(tile.c0 / p.BN) * b_bytes, b_bytes, &full[s]);   // all taps, already swizzled
-        bulk_load(sb + b_bytes, p.sfa_img + (size_t)tile_m_index(p, tile) * sfa_bytes, sfa_bytes, &full[s]);
-        bulk_load(sb + b_bytes + sfa_bytes, p.sfb_img + ((size_t)tile.cls * p.tiles_c + tile.c0 / p.BN) * sfb_bytes, sfb_bytes, &full[s]);
+        mbar_arrive_expect_tx(&full[s], (uint32_t)(p.nbox * p.halo_box_bytes + sfa_bytes));
+#pragma unroll 1
+        for (int b = 0; b < p.nbox; ++b) tma_load_4d(sa + (size_t)b * p.halo_box_bytes, &map_a, &full[s], 0, ws + b, tile.n0, hs);
+        bulk_load(sa + p.halo_a_bytes, p.sfa_img + (size_t)tile_m_index(p, tile) * sfa_bytes, sfa_bytes, &full[s]);
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
       PROF_END(0);
@@ -428,72 +558,100 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer: all taps of a tile per stage
     if (lane == 0) {
-      const uint64_t a_desc_base = smem_desc_base(16, (uint32_t)(p.WH * KB), LAYOUT);   // 8-row groups WH pixels apart
+      const uint64_t a_desc_base = smem_desc_base(16, (uint32_t)((p.nbox == 1 ? p.WH : 8) * KB), LAYOUT);
       const uint64_t b_desc_base = smem_desc_base(16, 8 * KB, LAYOUT);
-      const uint32_t sf_base = tmem + p.n_acc * p.BN;
+      const uint32_t sb16 = smem_u32(smem) >> 4;
       uint32_t idesc_id[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) idesc_id[i] = idesc_with_sf_ids(p.idesc, i, i);
-      uint32_t s = 0, phase = 0, tcount = 0;
+      uint32_t s = 0, phase = 0, tcount = 0, bcount = 0;
+      int cur_ct = -1;
+      constexpr int TU = TAPS > 0 ? TAPS : 1;
+      uint32_t ta[TU], tb[TU];
+#pragma unroll
+      for (int q = 0; q < TU; ++q) { ta[q] = tap_a[q]; tb[q] = tap_b[q]; }
+      const uint32_t acc_mask = (uint32_t)p.n_acc - 1, acc_shift = (uint32_t)p.n_acc - 1;   // n_acc is 1 or 2
       PROF_BEGIN();
       for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
-        const int acc = tcount % p.n_acc;
-        if (!PROF_WAIT(mbar_wait(&tempty[acc], ((tcount / p.n_acc) & 1) ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+        const int ct = p.tiles_c == 1 ? 0 : (int)((t / tiles_per_c) % (unsigned)p.tiles_c);
+        if (ct != cur_ct) {
+          if (!PROF_WAIT(mbar_wait(bfull, bcount & 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+          cur_ct = ct; ++bcount;
+        }
+        const int acc = (int)(tcount & acc_mask);
+        if (!PROF_WAIT(mbar_wait(&tempty[acc], ((tcount >> acc_shift) & 1) ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
         if (!PROF_WAIT(mbar_wait(&sffull[s], phase, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem + acc * p.BN;
-        const uint32_t sa = smem_u32(smem + (size_t)s * stage_bytes);
-        const uint32_t sb = sa + p.halo_a_bytes;
-        const uint32_t sf_t = sf_base + s * sf_cols_stage;
+        const uint32_t sa16 = smem_u32(stage0 + (size_t)s * stage_bytes) >> 4;
+        const uint32_t sfa_s = sfa_base + s * sfa_cols_stage;
         uint32_t accumulate = 0;
-        int q = 0;
-        for (int kh = 0; kh < p.Kh; ++kh)
-          for (int kw = 0; kw < p.Kw; ++kw, ++q) {
-            // tap q of the walk: forward reads halo row kh, column shift kw; the input gradient walks the taps in
-            // the same (kh, kw) order but its source pixel moves the other way
-            const int hrow = MODE == MQ_OP_FWD ? kh : p.Kh - 1 - kh, wsh = MODE == MQ_OP_FWD ? kw : p.Kw - 1 - kw;
-            const uint32_t a_addr = sa + (uint32_t)((hrow * p.WH * p.TN + wsh) * KB);
-            const uint32_t b_addr = sb + (uint32_t)((kh * p.Kw + kw) * p.BN * KB);
-            const int sfst = q / G;
-            const uint32_t sfa_t = sf_t + sfst * SF_COLS, sfb_t = sfa_t + 8;
+        const long long pc0 = PROF_CLK();
+        auto issue_tap = [&](int q, uint32_t a16, uint32_t b16) {
+          const int sfst = q / G;
+          const uint32_t sfa_t = sfa_s + sfst * 8, sfb_t = sfb_base + sfst * 16;
 #pragma unroll
-            for (int ja = 0; ja < APC; ++ja) {
-              const int atom = (q % G) * APC + ja;
-              const int g = (atom * SPA) >> 2, id = (atom * SPA) & 3;
-              const uint64_t ad = smem_desc(a_desc_base, a_addr + ja * 32);
-              const uint64_t bd = smem_desc(b_desc_base, b_addr + ja * 32);
-              if (FP4) mma_mxf4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accumulate);
-              else mma_mxf8f6f4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accumulate);
-              accumulate = 1;
-            }
+          for (int ja = 0; ja < APC; ++ja) {
+            const int atom = (q % G) * APC + ja;
+            const int g = (atom * SPA) >> 2, id = (atom * SPA) & 3;
+            const uint64_t ad = a_desc_base | (uint64_t)((a16 + 2 * ja) & 0x3FFF);
+            const uint64_t bd = b_desc_base | (uint64_t)((b16 + 2 * ja) & 0x3FFF);
+            if (FP4) mma_mxf4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accumulate);
+            else mma_mxf8f6f4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accumulate);
+            accumulate = 1;
           }
+        };
+        if (TAPS > 0) {
+#pragma unroll
+          for (int q = 0; q < TU; ++q) issue_tap(q, sa16 + ta[q], sb16 + tb[q]);
+        } else {
+#pragma unroll 1
+          for (int q = 0; q < taps; ++q) issue_tap(q, sa16 + tap_a[q], sb16 + tap_b[q]);
+        }
+        const long long pc1 = PROF_CLK();
         tc_commit(&empty[s]);
         tc_commit(&tfull[acc]);
+        PROF_ADD(4, 1, pc1 - pc0);
+        if (p.tiles_c > 1) {
+          const unsigned tn_ = t + gridDim.x;   // the block's next tile: release the weight tile if it needs another
+          if (tn_ < total && (int)((tn_ / tiles_per_c) % (unsigned)p.tiles_c) != ct) tc_commit(bempty);
+        }
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
       PROF_END(1);
     }
   } else if (warp == 2) {
-    // ------------------------------------------------------------------ scale copier: the tile's chunks smem -> TMEM
+    // ------------------------------------------------------------------ scale copier: chunks smem -> TMEM
     if (lane == 0) {
       const uint64_t sf_desc = smem_desc_base(0, 128, 0);
-      const uint32_t sf_base = tmem + p.n_acc * p.BN;
-      uint32_t s = 0, phase = 0;
+      uint32_t s = 0, phase = 0, bcount = 0;
+      int cur_ct = -1;
       PROF_BEGIN();
       for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x) {
+        const int ct = p.tiles_c == 1 ? 0 : (int)((t / tiles_per_c) % (unsigned)p.tiles_c);
+        const bool new_b = ct != cur_ct;
+        if (new_b) {
+          if (!PROF_WAIT(mbar_wait(bfull, bcount & 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+          cur_ct = ct; ++bcount;
+        }
         if (!PROF_WAIT(mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
         tc_fence_after_sync();
-        const uint32_t sfa_s = smem_u32(smem + (size_t)s * stage_bytes + p.halo_a_bytes + b_bytes);
-        const uint32_t sfb_s = sfa_s + sfa_bytes;
-        const uint32_t sf_t = sf_base + s * sf_cols_stage;
-        for (int st = 0; st < nsf; ++st) {
-          const uint32_t sfa_t = sf_t + st * SF_COLS, sfb_t = sfa_t + 8;
+        if (new_b) {
+          const uint32_t sfb_s = smem_u32(smem + b_bytes);
+#pragma unroll 1
+          for (int st = 0; st < nsf; ++st)
 #pragma unroll
-          for (int g = 0; g < SPA; ++g) {
-            tmem_cp_32x128b_warpx4(sfa_t + 4 * g, smem_desc(sf_desc, sfa_s + (st * SPA + g) * 512));
-            for (int a = 0; a < atoms_b; ++a)
-              tmem_cp_32x128b_warpx4(sfb_t + 4 * (g * atoms_b + a), smem_desc(sf_desc, sfb_s + ((st * SPA + g) * atoms_b + a) * 512));
-          }
+            for (int g = 0; g < SPA; ++g)
+#pragma unroll 1
+              for (int a = 0; a < atoms_b; ++a)
+                tmem_cp_32x128b_warpx4(sfb_base + st * 16 + 4 * (g * atoms_b + a), smem_desc(sf_desc, sfb_s + ((st * SPA + g) * atoms_b + a) * 512));
+        }
+        const uint32_t sfa_sm = smem_u32(stage0 + (size_t)s * stage_bytes + p.halo_a_bytes);
+        const uint32_t sfa_s = sfa_base + s * sfa_cols_stage;
+#pragma unroll 1
+        for (int st = 0; st < nsf; ++st) {
+#pragma unroll
+          for (int g = 0; g < SPA; ++g) tmem_cp_32x128b_warpx4(sfa_s + st * 8 + 4 * g, smem_desc(sf_desc, sfa_sm + (st * SPA + g) * 512));
         }
         tc_commit(&sffull[s]);
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
@@ -501,11 +659,21 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       PROF_END(2);
     }
   } else if (warp >= 4) {
-    epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
+    if (p.tma_store) epilogue_tma_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total);
+    else epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
   }
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem, 512);
+#ifdef MQ_TC_PROFILE
+  if (threadIdx.x == 0) {
+    unsigned long long gt2; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt2));
+    if (blockIdx.x < 160) {
+      unsigned smid; asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
+      g_blk[blockIdx.x][0] = smid; g_blk[blockIdx.x][1] = gt0; g_blk[blockIdx.x][2] = gt1; g_blk[blockIdx.x][3] = gt2;
+    }
+  }
+#endif
 }
 
 // ---- scale expansion --------------------------------------------------------------------------------
@@ -588,7 +756,7 @@ __global__ void __launch_bounds__(256) expand_conv_scales_kernel(const ConvTcPar
     const int st = (int)(idx % (unsigned)p.max_stages); idx /= (unsigned)p.max_stages;
     const int ct = (int)(idx % (unsigned)p.tiles_c);
     Tile tile;
-    tile.cls = (int)(idx / (unsigned)p.tiles_c); tile.c0 = ct * p.BN; tile.w0 = 0; tile.n0 = 0; tile.h = 0;
+    tile.cls = (int)(idx / (unsigned)p.tiles_c); tile.ct = ct; tile.c0 = ct * p.BN; tile.w0 = 0; tile.n0 = 0; tile.h = 0;
     TapWalk<MODE> tw;
     tw.init(p, tile);
     const int Q = tw.chunks(p);
@@ -682,12 +850,23 @@ EncodeTiledFn get_encoder() {
 
 }  // namespace
 
-extern "C" int mqdbg_read_prof(unsigned long long* out16) {
-  return cudaMemcpyFromSymbol(out16, g_prof, sizeof(unsigned long long) * 16) == cudaSuccess ? 0 : 1;
+#ifdef MQ_TC_PROFILE
+extern "C" int mqdbg_read_role(unsigned long long* out1280) {
+  return cudaMemcpyFromSymbol(out1280, g_role, sizeof(unsigned long long) * 1280) == cudaSuccess ? 0 : 1;
 }
+extern "C" int mqdbg_read_blk(unsigned long long* out640) {
+  return cudaMemcpyFromSymbol(out640, g_blk, sizeof(unsigned long long) * 640) == cudaSuccess ? 0 : 1;
+}
+extern "C" int mqdbg_read_prof(unsigned long long* out16) {
+  if (cudaMemcpyFromSymbol(out16, g_prof, sizeof(unsigned long long) * 16) != cudaSuccess) return 1;
+  unsigned long long z[16] = {0};
+  z[12] = ~0ull;
+  return cudaMemcpyToSymbol(g_prof, z, sizeof(z)) == cudaSuccess ? 0 : 1;
+}
+#endif
 
 bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes, const uint32_t* box,
-                          const uint32_t* elem_strides, int swizzle_bytes) {
+                          const uint32_t* elem_strides, int swizzle_bytes, bool f32) {
   EncodeTiledFn fn = get_encoder();
   if (!fn) return false;
   cuuint64_t d[5], st[4];
@@ -697,7 +876,7 @@ bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const ui
   CUtensorMapSwizzle sw = swizzle_bytes == 128 ? CU_TENSOR_MAP_SWIZZLE_128B
                         : swizzle_bytes == 64  ? CU_TENSOR_MAP_SWIZZLE_64B
                         : swizzle_bytes == 32  ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE;
-  CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
+  CUresult r = fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
                   CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
@@ -753,12 +932,13 @@ cudaError_t launch_expand_conv_scales(const ConvTcParams& p, cudaStream_t s) {
   return cudaErrorInvalidValue;
 }
 
-template <int MODE, int KB, bool FP4>
-cudaError_t launch_conv_tc_halo_inst(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s) {
+template <int MODE, int KB, bool FP4, int TAPS>
+cudaError_t launch_conv_tc_halo_taps(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s) {
   static bool attr_set = false;
-  const size_t smem = 1024 + (size_t)p.stages * p.halo_stage_bytes + (3 * (size_t)p.stages + 4) * 8 + 64;
+  const size_t smem = 1024 + (size_t)p.halo_b_bytes + (size_t)p.stages * p.halo_stage_bytes + (p.tma_store ? EPI_STAGING_BYTES : 0) +
+                      (3 * (size_t)p.stages + 6) * 8 + 16 + 2 * 64 * 4;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(conv_tc_halo_kernel<MODE, KB, FP4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(conv_tc_halo_kernel<MODE, KB, FP4, TAPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -766,9 +946,14 @@ cudaError_t launch_conv_tc_halo_inst(const ConvTcParams& p, const CUtensorMap& m
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const unsigned grid = (unsigned)(p.total_tiles < sms ? p.total_tiles : sms);
-  conv_tc_halo_kernel<MODE, KB, FP4><<<grid, TC_THREADS, smem, s>>>(map_a, map_b, p);
+  conv_tc_halo_kernel<MODE, KB, FP4, TAPS><<<grid, TC_THREADS, smem, s>>>(map_a, map_b, p);
   count_launches(1);
   return cudaGetLastError();
+}
+template <int MODE, int KB, bool FP4>
+cudaError_t launch_conv_tc_halo_inst(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s) {
+  if (p.Kh * p.Kw == 9) return launch_conv_tc_halo_taps<MODE, KB, FP4, 9>(p, map_a, map_b, s);
+  return launch_conv_tc_halo_taps<MODE, KB, FP4, 0>(p, map_a, map_b, s);
 }
 
 cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s) {

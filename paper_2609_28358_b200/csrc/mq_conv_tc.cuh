@@ -23,7 +23,7 @@ struct ConvTcParams {
   int BN;               // output channels per tile (multiple of 16, <= 256)
   int stages;
   int n_acc;            // accumulator buffers in TMEM (1 or 2)
-  int TW, TN, lgTW;     // tile = TW output columns x TN samples (TW * TN = 128), TW fastest among rows
+  int TW, TN, lgTW, lgTN;  // tile = TW output columns x TN samples (TW * TN = 128), TW fastest among rows
   // geometry
   int N, Nt;
   int Hs, Ws;           // spatial extent of the gathered source (fwd: H, W; bwd_data: Ho, Wo)
@@ -34,6 +34,7 @@ struct ConvTcParams {
   // tiles
   int tiles_c, tiles_w, tiles_n, tiles_h, classes;  // classes = sh*sw parity classes (bwd_data), else 1
   long long total_tiles;
+  uint32_t m_classes, m_tiles_w, m_tiles_h, m_tiles_c, m_sh, m_sw;   // ceil(2^32 / d) for the divisions by these (0: divide)
   // scales
   const uint8_t* a_scales;  // [Hs][Ws][Nt][Kblocks]
   const uint8_t* b_scales;  // [row blocks of 32][taps][Kblocks]
@@ -43,9 +44,13 @@ struct ConvTcParams {
   int max_stages;           // stages of the longest tile
   // whole-tile-per-stage variant (small channel counts, stride 1): see conv_tc_halo_kernel
   int halo;                 // 1: use it
-  int WH;                   // halo width in pixels = TW + Kw - 1
-  int halo_a_bytes;         // bytes of the activation halo of a tile (rounded up to 1024)
-  int halo_stage_bytes;     // bytes of one pipeline stage (halo + all taps of B + scale chunks)
+  int nbox;                 // activation boxes per tile: 1 (one box with the column halo) or Kw (one box per column shift)
+  int WH;                   // columns per box: TW + Kw - 1 (nbox == 1) or TW
+  int halo_box_bytes;       // bytes of one activation box = Kh * TN * WH * KB
+  int halo_a_bytes;         // bytes of a tile's activation boxes (rounded up to 1024)
+  int halo_stage_bytes;     // bytes of one pipeline stage (activation boxes + A-side scale chunks)
+  int halo_b_bytes;         // bytes of the resident weight image + its scale chunks (rounded up to 1024)
+  int tma_store;            // 1: NCHW output written by TMA stores from a staging buffer (the second tensor map is the output's)
   const uint8_t* b_codes;   // weight-like codes [rows][taps][b_rowbytes] (source of the images below)
   int b_rows_total, b_rowbytes;
   uint8_t* b_img;           // [channel tile][tap][BN rows][KB], each row stored with the KB-byte swizzle applied
@@ -107,8 +112,9 @@ cudaError_t launch_fp4_to_flat(const uint8_t* in, uint8_t* out, int Hs, int Ws, 
 // Adds the split partial sums in a fixed order and writes G_W in its final layout.
 cudaError_t launch_bwd_weight_reduce(const float* partial, float* out, const Geom& g, int splits, int layout, cudaStream_t s);
 
-// Host: encode a tiled tensor map over bytes.  dims / strides in bytes (stride[0] implied 1), fastest first.
+// Host: encode a tiled tensor map over bytes (or over fp32 elements when f32 is set: dims and box then count
+// elements).  Strides in bytes (stride[0] implied contiguous), fastest dimension first.
 bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-                          const uint32_t* box, const uint32_t* elem_strides, int swizzle_bytes);
+                          const uint32_t* box, const uint32_t* elem_strides, int swizzle_bytes, bool f32 = false);
 
 }  // namespace mq
