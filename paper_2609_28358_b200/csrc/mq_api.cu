@@ -192,6 +192,7 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
       while (hst >= 2 && p.BN + 16 * p.max_stages + 8 * p.max_stages * hst > 512) --hst;
       if (hst >= 2 && p.WH <= 256 && (p.halo_box_bytes % 1024 == 0 || nbox == 1)) {
         p.halo = 1;
+        p.fused = p.tiles_c == 1 && p.TN <= 32 && g.Kh * (p.TW + g.Kw - 1) * (p.KB / 32) * spa <= 128 && !env_int("MQ_TC_NO_FUSED", 0);
         p.stages = hst;
         p.n_acc = (2 * p.BN + 16 * p.max_stages + 8 * p.max_stages * hst <= 512) ? 2 : 1;
       }
@@ -241,9 +242,9 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
   p.sfb_img = base + pl.off_sfb;
   p.b_codes = b_codes; p.b_rows_total = pl.rows_b; p.b_rowbytes = pl.rowbytes; p.b_img = base + pl.off_bimg;
   p.out = out; p.out_layout = env_int("MQ_TC_SKIP_STORE", 0) ? 99 : layout; p.status = status;
-  if (launch_expand_conv_scales(p, stream) != cudaSuccess) return MQ_ERR_CUDA;
+  if (!(p.halo && p.fused) && launch_expand_conv_scales(p, stream) != cudaSuccess) return MQ_ERR_CUDA;
 
-  CUtensorMap map_a, map_b;
+  CUtensorMap map_a, map_b, map_w;
   {
     const uint64_t rb = (uint64_t)pl.rowbytes;
     const uint64_t dims[4] = {rb, (uint64_t)p.Ws, (uint64_t)g.N, (uint64_t)p.Hs};
@@ -253,6 +254,15 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
     if (p.halo) { box[1] = (uint32_t)p.WH; box[3] = (uint32_t)g.Kh; }   // the whole halo of a tile in one box
     const uint32_t es[4] = {1u, wst, 1u, 1u};
     if (!encode_tensor_map_u8(&map_a, qx_like->codes, 4, dims, strides, box, es, p.KB)) return MQ_ERR_CUDA;
+  }
+  map_w = map_a;
+  if (p.halo && p.fused) {
+    // all taps of the weight tile in one box: dims ordered (channel bytes, rows, taps)
+    const uint64_t rb = (uint64_t)pl.rowbytes;
+    const uint64_t dims[3] = {rb, (uint64_t)pl.rows_b, (uint64_t)taps};
+    const uint64_t strides[2] = {(uint64_t)taps * rb, rb};
+    const uint32_t box[3] = {(uint32_t)p.KB, (uint32_t)p.BN, (uint32_t)taps};
+    if (!encode_tensor_map_u8(&map_w, b_codes, 3, dims, strides, box, nullptr, p.KB)) return MQ_ERR_CUDA;
   }
   if (p.halo) {
     map_b = map_a;   // the weight tile comes as a pre-swizzled image by bulk copy; the second map is the output's
@@ -274,7 +284,7 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
     const uint32_t box[3] = {(uint32_t)p.KB, 1u, (uint32_t)p.BN};
     if (!encode_tensor_map_u8(&map_b, b_codes, 3, dims, strides, box, nullptr, p.KB)) return MQ_ERR_CUDA;
   }
-  return launch_conv_tc(p, map_a, map_b, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
+  return launch_conv_tc(p, map_a, map_b, map_w, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }
 
 // ---- weight gradient on tensor cores ---------------------------------------------------------------
@@ -309,20 +319,36 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   p.b_rows = flat ? (g.Cp < 128 ? g.Cp : 128) : 128;
   p.m_tiles = (g.Cout + 127) / 128;
   p.cb_tiles = (g.Cp + p.b_rows - 1) / p.b_rows;
-  p.j_tiles = g.Kh * g.Kw * p.cb_tiles;
+  // taps per block: a whole kernel row in the flat mode when its accumulators fit in tensor memory
+  p.TG = 1;
+  if (flat && g.Kw > 1 && g.Kw * p.b_rows + 2 * (8 + 8 * ((g.Kw * p.b_rows + 127) / 128)) <= 512 && !env_int("MQ_WGRAD_NO_GROUP", 0)) p.TG = g.Kw;
+  p.NB = (p.TG * p.b_rows + 127) / 128;
+  p.n0 = p.TG * p.b_rows < 256 ? p.TG * p.b_rows : 256;
+  p.n1 = p.TG * p.b_rows - p.n0;
+  p.j_tiles = (g.Kh * g.Kw / p.TG) * p.cb_tiles;
   const int items = p.m_tiles * p.j_tiles;
   int splits = env_int("MQ_WGRAD_SPLITS", 0);
   if (splits <= 0) splits = items >= 148 ? 1 : 148 / items;
   if (splits > p.stages_total) splits = p.stages_total;
   if (splits < 1) splits = 1;
   p.splits = splits;
-  p.stages = 6;
+  p.b_tile_bytes = flat ? (p.KPX + p.TG - 1) * p.b_rows * p.KBn : p.b_rows * 128;
+  p.stage_bytes = (128 * 128 + p.b_tile_bytes + (1 + p.NB) * 1024 + 1023) / 1024 * 1024;
+  {
+    int st = (227 * 1024 - 2048) / p.stage_bytes;
+    if (st > 6) st = 6;
+    while (st > 2 && p.TG * p.b_rows + st * (8 + 8 * p.NB) > 512) --st;
+    p.stages = st;
+    const int cols = p.TG * p.b_rows + st * (8 + 8 * p.NB);
+    p.tmem_cols = cols <= 256 ? 256 : 512;
+    if (st < 2 || cols > 512) return w;
+  }
   const int spa = fp4 ? 2 : 1;
   w.P_a = p.stages_total * p.KPX;
   w.P_b = (w.P_a + (g.Kh - 1) * p.Wp + g.Kw - 1 + 7) / 8 * 8;
   size_t o = up256((size_t)splits * g.Cout * g.Kh * g.Kw * g.Cp * sizeof(float));
   w.off_sfa = o; o += up256((size_t)p.m_tiles * p.stages_total * 512 * spa);
-  w.off_sfb = o; o += up256((size_t)p.cb_tiles * g.Kh * g.Kw * p.stages_total * 512 * spa);
+  w.off_sfb = o; o += up256((size_t)p.cb_tiles * (g.Kh * g.Kw / p.TG) * p.stages_total * p.NB * 512 * spa);
   w.off_xt = o;
   if (flat) { p.xt_block_bytes = (long long)w.P_b * p.b_rows * p.KBn; o += up256((size_t)p.cb_tiles * p.xt_block_bytes); }
   else if (fp4) o += up256((size_t)g.Cp * g.H * g.W * w.Npad / 2);
@@ -348,11 +374,11 @@ mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const 
     if (launch_fp4_to_flat(static_cast<const uint8_t*>(qx->codes), xt, g.H, g.W, g.N, g.Cp, w.P_b, p.Wp, g.ph, g.pw, p.b_rows, p.cb_tiles, p.KBn, stream) != cudaSuccess) return MQ_ERR_CUDA;
     if (launch_fp4_to_flat(static_cast<const uint8_t*>(qg->codes), gt, g.Ho, g.Wo, g.N, g.Cop, w.P_a, p.Wp, 0, 0, 128, p.m_tiles, p.KBn, stream) != cudaSuccess) return MQ_ERR_CUDA;
     p.xt = xt; p.gt = gt;
-    p.idesc = (1u << 7) | (1u << 10) | ((uint32_t)(p.b_rows >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
+    p.idesc = (1u << 7) | (1u << 10) | (1u << 23) | ((128u >> 4) << 24);
   } else if (p.mode == MQ_WG_FP4_PIXEL) {
     if (launch_fp4_to_n_major(static_cast<const uint8_t*>(qx->codes), xt, g.H * g.W, g.N, g.Cp, w.Npad, stream) != cudaSuccess) return MQ_ERR_CUDA;
     if (launch_fp4_to_n_major(static_cast<const uint8_t*>(qg->codes), gt, g.Ho * g.Wo, g.N, g.Cop, w.Npad, stream) != cudaSuccess) return MQ_ERR_CUDA;
-    p.idesc = (1u << 7) | (1u << 10) | ((128u >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
+    p.idesc = (1u << 7) | (1u << 10) | (1u << 23) | ((128u >> 4) << 24);
     const uint64_t nb = (uint64_t)w.Npad / 2;
     const int swz = p.KBn >= 32 ? p.KBn : 0;
     {
@@ -369,7 +395,7 @@ mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const 
     }
   } else {
     const uint32_t fa = qg->fmt == MQ_E5M2 ? 1u : 0u, fb = qx->fmt == MQ_E5M2 ? 1u : 0u;
-    p.idesc = (fa << 7) | (fb << 10) | (1u << 15) | (1u << 16) | ((128u >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
+    p.idesc = (fa << 7) | (fb << 10) | (1u << 15) | (1u << 16) | (1u << 23) | ((128u >> 4) << 24);
     {
       const uint64_t rb = (uint64_t)g.Cop;
       const uint64_t dims[4] = {rb, (uint64_t)g.N, (uint64_t)g.Wo, (uint64_t)g.Ho};

@@ -225,19 +225,46 @@ __global__ void __launch_bounds__(GT) bwd_weight_generic(ConvArgs a, int splits)
   }
 }
 
-__global__ void bwd_weight_reduce(const float* __restrict__ part, float* __restrict__ out, Geom g, int splits, int layout) {
+// Adds the split-K partial sums [split][Cout][taps][Cp] in a fixed order and writes G_W in its final layout.
+// The reads are `splits` times the writes, so threads follow the partials' own order (4 consecutive input
+// channels per thread, 16-byte loads); a block's four thread groups take every fourth split each and are
+// combined through shared memory in group order, so the result does not depend on scheduling.
+__global__ void __launch_bounds__(256) bwd_weight_reduce(const float* __restrict__ part, float* __restrict__ out, Geom g, int splits, int layout) {
+  __shared__ float4 sh[3][64];
   const int taps = g.Kh * g.Kw;
-  const long long total = (long long)g.Cout * taps * g.Cin;
-  const long long J = (long long)taps * g.Cp;
-  for (long long i = (long long)blockIdx.x * blockDim.x + threadIdx.x; i < total; i += (long long)gridDim.x * blockDim.x) {
-    // i enumerates the output in its own layout so that writes are coalesced
-    int co, ci, tap;
-    if (layout == MQ_NCHW) { tap = (int)(i % taps); long long q = i / taps; ci = (int)(q % g.Cin); co = (int)(q / g.Cin); }
-    else { ci = (int)(i % g.Cin); long long q = i / g.Cin; tap = (int)(q % taps); co = (int)(q / taps); }
-    const float* p = part + (long long)co * J + (long long)tap * g.Cp + ci;
-    float s = 0.f;
-    for (int k = 0; k < splits; ++k) s += p[(long long)k * g.Cout * J];
-    out[i] = s;
+  const int cq = g.Cp >> 2;                                   // float4 columns per (co, tap)
+  const long long quads = (long long)g.Cout * taps * cq;
+  const long long slab = (long long)g.Cout * taps * g.Cp;     // floats per split
+  const int col = threadIdx.x & 63, grp = threadIdx.x >> 6;
+  for (long long base = (long long)blockIdx.x * 64; base < quads; base += (long long)gridDim.x * 64) {
+    const long long qd = base + col;
+    float4 s = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (qd < quads) {
+      const float4* p = reinterpret_cast<const float4*>(part) + qd;
+#pragma unroll 4
+      for (int k = grp; k < splits; k += 4) {
+        const float4 v = __ldg(p + (long long)k * (slab >> 2));
+        s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w;
+      }
+    }
+    if (grp > 0) sh[grp - 1][col] = s;
+    __syncthreads();
+    if (grp == 0 && qd < quads) {
+#pragma unroll
+      for (int q = 0; q < 3; ++q) { const float4 v = sh[q][col]; s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w; }
+      const int c4 = (int)(qd % cq); const long long r = qd / cq;
+      const int tap = (int)(r % taps), co = (int)(r / taps);
+      const float vals[4] = {s.x, s.y, s.z, s.w};
+#pragma unroll
+      for (int e = 0; e < 4; ++e) {
+        const int ci = 4 * c4 + e;
+        if (ci < g.Cin) {
+          if (layout == MQ_NCHW) out[((long long)co * g.Cin + ci) * taps + tap] = vals[e];
+          else out[((long long)co * taps + tap) * g.Cin + ci] = vals[e];
+        }
+      }
+    }
+    __syncthreads();
   }
 }
 
@@ -260,8 +287,8 @@ size_t conv_generic_workspace(int op, const Geom& g) {
 }
 
 cudaError_t launch_bwd_weight_reduce(const float* partial, float* out, const Geom& g, int splits, int layout, cudaStream_t s) {
-  const long long total = (long long)g.Cout * g.Kh * g.Kw * g.Cin;
-  unsigned blocks = (unsigned)((total + 255) / 256);
+  const long long quads = (long long)g.Cout * g.Kh * g.Kw * (g.Cp / 4);
+  unsigned blocks = (unsigned)((quads + 63) / 64);
   if (blocks > 148u * 16) blocks = 148u * 16;
   bwd_weight_reduce<<<blocks, 256, 0, s>>>(partial, out, g, splits, layout);
   count_launches(1);
@@ -299,8 +326,8 @@ cudaError_t launch_conv_generic(int op, const ConvArgs& a, cudaStream_t s) {
     MQ_DISPATCH2(a.fmt_a, a.fmt_b, (bwd_weight_generic<A_, B_><<<grid, GT, 0, s>>>(a, splits)));
     cudaError_t e = cudaGetLastError();
     if (e != cudaSuccess) return e;
-    const long long total = (long long)g.Cout * g.Kh * g.Kw * g.Cin;
-    unsigned blocks = (unsigned)((total + 255) / 256);
+    const long long quads = (long long)g.Cout * g.Kh * g.Kw * (g.Cp / 4);
+    unsigned blocks = (unsigned)((quads + 63) / 64);
     if (blocks > 148u * 16) blocks = 148u * 16;
     bwd_weight_reduce<<<blocks, 256, 0, s>>>(reinterpret_cast<const float*>(a.workspace), a.out, g, splits, a.out_layout);
     count_launches(1);

@@ -442,6 +442,49 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if (warp == 1) tmem_dealloc(tmem, 512);
 }
 
+template <int BPC>
+__device__ __forceinline__ unsigned long long load_scale_bytes(const uint8_t* ptr) {
+  if (BPC == 1) return __ldg(ptr);
+  if (BPC == 2) return __ldg(reinterpret_cast<const unsigned short*>(ptr));
+  if (BPC == 4) return __ldg(reinterpret_cast<const unsigned int*>(ptr));
+  return __ldg(reinterpret_cast<const unsigned long long*>(ptr));
+}
+
+// Builds, in shared memory, the scale-vector chunks ([chunk][group][atom][512]) of the resident weight tile of
+// the whole-tile kernel (channel tile 0).  Called by all threads of the block before the roles start (stride 1:
+// tap q of the walk is weight tap q).
+template <int KB, bool FP4>
+__device__ __forceinline__ void halo_build_sfb(const ConvTcParams& p, uint8_t* s_sfb) {
+  constexpr int G = 128 / KB, APC = KB / 32, SPA = FP4 ? 2 : 1, BPC = APC * SPA;
+  const int taps = p.Kh * p.Kw;
+  const int atoms_b = (p.BN + 127) / 128;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+#pragma unroll 1
+  for (int st = warp; st < p.max_stages; st += nwarps) {
+    unsigned long long acc[8] = {0ull, 0ull, 0ull, 0ull, 0ull, 0ull, 0ull, 0ull};
+#pragma unroll 1
+    for (int c = 0; c < G; ++c) {
+      const int q = st * G + c;
+      if (q < taps) {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+          if (j < 4 * atoms_b && 32 * j < p.BN && 32 * j < p.Cd)
+            acc[j] |= load_scale_bytes<BPC>(p.b_scales + ((long long)j * taps + q) * p.Kblocks) << (8 * c * BPC);
+        }
+      }
+    }
+    uint8_t* dst = s_sfb + (size_t)st * (512 * SPA * atoms_b) + lane * 16;
+#pragma unroll
+    for (int g = 0; g < SPA; ++g)
+#pragma unroll 1
+      for (int a = 0; a < atoms_b; ++a)
+        *reinterpret_cast<uint4*>(dst + (g * atoms_b + a) * 512) =
+            make_uint4((uint32_t)(acc[4 * a] >> (32 * g)), (uint32_t)(acc[4 * a + 1] >> (32 * g)), (uint32_t)(acc[4 * a + 2] >> (32 * g)),
+                       (uint32_t)(acc[4 * a + 3] >> (32 * g)));
+  }
+  fence_proxy_async_smem();   // the scale copies read these through the async proxy
+}
+
 // ---- whole-tile-per-stage variant -------------------------------------------------------------------
 // For stride-1 layers whose tap has at most 64 bytes of channels (one chunk per tap), the per-tap TMA boxes
 // of the kernel above are tiny and their issue rate is the limit.  Here
@@ -457,11 +500,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 //                 128-row operand at ((kw * Kh + kh) * 128) * KB.  Longer runs of output columns per warp for
 //                 an NCHW store, at Kw times the shared-memory footprint.
 // Roles and barriers are those of conv_tc_kernel, plus bfull / bempty for the resident weight tile.
+// With a single channel tile (p.fused) no preparation kernel runs at all: every block builds the weight image and
+// its scale chunks in shared memory itself at start-up, and warp 3 expands each tile's activation scales (a
+// Kh x (TW + Kw - 1) patch of tile scales: all rows of a tile lie in one 32-sample block) into the scale-vector
+// chunks of the tile's stage, a few tiles ahead of the MMAs.
 // TAPS > 0 fixes the tap count at compile time (the MMA issue loop is then fully unrolled with the tap offsets in
 // registers: the single issuing thread is latency-bound, every instruction between two MMAs counts); 0 = any.
 template <int MODE, int KB, bool FP4, int TAPS>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_out, const ConvTcParams p) {
+conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_w,
+                    const ConvTcParams p) {
   constexpr int G = 128 / KB, APC = KB / 32, SPA = FP4 ? 2 : 1;
   constexpr int LAYOUT = KB == 128 ? 2 : (KB == 64 ? 4 : 6);
 #ifdef MQ_TC_PROFILE
@@ -489,18 +537,24 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   uint32_t* tap_a = tmem_slot + 4;                     // per tap: offset of its A view / B rows, in 16-byte units
   uint32_t* tap_b = tap_a + 64;
+  uint32_t* tap_p = tap_b + 64;                        // per tap: first pixel of its view in the tile's scale patch
+  uint8_t* sc_tbl = reinterpret_cast<uint8_t*>(tap_p + 64);   // the tile's patch of raw scale bytes (<= 512)
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const unsigned total = (unsigned)p.total_tiles;
   const unsigned tiles_per_c = (unsigned)(p.classes * p.tiles_w * p.tiles_h);   // tile order: (class, w, h) below the channel tile
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); }
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], p.fused ? 2 : 1); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 8); }
     mbar_init(bfull, 1); mbar_init(bempty, 1);
     *abort_flag = 0;
     mbar_fence_init();
     prefetch_tensormap(&map_a);
     if (p.tma_store) prefetch_tensormap(&map_out);
+    if (p.fused) {   // the weight tile, all taps: one box, swizzled by the copy engine, while the block finishes setting up
+      mbar_arrive_expect_tx(bfull, (uint32_t)b_bytes);
+      tma_load_3d(smem, &map_w, bfull, 0, 0, 0);
+    }
   }
   if ((int)threadIdx.x < taps) {
     const int kh = threadIdx.x / p.Kw, kw = threadIdx.x - kh * p.Kw;
@@ -510,7 +564,9 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     const int aoff = p.nbox == 1 ? (hrow * p.TN * p.WH + wsh) * KB : (wsh * p.Kh + hrow) * 128 * KB;
     tap_a[threadIdx.x] = (uint32_t)aoff >> 4;
     tap_b[threadIdx.x] = (uint32_t)(threadIdx.x * p.BN * KB) >> 4;
+    tap_p[threadIdx.x] = (uint32_t)(hrow * (p.TW + p.Kw - 1) + wsh);
   }
+  if (p.fused) halo_build_sfb<KB, FP4>(p, smem + b_bytes);
   if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
   tc_fence_before_sync();
   __syncthreads();
@@ -534,7 +590,7 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x) {
         const Tile tile = decode_tile(p, t);
         const int ct = tile.ct;
-        if (ct != cur_ct) {
+        if (!p.fused && ct != cur_ct) {
           // new weight tile: wait until the MMAs of the previous one have retired, then one copy of image + scales
           if (bcount > 0 && !PROF_WAIT(mbar_wait(bempty, (bcount - 1) & 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
           mbar_arrive_expect_tx(bfull, (uint32_t)(b_bytes + sfb_bytes));
@@ -547,10 +603,10 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // first source pixel of the halo: forward (h - ph, w0 - pw); input gradient (h + ph - (Kh-1), w0 + pw - (Kw-1))
         const int hs = MODE == MQ_OP_FWD ? tile.h - p.ph : tile.h + p.ph - (p.Kh - 1);
         const int ws = MODE == MQ_OP_FWD ? tile.w0 - p.pw : tile.w0 + p.pw - (p.Kw - 1);
-        mbar_arrive_expect_tx(&full[s], (uint32_t)(p.nbox * p.halo_box_bytes + sfa_bytes));
+        mbar_arrive_expect_tx(&full[s], (uint32_t)(p.nbox * p.halo_box_bytes + (p.fused ? 0 : sfa_bytes)));
 #pragma unroll 1
         for (int b = 0; b < p.nbox; ++b) tma_load_4d(sa + (size_t)b * p.halo_box_bytes, &map_a, &full[s], 0, ws + b, tile.n0, hs);
-        bulk_load(sa + p.halo_a_bytes, p.sfa_img + (size_t)tile_m_index(p, tile) * sfa_bytes, sfa_bytes, &full[s]);
+        if (!p.fused) bulk_load(sa + p.halo_a_bytes, p.sfa_img + (size_t)tile_m_index(p, tile) * sfa_bytes, sfa_bytes, &full[s]);
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
       PROF_END(0);
@@ -631,7 +687,7 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         const int ct = p.tiles_c == 1 ? 0 : (int)((t / tiles_per_c) % (unsigned)p.tiles_c);
         const bool new_b = ct != cur_ct;
         if (new_b) {
-          if (!PROF_WAIT(mbar_wait(bfull, bcount & 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+          if (!p.fused && !PROF_WAIT(mbar_wait(bfull, bcount & 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
           cur_ct = ct; ++bcount;
         }
         if (!PROF_WAIT(mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
@@ -658,6 +714,75 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       }
       PROF_END(2);
     }
+  } else if (warp == 3) {
+    // ------------------------------------------------------------------ activation-scale expander (fused mode)
+    if (p.fused) {
+      constexpr int BPC = APC * SPA;                       // scale bytes per tap per row = K-blocks of a tap
+      const int WT = p.TW + p.Kw - 1, npix = p.Kh * WT;
+      // this lane's patch entries e = lane + 32 i: (halo row, column, K-block), fixed for the whole kernel
+      int e_h[4], e_w[4], e_k[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        const int e = lane + 32 * i, pe = e / BPC;
+        e_k[i] = e - pe * BPC; e_h[i] = pe / WT; e_w[i] = pe - e_h[i] * WT;
+        if (pe >= npix) e_h[i] = -1;
+      }
+      int twj[4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) twj[j] = (32 * j + lane) & (p.TW - 1);
+      uint32_t s = 0, phase = 0;
+      for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x) {
+        const Tile tile = decode_tile(p, t);
+        const int hs = MODE == MQ_OP_FWD ? tile.h - p.ph : tile.h + p.ph - (p.Kh - 1);
+        const int ws = MODE == MQ_OP_FWD ? tile.w0 - p.pw : tile.w0 + p.pw - (p.Kw - 1);
+        const int nblk = tile.n0 >> 5;
+        // raw tile scales of the patch (zero outside the image: those codes are zero-filled anyway)
+        uint8_t raw[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const int hh = hs + e_h[i], ww = ws + e_w[i];
+          raw[i] = 0;
+          if (e_h[i] >= 0 && hh >= 0 && hh < p.Hs && ww >= 0 && ww < p.Ws)
+            raw[i] = __ldg(p.a_scales + (((long long)hh * p.Ws + ww) * p.Nt + nblk) * p.Kblocks + e_k[i]);
+        }
+        bool ok = true;
+        if (lane == 0) ok = mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT);
+        ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+        if (!ok) { *abort_flag = 1; break; }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) sc_tbl[lane + 32 * i] = raw[i];
+        __syncwarp();
+        uint8_t* dst = stage0 + (size_t)s * stage_bytes + p.halo_a_bytes + lane * 16;
+#pragma unroll 1
+        for (int st = 0; st < nsf; ++st) {
+          unsigned long long acc[4] = {0ull, 0ull, 0ull, 0ull};
+#pragma unroll
+          for (int c = 0; c < G; ++c) {
+            const int q = st * G + c;
+            if (q < taps) {
+              const uint32_t pb = tap_p[q];
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const uint8_t* src = sc_tbl + (pb + twj[j]) * BPC;
+                unsigned long long v;
+                if (BPC == 1) v = *src;
+                else if (BPC == 2) v = *reinterpret_cast<const unsigned short*>(src);
+                else v = *reinterpret_cast<const unsigned int*>(src);
+                acc[j] |= v << (8 * c * BPC);
+              }
+            }
+          }
+#pragma unroll
+          for (int g = 0; g < SPA; ++g)
+            *reinterpret_cast<uint4*>(dst + (st * SPA + g) * 512) =
+                make_uint4((uint32_t)(acc[0] >> (32 * g)), (uint32_t)(acc[1] >> (32 * g)), (uint32_t)(acc[2] >> (32 * g)), (uint32_t)(acc[3] >> (32 * g)));
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&full[s]);
+        if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
+      }
+    }
   } else if (warp >= 4) {
     if (p.tma_store) epilogue_tma_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
@@ -681,14 +806,6 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 // row r of the tile at byte (r % 32) * 16 + (r / 32) * 4, four consecutive K-blocks per 32-bit word --
 // from the compact tile scales.  A-side chunks exist per tile (without its channel index), B-side
 // chunks per (stride class, channel tile).
-template <int BPC>
-__device__ __forceinline__ unsigned long long load_scale_bytes(const uint8_t* ptr) {
-  if (BPC == 1) return __ldg(ptr);
-  if (BPC == 2) return __ldg(reinterpret_cast<const unsigned short*>(ptr));
-  if (BPC == 4) return __ldg(reinterpret_cast<const unsigned int*>(ptr));
-  return __ldg(reinterpret_cast<const unsigned long long*>(ptr));
-}
-
 template <int MODE, int KB, bool FP4>
 __global__ void __launch_bounds__(256) expand_conv_scales_kernel(const ConvTcParams p, unsigned n_tile_m) {
   constexpr int G = 128 / KB, APC = KB / 32, SPA = FP4 ? 2 : 1, BPC = APC * SPA;
@@ -933,10 +1050,10 @@ cudaError_t launch_expand_conv_scales(const ConvTcParams& p, cudaStream_t s) {
 }
 
 template <int MODE, int KB, bool FP4, int TAPS>
-cudaError_t launch_conv_tc_halo_taps(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s) {
+cudaError_t launch_conv_tc_halo_taps(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_w, cudaStream_t s) {
   static bool attr_set = false;
   const size_t smem = 1024 + (size_t)p.halo_b_bytes + (size_t)p.stages * p.halo_stage_bytes + (p.tma_store ? EPI_STAGING_BYTES : 0) +
-                      (3 * (size_t)p.stages + 6) * 8 + 16 + 2 * 64 * 4;
+                      (3 * (size_t)p.stages + 6) * 8 + 16 + 3 * 64 * 4 + 512;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(conv_tc_halo_kernel<MODE, KB, FP4, TAPS>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
@@ -946,20 +1063,20 @@ cudaError_t launch_conv_tc_halo_taps(const ConvTcParams& p, const CUtensorMap& m
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const unsigned grid = (unsigned)(p.total_tiles < sms ? p.total_tiles : sms);
-  conv_tc_halo_kernel<MODE, KB, FP4, TAPS><<<grid, TC_THREADS, smem, s>>>(map_a, map_b, p);
+  conv_tc_halo_kernel<MODE, KB, FP4, TAPS><<<grid, TC_THREADS, smem, s>>>(map_a, map_b, map_w, p);
   count_launches(1);
   return cudaGetLastError();
 }
 template <int MODE, int KB, bool FP4>
-cudaError_t launch_conv_tc_halo_inst(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s) {
-  if (p.Kh * p.Kw == 9) return launch_conv_tc_halo_taps<MODE, KB, FP4, 9>(p, map_a, map_b, s);
-  return launch_conv_tc_halo_taps<MODE, KB, FP4, 0>(p, map_a, map_b, s);
+cudaError_t launch_conv_tc_halo_inst(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_w, cudaStream_t s) {
+  if (p.Kh * p.Kw == 9) return launch_conv_tc_halo_taps<MODE, KB, FP4, 9>(p, map_a, map_b, map_w, s);
+  return launch_conv_tc_halo_taps<MODE, KB, FP4, 0>(p, map_a, map_b, map_w, s);
 }
 
-cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s) {
+cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_w, cudaStream_t s) {
   if (p.total_tiles <= 0 || p.total_tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
   if (p.halo) {
-#define MQ_TC_HCASE(M, K, F) if (p.mode == M && p.KB == K && (p.kind_fp4 != 0) == F) return launch_conv_tc_halo_inst<M, K, F>(p, map_a, map_b, s)
+#define MQ_TC_HCASE(M, K, F) if (p.mode == M && p.KB == K && (p.kind_fp4 != 0) == F) return launch_conv_tc_halo_inst<M, K, F>(p, map_a, map_b, map_w, s)
     MQ_TC_HCASE(MQ_OP_FWD, 64, false); MQ_TC_HCASE(MQ_OP_FWD, 32, false); MQ_TC_HCASE(MQ_OP_FWD, 64, true); MQ_TC_HCASE(MQ_OP_FWD, 32, true);
     MQ_TC_HCASE(MQ_OP_BWD_DATA, 64, false); MQ_TC_HCASE(MQ_OP_BWD_DATA, 32, false); MQ_TC_HCASE(MQ_OP_BWD_DATA, 64, true); MQ_TC_HCASE(MQ_OP_BWD_DATA, 32, true);
 #undef MQ_TC_HCASE

@@ -50,6 +50,8 @@ struct ConvTcParams {
   int halo_a_bytes;         // bytes of a tile's activation boxes (rounded up to 1024)
   int halo_stage_bytes;     // bytes of one pipeline stage (activation boxes + A-side scale chunks)
   int halo_b_bytes;         // bytes of the resident weight image + its scale chunks (rounded up to 1024)
+  int fused;                // 1: single channel tile, stride 1: no preparation kernel (the blocks build the weight image, its
+                            //    scale chunks and every tile's activation scale chunks themselves)
   int tma_store;            // 1: NCHW output written by TMA stores from a staging buffer (the second tensor map is the output's)
   const uint8_t* b_codes;   // weight-like codes [rows][taps][b_rowbytes] (source of the images below)
   int b_rows_total, b_rowbytes;
@@ -60,7 +62,9 @@ struct ConvTcParams {
   unsigned int* status;
 };
 
-cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s);
+// map_a: gathered activation codes.  map_b: weight codes per tap (per-tap kernel) or the fp32 output (whole-tile kernel
+// with TMA stores).  map_w: all taps of a weight tile in one box (whole-tile kernel, fused preparation).
+cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_w, cudaStream_t s);
 // Expands the compact tile scales into the per-stage scale-vector chunks the MMA reads (p.sfa_img, p.sfb_img).
 cudaError_t launch_expand_conv_scales(const ConvTcParams& p, cudaStream_t s);
 size_t conv_tc_sfa_bytes(const ConvTcParams& p);
@@ -78,7 +82,7 @@ struct WgradTcParams {
   int mode;             // MQ_WG_FP8: 8-bit operands as stored (MN-major TMA boxes); MQ_WG_FP4_PIXEL: E2M1 re-laid
                         // [pixel][c][n], one TMA box per pixel; MQ_WG_FP4_FLAT: stride 1, E2M1 re-laid as contiguous
                         // pre-swizzled pieces over the zero-padded, flattened pixel axis (bulk copies)
-  uint32_t idesc;
+  uint32_t idesc;       // instruction descriptor without the N field
   int stages;
   int N, Nt, Ho, Wo, H, W, Cout, Cp, Ct, Cot, Kh, Kw, sh, sw, ph, pw;
   int BPP;              // K-blocks (32 samples) taken per pixel per stage
@@ -89,14 +93,20 @@ struct WgradTcParams {
   int stages_total;     // pixel: Ho * groups_w * nchunks; flat: ceil(Ho * Wp / KPX)
   int Wp;               // flat: padded width W + 2 * pw
   int b_rows;           // rows (input channels) of a B tile: 128, or min(128, Cp) in flat mode
-  int m_tiles, j_tiles, cb_tiles, splits;
+  int m_tiles, j_tiles, cb_tiles, splits;   // j_tiles = (taps / TG) * cb_tiles
+  int TG;               // taps per block: 1, or Kw (flat mode: the taps of a kernel row share the stage's pixels)
+  int NB;               // 128-row chunks of the group's B rows = ceil(TG * b_rows / 128)
+  int n0, n1;           // MMA widths per K slice: n0 = min(TG * b_rows, 256) and the rest (0: one MMA)
+  int b_tile_bytes;     // bytes of X loaded per stage: b_rows * 128, flat mode (KPX + TG - 1) * b_rows * KBn
+  int stage_bytes;      // A tile + B tile + (1 + NB) scale chunks of 1024 bytes, rounded up to 1024
+  int tmem_cols;        // TMEM allocation: accumulators (TG * b_rows) + stages * (8 + 8 * NB), a power of two
   const uint8_t* g_scales;  // [Ho][Wo][Nt][Cot]
   const uint8_t* x_scales;  // [H][W][Nt][Ct]
   const uint8_t* gt;        // flat: [co block][padded pixel][128][KBn]
   const uint8_t* xt;        // flat: [ci block][padded pixel][b_rows][KBn]
   long long gt_block_bytes, xt_block_bytes;
   uint8_t* sfa_img;         // [m tile][stage][512 * SPA]
-  uint8_t* sfb_img;         // [ci block][tap][stage][512 * SPA]
+  uint8_t* sfb_img;         // [ci block][tap group][stage][NB][512 * SPA]
   float* partial;           // [splits][Cout][taps * Cp]
   unsigned int* status;
 };

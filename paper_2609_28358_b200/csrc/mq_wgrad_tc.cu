@@ -26,8 +26,6 @@ namespace {
 using namespace tc;
 
 constexpr int WG_THREADS = 256;
-constexpr int WG_STAGE_BYTES = 2 * 128 * 128 + 4 * 512;  // A 16 KB + B 16 KB + scale chunks (2 groups each)
-constexpr int WG_SF_COLS = 16;                           // TMEM columns of one stage's scale vectors (A 8 + B 8)
 
 // K-block b of stage st: output pixel and 32-sample block
 __device__ __forceinline__ void stage_block(const WgradTcParams& p, int st, int b, int& ho, int& wo, int& nb) {
@@ -50,9 +48,10 @@ __global__ void __launch_bounds__(256) expand_wgrad_scales_kernel(const WgradTcP
   const long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int taps = p.Kh * p.Kw;
   const long long nA = (long long)p.m_tiles * p.stages_total;
-  const long long nB = (long long)p.cb_tiles * taps * p.stages_total;
+  const int groups = taps / p.TG;
+  const long long nB = (long long)p.cb_tiles * groups * p.stages_total * p.NB;
   if (wid >= nA + nB) return;
-  // this lane's byte: channel block j of the tile (row group), K-block b of the stage
+  // this lane's byte: 32-row group j of the 128-row chunk, K-block b of the stage
   const int j = lane >> 3, b = lane & 7;
   uint32_t v = 0;
   uint8_t* dst;
@@ -66,12 +65,17 @@ __global__ void __launch_bounds__(256) expand_wgrad_scales_kernel(const WgradTcP
     }
     dst = p.sfa_img + wid * (512 * SPA);
   } else {
+    // B rows of a tap group: tap-in-group major, input channel minor; chunk c holds rows [128c, 128c + 128)
     long long idx = wid - nA;
+    const int c = (int)(idx % p.NB); idx /= p.NB;
     const int st = (int)(idx % p.stages_total); idx /= p.stages_total;
-    const int tap = (int)(idx % taps); const int cb = (int)(idx / taps);
+    const int tg = (int)(idx % groups); const int cb = (int)(idx / groups);
+    const int row0 = c * 128 + 32 * j;
+    const int tj = row0 / p.b_rows, rj = row0 - tj * p.b_rows;
+    const int tap = tg * p.TG + tj;
     const int kh = tap / p.Kw, kw = tap - kh * p.Kw;
-    const int cib = (cb * p.b_rows) / 32 + j;
-    if (b < NBS && 32 * j < p.b_rows && cib < p.Ct) {
+    const int cib = (cb * p.b_rows + rj) / 32;
+    if (b < NBS && tj < p.TG && cib < p.Ct) {
       int ho, wo, nb;
       stage_block(p, st, b, ho, wo, nb);
       const int h = ho * p.sh + kh - p.ph, w = wo * p.sw + kw - p.pw;
@@ -94,13 +98,20 @@ __global__ void __launch_bounds__(256) expand_wgrad_scales_kernel(const WgradTcP
   }
 }
 
+// A block's work item is (output-channel tile, tap group, input-channel block, K slice).  In the flat mode a tap
+// group is the Kw taps of one kernel row: their B operands are views of the same run of consecutive pixels,
+// shifted by one pixel (one piece) per tap, so a stage loads KPX + Kw - 1 pieces of X once and the stage's G_Y
+// tile feeds Kw accumulators (Kw times less shared-memory traffic per FLOP than one tap per block).
 template <bool FP4>
 __global__ void __launch_bounds__(WG_THREADS, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const WgradTcParams p) {
   constexpr int SPA = FP4 ? 2 : 1;     // scale bytes per MMA per row
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * WG_STAGE_BYTES);
+  const int TG = p.TG;
+  const int stage_bytes = p.stage_bytes;               // A tile | B tile | A scale chunk (1024) | NB B scale chunks
+  const int b_off = 128 * 128, sf_off = b_off + p.b_tile_bytes;
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * stage_bytes);
   uint64_t* empty = full + p.stages;
   uint64_t* sffull = empty + p.stages;
   uint64_t* tfull = sffull + p.stages;
@@ -113,21 +124,25 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   const int mt = item % p.m_tiles; item /= p.m_tiles;
   const int jt = item % p.j_tiles;
   const int split = item / p.j_tiles;
-  const int tap = jt / p.cb_tiles, cb = jt - tap * p.cb_tiles;
-  const int kh = tap / p.Kw, kw = tap - kh * p.Kw;
+  const int tgi = jt / p.cb_tiles, cb = jt - tgi * p.cb_tiles;
+  const int tap0 = tgi * TG;                            // first tap of the group (TG divides Kw)
+  const int kh = tap0 / p.Kw, kw = tap0 - kh * p.Kw;
   const int co0 = mt * 128, ci0 = cb * p.b_rows;
   const int st_begin = (int)((long long)p.stages_total * split / p.splits);
   const int st_end = (int)((long long)p.stages_total * (split + 1) / p.splits);
   const int nst = st_end - st_begin;
+  const uint32_t acc_cols = (uint32_t)(TG * p.b_rows);  // accumulators first, then the per-stage scale buffers
+  const uint32_t sf_cols = 8u + 8u * (uint32_t)p.NB;
 
   if (threadIdx.x == 0) {
+#pragma unroll 1
     for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); }
     mbar_init(tfull, 1);
     *abort_flag = 0;
     mbar_fence_init();
     if (p.mode != MQ_WG_FP4_FLAT) { prefetch_tensormap(&map_a); prefetch_tensormap(&map_b); }
   }
-  if (warp == 1) { tmem_alloc(tmem_slot, 256); tmem_relinquish(); }
+  if (warp == 1) { tmem_alloc(tmem_slot, p.tmem_cols); tmem_relinquish(); }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
@@ -138,26 +153,29 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     if (lane == 0) {
       const int taps = p.Kh * p.Kw;
       const uint8_t* sfa_src = p.sfa_img + ((size_t)mt * p.stages_total + st_begin) * (512 * SPA);
-      const uint8_t* sfb_src = p.sfb_img + (((size_t)cb * taps + tap) * p.stages_total + st_begin) * (512 * SPA);
-      const uint32_t a_bytes = 128 * 128, b_bytes = (uint32_t)p.b_rows * 128;
+      const uint32_t sfb_bytes = (uint32_t)p.NB * 512 * SPA;
+      const uint8_t* sfb_src = p.sfb_img + (((size_t)cb * (taps / TG) + tgi) * p.stages_total + st_begin) * sfb_bytes;
+      const uint32_t a_bytes = 128 * 128, b_step = (uint32_t)p.b_rows * 128, b_bytes = (uint32_t)p.b_tile_bytes;
       const uint8_t* ga = nullptr; const uint8_t* gb = nullptr;
       if (p.mode == MQ_WG_FP4_FLAT) {
         ga = p.gt + (size_t)mt * p.gt_block_bytes + (size_t)st_begin * a_bytes;
         gb = p.xt + (size_t)cb * p.xt_block_bytes + ((size_t)st_begin * p.KPX + (size_t)kh * p.Wp + kw) * ((size_t)p.b_rows * p.KBn);
       }
       uint32_t s = 0, phase = 0;
+#pragma unroll 1
       for (int i = 0; i < nst && !*abort_flag; ++i) {
         if (!mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
-        uint8_t* sa = smem + (size_t)s * WG_STAGE_BYTES;
-        uint8_t* sb = sa + 128 * 128;
-        mbar_arrive_expect_tx(&full[s], a_bytes + b_bytes + 2 * 512 * SPA);
-        bulk_load(sb + 128 * 128, sfa_src, 512 * SPA, &full[s]);
-        bulk_load(sb + 128 * 128 + 1024, sfb_src, 512 * SPA, &full[s]);
-        sfa_src += 512 * SPA; sfb_src += 512 * SPA;
+        uint8_t* sa = smem + (size_t)s * stage_bytes;
+        uint8_t* sb = sa + b_off;
+        uint8_t* ssf = sa + sf_off;
+        mbar_arrive_expect_tx(&full[s], a_bytes + b_bytes + 512 * SPA + sfb_bytes);
+        bulk_load(ssf, sfa_src, 512 * SPA, &full[s]);
+        bulk_load(ssf + 1024, sfb_src, sfb_bytes, &full[s]);
+        sfa_src += 512 * SPA; sfb_src += sfb_bytes;
         if (p.mode == MQ_WG_FP4_FLAT) {
           bulk_load(sa, ga, a_bytes, &full[s]);
-          bulk_load(sb, gb, b_bytes, &full[s]);
-          ga += a_bytes; gb += b_bytes;
+          bulk_load(sb, gb, b_bytes, &full[s]);          // KPX + TG - 1 consecutive pixels
+          ga += a_bytes; gb += b_step;
         } else {
           const int st = st_begin + i;
           const int nc = st % p.nchunks; const int t = st / p.nchunks;
@@ -165,6 +183,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           const int wo0 = wg * p.KPX;
           if (p.mode == MQ_WG_FP4_PIXEL) {
             // [pixel][c][n] re-laid codes: one box (n bytes, 128 channels) per pixel of the stage
+#pragma unroll 1
             for (int px = 0; px < p.KPX; ++px) {
               tma_load_4d(sa + px * 128 * p.KBn, &map_a, &full[s], nc * p.KBn, co0, wo0 + px, ho);
               tma_load_4d(sb + px * 128 * p.KBn, &map_b, &full[s], nc * p.KBn, ci0, (wo0 + px) * p.sw + kw - p.pw, ho * p.sh + kh - p.ph);
@@ -187,8 +206,14 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const uint32_t fp4_layout = p.KBn == 128 ? 2u : (p.KBn == 64 ? 4u : (p.KBn == 32 ? 6u : 0u));
       const uint32_t a_piece = 128 * p.KBn, b_piece = (uint32_t)p.b_rows * p.KBn;
       const uint64_t a_desc0 = smem_desc(FP4 ? smem_desc_base(a_piece, 8 * p.KBn, fp4_layout) : smem_desc_base(128 * 128, 1024, 2), smem_u32(smem));
-      const uint64_t b_desc0 = smem_desc(FP4 ? smem_desc_base(b_piece, 8 * p.KBn, fp4_layout) : smem_desc_base(128 * 128, 1024, 2), smem_u32(smem + 128 * 128));
-      const uint32_t stage16 = WG_STAGE_BYTES >> 4;
+      const uint64_t b_desc0 = smem_desc(FP4 ? smem_desc_base(b_piece, 8 * p.KBn, fp4_layout) : smem_desc_base(128 * 128, 1024, 2), smem_u32(smem + b_off));
+      const uint32_t stage16 = (uint32_t)stage_bytes >> 4;
+      // The taps of a group are ONE wide B operand: tap j's view starts j pieces (= b_rows / 8 row groups) further,
+      // which is exactly where rows [j * b_rows, (j + 1) * b_rows) of a (TG * b_rows)-row operand lie.  At most two
+      // MMAs per K slice: N = n0 (<= 256) and the remaining n1 rows.
+      const uint32_t idesc_n[2] = {p.idesc | ((uint32_t)(p.n0 >> 3) << 17), p.idesc | ((uint32_t)(p.n1 >> 3) << 17)};
+      const uint32_t row16_1 = ((uint32_t)p.n0 * p.KBn) >> 4;   // second MMA: B rows from n0 on (flat mode only)
+      const int nm = p.n1 > 0 ? 2 : 1;
       uint32_t ka16[4], kb16[4];   // offset of MMA a's K slice inside the stage's A / B tile, in 16-byte units
 #pragma unroll
       for (int a = 0; a < 4; ++a) {
@@ -197,23 +222,28 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           ka16[a] = (piece * a_piece + off) >> 4; kb16[a] = (piece * b_piece + off) >> 4;
         } else { ka16[a] = 256u * a; kb16[a] = 256u * a; }
       }
-      uint32_t idesc_id[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) idesc_id[i] = idesc_with_sf_ids(p.idesc, i, i);
-      const uint32_t sf_base = tmem + 128;
+      const uint32_t sf_base = tmem + acc_cols;
       uint32_t s = 0, phase = 0, accumulate = 0;
+#pragma unroll 1
       for (int i = 0; i < nst && !*abort_flag; ++i) {
         if (!mbar_wait(&sffull[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
         tc_fence_after_sync();
         const uint32_t so = s * stage16;
-        const uint32_t sfa_t = sf_base + s * WG_SF_COLS, sfb_t = sfa_t + 8;
+        const uint32_t sfa_t = sf_base + s * sf_cols, sfb_t = sfa_t + 8;
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
           const int g = (a * SPA) >> 2, id = (a * SPA) & 3;
-          if (FP4) mma_mxf4(tmem, a_desc0 + so + ka16[a], b_desc0 + so + kb16[a], idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g, accumulate);
-          else mma_mxf8f6f4(tmem, a_desc0 + so + ka16[a], b_desc0 + so + kb16[a], idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g, accumulate);
-          accumulate = 1;
+          const uint32_t accu = accumulate | (a > 0 ? 1u : 0u);
+#pragma unroll 1
+          for (int m = 0; m < nm; ++m) {
+            const uint32_t d_t = tmem + (m ? (uint32_t)p.n0 : 0u), bo = so + (m ? row16_1 : 0u);
+            const uint32_t idesc = idesc_with_sf_ids(idesc_n[m], id, id);
+            const uint32_t sfb_m = sfb_t + 4 * (g * p.NB + (m ? (p.n0 >> 7) : 0));
+            if (FP4) mma_mxf4(d_t, a_desc0 + so + ka16[a], b_desc0 + bo + kb16[a], idesc, sfa_t + 4 * g, sfb_m, accu);
+            else mma_mxf8f6f4(d_t, a_desc0 + so + ka16[a], b_desc0 + bo + kb16[a], idesc, sfa_t + 4 * g, sfb_m, accu);
+          }
         }
+        accumulate = 1;
         tc_commit(&empty[s]);
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
@@ -223,20 +253,22 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     // ------------------------------------------------------------------ scale copier (smem -> per-stage TMEM buffers)
     if (lane == 0) {
       const uint64_t sf_desc = smem_desc_base(0, 128, 0);
-      const uint64_t sfa_desc0 = smem_desc(sf_desc, smem_u32(smem + 2 * 128 * 128));
-      const uint64_t sfb_desc0 = smem_desc(sf_desc, smem_u32(smem + 2 * 128 * 128 + 1024));
-      const uint32_t stage16 = WG_STAGE_BYTES >> 4;
-      const uint32_t sf_base = tmem + 128;
+      const uint64_t sf_desc0 = smem_desc(sf_desc, smem_u32(smem + sf_off));
+      const uint32_t stage16 = (uint32_t)stage_bytes >> 4;
+      const uint32_t sf_base = tmem + acc_cols;
       uint32_t s = 0, phase = 0;
+#pragma unroll 1
       for (int i = 0; i < nst && !*abort_flag; ++i) {
         if (!mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
         tc_fence_after_sync();
         const uint32_t so = s * stage16;
-        const uint32_t sfa_t = sf_base + s * WG_SF_COLS, sfb_t = sfa_t + 8;
+        const uint32_t sf_t = sf_base + s * sf_cols;
 #pragma unroll
-        for (int g = 0; g < SPA; ++g) {
-          tmem_cp_32x128b_warpx4(sfa_t + 4 * g, sfa_desc0 + so + g * 32);
-          tmem_cp_32x128b_warpx4(sfb_t + 4 * g, sfb_desc0 + so + g * 32);
+        for (int g = 0; g < SPA; ++g) tmem_cp_32x128b_warpx4(sf_t + 4 * g, sf_desc0 + so + g * 32);
+#pragma unroll 1
+        for (int c = 0; c < p.NB; ++c) {     // B-side chunk c: rows [128c, 128c + 128) of the group's operand
+#pragma unroll
+          for (int g = 0; g < SPA; ++g) tmem_cp_32x128b_warpx4(sf_t + 8 + 4 * (g * p.NB + c), sf_desc0 + so + 64 + (c * SPA + g) * 32);
         }
         tc_commit(&sffull[s]);
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
@@ -253,29 +285,33 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       tc_fence_after_sync();
       const int co = co0 + r;
       const long long J = (long long)p.Kh * p.Kw * p.Cp;
-      float* out = p.partial + ((long long)split * p.Cout + co) * J + (long long)tap * p.Cp + ci0;
       const int ncols = min(p.b_rows, p.Cp - ci0);
-      const uint32_t taddr = tmem + ((uint32_t)(32 * quad) << 16);
-      for (int c = 0; c < ncols; c += 16) {
-        uint32_t v[16];
-        if (nst > 0) {
-          tmem_ld_32x32b_x16(taddr + c, v);
-          tmem_ld_wait();
-        } else {
+#pragma unroll 1
+      for (int j = 0; j < TG; ++j) {
+        float* out = p.partial + ((long long)split * p.Cout + co) * J + (long long)(tap0 + j) * p.Cp + ci0;
+        const uint32_t taddr = tmem + (uint32_t)(j * p.b_rows) + ((uint32_t)(32 * quad) << 16);
+#pragma unroll 1
+        for (int c = 0; c < ncols; c += 16) {
+          uint32_t v[16];
+          if (nst > 0) {
+            tmem_ld_32x32b_x16(taddr + c, v);
+            tmem_ld_wait();
+          } else {
 #pragma unroll
-          for (int q = 0; q < 16; ++q) v[q] = 0u;
-        }
-        if (co < p.Cout) {
+            for (int q = 0; q < 16; ++q) v[q] = 0u;
+          }
+          if (co < p.Cout) {
 #pragma unroll
-          for (int q = 0; q < 16; q += 4)   // Cp is a multiple of 32: whole float4s
-            *reinterpret_cast<float4*>(out + c + q) = make_float4(__uint_as_float(v[q]), __uint_as_float(v[q + 1]), __uint_as_float(v[q + 2]), __uint_as_float(v[q + 3]));
+            for (int q = 0; q < 16; q += 4)   // Cp is a multiple of 32: whole float4s
+              *reinterpret_cast<float4*>(out + c + q) = make_float4(__uint_as_float(v[q]), __uint_as_float(v[q + 1]), __uint_as_float(v[q + 2]), __uint_as_float(v[q + 3]));
+          }
         }
       }
     }
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem, 256);
+  if (warp == 1) tmem_dealloc(tmem, p.tmem_cols);
 }
 
 // ---- E2M1 re-layout: stored [pixel][n][Cp] nibbles -> [pixel][Cp][Npad] nibbles (n fastest, zero for n >= N) ----
@@ -358,7 +394,7 @@ __global__ void __launch_bounds__(256) fp4_to_flat_kernel(const uint8_t* __restr
 
 }  // namespace
 
-size_t wgrad_tc_smem_bytes(const WgradTcParams& p) { return 1024 + (size_t)p.stages * WG_STAGE_BYTES + (3 * (size_t)p.stages + 2) * 8 + 64; }
+size_t wgrad_tc_smem_bytes(const WgradTcParams& p) { return 1024 + (size_t)p.stages * p.stage_bytes + (3 * (size_t)p.stages + 2) * 8 + 64; }
 
 cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s) {
   static bool attr_set[2] = {false, false};
@@ -378,7 +414,7 @@ cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, co
 }
 
 cudaError_t launch_expand_wgrad_scales(const WgradTcParams& p, cudaStream_t s) {
-  const long long warps = (long long)p.m_tiles * p.stages_total + (long long)p.cb_tiles * p.Kh * p.Kw * p.stages_total;
+  const long long warps = (long long)p.m_tiles * p.stages_total + (long long)p.cb_tiles * (p.Kh * p.Kw / p.TG) * p.stages_total * p.NB;
   const unsigned blocks = (unsigned)((warps + 7) / 8);
   if (p.mode == MQ_WG_FP8) expand_wgrad_scales_kernel<false><<<blocks, 256, 0, s>>>(p);
   else expand_wgrad_scales_kernel<true><<<blocks, 256, 0, s>>>(p);
