@@ -371,8 +371,6 @@ mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const 
   uint8_t* gt = base + w.off_gt;
   CUtensorMap map_a{}, map_b{};
   if (p.mode == MQ_WG_FP4_FLAT) {
-    if (launch_fp4_to_flat(static_cast<const uint8_t*>(qx->codes), xt, g.H, g.W, g.N, g.Cp, w.P_b, p.Wp, g.ph, g.pw, p.b_rows, p.cb_tiles, p.KBn, stream) != cudaSuccess) return MQ_ERR_CUDA;
-    if (launch_fp4_to_flat(static_cast<const uint8_t*>(qg->codes), gt, g.Ho, g.Wo, g.N, g.Cop, w.P_a, p.Wp, 0, 0, 128, p.m_tiles, p.KBn, stream) != cudaSuccess) return MQ_ERR_CUDA;
     p.xt = xt; p.gt = gt;
     p.idesc = (1u << 7) | (1u << 10) | (1u << 23) | ((128u >> 4) << 24);
   } else if (p.mode == MQ_WG_FP4_PIXEL) {
@@ -412,8 +410,19 @@ mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const 
       if (!encode_tensor_map_u8(&map_b, qx->codes, 4, dims, strides, box, es, 128)) return MQ_ERR_CUDA;
     }
   }
-  if (launch_expand_wgrad_scales(p, stream) != cudaSuccess) return MQ_ERR_CUDA;
-  if (launch_wgrad_tc(p, map_a, map_b, stream) != cudaSuccess) return MQ_ERR_CUDA;
+  if (p.mode == MQ_WG_FP4_FLAT) {
+    if (launch_wgrad_flat_prep(p, static_cast<const uint8_t*>(qx->codes), xt, w.P_b, static_cast<const uint8_t*>(qg->codes), gt, w.P_a, stream) != cudaSuccess)
+      return MQ_ERR_CUDA;
+  } else if (launch_expand_wgrad_scales(p, stream) != cudaSuccess) return MQ_ERR_CUDA;
+  CUtensorMap map_p{};
+  {
+    const uint64_t J = (uint64_t)g.Kh * g.Kw * g.Cp;
+    const uint64_t dims[3] = {J, (uint64_t)g.Cout, (uint64_t)p.splits};
+    const uint64_t strides[2] = {J * 4, (uint64_t)g.Cout * J * 4};
+    const uint32_t box[3] = {32u, 32u, 1u};
+    if (!encode_tensor_map_u8(&map_p, partial, 3, dims, strides, box, nullptr, 128, true)) return MQ_ERR_CUDA;
+  }
+  if (launch_wgrad_tc(p, map_a, map_b, map_p, stream) != cudaSuccess) return MQ_ERR_CUDA;
   return launch_bwd_weight_reduce(partial, out, g, p.splits, layout, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }
 

@@ -110,15 +110,18 @@ struct WgradTcParams {
   float* partial;           // [splits][Cout][taps * Cp]
   unsigned int* status;
 };
-cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s);
+// map_p: the partial sums as an fp32 tensor (taps * Cp columns, C_out rows, splits), box 32 x 32 x 1, 128-byte swizzle
+cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_p, cudaStream_t s);
 cudaError_t launch_expand_wgrad_scales(const WgradTcParams& p, cudaStream_t s);
 // E2M1 codes [P][N][Cp] -> [P][Cp][Npad] (n fastest, zero-padded): a permutation of nibbles, no requantization.
 cudaError_t launch_fp4_to_n_major(const uint8_t* in, uint8_t* out, int P, int N, int Cp, int Npad, cudaStream_t s);
-// E2M1 codes [Hs][Ws][N][Cs_p] -> [channel block][q][rows][KBn] over q = hq * Wp + wq in [0, P_out), source pixel
-// (hq - off_h, wq - off_w), zero outside the image / beyond the channels, each [rows][KBn] piece stored with the
-// shared-memory swizzle of span KBn already applied.
-cudaError_t launch_fp4_to_flat(const uint8_t* in, uint8_t* out, int Hs, int Ws, int N, int Cs_p, int P_out, int Wp, int off_h, int off_w,
-                               int rows, int nblocks, int KBn, cudaStream_t s);
+// Flat-mode preparation in one launch.  E2M1 codes [Hs][Ws][N][Cs_p] -> [channel block][q][rows][KBn] over the
+// zero-padded, flattened pixel axis q = hq * Wp + wq in [0, P), source pixel (hq - off_h, wq - off_w), zero outside
+// the image / beyond the channels, each [rows][KBn] piece stored with the shared-memory swizzle of span KBn already
+// applied: X (P_b pixels, offsets = the padding, b_rows channels per block) and G_Y (P_a pixels, 128 channels per
+// block); then the scale chunks of expand_wgrad_scales.
+cudaError_t launch_wgrad_flat_prep(const WgradTcParams& p, const uint8_t* x_codes, uint8_t* xt, int P_b, const uint8_t* g_codes, uint8_t* gt, int P_a,
+                                   cudaStream_t s);
 // Adds the split partial sums in a fixed order and writes G_W in its final layout.
 cudaError_t launch_bwd_weight_reduce(const float* partial, float* out, const Geom& g, int splits, int layout, cudaStream_t s);
 

@@ -12,37 +12,50 @@ namespace {
 
 constexpr int IC_THREADS = 256;
 constexpr int IC_MAX_J = 1024;   // chunks of 16 bytes per X' row held in the offset table
+constexpr int IC_TABLE = 2048;   // table entries per block: PX pixels x J chunks
 
-__global__ void __launch_bounds__(IC_THREADS) im2col_kernel(Im2colArgs a, int rc, int J, unsigned n_main) {
+// PX consecutive output pixels per block amortise the block's fixed cost (launch, offset table, barrier) over
+// PX * 32 rows of X'.
+__global__ void __launch_bounds__(IC_THREADS) im2col_kernel(Im2colArgs a, int rc, int J, int PX, unsigned n_main) {
   const Geom& g = a.g;
-  __shared__ int soff[IC_MAX_J];   // source chunk offset of row chunk j relative to sample 0 of the source pixel, -1: zero
+  __shared__ int soff[IC_TABLE];   // source chunk offset of row chunk j of pixel px relative to sample 0, -1: zero
   const int taps = g.Kh * g.Kw;
   if (blockIdx.x < n_main) {
-    const unsigned pix = blockIdx.x / (unsigned)g.Nt;
-    const int nt = (int)(blockIdx.x - pix * (unsigned)g.Nt);
-    const int ho = (int)(pix / (unsigned)g.Wo), wo = (int)(pix - (unsigned)ho * (unsigned)g.Wo);
-    for (int j = threadIdx.x; j < J; j += IC_THREADS) {
+    const unsigned pg = blockIdx.x / (unsigned)g.Nt;
+    const int nt = (int)(blockIdx.x - pg * (unsigned)g.Nt);
+    const unsigned pix0 = pg * (unsigned)PX;
+    const unsigned npix = (unsigned)(g.Ho * g.Wo);
+    const int px_n = (int)min((unsigned)PX, npix - pix0);
+    for (int e = threadIdx.x; e < px_n * J; e += IC_THREADS) {
+      const int px = e / J, j = e - px * J;
+      const unsigned pix = pix0 + px;
+      const int ho = (int)(pix / (unsigned)g.Wo), wo = (int)(pix - (unsigned)ho * (unsigned)g.Wo);
       const int tap = j / rc, ch = j - tap * rc;
       const int kh = tap / g.Kw, kw = tap - kh * g.Kw;
       const int h = ho * g.sh + kh - g.ph, w = wo * g.sw + kw - g.pw;
-      soff[j] = (h >= 0 && h < g.H && w >= 0 && w < g.W) ? ((h * g.W + w) * g.N) * rc + ch : -1;   // < 2^31 chunks checked on the host
+      soff[e] = (h >= 0 && h < g.H && w >= 0 && w < g.W) ? ((h * g.W + w) * g.N) * rc + ch : -1;   // < 2^31 chunks checked on the host
     }
     __syncthreads();
     const int n0 = nt * 32;
     const int rows = min(32, g.N - n0);
     const int total = rows * J;
     const uint4* src = reinterpret_cast<const uint4*>(a.codes) + (long long)n0 * rc;
-    uint4* dst = reinterpret_cast<uint4*>(a.out_codes) + ((long long)pix * g.N + n0) * J;
-    // chunk i = n * J + j, advanced by IC_THREADS per step without divisions
-    int n = threadIdx.x / J, j = threadIdx.x - n * J;
     const int dn = IC_THREADS / J, dj = IC_THREADS - dn * J;
-    for (int i = threadIdx.x; i < total; i += IC_THREADS) {
-      const int so = soff[j];
-      uint4 v = make_uint4(0, 0, 0, 0);
-      if (so >= 0) v = __ldg(src + so + n * rc);
-      __stcs(dst + i, v);
-      n += dn; j += dj;
-      if (j >= J) { j -= J; ++n; }
+#pragma unroll 1
+    for (int px = 0; px < px_n; ++px) {
+      const int* so_px = soff + px * J;
+      uint4* dst = reinterpret_cast<uint4*>(a.out_codes) + ((long long)(pix0 + px) * g.N + n0) * J;
+      // chunk i = n * J + j, advanced by IC_THREADS per step without divisions
+      int n = threadIdx.x / J, j = threadIdx.x - n * J;
+#pragma unroll 2
+      for (int i = threadIdx.x; i < total; i += IC_THREADS) {
+        const int so = so_px[j];
+        uint4 v = make_uint4(0, 0, 0, 0);
+        if (so >= 0) v = __ldg(src + so + n * rc);
+        __stcs(dst + i, v);
+        n += dn; j += dj;
+        if (j >= J) { j -= J; ++n; }
+      }
     }
   } else {
     // scales [ho][wo][nt][kh][kw][ct]
@@ -105,14 +118,17 @@ cudaError_t launch_im2col(const Im2colArgs& a, cudaStream_t s) {
   const int taps = g.Kh * g.Kw;
   const long long J = (long long)taps * rc;
   const long long src_chunks = (long long)g.H * g.W * g.N * rc;
-  const long long n_main = (long long)g.Ho * g.Wo * g.Nt;
+  int PX = (int)(IC_TABLE / (J > 0 ? J : 1));
+  if (PX > 8) PX = 8;
+  if (PX < 1) PX = 1;
+  const long long n_main = (((long long)g.Ho * g.Wo + PX - 1) / PX) * g.Nt;
   const long long n_scales = (long long)g.Ho * g.Wo * g.Nt * taps * g.Ct;
   count_launches(1);
   if (J <= IC_MAX_J && src_chunks < 0x7fffffffLL && n_main < 0x7fff0000LL) {
     long long sc_blocks = (n_scales + IC_THREADS - 1) / IC_THREADS;
     if (sc_blocks > 148 * 4) sc_blocks = 148 * 4;
     if (sc_blocks < 1) sc_blocks = 1;
-    im2col_kernel<<<(unsigned)(n_main + sc_blocks), IC_THREADS, 0, s>>>(a, rc, (int)J, (unsigned)n_main);
+    im2col_kernel<<<(unsigned)(n_main + sc_blocks), IC_THREADS, 0, s>>>(a, rc, (int)J, PX, (unsigned)n_main);
     return cudaGetLastError();
   }
   const long long code_chunks = (long long)g.Ho * g.Wo * g.N * J;

@@ -24,6 +24,13 @@
 namespace mq {
 namespace {
 using namespace tc;
+#ifdef MQ_TC_PROFILE
+__device__ unsigned long long g_wblk[160][6];   // per block: start, after setup, producer done, MMA done, epilogue done, SM id
+__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
+#define WPROF(slot) do { if (blockIdx.x < 160) g_wblk[blockIdx.x][slot] = gtime(); } while (0)
+#else
+#define WPROF(slot) do { } while (0)
+#endif
 
 constexpr int WG_THREADS = 256;
 
@@ -42,10 +49,10 @@ __device__ __forceinline__ void stage_block(const WgradTcParams& p, int st, int 
 
 // ---- scale expansion: one warp per 512*SPA-byte chunk ----------------------------------------------------
 template <bool FP4>
-__global__ void __launch_bounds__(256) expand_wgrad_scales_kernel(const WgradTcParams p) {
+__device__ __forceinline__ void expand_wgrad_scales_body(const WgradTcParams& p, unsigned block) {
   constexpr int SPA = FP4 ? 2 : 1, NBS = 4 * SPA;
   const int lane = threadIdx.x & 31;
-  const long long wid = (long long)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const long long wid = (long long)block * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int taps = p.Kh * p.Kw;
   const long long nA = (long long)p.m_tiles * p.stages_total;
   const int groups = taps / p.TG;
@@ -103,9 +110,14 @@ __global__ void __launch_bounds__(256) expand_wgrad_scales_kernel(const WgradTcP
 // shifted by one pixel (one piece) per tap, so a stage loads KPX + Kw - 1 pieces of X once and the stage's G_Y
 // tile feeds Kw accumulators (Kw times less shared-memory traffic per FLOP than one tap per block).
 template <bool FP4>
+__global__ void __launch_bounds__(256) expand_wgrad_scales_kernel(const WgradTcParams p) { expand_wgrad_scales_body<FP4>(p, blockIdx.x); }
+
+template <bool FP4>
 __global__ void __launch_bounds__(WG_THREADS, 1)
-wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const WgradTcParams p) {
+wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_p,
+                const WgradTcParams p) {
   constexpr int SPA = FP4 ? 2 : 1;     // scale bytes per MMA per row
+  if (threadIdx.x == 0) WPROF(0);
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int TG = p.TG;
@@ -141,12 +153,14 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     *abort_flag = 0;
     mbar_fence_init();
     if (p.mode != MQ_WG_FP4_FLAT) { prefetch_tensormap(&map_a); prefetch_tensormap(&map_b); }
+    prefetch_tensormap(&map_p);
   }
   if (warp == 1) { tmem_alloc(tmem_slot, p.tmem_cols); tmem_relinquish(); }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
+  if (threadIdx.x == 0) WPROF(1);
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
@@ -196,6 +210,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         }
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
+      WPROF(2);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -248,6 +263,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
       if (nst > 0) tc_commit(tfull); else mbar_arrive(tfull);
+      WPROF(3);
     }
   } else if (warp == 2) {
     // ------------------------------------------------------------------ scale copier (smem -> per-stage TMEM buffers)
@@ -263,6 +279,9 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         tc_fence_after_sync();
         const uint32_t so = s * stage16;
         const uint32_t sf_t = sf_base + s * sf_cols;
+#ifdef MQ_WG_SKIPCP
+        if (i >= p.stages) { tc_commit(&sffull[s]); if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; } continue; }
+#endif
 #pragma unroll
         for (int g = 0; g < SPA; ++g) tmem_cp_32x128b_warpx4(sf_t + 4 * g, sf_desc0 + so + g * 32);
 #pragma unroll 1
@@ -276,42 +295,59 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     }
   } else if (warp >= 4) {
     // ------------------------------------------------------------------ epilogue: partial sums to scratch
+    // Each warp moves its 32 rows, 32 columns at a time: TMEM -> registers -> a [32 rows][128 bytes] staging tile
+    // (128-byte swizzle, so the 16-byte writes of a row do not collide) -> one TMA store into the partial-sum
+    // tensor (columns, rows, split): coalesced lines, clipped at C_out.  The pipeline's shared memory is free by
+    // now (tfull fires after the last MMA) and serves as staging, two tiles per warp.
     const int quad = warp & 3;
-    const int r = 32 * quad + lane;
     bool ok = true;
     if (lane == 0) ok = mbar_wait(tfull, 0, p.status, MQ_ERR_TIMEOUT);
     ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
     if (ok) {
       tc_fence_after_sync();
-      const int co = co0 + r;
-      const long long J = (long long)p.Kh * p.Kw * p.Cp;
       const int ncols = min(p.b_rows, p.Cp - ci0);
+      uint8_t* stg = smem + quad * (2 * 4096);
+      uint32_t nbuf = 0;
 #pragma unroll 1
       for (int j = 0; j < TG; ++j) {
-        float* out = p.partial + ((long long)split * p.Cout + co) * J + (long long)(tap0 + j) * p.Cp + ci0;
+        const int col0 = (tap0 + j) * p.Cp + ci0;
         const uint32_t taddr = tmem + (uint32_t)(j * p.b_rows) + ((uint32_t)(32 * quad) << 16);
 #pragma unroll 1
-        for (int c = 0; c < ncols; c += 16) {
-          uint32_t v[16];
+        for (int c = 0; c < ncols; c += 32, ++nbuf) {
+          uint32_t v[2][16];
           if (nst > 0) {
-            tmem_ld_32x32b_x16(taddr + c, v);
+            tmem_ld_32x32b_x16(taddr + c, v[0]);
+            tmem_ld_32x32b_x16(taddr + c + 16, v[1]);
             tmem_ld_wait();
           } else {
 #pragma unroll
-            for (int q = 0; q < 16; ++q) v[q] = 0u;
+            for (int q = 0; q < 16; ++q) { v[0][q] = 0u; v[1][q] = 0u; }
           }
-          if (co < p.Cout) {
+          uint8_t* buf = stg + (nbuf & 1) * 4096;
+          if (lane == 0) bulk_wait_group_read<1>();      // the store that used this buffer two tiles ago has read it
+          __syncwarp();
 #pragma unroll
-            for (int q = 0; q < 16; q += 4)   // Cp is a multiple of 32: whole float4s
-              *reinterpret_cast<float4*>(out + c + q) = make_float4(__uint_as_float(v[q]), __uint_as_float(v[q + 1]), __uint_as_float(v[q + 2]), __uint_as_float(v[q + 3]));
+          for (int h = 0; h < 2; ++h)
+#pragma unroll
+            for (int q = 0; q < 4; ++q)                  // 16-byte unit 4h + q of row `lane`
+              *reinterpret_cast<uint4*>(buf + lane * 128 + (((4 * h + q) ^ (lane & 7)) << 4)) = make_uint4(v[h][4 * q], v[h][4 * q + 1], v[h][4 * q + 2], v[h][4 * q + 3]);
+          fence_proxy_async_smem();
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_3d(&map_p, buf, col0 + c, co0 + 32 * quad, split);
+            bulk_commit_group();
           }
         }
       }
+      if (lane == 0) bulk_wait_group_all();
     }
   }
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem, p.tmem_cols);
+#ifdef MQ_TC_PROFILE
+  if (threadIdx.x == 0) { WPROF(4); unsigned smid; asm volatile("mov.u32 %0, %smid;" : "=r"(smid)); if (blockIdx.x < 160) g_wblk[blockIdx.x][5] = smid; }
+#endif
 }
 
 // ---- E2M1 re-layout: stored [pixel][n][Cp] nibbles -> [pixel][Cp][Npad] nibbles (n fastest, zero for n >= N) ----
@@ -349,54 +385,78 @@ __global__ void __launch_bounds__(256) fp4_to_n_major_kernel(const uint8_t* __re
 }
 
 // ---- E2M1 re-layout for the flat mode (see launch_fp4_to_flat) -------------------------------------------------
-// One block: 8 output pixels x 32 samples x 64 channels.
-__global__ void __launch_bounds__(256) fp4_to_flat_kernel(const uint8_t* __restrict__ in, uint8_t* __restrict__ out, int Hs, int Ws, int N, int Cs_p,
-                                                           int P_out, int Wp, int off_h, int off_w, int rows, int nblocks, int KBn) {
-  __shared__ uint8_t t[8][32][65];
-  const int q0 = blockIdx.x * 8, n0 = blockIdx.y * 32, c0 = blockIdx.z * 64;
-  const int tid = threadIdx.x;
-  for (int i = tid; i < 512; i += 256) {
-    const int px = i >> 6, n = (i >> 1) & 31, half = i & 1;
-    const int q = q0 + px;
-    const int hq = q / Wp, wq = q - hq * Wp;
-    const int h = hq - off_h, w = wq - off_w;
-    uint4 v = make_uint4(0, 0, 0, 0);
-    if (q < P_out && h >= 0 && h < Hs && w >= 0 && w < Ws && n0 + n < N && c0 + 32 * half < Cs_p)
-      v = *reinterpret_cast<const uint4*>(in + ((((long long)h * Ws + w) * N + n0 + n) * Cs_p + c0 + 32 * half) / 2);
-    const uint32_t wd[4] = {v.x, v.y, v.z, v.w};
+// One warp per (output pixel, 32-sample block, 64 channels): 1 KB in, 1 KB out, transposed in registers.  Lane
+// (k, ng) = (lane & 7, lane >> 3) reads the 32-bit word of channels 8k..8k+7 for samples 8ng..8ng+7, swaps the
+// 8 x 8 nibble block in three butterfly steps, and writes word ng of the 16-byte sample run of channels 8k..8k+7.
+__device__ __forceinline__ void nibble_transpose_8x8(uint32_t (&w)[8]) {
 #pragma unroll
-    for (int k = 0; k < 4; ++k)
+  for (int a = 0; a < 8; a += 2) { const uint32_t x = ((w[a] >> 4) ^ w[a + 1]) & 0x0F0F0F0Fu; w[a + 1] ^= x; w[a] ^= x << 4; }
 #pragma unroll
-      for (int b = 0; b < 8; ++b) t[px][n][32 * half + 8 * k + b] = (uint8_t)((wd[k] >> (4 * b)) & 0xF);
-  }
-  __syncthreads();
+  for (int a = 0; a < 8; ++a)
+    if ((a & 2) == 0) { const uint32_t x = ((w[a] >> 8) ^ w[a + 2]) & 0x00FF00FFu; w[a + 2] ^= x; w[a] ^= x << 8; }
+#pragma unroll
+  for (int a = 0; a < 4; ++a) { const uint32_t x = ((w[a] >> 16) ^ w[a + 4]) & 0x0000FFFFu; w[a + 4] ^= x; w[a] ^= x << 16; }
+}
+
+struct FlatArgs {
+  const uint8_t* in; uint8_t* out;
+  int Hs, Ws, N, Cs_p, P_out, Wp, off_h, off_w, rows, nblocks, KBn, ncg;
+  unsigned units, blocks;
+};
+__device__ __forceinline__ void fp4_to_flat_body(const FlatArgs& fa, unsigned block, unsigned nblocks_grid) {
+  const uint8_t* __restrict__ in = fa.in; uint8_t* __restrict__ out = fa.out;
+  const int Hs = fa.Hs, Ws = fa.Ws, N = fa.N, Cs_p = fa.Cs_p, P_out = fa.P_out, Wp = fa.Wp, off_h = fa.off_h, off_w = fa.off_w;
+  const int rows = fa.rows, nblocks = fa.nblocks, KBn = fa.KBn, ncg = fa.ncg;
+  const unsigned units = fa.units;
+  const int lane = threadIdx.x & 31;
+  const int k = lane & 7, ng = lane >> 3;
+  const int nbk = KBn >> 4;                        // 32-sample blocks per pixel
   const int cmax = nblocks * rows;
-  for (int i = tid; i < 512; i += 256) {
-    const int px = i >> 6, c = i & 63;
-    const int q = q0 + px, cc = c0 + c;
-    if (cc < cmax && q < P_out) {
-      uint32_t wd[4];
+  const unsigned per_q = (unsigned)(ncg * nbk);
+  for (unsigned u = block * 8u + (threadIdx.x >> 5); u < units; u += nblocks_grid * 8u) {
+    const unsigned q = u / per_q, rem = u - q * per_q;
+    const int nb = (int)(rem / (unsigned)ncg), cg = (int)(rem - (unsigned)nb * ncg);
+    const int hq = (int)(q / (unsigned)Wp), wq = (int)q - hq * Wp;
+    const int h = hq - off_h, w = wq - off_w;
+    const int c0 = cg * 64 + 8 * k;                // this lane's 8 channels
+    uint32_t wd[8];
+    const bool pix_ok = h >= 0 && h < Hs && w >= 0 && w < Ws && c0 < Cs_p;
+    const uint8_t* src = in + ((((long long)h * Ws + w) * N + nb * 32 + 8 * ng) * Cs_p + c0) / 2;
 #pragma unroll
-      for (int k = 0; k < 4; ++k) {
-        uint32_t acc = 0;
+    for (int j = 0; j < 8; ++j) {
+      wd[j] = 0u;
+      if (pix_ok && nb * 32 + 8 * ng + j < N) wd[j] = __ldg(reinterpret_cast<const uint32_t*>(src + (long long)j * (Cs_p / 2)));
+    }
+    nibble_transpose_8x8(wd);                       // wd[i]: channel c0 + i, samples 8ng .. 8ng + 7
+    if (c0 < cmax) {                                // rows is a multiple of 32: the lane's 8 channels share a block
+      const int blk = c0 / rows, r0 = c0 - blk * rows;
+      uint8_t* dst = out + (((long long)blk * P_out + q) * rows + r0) * KBn + 4 * ng;
 #pragma unroll
-        for (int b = 0; b < 8; ++b) acc |= (uint32_t)t[px][8 * k + b][c] << (4 * b);
-        wd[k] = acc;
+      for (int i = 0; i < 8; ++i) {
+        const int r = r0 + i;
+        const int sw = KBn == 128 ? (r & 7) : (KBn == 64 ? ((r >> 1) & 3) : (KBn == 32 ? ((r >> 2) & 1) : 0));
+        *reinterpret_cast<uint32_t*>(dst + (long long)i * KBn + ((nb ^ sw) << 4)) = wd[i];
       }
-      const int blk = cc / rows, r = cc - blk * rows;
-      const int chunk = n0 >> 5;   // 16-byte chunk of the row
-      const int sw = KBn == 128 ? (r & 7) : (KBn == 64 ? ((r >> 1) & 3) : (KBn == 32 ? ((r >> 2) & 1) : 0));
-      const long long off = (((long long)blk * P_out + q) * rows + r) * KBn + ((chunk ^ sw) << 4);
-      *reinterpret_cast<uint4*>(out + off) = make_uint4(wd[0], wd[1], wd[2], wd[3]);
     }
   }
 }
 
+// Preparation of the flat mode in one launch: blocks [0, x.blocks) re-lay X, the next g.blocks re-lay G_Y, the rest
+// expand the scale chunks.
+__global__ void __launch_bounds__(256) wgrad_flat_prep_kernel(const FlatArgs x, const FlatArgs gy, const WgradTcParams p) {
+  if (blockIdx.x < x.blocks) fp4_to_flat_body(x, blockIdx.x, x.blocks);
+  else if (blockIdx.x < x.blocks + gy.blocks) fp4_to_flat_body(gy, blockIdx.x - x.blocks, gy.blocks);
+  else expand_wgrad_scales_body<true>(p, blockIdx.x - x.blocks - gy.blocks);
+}
+
 }  // namespace
 
+#ifdef MQ_TC_PROFILE
+extern "C" int mqdbg_read_wblk(unsigned long long* out960) { return cudaMemcpyFromSymbol(out960, g_wblk, sizeof(unsigned long long) * 960) == cudaSuccess ? 0 : 1; }
+#endif
 size_t wgrad_tc_smem_bytes(const WgradTcParams& p) { return 1024 + (size_t)p.stages * p.stage_bytes + (3 * (size_t)p.stages + 2) * 8 + 64; }
 
-cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s) {
+cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_p, cudaStream_t s) {
   static bool attr_set[2] = {false, false};
   const size_t smem = wgrad_tc_smem_bytes(p);
   const int f = p.mode == MQ_WG_FP8 ? 0 : 1;
@@ -407,8 +467,8 @@ cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, co
     attr_set[f] = true;
   }
   const unsigned grid = (unsigned)(p.m_tiles * p.j_tiles * p.splits);
-  if (f) wgrad_tc_kernel<true><<<grid, WG_THREADS, smem, s>>>(map_a, map_b, p);
-  else wgrad_tc_kernel<false><<<grid, WG_THREADS, smem, s>>>(map_a, map_b, p);
+  if (f) wgrad_tc_kernel<true><<<grid, WG_THREADS, smem, s>>>(map_a, map_b, map_p, p);
+  else wgrad_tc_kernel<false><<<grid, WG_THREADS, smem, s>>>(map_a, map_b, map_p, p);
   count_launches(1);
   return cudaGetLastError();
 }
@@ -429,10 +489,29 @@ cudaError_t launch_fp4_to_n_major(const uint8_t* in, uint8_t* out, int P, int N,
   return cudaGetLastError();
 }
 
-cudaError_t launch_fp4_to_flat(const uint8_t* in, uint8_t* out, int Hs, int Ws, int N, int Cs_p, int P_out, int Wp, int off_h, int off_w,
-                               int rows, int nblocks, int KBn, cudaStream_t s) {
-  dim3 grid((P_out + 7) / 8, KBn / 16, (nblocks * rows + 63) / 64);
-  fp4_to_flat_kernel<<<grid, 256, 0, s>>>(in, out, Hs, Ws, N, Cs_p, P_out, Wp, off_h, off_w, rows, nblocks, KBn);
+static bool make_flat_args(FlatArgs* fa, const uint8_t* in, uint8_t* out, int Hs, int Ws, int N, int Cs_p, int P_out, int Wp, int off_h, int off_w, int rows,
+                           int nblocks, int KBn) {
+  fa->in = in; fa->out = out; fa->Hs = Hs; fa->Ws = Ws; fa->N = N; fa->Cs_p = Cs_p; fa->P_out = P_out; fa->Wp = Wp; fa->off_h = off_h; fa->off_w = off_w;
+  fa->rows = rows; fa->nblocks = nblocks; fa->KBn = KBn;
+  fa->ncg = (nblocks * rows + 63) / 64;
+  const long long units = (long long)P_out * (KBn / 16) * fa->ncg;
+  if (units >= 0xffffffffLL) return false;
+  fa->units = (unsigned)units;
+  long long blocks = (units + 7) / 8;
+  if (blocks > 148LL * 32) blocks = 148LL * 32;
+  if (blocks < 1) blocks = 1;
+  fa->blocks = (unsigned)blocks;
+  return true;
+}
+
+cudaError_t launch_wgrad_flat_prep(const WgradTcParams& p, const uint8_t* x_codes, uint8_t* xt, int P_b, const uint8_t* g_codes, uint8_t* gt, int P_a,
+                                   cudaStream_t s) {
+  FlatArgs fx, fg;
+  if (!make_flat_args(&fx, x_codes, xt, p.H, p.W, p.N, p.Cp, P_b, p.Wp, p.ph, p.pw, p.b_rows, p.cb_tiles, p.KBn)) return cudaErrorInvalidValue;
+  if (!make_flat_args(&fg, g_codes, gt, p.Ho, p.Wo, p.N, p.Cot * 32, P_a, p.Wp, 0, 0, 128, p.m_tiles, p.KBn)) return cudaErrorInvalidValue;
+  const long long warps = (long long)p.m_tiles * p.stages_total + (long long)p.cb_tiles * (p.Kh * p.Kw / p.TG) * p.stages_total * p.NB;
+  const unsigned sc_blocks = (unsigned)((warps + 7) / 8);
+  wgrad_flat_prep_kernel<<<fx.blocks + fg.blocks + sc_blocks, 256, 0, s>>>(fx, fg, p);
   count_launches(1);
   return cudaGetLastError();
 }
