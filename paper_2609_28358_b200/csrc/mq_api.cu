@@ -77,21 +77,25 @@ size_t wt_codes_bytes(const Geom& g, int fmt_w) {
 }
 size_t up256(size_t v) { return (v + 255) / 256 * 256; }
 
-// Output columns per tile.  Rows of a tile are TW consecutive output columns x TN = 128/TW samples with
-// the column index fastest, so an NCHW store writes runs of TW floats; TW >= 8 fills 32-byte sectors.
-int choose_tw(int w_eff, int N, int layout, bool wide) {
+// Output columns per tile.  Rows of a tile are TW consecutive output columns x TN = 128/TW samples with the
+// column index fastest.  An NCHW store writes runs of TW floats and the store path is bound by the NUMBER of
+// runs (about 2.2 cycles each per SM, measured), so the choice weighs the tile's MMA time against its store time
+// and both against the padding the tile shape wastes at the edges.
+//   k_bytes: bytes of K per tile row (taps x channel bytes); bn: output channels per tile.
+int choose_tw(int w_eff, int N, int layout, double k_bytes, int bn, bool thin) {
   const int forced = env_int("MQ_TC_TW", 0);
   if (forced > 0) return forced;
+  if (thin) return 8;   // the whole-tile kernel (8-column tiles): its per-tile loads beat any per-tap shape on thin layers
+  const double t_mma = k_bytes / 32.0 * 107.0 * (bn / 128.0 < 0.5 ? 0.5 : bn / 128.0);
   int best = 1;
   double best_cost = 1e30;
   for (int tw = 1; tw <= 32; tw *= 2) {
     const int tn = 128 / tw;
     const double waste = (double)((w_eff + tw - 1) / tw * tw) / w_eff * (double)((N + tn - 1) / tn * tn) / N;
-    double pen = 1.0;
-    if (layout == MQ_NCHW) pen = tw >= 8 ? 1.0 : (tw == 4 ? 1.25 : (tw == 2 ? 1.8 : 2.5));
-    if (layout == MQ_NCHW && wide && env_int("MQ_TC_WIDE", 0)) pen = tw >= 32 ? 1.0 : (tw == 16 ? 1.05 : (tw == 8 ? 1.2 : pen * 1.2));
-    const double cost = waste * pen;
-    if (cost < best_cost - 1e-9) { best_cost = cost; best = tw; }
+    double t_store = 128.0 * (bn * 4.0 / 128.0) * 2.2;          // [H][W][N][C] output: whole lines
+    if (layout == MQ_NCHW) t_store = 128.0 * bn / tw * 2.2 * (tw < 8 ? 8.0 / tw : 1.0);   // runs below a 32-byte sector cost a sector each
+    double cost = waste * (t_mma > t_store ? t_mma : t_store);
+    if (cost < best_cost * (1.0 - 1e-9)) { best_cost = cost; best = tw; }
   }
   return best;
 }
@@ -128,8 +132,12 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   p.G = 128 / p.KB;
   p.cpt = rowbytes / p.KB;
   const int w_eff = op == MQ_OP_FWD ? g.Wo : (g.W + g.sw - 1) / g.sw;
-  const bool thin = g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && g.Kw > 1;
-  p.TW = choose_tw(w_eff, g.N, layout, thin && !env_int("MQ_TC_NO_HALO", 0));
+  const bool thin = g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && !env_int("MQ_TC_NO_HALO", 0);
+  {
+    const int cd16_ = (p.Cd + 15) / 16 * 16;
+    const int nkh_ = op == MQ_OP_FWD ? g.Kh : (g.Kh + g.sh - 1) / g.sh, nkw_ = op == MQ_OP_FWD ? g.Kw : (g.Kw + g.sw - 1) / g.sw;
+    p.TW = choose_tw(w_eff, g.N, layout, (double)nkh_ * nkw_ * rowbytes, cd16_ < 128 ? cd16_ : 128, thin);
+  }
   if (p.TW < 1 || p.TW > 32 || (p.TW & (p.TW - 1))) return false;
   p.TN = 128 / p.TW;
   p.lgTW = 0;
@@ -156,8 +164,12 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
     p.m_sh = magic(g.sh); p.m_sw = magic(g.sw);
     if (!exact) return false;
   }
+  // NCHW output through TMA stores (unit-stride output columns, rows of 16-byte multiples): worth its 64 KB of
+  // staging only in the whole-tile kernel, whose pipeline is short; the per-tap kernel keeps its stages
+  const bool tma_store_ok = layout == MQ_NCHW && p.Wd % 4 == 0 && p.TW >= 4 && p.TW <= 32 && (op == MQ_OP_FWD || (g.sh == 1 && g.sw == 1));
+  p.tma_store = tma_store_ok && env_int("MQ_TC_TMA_STORE", 0) ? 1 : 0;
   const size_t stage_bytes = 128 * 128 + (size_t)p.BN * 128 + 3072;
-  int stages = (int)((227 * 1024 - 2048) / stage_bytes);
+  int stages = (int)((227 * 1024 - 2048 - (p.tma_store ? 65536 : 0)) / stage_bytes);
   if (stages > 8) stages = 8;
   if (stages < 2) return false;
   p.stages = stages;
@@ -184,14 +196,14 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
       p.halo_a_bytes = (nbox * p.halo_box_bytes + 1023) / 1024 * 1024;
       p.halo_stage_bytes = (p.halo_a_bytes + p.max_stages * 512 * spa + 1023) / 1024 * 1024;
       p.halo_b_bytes = (taps * p.BN * p.KB + p.max_stages * 512 * spa * atoms_b + 1023) / 1024 * 1024;
-      // NCHW output through TMA stores: rows of the output must be 16-byte multiples
-      p.tma_store = layout == MQ_NCHW && p.Wd % 4 == 0 && p.TW >= 4 && p.TW <= 32 && !env_int("MQ_TC_NO_TMA_STORE", 0);
-      int hst = (227 * 1024 - 4096 - p.halo_b_bytes - (p.tma_store ? 65536 : 0)) / p.halo_stage_bytes;
+      const int halo_tma = tma_store_ok && !env_int("MQ_TC_NO_TMA_STORE", 0) ? 1 : 0;
+      int hst = (227 * 1024 - 4096 - p.halo_b_bytes - (halo_tma ? 65536 : 0)) / p.halo_stage_bytes;
       if (hst > 4) hst = 4;
       // TMEM: accumulator(s), 16 columns per chunk of resident weight scales, 8 per chunk per stage
       while (hst >= 2 && p.BN + 16 * p.max_stages + 8 * p.max_stages * hst > 512) --hst;
       if (hst >= 2 && p.WH <= 256 && (p.halo_box_bytes % 1024 == 0 || nbox == 1)) {
         p.halo = 1;
+        p.tma_store = halo_tma;
         p.fused = p.tiles_c == 1 && p.TN <= 32 && g.Kh * (p.TW + g.Kw - 1) * (p.KB / 32) * spa <= 128 && !env_int("MQ_TC_NO_FUSED", 0);
         p.stages = hst;
         p.n_acc = (2 * p.BN + 16 * p.max_stages + 8 * p.max_stages * hst <= 512) ? 2 : 1;
@@ -244,7 +256,7 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
   p.out = out; p.out_layout = env_int("MQ_TC_SKIP_STORE", 0) ? 99 : layout; p.status = status;
   if (!(p.halo && p.fused) && launch_expand_conv_scales(p, stream) != cudaSuccess) return MQ_ERR_CUDA;
 
-  CUtensorMap map_a, map_b, map_w;
+  CUtensorMap map_a, map_w;
   {
     const uint64_t rb = (uint64_t)pl.rowbytes;
     const uint64_t dims[4] = {rb, (uint64_t)p.Ws, (uint64_t)g.N, (uint64_t)p.Hs};
@@ -256,35 +268,35 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
     if (!encode_tensor_map_u8(&map_a, qx_like->codes, 4, dims, strides, box, es, p.KB)) return MQ_ERR_CUDA;
   }
   map_w = map_a;
-  if (p.halo && p.fused) {
-    // all taps of the weight tile in one box: dims ordered (channel bytes, rows, taps)
-    const uint64_t rb = (uint64_t)pl.rowbytes;
-    const uint64_t dims[3] = {rb, (uint64_t)pl.rows_b, (uint64_t)taps};
-    const uint64_t strides[2] = {(uint64_t)taps * rb, rb};
-    const uint32_t box[3] = {(uint32_t)p.KB, (uint32_t)p.BN, (uint32_t)taps};
-    if (!encode_tensor_map_u8(&map_w, b_codes, 3, dims, strides, box, nullptr, p.KB)) return MQ_ERR_CUDA;
-  }
   if (p.halo) {
-    map_b = map_a;   // the weight tile comes as a pre-swizzled image by bulk copy; the second map is the output's
-    if (p.tma_store) {
-      if (reinterpret_cast<uintptr_t>(out) % 16 != 0) p.tma_store = 0;
-      else {
-        const uint64_t dims[4] = {(uint64_t)p.Wd, (uint64_t)g.N, (uint64_t)p.Cd, (uint64_t)p.Hd};
-        const uint64_t strides[3] = {(uint64_t)p.Cd * p.Hd * p.Wd * 4, (uint64_t)p.Hd * p.Wd * 4, (uint64_t)p.Wd * 4};
-        // one epilogue warp's 32 rows x the channels of a column half (at most 64)
-        const int half_cols = (p.BN / 2 + 15) & ~15;
-        const uint32_t box[4] = {(uint32_t)p.TW, (uint32_t)(32 / p.TW), (uint32_t)(half_cols < 64 ? half_cols : 64), 1u};
-        if (!encode_tensor_map_u8(&map_b, out, 4, dims, strides, box, nullptr, 0, true)) return MQ_ERR_CUDA;
-      }
+    if (p.fused) {
+      // all taps of the weight tile in one box: dims ordered (channel bytes, rows, taps)
+      const uint64_t rb = (uint64_t)pl.rowbytes;
+      const uint64_t dims[3] = {rb, (uint64_t)pl.rows_b, (uint64_t)taps};
+      const uint64_t strides[2] = {(uint64_t)taps * rb, rb};
+      const uint32_t box[3] = {(uint32_t)p.KB, (uint32_t)p.BN, (uint32_t)taps};
+      if (!encode_tensor_map_u8(&map_w, b_codes, 3, dims, strides, box, nullptr, p.KB)) return MQ_ERR_CUDA;
     }
   } else {
     const uint64_t rb = (uint64_t)pl.rowbytes;
     const uint64_t dims[3] = {rb, (uint64_t)taps, (uint64_t)pl.rows_b};
     const uint64_t strides[2] = {rb, (uint64_t)taps * rb};
     const uint32_t box[3] = {(uint32_t)p.KB, 1u, (uint32_t)p.BN};
-    if (!encode_tensor_map_u8(&map_b, b_codes, 3, dims, strides, box, nullptr, p.KB)) return MQ_ERR_CUDA;
+    if (!encode_tensor_map_u8(&map_w, b_codes, 3, dims, strides, box, nullptr, p.KB)) return MQ_ERR_CUDA;
   }
-  return launch_conv_tc(p, map_a, map_b, map_w, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
+  CUtensorMap map_out = map_a;
+  if (p.tma_store) {
+    if (reinterpret_cast<uintptr_t>(out) % 16 != 0) p.tma_store = 0;
+    else {
+      // the output seen as (W, N, C, H); one epilogue warp's 32 rows x the channels of a column half (at most 64)
+      const uint64_t dims[4] = {(uint64_t)p.Wd, (uint64_t)g.N, (uint64_t)p.Cd, (uint64_t)p.Hd};
+      const uint64_t strides[3] = {(uint64_t)p.Cd * p.Hd * p.Wd * 4, (uint64_t)p.Hd * p.Wd * 4, (uint64_t)p.Wd * 4};
+      const int half_cols = (p.BN / 2 + 15) & ~15;
+      const uint32_t box[4] = {(uint32_t)p.TW, (uint32_t)(32 / p.TW), (uint32_t)(half_cols < 64 ? half_cols : 64), 1u};
+      if (!encode_tensor_map_u8(&map_out, out, 4, dims, strides, box, nullptr, 0, true)) return MQ_ERR_CUDA;
+    }
+  }
+  return launch_conv_tc(p, map_a, map_w, map_out, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }
 
 // ---- weight gradient on tensor cores ---------------------------------------------------------------

@@ -276,7 +276,8 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
 
 template <int MODE, int KB, bool FP4>
 __global__ void __launch_bounds__(TC_THREADS, 1)
-conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const ConvTcParams p) {
+conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_out,
+               const ConvTcParams p) {
   constexpr int G = 128 / KB;          // chunks per stage
   constexpr int APC = KB / 32;         // MMA K-atoms (32 bytes) per chunk
   constexpr int SPA = FP4 ? 2 : 1;     // scale bytes per atom
@@ -287,7 +288,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int b_stage_bytes = p.BN * 128;
   const int stage_bytes = A_STAGE_BYTES + b_stage_bytes + SFA_BYTES + SFB_BYTES;
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * stage_bytes);
+  float* staging = reinterpret_cast<float*>(smem + (size_t)p.stages * stage_bytes);   // TMA-store epilogue only
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * stage_bytes + (p.tma_store ? EPI_STAGING_BYTES : 0));
   uint64_t* empty = full + p.stages;
   uint64_t* sffull = empty + p.stages;     // scale vectors of the stage have landed in TMEM
   uint64_t* tfull = sffull + p.stages;
@@ -306,6 +308,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     mbar_fence_init();
     prefetch_tensormap(&map_a);
     prefetch_tensormap(&map_b);
+    if (p.tma_store) prefetch_tensormap(&map_out);
   }
   if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
   tc_fence_before_sync();
@@ -434,7 +437,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else if (warp >= 4) {
-    epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
+    if (p.tma_store) epilogue_tma_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total);
+    else epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
   }
   // teardown: everyone meets here (all loops are bounded), then the allocating warp frees TMEM
   tc_fence_before_sync();
@@ -1000,11 +1004,11 @@ bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const ui
 
 size_t conv_tc_smem_bytes(const ConvTcParams& p) {
   const size_t stage = A_STAGE_BYTES + (size_t)p.BN * 128 + SFA_BYTES + SFB_BYTES;
-  return 1024 + (size_t)p.stages * stage + (3 * (size_t)p.stages + 4) * 8 + 64;
+  return 1024 + (size_t)p.stages * stage + (p.tma_store ? EPI_STAGING_BYTES : 0) + (3 * (size_t)p.stages + 4) * 8 + 64;
 }
 
 template <int MODE, int KB, bool FP4>
-cudaError_t launch_conv_tc_inst(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, cudaStream_t s) {
+cudaError_t launch_conv_tc_inst(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_out, cudaStream_t s) {
   static bool attr_set = false;
   const size_t smem = conv_tc_smem_bytes(p);
   if (!attr_set) {
@@ -1016,7 +1020,7 @@ cudaError_t launch_conv_tc_inst(const ConvTcParams& p, const CUtensorMap& map_a,
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const unsigned grid = (unsigned)(p.total_tiles < sms ? p.total_tiles : sms);
-  conv_tc_kernel<MODE, KB, FP4><<<grid, TC_THREADS, smem, s>>>(map_a, map_b, p);
+  conv_tc_kernel<MODE, KB, FP4><<<grid, TC_THREADS, smem, s>>>(map_a, map_b, map_out, p);
   count_launches(1);
   return cudaGetLastError();
 }
@@ -1073,16 +1077,16 @@ cudaError_t launch_conv_tc_halo_inst(const ConvTcParams& p, const CUtensorMap& m
   return launch_conv_tc_halo_taps<MODE, KB, FP4, 0>(p, map_a, map_b, map_w, s);
 }
 
-cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_w, cudaStream_t s) {
+cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_out, cudaStream_t s) {
   if (p.total_tiles <= 0 || p.total_tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
   if (p.halo) {
-#define MQ_TC_HCASE(M, K, F) if (p.mode == M && p.KB == K && (p.kind_fp4 != 0) == F) return launch_conv_tc_halo_inst<M, K, F>(p, map_a, map_b, map_w, s)
+#define MQ_TC_HCASE(M, K, F) if (p.mode == M && p.KB == K && (p.kind_fp4 != 0) == F) return launch_conv_tc_halo_inst<M, K, F>(p, map_a, map_out, map_w, s)
     MQ_TC_HCASE(MQ_OP_FWD, 64, false); MQ_TC_HCASE(MQ_OP_FWD, 32, false); MQ_TC_HCASE(MQ_OP_FWD, 64, true); MQ_TC_HCASE(MQ_OP_FWD, 32, true);
     MQ_TC_HCASE(MQ_OP_BWD_DATA, 64, false); MQ_TC_HCASE(MQ_OP_BWD_DATA, 32, false); MQ_TC_HCASE(MQ_OP_BWD_DATA, 64, true); MQ_TC_HCASE(MQ_OP_BWD_DATA, 32, true);
 #undef MQ_TC_HCASE
     return cudaErrorInvalidValue;
   }
-#define MQ_TC_CASE(M, K, F) if (p.mode == M && p.KB == K && (p.kind_fp4 != 0) == F) return launch_conv_tc_inst<M, K, F>(p, map_a, map_b, s)
+#define MQ_TC_CASE(M, K, F) if (p.mode == M && p.KB == K && (p.kind_fp4 != 0) == F) return launch_conv_tc_inst<M, K, F>(p, map_a, map_w, map_out, s)
   MQ_TC_CASE(MQ_OP_FWD, 128, false); MQ_TC_CASE(MQ_OP_FWD, 64, false); MQ_TC_CASE(MQ_OP_FWD, 32, false);
   MQ_TC_CASE(MQ_OP_FWD, 128, true);  MQ_TC_CASE(MQ_OP_FWD, 64, true);  MQ_TC_CASE(MQ_OP_FWD, 32, true);
   MQ_TC_CASE(MQ_OP_BWD_DATA, 128, false); MQ_TC_CASE(MQ_OP_BWD_DATA, 64, false); MQ_TC_CASE(MQ_OP_BWD_DATA, 32, false);

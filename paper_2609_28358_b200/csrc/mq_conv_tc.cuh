@@ -52,7 +52,7 @@ struct ConvTcParams {
   int halo_b_bytes;         // bytes of the resident weight image + its scale chunks (rounded up to 1024)
   int fused;                // 1: single channel tile, stride 1: no preparation kernel (the blocks build the weight image, its
                             //    scale chunks and every tile's activation scale chunks themselves)
-  int tma_store;            // 1: NCHW output written by TMA stores from a staging buffer (the second tensor map is the output's)
+  int tma_store;            // 1: NCHW output written by TMA stores from per-warp staging slices
   const uint8_t* b_codes;   // weight-like codes [rows][taps][b_rowbytes] (source of the images below)
   int b_rows_total, b_rowbytes;
   uint8_t* b_img;           // [channel tile][tap][BN rows][KB], each row stored with the KB-byte swizzle applied
@@ -62,9 +62,10 @@ struct ConvTcParams {
   unsigned int* status;
 };
 
-// map_a: gathered activation codes.  map_b: weight codes per tap (per-tap kernel) or the fp32 output (whole-tile kernel
-// with TMA stores).  map_w: all taps of a weight tile in one box (whole-tile kernel, fused preparation).
-cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_w, cudaStream_t s);
+// map_a: gathered activation codes.  map_w: weight codes, one tap per box (per-tap kernel) or all taps of a tile in one
+// box (whole-tile kernel with fused preparation).  map_out: the fp32 NCHW output seen as (W, N, C, H), used when
+// p.tma_store is set.
+cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_out, cudaStream_t s);
 // Expands the compact tile scales into the per-stage scale-vector chunks the MMA reads (p.sfa_img, p.sfb_img).
 cudaError_t launch_expand_conv_scales(const ConvTcParams& p, cudaStream_t s);
 size_t conv_tc_sfa_bytes(const ConvTcParams& p);
