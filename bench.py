@@ -34,9 +34,18 @@ FMT_BITS = {0: 8, 1: 8, 2: 4}
 # nominal dense tensor-core ratio to bf16 for the operand formats of a GEMM
 TENSOR_RATIO = {8: 2.0, 4: 4.0}
 
-# dram__bytes_read.sum + dram__bytes_write.sum per launch from an ncu capture of the named kernel
-# on the named workload (see profiles/); None until a capture exists for that pair.
-NCU_TRAFFIC = {}
+# dram__bytes_read.sum + dram__bytes_write.sum per call from ncu captures of the call's kernels on the named
+# workload (profiles/*_config2.md), summed over the kernels one call launches.  Config 2's tensors are of the size
+# of the 126 MB L2, so part of every output is still cached when the kernel ends: these figures are below the
+# algorithmic bytes for the write-heavy calls and are kept as measured.
+NCU_TRAFFIC = {
+    ("config2", "quantize_x"): 52831488,
+    ("config2", "quantize_dy"): 111208960,
+    ("config2", "cbf_im2col"): 12299008,
+    ("config2", "conv_fwd"): 60308224,          # conv_tc_halo_kernel<fwd>
+    ("config2", "conv_bwd_data"): 17835264,     # conv_tc_halo_kernel<bwd_data>; weight_transpose_kernel not captured
+    ("config2", "conv_bwd_weight"): 19729152 + 26230016,   # wgrad_flat_prep_kernel + wgrad_tc_kernel; the reduce not captured
+}
 
 
 def workloads():
