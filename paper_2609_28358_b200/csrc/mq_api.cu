@@ -482,6 +482,13 @@ mq_status run_conv(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int r
 }
 
 }  // namespace
+
+bool pdl_enabled() {
+  static int v = -1;
+  if (v < 0) v = env_int("MQ_NO_PDL", 0) ? 0 : 1;
+  return v != 0;
+}
+
 }  // namespace mq
 
 using namespace mq;

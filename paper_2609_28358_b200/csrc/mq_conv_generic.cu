@@ -230,6 +230,7 @@ __global__ void __launch_bounds__(GT) bwd_weight_generic(ConvArgs a, int splits)
 // channels per thread, 16-byte loads); a block's four thread groups take every fourth split each and are
 // combined through shared memory in group order, so the result does not depend on scheduling.
 __global__ void __launch_bounds__(256) bwd_weight_reduce(const float* __restrict__ part, float* __restrict__ out, Geom g, int splits, int layout) {
+  pdl_wait();
   __shared__ float4 sh[3][64];
   const int taps = g.Kh * g.Kw;
   const int cq = g.Cp >> 2;                                   // float4 columns per (co, tap)
@@ -290,9 +291,8 @@ cudaError_t launch_bwd_weight_reduce(const float* partial, float* out, const Geo
   const long long quads = (long long)g.Cout * g.Kh * g.Kw * (g.Cp / 4);
   unsigned blocks = (unsigned)((quads + 63) / 64);
   if (blocks > 148u * 16) blocks = 148u * 16;
-  bwd_weight_reduce<<<blocks, 256, 0, s>>>(partial, out, g, splits, layout);
   count_launches(1);
-  return cudaGetLastError();
+  return launch_pdl(bwd_weight_reduce, dim3(blocks), dim3(256), 0, s, partial, out, g, splits, layout);
 }
 
 #define MQ_DISPATCH2(FA, FB, CALL)                                                         \

@@ -278,6 +278,7 @@ template <int MODE, int KB, bool FP4>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_out,
                const ConvTcParams p) {
+  pdl_wait();
   constexpr int G = 128 / KB;          // chunks per stage
   constexpr int APC = KB / 32;         // MMA K-atoms (32 bytes) per chunk
   constexpr int SPA = FP4 ? 2 : 1;     // scale bytes per atom
@@ -514,6 +515,7 @@ template <int MODE, int KB, bool FP4, int TAPS>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_w,
                     const ConvTcParams p) {
+  pdl_wait();
   constexpr int G = 128 / KB, APC = KB / 32, SPA = FP4 ? 2 : 1;
   constexpr int LAYOUT = KB == 128 ? 2 : (KB == 64 ? 4 : 6);
 #ifdef MQ_TC_PROFILE
@@ -812,6 +814,7 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 // chunks per (stride class, channel tile).
 template <int MODE, int KB, bool FP4>
 __global__ void __launch_bounds__(256) expand_conv_scales_kernel(const ConvTcParams p, unsigned n_tile_m) {
+  pdl_wait();
   constexpr int G = 128 / KB, APC = KB / 32, SPA = FP4 ? 2 : 1, BPC = APC * SPA;
   const int lane = threadIdx.x & 31;
   const unsigned wid = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -916,6 +919,7 @@ __global__ void __launch_bounds__(256) expand_conv_scales_kernel(const ConvTcPar
 // in:  [C_out][taps][C_in_p] codes;  out: [C_in_p][taps][C_out_p] codes (zero for c_out >= C_out)
 __global__ void weight_transpose_kernel(const uint8_t* __restrict__ in, uint8_t* __restrict__ out, const uint8_t* __restrict__ sc_in,
                                         uint8_t* __restrict__ sc_out, int Cout, int Cop, int Cp, int taps, int fp4) {
+  pdl_wait();
   __shared__ uint8_t tile[32][33];  // [ci][co]
   const int tap = blockIdx.z;
   if (blockIdx.x == 0 && blockIdx.y == 0) {
@@ -1020,9 +1024,8 @@ cudaError_t launch_conv_tc_inst(const ConvTcParams& p, const CUtensorMap& map_a,
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const unsigned grid = (unsigned)(p.total_tiles < sms ? p.total_tiles : sms);
-  conv_tc_kernel<MODE, KB, FP4><<<grid, TC_THREADS, smem, s>>>(map_a, map_b, map_out, p);
   count_launches(1);
-  return cudaGetLastError();
+  return launch_pdl(conv_tc_kernel<MODE, KB, FP4>, dim3(grid), dim3(TC_THREADS), smem, s, map_a, map_b, map_out, p);
 }
 
 size_t conv_tc_sfa_bytes(const ConvTcParams& p) {
@@ -1038,9 +1041,8 @@ cudaError_t launch_expand_inst(const ConvTcParams& p, cudaStream_t s) {
   unsigned long long warps = (unsigned long long)n_tile_m * p.max_stages + (unsigned long long)p.classes * p.tiles_c * p.max_stages;
   if (p.halo) warps += ((unsigned long long)p.tiles_c * p.Kh * p.Kw * p.BN * (KB / 16) + 31) / 32;
   const unsigned blocks = (unsigned)((warps + 7) / 8);
-  expand_conv_scales_kernel<MODE, KB, FP4><<<blocks, 256, 0, s>>>(p, n_tile_m);
   count_launches(1);
-  return cudaGetLastError();
+  return launch_pdl(expand_conv_scales_kernel<MODE, KB, FP4>, dim3(blocks), dim3(256), 0, s, p, n_tile_m);
 }
 
 cudaError_t launch_expand_conv_scales(const ConvTcParams& p, cudaStream_t s) {
@@ -1067,9 +1069,8 @@ cudaError_t launch_conv_tc_halo_taps(const ConvTcParams& p, const CUtensorMap& m
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const unsigned grid = (unsigned)(p.total_tiles < sms ? p.total_tiles : sms);
-  conv_tc_halo_kernel<MODE, KB, FP4, TAPS><<<grid, TC_THREADS, smem, s>>>(map_a, map_b, map_w, p);
   count_launches(1);
-  return cudaGetLastError();
+  return launch_pdl(conv_tc_halo_kernel<MODE, KB, FP4, TAPS>, dim3(grid), dim3(TC_THREADS), smem, s, map_a, map_b, map_w, p);
 }
 template <int MODE, int KB, bool FP4>
 cudaError_t launch_conv_tc_halo_inst(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_w, cudaStream_t s) {
@@ -1098,9 +1099,8 @@ cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, cons
 cudaError_t launch_weight_transpose(const uint8_t* w_codes, const uint8_t* w_scales, uint8_t* wt_codes, uint8_t* wt_scales, const Geom& g, int fmt,
                                     cudaStream_t s) {
   dim3 grid(g.Cp / 32, g.Cop / 32, g.Kh * g.Kw), block(32, 8);
-  weight_transpose_kernel<<<grid, block, 0, s>>>(w_codes, wt_codes, w_scales, wt_scales, g.Cout, g.Cop, g.Cp, g.Kh * g.Kw, fmt == MQ_E2M1 ? 1 : 0);
   count_launches(1);
-  return cudaGetLastError();
+  return launch_pdl(weight_transpose_kernel, grid, block, 0, s, w_codes, wt_codes, w_scales, wt_scales, g.Cout, g.Cop, g.Cp, g.Kh * g.Kw, fmt == MQ_E2M1 ? 1 : 0);
 }
 
 }  // namespace mq

@@ -17,6 +17,7 @@ constexpr int IC_TABLE = 2048;   // table entries per block: PX pixels x J chunk
 // PX consecutive output pixels per block amortise the block's fixed cost (launch, offset table, barrier) over
 // PX * 32 rows of X'.
 __global__ void __launch_bounds__(IC_THREADS) im2col_kernel(Im2colArgs a, int rc, int J, int PX, unsigned n_main) {
+  pdl_wait();
   const Geom& g = a.g;
   __shared__ int soff[IC_TABLE];   // source chunk offset of row chunk j of pixel px relative to sample 0, -1: zero
   const int taps = g.Kh * g.Kw;
@@ -128,8 +129,7 @@ cudaError_t launch_im2col(const Im2colArgs& a, cudaStream_t s) {
     long long sc_blocks = (n_scales + IC_THREADS - 1) / IC_THREADS;
     if (sc_blocks > 148 * 4) sc_blocks = 148 * 4;
     if (sc_blocks < 1) sc_blocks = 1;
-    im2col_kernel<<<(unsigned)(n_main + sc_blocks), IC_THREADS, 0, s>>>(a, rc, (int)J, PX, (unsigned)n_main);
-    return cudaGetLastError();
+    return launch_pdl(im2col_kernel, dim3((unsigned)(n_main + sc_blocks)), dim3(IC_THREADS), 0, s, a, rc, (int)J, PX, (unsigned)n_main);
   }
   const long long code_chunks = (long long)g.Ho * g.Wo * g.N * J;
   const long long total = code_chunks + n_scales;

@@ -115,4 +115,22 @@ __device__ __forceinline__ void decode8(const uint8_t* codes_base, long long ele
 
 #endif  // __CUDACC__
 
+// ---- programmatic dependent launch --------------------------------------------------------------------------
+// Kernels of this library are launched with programmatic stream serialization: a kernel may be scheduled while its
+// predecessor in the stream is still draining, and executes pdl_wait() (griddepcontrol.wait: returns once the
+// predecessor grid has completed and its writes are visible) before its first access to global memory.  Every
+// kernel waits, so completion is transitive along the stream.  MQ_NO_PDL=1 launches them plainly.
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+bool pdl_enabled();
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s, Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr; cfg.numAttrs = pdl_enabled() ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
 }  // namespace mq

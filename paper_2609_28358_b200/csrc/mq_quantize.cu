@@ -80,6 +80,7 @@ __global__ void __launch_bounds__(NT) quantize_pipe_kernel(QuantArgs a, int n_ps
   uint8_t* stage = qsmem + 2 * QBUF_BYTES;                              // codes [p][r][32 B (FP8) | 16 B (FP4)]
   unsigned* red = reinterpret_cast<unsigned*>(stage + PS * 32 * 32);     // [warp][quad][4]
 
+  pdl_wait();
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
   // compute mapping: 4 adjacent channels x 2 rows x 4 positions per thread
   const int cq = t & 7, quad = (t >> 3) & 1, rs = t >> 4;
@@ -204,6 +205,7 @@ template <int FMT>
 __global__ void __launch_bounds__(QT_THREADS) quantize_simple_kernel(QuantArgs a, int n_pstrips, int Ct) {
   __shared__ __align__(16) unsigned red[8][2][4];
   __shared__ __align__(16) uint8_t stage[PS][32][32];   // one code per byte
+  pdl_wait();
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
   const Item q = item_of(blockIdx.x, n_pstrips, Ct);
   const int quad = t & 1, c = (t >> 1) & 31, rsub = t >> 6;
@@ -299,8 +301,7 @@ constexpr size_t QPIPE_SMEM = 2 * QBUF_BYTES + PS * 32 * 32 + 16 * 2 * 4 * sizeo
 template <int FMT>
 cudaError_t launch_q(const QuantArgs& a, int n_pstrips, int Ct, long long n_items, bool vec, cudaStream_t s) {
   if (!vec) {
-    quantize_simple_kernel<FMT><<<(unsigned)n_items, QT_THREADS, 0, s>>>(a, n_pstrips, Ct);
-    return cudaGetLastError();
+    return launch_pdl(quantize_simple_kernel<FMT>, dim3((unsigned)n_items), dim3(QT_THREADS), 0, s, a, n_pstrips, Ct);
   }
   static bool attr_set = false;
   static int ctas_per_sm = 2;   // 80 KB of shared memory per block
@@ -321,9 +322,8 @@ cudaError_t launch_q(const QuantArgs& a, int n_pstrips, int Ct, long long n_item
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   long long grid = (long long)sms * ctas_per_sm;
   if (grid > n_items) grid = n_items;
-  if (nt == 512) quantize_pipe_kernel<FMT, 512><<<(unsigned)grid, 512, QPIPE_SMEM, s>>>(a, n_pstrips, Ct, (unsigned)n_items);
-  else quantize_pipe_kernel<FMT, 256><<<(unsigned)grid, 256, QPIPE_SMEM, s>>>(a, n_pstrips, Ct, (unsigned)n_items);
-  return cudaGetLastError();
+  if (nt == 512) return launch_pdl(quantize_pipe_kernel<FMT, 512>, dim3((unsigned)grid), dim3(512), QPIPE_SMEM, s, a, n_pstrips, Ct, (unsigned)n_items);
+  return launch_pdl(quantize_pipe_kernel<FMT, 256>, dim3((unsigned)grid), dim3(256), QPIPE_SMEM, s, a, n_pstrips, Ct, (unsigned)n_items);
 }
 
 }  // namespace

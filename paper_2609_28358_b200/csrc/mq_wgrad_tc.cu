@@ -110,12 +110,13 @@ __device__ __forceinline__ void expand_wgrad_scales_body(const WgradTcParams& p,
 // shifted by one pixel (one piece) per tap, so a stage loads KPX + Kw - 1 pieces of X once and the stage's G_Y
 // tile feeds Kw accumulators (Kw times less shared-memory traffic per FLOP than one tap per block).
 template <bool FP4>
-__global__ void __launch_bounds__(256) expand_wgrad_scales_kernel(const WgradTcParams p) { expand_wgrad_scales_body<FP4>(p, blockIdx.x); }
+__global__ void __launch_bounds__(256) expand_wgrad_scales_kernel(const WgradTcParams p) { pdl_wait(); expand_wgrad_scales_body<FP4>(p, blockIdx.x); }
 
 template <bool FP4>
 __global__ void __launch_bounds__(WG_THREADS, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_p,
                 const WgradTcParams p) {
+  pdl_wait();
   constexpr int SPA = FP4 ? 2 : 1;     // scale bytes per MMA per row
   if (threadIdx.x == 0) WPROF(0);
   extern __shared__ uint8_t smem_raw[];
@@ -444,6 +445,7 @@ __device__ __forceinline__ void fp4_to_flat_body(const FlatArgs& fa, unsigned bl
 // Preparation of the flat mode in one launch: blocks [0, x.blocks) re-lay X, the next g.blocks re-lay G_Y, the rest
 // expand the scale chunks.
 __global__ void __launch_bounds__(256) wgrad_flat_prep_kernel(const FlatArgs x, const FlatArgs gy, const WgradTcParams p) {
+  pdl_wait();
   if (blockIdx.x < x.blocks) fp4_to_flat_body(x, blockIdx.x, x.blocks);
   else if (blockIdx.x < x.blocks + gy.blocks) fp4_to_flat_body(gy, blockIdx.x - x.blocks, gy.blocks);
   else expand_wgrad_scales_body<true>(p, blockIdx.x - x.blocks - gy.blocks);
@@ -467,19 +469,17 @@ cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, co
     attr_set[f] = true;
   }
   const unsigned grid = (unsigned)(p.m_tiles * p.j_tiles * p.splits);
-  if (f) wgrad_tc_kernel<true><<<grid, WG_THREADS, smem, s>>>(map_a, map_b, map_p, p);
-  else wgrad_tc_kernel<false><<<grid, WG_THREADS, smem, s>>>(map_a, map_b, map_p, p);
   count_launches(1);
-  return cudaGetLastError();
+  if (f) return launch_pdl(wgrad_tc_kernel<true>, dim3(grid), dim3(WG_THREADS), smem, s, map_a, map_b, map_p, p);
+  return launch_pdl(wgrad_tc_kernel<false>, dim3(grid), dim3(WG_THREADS), smem, s, map_a, map_b, map_p, p);
 }
 
 cudaError_t launch_expand_wgrad_scales(const WgradTcParams& p, cudaStream_t s) {
   const long long warps = (long long)p.m_tiles * p.stages_total + (long long)p.cb_tiles * (p.Kh * p.Kw / p.TG) * p.stages_total * p.NB;
   const unsigned blocks = (unsigned)((warps + 7) / 8);
-  if (p.mode == MQ_WG_FP8) expand_wgrad_scales_kernel<false><<<blocks, 256, 0, s>>>(p);
-  else expand_wgrad_scales_kernel<true><<<blocks, 256, 0, s>>>(p);
   count_launches(1);
-  return cudaGetLastError();
+  if (p.mode == MQ_WG_FP8) return launch_pdl(expand_wgrad_scales_kernel<false>, dim3(blocks), dim3(256), 0, s, p);
+  return launch_pdl(expand_wgrad_scales_kernel<true>, dim3(blocks), dim3(256), 0, s, p);
 }
 
 cudaError_t launch_fp4_to_n_major(const uint8_t* in, uint8_t* out, int P, int N, int Cp, int Npad, cudaStream_t s) {
@@ -511,9 +511,8 @@ cudaError_t launch_wgrad_flat_prep(const WgradTcParams& p, const uint8_t* x_code
   if (!make_flat_args(&fg, g_codes, gt, p.Ho, p.Wo, p.N, p.Cot * 32, P_a, p.Wp, 0, 0, 128, p.m_tiles, p.KBn)) return cudaErrorInvalidValue;
   const long long warps = (long long)p.m_tiles * p.stages_total + (long long)p.cb_tiles * (p.Kh * p.Kw / p.TG) * p.stages_total * p.NB;
   const unsigned sc_blocks = (unsigned)((warps + 7) / 8);
-  wgrad_flat_prep_kernel<<<fx.blocks + fg.blocks + sc_blocks, 256, 0, s>>>(fx, fg, p);
   count_launches(1);
-  return cudaGetLastError();
+  return launch_pdl(wgrad_flat_prep_kernel, dim3(fx.blocks + fg.blocks + sc_blocks), dim3(256), 0, s, fx, fg, p);
 }
 
 }  // namespace mq
