@@ -333,6 +333,9 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   p.Wp = g.W + 2 * g.pw;
   p.stages_total = flat ? (g.Ho * p.Wp + p.KPX - 1) / p.KPX : g.Ho * p.groups_w * p.nchunks;
   p.b_rows = flat ? (g.Cp < 128 ? g.Cp : 128) : 128;
+  // 8-bit operands: 256 input channels per MMA when the layer has them (the kernel is bound by the tensor core's
+  // shared-memory operand reads, and a wider N reads the G_Y tile once for twice the work)
+  if (fp8 && g.Cp >= 256 && !env_int("MQ_WGRAD_N128", 0)) p.b_rows = 256;
   p.m_tiles = (g.Cout + 127) / 128;
   p.cb_tiles = (g.Cp + p.b_rows - 1) / p.b_rows;
   // taps per block: a whole kernel row in the flat mode when its accumulators fit in tensor memory

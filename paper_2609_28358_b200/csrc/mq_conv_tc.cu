@@ -278,7 +278,6 @@ template <int MODE, int KB, bool FP4>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_out,
                const ConvTcParams p) {
-  pdl_wait();
   constexpr int G = 128 / KB;          // chunks per stage
   constexpr int APC = KB / 32;         // MMA K-atoms (32 bytes) per chunk
   constexpr int SPA = FP4 ? 2 : 1;     // scale bytes per atom
@@ -316,6 +315,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
+  pdl_wait();   // set-up above touched only shared memory, tensor memory and the kernel parameters
 
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
@@ -515,7 +515,6 @@ template <int MODE, int KB, bool FP4, int TAPS>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_w,
                     const ConvTcParams p) {
-  pdl_wait();
   constexpr int G = 128 / KB, APC = KB / 32, SPA = FP4 ? 2 : 1;
   constexpr int LAYOUT = KB == 128 ? 2 : (KB == 64 ? 4 : 6);
 #ifdef MQ_TC_PROFILE
@@ -557,6 +556,7 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     mbar_fence_init();
     prefetch_tensormap(&map_a);
     if (p.tma_store) prefetch_tensormap(&map_out);
+    pdl_wait();      // everything above touches only this block's shared memory and the kernel parameters
     if (p.fused) {   // the weight tile, all taps: one box, swizzled by the copy engine, while the block finishes setting up
       mbar_arrive_expect_tx(bfull, (uint32_t)b_bytes);
       tma_load_3d(smem, &map_w, bfull, 0, 0, 0);
@@ -572,8 +572,9 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     tap_b[threadIdx.x] = (uint32_t)(threadIdx.x * p.BN * KB) >> 4;
     tap_p[threadIdx.x] = (uint32_t)(hrow * (p.TW + p.Kw - 1) + wsh);
   }
-  if (p.fused) halo_build_sfb<KB, FP4>(p, smem + b_bytes);
   if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  pdl_wait();
+  if (p.fused) halo_build_sfb<KB, FP4>(p, smem + b_bytes);
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();

@@ -116,7 +116,6 @@ template <bool FP4>
 __global__ void __launch_bounds__(WG_THREADS, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_p,
                 const WgradTcParams p) {
-  pdl_wait();
   constexpr int SPA = FP4 ? 2 : 1;     // scale bytes per MMA per row
   if (threadIdx.x == 0) WPROF(0);
   extern __shared__ uint8_t smem_raw[];
@@ -161,6 +160,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
+  pdl_wait();   // set-up above touched only shared memory, tensor memory and the kernel parameters
   if (threadIdx.x == 0) WPROF(1);
 
   if (warp == 0) {
@@ -207,6 +207,8 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             // stored [ho][wo][n][c] codes: box (128 channel bytes, n rows, pixels, 1)
             tma_load_4d(sa, &map_a, &full[s], co0, nc * p.BPP * 32, wo0, ho);
             tma_load_4d(sb, &map_b, &full[s], ci0, nc * p.BPP * 32, wo0 * p.sw + kw - p.pw, ho * p.sh + kh - p.ph);
+            if (p.b_rows > 128)   // second 128-channel panel of a 256-channel tile
+              tma_load_4d(sb + 128 * 128, &map_b, &full[s], ci0 + 128, nc * p.BPP * 32, wo0 * p.sw + kw - p.pw, ho * p.sh + kh - p.ph);
           }
         }
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
