@@ -32,6 +32,9 @@ SMALL_SHAPES = [
     ("k5", (8, 16, 12, 12, 24, 5, 2, 2)),          # 5x5, C < 32
     ("nopad", (16, 32, 7, 7, 32, 3, 1, 0)),        # no padding
     ("rect", (4, 35, 6, 10, 33, 3, 1, 1)),
+    ("thin_wide", (16, 32, 6, 8, 160, 3, 1, 1)),   # thin contraction, two output-channel tiles (weight tile reloaded) in fwd
+    ("wide_thin", (16, 160, 6, 8, 32, 3, 1, 1)),   # the same situation in the input gradient
+    ("wide", (32, 256, 4, 8, 288, 3, 1, 1)),       # 256-channel MMAs (8-bit) and a remainder channel tile
 ]
 
 
