@@ -89,8 +89,10 @@ mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt
  *   per tile: amax = max |x| over the valid elements; scale code = clamp(floor(log2 amax) - emax
  *   + 127, 0, 254) (0 if amax = 0); element = round-to-nearest-even(x * 2^(127 - code)) on the
  *   element format's grid, saturating at its largest finite magnitude, sign kept.
- * src: fp32, `src_layout` = MQ_NCHW (X: NCHW, W: OIHW, G_Y: N.C_out.Ho.Wo); MQ_HWNC is not
- * implemented (MQ_ERR_UNSUPPORTED).  dst->codes / dst->scales receive the stored tensor; dst->fmt and
+ * src: fp32 device memory, 16-byte aligned; `src_layout` = MQ_NCHW (X: [N][C_in][H][W], W: [C_out][C_in][Kh][Kw],
+ * G_Y: [N][C_out][Ho][Wo]) or MQ_HWNC, the channel-fastest order the convolution entry points can emit
+ * (X: [H][W][N][C_in], W: [C_out][Kh][Kw][C_in], G_Y: [Ho][Wo][N][C_out]); both give the same stored
+ * tensor bit for bit.  dst->codes / dst->scales receive the stored tensor; dst->fmt and
  * dst->role select format and role; the *_bytes fields must be at least mq_qtensor_sizes().
  * Non-finite inputs are outside the contract (result unspecified, no fault). */
 mq_status mq_quantize(const mq_conv_desc* desc, const void* src, int src_layout, mq_qtensor* dst, void* stream);

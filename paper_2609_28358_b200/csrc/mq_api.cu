@@ -537,7 +537,6 @@ mq_status mq_quantize(const mq_conv_desc* desc, const void* src, int src_layout,
   if (st != MQ_OK) return st;
   if (!src || !dst || !valid_role(dst->role)) return MQ_ERR_INVALID_ARG;
   if (src_layout != MQ_NCHW && src_layout != MQ_HWNC) return MQ_ERR_INVALID_ARG;
-  if (src_layout != MQ_NCHW) return MQ_ERR_UNSUPPORTED;
   Geom g = make_geom(*desc);
   if ((st = check_qtensor(g, dst, dst->role)) != MQ_OK) return st;
   if (!aligned16(src)) return MQ_ERR_ALIGNMENT;
@@ -556,6 +555,11 @@ mq_status mq_quantize(const mq_conv_desc* desc, const void* src, int src_layout,
     a.sc_stride_p = Rt * Ct; a.sc_stride_r = Ct;
   }
   a.fmt = dst->fmt;
+  a.src_stride_p = 0; a.src_stride_r = 0;
+  if (src_layout == MQ_HWNC) {   // channel-fastest source: activations / gradients [pixel][n][c], weights [cout][tap][cin]
+    if (dst->role == MQ_ROLE_W) { a.src_stride_p = v.C; a.src_stride_r = v.P * v.C; }
+    else { a.src_stride_p = v.R * v.C; a.src_stride_r = v.C; }
+  }
   cudaError_t e = launch_quantize(a, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }

@@ -49,6 +49,9 @@ struct QuantArgs {
   long long out_stride_p, out_stride_r;  // in elements of the codes tensor
   long long sc_stride_p, sc_stride_r;    // in scale bytes
   int fmt;
+  // source strides in floats when the source has the channel axis fastest (fp32 [H][W][N][C] / [Cout][Kh][Kw][Cin]):
+  // element (p, r, c) at p * src_stride_p + r * src_stride_r + c; both zero for the NCHW / OIHW source
+  long long src_stride_p, src_stride_r;
 };
 cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s);
 

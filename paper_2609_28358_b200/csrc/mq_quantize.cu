@@ -296,6 +296,73 @@ __global__ void __launch_bounds__(QT_THREADS) quantize_simple_kernel(QuantArgs a
   }
 }
 
+// ---- channel-fastest source ([H][W][N][C] activations / gradients, [Cout][Kh][Kw][Cin] weights) ------------------
+// No re-layout is needed: a tile's 32 rows are runs of 32 consecutive floats.  One warp per (position, tile): lane
+// (cq, rq) = (lane & 7, lane >> 3) loads 4 adjacent channels of rows rq, rq + 4, ... as one 128-bit load each (8 in
+// flight), the amax is a per-lane max plus one redux.sync, and the codes leave as 32-bit words (FP8) or, pairing
+// neighbouring lanes, 32-bit words of 8 E2M1 codes.  VEC = false takes any C and alignment with scalar loads.
+template <int FMT, bool VEC>
+__global__ void __launch_bounds__(256) quantize_cfast_kernel(QuantArgs a, unsigned Rt, unsigned Ct, unsigned n_items) {
+  pdl_wait();
+  const int lane = threadIdx.x & 31;
+  const int cq = lane & 7, rq = lane >> 3;
+#pragma unroll 1
+  for (unsigned it = blockIdx.x * 8u + (threadIdx.x >> 5); it < n_items; it += gridDim.x * 8u) {
+    // channel tile fastest, then row tile, then position: consecutive warps read consecutive memory
+    const unsigned ct = it % Ct; const unsigned u = it / Ct;
+    const unsigned rt = u % Rt; const unsigned pos = u / Rt;
+    const int r0 = (int)rt * 32 + rq, c0 = (int)ct * 32 + 4 * cq;
+    const float* src = a.src + (long long)pos * a.src_stride_p + (long long)r0 * a.src_stride_r + c0;
+    float4 v[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      v[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+      const float* q = src + (long long)(4 * i) * a.src_stride_r;
+      if (r0 + 4 * i < a.R) {
+        if (VEC) { if (c0 < a.C) v[i] = __ldg(reinterpret_cast<const float4*>(q)); }   // C % 4 == 0: whole quads
+        else {
+          if (c0 + 0 < a.C) v[i].x = __ldg(q + 0);
+          if (c0 + 1 < a.C) v[i].y = __ldg(q + 1);
+          if (c0 + 2 < a.C) v[i].z = __ldg(q + 2);
+          if (c0 + 3 < a.C) v[i].w = __ldg(q + 3);
+        }
+      }
+    }
+    float m = 0.f;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) m = fmaxf(fmaxf(m, fmaxf(fabsf(v[i].x), fabsf(v[i].y))), fmaxf(fabsf(v[i].z), fabsf(v[i].w)));
+    const int code = scale_code_of(__reduce_max_sync(0xffffffffu, __float_as_uint(m)), fmt_emax(FMT));
+    if (lane == 0) a.scales[(long long)pos * a.sc_stride_p + (long long)rt * a.sc_stride_r + ct] = (uint8_t)code;
+    const float f = scale_factor(code);
+    const long long pbase = (long long)pos * a.out_stride_p + c0;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      const int r = r0 + 4 * i;
+      const unsigned lo = encode2<FMT>(v[i].x * f, v[i].y * f), hi = encode2<FMT>(v[i].z * f, v[i].w * f);
+      const long long e = pbase + (long long)r * a.out_stride_r;
+      if (FMT == MQ_E2M1) {
+        const unsigned mine = lo | (hi << 8);                       // 4 codes; the odd lane's go above the even lane's
+        const unsigned other = __shfl_xor_sync(0xffffffffu, mine, 1);
+        if ((lane & 1) == 0 && r < a.R) *reinterpret_cast<unsigned*>(a.codes + (e >> 1)) = mine | (other << 16);
+      } else {
+        if (r < a.R) *reinterpret_cast<unsigned*>(a.codes + e) = lo | (hi << 16);
+      }
+    }
+  }
+}
+
+template <int FMT>
+cudaError_t launch_q_cfast(const QuantArgs& a, int Ct, cudaStream_t s) {
+  const long long Rt = (a.R + 31) / 32;
+  const long long items = (long long)a.P * Rt * Ct;
+  if (items <= 0 || items > 0xffffffffLL) return cudaErrorInvalidValue;
+  const bool vec = a.C % 4 == 0 && a.src_stride_p % 4 == 0 && a.src_stride_r % 4 == 0 && (reinterpret_cast<uintptr_t>(a.src) & 15) == 0;
+  long long blocks = (items + 7) / 8;
+  if (blocks > 148LL * 64) blocks = 148LL * 64;
+  if (vec) return launch_pdl(quantize_cfast_kernel<FMT, true>, dim3((unsigned)blocks), dim3(256), 0, s, a, (unsigned)Rt, (unsigned)Ct, (unsigned)items);
+  return launch_pdl(quantize_cfast_kernel<FMT, false>, dim3((unsigned)blocks), dim3(256), 0, s, a, (unsigned)Rt, (unsigned)Ct, (unsigned)items);
+}
+
 constexpr size_t QPIPE_SMEM = 2 * QBUF_BYTES + PS * 32 * 32 + 16 * 2 * 4 * sizeof(unsigned);
 
 template <int FMT>
@@ -335,6 +402,16 @@ cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s) {
   if (n_items <= 0 || n_items > 0x7fffffffLL) return cudaErrorInvalidValue;
   const bool vec = (a.P % 4 == 0) && ((reinterpret_cast<uintptr_t>(a.src) & 15) == 0);
   cudaError_t e;
+  if (a.src_stride_r != 0) {   // channel-fastest source
+    switch (a.fmt) {
+      case MQ_E4M3: e = launch_q_cfast<MQ_E4M3>(a, Ct, s); break;
+      case MQ_E5M2: e = launch_q_cfast<MQ_E5M2>(a, Ct, s); break;
+      case MQ_E2M1: e = launch_q_cfast<MQ_E2M1>(a, Ct, s); break;
+      default: return cudaErrorInvalidValue;
+    }
+    count_launches(1);
+    return e;
+  }
   switch (a.fmt) {
     case MQ_E4M3: e = launch_q<MQ_E4M3>(a, n_pstrips, Ct, n_items, vec, s); break;
     case MQ_E5M2: e = launch_q<MQ_E5M2>(a, n_pstrips, Ct, n_items, vec, s); break;

@@ -105,7 +105,7 @@ def empty_qtensor(desc, role, fmt, device="cuda"):
 
 
 def quantize(desc, role, fmt, src, out=None, src_layout=NCHW, stream=None):
-    """mq_quantize: fp32 device tensor (NCHW / OIHW) -> stored MX tensor."""
+    """mq_quantize: fp32 device tensor (NCHW / OIHW, or channel-fastest with src_layout=HWNC) -> stored MX tensor."""
     assert src.is_cuda and src.dtype == torch.float32 and src.is_contiguous()
     if out is None:
         out = empty_qtensor(desc, role, fmt, src.device)

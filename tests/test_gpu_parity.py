@@ -49,6 +49,21 @@ def test_small_layers_all_steps(name, shape, fmts):
 
 
 @pytest.mark.parametrize("fmt", [E4M3, E5M2, E2M1])
+@pytest.mark.parametrize("shape", [(40, 48, 5, 6, 70, 3, 1, 1), (64, 96, 8, 8, 64, 3, 1, 1), (33, 35, 6, 7, 34, 3, 2, 1)],
+                         ids=["ragged", "aligned", "odd-channels"])
+def test_quantize_channel_fastest_source(shape, fmt):
+    """The same logical tensors handed over as fp32 [H][W][N][C] / [Cout][Kh][Kw][Cin] give the oracle's stored bytes."""
+    d = inputs.conv_desc(*shape)
+    ol = OracleLayer(make_layer("hwnc_src", d, (fmt, fmt, fmt), seed=7, kinds=("relu", "kaiming", "gauss")))
+    x, w, g = ol.src
+    srcs = (np.ascontiguousarray(x.transpose(2, 3, 0, 1)), np.ascontiguousarray(w.transpose(0, 2, 3, 1)), np.ascontiguousarray(g.transpose(2, 3, 0, 1)))
+    for role, name, src, (c, s_) in zip((0, 1, 2), ("X", "W", "dY"), srcs, ol.q):
+        q = mq.quantize(d, role, fmt, torch.from_numpy(src).cuda(), src_layout=mq.HWNC)
+        assert_same_bytes(q.scales, s_, f"{name} scales from channel-fastest source")
+        assert_same_bytes(q.codes, c, f"{name} codes from channel-fastest source")
+
+
+@pytest.mark.parametrize("fmt", [E4M3, E5M2, E2M1])
 def test_quantize_edge_values(fmt):
     """Zero tiles, -0, ties, saturation, huge and tiny magnitudes, fp32 subnormals."""
     d = inputs.conv_desc(64, 64, 4, 4, 32, 1, 1, 0)
