@@ -76,7 +76,7 @@ def test_bad_arguments_are_rejected_on_the_host(mq):
     q = mq._QTensor(0x1008, 0x2000, 1 << 30, 1 << 30, 0, 0)
     assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), 0, ctypes.byref(q), None) == 3  # alignment
     q = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 0)
-    assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), 1, ctypes.byref(q), None) == 2  # HWNC source
+    assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), 7, ctypes.byref(q), None) == 1  # no such source layout
     assert L.mq_cbf_im2col(ctypes.byref(good), ctypes.byref(q), None, None, None) == 1
     qw = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 1)
     assert L.mq_conv_fwd(ctypes.byref(good), ctypes.byref(qw), ctypes.byref(qw), ctypes.c_void_p(0x4000), 0, None, 0, None) == 1  # wrong role
