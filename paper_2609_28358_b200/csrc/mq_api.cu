@@ -170,7 +170,8 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   }
   // NCHW output through TMA stores (unit-stride output columns, rows of 16-byte multiples): worth its 64 KB of
   // staging only in the whole-tile kernel, whose pipeline is short; the per-tap kernel keeps its stages
-  const bool tma_store_ok = layout == MQ_NCHW && p.Wd % 4 == 0 && p.TW >= 4 && p.TW <= 32 && (op == MQ_OP_FWD || (g.sh == 1 && g.sw == 1));
+  const bool tma_store_ok = (op == MQ_OP_FWD || (g.sh == 1 && g.sw == 1)) && p.TW >= 4 && p.TW <= 32 &&
+                            (layout == MQ_NCHW ? p.Wd % 4 == 0 : (p.Cd % 4 == 0 && p.BN % 64 == 0));   // [H][W][N][C]: whole 32-channel groups per column half
   p.tma_store = tma_store_ok && env_int("MQ_TC_TMA_STORE", 0) ? 1 : 0;
   const size_t stage_bytes = 128 * 128 + (size_t)p.BN * 128 + 3072;
   int stages = (int)((227 * 1024 - 2048 - (p.tma_store ? 65536 : 0)) / stage_bytes);
@@ -292,12 +293,21 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
   if (p.tma_store) {
     if (reinterpret_cast<uintptr_t>(out) % 16 != 0) p.tma_store = 0;
     else {
-      // the output seen as (W, N, C, H); one epilogue warp's 32 rows x the channels of a column half (at most 64)
-      const uint64_t dims[4] = {(uint64_t)p.Wd, (uint64_t)g.N, (uint64_t)p.Cd, (uint64_t)p.Hd};
-      const uint64_t strides[3] = {(uint64_t)p.Cd * p.Hd * p.Wd * 4, (uint64_t)p.Hd * p.Wd * 4, (uint64_t)p.Wd * 4};
-      const int half_cols = (p.BN / 2 + 15) & ~15;
-      const uint32_t box[4] = {(uint32_t)p.TW, (uint32_t)(32 / p.TW), (uint32_t)(half_cols < 64 ? half_cols : 64), 1u};
-      if (!encode_tensor_map_u8(&map_out, out, 4, dims, strides, box, nullptr, 0, true)) return MQ_ERR_CUDA;
+      if (layout == MQ_NCHW) {
+        // the output seen as (W, N, C, H); one epilogue warp's 32 rows x the channels of a column half (at most 64)
+        const uint64_t dims[4] = {(uint64_t)p.Wd, (uint64_t)g.N, (uint64_t)p.Cd, (uint64_t)p.Hd};
+        const uint64_t strides[3] = {(uint64_t)p.Cd * p.Hd * p.Wd * 4, (uint64_t)p.Hd * p.Wd * 4, (uint64_t)p.Wd * 4};
+        const int half_cols = (p.BN / 2 + 15) & ~15;
+        const uint32_t box[4] = {(uint32_t)p.TW, (uint32_t)(32 / p.TW), (uint32_t)(half_cols < 64 ? half_cols : 64), 1u};
+        if (!encode_tensor_map_u8(&map_out, out, 4, dims, strides, box, nullptr, 0, true)) return MQ_ERR_CUDA;
+      } else {
+        // [Ho][Wo][N][C] seen as (C, W, N, H) -- the order of a tile's rows: a warp's 32 rows x 32 channels, rows of 128
+        // bytes with the 128-byte swizzle
+        const uint64_t dims[4] = {(uint64_t)p.Cd, (uint64_t)p.Wd, (uint64_t)g.N, (uint64_t)p.Hd};
+        const uint64_t strides[3] = {(uint64_t)g.N * p.Cd * 4, (uint64_t)p.Cd * 4, (uint64_t)p.Wd * g.N * p.Cd * 4};
+        const uint32_t box[4] = {32u, (uint32_t)p.TW, (uint32_t)(32 / p.TW), 1u};
+        if (!encode_tensor_map_u8(&map_out, out, 4, dims, strides, box, nullptr, 128, true)) return MQ_ERR_CUDA;
+      }
     }
   }
   return launch_conv_tc(p, map_a, map_w, map_out, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;

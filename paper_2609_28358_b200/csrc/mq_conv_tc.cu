@@ -217,6 +217,8 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
     const int cend = half == 0 ? ((p.BN / 2 + 15) & ~15) : p.BN;
     float* buf = staging + (warp - 4) * (64 * 32);
     const int n_off = quad * (32 >> p.lgTW);          // first sample of this warp's rows inside the tile
+    const bool hwnc = p.out_layout == MQ_HWNC;
+    const int hrow = lane;   // the [H][W][N][C] store's box walks (sample, column) in the rows' own order
     uint32_t tcount = 0;
     PROF_BEGIN();
     for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
@@ -253,9 +255,18 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
 #pragma unroll
             for (int j = 0; j < 16; ++j) v[j] = 0u;
           }
-          float* bi = buf + (16 * i) * 32 + lane;
+          if (!hwnc) {
+            float* bi = buf + (16 * i) * 32 + lane;
 #pragma unroll
-          for (int j = 0; j < 16; ++j) bi[j * 32] = __uint_as_float(v[j]);
+            for (int j = 0; j < 16; ++j) bi[j * 32] = __uint_as_float(v[j]);
+          } else {
+            // [Ho][Wo][N][C] output: rows of 32 channels (128 bytes, 128-byte swizzle: consecutive lanes hit different
+            // bank groups); chunk i is the 16-byte units 4 (i & 1) .. + 3 of 32-channel group i >> 1
+            uint8_t* bg = reinterpret_cast<uint8_t*>(buf) + (i >> 1) * 4096 + hrow * 128;
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+              *reinterpret_cast<uint4*>(bg + ((((i & 1) * 4 + u) ^ (hrow & 7)) << 4)) = make_uint4(v[4 * u], v[4 * u + 1], v[4 * u + 2], v[4 * u + 3]);
+          }
         }
         if (c0 + 64 >= cend) {   // the accumulator has been read: hand it back before the store
           tc_fence_before_sync();
@@ -265,7 +276,11 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0 && p.out_layout != 99) {
-          tma_store_4d(map_out, buf, tile.w0, tile.n0 + n_off, tile.c0 + c0, yo);
+          if (!hwnc) tma_store_4d(map_out, buf, tile.w0, tile.n0 + n_off, tile.c0 + c0, yo);
+          else {
+            tma_store_4d(map_out, buf, tile.c0 + c0, tile.w0, tile.n0 + n_off, yo);
+            if (nch > 2) tma_store_4d(map_out, buf + 1024, tile.c0 + c0 + 32, tile.w0, tile.n0 + n_off, yo);
+          }
           bulk_commit_group();
         }
       }
