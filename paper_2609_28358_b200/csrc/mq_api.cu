@@ -181,6 +181,8 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   // TMEM (512 columns): accumulators (BN columns each) + one 24-column scale buffer per pipeline stage
   p.n_acc = (2 * p.BN + 24 * stages <= 512) ? 2 : 1;
   if (p.n_acc * p.BN + 24 * stages > 512) return false;
+  p.pair = op == MQ_OP_BWD_DATA && g.sw == 2 && layout == MQ_NCHW && p.Wd % 2 == 0 && p.n_acc == 2 && p.total_tiles % 2 == 0 &&
+           !env_int("MQ_TC_NO_PAIR", 0);
   const int nkh = op == MQ_OP_FWD ? g.Kh : (g.Kh + g.sh - 1) / g.sh, nkw = op == MQ_OP_FWD ? g.Kw : (g.Kw + g.sw - 1) / g.sw;
   p.max_stages = (nkh * nkw * p.cpt + p.G - 1) / p.G;
   const uint32_t fa = fp4 ? 1u : (fmt_x_like == MQ_E5M2 ? 1u : 0u);

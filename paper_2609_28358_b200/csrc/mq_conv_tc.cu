@@ -84,6 +84,14 @@ __device__ __forceinline__ Tile tile_of_m_index(const ConvTcParams& p, unsigned 
   return q;
 }
 
+// The i-th tile of this block.  Plain mode: round robin over the blocks.  Pair mode (input gradient with a column
+// stride of 2, NCHW output): tiles 2k and 2k + 1 are the two column-parity classes of the same output positions
+// (the class is the fastest tile index) and go to the same block back to back, into the two accumulators, so
+// that the epilogue can interleave them into contiguous stores.
+__device__ __forceinline__ unsigned tile_of_iter(const ConvTcParams& p, unsigned i) {
+  return p.pair ? 2u * (blockIdx.x + (i >> 1) * gridDim.x) + (i & 1u) : blockIdx.x + i * gridDim.x;
+}
+
 // The taps that contribute to a tile, as a small 2-D range walked without divisions.
 // Forward: all (kh, kw); source pixel = (ho*sh - ph + kh, wo*sw - pw + kw).
 // Input gradient: the taps whose offset has the parity of the tile's class (h + ph - kh and w + pw - kw
@@ -199,6 +207,66 @@ __device__ __forceinline__ void epilogue_role(const ConvTcParams& p, uint32_t tm
       if (lane == 0) mbar_arrive(&tempty[acc]);
     }
     if (lane == 0 && warp == 4) PROF_END(3);
+}
+
+// Epilogue role of the pair mode (see tile_of_iter): both accumulators hold the same output rows and channels for the
+// even and the odd output columns; a thread writes them as float2 (x = 2 (w0 + tw), x + 1), so a warp's store covers
+// 64-byte runs per sample instead of every other float.
+template <int MODE>
+__device__ __forceinline__ void epilogue_pair_role(const ConvTcParams& p, uint32_t tmem, uint64_t* tfull, uint64_t* tempty, volatile int* abort_flag,
+                                                   int warp, int lane, unsigned total) {
+    const int quad = warp & 3;
+    const int half = (warp - 4) >> 2;
+    const int r = 32 * quad + lane;
+    const int tw_ = r & (p.TW - 1), tn = r >> p.lgTW;
+    const int cbeg = half == 0 ? 0 : ((p.BN / 2 + 15) & ~15);
+    const int cend = half == 0 ? ((p.BN / 2 + 15) & ~15) : p.BN;
+    const long long cs = (long long)p.Hd * p.Wd;
+#pragma unroll 1
+    for (unsigned j = 0, t; (t = tile_of_iter(p, 2 * j)) < total && !*abort_flag; ++j) {
+      const Tile t0 = decode_tile(p, t), t1 = decode_tile(p, t + 1);
+      TapWalk<MODE> w0, w1;
+      w0.init(p, t0); w1.init(p, t1);
+      const int Q0 = w0.chunks(p), Q1 = w1.chunks(p);
+      bool ok = true;
+      if (lane == 0) ok = mbar_wait(&tfull[0], j & 1, p.status, MQ_ERR_TIMEOUT) && mbar_wait(&tfull[1], j & 1, p.status, MQ_ERR_TIMEOUT);
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) { *abort_flag = 1; break; }
+      tc_fence_after_sync();
+      const int ch = (int)fdiv((unsigned)t0.cls, p.sw, p.m_sw);
+      const int yo = ch + p.sh * t0.h, xo = p.sw * (t0.w0 + tw_);     // even column; the odd class writes xo + 1
+      const int n = t0.n0 + tn;
+      const bool row_ok = yo < p.Hd && xo < p.Wd && n < p.N;          // Wd is even in this mode: xo + 1 < Wd as well
+      const uint32_t taddr = tmem + ((uint32_t)(32 * quad) << 16);
+      float* o = p.out + (((long long)n * p.Cd + t0.c0 + cbeg) * p.Hd + yo) * p.Wd + xo;
+#pragma unroll 1
+      for (int c = cbeg; c < cend; c += 16) {
+        uint32_t v0[16], v1[16];
+        if (Q0 > 0) tmem_ld_32x32b_x16(taddr + c, v0);
+        if (Q1 > 0) tmem_ld_32x32b_x16(taddr + p.BN + c, v1);
+        tmem_ld_wait();
+        if (Q0 == 0) {
+#pragma unroll
+          for (int q = 0; q < 16; ++q) v0[q] = 0u;
+        }
+        if (Q1 == 0) {
+#pragma unroll
+          for (int q = 0; q < 16; ++q) v1[q] = 0u;
+        }
+        if (row_ok && p.out_layout != 99) {
+#pragma unroll
+          for (int q = 0; q < 16; ++q) {
+            if (t0.c0 + c + q < p.Cd) *reinterpret_cast<float2*>(o) = make_float2(__uint_as_float(v0[q]), __uint_as_float(v1[q]));
+            o += cs;
+          }
+        } else {
+          o += 16 * cs;
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(&tempty[0]); mbar_arrive(&tempty[1]); }
+    }
 }
 
 // Epilogue role with TMA stores, NCHW output (warps 4-11).  Each warp moves its 32 rows x up to 64 channels on
@@ -337,7 +405,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (lane == 0) {
       PROF_BEGIN();
       uint32_t s = 0, phase = 0;
-      for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x) {
+      for (unsigned i = 0, t; (t = tile_of_iter(p, i)) < total && !*abort_flag; ++i) {
         const Tile tile = decode_tile(p, t);
         TapWalk<MODE> tw;
         tw.init(p, tile);
@@ -383,7 +451,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       for (int i = 0; i < 4; ++i) idesc_id[i] = idesc_with_sf_ids(p.idesc, i, i);
       uint32_t s = 0, phase = 0, tcount = 0;
       PROF_BEGIN();
-      for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
+      for (unsigned t; (t = tile_of_iter(p, tcount)) < total && !*abort_flag; ++tcount) {
         const Tile tile = decode_tile(p, t);
         TapWalk<MODE> tw;
         tw.init(p, tile);
@@ -432,7 +500,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const uint64_t sfb_desc0 = smem_desc(sf_desc, smem_u32(smem + A_STAGE_BYTES + b_stage_bytes + SFA_BYTES));
       uint32_t s = 0, phase = 0;
       bool alive = true;
-      for (unsigned t = blockIdx.x; t < total && alive && !*abort_flag; t += gridDim.x) {
+      for (unsigned i = 0, t; (t = tile_of_iter(p, i)) < total && alive && !*abort_flag; ++i) {
         const Tile tile = decode_tile(p, t);
         TapWalk<MODE> tw;
         tw.init(p, tile);
@@ -453,7 +521,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else if (warp >= 4) {
-    if (p.tma_store) epilogue_tma_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total);
+    if (p.pair) epilogue_pair_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
+    else if (p.tma_store) epilogue_tma_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
   }
   // teardown: everyone meets here (all loops are bounded), then the allocating warp frees TMEM
@@ -1039,7 +1108,8 @@ cudaError_t launch_conv_tc_inst(const ConvTcParams& p, const CUtensorMap& map_a,
   int dev = 0, sms = 148;
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  const unsigned grid = (unsigned)(p.total_tiles < sms ? p.total_tiles : sms);
+  const long long units = p.pair ? p.total_tiles / 2 : p.total_tiles;
+  const unsigned grid = (unsigned)(units < sms ? units : sms);
   count_launches(1);
   return launch_pdl(conv_tc_kernel<MODE, KB, FP4>, dim3(grid), dim3(TC_THREADS), smem, s, map_a, map_b, map_out, p);
 }

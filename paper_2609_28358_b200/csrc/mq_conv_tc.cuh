@@ -52,6 +52,7 @@ struct ConvTcParams {
   int halo_b_bytes;         // bytes of the resident weight image + its scale chunks (rounded up to 1024)
   int fused;                // 1: single channel tile, stride 1: no preparation kernel (the blocks build the weight image, its
                             //    scale chunks and every tile's activation scale chunks themselves)
+  int pair;                 // per-tap kernel, input gradient with column stride 2, NCHW output: see tile_of_iter
   int tma_store;            // 1: NCHW output written by TMA stores from per-warp staging slices
   const uint8_t* b_codes;   // weight-like codes [rows][taps][b_rowbytes] (source of the images below)
   int b_rows_total, b_rowbytes;
