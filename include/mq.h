@@ -153,7 +153,10 @@ mq_status mq_conv_bwd_weight(const mq_conv_desc* desc, const mq_qtensor* xq, con
  * copies X, W, G_Y (fp32; NCHW / OIHW / N.C_out.Ho.Wo; pinned memory makes the copies asynchronous)
  * into `arena`, runs mq_quantize on each once, mq_cbf_im2col, mq_conv_fwd, mq_conv_bwd_data and
  * mq_conv_bwd_weight, and copies Y, G_X, G_W (fp32, MQ_NCHW layouts) back to the host buffers.
- * Everything is enqueued on `stream`; the host results are valid after the stream is synchronised.
+ * The kernels are enqueued on `stream`; the copies run on two library-owned side streams (one per direction,
+ * created on first use, no device memory involved) tied to `stream` by events, so uploads and downloads
+ * overlap the kernels; `stream` waits for the last download, so the host results are valid after `stream`
+ * is synchronised and successive calls on one stream stay ordered.
  * arena: device memory, arena_bytes >= mq_conv_layer_host_arena_size(); contents are scratch. */
 mq_status mq_conv_layer_host_arena_size(const mq_conv_desc* desc, int fmt_x, int fmt_w, int fmt_dy, size_t* bytes);
 mq_status mq_conv_layer_host(const mq_conv_desc* desc, int fmt_x, int fmt_w, int fmt_dy, const float* x_host, const float* w_host,

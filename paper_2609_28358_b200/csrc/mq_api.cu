@@ -669,6 +669,23 @@ LayerArena layer_arena(const mq_conv_desc* desc, const int fmts[3]) {
 }
 }  // namespace
 
+// Side streams and events of mq_conv_layer_host, created once per device (no device memory is allocated).
+struct HostPipe { cudaStream_t h2d, d2h; cudaEvent_t ev[8]; bool ready; };
+static HostPipe* host_pipe() {
+  static HostPipe pipes[32];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 32) return nullptr;
+  HostPipe* hp = &pipes[dev];
+  if (!hp->ready) {
+    if (cudaStreamCreateWithFlags(&hp->h2d, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    if (cudaStreamCreateWithFlags(&hp->d2h, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
+    for (int i = 0; i < 8; ++i)
+      if (cudaEventCreateWithFlags(&hp->ev[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
+    hp->ready = true;
+  }
+  return hp;
+}
+
 mq_status mq_conv_layer_host_arena_size(const mq_conv_desc* desc, int fmt_x, int fmt_w, int fmt_dy, size_t* bytes) {
   mq_status st = check_desc(desc);
   if (st != MQ_OK) return st;
@@ -691,24 +708,41 @@ mq_status mq_conv_layer_host(const mq_conv_desc* desc, int fmt_x, int fmt_w, int
   if (arena_bytes < L.total) return MQ_ERR_BUFFER_TOO_SMALL;
   uint8_t* base = static_cast<uint8_t*>(arena);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
-  if (cudaMemcpyAsync(base + L.off_x, x_host, L.nx, cudaMemcpyHostToDevice, s) != cudaSuccess) return MQ_ERR_CUDA;
-  if (cudaMemcpyAsync(base + L.off_w, w_host, L.nw, cudaMemcpyHostToDevice, s) != cudaSuccess) return MQ_ERR_CUDA;
-  if (cudaMemcpyAsync(base + L.off_g, dy_host, L.ng, cudaMemcpyHostToDevice, s) != cudaSuccess) return MQ_ERR_CUDA;
+  // Copies run on two side streams of their own (one per direction: the copy engines are full duplex) and are tied to
+  // the caller's stream by events, so the upload of G_Y overlaps the forward half of the step and the download of Y
+  // overlaps the backward half.  The caller's stream waits for the last download: synchronising it is enough.
+  HostPipe* hp = host_pipe();
+  if (!hp) return MQ_ERR_CUDA;
+  auto ok = [](cudaError_t e) { return e == cudaSuccess; };
+  if (!ok(cudaEventRecord(hp->ev[0], s)) || !ok(cudaStreamWaitEvent(hp->h2d, hp->ev[0], 0)) || !ok(cudaStreamWaitEvent(hp->d2h, hp->ev[0], 0)))
+    return MQ_ERR_CUDA;
+  if (!ok(cudaMemcpyAsync(base + L.off_x, x_host, L.nx, cudaMemcpyHostToDevice, hp->h2d)) || !ok(cudaEventRecord(hp->ev[1], hp->h2d))) return MQ_ERR_CUDA;
+  if (!ok(cudaMemcpyAsync(base + L.off_w, w_host, L.nw, cudaMemcpyHostToDevice, hp->h2d)) || !ok(cudaEventRecord(hp->ev[2], hp->h2d))) return MQ_ERR_CUDA;
+  if (!ok(cudaMemcpyAsync(base + L.off_g, dy_host, L.ng, cudaMemcpyHostToDevice, hp->h2d)) || !ok(cudaEventRecord(hp->ev[3], hp->h2d))) return MQ_ERR_CUDA;
   mq_qtensor q[3];
   const size_t src_off[3] = {L.off_x, L.off_w, L.off_g};
   for (int r = 0; r < 3; ++r) {
     q[r].codes = base + L.off_qc[r]; q[r].scales = base + L.off_qs[r];
     q[r].codes_bytes = L.qc[r]; q[r].scales_bytes = L.qs[r]; q[r].fmt = fmts[r]; q[r].role = r;
-    if ((st = mq_quantize(desc, base + src_off[r], MQ_NCHW, &q[r], stream)) != MQ_OK) return st;
   }
-  if ((st = mq_cbf_im2col(desc, &q[0], base + L.off_ic, base + L.off_is, stream)) != MQ_OK) return st;
   void* ws = L.ws ? base + L.off_ws : nullptr;
+  if (!ok(cudaStreamWaitEvent(s, hp->ev[1], 0))) return MQ_ERR_CUDA;
+  if ((st = mq_quantize(desc, base + src_off[0], MQ_NCHW, &q[0], stream)) != MQ_OK) return st;
+  if (!ok(cudaStreamWaitEvent(s, hp->ev[2], 0))) return MQ_ERR_CUDA;
+  if ((st = mq_quantize(desc, base + src_off[1], MQ_NCHW, &q[1], stream)) != MQ_OK) return st;
+  if ((st = mq_cbf_im2col(desc, &q[0], base + L.off_ic, base + L.off_is, stream)) != MQ_OK) return st;
   if ((st = mq_conv_fwd(desc, &q[0], &q[1], base + L.off_y, MQ_NCHW, ws, L.ws, stream)) != MQ_OK) return st;
+  if (!ok(cudaEventRecord(hp->ev[4], s)) || !ok(cudaStreamWaitEvent(hp->d2h, hp->ev[4], 0))) return MQ_ERR_CUDA;
+  if (!ok(cudaMemcpyAsync(y_host, base + L.off_y, L.ng, cudaMemcpyDeviceToHost, hp->d2h))) return MQ_ERR_CUDA;
+  if (!ok(cudaStreamWaitEvent(s, hp->ev[3], 0))) return MQ_ERR_CUDA;
+  if ((st = mq_quantize(desc, base + src_off[2], MQ_NCHW, &q[2], stream)) != MQ_OK) return st;
   if ((st = mq_conv_bwd_data(desc, &q[1], &q[2], base + L.off_dx, MQ_NCHW, ws, L.ws, stream)) != MQ_OK) return st;
+  if (!ok(cudaEventRecord(hp->ev[5], s)) || !ok(cudaStreamWaitEvent(hp->d2h, hp->ev[5], 0))) return MQ_ERR_CUDA;
+  if (!ok(cudaMemcpyAsync(dx_host, base + L.off_dx, L.nx, cudaMemcpyDeviceToHost, hp->d2h))) return MQ_ERR_CUDA;
   if ((st = mq_conv_bwd_weight(desc, &q[0], &q[2], base + L.off_dw, MQ_NCHW, ws, L.ws, stream)) != MQ_OK) return st;
-  if (cudaMemcpyAsync(y_host, base + L.off_y, L.ng, cudaMemcpyDeviceToHost, s) != cudaSuccess) return MQ_ERR_CUDA;
-  if (cudaMemcpyAsync(dx_host, base + L.off_dx, L.nx, cudaMemcpyDeviceToHost, s) != cudaSuccess) return MQ_ERR_CUDA;
-  if (cudaMemcpyAsync(dw_host, base + L.off_dw, L.nw, cudaMemcpyDeviceToHost, s) != cudaSuccess) return MQ_ERR_CUDA;
+  if (!ok(cudaEventRecord(hp->ev[6], s)) || !ok(cudaStreamWaitEvent(hp->d2h, hp->ev[6], 0))) return MQ_ERR_CUDA;
+  if (!ok(cudaMemcpyAsync(dw_host, base + L.off_dw, L.nw, cudaMemcpyDeviceToHost, hp->d2h))) return MQ_ERR_CUDA;
+  if (!ok(cudaEventRecord(hp->ev[7], hp->d2h)) || !ok(cudaStreamWaitEvent(s, hp->ev[7], 0))) return MQ_ERR_CUDA;
   return MQ_OK;
 }
 
