@@ -157,3 +157,25 @@ def test_config5_points_full_size(name):
     qs = check_quantize(ol)
     check_im2col(ol, qs[0])
     check_convs(ol, qs, samples=4000)
+
+
+@pytest.mark.parametrize("fmts", [(E4M3, E4M3, E5M2), (E2M1, E2M1, E2M1)], ids=["fp8", "fp4"])
+def test_layer_from_host_buffers_matches_the_device_calls(fmts):
+    """mq_conv_layer_host (pinned host tensors in, host results out, copies overlapped with the kernels) gives, twice in a
+    row, exactly what the separate device-side calls give."""
+    d = inputs.conv_desc(64, 64, 12, 16, 96, 3, 1, 1)
+    layer = make_layer("host", d, fmts, seed=11, kinds=("relu", "kaiming", "gauss"))
+    x, w, g = inputs.layer_tensors(layer)
+    q = [mq.quantize(d, r, f, torch.from_numpy(t).cuda()) for r, f, t in zip((0, 1, 2), fmts, (x, w, g))]
+    want = (mq.conv_fwd(d, q[0], q[1]).cpu(), mq.conv_bwd_data(d, q[1], q[2]).cpu(), mq.conv_bwd_weight(d, q[0], q[2]).cpu())
+    hx, hw, hg = [torch.from_numpy(t).pin_memory() for t in (x, w, g)]
+    outs = [torch.empty(t.shape, dtype=torch.float32).pin_memory() for t in want]
+    arena = torch.empty(mq.conv_layer_host_arena_size(d, *fmts), dtype=torch.uint8, device="cuda")
+    for _ in range(2):
+        for o in outs:
+            o.fill_(float("nan"))
+        mq.conv_layer_host(d, fmts, hx, hw, hg, outs[0], outs[1], outs[2], arena)
+        torch.cuda.synchronize()
+        for name, got, exp in zip(("Y", "dX", "dW"), outs, want):
+            assert torch.equal(got, exp), f"{name} from host buffers differs from the device call"
+    assert mq.last_device_status() == 0
