@@ -193,14 +193,10 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   p.halo = 0;
   if (g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && taps <= 64 && !env_int("MQ_TC_NO_HALO", 0)) {
     const int spa = fp4 ? 2 : 1, atoms_b = (p.BN + 127) / 128;
-    int nbox = env_int("MQ_TC_NBOX", 0);
-    if (nbox != 1 && nbox != g.Kw) nbox = (layout == MQ_NCHW && p.TW >= 16) ? g.Kw : 1;
-    if (g.Kw == 1) nbox = 1;
-    if ((nbox == 1 && p.TW == 8) || (nbox > 1 && p.TW >= 8)) {
-      p.nbox = nbox;
-      p.WH = nbox == 1 ? p.TW + g.Kw - 1 : p.TW;
+    if (p.TW == 8) {
+      p.WH = p.TW + g.Kw - 1;
       p.halo_box_bytes = g.Kh * p.WH * p.TN * p.KB;
-      p.halo_a_bytes = (nbox * p.halo_box_bytes + 1023) / 1024 * 1024;
+      p.halo_a_bytes = (p.halo_box_bytes + 1023) / 1024 * 1024;
       p.halo_stage_bytes = (p.halo_a_bytes + p.max_stages * 512 * spa + 1023) / 1024 * 1024;
       p.halo_b_bytes = (taps * p.BN * p.KB + p.max_stages * 512 * spa * atoms_b + 1023) / 1024 * 1024;
       const int halo_tma = tma_store_ok && !env_int("MQ_TC_NO_TMA_STORE", 0) ? 1 : 0;
@@ -208,7 +204,7 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
       if (hst > 4) hst = 4;
       // TMEM: accumulator(s), 16 columns per chunk of resident weight scales, 8 per chunk per stage
       while (hst >= 2 && p.BN + 16 * p.max_stages + 8 * p.max_stages * hst > 512) --hst;
-      if (hst >= 2 && p.WH <= 256 && (p.halo_box_bytes % 1024 == 0 || nbox == 1)) {
+      if (hst >= 2 && p.WH <= 256) {
         p.halo = 1;
         p.tma_store = halo_tma;
         p.fused = p.tiles_c == 1 && p.TN <= 32 && g.Kh * (p.TW + g.Kw - 1) * (p.KB / 32) * spa <= 128 && !env_int("MQ_TC_NO_FUSED", 0);
@@ -260,7 +256,7 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
   p.sfa_img = base + pl.off_sfa;
   p.sfb_img = base + pl.off_sfb;
   p.b_codes = b_codes; p.b_rows_total = pl.rows_b; p.b_rowbytes = pl.rowbytes; p.b_img = base + pl.off_bimg;
-  p.out = out; p.out_layout = env_int("MQ_TC_SKIP_STORE", 0) ? 99 : layout; p.status = status;
+  p.out = out; p.out_layout = layout; p.status = status;
   if (!(p.halo && p.fused) && launch_expand_conv_scales(p, stream) != cudaSuccess) return MQ_ERR_CUDA;
 
   CUtensorMap map_a, map_w;
@@ -457,13 +453,16 @@ mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const 
   return launch_bwd_weight_reduce(partial, out, g, p.splits, layout, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }
 
+// address of the current device's status word (a __device__ variable has one instance per device)
 unsigned int* device_status_ptr() {
-  static unsigned int* ptr = nullptr;
-  if (!ptr) {
+  static unsigned int* ptrs[64] = {nullptr};
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  if (!ptrs[dev]) {
     void* q = nullptr;
-    if (cudaGetSymbolAddress(&q, g_device_status) == cudaSuccess) ptr = static_cast<unsigned int*>(q);
+    if (cudaGetSymbolAddress(&q, g_device_status) == cudaSuccess) ptrs[dev] = static_cast<unsigned int*>(q);
   }
-  return ptr;
+  return ptrs[dev];
 }
 
 mq_status run_conv(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int role_a, const mq_qtensor* qb, int role_b,

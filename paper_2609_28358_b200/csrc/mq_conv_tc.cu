@@ -184,7 +184,7 @@ __device__ __forceinline__ void epilogue_role(const ConvTcParams& p, uint32_t tm
 #pragma unroll
           for (int j = 0; j < 16; ++j) v[j] = 0u;
         }
-        if (row_ok && p.out_layout != 99) {
+        if (row_ok) {
           if (p.out_layout == MQ_NCHW) {
 #pragma unroll
             for (int j = 0; j < 16; ++j) { if (full_cols || tile.c0 + c + j < p.Cd) *o_nchw = __uint_as_float(v[j]); o_nchw += cs; }
@@ -253,7 +253,7 @@ __device__ __forceinline__ void epilogue_pair_role(const ConvTcParams& p, uint32
 #pragma unroll
           for (int q = 0; q < 16; ++q) v1[q] = 0u;
         }
-        if (row_ok && p.out_layout != 99) {
+        if (row_ok) {
 #pragma unroll
           for (int q = 0; q < 16; ++q) {
             if (t0.c0 + c + q < p.Cd) *reinterpret_cast<float2*>(o) = make_float2(__uint_as_float(v0[q]), __uint_as_float(v1[q]));
@@ -343,7 +343,7 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
         }
         fence_proxy_async_smem();
         __syncwarp();
-        if (lane == 0 && p.out_layout != 99) {
+        if (lane == 0) {
           if (!hwnc) tma_store_4d(map_out, buf, tile.w0, tile.n0 + n_off, tile.c0 + c0, yo);
           else {
             tma_store_4d(map_out, buf, tile.c0 + c0, tile.w0, tile.n0 + n_off, yo);
@@ -581,13 +581,9 @@ __device__ __forceinline__ void halo_build_sfb(const ConvTcParams& p, uint8_t* s
 //    RESIDENT: one bulk copy when the channel tile changes (never, when the layer has a single channel tile),
 //    its scale vectors copied to TMEM once;
 //  * a pipeline stage holds the whole K range of a tile's activations, every stored pixel once (the data reuse
-//    of Sec. IV-A), and each tap's A operand is a view into it.  Two shapes:
-//      nbox == 1  one TMA box [Kh rows][TN samples][TW + Kw - 1 columns][KB]; tap (kh, kw) starts at
-//                 (kh * TN * WH + kw) * KB with 8-row groups WH * KB bytes apart (TW = 8: one 8-row swizzle
-//                 group per sample);
-//      nbox == Kw one box [Kh][TN][TW][KB] per column shift (TW = 8, 16 or 32); tap (kh, kw) is the plain
-//                 128-row operand at ((kw * Kh + kh) * 128) * KB.  Longer runs of output columns per warp for
-//                 an NCHW store, at Kw times the shared-memory footprint.
+//    of Sec. IV-A): ONE TMA box [Kh rows][TN samples][TW + Kw - 1 columns][KB], and each tap's A operand is a
+//    view into it: tap (kh, kw) starts at (kh * TN * WH + kw) * KB with 8-row groups WH * KB bytes apart (TW = 8:
+//    one 8-row swizzle group per sample).
 // Roles and barriers are those of conv_tc_kernel, plus bfull / bempty for the resident weight tile.
 // With a single channel tile (p.fused) no preparation kernel runs at all: every block builds the weight image and
 // its scale chunks in shared memory itself at start-up, and warp 3 expands each tile's activation scales (a
@@ -651,7 +647,7 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     // forward reads halo row kh, column shift kw; the input gradient walks the taps in the same order but its
     // source pixel moves the other way
     const int hrow = MODE == MQ_OP_FWD ? kh : p.Kh - 1 - kh, wsh = MODE == MQ_OP_FWD ? kw : p.Kw - 1 - kw;
-    const int aoff = p.nbox == 1 ? (hrow * p.TN * p.WH + wsh) * KB : (wsh * p.Kh + hrow) * 128 * KB;
+    const int aoff = (hrow * p.TN * p.WH + wsh) * KB;
     tap_a[threadIdx.x] = (uint32_t)aoff >> 4;
     tap_b[threadIdx.x] = (uint32_t)(threadIdx.x * p.BN * KB) >> 4;
     tap_p[threadIdx.x] = (uint32_t)(hrow * (p.TW + p.Kw - 1) + wsh);
@@ -694,9 +690,8 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // first source pixel of the halo: forward (h - ph, w0 - pw); input gradient (h + ph - (Kh-1), w0 + pw - (Kw-1))
         const int hs = MODE == MQ_OP_FWD ? tile.h - p.ph : tile.h + p.ph - (p.Kh - 1);
         const int ws = MODE == MQ_OP_FWD ? tile.w0 - p.pw : tile.w0 + p.pw - (p.Kw - 1);
-        mbar_arrive_expect_tx(&full[s], (uint32_t)(p.nbox * p.halo_box_bytes + (p.fused ? 0 : sfa_bytes)));
-#pragma unroll 1
-        for (int b = 0; b < p.nbox; ++b) tma_load_4d(sa + (size_t)b * p.halo_box_bytes, &map_a, &full[s], 0, ws + b, tile.n0, hs);
+        mbar_arrive_expect_tx(&full[s], (uint32_t)(p.halo_box_bytes + (p.fused ? 0 : sfa_bytes)));
+        tma_load_4d(sa, &map_a, &full[s], 0, ws, tile.n0, hs);
         if (!p.fused) bulk_load(sa + p.halo_a_bytes, p.sfa_img + (size_t)tile_m_index(p, tile) * sfa_bytes, sfa_bytes, &full[s]);
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
@@ -705,7 +700,7 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer: all taps of a tile per stage
     if (lane == 0) {
-      const uint64_t a_desc_base = smem_desc_base(16, (uint32_t)((p.nbox == 1 ? p.WH : 8) * KB), LAYOUT);
+      const uint64_t a_desc_base = smem_desc_base(16, (uint32_t)(p.WH * KB), LAYOUT);   // 8-row groups one halo row apart
       const uint64_t b_desc_base = smem_desc_base(16, 8 * KB, LAYOUT);
       const uint32_t sb16 = smem_u32(smem) >> 4;
       uint32_t idesc_id[4];

@@ -44,8 +44,7 @@ struct ConvTcParams {
   int max_stages;           // stages of the longest tile
   // whole-tile-per-stage variant (small channel counts, stride 1): see conv_tc_halo_kernel
   int halo;                 // 1: use it
-  int nbox;                 // activation boxes per tile: 1 (one box with the column halo) or Kw (one box per column shift)
-  int WH;                   // columns per box: TW + Kw - 1 (nbox == 1) or TW
+  int WH;                   // columns of the activation halo box = TW + Kw - 1
   int halo_box_bytes;       // bytes of one activation box = Kh * TN * WH * KB
   int halo_a_bytes;         // bytes of a tile's activation boxes (rounded up to 1024)
   int halo_stage_bytes;     // bytes of one pipeline stage (activation boxes + A-side scale chunks)
