@@ -345,6 +345,11 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   // shared-memory operand reads, and a wider N reads the G_Y tile once for twice the work)
   if (fp8 && g.Cp >= 256 && !env_int("MQ_WGRAD_N128", 0)) p.b_rows = 256;
   p.m_tiles = (g.Cout + 127) / 128;
+  p.m_tiles128 = p.m_tiles;
+  // Pairs of blocks on 256 x 256 tiles (cta_group::2): correct, but measured 1.35x slower than single blocks on
+  // 128 x 256 tiles, whose neighbours already share their X loads on the way from L2; opt-in only.
+  p.cta2 = fp8 && p.b_rows == 256 && g.Cout >= 256 && env_int("MQ_WGRAD_CTA2", 0);
+  if (p.cta2) { p.m_tiles = (g.Cout + 255) / 256; p.m_tiles128 = 2 * p.m_tiles; }
   p.cb_tiles = (g.Cp + p.b_rows - 1) / p.b_rows;
   // taps per block: a whole kernel row in the flat mode when its accumulators fit in tensor memory
   p.TG = 1;
@@ -355,11 +360,12 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   p.j_tiles = (g.Kh * g.Kw / p.TG) * p.cb_tiles;
   const int items = p.m_tiles * p.j_tiles;
   int splits = env_int("MQ_WGRAD_SPLITS", 0);
-  if (splits <= 0) splits = items >= 148 ? 1 : 148 / items;
+  const int units = p.cta2 ? 74 : 148;   // blocks, or pairs of blocks, that run at once
+  if (splits <= 0) splits = items >= units ? 1 : units / items;
   if (splits > p.stages_total) splits = p.stages_total;
   if (splits < 1) splits = 1;
   p.splits = splits;
-  p.b_tile_bytes = flat ? (p.KPX + p.TG - 1) * p.b_rows * p.KBn : p.b_rows * 128;
+  p.b_tile_bytes = flat ? (p.KPX + p.TG - 1) * p.b_rows * p.KBn : (p.cta2 ? 128 : p.b_rows) * 128;   // a pair's blocks load half of X each
   p.stage_bytes = (128 * 128 + p.b_tile_bytes + (1 + p.NB) * 1024 + 1023) / 1024 * 1024;
   {
     int st = (227 * 1024 - 2048) / p.stage_bytes;
@@ -374,7 +380,7 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   w.P_a = p.stages_total * p.KPX;
   w.P_b = (w.P_a + (g.Kh - 1) * p.Wp + g.Kw - 1 + 7) / 8 * 8;
   size_t o = up256((size_t)splits * g.Cout * g.Kh * g.Kw * g.Cp * sizeof(float));
-  w.off_sfa = o; o += up256((size_t)p.m_tiles * p.stages_total * 512 * spa);
+  w.off_sfa = o; o += up256((size_t)p.m_tiles128 * p.stages_total * 512 * spa);
   w.off_sfb = o; o += up256((size_t)p.cb_tiles * (g.Kh * g.Kw / p.TG) * p.stages_total * p.NB * 512 * spa);
   w.off_xt = o;
   if (flat) { p.xt_block_bytes = (long long)w.P_b * p.b_rows * p.KBn; o += up256((size_t)p.cb_tiles * p.xt_block_bytes); }
@@ -420,7 +426,7 @@ mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const 
     }
   } else {
     const uint32_t fa = qg->fmt == MQ_E5M2 ? 1u : 0u, fb = qx->fmt == MQ_E5M2 ? 1u : 0u;
-    p.idesc = (fa << 7) | (fb << 10) | (1u << 15) | (1u << 16) | (1u << 23) | ((128u >> 4) << 24);
+    p.idesc = (fa << 7) | (fb << 10) | (1u << 15) | (1u << 16) | (1u << 23) | (((p.cta2 ? 256u : 128u) >> 4) << 24);
     {
       const uint64_t rb = (uint64_t)g.Cop;
       const uint64_t dims[4] = {rb, (uint64_t)g.N, (uint64_t)g.Wo, (uint64_t)g.Ho};

@@ -94,7 +94,9 @@ struct WgradTcParams {
   int stages_total;     // pixel: Ho * groups_w * nchunks; flat: ceil(Ho * Wp / KPX)
   int Wp;               // flat: padded width W + 2 * pw
   int b_rows;           // rows (input channels) of a B tile: 128, or min(128, Cp) in flat mode
-  int m_tiles, j_tiles, cb_tiles, splits;   // j_tiles = (taps / TG) * cb_tiles
+  int m_tiles, j_tiles, cb_tiles, splits;   // j_tiles = (taps / TG) * cb_tiles; m_tiles counts work units along C_out
+  int m_tiles128;       // 128-row tiles of output channels (= m_tiles, or 2 * m_tiles when cta2)
+  int cta2;             // 1: pairs of blocks (clusters of 2) compute 256 x 256 tiles with cta_group::2 MMAs
   int TG;               // taps per block: 1, or Kw (flat mode: the taps of a kernel row share the stage's pixels)
   int NB;               // 128-row chunks of the group's B rows = ceil(TG * b_rows / 128)
   int n0, n1;           // MMA widths per K slice: n0 = min(TG * b_rows, 256) and the rest (0: one MMA)

@@ -54,7 +54,7 @@ __device__ __forceinline__ void expand_wgrad_scales_body(const WgradTcParams& p,
   const int lane = threadIdx.x & 31;
   const long long wid = (long long)block * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const int taps = p.Kh * p.Kw;
-  const long long nA = (long long)p.m_tiles * p.stages_total;
+  const long long nA = (long long)p.m_tiles128 * p.stages_total;
   const int groups = taps / p.TG;
   const long long nB = (long long)p.cb_tiles * groups * p.stages_total * p.NB;
   if (wid >= nA + nB) return;
@@ -112,7 +112,14 @@ __device__ __forceinline__ void expand_wgrad_scales_body(const WgradTcParams& p,
 template <bool FP4>
 __global__ void __launch_bounds__(256) expand_wgrad_scales_kernel(const WgradTcParams p) { pdl_wait(); expand_wgrad_scales_body<FP4>(p, blockIdx.x); }
 
-template <bool FP4>
+//
+// CTA2 (8-bit operands, C_out and C_in >= 256): the two blocks of a cluster compute a 256 x 256 tile with
+// cta_group::2 MMAs.  Each block loads its own 128 output channels of G_Y and its own 128 of the tile's 256 input
+// channels of X, so a block's shared memory receives and supplies two thirds of the bytes per FLOP of the one-block
+// 128 x 256 tile -- and the shared-memory operand path is what bounds these kernels.  The leader block's threads issue
+// the scale copies, MMAs and commits for the pair; the other block only loads, relays "my stage has landed" to the
+// leader's barrier, and stores its half of the result.
+template <bool FP4, bool CTA2>
 __global__ void __launch_bounds__(WG_THREADS, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_p,
                 const WgradTcParams p) {
@@ -127,19 +134,23 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   uint64_t* empty = full + p.stages;
   uint64_t* sffull = empty + p.stages;
   uint64_t* tfull = sffull + p.stages;
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tfull + 1);
+  uint64_t* pfull = tfull + 1;                         // CTA2, leader: the peer block's stage has landed
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pfull + p.stages);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
 
   // work item
-  int item = blockIdx.x;
-  const int mt = item % p.m_tiles; item /= p.m_tiles;
+  const uint32_t rank = CTA2 ? cluster_ctarank() : 0u;  // 0: leader
+  int item = CTA2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
+  const int mu = item % p.m_tiles; item /= p.m_tiles;
+  const int mt = CTA2 ? 2 * mu + (int)rank : mu;        // 128-row tile of output channels
   const int jt = item % p.j_tiles;
   const int split = item / p.j_tiles;
   const int tgi = jt / p.cb_tiles, cb = jt - tgi * p.cb_tiles;
   const int tap0 = tgi * TG;                            // first tap of the group (TG divides Kw)
   const int kh = tap0 / p.Kw, kw = tap0 - kh * p.Kw;
-  const int co0 = mt * 128, ci0 = cb * p.b_rows;
+  const int co0 = mt * 128, ci0 = cb * p.b_rows;         // the tile's first output / input channel
+  const int ci_ld = ci0 + (CTA2 ? 128 * (int)rank : 0);  // first input channel this block loads (its half, in a pair)
   const int st_begin = (int)((long long)p.stages_total * split / p.splits);
   const int st_end = (int)((long long)p.stages_total * (split + 1) / p.splits);
   const int nst = st_end - st_begin;
@@ -148,16 +159,20 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 
   if (threadIdx.x == 0) {
 #pragma unroll 1
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); }
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); mbar_init(&pfull[s], 1); }
     mbar_init(tfull, 1);
     *abort_flag = 0;
     mbar_fence_init();
     if (p.mode != MQ_WG_FP4_FLAT) { prefetch_tensormap(&map_a); prefetch_tensormap(&map_b); }
     prefetch_tensormap(&map_p);
   }
-  if (warp == 1) { tmem_alloc(tmem_slot, p.tmem_cols); tmem_relinquish(); }
+  if (warp == 1) {
+    if (CTA2) { tmem_alloc_2(tmem_slot, p.tmem_cols); tmem_relinquish_2(); }
+    else { tmem_alloc(tmem_slot, p.tmem_cols); tmem_relinquish(); }
+  }
   tc_fence_before_sync();
   __syncthreads();
+  if (CTA2) cluster_sync_all();   // both blocks' barriers and tensor memory exist before anything crosses over
   tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
   pdl_wait();   // set-up above touched only shared memory, tensor memory and the kernel parameters
@@ -206,8 +221,8 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           } else {
             // stored [ho][wo][n][c] codes: box (128 channel bytes, n rows, pixels, 1)
             tma_load_4d(sa, &map_a, &full[s], co0, nc * p.BPP * 32, wo0, ho);
-            tma_load_4d(sb, &map_b, &full[s], ci0, nc * p.BPP * 32, wo0 * p.sw + kw - p.pw, ho * p.sh + kh - p.ph);
-            if (p.b_rows > 128)   // second 128-channel panel of a 256-channel tile
+            tma_load_4d(sb, &map_b, &full[s], ci_ld, nc * p.BPP * 32, wo0 * p.sw + kw - p.pw, ho * p.sh + kh - p.ph);
+            if (!CTA2 && p.b_rows > 128)   // second 128-channel panel of a 256-channel tile (the peer block's in a pair)
               tma_load_4d(sb + 128 * 128, &map_b, &full[s], ci0 + 128, nc * p.BPP * 32, wo0 * p.sw + kw - p.pw, ho * p.sh + kh - p.ph);
           }
         }
@@ -216,8 +231,8 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       WPROF(2);
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    // ------------------------------------------------------------------ MMA issuer (the leader's, in a pair)
+    if (lane == 0 && rank == 0) {
       // 8-bit: MN-major tiles [K row][128 bytes], 128-byte swizzle, 8-row groups 1024 bytes apart; an MMA
       // takes 32 K rows (4096 bytes).  E2M1: K-major pieces [rows][KBn bytes], swizzle span = KBn (none for
       // 16: 8x16-byte core matrices, the next 16 bytes of K one piece further); an MMA takes 32 bytes of K.
@@ -258,14 +273,19 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             const uint32_t idesc = idesc_with_sf_ids(idesc_n[m], id, id);
             const uint32_t sfb_m = sfb_t + 4 * (g * p.NB + (m ? (p.n0 >> 7) : 0));
             if (FP4) mma_mxf4(d_t, a_desc0 + so + ka16[a], b_desc0 + bo + kb16[a], idesc, sfa_t + 4 * g, sfb_m, accu);
+            else if (CTA2) mma_mxf8f6f4_2(d_t, a_desc0 + so + ka16[a], b_desc0 + bo + kb16[a], idesc, sfa_t + 4 * g, sfb_m, accu);
             else mma_mxf8f6f4(d_t, a_desc0 + so + ka16[a], b_desc0 + bo + kb16[a], idesc, sfa_t + 4 * g, sfb_m, accu);
           }
         }
         accumulate = 1;
-        tc_commit(&empty[s]);
+        if (CTA2) tc_commit_2_multicast(&empty[s], 3); else tc_commit(&empty[s]);   // frees the stage in both blocks
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
-      if (nst > 0) tc_commit(tfull); else mbar_arrive(tfull);
+      if (CTA2) {
+        if (nst > 0) tc_commit_2_multicast(tfull, 3); else { mbar_arrive(tfull); mbar_arrive_remote(tfull, 1); }
+      } else {
+        if (nst > 0) tc_commit(tfull); else mbar_arrive(tfull);
+      }
       WPROF(3);
     }
   } else if (warp == 2) {
@@ -279,20 +299,31 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 #pragma unroll 1
       for (int i = 0; i < nst && !*abort_flag; ++i) {
         if (!mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+        if (CTA2) {
+          if (rank != 0) {   // relay to the leader; its copier issues the copies for both blocks
+            mbar_arrive_remote(&pfull[s], 0);
+            if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
+            continue;
+          }
+          if (!mbar_wait(&pfull[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+        }
         tc_fence_after_sync();
         const uint32_t so = s * stage16;
         const uint32_t sf_t = sf_base + s * sf_cols;
-#ifdef MQ_WG_SKIPCP
-        if (i >= p.stages) { tc_commit(&sffull[s]); if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; } continue; }
-#endif
 #pragma unroll
-        for (int g = 0; g < SPA; ++g) tmem_cp_32x128b_warpx4(sf_t + 4 * g, sf_desc0 + so + g * 32);
+        for (int g = 0; g < SPA; ++g) {
+          if (CTA2) tmem_cp_32x128b_warpx4_2(sf_t + 4 * g, sf_desc0 + so + g * 32);
+          else tmem_cp_32x128b_warpx4(sf_t + 4 * g, sf_desc0 + so + g * 32);
+        }
 #pragma unroll 1
         for (int c = 0; c < p.NB; ++c) {     // B-side chunk c: rows [128c, 128c + 128) of the group's operand
 #pragma unroll
-          for (int g = 0; g < SPA; ++g) tmem_cp_32x128b_warpx4(sf_t + 8 + 4 * (g * p.NB + c), sf_desc0 + so + 64 + (c * SPA + g) * 32);
+          for (int g = 0; g < SPA; ++g) {
+            if (CTA2) tmem_cp_32x128b_warpx4_2(sf_t + 8 + 4 * (g * p.NB + c), sf_desc0 + so + 64 + (c * SPA + g) * 32);
+            else tmem_cp_32x128b_warpx4(sf_t + 8 + 4 * (g * p.NB + c), sf_desc0 + so + 64 + (c * SPA + g) * 32);
+          }
         }
-        tc_commit(&sffull[s]);
+        if (CTA2) tc_commit_2(&sffull[s]); else tc_commit(&sffull[s]);
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
     }
@@ -347,7 +378,8 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem, p.tmem_cols);
+  if (CTA2) cluster_sync_all();   // nothing of the peer block is touched after this point
+  if (warp == 1) { if (CTA2) tmem_dealloc_2(tmem, p.tmem_cols); else tmem_dealloc(tmem, p.tmem_cols); }
 #ifdef MQ_TC_PROFILE
   if (threadIdx.x == 0) { WPROF(4); unsigned smid; asm volatile("mov.u32 %0, %smid;" : "=r"(smid)); if (blockIdx.x < 160) g_wblk[blockIdx.x][5] = smid; }
 #endif
@@ -458,26 +490,28 @@ __global__ void __launch_bounds__(256) wgrad_flat_prep_kernel(const FlatArgs x, 
 #ifdef MQ_TC_PROFILE
 extern "C" int mqdbg_read_wblk(unsigned long long* out960) { return cudaMemcpyFromSymbol(out960, g_wblk, sizeof(unsigned long long) * 960) == cudaSuccess ? 0 : 1; }
 #endif
-size_t wgrad_tc_smem_bytes(const WgradTcParams& p) { return 1024 + (size_t)p.stages * p.stage_bytes + (3 * (size_t)p.stages + 2) * 8 + 64; }
+size_t wgrad_tc_smem_bytes(const WgradTcParams& p) { return 1024 + (size_t)p.stages * p.stage_bytes + (4 * (size_t)p.stages + 2) * 8 + 64; }
 
 cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_p, cudaStream_t s) {
-  static bool attr_set[2] = {false, false};
+  static bool attr_set[3] = {false, false, false};
   const size_t smem = wgrad_tc_smem_bytes(p);
-  const int f = p.mode == MQ_WG_FP8 ? 0 : 1;
+  const int f = p.cta2 ? 2 : (p.mode == MQ_WG_FP8 ? 0 : 1);
   if (!attr_set[f]) {
-    cudaError_t e = f ? cudaFuncSetAttribute(wgrad_tc_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)
-                      : cudaFuncSetAttribute(wgrad_tc_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = f == 2 ? cudaFuncSetAttribute(wgrad_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)
+                  : f == 1 ? cudaFuncSetAttribute(wgrad_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)
+                           : cudaFuncSetAttribute(wgrad_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_set[f] = true;
   }
-  const unsigned grid = (unsigned)(p.m_tiles * p.j_tiles * p.splits);
+  const unsigned grid = (unsigned)(p.m_tiles * p.j_tiles * p.splits) * (p.cta2 ? 2u : 1u);
   count_launches(1);
-  if (f) return launch_pdl(wgrad_tc_kernel<true>, dim3(grid), dim3(WG_THREADS), smem, s, map_a, map_b, map_p, p);
-  return launch_pdl(wgrad_tc_kernel<false>, dim3(grid), dim3(WG_THREADS), smem, s, map_a, map_b, map_p, p);
+  if (f == 2) return launch_pdl_cluster(wgrad_tc_kernel<false, true>, dim3(grid), dim3(WG_THREADS), smem, s, 2u, map_a, map_b, map_p, p);
+  if (f == 1) return launch_pdl(wgrad_tc_kernel<true, false>, dim3(grid), dim3(WG_THREADS), smem, s, map_a, map_b, map_p, p);
+  return launch_pdl(wgrad_tc_kernel<false, false>, dim3(grid), dim3(WG_THREADS), smem, s, map_a, map_b, map_p, p);
 }
 
 cudaError_t launch_expand_wgrad_scales(const WgradTcParams& p, cudaStream_t s) {
-  const long long warps = (long long)p.m_tiles * p.stages_total + (long long)p.cb_tiles * (p.Kh * p.Kw / p.TG) * p.stages_total * p.NB;
+  const long long warps = (long long)p.m_tiles128 * p.stages_total + (long long)p.cb_tiles * (p.Kh * p.Kw / p.TG) * p.stages_total * p.NB;
   const unsigned blocks = (unsigned)((warps + 7) / 8);
   count_launches(1);
   if (p.mode == MQ_WG_FP8) return launch_pdl(expand_wgrad_scales_kernel<false>, dim3(blocks), dim3(256), 0, s, p);
@@ -511,7 +545,7 @@ cudaError_t launch_wgrad_flat_prep(const WgradTcParams& p, const uint8_t* x_code
   FlatArgs fx, fg;
   if (!make_flat_args(&fx, x_codes, xt, p.H, p.W, p.N, p.Cp, P_b, p.Wp, p.ph, p.pw, p.b_rows, p.cb_tiles, p.KBn)) return cudaErrorInvalidValue;
   if (!make_flat_args(&fg, g_codes, gt, p.Ho, p.Wo, p.N, p.Cot * 32, P_a, p.Wp, 0, 0, 128, p.m_tiles, p.KBn)) return cudaErrorInvalidValue;
-  const long long warps = (long long)p.m_tiles * p.stages_total + (long long)p.cb_tiles * (p.Kh * p.Kw / p.TG) * p.stages_total * p.NB;
+  const long long warps = (long long)p.m_tiles128 * p.stages_total + (long long)p.cb_tiles * (p.Kh * p.Kw / p.TG) * p.stages_total * p.NB;
   const unsigned sc_blocks = (unsigned)((warps + 7) / 8);
   count_launches(1);
   return launch_pdl(wgrad_flat_prep_kernel, dim3(fx.blocks + fg.blocks + sc_blocks), dim3(256), 0, s, fx, fg, p);
