@@ -28,11 +28,15 @@ using namespace tc;
 __device__ unsigned long long g_wblk[160][6];   // per block: start, after setup, producer done, MMA done, epilogue done, SM id
 __device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
 #define WPROF(slot) do { if (blockIdx.x < 160) g_wblk[blockIdx.x][slot] = gtime(); } while (0)
+__device__ unsigned long long g_wtrace[2][4][256];   // blocks 0 and 1: per stage TMA issue, landed, scales copied, MMAs issued
+#define WTRACE(k, i) do { if (blockIdx.x < 2 && (i) < 256) g_wtrace[blockIdx.x][k][i] = gtime(); } while (0)
 #else
 #define WPROF(slot) do { } while (0)
+#define WTRACE(k, i) do { } while (0)
 #endif
 
 constexpr int WG_THREADS = 256;
+constexpr int WG_PREFETCH = 8;   // stages between an L2 prefetch and the load it serves
 
 // K-block b of stage st: output pixel and 32-sample block
 __device__ __forceinline__ void stage_block(const WgradTcParams& p, int st, int b, int& ho, int& wo, int& nb) {
@@ -137,10 +141,16 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   uint64_t* pfull = tfull + 1;                         // CTA2, leader: the peer block's stage has landed
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pfull + p.stages);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  volatile int* progress = abort_flag + 1;             // stages the G_Y loader has issued (paces the prefetchers)
+  // Warp index and cluster rank go through a shuffle so that the compiler knows them to be warp-uniform: the role
+  // loops below are run by whole warps, their arithmetic stays in the uniform datapath, and only the bulk-copy / MMA /
+  // commit instructions themselves are issued by one elected lane.  (With `if (lane == 0)` around a role, every
+  // operand of those instructions is first moved from a per-thread register, which more than doubles the cycles a
+  // thread spends per MMA or copy.)
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
 
   // work item
-  const uint32_t rank = CTA2 ? cluster_ctarank() : 0u;  // 0: leader
+  const uint32_t rank = CTA2 ? __shfl_sync(0xffffffffu, cluster_ctarank(), 0) : 0u;  // 0: leader
   int item = CTA2 ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;
   const int mu = item % p.m_tiles; item /= p.m_tiles;
   const int mt = CTA2 ? 2 * mu + (int)rank : mu;        // 128-row tile of output channels
@@ -156,12 +166,14 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   const int nst = st_end - st_begin;
   const uint32_t acc_cols = (uint32_t)(TG * p.b_rows);  // accumulators first, then the per-stage scale buffers
   const uint32_t sf_cols = 8u + 8u * (uint32_t)p.NB;
+  const bool has_b1 = p.mode == MQ_WG_FP8 && !CTA2 && p.b_rows > 128;   // a fifth loader: second X panel
 
   if (threadIdx.x == 0) {
 #pragma unroll 1
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); mbar_init(&pfull[s], 1); }
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], has_b1 ? 4 : 3); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); mbar_init(&pfull[s], 1); }
     mbar_init(tfull, 1);
     *abort_flag = 0;
+    *progress = 0;
     mbar_fence_init();
     if (p.mode != MQ_WG_FP4_FLAT) { prefetch_tensormap(&map_a); prefetch_tensormap(&map_b); }
     prefetch_tensormap(&map_p);
@@ -178,61 +190,90 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   pdl_wait();   // set-up above touched only shared memory, tensor memory and the kernel parameters
   if (threadIdx.x == 0) WPROF(1);
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ producer
-    if (lane == 0) {
-      const int taps = p.Kh * p.Kw;
-      const uint8_t* sfa_src = p.sfa_img + ((size_t)mt * p.stages_total + st_begin) * (512 * SPA);
-      const uint32_t sfb_bytes = (uint32_t)p.NB * 512 * SPA;
-      const uint8_t* sfb_src = p.sfb_img + (((size_t)cb * (taps / TG) + tgi) * p.stages_total + st_begin) * sfb_bytes;
-      const uint32_t a_bytes = 128 * 128, b_step = (uint32_t)p.b_rows * 128, b_bytes = (uint32_t)p.b_tile_bytes;
-      const uint8_t* ga = nullptr; const uint8_t* gb = nullptr;
-      if (p.mode == MQ_WG_FP4_FLAT) {
-        ga = p.gt + (size_t)mt * p.gt_block_bytes + (size_t)st_begin * a_bytes;
-        gb = p.xt + (size_t)cb * p.xt_block_bytes + ((size_t)st_begin * p.KPX + (size_t)kh * p.Wp + kw) * ((size_t)p.b_rows * p.KBn);
-      }
-      uint32_t s = 0, phase = 0;
-#pragma unroll 1
-      for (int i = 0; i < nst && !*abort_flag; ++i) {
-        if (!mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
-        uint8_t* sa = smem + (size_t)s * stage_bytes;
-        uint8_t* sb = sa + b_off;
-        uint8_t* ssf = sa + sf_off;
-        mbar_arrive_expect_tx(&full[s], a_bytes + b_bytes + 512 * SPA + sfb_bytes);
-        bulk_load(ssf, sfa_src, 512 * SPA, &full[s]);
-        bulk_load(ssf + 1024, sfb_src, sfb_bytes, &full[s]);
-        sfa_src += 512 * SPA; sfb_src += sfb_bytes;
-        if (p.mode == MQ_WG_FP4_FLAT) {
-          bulk_load(sa, ga, a_bytes, &full[s]);
-          bulk_load(sb, gb, b_bytes, &full[s]);          // KPX + TG - 1 consecutive pixels
-          ga += a_bytes; gb += b_step;
-        } else {
-          const int st = st_begin + i;
-          const int nc = st % p.nchunks; const int t = st / p.nchunks;
-          const int wg = t % p.groups_w, ho = t / p.groups_w;
-          const int wo0 = wg * p.KPX;
-          if (p.mode == MQ_WG_FP4_PIXEL) {
-            // [pixel][c][n] re-laid codes: one box (n bytes, 128 channels) per pixel of the stage
-#pragma unroll 1
-            for (int px = 0; px < p.KPX; ++px) {
-              tma_load_4d(sa + px * 128 * p.KBn, &map_a, &full[s], nc * p.KBn, co0, wo0 + px, ho);
-              tma_load_4d(sb + px * 128 * p.KBn, &map_b, &full[s], nc * p.KBn, ci0, (wo0 + px) * p.sw + kw - p.pw, ho * p.sh + kh - p.ph);
-            }
-          } else {
-            // stored [ho][wo][n][c] codes: box (128 channel bytes, n rows, pixels, 1)
-            tma_load_4d(sa, &map_a, &full[s], co0, nc * p.BPP * 32, wo0, ho);
-            tma_load_4d(sb, &map_b, &full[s], ci_ld, nc * p.BPP * 32, wo0 * p.sw + kw - p.pw, ho * p.sh + kh - p.ph);
-            if (!CTA2 && p.b_rows > 128)   // second 128-channel panel of a 256-channel tile (the peer block's in a pair)
-              tma_load_4d(sb + 128 * 128, &map_b, &full[s], ci0 + 128, nc * p.BPP * 32, wo0 * p.sw + kw - p.pw, ho * p.sh + kh - p.ph);
-          }
-        }
-        if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
-      }
-      WPROF(2);
+  // ------------------------------------------------------------------ loaders
+  // A thread gets one bulk copy accepted per ~265 cycles whatever its size, so a stage's copies are issued by
+  // different warps (one lane each).  Every loader arrives on the stage's barrier with its own byte count.  Four of
+  // these threads belong to the epilogue warps, which have nothing else to do until the accumulators are final.
+  // roles: 0 G_Y tile, 1 X tile (first panel), 2 second X panel, 3 both scale-chunk copies; 4 and 5 prefetch the G_Y and
+  // X boxes of the stage WG_PREFETCH stages ahead into L2 (about a quarter of the lines miss L2, and a box lands only
+  // when its slowest line has: the prefetch takes the DRAM latency out of the pipeline's loop).
+  const int role = warp == 0 ? 0 : (warp == 3 ? 1 : (warp >= 4 ? warp - 2 : -1));
+  if (role >= 0 && (role != 2 || has_b1) && (role < 4 || p.mode != MQ_WG_FP4_PIXEL)) {
+    const int taps = p.Kh * p.Kw;
+    const uint8_t* sfa_src = p.sfa_img + ((size_t)mt * p.stages_total + st_begin) * (512 * SPA);
+    const uint32_t sfb_bytes = (uint32_t)p.NB * 512 * SPA;
+    const uint8_t* sfb_src = p.sfb_img + (((size_t)cb * (taps / TG) + tgi) * p.stages_total + st_begin) * sfb_bytes;
+    const uint32_t a_bytes = 128 * 128, b_step = (uint32_t)p.b_rows * 128;
+    const uint32_t b_bytes = p.mode == MQ_WG_FP8 ? 128u * 128u : (uint32_t)p.b_tile_bytes;   // per loader
+    const uint8_t* ga = nullptr; const uint8_t* gb = nullptr;
+    if (p.mode == MQ_WG_FP4_FLAT) {
+      ga = p.gt + (size_t)mt * p.gt_block_bytes + (size_t)st_begin * a_bytes;
+      gb = p.xt + (size_t)cb * p.xt_block_bytes + ((size_t)st_begin * p.KPX + (size_t)kh * p.Wp + kw) * ((size_t)p.b_rows * p.KBn);
     }
-  } else if (warp == 1) {
+    const uint32_t my_bytes = role == 0 ? a_bytes : (role <= 2 ? b_bytes : 512u * SPA + sfb_bytes);
+    const bool prefetcher = role >= 4;
+    int nc, wg, ho;                                            // of the first stage this warp handles
+    {
+      const int st = st_begin + (prefetcher ? p.stages : 0);
+      nc = st % p.nchunks; const int t = st / p.nchunks;
+      wg = t % p.groups_w; ho = t / p.groups_w;
+    }
+    uint32_t s = 0, phase = 0;
+#pragma unroll 1
+    for (int i = 0; i < nst && !*abort_flag; ++i) {
+      const int ii = prefetcher ? i + p.stages : i;          // the stage this warp's copy is for
+      if (ii >= nst) break;
+      if (prefetcher) {
+        // not a party to the pipeline's barriers: stay at most WG_PREFETCH stages ahead of the loader's counter
+        uint32_t spins = 0;
+        while (ii - *progress > WG_PREFETCH && !*abort_flag && ++spins < kWaitLimit) __nanosleep(64);
+      } else if (!mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+      uint8_t* sa = smem + (size_t)s * stage_bytes;
+      uint8_t* sb = sa + b_off;
+      uint8_t* ssf = sa + sf_off;
+      uint64_t* bar = &full[s];
+      if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
+      const int wo0 = wg * p.KPX;
+      const int xw = wo0 * p.sw + kw - p.pw, xh = ho * p.sh + kh - p.ph;
+      if (elect_one()) {
+        if (role == 0) { WTRACE(0, i); *progress = i; }
+        if (!prefetcher) mbar_arrive_expect_tx(bar, my_bytes);
+        if (role == 3) {
+          bulk_load(ssf, sfa_src + (size_t)i * (512 * SPA), 512 * SPA, bar);
+          bulk_load(ssf + 1024, sfb_src + (size_t)i * sfb_bytes, sfb_bytes, bar);
+        } else if (p.mode == MQ_WG_FP4_FLAT) {
+          if (role == 0) bulk_load(sa, ga + (size_t)i * a_bytes, a_bytes, bar);
+          else if (role == 1) bulk_load(sb, gb + (size_t)i * b_step, b_bytes, bar);          // KPX + TG - 1 consecutive pixels
+          else if (role == 4) bulk_prefetch(ga + (size_t)ii * a_bytes, a_bytes);
+          else bulk_prefetch(gb + (size_t)ii * b_step + (b_bytes - b_step), b_step);          // the pixels stage ii adds
+        } else if (p.mode == MQ_WG_FP4_PIXEL) {
+          // [pixel][c][n] re-laid codes: one box (n bytes, 128 channels) per pixel of the stage
+#pragma unroll 1
+          for (int px = 0; px < p.KPX; ++px) {
+            if (role == 0) tma_load_4d(sa + px * 128 * p.KBn, &map_a, bar, nc * p.KBn, co0, wo0 + px, ho);
+            else tma_load_4d(sb + px * 128 * p.KBn, &map_b, bar, nc * p.KBn, ci0, (wo0 + px) * p.sw + kw - p.pw, xh);
+          }
+        } else {
+          // stored [ho][wo][n][c] codes: box (128 channel bytes, n rows, pixels, 1); role 2 brings the second
+          // 128-channel panel of a 256-channel tile (the peer block brings it in a pair; the prefetch of the first
+          // panel covers it: the tensor maps promote L2 fills to 256 bytes)
+          if (role == 0) tma_load_4d(sa, &map_a, bar, co0, nc * p.BPP * 32, wo0, ho);
+          else if (role <= 2) tma_load_4d(sb + (role == 2 ? 128 * 128 : 0), &map_b, bar, ci_ld + (role == 2 ? 128 : 0), nc * p.BPP * 32, xw, xh);
+          else if (role == 4) tma_prefetch_4d(&map_a, co0, nc * p.BPP * 32, wo0, ho);
+          else tma_prefetch_4d(&map_b, ci_ld, nc * p.BPP * 32, xw, xh);
+        }
+      }
+      __syncwarp();
+      // next stage's (sample chunk, pixel group, row): counters, not divisions - this arithmetic sits in the
+      // pipeline's loop
+      if (++nc == p.nchunks) { nc = 0; if (++wg == p.groups_w) { wg = 0; ++ho; } }
+    }
+    if (role == 0 && lane == 0) WPROF(2);
+  }
+  __syncwarp();
+  if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer (the leader's, in a pair)
-    if (lane == 0 && rank == 0) {
+    if (rank == 0) {
       // 8-bit: MN-major tiles [K row][128 bytes], 128-byte swizzle, 8-row groups 1024 bytes apart; an MMA
       // takes 32 K rows (4096 bytes).  E2M1: K-major pieces [rows][KBn bytes], swizzle span = KBn (none for
       // 16: 8x16-byte core matrices, the next 16 bytes of K one piece further); an MMA takes 32 bytes of K.
@@ -256,41 +297,79 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         } else { ka16[a] = 256u * a; kb16[a] = 256u * a; }
       }
       const uint32_t sf_base = tmem + acc_cols;
+      // Everything that does not depend on the stage is hoisted: this thread must hand the tensor core one MMA per
+      // 128 cycles, and its own instructions are one dependent chain.
+      uint32_t idesc_a[2][4], sfa_off[4], sfb_off[2][4];
+#pragma unroll
+      for (int a = 0; a < 4; ++a) {
+        const uint32_t g = (uint32_t)(a * SPA) >> 2, id = (uint32_t)(a * SPA) & 3;
+        sfa_off[a] = 4 * g;
+#pragma unroll
+        for (int m = 0; m < 2; ++m) {
+          idesc_a[m][a] = idesc_with_sf_ids(idesc_n[m], id, id);
+          sfb_off[m][a] = 8 + 4 * (g * (uint32_t)p.NB + (m ? (uint32_t)(p.n0 >> 7) : 0u));
+        }
+      }
+      const uint32_t d1 = tmem + (uint32_t)p.n0;
       uint32_t s = 0, phase = 0, accumulate = 0;
+#ifdef MQ_TC_PROFILE
+      long long cw = 0, ci = 0, cc = 0;
+#endif
 #pragma unroll 1
-      for (int i = 0; i < nst && !*abort_flag; ++i) {
+      for (int i = 0; i < nst; ++i) {   // another role's abort shows here as this thread's own bounded wait running out
+#ifdef MQ_TC_PROFILE
+        const long long q0 = clock64();
+#endif
         if (!mbar_wait(&sffull[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+#ifdef MQ_TC_PROFILE
+        const long long q1 = clock64();
+#endif
         tc_fence_after_sync();
         const uint32_t so = s * stage16;
-        const uint32_t sfa_t = sf_base + s * sf_cols, sfb_t = sfa_t + 8;
+        const uint32_t sf_t = sf_base + s * sf_cols;
+        const uint64_t ad = a_desc0 + so, bd = b_desc0 + so;
+        if (elect_one()) {
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
-          const int g = (a * SPA) >> 2, id = (a * SPA) & 3;
-          const uint32_t accu = accumulate | (a > 0 ? 1u : 0u);
-#pragma unroll 1
-          for (int m = 0; m < nm; ++m) {
-            const uint32_t d_t = tmem + (m ? (uint32_t)p.n0 : 0u), bo = so + (m ? row16_1 : 0u);
-            const uint32_t idesc = idesc_with_sf_ids(idesc_n[m], id, id);
-            const uint32_t sfb_m = sfb_t + 4 * (g * p.NB + (m ? (p.n0 >> 7) : 0));
-            if (FP4) mma_mxf4(d_t, a_desc0 + so + ka16[a], b_desc0 + bo + kb16[a], idesc, sfa_t + 4 * g, sfb_m, accu);
-            else if (CTA2) mma_mxf8f6f4_2(d_t, a_desc0 + so + ka16[a], b_desc0 + bo + kb16[a], idesc, sfa_t + 4 * g, sfb_m, accu);
-            else mma_mxf8f6f4(d_t, a_desc0 + so + ka16[a], b_desc0 + bo + kb16[a], idesc, sfa_t + 4 * g, sfb_m, accu);
+          const uint32_t accu = a > 0 ? 1u : accumulate;
+          if (FP4) mma_mxf4(tmem, ad + ka16[a], bd + kb16[a], idesc_a[0][a], sf_t + sfa_off[a], sf_t + sfb_off[0][a], accu);
+          else if (CTA2) mma_mxf8f6f4_2(tmem, ad + ka16[a], bd + kb16[a], idesc_a[0][a], sf_t + sfa_off[a], sf_t + sfb_off[0][a], accu);
+          else mma_mxf8f6f4(tmem, ad + ka16[a], bd + kb16[a], idesc_a[0][a], sf_t + sfa_off[a], sf_t + sfb_off[0][a], accu);
+          if (nm == 2) {   // the remaining n1 rows of a tap group's operand (flat mode only)
+            if (FP4) mma_mxf4(d1, ad + ka16[a], bd + row16_1 + kb16[a], idesc_a[1][a], sf_t + sfa_off[a], sf_t + sfb_off[1][a], accu);
+            else mma_mxf8f6f4(d1, ad + ka16[a], bd + row16_1 + kb16[a], idesc_a[1][a], sf_t + sfa_off[a], sf_t + sfb_off[1][a], accu);
           }
         }
-        accumulate = 1;
+        WTRACE(3, i);
         if (CTA2) tc_commit_2_multicast(&empty[s], 3); else tc_commit(&empty[s]);   // frees the stage in both blocks
+        }
+        __syncwarp();
+        accumulate = 1;
+#ifdef MQ_TC_PROFILE
+        const long long q2 = clock64();
+#endif
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
+#ifdef MQ_TC_PROFILE
+        const long long q3 = clock64();
+        cw += q1 - q0; ci += q2 - q1; cc += q3 - q2;
+#endif
       }
-      if (CTA2) {
-        if (nst > 0) tc_commit_2_multicast(tfull, 3); else { mbar_arrive(tfull); mbar_arrive_remote(tfull, 1); }
-      } else {
-        if (nst > 0) tc_commit(tfull); else mbar_arrive(tfull);
+#ifdef MQ_TC_PROFILE
+      if (blockIdx.x < 2 && lane == 0) { g_wtrace[blockIdx.x][0][253] = (unsigned long long)cw; g_wtrace[blockIdx.x][0][254] = (unsigned long long)ci; g_wtrace[blockIdx.x][0][255] = (unsigned long long)cc; }
+#endif
+      if (elect_one()) {
+        if (CTA2) {
+          if (nst > 0) tc_commit_2_multicast(tfull, 3); else { mbar_arrive(tfull); mbar_arrive_remote(tfull, 1); }
+        } else {
+          if (nst > 0) tc_commit(tfull); else mbar_arrive(tfull);
+        }
+        WPROF(3);
       }
-      WPROF(3);
+      __syncwarp();
     }
   } else if (warp == 2) {
     // ------------------------------------------------------------------ scale copier (smem -> per-stage TMEM buffers)
-    if (lane == 0) {
+    {
       const uint64_t sf_desc = smem_desc_base(0, 128, 0);
       const uint64_t sf_desc0 = smem_desc(sf_desc, smem_u32(smem + sf_off));
       const uint32_t stage16 = (uint32_t)stage_bytes >> 4;
@@ -299,9 +378,11 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 #pragma unroll 1
       for (int i = 0; i < nst && !*abort_flag; ++i) {
         if (!mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+        if (lane == 0) WTRACE(1, i);
         if (CTA2) {
           if (rank != 0) {   // relay to the leader; its copier issues the copies for both blocks
-            mbar_arrive_remote(&pfull[s], 0);
+            if (elect_one()) mbar_arrive_remote(&pfull[s], 0);
+            __syncwarp();
             if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
             continue;
           }
@@ -310,20 +391,24 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         tc_fence_after_sync();
         const uint32_t so = s * stage16;
         const uint32_t sf_t = sf_base + s * sf_cols;
-#pragma unroll
-        for (int g = 0; g < SPA; ++g) {
-          if (CTA2) tmem_cp_32x128b_warpx4_2(sf_t + 4 * g, sf_desc0 + so + g * 32);
-          else tmem_cp_32x128b_warpx4(sf_t + 4 * g, sf_desc0 + so + g * 32);
-        }
-#pragma unroll 1
-        for (int c = 0; c < p.NB; ++c) {     // B-side chunk c: rows [128c, 128c + 128) of the group's operand
+        if (elect_one()) {
 #pragma unroll
           for (int g = 0; g < SPA; ++g) {
-            if (CTA2) tmem_cp_32x128b_warpx4_2(sf_t + 8 + 4 * (g * p.NB + c), sf_desc0 + so + 64 + (c * SPA + g) * 32);
-            else tmem_cp_32x128b_warpx4(sf_t + 8 + 4 * (g * p.NB + c), sf_desc0 + so + 64 + (c * SPA + g) * 32);
+            if (CTA2) tmem_cp_32x128b_warpx4_2(sf_t + 4 * g, sf_desc0 + so + g * 32);
+            else tmem_cp_32x128b_warpx4(sf_t + 4 * g, sf_desc0 + so + g * 32);
           }
+#pragma unroll 1
+          for (int c = 0; c < p.NB; ++c) {     // B-side chunk c: rows [128c, 128c + 128) of the group's operand
+#pragma unroll
+            for (int g = 0; g < SPA; ++g) {
+              if (CTA2) tmem_cp_32x128b_warpx4_2(sf_t + 8 + 4 * (g * p.NB + c), sf_desc0 + so + 64 + (c * SPA + g) * 32);
+              else tmem_cp_32x128b_warpx4(sf_t + 8 + 4 * (g * p.NB + c), sf_desc0 + so + 64 + (c * SPA + g) * 32);
+            }
+          }
+          WTRACE(2, i);
+          if (CTA2) tc_commit_2(&sffull[s]); else tc_commit(&sffull[s]);
         }
-        if (CTA2) tc_commit_2(&sffull[s]); else tc_commit(&sffull[s]);
+        __syncwarp();
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
     }
@@ -488,6 +573,7 @@ __global__ void __launch_bounds__(256) wgrad_flat_prep_kernel(const FlatArgs x, 
 }  // namespace
 
 #ifdef MQ_TC_PROFILE
+extern "C" int mqdbg_read_wtrace(unsigned long long* out2048) { return cudaMemcpyFromSymbol(out2048, g_wtrace, sizeof(unsigned long long) * 2048) == cudaSuccess ? 0 : 1; }
 extern "C" int mqdbg_read_wblk(unsigned long long* out960) { return cudaMemcpyFromSymbol(out960, g_wblk, sizeof(unsigned long long) * 960) == cudaSuccess ? 0 : 1; }
 #endif
 size_t wgrad_tc_smem_bytes(const WgradTcParams& p) { return 1024 + (size_t)p.stages * p.stage_bytes + (4 * (size_t)p.stages + 2) * 8 + 64; }
