@@ -18,6 +18,7 @@
 // A pipeline stage holds 128 bytes of K per row (four MMAs): one 128-byte box, or 128/KB boxes of KB
 // bytes when a tap has fewer than 128 bytes of channels (then several taps share a stage).
 // Every wait is bounded; on expiry the kernel records MQ_ERR_TIMEOUT in the status word and drains.
+#include <cstdlib>
 #include "mq_conv_tc.cuh"
 #include "mq_tcgen05.cuh"
 
@@ -380,12 +381,16 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  // The warp index goes through a shuffle so that the compiler knows it to be warp-uniform: the role loops below are
+  // run by whole warps, their arithmetic stays in the uniform datapath, and only the copy / MMA / commit instructions
+  // are issued by one elected lane (around `if (lane == 0)` every operand of those instructions would first be moved
+  // out of a per-thread register, which more than doubles the issuing thread's cycles per instruction).
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
   const int atoms_b = (p.BN + 127) / 128;
   const unsigned total = (unsigned)p.total_tiles;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 1); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); }
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 2); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 8); }
     *abort_flag = 0;
     mbar_fence_init();
@@ -400,11 +405,17 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const uint32_t tmem = *tmem_slot;
   pdl_wait();   // set-up above touched only shared memory, tensor memory and the kernel parameters
 
-  if (warp == 0) {
-    // ------------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+  if (warp == 0 || warp == 3) {
+    // ------------------------------------------------------------------ TMA producers
+    // Two warps, one copy stream each (a thread gets a bulk copy accepted only every few hundred cycles): warp 0
+    // brings the activation boxes and their scale chunk, warp 3 the weight boxes and theirs.  Both arrive on the
+    // stage's barrier with their own byte counts.
+    {
+      const bool side_b = warp == 3;
       PROF_BEGIN();
       uint32_t s = 0, phase = 0;
+      const uint32_t row_bytes = side_b ? (uint32_t)p.BN * KB : 128u * KB;
+      const uint32_t sf_bytes = side_b ? 512u * SPA * atoms_b : 512u * SPA;
       for (unsigned i = 0, t; (t = tile_of_iter(p, i)) < total && !*abort_flag; ++i) {
         const Tile tile = decode_tile(p, t);
         TapWalk<MODE> tw;
@@ -412,34 +423,38 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int Q = tw.chunks(p);
         ChunkPos pos;
         pos.reset();
-        const uint8_t* sfa_src = p.sfa_img + (size_t)tile_m_index(p, tile) * p.max_stages * (512 * SPA);
-        const uint8_t* sfb_src = p.sfb_img + ((size_t)tile.cls * p.tiles_c + tile.ct) * p.max_stages * (512 * SPA * atoms_b);
+        const uint8_t* sf_src = side_b ? p.sfb_img + ((size_t)tile.cls * p.tiles_c + tile.ct) * p.max_stages * (512 * SPA * atoms_b)
+                                       : p.sfa_img + (size_t)tile_m_index(p, tile) * p.max_stages * (512 * SPA);
         for (int q0 = 0; q0 < Q; q0 += G) {
           if (!PROF_WAIT(mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
           const int nch = min(G, Q - q0);
           uint8_t* sa = smem + (size_t)s * stage_bytes;
           uint8_t* sb = sa + A_STAGE_BYTES;
-          mbar_arrive_expect_tx(&full[s], (uint32_t)nch * (128 + p.BN) * KB + 512 * SPA * (1 + atoms_b));
-          bulk_load(sb + b_stage_bytes, sfa_src, 512 * SPA, &full[s]);
-          bulk_load(sb + b_stage_bytes + SFA_BYTES, sfb_src, 512 * SPA * atoms_b, &full[s]);
-          sfa_src += 512 * SPA;
-          sfb_src += 512 * SPA * atoms_b;
+          const bool leader = elect_one();
+          if (leader) {
+            mbar_arrive_expect_tx(&full[s], (uint32_t)nch * row_bytes + sf_bytes);
+            bulk_load(sb + b_stage_bytes + (side_b ? SFA_BYTES : 0), sf_src, sf_bytes, &full[s]);
+          }
+          sf_src += sf_bytes;
 #pragma unroll
           for (int c = 0; c < G; ++c) {
             if (c < nch) {
-              tma_load_4d(sa + c * 128 * KB, &map_a, &full[s], pos.cc * KB, src_w0(tw, pos), tile.n0, src_h(tw, pos));
-              tma_load_3d(sb + c * p.BN * KB, &map_b, &full[s], pos.cc * KB, tap_index(tw, pos), tile.c0);
+              if (leader) {
+                if (side_b) tma_load_3d(sb + c * p.BN * KB, &map_b, &full[s], pos.cc * KB, tap_index(tw, pos), tile.c0);
+                else tma_load_4d(sa + c * 128 * KB, &map_a, &full[s], pos.cc * KB, src_w0(tw, pos), tile.n0, src_h(tw, pos));
+              }
               pos.advance(tw, p.cpt);
             }
           }
+          __syncwarp();
           if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
         }
       }
-      PROF_END(0);
+      if (!side_b) PROF_END(0);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
+    {
       const uint64_t op_desc = smem_desc_base(16, 8 * KB, LAYOUT);
       const uint32_t sf_base = tmem + p.n_acc * p.BN;
       const uint32_t stage16 = (uint32_t)stage_bytes >> 4;
@@ -468,22 +483,28 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const uint32_t so = s * stage16;
           const uint32_t sfa_t = sf_base + s * SF_COLS, sfb_t = sfa_t + 8;
           const int natoms = min(G, Q - q0) * APC;
+          if (elect_one()) {
+            uint32_t accu = accumulate;
 #pragma unroll
-          for (int a = 0; a < 4; ++a) {
-            if (a < natoms) {
-              const int c = a / APC, ja = a % APC;
-              const uint64_t ad = a_desc0 + so + c * ((128 * KB) >> 4) + ja * 2;
-              const uint64_t bd = b_desc0 + so + c * b_chunk16 + ja * 2;
-              const int g = (a * SPA) >> 2, id = (a * SPA) & 3;
-              if (FP4) mma_mxf4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accumulate);
-              else mma_mxf8f6f4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accumulate);
-              accumulate = 1;
+            for (int a = 0; a < 4; ++a) {
+              if (a < natoms) {
+                const int c = a / APC, ja = a % APC;
+                const uint64_t ad = a_desc0 + so + c * ((128 * KB) >> 4) + ja * 2;
+                const uint64_t bd = b_desc0 + so + c * b_chunk16 + ja * 2;
+                const int g = (a * SPA) >> 2, id = (a * SPA) & 3;
+                if (FP4) mma_mxf4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accu);
+                else mma_mxf8f6f4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accu);
+                accu = 1;
+              }
             }
+            tc_commit(&empty[s]);
           }
-          tc_commit(&empty[s]);
+          __syncwarp();
+          accumulate = 1;
           if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
         }
-        if (Q > 0) tc_commit(&tfull[acc]); else mbar_arrive(&tfull[acc]);
+        if (elect_one()) { if (Q > 0) tc_commit(&tfull[acc]); else mbar_arrive(&tfull[acc]); }
+        __syncwarp();
       }
       PROF_END(1);
     }
@@ -491,8 +512,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // ------------------------------------------------------------------ scale copier
     // Copies the stage's scale chunks smem -> TMEM (one TMEM scale buffer per pipeline stage) from its own
     // thread, so these copies overlap the MMA issuer's work on earlier stages.  The buffer of stage s is free
-    // whenever full[s] completes: the producer refilled the stage only after the MMAs that read it committed.
-    if (lane == 0) {
+    // whenever full[s] completes: the producers refilled the stage only after the MMAs that read it committed.
+    {
       const uint64_t sf_desc = smem_desc_base(0, 128, 0);
       const uint32_t sf_base = tmem + p.n_acc * p.BN;
       const uint32_t stage16 = (uint32_t)stage_bytes >> 4;
@@ -510,12 +531,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           tc_fence_after_sync();
           const uint32_t so = s * stage16;
           const uint32_t sfa_t = sf_base + s * SF_COLS, sfb_t = sfa_t + 8;
+          if (elect_one()) {
 #pragma unroll
-          for (int g = 0; g < SPA; ++g) {
-            tmem_cp_32x128b_warpx4(sfa_t + 4 * g, sfa_desc0 + so + g * 32);
-            for (int a = 0; a < atoms_b; ++a) tmem_cp_32x128b_warpx4(sfb_t + 4 * (g * atoms_b + a), sfb_desc0 + so + (g * atoms_b + a) * 32);
+            for (int g = 0; g < SPA; ++g) {
+              tmem_cp_32x128b_warpx4(sfa_t + 4 * g, sfa_desc0 + so + g * 32);
+              for (int a = 0; a < atoms_b; ++a) tmem_cp_32x128b_warpx4(sfb_t + 4 * (g * atoms_b + a), sfb_desc0 + so + (g * atoms_b + a) * 32);
+            }
+            tc_commit(&sffull[s]);
           }
-          tc_commit(&sffull[s]);
+          __syncwarp();
           if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
         }
       }
@@ -624,7 +648,7 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   uint32_t* tap_b = tap_a + 64;
   uint32_t* tap_p = tap_b + 64;                        // per tap: first pixel of its view in the tile's scale patch
   uint8_t* sc_tbl = reinterpret_cast<uint8_t*>(tap_p + 64);   // the tile's patch of raw scale bytes (<= 512)
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;   // warp-uniform, see conv_tc_kernel
   const unsigned total = (unsigned)p.total_tiles;
   const unsigned tiles_per_c = (unsigned)(p.classes * p.tiles_w * p.tiles_h);   // tile order: (class, w, h) below the channel tile
 
@@ -670,7 +694,7 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 
   if (warp == 0) {
     // ------------------------------------------------------------------ producer
-    if (lane == 0) {
+    {
       uint32_t s = 0, phase = 0, bcount = 0;
       int cur_ct = -1;
       PROF_BEGIN();
@@ -680,9 +704,12 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         if (!p.fused && ct != cur_ct) {
           // new weight tile: wait until the MMAs of the previous one have retired, then one copy of image + scales
           if (bcount > 0 && !PROF_WAIT(mbar_wait(bempty, (bcount - 1) & 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
-          mbar_arrive_expect_tx(bfull, (uint32_t)(b_bytes + sfb_bytes));
-          bulk_load(smem, p.b_img + (size_t)ct * b_bytes, b_bytes, bfull);
-          bulk_load(smem + b_bytes, p.sfb_img + ((size_t)tile.cls * p.tiles_c + ct) * sfb_bytes, sfb_bytes, bfull);
+          if (elect_one()) {
+            mbar_arrive_expect_tx(bfull, (uint32_t)(b_bytes + sfb_bytes));
+            bulk_load(smem, p.b_img + (size_t)ct * b_bytes, b_bytes, bfull);
+            bulk_load(smem + b_bytes, p.sfb_img + ((size_t)tile.cls * p.tiles_c + ct) * sfb_bytes, sfb_bytes, bfull);
+          }
+          __syncwarp();
           cur_ct = ct; ++bcount;
         }
         if (!PROF_WAIT(mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
@@ -690,16 +717,19 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         // first source pixel of the halo: forward (h - ph, w0 - pw); input gradient (h + ph - (Kh-1), w0 + pw - (Kw-1))
         const int hs = MODE == MQ_OP_FWD ? tile.h - p.ph : tile.h + p.ph - (p.Kh - 1);
         const int ws = MODE == MQ_OP_FWD ? tile.w0 - p.pw : tile.w0 + p.pw - (p.Kw - 1);
-        mbar_arrive_expect_tx(&full[s], (uint32_t)(p.halo_box_bytes + (p.fused ? 0 : sfa_bytes)));
-        tma_load_4d(sa, &map_a, &full[s], 0, ws, tile.n0, hs);
-        if (!p.fused) bulk_load(sa + p.halo_a_bytes, p.sfa_img + (size_t)tile_m_index(p, tile) * sfa_bytes, sfa_bytes, &full[s]);
+        if (elect_one()) {
+          mbar_arrive_expect_tx(&full[s], (uint32_t)(p.halo_box_bytes + (p.fused ? 0 : sfa_bytes)));
+          tma_load_4d(sa, &map_a, &full[s], 0, ws, tile.n0, hs);
+          if (!p.fused) bulk_load(sa + p.halo_a_bytes, p.sfa_img + (size_t)tile_m_index(p, tile) * sfa_bytes, sfa_bytes, &full[s]);
+        }
+        __syncwarp();
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
       PROF_END(0);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer: all taps of a tile per stage
-    if (lane == 0) {
+    {
       const uint64_t a_desc_base = smem_desc_base(16, (uint32_t)(p.WH * KB), LAYOUT);   // 8-row groups one halo row apart
       const uint64_t b_desc_base = smem_desc_base(16, 8 * KB, LAYOUT);
       const uint32_t sb16 = smem_u32(smem) >> 4;
@@ -727,8 +757,9 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         const uint32_t d_tmem = tmem + acc * p.BN;
         const uint32_t sa16 = smem_u32(stage0 + (size_t)s * stage_bytes) >> 4;
         const uint32_t sfa_s = sfa_base + s * sfa_cols_stage;
-        uint32_t accumulate = 0;
         const long long pc0 = PROF_CLK();
+        if (elect_one()) {
+        uint32_t accumulate = 0;
         auto issue_tap = [&](int q, uint32_t a16, uint32_t b16) {
           const int sfst = q / G;
           const uint32_t sfa_t = sfa_s + sfst * 8, sfb_t = sfb_base + sfst * 16;
@@ -750,21 +781,23 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 #pragma unroll 1
           for (int q = 0; q < taps; ++q) issue_tap(q, sa16 + tap_a[q], sb16 + tap_b[q]);
         }
-        const long long pc1 = PROF_CLK();
         tc_commit(&empty[s]);
         tc_commit(&tfull[acc]);
-        PROF_ADD(4, 1, pc1 - pc0);
         if (p.tiles_c > 1) {
           const unsigned tn_ = t + gridDim.x;   // the block's next tile: release the weight tile if it needs another
           if (tn_ < total && (int)((tn_ / tiles_per_c) % (unsigned)p.tiles_c) != ct) tc_commit(bempty);
         }
+        }
+        __syncwarp();
+        const long long pc1 = PROF_CLK();
+        PROF_ADD(4, 1, pc1 - pc0);
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
       PROF_END(1);
     }
   } else if (warp == 2) {
     // ------------------------------------------------------------------ scale copier: chunks smem -> TMEM
-    if (lane == 0) {
+    {
       const uint64_t sf_desc = smem_desc_base(0, 128, 0);
       uint32_t s = 0, phase = 0, bcount = 0;
       int cur_ct = -1;
@@ -778,6 +811,7 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         }
         if (!PROF_WAIT(mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
         tc_fence_after_sync();
+        if (elect_one()) {
         if (new_b) {
           const uint32_t sfb_s = smem_u32(smem + b_bytes);
 #pragma unroll 1
@@ -796,6 +830,8 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           for (int g = 0; g < SPA; ++g) tmem_cp_32x128b_warpx4(sfa_s + st * 8 + 4 * g, smem_desc(sf_desc, sfa_sm + (st * SPA + g) * 512));
         }
         tc_commit(&sffull[s]);
+        }
+        __syncwarp();
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
       PROF_END(2);
@@ -1070,6 +1106,11 @@ extern "C" int mqdbg_read_prof(unsigned long long* out16) {
 }
 #endif
 
+static CUtensorMapL2promotion l2promo() {
+  const char* e = getenv("MQ_TMA_L2PROMO");
+  const int v = e ? atoi(e) : 3;
+  return v == 0 ? CU_TENSOR_MAP_L2_PROMOTION_NONE : v == 1 ? CU_TENSOR_MAP_L2_PROMOTION_L2_64B : v == 2 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
+}
 bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes, const uint32_t* box,
                           const uint32_t* elem_strides, int swizzle_bytes, bool f32) {
   EncodeTiledFn fn = get_encoder();
@@ -1082,7 +1123,7 @@ bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const ui
                         : swizzle_bytes == 64  ? CU_TENSOR_MAP_SWIZZLE_64B
                         : swizzle_bytes == 32  ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE;
   CUresult r = fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
-                  CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                  l2promo(), CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 
