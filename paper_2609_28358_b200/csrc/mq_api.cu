@@ -346,9 +346,9 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   if (fp8 && g.Cp >= 256 && !env_int("MQ_WGRAD_N128", 0)) p.b_rows = 256;
   p.m_tiles = (g.Cout + 127) / 128;
   p.m_tiles128 = p.m_tiles;
-  // Pairs of blocks on 256 x 256 tiles (cta_group::2): correct, but measured 1.35x slower than single blocks on
-  // 128 x 256 tiles, whose neighbours already share their X loads on the way from L2; opt-in only.
-  p.cta2 = fp8 && p.b_rows == 256 && g.Cout >= 256 && env_int("MQ_WGRAD_CTA2", 0);
+  // Pairs of blocks on 256 x 256 tiles (cta_group::2) when both channel counts allow it: half the X bytes per block
+  // and stage, so six pipeline stages instead of four, and one MMA instruction per 256 x 256 x 32 for the issuing lane.
+  p.cta2 = fp8 && p.b_rows == 256 && g.Cout >= 256 && !env_int("MQ_WGRAD_NO_CTA2", 0);
   if (p.cta2) { p.m_tiles = (g.Cout + 255) / 256; p.m_tiles128 = 2 * p.m_tiles; }
   p.cb_tiles = (g.Cp + p.b_rows - 1) / p.b_rows;
   // taps per block: a whole kernel row in the flat mode when its accumulators fit in tensor memory
@@ -455,7 +455,17 @@ mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const 
     const uint32_t box[3] = {32u, 32u, 1u};
     if (!encode_tensor_map_u8(&map_p, partial, 3, dims, strides, box, nullptr, 128, true)) return MQ_ERR_CUDA;
   }
-  if (launch_wgrad_tc(p, map_a, map_b, map_p, stream) != cudaSuccess) return MQ_ERR_CUDA;
+  CUtensorMap map_sfa{}, map_sfb{};
+  if (p.cta2) {   // a pair's scale chunks travel as tiled copies too (rows of 256 bytes), so that they can count on the leader's barrier
+    const int spa = 1;   // 8-bit operands only
+    const uint64_t rows_a = (uint64_t)p.m_tiles128 * p.stages_total * 2 * spa;
+    const uint64_t rows_b = (uint64_t)p.cb_tiles * (g.Kh * g.Kw / p.TG) * p.stages_total * p.NB * 2 * spa;
+    const uint64_t da[2] = {256, rows_a}, db[2] = {256, rows_b}, st[1] = {256};
+    const uint32_t ba[2] = {256u, (uint32_t)(2 * spa)}, bb[2] = {256u, (uint32_t)(2 * spa * p.NB)};
+    if (!encode_tensor_map_u8(&map_sfa, p.sfa_img, 2, da, st, ba, nullptr, 0)) return MQ_ERR_CUDA;
+    if (!encode_tensor_map_u8(&map_sfb, p.sfb_img, 2, db, st, bb, nullptr, 0)) return MQ_ERR_CUDA;
+  }
+  if (launch_wgrad_tc(p, map_a, map_b, map_p, map_sfa, map_sfb, stream) != cudaSuccess) return MQ_ERR_CUDA;
   return launch_bwd_weight_reduce(partial, out, g, p.splits, layout, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }
 

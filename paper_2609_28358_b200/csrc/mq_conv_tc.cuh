@@ -114,7 +114,8 @@ struct WgradTcParams {
   unsigned int* status;
 };
 // map_p: the partial sums as an fp32 tensor (taps * Cp columns, C_out rows, splits), box 32 x 32 x 1, 128-byte swizzle
-cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_p, cudaStream_t s);
+cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_p, const CUtensorMap& map_sfa,
+                            const CUtensorMap& map_sfb, cudaStream_t s);
 cudaError_t launch_expand_wgrad_scales(const WgradTcParams& p, cudaStream_t s);
 // E2M1 codes [P][N][Cp] -> [P][Cp][Npad] (n fastest, zero-padded): a permutation of nibbles, no requantization.
 cudaError_t launch_fp4_to_n_major(const uint8_t* in, uint8_t* out, int P, int N, int Cp, int Npad, cudaStream_t s);

@@ -35,8 +35,7 @@ __device__ unsigned long long g_wtrace[2][4][256];   // blocks 0 and 1: per stag
 #define WTRACE(k, i) do { } while (0)
 #endif
 
-constexpr int WG_THREADS = 256;
-constexpr int WG_PREFETCH = 8;   // stages between an L2 prefetch and the load it serves
+constexpr int WG_THREADS = 320;   // MMA warp, scale copier / loader, eight more loader warps (four of them the epilogue)
 
 // K-block b of stage st: output pixel and 32-sample block
 __device__ __forceinline__ void stage_block(const WgradTcParams& p, int st, int b, int& ho, int& wo, int& nb) {
@@ -126,7 +125,7 @@ __global__ void __launch_bounds__(256) expand_wgrad_scales_kernel(const WgradTcP
 template <bool FP4, bool CTA2>
 __global__ void __launch_bounds__(WG_THREADS, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_p,
-                const WgradTcParams p) {
+                const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb, const WgradTcParams p) {
   constexpr int SPA = FP4 ? 2 : 1;     // scale bytes per MMA per row
   if (threadIdx.x == 0) WPROF(0);
   extern __shared__ uint8_t smem_raw[];
@@ -138,10 +137,9 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   uint64_t* empty = full + p.stages;
   uint64_t* sffull = empty + p.stages;
   uint64_t* tfull = sffull + p.stages;
-  uint64_t* pfull = tfull + 1;                         // CTA2, leader: the peer block's stage has landed
+  uint64_t* pfull = tfull + 1;                         // (spare)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(pfull + p.stages);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-  volatile int* progress = abort_flag + 1;             // stages the G_Y loader has issued (paces the prefetchers)
   // Warp index and cluster rank go through a shuffle so that the compiler knows them to be warp-uniform: the role
   // loops below are run by whole warps, their arithmetic stays in the uniform datapath, and only the bulk-copy / MMA /
   // commit instructions themselves are issued by one elected lane.  (With `if (lane == 0)` around a role, every
@@ -170,10 +168,10 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 
   if (threadIdx.x == 0) {
 #pragma unroll 1
+    // full: one arrival per kind of copy
     for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], has_b1 ? 4 : 3); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); mbar_init(&pfull[s], 1); }
     mbar_init(tfull, 1);
     *abort_flag = 0;
-    *progress = 0;
     mbar_fence_init();
     if (p.mode != MQ_WG_FP4_FLAT) { prefetch_tensormap(&map_a); prefetch_tensormap(&map_b); }
     prefetch_tensormap(&map_p);
@@ -191,14 +189,19 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   if (threadIdx.x == 0) WPROF(1);
 
   // ------------------------------------------------------------------ loaders
-  // A thread gets one bulk copy accepted per ~265 cycles whatever its size, so a stage's copies are issued by
-  // different warps (one lane each).  Every loader arrives on the stage's barrier with its own byte count.  Four of
-  // these threads belong to the epilogue warps, which have nothing else to do until the accumulators are final.
-  // roles: 0 G_Y tile, 1 X tile (first panel), 2 second X panel, 3 both scale-chunk copies; 4 and 5 prefetch the G_Y and
-  // X boxes of the stage WG_PREFETCH stages ahead into L2 (about a quarter of the lines miss L2, and a box lands only
-  // when its slowest line has: the prefetch takes the DRAM latency out of the pipeline's loop).
-  const int role = warp == 0 ? 0 : (warp == 3 ? 1 : (warp >= 4 ? warp - 2 : -1));
-  if (role >= 0 && (role != 2 || has_b1) && (role < 4 || p.mode != MQ_WG_FP4_PIXEL)) {
+  // A warp gets one bulk copy accepted per ~170 cycles whatever its size, and its loop around that copy (barrier
+  // wait, addresses, coordinates) is a chain of dependent instructions, so the copies of a stage are spread over
+  // warps: one KIND of copy per pair of warps (G_Y tile; X tile, one or two 128-channel panels; the two scale
+  // chunks), the two warps of a kind taking even and odd stages.  Each kind arrives once per stage on the stage's
+  // barrier with its own byte count.  The loaders include the epilogue warps, idle until the accumulators are final.
+  // In a pair of blocks every copy of either block is counted on the LEADER's barrier: its loaders announce both
+  // blocks' bytes, the peer's loaders only issue (no relay thread, no remote arrive in the loop).
+  const int nkinds = has_b1 ? 4 : 3;
+  const int lslot = FP4 ? (warp == 0 ? 0 : (warp >= 3 ? warp - 2 : -1))          // E2M1: warp 2 is the scale copier
+                        : (warp == 0 ? 0 : (warp == 2 ? 1 : (warp >= 3 ? warp - 1 : -1)));
+  if (lslot >= 0 && lslot < 2 * nkinds) {
+    const int kidx = lslot >> 1, half = lslot & 1;
+    const int kind = kidx == 0 ? 0 : (kidx == 1 ? 1 : ((kidx == 2 && has_b1) ? 2 : 3));   // 0 G_Y, 1 X, 2 second X panel, 3 scales
     const int taps = p.Kh * p.Kw;
     const uint8_t* sfa_src = p.sfa_img + ((size_t)mt * p.stages_total + st_begin) * (512 * SPA);
     const uint32_t sfb_bytes = (uint32_t)p.NB * 512 * SPA;
@@ -210,65 +213,66 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       ga = p.gt + (size_t)mt * p.gt_block_bytes + (size_t)st_begin * a_bytes;
       gb = p.xt + (size_t)cb * p.xt_block_bytes + ((size_t)st_begin * p.KPX + (size_t)kh * p.Wp + kw) * ((size_t)p.b_rows * p.KBn);
     }
-    const uint32_t my_bytes = role == 0 ? a_bytes : (role <= 2 ? b_bytes : 512u * SPA + sfb_bytes);
-    const bool prefetcher = role >= 4;
+    const uint32_t my_bytes = (kind == 0 ? a_bytes : (kind <= 2 ? b_bytes : 512u * SPA + sfb_bytes)) * (CTA2 ? 2u : 1u);
+    const int sfa_row0 = (int)(((size_t)mt * p.stages_total + st_begin) * (2 * SPA));          // rows of 256 bytes (pair mode maps)
+    const int sfb_row0 = (int)((((size_t)cb * (taps / TG) + tgi) * p.stages_total + st_begin) * (2 * SPA * p.NB));
     int nc, wg, ho;                                            // of the first stage this warp handles
     {
-      const int st = st_begin + (prefetcher ? p.stages : 0);
+      const int st = st_begin + half;
       nc = st % p.nchunks; const int t = st / p.nchunks;
       wg = t % p.groups_w; ho = t / p.groups_w;
     }
-    uint32_t s = 0, phase = 0;
+    uint32_t s = (uint32_t)half % (uint32_t)p.stages, phase = 0;   // stages >= 2
 #pragma unroll 1
-    for (int i = 0; i < nst && !*abort_flag; ++i) {
-      const int ii = prefetcher ? i + p.stages : i;          // the stage this warp's copy is for
-      if (ii >= nst) break;
-      if (prefetcher) {
-        // not a party to the pipeline's barriers: stay at most WG_PREFETCH stages ahead of the loader's counter
-        uint32_t spins = 0;
-        while (ii - *progress > WG_PREFETCH && !*abort_flag && ++spins < kWaitLimit) __nanosleep(64);
-      } else if (!mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+    for (int i = half; i < nst; i += 2) {
+      // everything that does not depend on the stage being free comes before the wait
       uint8_t* sa = smem + (size_t)s * stage_bytes;
       uint8_t* sb = sa + b_off;
       uint8_t* ssf = sa + sf_off;
       uint64_t* bar = &full[s];
-      if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
+      const uint32_t lbar = CTA2 ? cluster_addr_of(bar, 0) : 0u;
       const int wo0 = wg * p.KPX;
       const int xw = wo0 * p.sw + kw - p.pw, xh = ho * p.sh + kh - p.ph;
+      const int nrow = nc * p.BPP * 32;
+      if (*abort_flag) break;
+      if (!mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
       if (elect_one()) {
-        if (role == 0) { WTRACE(0, i); *progress = i; }
-        if (!prefetcher) mbar_arrive_expect_tx(bar, my_bytes);
-        if (role == 3) {
+        if (kind == 0) WTRACE(0, i);
+        if (rank == 0) mbar_arrive_expect_tx(bar, my_bytes);
+        if (CTA2) {
+          if (kind == 0) tma_load_4d_pair(sa, &map_a, lbar, co0, nrow, wo0, ho);
+          else if (kind == 1) tma_load_4d_pair(sb, &map_b, lbar, ci_ld, nrow, xw, xh);
+          else {
+            tma_load_2d_pair(ssf, &map_sfa, lbar, 0, sfa_row0 + i * (2 * SPA));
+            tma_load_2d_pair(ssf + 1024, &map_sfb, lbar, 0, sfb_row0 + i * (2 * SPA * p.NB));
+          }
+        } else if (kind == 3) {
           bulk_load(ssf, sfa_src + (size_t)i * (512 * SPA), 512 * SPA, bar);
           bulk_load(ssf + 1024, sfb_src + (size_t)i * sfb_bytes, sfb_bytes, bar);
         } else if (p.mode == MQ_WG_FP4_FLAT) {
-          if (role == 0) bulk_load(sa, ga + (size_t)i * a_bytes, a_bytes, bar);
-          else if (role == 1) bulk_load(sb, gb + (size_t)i * b_step, b_bytes, bar);          // KPX + TG - 1 consecutive pixels
-          else if (role == 4) bulk_prefetch(ga + (size_t)ii * a_bytes, a_bytes);
-          else bulk_prefetch(gb + (size_t)ii * b_step + (b_bytes - b_step), b_step);          // the pixels stage ii adds
+          if (kind == 0) bulk_load(sa, ga + (size_t)i * a_bytes, a_bytes, bar);
+          else bulk_load(sb, gb + (size_t)i * b_step, b_bytes, bar);          // KPX + TG - 1 consecutive pixels
         } else if (p.mode == MQ_WG_FP4_PIXEL) {
           // [pixel][c][n] re-laid codes: one box (n bytes, 128 channels) per pixel of the stage
 #pragma unroll 1
           for (int px = 0; px < p.KPX; ++px) {
-            if (role == 0) tma_load_4d(sa + px * 128 * p.KBn, &map_a, bar, nc * p.KBn, co0, wo0 + px, ho);
+            if (kind == 0) tma_load_4d(sa + px * 128 * p.KBn, &map_a, bar, nc * p.KBn, co0, wo0 + px, ho);
             else tma_load_4d(sb + px * 128 * p.KBn, &map_b, bar, nc * p.KBn, ci0, (wo0 + px) * p.sw + kw - p.pw, xh);
           }
         } else {
-          // stored [ho][wo][n][c] codes: box (128 channel bytes, n rows, pixels, 1); role 2 brings the second
-          // 128-channel panel of a 256-channel tile (the peer block brings it in a pair; the prefetch of the first
-          // panel covers it: the tensor maps promote L2 fills to 256 bytes)
-          if (role == 0) tma_load_4d(sa, &map_a, bar, co0, nc * p.BPP * 32, wo0, ho);
-          else if (role <= 2) tma_load_4d(sb + (role == 2 ? 128 * 128 : 0), &map_b, bar, ci_ld + (role == 2 ? 128 : 0), nc * p.BPP * 32, xw, xh);
-          else if (role == 4) tma_prefetch_4d(&map_a, co0, nc * p.BPP * 32, wo0, ho);
-          else tma_prefetch_4d(&map_b, ci_ld, nc * p.BPP * 32, xw, xh);
+          // stored [ho][wo][n][c] codes: box (128 channel bytes, n rows, pixels, 1)
+          if (kind == 0) tma_load_4d(sa, &map_a, bar, co0, nrow, wo0, ho);
+          else tma_load_4d(sb + (kind == 2 ? 128 * 128 : 0), &map_b, bar, ci_ld + (kind == 2 ? 128 : 0), nrow, xw, xh);
         }
       }
       __syncwarp();
-      // next stage's (sample chunk, pixel group, row): counters, not divisions - this arithmetic sits in the
-      // pipeline's loop
-      if (++nc == p.nchunks) { nc = 0; if (++wg == p.groups_w) { wg = 0; ++ho; } }
+      // two stages on: slot, then (sample chunk, pixel group, row) by counters, not divisions
+      s += 2; if (s >= (uint32_t)p.stages) { s -= (uint32_t)p.stages; phase ^= 1; }
+#pragma unroll
+      for (int r = 0; r < 2; ++r)
+        if (++nc == p.nchunks) { nc = 0; if (++wg == p.groups_w) { wg = 0; ++ho; } }
     }
-    if (role == 0 && lane == 0) WPROF(2);
+    if (kind == 0 && half == 0 && lane == 0) WPROF(2);
   }
   __syncwarp();
   if (warp == 1) {
@@ -297,6 +301,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         } else { ka16[a] = 256u * a; kb16[a] = 256u * a; }
       }
       const uint32_t sf_base = tmem + acc_cols;
+      const uint64_t sf_desc0 = smem_desc(smem_desc_base(0, 128, 0), smem_u32(smem + sf_off));
       // Everything that does not depend on the stage is hoisted: this thread must hand the tensor core one MMA per
       // 128 cycles, and its own instructions are one dependent chain.
       uint32_t idesc_a[2][4], sfa_off[4], sfb_off[2][4];
@@ -314,20 +319,50 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       uint32_t s = 0, phase = 0, accumulate = 0;
 #ifdef MQ_TC_PROFILE
       long long cw = 0, ci = 0, cc = 0;
+      const long long loop_c0 = clock64(); const unsigned long long loop_g0 = gtime();
 #endif
 #pragma unroll 1
       for (int i = 0; i < nst; ++i) {   // another role's abort shows here as this thread's own bounded wait running out
 #ifdef MQ_TC_PROFILE
         const long long q0 = clock64();
 #endif
-        if (!mbar_wait(&sffull[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+        if (!mbar_wait(FP4 ? &sffull[s] : &full[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
 #ifdef MQ_TC_PROFILE
         const long long q1 = clock64();
+        if (!FP4 && lane == 0) WTRACE(1, i);
 #endif
         tc_fence_after_sync();
         const uint32_t so = s * stage16;
         const uint32_t sf_t = sf_base + s * sf_cols;
         const uint64_t ad = a_desc0 + so, bd = b_desc0 + so;
+        if (!FP4 && nm == 1) {
+          // 8-bit operands: this lane also issues the stage's three scale copies, right before the MMAs that read
+          // them (same thread, so the tensor pipe keeps them in order).  A separate copier's copies would queue behind
+          // the MMAs already issued and its completion signal would arrive only when those retire - one pipeline
+          // bubble per stage.
+          if (elect_one()) {
+            const uint64_t sfd = sf_desc0 + so;
+            if (CTA2) {
+              tmem_cp_32x128b_warpx4_2(sf_t, sfd);
+              tmem_cp_32x128b_warpx4_2(sf_t + 8, sfd + 64);
+              tmem_cp_32x128b_warpx4_2(sf_t + 12, sfd + 96);
+            } else {
+              tmem_cp_32x128b_warpx4(sf_t, sfd);
+              tmem_cp_32x128b_warpx4(sf_t + 8, sfd + 64);
+              if (p.NB > 1) tmem_cp_32x128b_warpx4(sf_t + 12, sfd + 96);
+            }
+            WTRACE(2, i);
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+              const uint32_t accu = a > 0 ? 1u : accumulate;
+              const uint32_t id = idesc_n[0] | ((uint32_t)a << 4) | ((uint32_t)a << 29);
+              if (CTA2) mma_mxf8f6f4_2(tmem, ad + 256u * a, bd + 256u * a, id, sf_t, sf_t + 8, accu);
+              else mma_mxf8f6f4(tmem, ad + 256u * a, bd + 256u * a, id, sf_t, sf_t + 8, accu);
+            }
+            if (CTA2) tc_commit_2_multicast(&empty[s], 3); else tc_commit(&empty[s]);
+            WTRACE(3, i);
+          }
+        } else
         if (elect_one()) {
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
@@ -355,6 +390,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 #endif
       }
 #ifdef MQ_TC_PROFILE
+      if (blockIdx.x < 2 && lane == 0) { g_wtrace[blockIdx.x][1][254] = (unsigned long long)(clock64() - loop_c0); g_wtrace[blockIdx.x][1][255] = gtime() - loop_g0; }
       if (blockIdx.x < 2 && lane == 0) { g_wtrace[blockIdx.x][0][253] = (unsigned long long)cw; g_wtrace[blockIdx.x][0][254] = (unsigned long long)ci; g_wtrace[blockIdx.x][0][255] = (unsigned long long)cc; }
 #endif
       if (elect_one()) {
@@ -369,7 +405,8 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     }
   } else if (warp == 2) {
     // ------------------------------------------------------------------ scale copier (smem -> per-stage TMEM buffers)
-    {
+    // E2M1 only (twice the scale bytes, up to eight copies per stage); for 8-bit operands the MMA lane issues them.
+    if (FP4) {
       const uint64_t sf_desc = smem_desc_base(0, 128, 0);
       const uint64_t sf_desc0 = smem_desc(sf_desc, smem_u32(smem + sf_off));
       const uint32_t stage16 = (uint32_t)stage_bytes >> 4;
@@ -379,19 +416,14 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       for (int i = 0; i < nst && !*abort_flag; ++i) {
         if (!mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
         if (lane == 0) WTRACE(1, i);
-        if (CTA2) {
-          if (rank != 0) {   // relay to the leader; its copier issues the copies for both blocks
-            if (elect_one()) mbar_arrive_remote(&pfull[s], 0);
-            __syncwarp();
-            if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
-            continue;
-          }
-          if (!mbar_wait(&pfull[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
-        }
         tc_fence_after_sync();
         const uint32_t so = s * stage16;
         const uint32_t sf_t = sf_base + s * sf_cols;
         if (elect_one()) {
+#ifdef MQ_WG_SKIPCP
+          if (i < p.stages)
+#endif
+          {
 #pragma unroll
           for (int g = 0; g < SPA; ++g) {
             if (CTA2) tmem_cp_32x128b_warpx4_2(sf_t + 4 * g, sf_desc0 + so + g * 32);
@@ -405,6 +437,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
               else tmem_cp_32x128b_warpx4(sf_t + 8 + 4 * (g * p.NB + c), sf_desc0 + so + 64 + (c * SPA + g) * 32);
             }
           }
+          }
           WTRACE(2, i);
           if (CTA2) tc_commit_2(&sffull[s]); else tc_commit(&sffull[s]);
         }
@@ -412,7 +445,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
     }
-  } else if (warp >= 4) {
+  } else if (warp >= 4 && warp < 8) {
     // ------------------------------------------------------------------ epilogue: partial sums to scratch
     // Each warp moves its 32 rows, 32 columns at a time: TMEM -> registers -> a [32 rows][128 bytes] staging tile
     // (128-byte swizzle, so the 16-byte writes of a row do not collide) -> one TMA store into the partial-sum
@@ -578,7 +611,8 @@ extern "C" int mqdbg_read_wblk(unsigned long long* out960) { return cudaMemcpyFr
 #endif
 size_t wgrad_tc_smem_bytes(const WgradTcParams& p) { return 1024 + (size_t)p.stages * p.stage_bytes + (4 * (size_t)p.stages + 2) * 8 + 64; }
 
-cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_p, cudaStream_t s) {
+cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_p, const CUtensorMap& map_sfa,
+                            const CUtensorMap& map_sfb, cudaStream_t s) {
   static bool attr_set[3] = {false, false, false};
   const size_t smem = wgrad_tc_smem_bytes(p);
   const int f = p.cta2 ? 2 : (p.mode == MQ_WG_FP8 ? 0 : 1);
@@ -591,9 +625,9 @@ cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, co
   }
   const unsigned grid = (unsigned)(p.m_tiles * p.j_tiles * p.splits) * (p.cta2 ? 2u : 1u);
   count_launches(1);
-  if (f == 2) return launch_pdl_cluster(wgrad_tc_kernel<false, true>, dim3(grid), dim3(WG_THREADS), smem, s, 2u, map_a, map_b, map_p, p);
-  if (f == 1) return launch_pdl(wgrad_tc_kernel<true, false>, dim3(grid), dim3(WG_THREADS), smem, s, map_a, map_b, map_p, p);
-  return launch_pdl(wgrad_tc_kernel<false, false>, dim3(grid), dim3(WG_THREADS), smem, s, map_a, map_b, map_p, p);
+  if (f == 2) return launch_pdl_cluster(wgrad_tc_kernel<false, true>, dim3(grid), dim3(WG_THREADS), smem, s, 2u, map_a, map_b, map_p, map_sfa, map_sfb, p);
+  if (f == 1) return launch_pdl(wgrad_tc_kernel<true, false>, dim3(grid), dim3(WG_THREADS), smem, s, map_a, map_b, map_p, map_sfa, map_sfb, p);
+  return launch_pdl(wgrad_tc_kernel<false, false>, dim3(grid), dim3(WG_THREADS), smem, s, map_a, map_b, map_p, map_sfa, map_sfb, p);
 }
 
 cudaError_t launch_expand_wgrad_scales(const WgradTcParams& p, cudaStream_t s) {
