@@ -26,7 +26,7 @@ namespace mq {
 namespace {
 using namespace tc;
 
-constexpr int TC_THREADS = 384;   // 12 warps: TMA, MMA, 2 scale expanders, 8 epilogue
+constexpr int TC_THREADS = 512;   // 16 warps: MMA, scale copier, scale expander / loader, 8 epilogue, 5 more loaders
 constexpr int A_STAGE_BYTES = 128 * 128;
 constexpr int SFA_BYTES = 1024;   // up to 2 groups of 4 scale bytes per row
 constexpr int SFB_BYTES = 2048;   // up to 2 groups x 2 atoms of 128 rows
@@ -390,7 +390,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const unsigned total = (unsigned)p.total_tiles;
 
   if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 2); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); }
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 3); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); }
     for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 8); }
     *abort_flag = 0;
     mbar_fence_init();
@@ -405,17 +405,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   const uint32_t tmem = *tmem_slot;
   pdl_wait();   // set-up above touched only shared memory, tensor memory and the kernel parameters
 
-  if (warp == 0 || warp == 3) {
-    // ------------------------------------------------------------------ TMA producers
-    // Two warps, one copy stream each (a thread gets a bulk copy accepted only every few hundred cycles): warp 0
-    // brings the activation boxes and their scale chunk, warp 3 the weight boxes and theirs.  Both arrive on the
-    // stage's barrier with their own byte counts.
+  // loader warps: (kind, parity of the stages it serves)
+  const int lkind = (warp == 0 || warp == 12) ? 0 : ((warp == 3 || warp == 13) ? 1 : (warp >= 14 ? 2 : -1));
+  const int lhalf = (warp == 12 || warp == 13 || warp == 15) ? 1 : 0;
+  if (lkind >= 0) {
+    // ------------------------------------------------------------------ TMA loaders
+    // A warp gets one bulk copy accepted per ~170 cycles whatever its size, and the loop around it is a chain of
+    // dependent instructions, so a stage's copies are spread over warps: one KIND of copy (activation boxes, weight
+    // boxes, the two scale chunks) per pair of warps, which take even and odd stages.  Every warp walks all stages
+    // (the walk is a few additions) but waits and issues only for its own; each kind arrives once per stage on the
+    // stage's barrier with its own byte count.
     {
-      const bool side_b = warp == 3;
       PROF_BEGIN();
-      uint32_t s = 0, phase = 0;
-      const uint32_t row_bytes = side_b ? (uint32_t)p.BN * KB : 128u * KB;
-      const uint32_t sf_bytes = side_b ? 512u * SPA * atoms_b : 512u * SPA;
+      uint32_t s = 0, phase = 0, gi = 0;
+      const uint32_t row_bytes = lkind == 1 ? (uint32_t)p.BN * KB : 128u * KB;
       for (unsigned i = 0, t; (t = tile_of_iter(p, i)) < total && !*abort_flag; ++i) {
         const Tile tile = decode_tile(p, t);
         TapWalk<MODE> tw;
@@ -423,34 +426,50 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         const int Q = tw.chunks(p);
         ChunkPos pos;
         pos.reset();
-        const uint8_t* sf_src = side_b ? p.sfb_img + ((size_t)tile.cls * p.tiles_c + tile.ct) * p.max_stages * (512 * SPA * atoms_b)
-                                       : p.sfa_img + (size_t)tile_m_index(p, tile) * p.max_stages * (512 * SPA);
-        for (int q0 = 0; q0 < Q; q0 += G) {
-          if (!PROF_WAIT(mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+        const uint8_t* sfa_src = p.sfa_img + (size_t)tile_m_index(p, tile) * p.max_stages * (512 * SPA);
+        const uint8_t* sfb_src = p.sfb_img + ((size_t)tile.cls * p.tiles_c + tile.ct) * p.max_stages * (512 * SPA * atoms_b);
+        for (int q0 = 0; q0 < Q; q0 += G, ++gi) {
           const int nch = min(G, Q - q0);
-          uint8_t* sa = smem + (size_t)s * stage_bytes;
-          uint8_t* sb = sa + A_STAGE_BYTES;
-          const bool leader = elect_one();
-          if (leader) {
-            mbar_arrive_expect_tx(&full[s], (uint32_t)nch * row_bytes + sf_bytes);
-            bulk_load(sb + b_stage_bytes + (side_b ? SFA_BYTES : 0), sf_src, sf_bytes, &full[s]);
-          }
-          sf_src += sf_bytes;
+          const bool mine = (gi & 1u) == (uint32_t)lhalf;
+          // coordinates of the stage's boxes, before the wait
+          int c0[G], c1[G], c2[G];
 #pragma unroll
           for (int c = 0; c < G; ++c) {
             if (c < nch) {
-              if (leader) {
-                if (side_b) tma_load_3d(sb + c * p.BN * KB, &map_b, &full[s], pos.cc * KB, tap_index(tw, pos), tile.c0);
-                else tma_load_4d(sa + c * 128 * KB, &map_a, &full[s], pos.cc * KB, src_w0(tw, pos), tile.n0, src_h(tw, pos));
-              }
+              c0[c] = pos.cc * KB;
+              c1[c] = lkind == 1 ? tap_index(tw, pos) : src_w0(tw, pos);
+              c2[c] = src_h(tw, pos);
               pos.advance(tw, p.cpt);
             }
           }
-          __syncwarp();
+          if (mine) {
+            uint8_t* sa = smem + (size_t)s * stage_bytes;
+            uint8_t* sb = sa + A_STAGE_BYTES;
+            if (!PROF_WAIT(mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+            if (elect_one()) {
+              if (lkind == 2) {
+                mbar_arrive_expect_tx(&full[s], 512u * SPA * (1 + atoms_b));
+                bulk_load(sb + b_stage_bytes, sfa_src, 512 * SPA, &full[s]);
+                bulk_load(sb + b_stage_bytes + SFA_BYTES, sfb_src, 512 * SPA * atoms_b, &full[s]);
+              } else {
+                mbar_arrive_expect_tx(&full[s], (uint32_t)nch * row_bytes);
+#pragma unroll
+                for (int c = 0; c < G; ++c) {
+                  if (c < nch) {
+                    if (lkind == 1) tma_load_3d(sb + c * p.BN * KB, &map_b, &full[s], c0[c], c1[c], tile.c0);
+                    else tma_load_4d(sa + c * 128 * KB, &map_a, &full[s], c0[c], c1[c], tile.n0, c2[c]);
+                  }
+                }
+              }
+            }
+            __syncwarp();
+          }
+          sfa_src += 512 * SPA;
+          sfb_src += 512 * SPA * atoms_b;
           if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
         }
       }
-      if (!side_b) PROF_END(0);
+      if (warp == 0) PROF_END(0);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -461,6 +480,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const uint64_t a_desc0 = smem_desc(op_desc, smem_u32(smem));
       const uint64_t b_desc0 = smem_desc(op_desc, smem_u32(smem + A_STAGE_BYTES));
       const uint32_t b_chunk16 = (uint32_t)(p.BN * KB) >> 4;
+      const uint64_t sf_desc = smem_desc_base(0, 128, 0);
+      const uint64_t sfa_desc0 = smem_desc(sf_desc, smem_u32(smem + A_STAGE_BYTES + b_stage_bytes));
+      const uint64_t sfb_desc0 = smem_desc(sf_desc, smem_u32(smem + A_STAGE_BYTES + b_stage_bytes + SFA_BYTES));
       uint32_t idesc_id[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) idesc_id[i] = idesc_with_sf_ids(p.idesc, i, i);
@@ -478,12 +500,20 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         uint32_t accumulate = 0;
         for (int q0 = 0; q0 < Q; q0 += G) {
           // the scale copier signals sffull[s] once the stage's operands are in smem and its scale vectors in TMEM
-          if (!PROF_WAIT(mbar_wait(&sffull[s], phase, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+          // E2M1: the scale copier signals sffull[s] once the stage's scale vectors are in TMEM.  8-bit operands: this
+          // warp waits for the stage itself and its lane issues the (three) scale copies right before the MMAs that
+          // read them - same thread, so the tensor pipe keeps the order, and no copy queues behind MMAs issued earlier.
+          if (!PROF_WAIT(mbar_wait(FP4 ? &sffull[s] : &full[s], phase, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
           tc_fence_after_sync();
           const uint32_t so = s * stage16;
           const uint32_t sfa_t = sf_base + s * SF_COLS, sfb_t = sfa_t + 8;
           const int natoms = min(G, Q - q0) * APC;
           if (elect_one()) {
+            if (!FP4) {
+              tmem_cp_32x128b_warpx4(sfa_t, sfa_desc0 + so);
+              tmem_cp_32x128b_warpx4(sfb_t, sfb_desc0 + so);
+              if (atoms_b > 1) tmem_cp_32x128b_warpx4(sfb_t + 4, sfb_desc0 + so + 32);
+            }
             uint32_t accu = accumulate;
 #pragma unroll
             for (int a = 0; a < 4; ++a) {
@@ -513,7 +543,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // Copies the stage's scale chunks smem -> TMEM (one TMEM scale buffer per pipeline stage) from its own
     // thread, so these copies overlap the MMA issuer's work on earlier stages.  The buffer of stage s is free
     // whenever full[s] completes: the producers refilled the stage only after the MMAs that read it committed.
-    {
+    // E2M1 only (twice the scale bytes, up to six copies per stage); for 8-bit operands the MMA lane issues them.
+    if (FP4) {
       const uint64_t sf_desc = smem_desc_base(0, 128, 0);
       const uint32_t sf_base = tmem + p.n_acc * p.BN;
       const uint32_t stage16 = (uint32_t)stage_bytes >> 4;
@@ -544,7 +575,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
       }
     }
-  } else if (warp >= 4) {
+  } else if (warp >= 4 && warp < 12) {
     if (p.pair) epilogue_pair_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else if (p.tma_store) epilogue_tma_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
@@ -905,7 +936,7 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
     }
-  } else if (warp >= 4) {
+  } else if (warp >= 4 && warp < 12) {
     if (p.tma_store) epilogue_tma_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
   }
