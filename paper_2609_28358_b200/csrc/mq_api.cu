@@ -82,7 +82,8 @@ size_t up256(size_t v) { return (v + 255) / 256 * 256; }
 // runs (about 2.2 cycles each per SM, measured), so the choice weighs the tile's MMA time against its store time
 // and both against the padding the tile shape wastes at the edges.
 //   k_bytes: bytes of K per tile row (taps x channel bytes); bn: output channels per tile.
-int choose_tw(int w_eff, int N, int layout, double k_bytes, int bn, bool thin) {
+//   serial: the tile's store is not overlapped with the next tile's MMAs (a single 256-column accumulator).
+int choose_tw(int w_eff, int N, int layout, double k_bytes, int bn, bool thin, bool serial) {
   const int forced = env_int("MQ_TC_TW", 0);
   if (forced > 0) return forced;
   if (thin) return 8;   // the whole-tile kernel (8-column tiles): its per-tile loads beat any per-tap shape on thin layers
@@ -94,7 +95,7 @@ int choose_tw(int w_eff, int N, int layout, double k_bytes, int bn, bool thin) {
     const double waste = (double)((w_eff + tw - 1) / tw * tw) / w_eff * (double)((N + tn - 1) / tn * tn) / N;
     double t_store = 128.0 * (bn * 4.0 / 128.0) * 2.2;          // [H][W][N][C] output: whole lines
     if (layout == MQ_NCHW) t_store = 128.0 * bn / tw * 2.2 * (tw < 8 ? 8.0 / tw : 1.0);   // runs below a 32-byte sector cost a sector each
-    double cost = waste * (t_mma > t_store ? t_mma : t_store);
+    double cost = waste * (serial ? t_mma + t_store : (t_mma > t_store ? t_mma : t_store));
     if (cost < best_cost * (1.0 - 1e-9)) { best_cost = cost; best = tw; }
   }
   return best;
@@ -133,26 +134,29 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   p.cpt = rowbytes / p.KB;
   const int w_eff = op == MQ_OP_FWD ? g.Wo : (g.W + g.sw - 1) / g.sw;
   const bool thin = g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && !env_int("MQ_TC_NO_HALO", 0);
+  const int cd16 = (p.Cd + 15) / 16 * 16;
+  p.BN = cd16 <= 128 ? cd16 : 128;
+  // 256-channel tiles halve the re-reads of the activation tile but leave tensor memory for one accumulator only, so
+  // the epilogue no longer overlaps the next tile: worth it for 8-bit layers whose main loop is long (measured: +30 %
+  // at 2304+ bytes of K per row)
+  if (!fp4 && p.Cd >= 256 && (double)taps * rowbytes >= 2048.0 && (op == MQ_OP_FWD || (g.sh == 1 && g.sw == 1))) p.BN = 256;
+  // E2M1: the same trade pays once the activation codes no longer stay in L2 between their re-reads (measured on
+  // 512 channels: 56x56x256 samples, 205 MB of codes, -10 %; 28x28, 51 MB, +4 %)
+  const double act_bytes = (double)p.Hs * p.Ws * g.N * rowbytes;
+  if (fp4 && p.Cd >= 256 && (double)taps * rowbytes >= 2048.0 && (op == MQ_OP_FWD || (g.sh == 1 && g.sw == 1)) && act_bytes > 96e6) p.BN = 256;
   {
-    const int cd16_ = (p.Cd + 15) / 16 * 16;
+    const int forced_bn_ = env_int("MQ_TC_BN", 0);
+    const int bn_ = (forced_bn_ >= 32 && forced_bn_ <= 256 && forced_bn_ % 32 == 0) ? (forced_bn_ < cd16 ? forced_bn_ : cd16) : p.BN;
     const int nkh_ = op == MQ_OP_FWD ? g.Kh : (g.Kh + g.sh - 1) / g.sh, nkw_ = op == MQ_OP_FWD ? g.Kw : (g.Kw + g.sw - 1) / g.sw;
-    p.TW = choose_tw(w_eff, g.N, layout, (double)nkh_ * nkw_ * rowbytes, cd16_ < 128 ? cd16_ : 128, thin);
+    // with a single accumulator the store time adds to the tile's time instead of hiding behind the next tile: wider
+    // tiles (longer store runs) then win - as long as the activations stay in L2 (measured: 28x28 -11 %, 56x56 +11 %)
+    const bool serial = bn_ > 128 && act_bytes <= 110e6;
+    p.TW = choose_tw(w_eff, g.N, layout, (double)nkh_ * nkw_ * rowbytes, bn_ < 128 ? bn_ : (serial ? bn_ : 128), thin, serial);
   }
   if (p.TW < 1 || p.TW > 32 || (p.TW & (p.TW - 1))) return false;
   p.TN = 128 / p.TW;
   p.lgTW = 0;
   while ((1 << p.lgTW) < p.TW) ++p.lgTW;
-  const int cd16 = (p.Cd + 15) / 16 * 16;
-  p.BN = cd16 <= 128 ? cd16 : 128;
-  // 256-channel tiles halve the re-reads of the activation tile (the per-tap kernel is bound by L2 -> SM bytes) but
-  // leave tensor memory for one accumulator only, so the epilogue no longer overlaps the next tile: worth it for
-  // 8-bit layers whose main loop is long (measured: +30 % at 2304+ bytes of K per row, nothing for E2M1)
-  if (!fp4 && p.Cd >= 256 && (double)taps * rowbytes >= 2048.0 && (op == MQ_OP_FWD || (g.sh == 1 && g.sw == 1))) p.BN = 256;
-  // E2M1: the same trade pays once the activation codes no longer stay in L2 between their re-reads (measured on
-  // 512 channels: 56x56x256 samples, 205 MB of codes, -10 %; 28x28, 51 MB, +4 %)
-  if (fp4 && p.Cd >= 256 && (double)taps * rowbytes >= 2048.0 && (op == MQ_OP_FWD || (g.sh == 1 && g.sw == 1)) &&
-      (double)p.Hs * p.Ws * g.N * rowbytes > 96e6)
-    p.BN = 256;
   const int forced_bn = env_int("MQ_TC_BN", 0);
   if (forced_bn >= 32 && forced_bn <= 256 && forced_bn % 32 == 0) p.BN = forced_bn < cd16 ? forced_bn : cd16;
   p.tiles_c = (p.Cd + p.BN - 1) / p.BN;
