@@ -83,7 +83,9 @@ size_t up256(size_t v) { return (v + 255) / 256 * 256; }
 // and both against the padding the tile shape wastes at the edges.
 //   k_bytes: bytes of K per tile row (taps x channel bytes); bn: output channels per tile.
 //   serial: the tile's store is not overlapped with the next tile's MMAs (a single 256-column accumulator).
-int choose_tw(int w_eff, int N, int layout, double k_bytes, int bn, bool thin, bool serial) {
+//   pair: the tiles of the even and the odd output columns are stored together (stride-2 input gradient): runs of
+//   2 tw floats, and the two accumulators belong to one pair, so the store is not overlapped either.
+int choose_tw(int w_eff, int N, int layout, double k_bytes, int bn, bool thin, bool serial, bool pair) {
   const int forced = env_int("MQ_TC_TW", 0);
   if (forced > 0) return forced;
   if (thin) return 8;   // the whole-tile kernel (8-column tiles): its per-tile loads beat any per-tap shape on thin layers
@@ -94,8 +96,9 @@ int choose_tw(int w_eff, int N, int layout, double k_bytes, int bn, bool thin, b
     const int tn = 128 / tw;
     const double waste = (double)((w_eff + tw - 1) / tw * tw) / w_eff * (double)((N + tn - 1) / tn * tn) / N;
     double t_store = 128.0 * (bn * 4.0 / 128.0) * 2.2;          // [H][W][N][C] output: whole lines
-    if (layout == MQ_NCHW) t_store = 128.0 * bn / tw * 2.2 * (tw < 8 ? 8.0 / tw : 1.0);   // runs below a 32-byte sector cost a sector each
-    double cost = waste * (serial ? t_mma + t_store : (t_mma > t_store ? t_mma : t_store));
+    const int run = pair ? 2 * tw : tw;
+    if (layout == MQ_NCHW) t_store = 128.0 * bn / run * 2.2 * (run < 8 ? 8.0 / run : 1.0);   // runs below a 32-byte sector cost a sector each
+    double cost = waste * ((serial || pair) ? t_mma + t_store : (t_mma > t_store ? t_mma : t_store));
     if (cost < best_cost * (1.0 - 1e-9)) { best_cost = cost; best = tw; }
   }
   return best;
@@ -151,7 +154,8 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
     // with a single accumulator the store time adds to the tile's time instead of hiding behind the next tile: wider
     // tiles (longer store runs) then win - as long as the activations stay in L2 (measured: 28x28 -11 %, 56x56 +11 %)
     const bool serial = bn_ > 128 && act_bytes <= 110e6;
-    p.TW = choose_tw(w_eff, g.N, layout, (double)nkh_ * nkw_ * rowbytes, bn_ < 128 ? bn_ : (serial ? bn_ : 128), thin, serial);
+    const bool pair_hint = op == MQ_OP_BWD_DATA && g.sw == 2 && layout == MQ_NCHW && p.Wd % 2 == 0 && bn_ <= 128 && !env_int("MQ_TC_NO_PAIR", 0);
+    p.TW = choose_tw(w_eff, g.N, layout, (double)nkh_ * nkw_ * rowbytes, bn_ < 128 ? bn_ : (serial ? bn_ : 128), thin, serial, pair_hint);
   }
   if (p.TW < 1 || p.TW > 32 || (p.TW & (p.TW - 1))) return false;
   p.TN = 128 / p.TW;
