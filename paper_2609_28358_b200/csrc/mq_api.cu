@@ -352,6 +352,7 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   w.Npad = 32 * p.BPP * p.nchunks;
   p.groups_w = (g.Wo + p.KPX - 1) / p.KPX;
   p.Wp = g.W + 2 * g.pw;
+  p.Hp = g.H + 2 * g.ph;
   p.stages_total = flat ? (g.Ho * p.Wp + p.KPX - 1) / p.KPX : g.Ho * p.groups_w * p.nchunks;
   p.b_rows = flat ? (g.Cp < 128 ? g.Cp : 128) : 128;
   // 8-bit operands: 256 input channels per MMA when the layer has them (the kernel is bound by the tensor core's
@@ -394,7 +395,7 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   w.P_b = (w.P_a + (g.Kh - 1) * p.Wp + g.Kw - 1 + 7) / 8 * 8;
   size_t o = up256((size_t)splits * g.Cout * g.Kh * g.Kw * g.Cp * sizeof(float));
   w.off_sfa = o; o += up256((size_t)p.m_tiles128 * p.stages_total * 512 * spa);
-  w.off_sfb = o; o += up256((size_t)p.cb_tiles * (g.Kh * g.Kw / p.TG) * p.stages_total * p.NB * 512 * spa);
+  w.off_sfb = o; o += up256(fp8 ? (size_t)p.cb_tiles * p.Hp * p.Wp * p.nchunks * p.NB * 512 : (size_t)p.cb_tiles * (g.Kh * g.Kw / p.TG) * p.stages_total * p.NB * 512 * spa);
   w.off_xt = o;
   if (flat) { p.xt_block_bytes = (long long)w.P_b * p.b_rows * p.KBn; o += up256((size_t)p.cb_tiles * p.xt_block_bytes); }
   else if (fp4) o += up256((size_t)g.Cp * g.H * g.W * w.Npad / 2);
@@ -472,7 +473,7 @@ mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const 
   if (p.cta2) {   // a pair's scale chunks travel as tiled copies too (rows of 256 bytes), so that they can count on the leader's barrier
     const int spa = 1;   // 8-bit operands only
     const uint64_t rows_a = (uint64_t)p.m_tiles128 * p.stages_total * 2 * spa;
-    const uint64_t rows_b = (uint64_t)p.cb_tiles * (g.Kh * g.Kw / p.TG) * p.stages_total * p.NB * 2 * spa;
+    const uint64_t rows_b = (uint64_t)p.cb_tiles * p.Hp * p.Wp * p.nchunks * p.NB * 2 * spa;
     const uint64_t da[2] = {256, rows_a}, db[2] = {256, rows_b}, st[1] = {256};
     const uint32_t ba[2] = {256u, (uint32_t)(2 * spa)}, bb[2] = {256u, (uint32_t)(2 * spa * p.NB)};
     if (!encode_tensor_map_u8(&map_sfa, p.sfa_img, 2, da, st, ba, nullptr, 0)) return MQ_ERR_CUDA;

@@ -92,7 +92,8 @@ struct WgradTcParams {
   int nchunks;          // stages per pixel group
   int groups_w;         // ceil(Wo / KPX)
   int stages_total;     // pixel: Ho * groups_w * nchunks; flat: ceil(Ho * Wp / KPX)
-  int Wp;               // flat: padded width W + 2 * pw
+  int Wp;               // padded width W + 2 * pw
+  int Hp;               // padded height H + 2 * ph
   int b_rows;           // rows (input channels) of a B tile: 128, or min(128, Cp) in flat mode
   int m_tiles, j_tiles, cb_tiles, splits;   // j_tiles = (taps / TG) * cb_tiles; m_tiles counts work units along C_out
   int m_tiles128;       // 128-row tiles of output channels (= m_tiles, or 2 * m_tiles when cta2)
@@ -109,7 +110,7 @@ struct WgradTcParams {
   const uint8_t* xt;        // flat: [ci block][padded pixel][b_rows][KBn]
   long long gt_block_bytes, xt_block_bytes;
   uint8_t* sfa_img;         // [m tile][stage][512 * SPA]
-  uint8_t* sfb_img;         // [ci block][tap group][stage][NB][512 * SPA]
+  uint8_t* sfb_img;         // E2M1: [ci block][tap group][stage][NB][512 * SPA]; 8-bit: [ci block][Hp][Wp][sample chunk][NB][512]
   float* partial;           // [splits][Cout][taps * Cp]
   unsigned int* status;
 };

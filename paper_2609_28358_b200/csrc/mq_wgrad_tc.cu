@@ -59,7 +59,9 @@ __device__ __forceinline__ void expand_wgrad_scales_body(const WgradTcParams& p,
   const int taps = p.Kh * p.Kw;
   const long long nA = (long long)p.m_tiles128 * p.stages_total;
   const int groups = taps / p.TG;
-  const long long nB = (long long)p.cb_tiles * groups * p.stages_total * p.NB;
+  // B-side chunks: E2M1 modes one per (channel block, tap group, stage); 8-bit mode one per (channel block, padded X
+  // pixel, sample chunk) - a stage's chunk depends only on where its taps' pixels start, so the taps share them
+  const long long nB = FP4 ? (long long)p.cb_tiles * groups * p.stages_total * p.NB : (long long)p.cb_tiles * p.Hp * p.Wp * p.nchunks * p.NB;
   if (wid >= nA + nB) return;
   // this lane's byte: 32-row group j of the 128-row chunk, K-block b of the stage
   const int j = lane >> 3, b = lane & 7;
@@ -75,9 +77,21 @@ __device__ __forceinline__ void expand_wgrad_scales_body(const WgradTcParams& p,
     }
     dst = p.sfa_img + wid * (512 * SPA);
   } else {
-    // B rows of a tap group: tap-in-group major, input channel minor; chunk c holds rows [128c, 128c + 128)
     long long idx = wid - nA;
     const int c = (int)(idx % p.NB); idx /= p.NB;
+    if (!FP4) {
+      // chunk (cb, hp, wp, nc): K-block b is pixel (hp - ph, wp - pw + (b / BPP) sw), sample block nc BPP + b % BPP
+      const int nc = (int)(idx % p.nchunks); idx /= p.nchunks;
+      const int wp = (int)(idx % p.Wp); idx /= p.Wp;
+      const int hp = (int)(idx % p.Hp); const int cb = (int)(idx / p.Hp);
+      const int cib = (cb * p.b_rows + c * 128 + 32 * j) / 32;
+      if (b < NBS && cib < p.Ct) {
+        const int px = b / p.BPP, nb = nc * p.BPP + (b - px * p.BPP);
+        const int h = hp - p.ph, w = wp - p.pw + px * p.sw;
+        if (nb < p.Nt && h >= 0 && h < p.H && w >= 0 && w < p.W) v = __ldg(p.x_scales + (((long long)h * p.W + w) * p.Nt + nb) * p.Ct + cib);
+      }
+    } else {
+    // B rows of a tap group: tap-in-group major, input channel minor; chunk c holds rows [128c, 128c + 128)
     const int st = (int)(idx % p.stages_total); idx /= p.stages_total;
     const int tg = (int)(idx % groups); const int cb = (int)(idx / groups);
     const int row0 = c * 128 + 32 * j;
@@ -91,6 +105,7 @@ __device__ __forceinline__ void expand_wgrad_scales_body(const WgradTcParams& p,
       const int h = ho * p.sh + kh - p.ph, w = wo * p.sw + kw - p.pw;
       if (ho < p.Ho && wo < p.Wo && nb < p.Nt && h >= 0 && h < p.H && w >= 0 && w < p.W)
         v = __ldg(p.x_scales + (((long long)h * p.W + w) * p.Nt + nb) * p.Ct + cib);
+    }
     }
     dst = p.sfb_img + (wid - nA) * (512 * SPA);
   }
@@ -215,7 +230,6 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     }
     const uint32_t my_bytes = (kind == 0 ? a_bytes : (kind <= 2 ? b_bytes : 512u * SPA + sfb_bytes)) * (CTA2 ? 2u : 1u);
     const int sfa_row0 = (int)(((size_t)mt * p.stages_total + st_begin) * (2 * SPA));          // rows of 256 bytes (pair mode maps)
-    const int sfb_row0 = (int)((((size_t)cb * (taps / TG) + tgi) * p.stages_total + st_begin) * (2 * SPA * p.NB));
     int nc, wg, ho;                                            // of the first stage this warp handles
     {
       const int st = st_begin + half;
@@ -239,16 +253,18 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       if (elect_one()) {
         if (kind == 0) WTRACE(0, i);
         if (rank == 0) mbar_arrive_expect_tx(bar, my_bytes);
+        // 8-bit mode: the X-side chunk of (padded pixel, sample chunk); E2M1: of (tap group, stage)
+        const long long xchunk = !FP4 ? ((((long long)cb * p.Hp + (xh + p.ph)) * p.Wp + (xw + p.pw)) * p.nchunks + nc) : 0;
         if (CTA2) {
           if (kind == 0) tma_load_4d_pair(sa, &map_a, lbar, co0, nrow, wo0, ho);
           else if (kind == 1) tma_load_4d_pair(sb, &map_b, lbar, ci_ld, nrow, xw, xh);
           else {
             tma_load_2d_pair(ssf, &map_sfa, lbar, 0, sfa_row0 + i * (2 * SPA));
-            tma_load_2d_pair(ssf + 1024, &map_sfb, lbar, 0, sfb_row0 + i * (2 * SPA * p.NB));
+            tma_load_2d_pair(ssf + 1024, &map_sfb, lbar, 0, (int)(xchunk * (2 * SPA * p.NB)));
           }
         } else if (kind == 3) {
           bulk_load(ssf, sfa_src + (size_t)i * (512 * SPA), 512 * SPA, bar);
-          bulk_load(ssf + 1024, sfb_src + (size_t)i * sfb_bytes, sfb_bytes, bar);
+          bulk_load(ssf + 1024, FP4 ? sfb_src + (size_t)i * sfb_bytes : p.sfb_img + (size_t)xchunk * sfb_bytes, sfb_bytes, bar);
         } else if (p.mode == MQ_WG_FP4_FLAT) {
           if (kind == 0) bulk_load(sa, ga + (size_t)i * a_bytes, a_bytes, bar);
           else bulk_load(sb, gb + (size_t)i * b_step, b_bytes, bar);          // KPX + TG - 1 consecutive pixels
@@ -631,7 +647,8 @@ cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, co
 }
 
 cudaError_t launch_expand_wgrad_scales(const WgradTcParams& p, cudaStream_t s) {
-  const long long warps = (long long)p.m_tiles128 * p.stages_total + (long long)p.cb_tiles * (p.Kh * p.Kw / p.TG) * p.stages_total * p.NB;
+  const long long nb = p.mode == MQ_WG_FP8 ? (long long)p.cb_tiles * p.Hp * p.Wp * p.nchunks * p.NB : (long long)p.cb_tiles * (p.Kh * p.Kw / p.TG) * p.stages_total * p.NB;
+  const long long warps = (long long)p.m_tiles128 * p.stages_total + nb;
   const unsigned blocks = (unsigned)((warps + 7) / 8);
   count_launches(1);
   if (p.mode == MQ_WG_FP8) return launch_pdl(expand_wgrad_scales_kernel<false>, dim3(blocks), dim3(256), 0, s, p);
