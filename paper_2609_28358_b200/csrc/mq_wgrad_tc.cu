@@ -18,6 +18,7 @@
 // One thread block per work item (128 output channels x one tap's block of input channels x a slice of
 // the K range); partial sums go to scratch and are added in a fixed order by bwd_weight_reduce.
 // Warps: 0 producer (TMA / bulk copies), 1 MMA issuer, 2 scale copier (smem -> TMEM), 4-7 epilogue.
+#include <cstdlib>
 #include "mq_conv_tc.cuh"
 #include "mq_tcgen05.cuh"
 
@@ -571,7 +572,10 @@ struct FlatArgs {
   const uint8_t* in; uint8_t* out;
   int Hs, Ws, N, Cs_p, P_out, Wp, off_h, off_w, rows, nblocks, KBn, ncg;
   unsigned units, blocks;
+  int wide;   // 1: 256 samples x 256 channels per block through shared memory (whole lines in and out)
 };
+constexpr int FLAT_WIDE_PITCH = 33;                                   // words per staged row (132 bytes: conflict-free columns)
+constexpr int FLAT_WIDE_SMEM = 2 * 256 * FLAT_WIDE_PITCH * 4;         // input tile + output tile
 __device__ __forceinline__ void fp4_to_flat_body(const FlatArgs& fa, unsigned block, unsigned nblocks_grid) {
   const uint8_t* __restrict__ in = fa.in; uint8_t* __restrict__ out = fa.out;
   const int Hs = fa.Hs, Ws = fa.Ws, N = fa.N, Cs_p = fa.Cs_p, P_out = fa.P_out, Wp = fa.Wp, off_h = fa.off_h, off_w = fa.off_w;
@@ -610,13 +614,72 @@ __device__ __forceinline__ void fp4_to_flat_body(const FlatArgs& fa, unsigned bl
   }
 }
 
+// Wide variant (256 samples per pixel, i.e. 128-byte pieces): a block takes (padded pixel, 256 channels), reads its
+// 256 sample rows x 128 bytes as whole lines into shared memory, the warps transpose 32 x 64 sub-blocks in registers as
+// above, and the 256 channel rows x 128 bytes leave as whole lines (the narrow variant reads 32-byte and writes
+// 16-byte runs, which costs a memory request each).
+__device__ __forceinline__ void fp4_to_flat_wide_body(const FlatArgs& fa, unsigned block, unsigned nblocks_grid, uint32_t* sm) {
+  const uint8_t* __restrict__ in = fa.in; uint8_t* __restrict__ out = fa.out;
+  uint32_t* sin = sm;
+  uint32_t* sout = sm + 256 * FLAT_WIDE_PITCH;
+  const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
+  const int k = lane & 7, ng = lane >> 3;
+  const int ncgw = fa.ncg;                        // 256-channel groups
+  const int cmax = fa.nblocks * fa.rows;
+  const int row_t = t >> 3, ch_t = t & 7;          // this thread's row (+ 32 m) and 16-byte chunk of a 128-byte line
+#pragma unroll 1
+  for (unsigned u = block; u < fa.units; u += nblocks_grid) {
+    const unsigned q = u / (unsigned)ncgw;
+    const int cgw = (int)(u - q * (unsigned)ncgw);
+    const int hq = (int)(q / (unsigned)fa.Wp), wq = (int)q - hq * fa.Wp;
+    const int h = hq - fa.off_h, w = wq - fa.off_w;
+    const bool pix_ok = h >= 0 && h < fa.Hs && w >= 0 && w < fa.Ws;
+    const int cbase = cgw * 256;
+#pragma unroll
+    for (int m = 0; m < 8; ++m) {
+      const int row = row_t + 32 * m;
+      uint4 v = make_uint4(0u, 0u, 0u, 0u);
+      if (pix_ok && row < fa.N && cbase + 32 * ch_t < fa.Cs_p)
+        v = __ldg(reinterpret_cast<const uint4*>(in + ((((long long)h * fa.Ws + w) * fa.N + row) * fa.Cs_p + cbase + 32 * ch_t) / 2));
+      uint32_t* d = sin + row * FLAT_WIDE_PITCH + 4 * ch_t;
+      d[0] = v.x; d[1] = v.y; d[2] = v.z; d[3] = v.w;
+    }
+    __syncthreads();
+#pragma unroll 1
+    for (int sb = warp; sb < 32; sb += 8) {
+      const int nb = sb >> 2, cg = sb & 3;
+      uint32_t wd[8];
+#pragma unroll
+      for (int j = 0; j < 8; ++j) wd[j] = sin[(nb * 32 + 8 * ng + j) * FLAT_WIDE_PITCH + cg * 8 + k];
+      nibble_transpose_8x8(wd);                     // wd[i]: channel cg * 64 + 8k + i, samples nb * 32 + 8ng .. + 7
+#pragma unroll
+      for (int i = 0; i < 8; ++i) sout[(cg * 64 + 8 * k + i) * FLAT_WIDE_PITCH + ((nb ^ i) << 2) + ng] = wd[i];   // 128-byte swizzle: chunk nb ^ (row & 7)
+    }
+    __syncthreads();
+#pragma unroll
+    for (int m = 0; m < 8; ++m) {
+      const int row = row_t + 32 * m;
+      const int c = cbase + row;
+      if (c < cmax) {
+        const int blk = c / fa.rows, r = c - blk * fa.rows;
+        const uint32_t* sp = sout + row * FLAT_WIDE_PITCH + 4 * ch_t;
+        *reinterpret_cast<uint4*>(out + (((long long)blk * fa.P_out + q) * fa.rows + r) * 128 + 16 * ch_t) = make_uint4(sp[0], sp[1], sp[2], sp[3]);
+      }
+    }
+    // the next unit's fill of `sin` is ordered after this unit's reads of it by the second barrier above; its writes
+    // to `sout` come after its own first barrier, which every thread reaches only after these reads
+  }
+}
+
 // Preparation of the flat mode in one launch: blocks [0, x.blocks) re-lay X, the next g.blocks re-lay G_Y, the rest
 // expand the scale chunks.
 __global__ void __launch_bounds__(256) wgrad_flat_prep_kernel(const FlatArgs x, const FlatArgs gy, const WgradTcParams p) {
+  extern __shared__ __align__(16) uint32_t flat_sm[];
   pdl_wait();
-  if (blockIdx.x < x.blocks) fp4_to_flat_body(x, blockIdx.x, x.blocks);
-  else if (blockIdx.x < x.blocks + gy.blocks) fp4_to_flat_body(gy, blockIdx.x - x.blocks, gy.blocks);
-  else expand_wgrad_scales_body<true>(p, blockIdx.x - x.blocks - gy.blocks);
+  if (blockIdx.x < x.blocks) { if (x.wide) fp4_to_flat_wide_body(x, blockIdx.x, x.blocks, flat_sm); else fp4_to_flat_body(x, blockIdx.x, x.blocks); }
+  else if (blockIdx.x < x.blocks + gy.blocks) {
+    if (gy.wide) fp4_to_flat_wide_body(gy, blockIdx.x - x.blocks, gy.blocks, flat_sm); else fp4_to_flat_body(gy, blockIdx.x - x.blocks, gy.blocks);
+  } else expand_wgrad_scales_body<true>(p, blockIdx.x - x.blocks - gy.blocks);
 }
 
 }  // namespace
@@ -666,6 +729,15 @@ static bool make_flat_args(FlatArgs* fa, const uint8_t* in, uint8_t* out, int Hs
                            int nblocks, int KBn) {
   fa->in = in; fa->out = out; fa->Hs = Hs; fa->Ws = Ws; fa->N = N; fa->Cs_p = Cs_p; fa->P_out = P_out; fa->Wp = Wp; fa->off_h = off_h; fa->off_w = off_w;
   fa->rows = rows; fa->nblocks = nblocks; fa->KBn = KBn;
+  fa->wide = (KBn == 128 && nblocks * rows >= 256 && N <= 256 && !getenv("MQ_WGRAD_NO_WIDE_PREP")) ? 1 : 0;
+  if (fa->wide) {
+    fa->ncg = (nblocks * rows + 255) / 256;
+    const long long units = (long long)P_out * fa->ncg;
+    if (units >= 0xffffffffLL) return false;
+    fa->units = (unsigned)units;
+    fa->blocks = (unsigned)(units < 148LL * 3 ? (units < 1 ? 1 : units) : 148LL * 3);
+    return true;
+  }
   fa->ncg = (nblocks * rows + 63) / 64;
   const long long units = (long long)P_out * (KBn / 16) * fa->ncg;
   if (units >= 0xffffffffLL) return false;
@@ -685,7 +757,13 @@ cudaError_t launch_wgrad_flat_prep(const WgradTcParams& p, const uint8_t* x_code
   const long long warps = (long long)p.m_tiles128 * p.stages_total + (long long)p.cb_tiles * (p.Kh * p.Kw / p.TG) * p.stages_total * p.NB;
   const unsigned sc_blocks = (unsigned)((warps + 7) / 8);
   count_launches(1);
-  return launch_pdl(wgrad_flat_prep_kernel, dim3(fx.blocks + fg.blocks + sc_blocks), dim3(256), 0, s, fx, fg, p);
+  const size_t smem = (fx.wide || fg.wide) ? (size_t)FLAT_WIDE_SMEM : 0;
+  static bool attr_set = false;
+  if (smem && !attr_set) {
+    if (cudaFuncSetAttribute(wgrad_flat_prep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, FLAT_WIDE_SMEM) != cudaSuccess) return cudaErrorInvalidValue;
+    attr_set = true;
+  }
+  return launch_pdl(wgrad_flat_prep_kernel, dim3(fx.blocks + fg.blocks + sc_blocks), dim3(256), smem, s, fx, fg, p);
 }
 
 }  // namespace mq

@@ -35,6 +35,7 @@ SMALL_SHAPES = [
     ("thin_wide", (16, 32, 6, 8, 160, 3, 1, 1)),   # thin contraction, two output-channel tiles (weight tile reloaded) in fwd
     ("wide_thin", (16, 160, 6, 8, 32, 3, 1, 1)),   # the same situation in the input gradient
     ("wide", (32, 256, 4, 8, 288, 3, 1, 1)),       # 256-channel MMAs (8-bit) and a remainder channel tile
+    ("deep_batch", (250, 320, 3, 4, 288, 3, 1, 1)),  # 8 sample tiles (ragged): E2M1 whole-line re-layout with partial channel groups, block pairs
 ]
 
 
@@ -147,7 +148,8 @@ def test_config3_layers_full_size(li):
 
 
 CFG5_POINTS = ["cfg5_e4m3_k3s1_c64_hw14", "cfg5_e4m3_k3s2_c128_hw28", "cfg5_e4m3_k1s1_c256_hw14", "cfg5_e2m1_k3s1_c128_hw14",
-               "cfg5_e2m1_k1s2_c64_hw28", "cfg5_e2m1_k3s2_c256_hw14", "cfg5_e4m3_k3s1_c512_hw14", "cfg5_e4m3_k3s1_c64_hw56"]
+               "cfg5_e2m1_k1s2_c64_hw28", "cfg5_e2m1_k3s2_c256_hw14", "cfg5_e4m3_k3s1_c512_hw14", "cfg5_e4m3_k3s1_c64_hw56",
+               "cfg5_e2m1_k3s1_c256_hw14"]
 
 
 @pytest.mark.parametrize("name", CFG5_POINTS)
