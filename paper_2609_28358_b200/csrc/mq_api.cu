@@ -143,10 +143,10 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   // the epilogue no longer overlaps the next tile: worth it for 8-bit layers whose main loop is long (measured: +30 %
   // at 2304+ bytes of K per row)
   if (!fp4 && p.Cd >= 256 && (double)taps * rowbytes >= 2048.0 && (op == MQ_OP_FWD || (g.sh == 1 && g.sw == 1))) p.BN = 256;
-  // E2M1: the same trade pays once the activation codes no longer stay in L2 between their re-reads (measured on
-  // 512 channels: 56x56x256 samples, 205 MB of codes, -10 %; 28x28, 51 MB, +4 %)
+  // E2M1: the same trade (measured with the tile widths chosen below: 256 channels 28x28 -13 %, 512 channels 14x14 -6 %,
+  // 56x56 -10 %)
   const double act_bytes = (double)p.Hs * p.Ws * g.N * rowbytes;
-  if (fp4 && p.Cd >= 256 && (double)taps * rowbytes >= 2048.0 && (op == MQ_OP_FWD || (g.sh == 1 && g.sw == 1)) && act_bytes > 96e6) p.BN = 256;
+  if (fp4 && p.Cd >= 256 && (double)taps * rowbytes >= 1024.0 && (op == MQ_OP_FWD || (g.sh == 1 && g.sw == 1)) && !env_int("MQ_TC_FP4_BN128", 0)) p.BN = 256;
   {
     const int forced_bn_ = env_int("MQ_TC_BN", 0);
     const int bn_ = (forced_bn_ >= 32 && forced_bn_ <= 256 && forced_bn_ % 32 == 0) ? (forced_bn_ < cd16 ? forced_bn_ : cd16) : p.BN;
@@ -194,6 +194,7 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   // TMEM (512 columns): accumulators (BN columns each) + one 24-column scale buffer per pipeline stage
   p.n_acc = (2 * p.BN + 24 * stages <= 512) ? 2 : 1;
   if (p.n_acc * p.BN + 24 * stages > 512) return false;
+  p.mma_cp = env_int("MQ_TC_NO_MMA_CP", 0) ? 0 : 1;   // E2M1 too: the bubble behind a copier warp costs more than the lane's extra issues
   p.pair = op == MQ_OP_BWD_DATA && g.sw == 2 && layout == MQ_NCHW && p.Wd % 2 == 0 && p.n_acc == 2 && p.total_tiles % 2 == 0 &&
            !env_int("MQ_TC_NO_PAIR", 0);
   const int nkh = op == MQ_OP_FWD ? g.Kh : (g.Kh + g.sh - 1) / g.sh, nkw = op == MQ_OP_FWD ? g.Kw : (g.Kw + g.sw - 1) / g.sw;
@@ -353,6 +354,7 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   p.groups_w = (g.Wo + p.KPX - 1) / p.KPX;
   p.Wp = g.W + 2 * g.pw;
   p.Hp = g.H + 2 * g.ph;
+  p.mma_cp = env_int("MQ_WGRAD_MMA_CP", 0);
   p.stages_total = flat ? (g.Ho * p.Wp + p.KPX - 1) / p.KPX : g.Ho * p.groups_w * p.nchunks;
   p.b_rows = flat ? (g.Cp < 128 ? g.Cp : 128) : 128;
   // 8-bit operands: 256 input channels per MMA when the layer has them (the kernel is bound by the tensor core's

@@ -486,6 +486,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       uint32_t idesc_id[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) idesc_id[i] = idesc_with_sf_ids(p.idesc, i, i);
+      const bool self_cp = !FP4 || p.mma_cp;
       uint32_t s = 0, phase = 0, tcount = 0;
       PROF_BEGIN();
       for (unsigned t; (t = tile_of_iter(p, tcount)) < total && !*abort_flag; ++tcount) {
@@ -503,16 +504,19 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           // E2M1: the scale copier signals sffull[s] once the stage's scale vectors are in TMEM.  8-bit operands: this
           // warp waits for the stage itself and its lane issues the (three) scale copies right before the MMAs that
           // read them - same thread, so the tensor pipe keeps the order, and no copy queues behind MMAs issued earlier.
-          if (!PROF_WAIT(mbar_wait(FP4 ? &sffull[s] : &full[s], phase, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+          if (!PROF_WAIT(mbar_wait(self_cp ? &full[s] : &sffull[s], phase, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
           tc_fence_after_sync();
           const uint32_t so = s * stage16;
           const uint32_t sfa_t = sf_base + s * SF_COLS, sfb_t = sfa_t + 8;
           const int natoms = min(G, Q - q0) * APC;
           if (elect_one()) {
-            if (!FP4) {
-              tmem_cp_32x128b_warpx4(sfa_t, sfa_desc0 + so);
-              tmem_cp_32x128b_warpx4(sfb_t, sfb_desc0 + so);
-              if (atoms_b > 1) tmem_cp_32x128b_warpx4(sfb_t + 4, sfb_desc0 + so + 32);
+            if (self_cp) {
+#pragma unroll
+              for (int g = 0; g < SPA; ++g) {
+                tmem_cp_32x128b_warpx4(sfa_t + 4 * g, sfa_desc0 + so + g * 32);
+                tmem_cp_32x128b_warpx4(sfb_t + 4 * g * atoms_b, sfb_desc0 + so + g * atoms_b * 32);
+                if (atoms_b > 1) tmem_cp_32x128b_warpx4(sfb_t + 4 * (g * atoms_b + 1), sfb_desc0 + so + (g * atoms_b + 1) * 32);
+              }
             }
             uint32_t accu = accumulate;
 #pragma unroll
@@ -544,7 +548,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // thread, so these copies overlap the MMA issuer's work on earlier stages.  The buffer of stage s is free
     // whenever full[s] completes: the producers refilled the stage only after the MMAs that read it committed.
     // E2M1 only (twice the scale bytes, up to six copies per stage); for 8-bit operands the MMA lane issues them.
-    if (FP4) {
+    if (FP4 && !p.mma_cp) {
       const uint64_t sf_desc = smem_desc_base(0, 128, 0);
       const uint32_t sf_base = tmem + p.n_acc * p.BN;
       const uint32_t stage16 = (uint32_t)stage_bytes >> 4;

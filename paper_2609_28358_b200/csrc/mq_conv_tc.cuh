@@ -51,6 +51,7 @@ struct ConvTcParams {
   int halo_b_bytes;         // bytes of the resident weight image + its scale chunks (rounded up to 1024)
   int fused;                // 1: single channel tile, stride 1: no preparation kernel (the blocks build the weight image, its
                             //    scale chunks and every tile's activation scale chunks themselves)
+  int mma_cp;             // E2M1: 1 = the MMA lane issues the scale copies itself (no copier warp)
   int pair;                 // per-tap kernel, input gradient with column stride 2, NCHW output: see tile_of_iter
   int tma_store;            // 1: NCHW output written by TMA stores from per-warp staging slices
   const uint8_t* b_codes;   // weight-like codes [rows][taps][b_rowbytes] (source of the images below)
@@ -97,6 +98,7 @@ struct WgradTcParams {
   int b_rows;           // rows (input channels) of a B tile: 128, or min(128, Cp) in flat mode
   int m_tiles, j_tiles, cb_tiles, splits;   // j_tiles = (taps / TG) * cb_tiles; m_tiles counts work units along C_out
   int m_tiles128;       // 128-row tiles of output channels (= m_tiles, or 2 * m_tiles when cta2)
+  int mma_cp;           // E2M1: 1 = the MMA lane issues the scale copies itself (no copier warp)
   int cta2;             // 1: pairs of blocks (clusters of 2) compute 256 x 256 tiles with cta_group::2 MMAs
   int TG;               // taps per block: 1, or Kw (flat mode: the taps of a kernel row share the stage's pixels)
   int NB;               // 128-row chunks of the group's B rows = ceil(TG * b_rows / 128)

@@ -343,7 +343,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 #ifdef MQ_TC_PROFILE
         const long long q0 = clock64();
 #endif
-        if (!mbar_wait(FP4 ? &sffull[s] : &full[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+        if (!mbar_wait((FP4 && !p.mma_cp) ? &sffull[s] : &full[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
 #ifdef MQ_TC_PROFILE
         const long long q1 = clock64();
         if (!FP4 && lane == 0) WTRACE(1, i);
@@ -381,6 +381,15 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           }
         } else
         if (elect_one()) {
+        if (FP4 && p.mma_cp) {
+          const uint64_t sfd = sf_desc0 + so;
+#pragma unroll
+          for (int g = 0; g < SPA; ++g) tmem_cp_32x128b_warpx4(sf_t + 4 * g, sfd + g * 32);
+#pragma unroll 1
+          for (int c = 0; c < p.NB; ++c)
+#pragma unroll
+            for (int g = 0; g < SPA; ++g) tmem_cp_32x128b_warpx4(sf_t + 8 + 4 * (g * p.NB + c), sfd + 64 + (c * SPA + g) * 32);
+        }
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
           const uint32_t accu = a > 0 ? 1u : accumulate;
@@ -423,7 +432,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   } else if (warp == 2) {
     // ------------------------------------------------------------------ scale copier (smem -> per-stage TMEM buffers)
     // E2M1 only (twice the scale bytes, up to eight copies per stage); for 8-bit operands the MMA lane issues them.
-    if (FP4) {
+    if (FP4 && !p.mma_cp) {
       const uint64_t sf_desc = smem_desc_base(0, 128, 0);
       const uint64_t sf_desc0 = smem_desc(sf_desc, smem_u32(smem + sf_off));
       const uint32_t stage16 = (uint32_t)stage_bytes >> 4;
