@@ -781,19 +781,39 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       PROF_BEGIN();
       for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
         const int ct = p.tiles_c == 1 ? 0 : (int)((t / tiles_per_c) % (unsigned)p.tiles_c);
-        if (ct != cur_ct) {
+        const bool new_b = ct != cur_ct;
+        if (new_b) {
           if (!PROF_WAIT(mbar_wait(bfull, bcount & 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
           cur_ct = ct; ++bcount;
         }
         const int acc = (int)(tcount & acc_mask);
         if (!PROF_WAIT(mbar_wait(&tempty[acc], ((tcount >> acc_shift) & 1) ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
-        if (!PROF_WAIT(mbar_wait(&sffull[s], phase, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+        if (!PROF_WAIT(mbar_wait(p.mma_cp ? &full[s] : &sffull[s], phase, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem + acc * p.BN;
         const uint32_t sa16 = smem_u32(stage0 + (size_t)s * stage_bytes) >> 4;
         const uint32_t sfa_s = sfa_base + s * sfa_cols_stage;
         const long long pc0 = PROF_CLK();
         if (elect_one()) {
+        if (p.mma_cp) {   // this lane issues the scale copies itself, right before the MMAs that read them
+          const uint64_t sf_desc = smem_desc_base(0, 128, 0);
+          if (new_b) {
+            const uint32_t sfb_s = smem_u32(smem + b_bytes);
+#pragma unroll 1
+            for (int st = 0; st < nsf; ++st)
+#pragma unroll
+              for (int g = 0; g < SPA; ++g)
+#pragma unroll 1
+                for (int a2 = 0; a2 < atoms_b; ++a2)
+                  tmem_cp_32x128b_warpx4(sfb_base + st * 16 + 4 * (g * atoms_b + a2), smem_desc(sf_desc, sfb_s + ((st * SPA + g) * atoms_b + a2) * 512));
+          }
+          const uint32_t sfa_sm = smem_u32(stage0 + (size_t)s * stage_bytes + p.halo_a_bytes);
+#pragma unroll 1
+          for (int st = 0; st < nsf; ++st) {
+#pragma unroll
+            for (int g = 0; g < SPA; ++g) tmem_cp_32x128b_warpx4(sfa_s + st * 8 + 4 * g, smem_desc(sf_desc, sfa_sm + (st * SPA + g) * 512));
+          }
+        }
         uint32_t accumulate = 0;
         auto issue_tap = [&](int q, uint32_t a16, uint32_t b16) {
           const int sfst = q / G;
@@ -832,7 +852,7 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     }
   } else if (warp == 2) {
     // ------------------------------------------------------------------ scale copier: chunks smem -> TMEM
-    {
+    if (!p.mma_cp) {
       const uint64_t sf_desc = smem_desc_base(0, 128, 0);
       uint32_t s = 0, phase = 0, bcount = 0;
       int cur_ct = -1;
