@@ -194,6 +194,19 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   // TMEM (512 columns): accumulators (BN columns each) + one 24-column scale buffer per pipeline stage
   p.n_acc = (2 * p.BN + 24 * stages <= 512) ? 2 : 1;
   if (p.n_acc * p.BN + 24 * stages > 512) return false;
+  // pairs of blocks (cta_group::2) on two neighbouring tiles that share the weight tile: 128-byte K chunks, 256-channel
+  // tiles, no stride classes, and an even number of tiles per channel tile so that a pair never straddles two of them
+  // Opt-in (MQ_TC_CTA2=1): measured within +-5 % of single blocks (512 channels 28x28 8-bit -2.5 %, E2M1 56x56 -5 %,
+  // 256 channels +2 %) - with one 256-column accumulator these kernels wait on their NCHW stores, not on loads or issue.
+  p.cta2 = (p.BN == 256 && p.KB == 128 && p.classes == 1 && ((long long)p.tiles_w * p.tiles_h) % 2 == 0 && p.total_tiles >= 2 &&
+            env_int("MQ_TC_CTA2", 0)) ? 1 : 0;
+  if (p.cta2) {
+    const size_t sb2 = 128 * 128 + 128 * 128 + 3072;
+    int st2 = (int)((227 * 1024 - 2048 - (p.tma_store ? 65536 : 0)) / sb2);
+    if (st2 > 8) st2 = 8;
+    if (st2 < 2 || 256 + 24 * st2 > 512) p.cta2 = 0;
+    else { p.stages = st2; p.n_acc = 1; }
+  }
   p.mma_cp = env_int("MQ_TC_NO_MMA_CP", 0) ? 0 : 1;   // E2M1 too: the bubble behind a copier warp costs more than the lane's extra issues
   p.pair = op == MQ_OP_BWD_DATA && g.sw == 2 && layout == MQ_NCHW && p.Wd % 2 == 0 && p.n_acc == 2 && p.total_tiles % 2 == 0 &&
            !env_int("MQ_TC_NO_PAIR", 0);
@@ -298,8 +311,19 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
     const uint64_t rb = (uint64_t)pl.rowbytes;
     const uint64_t dims[3] = {rb, (uint64_t)taps, (uint64_t)pl.rows_b};
     const uint64_t strides[2] = {rb, (uint64_t)taps * rb};
-    const uint32_t box[3] = {(uint32_t)p.KB, 1u, (uint32_t)p.BN};
+    const uint32_t box[3] = {(uint32_t)p.KB, 1u, (uint32_t)(p.cta2 ? 128 : p.BN)};   // a pair's blocks load half of the weight rows each
     if (!encode_tensor_map_u8(&map_w, b_codes, 3, dims, strides, box, nullptr, p.KB)) return MQ_ERR_CUDA;
+  }
+  CUtensorMap map_sfa = map_a, map_sfb = map_a;
+  if (p.cta2) {   // a pair's scale chunks travel as tiled copies (rows of 256 bytes), so that they can count on the leader's barrier
+    const int spa = p.kind_fp4 ? 2 : 1;
+    const uint64_t tiles_m = (uint64_t)p.tiles_n * p.tiles_h * p.tiles_w * p.classes;
+    const uint64_t rows_a = tiles_m * p.max_stages * 2 * spa;
+    const uint64_t rows_b = (uint64_t)p.classes * p.tiles_c * p.max_stages * 2 * spa * 2;
+    const uint64_t da[2] = {256, rows_a}, db[2] = {256, rows_b}, st[1] = {256};
+    const uint32_t ba[2] = {256u, (uint32_t)(2 * spa)}, bb[2] = {256u, (uint32_t)(2 * spa * 2)};
+    if (!encode_tensor_map_u8(&map_sfa, p.sfa_img, 2, da, st, ba, nullptr, 0)) return MQ_ERR_CUDA;
+    if (!encode_tensor_map_u8(&map_sfb, p.sfb_img, 2, db, st, bb, nullptr, 0)) return MQ_ERR_CUDA;
   }
   CUtensorMap map_out = map_a;
   if (p.tma_store) {
@@ -322,7 +346,7 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
       }
     }
   }
-  return launch_conv_tc(p, map_a, map_w, map_out, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
+  return launch_conv_tc(p, map_a, map_w, map_out, map_sfa, map_sfb, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }
 
 // ---- weight gradient on tensor cores ---------------------------------------------------------------

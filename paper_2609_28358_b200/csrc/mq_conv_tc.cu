@@ -136,11 +136,17 @@ __device__ __forceinline__ int src_w0(const TapWalk<MODE>& w, const ChunkPos& c)
 template <int MODE>
 __device__ __forceinline__ int tap_index(const TapWalk<MODE>& w, const ChunkPos& c) { return w.tap0 + c.ia * w.tap_dh + c.ib * w.tap_dw; }
 
+// An epilogue warp hands its accumulator back: to this block's barrier, or (a pair of blocks: the peer's warps) to the
+// leader's, whose MMA warp waits for the epilogues of both blocks.
+__device__ __forceinline__ void release_acc(uint64_t* bar, int leader_remote) {
+  if (leader_remote) mbar_arrive_remote(bar, 0); else mbar_arrive(bar);
+}
+
 // Epilogue role (warps 4-11): TMEM -> registers -> global (fp32), two warps per TMEM lane quadrant, each
 // taking half of the tile's columns.
 template <int MODE>
 __device__ __forceinline__ void epilogue_role(const ConvTcParams& p, uint32_t tmem, uint64_t* tfull, uint64_t* tempty, volatile int* abort_flag,
-                                              int warp, int lane, unsigned total) {
+                                              int warp, int lane, unsigned total, int leader_remote = 0) {
     const int quad = warp & 3;           // TMEM lane quadrant this warp may read
     const int half = (warp - 4) >> 2;    // warps 4-7 take the first half of the tile's columns, 8-11 the second
     const int r = 32 * quad + lane;
@@ -173,8 +179,9 @@ __device__ __forceinline__ void epilogue_role(const ConvTcParams& p, uint32_t tm
       const bool full_cols = tile.c0 + p.BN <= p.Cd;
       float* o_nchw = p.out + (((long long)n * p.Cd + tile.c0 + cbeg) * p.Hd + yo) * p.Wd + xo;
       float* o_hwnc = p.out + (((long long)yo * p.Wd + xo) * p.N + n) * p.Cd + tile.c0 + cbeg;
-      // one 16-column chunk at a time and no unrolling over chunks: this path serves the layouts the TMA-store
-      // epilogue cannot, and its code size matters more (instruction-cache misses stall every role) than its latency
+      // one 16-column chunk at a time and no unrolling over chunks: its code size matters more (instruction-cache
+      // misses stall every role) than its latency (double-buffering the TMEM loads was measured: no change - the
+      // NCHW stores themselves are the bound)
 #pragma unroll 1
       for (int c = cbeg; c < cend; c += 16) {
         uint32_t v[16];
@@ -205,7 +212,7 @@ __device__ __forceinline__ void epilogue_role(const ConvTcParams& p, uint32_t tm
       }
       tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&tempty[acc]);
+      if (lane == 0) release_acc(&tempty[acc], leader_remote);
     }
     if (lane == 0 && warp == 4) PROF_END(3);
 }
@@ -279,7 +286,8 @@ __device__ __forceinline__ void epilogue_pair_role(const ConvTcParams& p, uint32
 constexpr int EPI_STAGING_BYTES = 8 * 64 * 32 * 4;   // warps x [64 channels][32 rows] floats
 template <int MODE>
 __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const CUtensorMap* map_out, float* staging, uint32_t tmem,
-                                                  uint64_t* tfull, uint64_t* tempty, volatile int* abort_flag, int warp, int lane, unsigned total) {
+                                                  uint64_t* tfull, uint64_t* tempty, volatile int* abort_flag, int warp, int lane, unsigned total,
+                                                  int leader_remote = 0) {
     const int quad = warp & 3;
     const int half = (warp - 4) >> 2;
     const int cbeg = half == 0 ? 0 : ((p.BN / 2 + 15) & ~15);
@@ -306,7 +314,7 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
       if (cbeg >= cend) {      // a tile of 16 channels leaves the second half without columns
         tc_fence_before_sync();
         __syncwarp();
-        if (lane == 0) mbar_arrive(&tempty[acc]);
+        if (lane == 0) release_acc(&tempty[acc], leader_remote);
       }
 #pragma unroll 1
       for (int c0 = cbeg; c0 < cend; c0 += 64) {
@@ -340,7 +348,7 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
         if (c0 + 64 >= cend) {   // the accumulator has been read: hand it back before the store
           tc_fence_before_sync();
           __syncwarp();
-          if (lane == 0) mbar_arrive(&tempty[acc]);
+          if (lane == 0) release_acc(&tempty[acc], leader_remote);
         }
         fence_proxy_async_smem();
         __syncwarp();
@@ -588,6 +596,163 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem, 512);
+}
+
+// ---- the per-tap kernel on PAIRS of blocks (clusters of two, tcgen05 cta_group::2) -------------------------------
+// Tiles 2k and 2k + 1 (neighbours in the tile order: same channel tile, same taps) form one 256-row x 256-channel MMA
+// tile: each block loads the activation boxes of ITS 128 rows and HALF of the weight rows (128 of the 256 channels)
+// plus its scale chunks, all with .cta_group::2 tiled loads that count their bytes on the LEADER's barrier.  The
+// leader's MMA lane issues the scale copies, the MMAs (M = 256) and multicast commits that free the stage and
+// publish the accumulator in both blocks; every block drains its own 128 rows.  Half the weight bytes per block
+// and stage buy six pipeline stages instead of four, and one issuing lane feeds two tensor cores.
+// KB = 128 only (>= 128 bytes of channels per tap), 256-channel tiles, one accumulator, no stride classes.
+template <int MODE, bool FP4>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+conv_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_out,
+                    const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb, const ConvTcParams p) {
+  constexpr int KB = 128;
+  constexpr int SPA = FP4 ? 2 : 1;     // scale bytes per atom
+  constexpr int LAYOUT = 2;
+  constexpr int B_HALF_BYTES = 128 * 128;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+  constexpr int stage_bytes = A_STAGE_BYTES + B_HALF_BYTES + SFA_BYTES + SFB_BYTES;
+  float* staging = reinterpret_cast<float*>(smem + (size_t)p.stages * stage_bytes);   // TMA-store epilogue only
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * stage_bytes + (p.tma_store ? EPI_STAGING_BYTES : 0));
+  uint64_t* empty = full + p.stages;
+  uint64_t* tfull = empty + p.stages;      // [2], one used
+  uint64_t* tempty = tfull + 2;            // [2], one used (the leader's: 16 epilogue warps arrive)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
+  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;   // warp-uniform, see conv_tc_kernel
+  const uint32_t rank = __shfl_sync(0xffffffffu, cluster_ctarank(), 0);                            // 0: leader
+  const unsigned total = (unsigned)p.total_tiles;
+
+  if (threadIdx.x == 0) {
+    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 3); mbar_init(&empty[s], 1); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 16); }
+    *abort_flag = 0;
+    mbar_fence_init();
+    prefetch_tensormap(&map_a);
+    prefetch_tensormap(&map_b);
+    prefetch_tensormap(&map_sfa);
+    prefetch_tensormap(&map_sfb);
+    if (p.tma_store) prefetch_tensormap(&map_out);
+  }
+  if (warp == 1) { tmem_alloc_2(tmem_slot, 512); tmem_relinquish_2(); }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();   // both blocks' barriers and tensor memory exist before anything crosses over
+  tc_fence_after_sync();
+  const uint32_t tmem = *tmem_slot;
+  pdl_wait();
+
+  // loader warps: (kind, parity of the stages it serves), as in conv_tc_kernel
+  const int lkind = (warp == 0 || warp == 12) ? 0 : ((warp == 3 || warp == 13) ? 1 : (warp >= 14 ? 2 : -1));
+  const int lhalf = (warp == 12 || warp == 13 || warp == 15) ? 1 : 0;
+  if (lkind >= 0) {
+    uint32_t s = 0, phase = 0, gi = 0;
+    // the leader announces both blocks' bytes; the peer only issues
+    const uint32_t kind_bytes = 2u * (lkind == 2 ? 512u * SPA * 3u : 128u * KB);
+    for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x) {
+      const Tile tile = decode_tile(p, t);
+      TapWalk<MODE> tw;
+      tw.init(p, tile);
+      const int Q = tw.chunks(p);
+      ChunkPos pos;
+      pos.reset();
+      const int sfa_row0 = (int)(tile_m_index(p, tile) * (unsigned)p.max_stages) * (2 * SPA);                   // rows of 256 bytes
+      const int sfb_row0 = (int)((unsigned)(tile.cls * p.tiles_c + tile.ct) * (unsigned)p.max_stages) * (2 * SPA * 2);
+      for (int q = 0; q < Q; ++q, ++gi) {
+        const bool mine = (gi & 1u) == (uint32_t)lhalf;
+        const int c0 = pos.cc * KB;
+        const int c1 = lkind == 1 ? tap_index(tw, pos) : src_w0(tw, pos);
+        const int c2 = src_h(tw, pos);
+        pos.advance(tw, p.cpt);
+        if (mine) {
+          uint8_t* sa = smem + (size_t)s * stage_bytes;
+          uint8_t* sb = sa + A_STAGE_BYTES;
+          const uint32_t lbar = cluster_addr_of(&full[s], 0);
+          if (!mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+          if (elect_one()) {
+            if (rank == 0) mbar_arrive_expect_tx(&full[s], kind_bytes);
+            if (lkind == 2) {
+              tma_load_2d_pair(sb + B_HALF_BYTES, &map_sfa, lbar, 0, sfa_row0 + q * (2 * SPA));
+              tma_load_2d_pair(sb + B_HALF_BYTES + SFA_BYTES, &map_sfb, lbar, 0, sfb_row0 + q * (2 * SPA * 2));
+            } else if (lkind == 1) {
+              tma_load_3d_pair(sb, &map_b, lbar, c0, c1, tile.c0 + 128 * (int)rank);
+            } else {
+              tma_load_4d_pair(sa, &map_a, lbar, c0, c1, tile.n0, c2);
+            }
+          }
+          __syncwarp();
+        }
+        if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer (the leader's)
+    if (rank == 0) {
+      const uint64_t op_desc = smem_desc_base(16, 8 * KB, LAYOUT);
+      const uint32_t sf_base = tmem + (uint32_t)p.BN;
+      constexpr uint32_t stage16 = (uint32_t)stage_bytes >> 4;
+      const uint64_t a_desc0 = smem_desc(op_desc, smem_u32(smem));
+      const uint64_t b_desc0 = smem_desc(op_desc, smem_u32(smem + A_STAGE_BYTES));
+      const uint64_t sf_desc = smem_desc_base(0, 128, 0);
+      const uint64_t sfa_desc0 = smem_desc(sf_desc, smem_u32(smem + A_STAGE_BYTES + B_HALF_BYTES));
+      const uint64_t sfb_desc0 = smem_desc(sf_desc, smem_u32(smem + A_STAGE_BYTES + B_HALF_BYTES + SFA_BYTES));
+      const uint32_t idesc = (p.idesc & ~(0x1Fu << 24)) | ((256u >> 4) << 24);   // M = 256 over the pair
+      uint32_t s = 0, phase = 0, tcount = 0;
+      for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
+        const Tile tile = decode_tile(p, t);
+        TapWalk<MODE> tw;
+        tw.init(p, tile);
+        const int Q = tw.chunks(p);
+        if (!mbar_wait(&tempty[0], (tcount & 1) ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+        tc_fence_after_sync();
+        uint32_t accumulate = 0;
+        for (int q = 0; q < Q; ++q) {
+          if (!mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+          tc_fence_after_sync();
+          const uint32_t so = s * stage16;
+          const uint32_t sfa_t = sf_base + s * SF_COLS, sfb_t = sfa_t + 8;
+          if (elect_one()) {
+#pragma unroll
+            for (int g = 0; g < SPA; ++g) {
+              tmem_cp_32x128b_warpx4_2(sfa_t + 4 * g, sfa_desc0 + so + g * 32);
+              tmem_cp_32x128b_warpx4_2(sfb_t + 8 * g, sfb_desc0 + so + g * 64);
+              tmem_cp_32x128b_warpx4_2(sfb_t + 8 * g + 4, sfb_desc0 + so + g * 64 + 32);
+            }
+            uint32_t accu = accumulate;
+#pragma unroll
+            for (int a = 0; a < 4; ++a) {
+              const uint64_t ad = a_desc0 + so + a * 2;
+              const uint64_t bd = b_desc0 + so + a * 2;
+              const int g = (a * SPA) >> 2, id = (a * SPA) & 3;
+              const uint32_t idd = idesc_with_sf_ids(idesc, id, id);
+              if (FP4) mma_mxf4_2(tmem, ad, bd, idd, sfa_t + 4 * g, sfb_t + 8 * g, accu);
+              else mma_mxf8f6f4_2(tmem, ad, bd, idd, sfa_t + 4 * g, sfb_t + 8 * g, accu);
+              accu = 1;
+            }
+            tc_commit_2_multicast(&empty[s], 3);   // frees the stage in both blocks
+          }
+          __syncwarp();
+          accumulate = 1;
+          if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
+        }
+        if (elect_one()) { if (Q > 0) tc_commit_2_multicast(&tfull[0], 3); else { mbar_arrive(&tfull[0]); mbar_arrive_remote(&tfull[0], 1); } }
+        __syncwarp();
+      }
+    }
+  } else if (warp >= 4 && warp < 12) {
+    if (p.tma_store) epilogue_tma_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total, (int)rank);
+    else epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total, (int)rank);
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();   // nothing of the peer block is touched after this point
+  if (warp == 1) tmem_dealloc_2(tmem, 512);
 }
 
 template <int BPC>
@@ -1255,8 +1420,40 @@ cudaError_t launch_conv_tc_halo_inst(const ConvTcParams& p, const CUtensorMap& m
   return launch_conv_tc_halo_taps<MODE, KB, FP4, 0>(p, map_a, map_b, map_w, s);
 }
 
-cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_out, cudaStream_t s) {
+size_t conv_tc_pair_smem_bytes(const ConvTcParams& p) {
+  const size_t stage = A_STAGE_BYTES + 128 * 128 + SFA_BYTES + SFB_BYTES;
+  return 1024 + (size_t)p.stages * stage + (p.tma_store ? EPI_STAGING_BYTES : 0) + (2 * (size_t)p.stages + 4) * 8 + 64;
+}
+template <int MODE, bool FP4>
+cudaError_t launch_conv_tc_pair_inst(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_out, const CUtensorMap& map_sfa,
+                                     const CUtensorMap& map_sfb, cudaStream_t s) {
+  static bool attr_set = false;
+  const size_t smem = conv_tc_pair_smem_bytes(p);
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(conv_tc_pair_kernel<MODE, FP4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  int dev = 0, sms = 148;
+  cudaGetDevice(&dev);
+  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  unsigned grid = (unsigned)(p.total_tiles < sms ? p.total_tiles : sms);
+  grid &= ~1u;   // whole pairs (the tile count is even in this mode)
+  if (grid < 2) return cudaErrorInvalidValue;
+  count_launches(1);
+  return launch_pdl_cluster(conv_tc_pair_kernel<MODE, FP4>, dim3(grid), dim3(TC_THREADS), smem, s, 2u, map_a, map_b, map_out, map_sfa, map_sfb, p);
+}
+
+cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_out, const CUtensorMap& map_sfa,
+                           const CUtensorMap& map_sfb, cudaStream_t s) {
   if (p.total_tiles <= 0 || p.total_tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
+  if (p.cta2) {
+    const bool f4 = p.kind_fp4 != 0;
+    if (p.mode == MQ_OP_FWD) return f4 ? launch_conv_tc_pair_inst<MQ_OP_FWD, true>(p, map_a, map_w, map_out, map_sfa, map_sfb, s)
+                                       : launch_conv_tc_pair_inst<MQ_OP_FWD, false>(p, map_a, map_w, map_out, map_sfa, map_sfb, s);
+    return f4 ? launch_conv_tc_pair_inst<MQ_OP_BWD_DATA, true>(p, map_a, map_w, map_out, map_sfa, map_sfb, s)
+              : launch_conv_tc_pair_inst<MQ_OP_BWD_DATA, false>(p, map_a, map_w, map_out, map_sfa, map_sfb, s);
+  }
   if (p.halo) {
 #define MQ_TC_HCASE(M, K, F) if (p.mode == M && p.KB == K && (p.kind_fp4 != 0) == F) return launch_conv_tc_halo_inst<M, K, F>(p, map_a, map_out, map_w, s)
     MQ_TC_HCASE(MQ_OP_FWD, 64, false); MQ_TC_HCASE(MQ_OP_FWD, 32, false); MQ_TC_HCASE(MQ_OP_FWD, 64, true); MQ_TC_HCASE(MQ_OP_FWD, 32, true);

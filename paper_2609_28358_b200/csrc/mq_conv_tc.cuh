@@ -52,6 +52,7 @@ struct ConvTcParams {
   int fused;                // 1: single channel tile, stride 1: no preparation kernel (the blocks build the weight image, its
                             //    scale chunks and every tile's activation scale chunks themselves)
   int mma_cp;             // E2M1: 1 = the MMA lane issues the scale copies itself (no copier warp)
+  int cta2;               // 1: pairs of blocks (clusters of 2) on 256-row x 256-channel tiles, conv_tc_pair_kernel
   int pair;                 // per-tap kernel, input gradient with column stride 2, NCHW output: see tile_of_iter
   int tma_store;            // 1: NCHW output written by TMA stores from per-warp staging slices
   const uint8_t* b_codes;   // weight-like codes [rows][taps][b_rowbytes] (source of the images below)
@@ -66,7 +67,8 @@ struct ConvTcParams {
 // map_a: gathered activation codes.  map_w: weight codes, one tap per box (per-tap kernel) or all taps of a tile in one
 // box (whole-tile kernel with fused preparation).  map_out: the fp32 NCHW output seen as (W, N, C, H), used when
 // p.tma_store is set.
-cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_out, cudaStream_t s);
+cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_out, const CUtensorMap& map_sfa,
+                           const CUtensorMap& map_sfb, cudaStream_t s);
 // Expands the compact tile scales into the per-stage scale-vector chunks the MMA reads (p.sfa_img, p.sfb_img).
 cudaError_t launch_expand_conv_scales(const ConvTcParams& p, cudaStream_t s);
 size_t conv_tc_sfa_bytes(const ConvTcParams& p);

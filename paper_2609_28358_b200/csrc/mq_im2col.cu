@@ -42,21 +42,31 @@ __global__ void __launch_bounds__(IC_THREADS) im2col_kernel(Im2colArgs a, int rc
     const int total = rows * J;
     const uint4* src = reinterpret_cast<const uint4*>(a.codes) + (long long)n0 * rc;
     const int dn = IC_THREADS / J, dj = IC_THREADS - dn * J;
+    uint4* dst0 = reinterpret_cast<uint4*>(a.out_codes) + ((long long)pix0 * g.N + n0) * J;
+    const long long px_stride = (long long)g.N * J;      // chunks between the rows of consecutive pixels
+    // chunk i = n * J + j of every pixel of the block, advanced by IC_THREADS per step without divisions; the loads of
+    // four pixels are issued before their stores (the kernel waits on L2 latency, not on bandwidth)
+    int n = threadIdx.x / J, j = threadIdx.x - n * J;
 #pragma unroll 1
-    for (int px = 0; px < px_n; ++px) {
-      const int* so_px = soff + px * J;
-      uint4* dst = reinterpret_cast<uint4*>(a.out_codes) + ((long long)(pix0 + px) * g.N + n0) * J;
-      // chunk i = n * J + j, advanced by IC_THREADS per step without divisions
-      int n = threadIdx.x / J, j = threadIdx.x - n * J;
-#pragma unroll 2
-      for (int i = threadIdx.x; i < total; i += IC_THREADS) {
-        const int so = so_px[j];
-        uint4 v = make_uint4(0, 0, 0, 0);
-        if (so >= 0) v = __ldg(src + so + n * rc);
-        __stcs(dst + i, v);
-        n += dn; j += dj;
-        if (j >= J) { j -= J; ++n; }
+    for (int i = threadIdx.x; i < total; i += IC_THREADS) {
+      const uint4* s_n = src + n * rc;
+#pragma unroll 1
+      for (int px0 = 0; px0 < px_n; px0 += 4) {
+        uint4 v[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+          v[q] = make_uint4(0, 0, 0, 0);
+          if (px0 + q < px_n) {
+            const int so = soff[(px0 + q) * J + j];
+            if (so >= 0) v[q] = __ldg(s_n + so);
+          }
+        }
+#pragma unroll
+        for (int q = 0; q < 4; ++q)
+          if (px0 + q < px_n) __stcs(dst0 + (px0 + q) * px_stride + i, v[q]);
       }
+      n += dn; j += dj;
+      if (j >= J) { j -= J; ++n; }
     }
   } else {
     // scales [ho][wo][nt][kh][kw][ct]
