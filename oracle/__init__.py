@@ -7,7 +7,7 @@ library and its Python binding never do, and nothing here imports them.
 All arrays are host numpy arrays.  Conventions (Sec. II-A, IV-A, IV-B of the paper):
   * ``desc`` = ConvDesc(N, C_in, H, W, C_out, Kh, Kw, stride_h, stride_w, pad_h, pad_w)
   * roles: X (activations, NCHW), W (weights, OIHW), DY (output gradient, N.Cout.Ho.Wo)
-  * element formats: E4M3, E5M2 (one byte per code), E2M1 (two codes per byte, lower index in
+  * element formats: E4M3, E5M2, E3M2, E2M3 (one byte per code), E2M1 (two codes per byte, lower index in
     the low nibble); block scale E8M0
   * block shape (br, bc): br along N (X, DY) or Cout (W); bc along the channel axis that is
     stored fastest.  (32, 32) is the square block, (1, 32) the line block.
@@ -21,10 +21,10 @@ from collections import namedtuple
 
 import numpy as np
 
-E4M3, E5M2, E2M1 = 0, 1, 2
+E4M3, E5M2, E2M1, E3M2, E2M3 = 0, 1, 2, 3, 4
 ROLE_X, ROLE_W, ROLE_DY = 0, 1, 2
-FMT_BITS = {E4M3: 8, E5M2: 8, E2M1: 4}
-FMT_EMAX = {E4M3: 8, E5M2: 15, E2M1: 2}
+FMT_BITS = {E4M3: 8, E5M2: 8, E2M1: 4, E3M2: 8, E2M3: 8}   # stored bits per code (6-bit codes: one per byte)
+FMT_EMAX = {E4M3: 8, E5M2: 15, E2M1: 2, E3M2: 4, E2M3: 2}
 
 ConvDesc = namedtuple("ConvDesc", "N C_in H W C_out Kh Kw stride_h stride_w pad_h pad_w")
 

@@ -18,7 +18,7 @@
 //
 // Readings of the paper taken here (the paper is silent or uses another variant):
 //  * block scale is E8M0 (the "original microscaling format", Sec. II-D) with the OCP floor
-//    rule, no per-tensor scale; elements E2M1 / E4M3 / E5M2, round-to-nearest-even, saturating;
+//    rule, no per-tensor scale; elements E2M1 / E4M3 / E5M2 / E3M2 / E2M3, round-to-nearest-even, saturating;
 //  * a quantization block is a br x bc rectangle over the two axes Sec. IV-B names for each
 //    tensor (X: N x Cin, W: Cout x Cin, G_Y: N x Cout) at one spatial / tap position;
 //    32 x 32 is the square of Sec. IV-B with sqrt(B) = 32, 1 x 32 is the line block of Sec. III-A;
@@ -46,16 +46,20 @@ Conv conv_from(const int* d) {
   return c;
 }
 
-enum Fmt { E4M3 = 0, E5M2 = 1, E2M1 = 2 };
+enum Fmt { E4M3 = 0, E5M2 = 1, E2M1 = 2, E3M2 = 3, E2M3 = 4 };
 enum Role { ROLE_X = 0, ROLE_W = 1, ROLE_DY = 2 };
 
 // ---- element formats (OCP MX v1.0 / OFP8 definitions cited in Sec. II-D) -------------------
-struct FmtInfo { int ebits, mbits, bias, emax, max_code, bits; };
+// bits: width of a code, sign included; store_bits: bits a code occupies in the stored tensor (the 6-bit formats of
+// MicroQonv+ / "-6", Sec. V, are kept one code per byte, value in the low six bits)
+struct FmtInfo { int ebits, mbits, bias, emax, max_code, bits, store_bits; };
 FmtInfo fmt_info(int fmt) {
   switch (fmt) {
-    case E4M3: return {4, 3, 7, 8, 0x7E, 8};    // no Inf; S.1111.111 is NaN; max 448
-    case E5M2: return {5, 2, 15, 15, 0x7B, 8};  // IEEE-like: 0x7C Inf, 0x7D..0x7F NaN; max 57344
-    default:   return {2, 1, 1, 2, 0x7, 4};     // E2M1: no Inf/NaN; max 6
+    case E4M3: return {4, 3, 7, 8, 0x7E, 8, 8};    // no Inf; S.1111.111 is NaN; max 448
+    case E5M2: return {5, 2, 15, 15, 0x7B, 8, 8};  // IEEE-like: 0x7C Inf, 0x7D..0x7F NaN; max 57344
+    case E3M2: return {3, 2, 3, 4, 0x1F, 6, 8};    // no Inf/NaN; max 1.75 * 2^4 = 28
+    case E2M3: return {2, 3, 1, 2, 0x1F, 6, 8};    // no Inf/NaN; max 1.875 * 2^2 = 7.5
+    default:   return {2, 1, 1, 2, 0x7, 4, 4};     // E2M1: no Inf/NaN; max 6
   }
 }
 
@@ -183,7 +187,7 @@ int orc_qtensor_sizes(const int* d, int role, int fmt, int br, int bc, int64_t* 
   Conv c = conv_from(d);
   View v = view_of(c, role);
   int64_t elems = (int64_t)v.P * v.R * v.Cp;
-  *codes_bytes = elems * fmt_info(fmt).bits / 8;
+  *codes_bytes = elems * fmt_info(fmt).store_bits / 8;
   *scales_bytes = (int64_t)v.P * ((v.R + br - 1) / br) * (v.Cp / bc);
   return 0;
 }
@@ -245,7 +249,7 @@ int orc_im2col_sizes(const int* d, int fmt, int br, int bc, int64_t* codes_bytes
   Conv c = conv_from(d);
   int Cp = (c.Cin + 31) / 32 * 32;
   int64_t rows = (int64_t)c.Ho() * c.Wo() * c.N;
-  *codes_bytes = rows * c.Kh * c.Kw * Cp * fmt_info(fmt).bits / 8;
+  *codes_bytes = rows * c.Kh * c.Kw * Cp * fmt_info(fmt).store_bits / 8;
   *scales_bytes = (int64_t)c.Ho() * c.Wo() * ((c.N + br - 1) / br) * c.Kh * c.Kw * (Cp / bc);
   return 0;
 }

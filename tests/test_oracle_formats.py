@@ -12,10 +12,10 @@ import pytest
 import torch
 
 import oracle
-from oracle import E2M1, E4M3, E5M2
+from oracle import E2M1, E2M3, E3M2, E4M3, E5M2
 
 GOLD = os.path.join(os.path.dirname(__file__), "golden")
-FMT = {"E4M3": E4M3, "E5M2": E5M2, "E2M1": E2M1}
+FMT = {"E4M3": E4M3, "E5M2": E5M2, "E2M1": E2M1, "E3M2": E3M2, "E2M3": E2M3}
 
 
 def test_e2m1_decode_grid():
@@ -24,6 +24,37 @@ def test_e2m1_decode_grid():
         assert oracle.decode_elem(E2M1, c) == grid[c]
         assert oracle.decode_elem(E2M1, c | 8) == -grid[c]
     assert math.copysign(1.0, oracle.decode_elem(E2M1, 8)) == -1.0  # 0x8 is -0
+
+
+def test_fp6_decode_grids():
+    """The 6-bit element formats of the OCP MX definition (the activations of MicroQonv+ and the "-6" variant,
+    Sec. V), written out as explicit value grids: E3M2 bias 3 (subnormal step 2^-4, largest 28), E2M3 bias 1
+    (subnormal step 2^-3, largest 7.5); no infinities or NaNs; the sign is bit 5."""
+    e3m2 = [0.0, 0.0625, 0.125, 0.1875] + [(1 + m / 4) * 2.0 ** (e - 3) for e in range(1, 8) for m in range(4)]
+    e2m3 = [k * 0.125 for k in range(8)] + [(1 + m / 8) * 2.0 ** (e - 1) for e in range(1, 4) for m in range(8)]
+    assert len(e3m2) == 32 and len(e2m3) == 32
+    assert e3m2[4] == 0.25 and e3m2[31] == 28.0 and e3m2[1] == 2.0 ** -4     # smallest normal, largest, smallest subnormal
+    assert e2m3[8] == 1.0 and e2m3[31] == 7.5 and e2m3[1] == 2.0 ** -3
+    for fmt, grid in ((E3M2, e3m2), (E2M3, e2m3)):
+        for c in range(32):
+            assert oracle.decode_elem(fmt, c) == grid[c], (fmt, c)
+            assert oracle.decode_elem(fmt, c | 32) == -grid[c]
+        assert math.copysign(1.0, oracle.decode_elem(fmt, 32)) == -1.0
+        assert all(math.isfinite(oracle.decode_elem(fmt, c)) for c in range(64))
+
+
+def test_fp6_encode_explicit_cases():
+    # ties go to the code with an even low bit; magnitudes beyond the largest value saturate
+    cases = {
+        E2M3: [(1.0, 0x08), (1.0625, 0x08), (1.07, 0x09), (1.1875, 0x0A), (7.5, 0x1F), (7.75, 0x1F), (1e9, 0x1F), (0.0625, 0x00), (0.07, 0x01),
+               (0.1875, 0x02), (3.75, 0x17), (3.875, 0x18)],
+        E3M2: [(0.25, 0x04), (0.03125, 0x00), (0.04, 0x01), (0.09375, 0x02), (24.0, 0x1E), (26.0, 0x1E), (26.1, 0x1F), (28.0, 0x1F), (40.0, 0x1F),
+               (1.125, 0x0C), (1.126, 0x0D), (1.375, 0x0E)],
+    }
+    for fmt, rows in cases.items():
+        for v, code in rows:
+            assert oracle.encode_elem(fmt, v) == code, (fmt, v)
+            assert oracle.encode_elem(fmt, -v) == code | 32, (fmt, v)
 
 
 @pytest.mark.parametrize("fmt,tdtype", [(E4M3, torch.float8_e4m3fn), (E5M2, torch.float8_e5m2)])
@@ -48,7 +79,7 @@ def test_fp8_landmarks():
     assert math.isinf(oracle.decode_elem(E5M2, 0x7C))
 
 
-@pytest.mark.parametrize("fmt,ncodes,maxc", [(E2M1, 16, 0x7), (E4M3, 256, 0x7E), (E5M2, 256, 0x7B)])
+@pytest.mark.parametrize("fmt,ncodes,maxc", [(E2M1, 16, 0x7), (E4M3, 256, 0x7E), (E5M2, 256, 0x7B), (E3M2, 64, 0x1F), (E2M3, 64, 0x1F)])
 def test_encode_roundtrip_midpoints_saturation(fmt, ncodes, maxc):
     half = ncodes // 2
     for m in range(maxc + 1):
@@ -94,7 +125,7 @@ def test_fp8_encode_matches_library_cast(fmt, tdtype, top):
         assert oracle.encode_elem(fmt, float(x)) == int(c), (x, c)
 
 
-@pytest.mark.parametrize("fmt,emax", [(E2M1, 2), (E4M3, 8), (E5M2, 15)])
+@pytest.mark.parametrize("fmt,emax", [(E2M1, 2), (E4M3, 8), (E5M2, 15), (E3M2, 4), (E2M3, 2)])
 def test_scale_closed_form(fmt, emax):
     assert oracle.scale_code(fmt, 0.0) == 0
     for k in range(-140, 128):
