@@ -29,8 +29,8 @@ import numpy as np  # noqa: E402
 from paper_2609_28358_b200 import inputs  # noqa: E402
 
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
-FMT_NAME = {0: "e4m3", 1: "e5m2", 2: "e2m1"}
-FMT_BITS = {0: 8, 1: 8, 2: 4}
+FMT_NAME = {0: "e4m3", 1: "e5m2", 2: "e2m1", 3: "e3m2", 4: "e2m3"}
+FMT_BITS = {0: 8, 1: 8, 2: 4, 3: 8, 4: 8}   # stored bits per code (the 6-bit formats sit one per byte and run at the 8-bit tensor rate)
 # nominal dense tensor-core ratio to bf16 for the operand formats of a GEMM
 TENSOR_RATIO = {8: 2.0, 4: 4.0}
 
@@ -59,6 +59,8 @@ def workloads():
         w[l.name] = l
     for l in inputs.config3():
         w["cfg3_" + l.name] = l
+    for l in inputs.fp6_layers():
+        w[l.name] = l
     return w
 
 

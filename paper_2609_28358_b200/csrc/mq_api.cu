@@ -14,7 +14,7 @@ void count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::me
 
 namespace {
 
-bool valid_fmt(int f) { return f == MQ_E4M3 || f == MQ_E5M2 || f == MQ_E2M1; }
+bool valid_fmt(int f) { return f == MQ_E4M3 || f == MQ_E5M2 || f == MQ_E2M1 || f == MQ_E3M2 || f == MQ_E2M3; }
 bool valid_role(int r) { return r == MQ_ROLE_X || r == MQ_ROLE_W || r == MQ_ROLE_DY; }
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -67,6 +67,9 @@ bool conv_tc_eligible(int op, const Geom& g, int fmt_x_like, int fmt_w) {
   const bool fp4 = fmt_x_like == MQ_E2M1 && fmt_w == MQ_E2M1;
   const bool fp8 = fmt_x_like != MQ_E2M1 && fmt_w != MQ_E2M1;
   if (!fp4 && !fp8) return false;
+  // 6-bit operands: the tensor core reads them as 16 codes packed into 12 bytes + 4 bytes of padding, not one code per
+  // byte as they are stored here; they run on the CUDA-core kernels
+  if (fmt_is_6bit(fmt_x_like) || fmt_is_6bit(fmt_w)) return false;
   const int Kp = op == MQ_OP_FWD ? g.Cp : g.Cop;
   const int rowbytes = Kp * (fp4 ? 4 : 8) / 8;
   return rowbytes % 32 == 0;
@@ -212,8 +215,8 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
            !env_int("MQ_TC_NO_PAIR", 0);
   const int nkh = op == MQ_OP_FWD ? g.Kh : (g.Kh + g.sh - 1) / g.sh, nkw = op == MQ_OP_FWD ? g.Kw : (g.Kw + g.sw - 1) / g.sw;
   p.max_stages = (nkh * nkw * p.cpt + p.G - 1) / p.G;
-  const uint32_t fa = fp4 ? 1u : (fmt_x_like == MQ_E5M2 ? 1u : 0u);
-  const uint32_t fb = fp4 ? 1u : (fmt_w == MQ_E5M2 ? 1u : 0u);
+  const uint32_t fa = fp4 ? 1u : fmt_mma_code(fmt_x_like);   // kind::mxf4: 1 = E2M1; kind::mxf8f6f4: E4M3 0, E5M2 1, E2M3 3, E3M2 4
+  const uint32_t fb = fp4 ? 1u : fmt_mma_code(fmt_w);
   p.idesc = (fa << 7) | (fb << 10) | ((uint32_t)(p.BN >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
   // whole-tile-per-stage variant: stride 1, one chunk per tap (<= 64 bytes of channels).  One box with the column
   // halo needs 8-column tiles; one box per column shift takes 8, 16 or 32 columns (longer NCHW store runs).
@@ -364,6 +367,7 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   const bool fp4 = fmt_x == MQ_E2M1 && fmt_g == MQ_E2M1;
   const bool fp8 = fmt_x != MQ_E2M1 && fmt_g != MQ_E2M1;
   if (!fp4 && !fp8) return w;
+  if (fmt_is_6bit(fmt_x) || fmt_is_6bit(fmt_g)) return w;   // see conv_tc_eligible
   WgradTcParams& p = w.p;
   p.N = g.N; p.Nt = g.Nt; p.Ho = g.Ho; p.Wo = g.Wo; p.H = g.H; p.W = g.W; p.Cout = g.Cout; p.Cp = g.Cp; p.Ct = g.Ct; p.Cot = g.Cot;
   p.Kh = g.Kh; p.Kw = g.Kw; p.sh = g.sh; p.sw = g.sw; p.ph = g.ph; p.pw = g.pw;
@@ -465,7 +469,7 @@ mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const 
       if (!encode_tensor_map_u8(&map_b, xt, 4, dims, strides, box, nullptr, swz)) return MQ_ERR_CUDA;
     }
   } else {
-    const uint32_t fa = qg->fmt == MQ_E5M2 ? 1u : 0u, fb = qx->fmt == MQ_E5M2 ? 1u : 0u;
+    const uint32_t fa = fmt_mma_code(qg->fmt), fb = fmt_mma_code(qx->fmt);
     p.idesc = (fa << 7) | (fb << 10) | (1u << 15) | (1u << 16) | (1u << 23) | (((p.cta2 ? 256u : 128u) >> 4) << 24);
     {
       const uint64_t rb = (uint64_t)g.Cop;

@@ -74,11 +74,11 @@ __global__ void __launch_bounds__(GT) fwd_generic(ConvArgs a) {
       float va[8], vb[8];
       if (pix_ok) {
         float s = e8m0_to_float(a.a_scales[(pix * g.Nt + (n >> 5)) * g.Ct + kb]);
-        decode8<FX>(a.a_codes, (pix * g.N + n) * g.Cp + kb * 32 + kq * 8, s, va);
+        decode8<FX>(a.a_codes, (pix * g.N + n) * g.Cp + kb * 32 + kq * 8, s, va, a.fmt_a);
       } else zero8(va);
       if (co_ok) {
         float s = e8m0_to_float(a.b_scales[((long long)(co >> 5) * taps + tap) * g.Ct + kb]);
-        decode8<FW>(a.b_codes, ((long long)co * taps + tap) * g.Cp + kb * 32 + kq * 8, s, vb);
+        decode8<FW>(a.b_codes, ((long long)co * taps + tap) * g.Cp + kb * 32 + kq * 8, s, vb, a.fmt_b);
       } else zero8(vb);
       __syncthreads();
       store_kmajor(sm.As, row_l, kq, va);
@@ -135,12 +135,12 @@ __global__ void __launch_bounds__(GT) bwd_data_generic(ConvArgs a) {
       float va[8], vb[8];
       if (pix_ok) {
         float s = e8m0_to_float(a.b_scales[(pix * g.Nt + (n >> 5)) * g.Cot + kb]);
-        decode8<FG>(a.b_codes, (pix * g.N + n) * g.Cop + kb * 32 + kq * 8, s, va);
+        decode8<FG>(a.b_codes, (pix * g.N + n) * g.Cop + kb * 32 + kq * 8, s, va, a.fmt_b);
       } else zero8(va);
       const int co = kb * 32 + k_l;
       if (ci_ok && co < g.Cout) {
         float s = e8m0_to_float(a.a_scales[((long long)kb * taps + tap) * g.Ct + (ci0 >> 5)]);
-        decode8<FW>(a.a_codes, ((long long)co * taps + tap) * g.Cp + ci0, s, vb);
+        decode8<FW>(a.a_codes, ((long long)co * taps + tap) * g.Cp + ci0, s, vb, a.fmt_a);
       } else zero8(vb);
       __syncthreads();
       store_kmajor(sm.As, row_l, kq, va);
@@ -199,11 +199,11 @@ __global__ void __launch_bounds__(GT) bwd_weight_generic(ConvArgs a, int splits)
       float va[8], vb[8];
       if (co_ok && n < g.N) {
         float s = e8m0_to_float(a.b_scales[((long long)pix * g.Nt + kb) * g.Cot + (co0 >> 5)]);
-        decode8<FG>(a.b_codes, ((long long)pix * g.N + n) * g.Cop + co0, s, va);
+        decode8<FG>(a.b_codes, ((long long)pix * g.N + n) * g.Cop + co0, s, va, a.fmt_b);
       } else zero8(va);
       if (x_ok && n < g.N) {
         float s = e8m0_to_float(a.a_scales[(xpix * g.Nt + kb) * g.Ct + (ci0 >> 5)]);
-        decode8<FX>(a.a_codes, (xpix * g.N + n) * g.Cp + ci0, s, vb);
+        decode8<FX>(a.a_codes, (xpix * g.N + n) * g.Cp + ci0, s, vb, a.fmt_a);
       } else zero8(vb);
       __syncthreads();
       store_mnmajor(sm.As, k_l, q8, va);
@@ -295,17 +295,13 @@ cudaError_t launch_bwd_weight_reduce(const float* partial, float* out, const Geo
   return launch_pdl(bwd_weight_reduce, dim3(blocks), dim3(256), 0, s, partial, out, g, splits, layout);
 }
 
+// Two template classes per operand: packed E2M1 (2) or one byte per code (0; the format itself is read at run time)
 #define MQ_DISPATCH2(FA, FB, CALL)                                                         \
-  switch ((FA) * 3 + (FB)) {                                                               \
+  switch (((FA) == MQ_E2M1 ? 2 : 0) + ((FB) == MQ_E2M1 ? 1 : 0)) {                            \
     case 0: { constexpr int A_ = 0, B_ = 0; CALL; } break;                                 \
-    case 1: { constexpr int A_ = 0, B_ = 1; CALL; } break;                                 \
-    case 2: { constexpr int A_ = 0, B_ = 2; CALL; } break;                                 \
-    case 3: { constexpr int A_ = 1, B_ = 0; CALL; } break;                                 \
-    case 4: { constexpr int A_ = 1, B_ = 1; CALL; } break;                                 \
-    case 5: { constexpr int A_ = 1, B_ = 2; CALL; } break;                                 \
-    case 6: { constexpr int A_ = 2, B_ = 0; CALL; } break;                                 \
-    case 7: { constexpr int A_ = 2, B_ = 1; CALL; } break;                                 \
-    case 8: { constexpr int A_ = 2, B_ = 2; CALL; } break;                                 \
+    case 1: { constexpr int A_ = 0, B_ = 2; CALL; } break;                                 \
+    case 2: { constexpr int A_ = 2, B_ = 0; CALL; } break;                                 \
+    case 3: { constexpr int A_ = 2, B_ = 2; CALL; } break;                                 \
     default: return cudaErrorInvalidValue;                                                 \
   }
 

@@ -5,6 +5,7 @@
 #include <cuda_fp16.h>
 #include <cuda_fp8.h>
 #include <cuda_fp4.h>
+#include <cuda_fp6.h>
 #include <stdint.h>
 
 #include "mq.h"
@@ -35,7 +36,10 @@ inline Geom make_geom(const mq_conv_desc& d) {
 }
 
 __host__ __device__ inline int fmt_bits(int fmt) { return fmt == MQ_E2M1 ? 4 : 8; }
-__host__ __device__ inline int fmt_emax(int fmt) { return fmt == MQ_E4M3 ? 8 : (fmt == MQ_E5M2 ? 15 : 2); }
+__host__ __device__ inline int fmt_emax(int fmt) { return fmt == MQ_E4M3 ? 8 : (fmt == MQ_E5M2 ? 15 : (fmt == MQ_E3M2 ? 4 : 2)); }
+__host__ __device__ inline bool fmt_is_6bit(int fmt) { return fmt == MQ_E3M2 || fmt == MQ_E2M3; }
+// format field of the tcgen05 instruction descriptor (kind::mxf8f6f4)
+__host__ __device__ inline unsigned fmt_mma_code(int fmt) { return fmt == MQ_E4M3 ? 0u : (fmt == MQ_E5M2 ? 1u : (fmt == MQ_E2M3 ? 3u : (fmt == MQ_E3M2 ? 4u : 5u))); }
 
 // Number of kernels the library has launched in this process (diagnostic; see mq_kernel_launch_count).
 void count_launches(int n);
@@ -92,7 +96,8 @@ __device__ __forceinline__ float e8m0_to_float(unsigned code) {
 
 // Exact decode of 8 consecutive codes (K- or MN-contiguous in memory) to fp32, times `scale`.
 template <int FMT>
-__device__ __forceinline__ void decode8(const uint8_t* codes_base, long long elem_off, float scale, float* out) {
+__device__ __forceinline__ void decode8(const uint8_t* codes_base, long long elem_off, float scale, float* out, int fmt8 = FMT) {
+  // FMT: MQ_E2M1 (packed nibbles) or any other value for the one-byte-per-code formats, whose actual format is fmt8
   if (FMT == MQ_E2M1) {
     uint32_t v = *reinterpret_cast<const uint32_t*>(codes_base + (elem_off >> 1));
 #pragma unroll
@@ -108,7 +113,11 @@ __device__ __forceinline__ void decode8(const uint8_t* codes_base, long long ele
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
       unsigned short pair = (unsigned short)((w[i >> 1] >> (16 * (i & 1))) & 0xFFFF);
-      __half2_raw h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)pair, FMT == MQ_E4M3 ? __NV_E4M3 : __NV_E5M2);
+      __half2_raw h;
+      if (fmt8 == MQ_E4M3) h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)pair, __NV_E4M3);
+      else if (fmt8 == MQ_E5M2) h = __nv_cvt_fp8x2_to_halfraw2((__nv_fp8x2_storage_t)pair, __NV_E5M2);
+      else if (fmt8 == MQ_E3M2) h = __nv_cvt_fp6x2_to_halfraw2((__nv_fp6x2_storage_t)pair, __NV_E3M2);
+      else h = __nv_cvt_fp6x2_to_halfraw2((__nv_fp6x2_storage_t)pair, __NV_E2M3);
       float2 f = __half22float2(*reinterpret_cast<__half2*>(&h));
       out[2 * i] = f.x * scale;
       out[2 * i + 1] = f.y * scale;

@@ -31,6 +31,9 @@ __device__ __forceinline__ unsigned encode2(float lo, float hi) {
   // two elements -> two codes (lo in the low byte / nibble), round-to-nearest-even, saturating
   if (FMT == MQ_E2M1) {
     return (unsigned)__nv_cvt_float2_to_fp4x2(make_float2(lo, hi), __NV_E2M1, cudaRoundNearest);
+  } else if (FMT == MQ_E3M2 || FMT == MQ_E2M3) {
+    // two 6-bit codes, each in the low six bits of its byte (the container the tensor core reads)
+    return (unsigned)__nv_cvt_float2_to_fp6x2(make_float2(lo, hi), FMT == MQ_E3M2 ? __NV_E3M2 : __NV_E2M3, cudaRoundNearest);
   } else {
     return (unsigned)__nv_cvt_float2_to_fp8x2(make_float2(lo, hi), __NV_SATFINITE, FMT == MQ_E4M3 ? __NV_E4M3 : __NV_E5M2);
   }
@@ -407,6 +410,8 @@ cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s) {
       case MQ_E4M3: e = launch_q_cfast<MQ_E4M3>(a, Ct, s); break;
       case MQ_E5M2: e = launch_q_cfast<MQ_E5M2>(a, Ct, s); break;
       case MQ_E2M1: e = launch_q_cfast<MQ_E2M1>(a, Ct, s); break;
+      case MQ_E3M2: e = launch_q_cfast<MQ_E3M2>(a, Ct, s); break;
+      case MQ_E2M3: e = launch_q_cfast<MQ_E2M3>(a, Ct, s); break;
       default: return cudaErrorInvalidValue;
     }
     count_launches(1);
@@ -416,6 +421,8 @@ cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s) {
     case MQ_E4M3: e = launch_q<MQ_E4M3>(a, n_pstrips, Ct, n_items, vec, s); break;
     case MQ_E5M2: e = launch_q<MQ_E5M2>(a, n_pstrips, Ct, n_items, vec, s); break;
     case MQ_E2M1: e = launch_q<MQ_E2M1>(a, n_pstrips, Ct, n_items, vec, s); break;
+    case MQ_E3M2: e = launch_q<MQ_E3M2>(a, n_pstrips, Ct, n_items, vec, s); break;
+    case MQ_E2M3: e = launch_q<MQ_E2M3>(a, n_pstrips, Ct, n_items, vec, s); break;
     default: return cudaErrorInvalidValue;
   }
   count_launches(1);

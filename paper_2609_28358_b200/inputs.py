@@ -19,7 +19,7 @@ import numpy as np
 ConvDesc = namedtuple("ConvDesc", "N C_in H W C_out Kh Kw stride_h stride_w pad_h pad_w")
 
 # element formats / roles: plain integers shared by name with both sides' own enums
-E4M3, E5M2, E2M1 = 0, 1, 2
+E4M3, E5M2, E2M1, E3M2, E2M3 = 0, 1, 2, 3, 4
 ROLE_X, ROLE_W, ROLE_DY = 0, 1, 2
 
 _TENSOR_IDS = {"x": 1, "w": 2, "dy": 3, "outlier": 4}
@@ -156,6 +156,15 @@ def config5(channels=(64, 128, 256, 512), sizes=(14, 28, 56), N=256):
                         layers.append(Layer(f"cfg5_{fname}_k{k}s{s}_c{c}_hw{hw}", conv_desc(N, c, hw, hw, c, k, s),
                                             fmt, fmt, fmt, "gauss", "kaiming", "gauss", seed))
     return layers
+
+
+def fp6_layers(N=256):
+    """Two mid-size 3x3 layers in the 6-bit element formats: E3M2 activations with E4M3 weights and E5M2 gradients
+    (the MicroQonv+ mix), and E2M3 everywhere (the "-6" variant); Gaussian tensors as in the sweep."""
+    return [
+        Layer("fp6_e3m2act_k3s1_c256_hw28", conv_desc(N, 256, 28, 28, 256, 3), E3M2, E4M3, E5M2, "gauss", "kaiming", "gauss", 6001),
+        Layer("fp6_e2m3_k3s1_c256_hw28", conv_desc(N, 256, 28, 28, 256, 3), E2M3, E2M3, E2M3, "gauss", "kaiming", "gauss", 6002),
+    ]
 
 
 CONFIGS = {"config1": config1, "config2": config2, "config3": config3, "config4": config4, "config5": config5}

@@ -13,7 +13,7 @@ import torch
 
 ConvDesc = namedtuple("ConvDesc", "N C_in H W C_out Kh Kw stride_h stride_w pad_h pad_w")
 
-E4M3, E5M2, E2M1 = 0, 1, 2
+E4M3, E5M2, E2M1, E3M2, E2M3 = 0, 1, 2, 3, 4
 ROLE_X, ROLE_W, ROLE_DY = 0, 1, 2
 NCHW, HWNC = 0, 1
 OP_FWD, OP_BWD_DATA, OP_BWD_WEIGHT = 0, 1, 2

@@ -47,7 +47,7 @@ def test_status_strings(mq):
 @pytest.mark.parametrize("desc", [inputs.conv_desc(8, 32, 32, 32, 64, 3), inputs.conv_desc(37, 48, 9, 7, 70, 3, 2),
                                   inputs.conv_desc(256, 512, 14, 14, 512, 1, 1, 0)])
 def test_size_queries_match_oracle(mq, desc):
-    for fmt in (mq.E4M3, mq.E5M2, mq.E2M1):
+    for fmt in (mq.E4M3, mq.E5M2, mq.E2M1, mq.E3M2, mq.E2M3):
         for role in (mq.ROLE_X, mq.ROLE_W, mq.ROLE_DY):
             assert mq.qtensor_sizes(desc, role, fmt) == oracle.qtensor_sizes(desc, role, fmt)
         assert mq.im2col_sizes(desc, fmt) == oracle.im2col_sizes(desc, fmt)

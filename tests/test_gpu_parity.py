@@ -14,8 +14,9 @@ from parity_util import (OracleLayer, assert_same_bytes, check_convs, check_im2c
 
 pytestmark = pytest.mark.gpu
 
-E4M3, E5M2, E2M1 = mq.E4M3, mq.E5M2, mq.E2M1
-FMT_SETS = [(E4M3, E4M3, E5M2), (E2M1, E2M1, E2M1), (E5M2, E4M3, E4M3), (E2M1, E4M3, E5M2)]
+E4M3, E5M2, E2M1, E3M2, E2M3 = mq.E4M3, mq.E5M2, mq.E2M1, mq.E3M2, mq.E2M3
+FMT_SETS = [(E4M3, E4M3, E5M2), (E2M1, E2M1, E2M1), (E5M2, E4M3, E4M3), (E2M1, E4M3, E5M2),
+            (E3M2, E4M3, E5M2), (E2M3, E2M3, E2M3), (E3M2, E2M3, E3M2)]   # the 6-bit formats: MicroQonv+ activations, "-6", mixed
 
 
 def make_layer(name, desc, fmts, seed, kinds=("relu", "kaiming", "small")):
