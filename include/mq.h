@@ -52,8 +52,8 @@ typedef enum {
 typedef enum { MQ_E4M3 = 0, MQ_E5M2 = 1, MQ_E2M1 = 2,
                MQ_E3M2 = 3, MQ_E2M3 = 4 } mq_elem;   /* element format, Sec. II-D; the 6-bit formats (Sec. V: the
                                                         activations of MicroQonv+, the "-6" variant) are stored one code
-                                                        per byte, value in the low six bits, sign in bit 5; their GEMMs
-                                                        run on the CUDA-core kernels */
+                                                        per byte, value in the low six bits, sign in bit 5 (the
+                                                        convolution calls pack or re-encode them in their scratch) */
 typedef enum { MQ_ROLE_X = 0, MQ_ROLE_W = 1, MQ_ROLE_DY = 2 } mq_role; /* which tensor, Sec. IV-B   */
 typedef enum { MQ_NCHW = 0, MQ_HWNC = 1 } mq_layout;                   /* fp32 tensor layout        */
 typedef enum { MQ_OP_FWD = 0, MQ_OP_BWD_DATA = 1, MQ_OP_BWD_WEIGHT = 2 } mq_op;

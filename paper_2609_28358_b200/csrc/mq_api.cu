@@ -67,9 +67,9 @@ bool conv_tc_eligible(int op, const Geom& g, int fmt_x_like, int fmt_w) {
   const bool fp4 = fmt_x_like == MQ_E2M1 && fmt_w == MQ_E2M1;
   const bool fp8 = fmt_x_like != MQ_E2M1 && fmt_w != MQ_E2M1;
   if (!fp4 && !fp8) return false;
-  // 6-bit operands: the tensor core reads them as 16 codes packed into 12 bytes + 4 bytes of padding, not one code per
-  // byte as they are stored here; they run on the CUDA-core kernels
-  if (fmt_is_6bit(fmt_x_like) || fmt_is_6bit(fmt_w)) return false;
+  // 6-bit operands: the tensor core reads them as 16 codes packed into 12 bytes + 4 bytes of padding (along K), not one
+  // code per byte as they are stored; run_conv_tc packs them into scratch first (MQ_TC_NO_FP6=1: CUDA-core kernels)
+  if ((fmt_is_6bit(fmt_x_like) || fmt_is_6bit(fmt_w)) && env_int("MQ_TC_NO_FP6", 0)) return false;
   const int Kp = op == MQ_OP_FWD ? g.Cp : g.Cop;
   const int rowbytes = Kp * (fp4 ? 4 : 8) / 8;
   return rowbytes % 32 == 0;
@@ -112,7 +112,7 @@ int choose_tw(int w_eff, int N, int layout, double k_bytes, int bn, bool thin, b
 struct ConvTcPlan {
   ConvTcParams p;
   int rowbytes, rows_b;
-  size_t off_wt_scales, off_sfa, off_sfb, off_bimg, total;
+  size_t off_wt_scales, off_sfa, off_sfb, off_bimg, off_pack_a, off_pack_b, total;   // off_pack_*: packed copies of 6-bit operands
 };
 
 bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, ConvTcPlan* out) {
@@ -251,6 +251,10 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   out->off_sfb = o; o += up256(conv_tc_sfb_bytes(p));
   out->off_bimg = o;
   if (p.halo) o += up256((size_t)p.tiles_c * taps * p.BN * p.KB);
+  out->off_pack_a = o;
+  if (fmt_is_6bit(fmt_x_like)) o += up256((size_t)p.Hs * p.Ws * g.N * rowbytes);
+  out->off_pack_b = o;
+  if (fmt_is_6bit(fmt_w)) o += up256((size_t)out->rows_b * taps * rowbytes);
   out->total = o;
   return true;
 }
@@ -282,6 +286,19 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
     b_codes = base;
     p.b_scales = wt_scales;
   }
+  // 6-bit operands: 16 codes -> 12 packed bytes + 4 bytes of padding per 16-byte chunk (the container of the MMA's
+  // 6-bit types), written to scratch; every later step moves whole 16-byte chunks and is unchanged
+  const uint8_t* a_codes = static_cast<const uint8_t*>(qx_like->codes);
+  if (fmt_is_6bit(qx_like->fmt)) {
+    const size_t nbytes = (size_t)p.Hs * p.Ws * g.N * pl.rowbytes;
+    if (launch_pack6(a_codes, base + pl.off_pack_a, nbytes, stream) != cudaSuccess) return MQ_ERR_CUDA;
+    a_codes = base + pl.off_pack_a;
+  }
+  if (fmt_is_6bit(qw->fmt)) {
+    const size_t nbytes = (size_t)pl.rows_b * taps * pl.rowbytes;
+    if (launch_pack6(b_codes, base + pl.off_pack_b, nbytes, stream) != cudaSuccess) return MQ_ERR_CUDA;
+    b_codes = base + pl.off_pack_b;
+  }
   p.a_scales = qx_like->scales;
   p.sfa_img = base + pl.off_sfa;
   p.sfb_img = base + pl.off_sfb;
@@ -298,7 +315,7 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
     uint32_t box[4] = {(uint32_t)p.KB, (uint32_t)((p.TW - 1) * wst + 1), (uint32_t)p.TN, 1u};
     if (p.halo) { box[1] = (uint32_t)p.WH; box[3] = (uint32_t)g.Kh; }   // the whole halo of a tile in one box
     const uint32_t es[4] = {1u, wst, 1u, 1u};
-    if (!encode_tensor_map_u8(&map_a, qx_like->codes, 4, dims, strides, box, es, p.KB)) return MQ_ERR_CUDA;
+    if (!encode_tensor_map_u8(&map_a, a_codes, 4, dims, strides, box, es, p.KB)) return MQ_ERR_CUDA;
   }
   map_w = map_a;
   if (p.halo) {
@@ -367,7 +384,10 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   const bool fp4 = fmt_x == MQ_E2M1 && fmt_g == MQ_E2M1;
   const bool fp8 = fmt_x != MQ_E2M1 && fmt_g != MQ_E2M1;
   if (!fp4 && !fp8) return w;
-  if (fmt_is_6bit(fmt_x) || fmt_is_6bit(fmt_g)) return w;   // see conv_tc_eligible
+  // 6-bit operands: this GEMM reads its operands MN-major (K = samples), where the MMA's packed 6-bit container (packed
+  // along K) does not apply; every E3M2 / E2M3 value is also an E4M3 value, so the codes are re-encoded exactly as
+  // E4M3 bytes in scratch and the 8-bit path runs unchanged (MQ_TC_NO_FP6=1: CUDA-core kernels)
+  if ((fmt_is_6bit(fmt_x) || fmt_is_6bit(fmt_g)) && env_int("MQ_TC_NO_FP6", 0)) return w;
   WgradTcParams& p = w.p;
   p.N = g.N; p.Nt = g.Nt; p.Ho = g.Ho; p.Wo = g.Wo; p.H = g.H; p.W = g.W; p.Cout = g.Cout; p.Cp = g.Cp; p.Ct = g.Ct; p.Cot = g.Cot;
   p.Kh = g.Kh; p.Kw = g.Kw; p.sh = g.sh; p.sw = g.sw; p.ph = g.ph; p.pw = g.pw;
@@ -429,9 +449,11 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   w.off_xt = o;
   if (flat) { p.xt_block_bytes = (long long)w.P_b * p.b_rows * p.KBn; o += up256((size_t)p.cb_tiles * p.xt_block_bytes); }
   else if (fp4) o += up256((size_t)g.Cp * g.H * g.W * w.Npad / 2);
+  else if (fmt_is_6bit(fmt_x)) o += up256((size_t)g.H * g.W * g.N * g.Cp);     // X re-encoded as E4M3
   w.off_gt = o;
   if (flat) { p.gt_block_bytes = (long long)w.P_a * 128 * p.KBn; o += up256((size_t)p.m_tiles * p.gt_block_bytes); }
   else if (fp4) o += up256((size_t)g.Cop * g.Ho * g.Wo * w.Npad / 2);
+  else if (fmt_is_6bit(fmt_g)) o += up256((size_t)g.Ho * g.Wo * g.N * g.Cop);  // G_Y re-encoded as E4M3
   w.total = o;
   w.ok = true;
   return w;
@@ -469,14 +491,25 @@ mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const 
       if (!encode_tensor_map_u8(&map_b, xt, 4, dims, strides, box, nullptr, swz)) return MQ_ERR_CUDA;
     }
   } else {
-    const uint32_t fa = fmt_mma_code(qg->fmt), fb = fmt_mma_code(qx->fmt);
+    const uint8_t* g_codes = static_cast<const uint8_t*>(qg->codes);
+    const uint8_t* x_codes = static_cast<const uint8_t*>(qx->codes);
+    int fmt_g_eff = qg->fmt, fmt_x_eff = qx->fmt;
+    if (fmt_is_6bit(qx->fmt)) {
+      if (launch_recode6_e4m3(x_codes, xt, (size_t)g.H * g.W * g.N * g.Cp, qx->fmt, stream) != cudaSuccess) return MQ_ERR_CUDA;
+      x_codes = xt; fmt_x_eff = MQ_E4M3;
+    }
+    if (fmt_is_6bit(qg->fmt)) {
+      if (launch_recode6_e4m3(g_codes, gt, (size_t)g.Ho * g.Wo * g.N * g.Cop, qg->fmt, stream) != cudaSuccess) return MQ_ERR_CUDA;
+      g_codes = gt; fmt_g_eff = MQ_E4M3;
+    }
+    const uint32_t fa = fmt_mma_code(fmt_g_eff), fb = fmt_mma_code(fmt_x_eff);
     p.idesc = (fa << 7) | (fb << 10) | (1u << 15) | (1u << 16) | (1u << 23) | (((p.cta2 ? 256u : 128u) >> 4) << 24);
     {
       const uint64_t rb = (uint64_t)g.Cop;
       const uint64_t dims[4] = {rb, (uint64_t)g.N, (uint64_t)g.Wo, (uint64_t)g.Ho};
       const uint64_t strides[3] = {rb, (uint64_t)g.N * rb, (uint64_t)g.Wo * g.N * rb};
       const uint32_t box[4] = {128u, (uint32_t)(p.BPP * 32), (uint32_t)p.KPX, 1u};
-      if (!encode_tensor_map_u8(&map_a, qg->codes, 4, dims, strides, box, nullptr, 128)) return MQ_ERR_CUDA;
+      if (!encode_tensor_map_u8(&map_a, g_codes, 4, dims, strides, box, nullptr, 128)) return MQ_ERR_CUDA;
     }
     {
       const uint64_t rb = (uint64_t)g.Cp;
@@ -484,7 +517,7 @@ mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const 
       const uint64_t strides[3] = {rb, (uint64_t)g.N * rb, (uint64_t)g.W * g.N * rb};
       const uint32_t box[4] = {128u, (uint32_t)(p.BPP * 32), (uint32_t)((p.KPX - 1) * g.sw + 1), 1u};
       const uint32_t es[4] = {1u, 1u, (uint32_t)g.sw, 1u};
-      if (!encode_tensor_map_u8(&map_b, qx->codes, 4, dims, strides, box, es, 128)) return MQ_ERR_CUDA;
+      if (!encode_tensor_map_u8(&map_b, x_codes, 4, dims, strides, box, es, 128)) return MQ_ERR_CUDA;
     }
   }
   if (p.mode == MQ_WG_FP4_FLAT) {

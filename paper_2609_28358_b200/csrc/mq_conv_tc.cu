@@ -1420,6 +1420,61 @@ cudaError_t launch_conv_tc_halo_inst(const ConvTcParams& p, const CUtensorMap& m
   return launch_conv_tc_halo_taps<MODE, KB, FP4, 0>(p, map_a, map_b, map_w, s);
 }
 
+__global__ void __launch_bounds__(256) pack6_kernel(const uint4* __restrict__ in, uint4* __restrict__ out, size_t nchunks) {
+  pdl_wait();
+  for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < nchunks; i += (size_t)gridDim.x * 256) {
+    const uint4 v = __ldg(in + i);
+    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+    unsigned long long lo = 0ull, hi = 0ull;   // bits 0..63 and 64..95 of the 96-bit field
+#pragma unroll
+    for (int e = 0; e < 16; ++e) {
+      const unsigned long long c = (w[e >> 2] >> (8 * (e & 3))) & 0x3Fu;
+      const int bit = 6 * e;
+      if (bit < 64) { lo |= c << bit; if (bit > 58) hi |= c >> (64 - bit); }
+      else hi |= c << (bit - 64);
+    }
+    out[i] = make_uint4((uint32_t)lo, (uint32_t)(lo >> 32), (uint32_t)hi, 0u);
+  }
+}
+cudaError_t launch_pack6(const uint8_t* in, uint8_t* out, size_t nbytes, cudaStream_t s) {
+  const size_t nchunks = nbytes / 16;
+  if (nchunks == 0) return cudaSuccess;
+  size_t blocks = (nchunks + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  count_launches(1);
+  return launch_pdl(pack6_kernel, dim3((unsigned)blocks), dim3(256), 0, s, reinterpret_cast<const uint4*>(in), reinterpret_cast<uint4*>(out), nchunks);
+}
+
+template <bool IS_E3M2>
+__global__ void __launch_bounds__(256) recode6_kernel(const uint4* __restrict__ in, uint4* __restrict__ out, size_t nchunks) {
+  pdl_wait();
+  for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < nchunks; i += (size_t)gridDim.x * 256) {
+    const uint4 v = __ldg(in + i);
+    uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      uint32_t r = 0;
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const unsigned short pair = (unsigned short)((w[q] >> (16 * h)) & 0xFFFF);
+        const __half2_raw hr = __nv_cvt_fp6x2_to_halfraw2((__nv_fp6x2_storage_t)pair, IS_E3M2 ? __NV_E3M2 : __NV_E2M3);
+        r |= (uint32_t)__nv_cvt_halfraw2_to_fp8x2(hr, __NV_SATFINITE, __NV_E4M3) << (16 * h);   // exact: the value is representable
+      }
+      w[q] = r;
+    }
+    out[i] = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+cudaError_t launch_recode6_e4m3(const uint8_t* in, uint8_t* out, size_t nbytes, int fmt6, cudaStream_t s) {
+  const size_t nchunks = nbytes / 16;
+  if (nchunks == 0) return cudaSuccess;
+  size_t blocks = (nchunks + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  count_launches(1);
+  if (fmt6 == MQ_E3M2) return launch_pdl(recode6_kernel<true>, dim3((unsigned)blocks), dim3(256), 0, s, reinterpret_cast<const uint4*>(in), reinterpret_cast<uint4*>(out), nchunks);
+  return launch_pdl(recode6_kernel<false>, dim3((unsigned)blocks), dim3(256), 0, s, reinterpret_cast<const uint4*>(in), reinterpret_cast<uint4*>(out), nchunks);
+}
+
 size_t conv_tc_pair_smem_bytes(const ConvTcParams& p) {
   const size_t stage = A_STAGE_BYTES + 128 * 128 + SFA_BYTES + SFB_BYTES;
   return 1024 + (size_t)p.stages * stage + (p.tma_store ? EPI_STAGING_BYTES : 0) + (2 * (size_t)p.stages + 4) * 8 + 64;

@@ -67,6 +67,10 @@ struct ConvTcParams {
 // map_a: gathered activation codes.  map_w: weight codes, one tap per box (per-tap kernel) or all taps of a tile in one
 // box (whole-tile kernel with fused preparation).  map_out: the fp32 NCHW output seen as (W, N, C, H), used when
 // p.tma_store is set.
+// 16-byte chunks of one-code-per-byte 6-bit codes -> 12 packed bytes (code i at bit 6 i) + 4 zero bytes
+cudaError_t launch_pack6(const uint8_t* in, uint8_t* out, size_t nbytes, cudaStream_t s);
+// one-code-per-byte E3M2 / E2M3 codes -> the E4M3 codes of the same values (every 6-bit value is an E4M3 value)
+cudaError_t launch_recode6_e4m3(const uint8_t* in, uint8_t* out, size_t nbytes, int fmt6, cudaStream_t s);
 cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_out, const CUtensorMap& map_sfa,
                            const CUtensorMap& map_sfb, cudaStream_t s);
 // Expands the compact tile scales into the per-stage scale-vector chunks the MMA reads (p.sfa_img, p.sfb_img).

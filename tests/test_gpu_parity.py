@@ -184,6 +184,17 @@ def test_layer_from_host_buffers_matches_the_device_calls(fmts):
     assert mq.last_device_status() == 0
 
 
+def test_6bit_gemms_on_cuda_cores(monkeypatch):
+    """The CUDA-core route of 6-bit operands (the default packs them for the tensor cores; the weight gradient always
+    takes this route)."""
+    monkeypatch.setenv("MQ_TC_NO_FP6", "1")
+    d = inputs.conv_desc(64, 96, 8, 8, 64, 3, 1, 1)
+    for fmts in ((E3M2, E4M3, E5M2), (E2M3, E2M3, E2M3)):
+        ol = OracleLayer(make_layer("fp6_cuda_cores", d, fmts, seed=31, kinds=("relu", "kaiming", "gauss")))
+        qs = check_quantize(ol)
+        check_convs(ol, qs, samples=20000, layouts=(mq.NCHW, mq.HWNC))
+
+
 ALT_PATHS = [("MQ_TC_NO_HALO", "1"), ("MQ_TC_NO_FUSED", "1"), ("MQ_TC_NO_TMA_STORE", "1"), ("MQ_TC_TMA_STORE", "1"), ("MQ_TC_NO_PAIR", "1"),
              ("MQ_TC_BN", "256"), ("MQ_TC_TW", "4"), ("MQ_TC_TW", "16"), ("MQ_TC_TW", "32"), ("MQ_WGRAD_NO_FLAT", "1"),
              ("MQ_WGRAD_NO_GROUP", "1"), ("MQ_WGRAD_N128", "1"), ("MQ_WGRAD_NO_CTA2", "1"), ("MQ_TC_NO_MMA_CP", "1"), ("MQ_WGRAD_MMA_CP", "1"), ("MQ_TC_FP4_BN128", "1"), ("MQ_TC_CTA2", "1"), ("MQ_WGRAD_SPLITS", "3"), ("MQ_DISABLE_TC_WGRAD", "1"), ("MQ_DISABLE_TC", "1")]
