@@ -347,6 +347,7 @@ def run_ours(args):
                                  "value": 3.0 * layer_flops(d) / (ms_cl * 1e-3) / 1e12, "unit": "TFLOPS", "ms_per_step": ms_cl,
                                  "ms_per_call": {n: float(np.mean(v)) for n, v in per_cl.items()}},
         "device_status": dev_status,
+        "quantization_accounting": quantization_accounting(d, fmts),
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(layer, budget_s=args.cpu_budget)
@@ -354,6 +355,26 @@ def run_ours(args):
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def quantization_accounting(d, fmts):
+    """Counts of the kind the paper tabulates (Table I): elements that pass through a quantizer per training step of the
+    layer, and bytes of the activation kept for the backward pass, for this library's path (square tiles: each tensor
+    quantized once, usable in both contraction directions) next to two stand-ins built from their descriptions in the
+    paper - a line-block scheme (blocks along one contraction axis only, so every tensor is quantized again for its
+    second GEMM and the activation is kept in fp32 for that) and a scheme that quantizes the expanded im2col matrix and
+    keeps it.  Pure arithmetic on the layer shape; nothing here is measured."""
+    ho, wo = inputs.out_hw(d)
+    nx, nw, ng = d.N * d.C_in * d.H * d.W, d.C_out * d.C_in * d.Kh * d.Kw, d.N * d.C_out * ho * wo
+    nxp = ho * wo * d.N * d.Kh * d.Kw * d.C_in                      # elements of the expanded X'
+    bx = FMT_BITS[fmts[0]] / 8.0
+    return {
+        "unit": {"quantized_elements": "elements per fwd+bwd step", "activation_kept": "bytes"},
+        "square_tiles_once": {"quantized_elements": nx + nw + ng, "activation_kept": nx * bx * (1 + 1 / 1024)},
+        "line_blocks_requantize": {"quantized_elements": 2 * (nx + nw + ng), "activation_kept": nx * 4.0},
+        "quantize_expanded_im2col": {"quantized_elements": nxp + nw + ng, "activation_kept": nxp * bx * (1 + 1 / 32)},
+        "expansion_factor": nxp / nx,
+    }
 
 
 # ----------------------------------------------------------------------------------- CPU oracle
