@@ -376,14 +376,23 @@ struct WgradPlan {
   WgradTcParams p;
   int Npad, P_a, P_b;
   size_t off_sfa, off_sfb, off_xt, off_gt, total;
+  bool recode4;   // E2M1 operands re-encoded as E4M3 bytes for the 8-bit path
 };
 
 WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   WgradPlan w{};
   if (env_int("MQ_DISABLE_TC", 0) || env_int("MQ_DISABLE_TC_WGRAD", 0)) return w;
-  const bool fp4 = fmt_x == MQ_E2M1 && fmt_g == MQ_E2M1;
-  const bool fp8 = fmt_x != MQ_E2M1 && fmt_g != MQ_E2M1;
-  if (!fp4 && !fp8) return w;
+  const bool fp4_in = fmt_x == MQ_E2M1 && fmt_g == MQ_E2M1;
+  const bool fp8_in = fmt_x != MQ_E2M1 && fmt_g != MQ_E2M1;
+  if (!fp4_in && !fp8_in) return w;
+  // E2M1 layers that the flat mode below does not take (stride 2, batches that are not 1, 2, 4 or 8 sample tiles): every
+  // E2M1 value is an E4M3 value, so the codes are re-encoded exactly as E4M3 bytes in scratch and the 8-bit path (stored
+  // order read MN-major, block pairs) runs - faster than the per-pixel E2M1 mode (MQ_WGRAD_FP4_PIXEL=1 keeps that mode)
+  const bool flat_ok = fp4_in && g.sh == 1 && g.sw == 1 && (g.Nt == 1 || g.Nt == 2 || g.Nt == 4 || g.Nt == 8) && !env_int("MQ_WGRAD_NO_FLAT", 0);
+  const bool recode4 = fp4_in && !flat_ok && !env_int("MQ_WGRAD_FP4_PIXEL", 0);
+  const bool fp4 = fp4_in && !recode4;
+  const bool fp8 = fp8_in || recode4;
+  w.recode4 = recode4;
   // 6-bit operands: this GEMM reads its operands MN-major (K = samples), where the MMA's packed 6-bit container (packed
   // along K) does not apply; every E3M2 / E2M3 value is also an E4M3 value, so the codes are re-encoded exactly as
   // E4M3 bytes in scratch and the 8-bit path runs unchanged (MQ_TC_NO_FP6=1: CUDA-core kernels)
@@ -449,11 +458,11 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   w.off_xt = o;
   if (flat) { p.xt_block_bytes = (long long)w.P_b * p.b_rows * p.KBn; o += up256((size_t)p.cb_tiles * p.xt_block_bytes); }
   else if (fp4) o += up256((size_t)g.Cp * g.H * g.W * w.Npad / 2);
-  else if (fmt_is_6bit(fmt_x)) o += up256((size_t)g.H * g.W * g.N * g.Cp);     // X re-encoded as E4M3
+  else if (fmt_is_6bit(fmt_x) || recode4) o += up256((size_t)g.H * g.W * g.N * g.Cp);     // X re-encoded as E4M3
   w.off_gt = o;
   if (flat) { p.gt_block_bytes = (long long)w.P_a * 128 * p.KBn; o += up256((size_t)p.m_tiles * p.gt_block_bytes); }
   else if (fp4) o += up256((size_t)g.Cop * g.Ho * g.Wo * w.Npad / 2);
-  else if (fmt_is_6bit(fmt_g)) o += up256((size_t)g.Ho * g.Wo * g.N * g.Cop);  // G_Y re-encoded as E4M3
+  else if (fmt_is_6bit(fmt_g) || recode4) o += up256((size_t)g.Ho * g.Wo * g.N * g.Cop);  // G_Y re-encoded as E4M3
   w.total = o;
   w.ok = true;
   return w;
@@ -501,6 +510,11 @@ mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const 
     if (fmt_is_6bit(qg->fmt)) {
       if (launch_recode6_e4m3(g_codes, gt, (size_t)g.Ho * g.Wo * g.N * g.Cop, qg->fmt, stream) != cudaSuccess) return MQ_ERR_CUDA;
       g_codes = gt; fmt_g_eff = MQ_E4M3;
+    }
+    if (w.recode4) {
+      if (launch_recode4_e4m3(x_codes, xt, (size_t)g.H * g.W * g.N * g.Cp, stream) != cudaSuccess) return MQ_ERR_CUDA;
+      if (launch_recode4_e4m3(g_codes, gt, (size_t)g.Ho * g.Wo * g.N * g.Cop, stream) != cudaSuccess) return MQ_ERR_CUDA;
+      x_codes = xt; g_codes = gt; fmt_x_eff = MQ_E4M3; fmt_g_eff = MQ_E4M3;
     }
     const uint32_t fa = fmt_mma_code(fmt_g_eff), fb = fmt_mma_code(fmt_x_eff);
     p.idesc = (fa << 7) | (fb << 10) | (1u << 15) | (1u << 16) | (1u << 23) | (((p.cta2 ? 256u : 128u) >> 4) << 24);

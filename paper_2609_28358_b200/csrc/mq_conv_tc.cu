@@ -1475,6 +1475,36 @@ cudaError_t launch_recode6_e4m3(const uint8_t* in, uint8_t* out, size_t nbytes, 
   return launch_pdl(recode6_kernel<false>, dim3((unsigned)blocks), dim3(256), 0, s, reinterpret_cast<const uint4*>(in), reinterpret_cast<uint4*>(out), nchunks);
 }
 
+__global__ void __launch_bounds__(256) recode4_kernel(const uint2* __restrict__ in, uint4* __restrict__ out, size_t nchunks) {
+  pdl_wait();
+  // E2M1 magnitudes 0, .5, 1, 1.5, 2, 3, 4, 6 as E4M3 bytes; the sign moves from bit 3 of the nibble to bit 7 of the byte
+  const uint32_t lut_lo = 0x3C383000u, lut_hi = 0x4C484440u;
+  for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < nchunks; i += (size_t)gridDim.x * 256) {
+    const uint2 v = __ldg(in + i);
+    const uint32_t src[2] = {v.x, v.y};
+    uint32_t w[4];
+#pragma unroll
+    for (int q = 0; q < 4; ++q) {
+      uint32_t r = 0;
+#pragma unroll
+      for (int b = 0; b < 4; ++b) {
+        const uint32_t nib = (src[q >> 1] >> (16 * (q & 1) + 4 * b)) & 0xFu;
+        r |= (__byte_perm(lut_lo, lut_hi, nib & 7u) & 0xFFu | ((nib & 8u) << 4)) << (8 * b);
+      }
+      w[q] = r;
+    }
+    out[i] = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+cudaError_t launch_recode4_e4m3(const uint8_t* in, uint8_t* out, size_t n_out, cudaStream_t s) {
+  const size_t nchunks = n_out / 16;
+  if (nchunks == 0) return cudaSuccess;
+  size_t blocks = (nchunks + 255) / 256;
+  if (blocks > 148 * 16) blocks = 148 * 16;
+  count_launches(1);
+  return launch_pdl(recode4_kernel, dim3((unsigned)blocks), dim3(256), 0, s, reinterpret_cast<const uint2*>(in), reinterpret_cast<uint4*>(out), nchunks);
+}
+
 size_t conv_tc_pair_smem_bytes(const ConvTcParams& p) {
   const size_t stage = A_STAGE_BYTES + 128 * 128 + SFA_BYTES + SFB_BYTES;
   return 1024 + (size_t)p.stages * stage + (p.tma_store ? EPI_STAGING_BYTES : 0) + (2 * (size_t)p.stages + 4) * 8 + 64;

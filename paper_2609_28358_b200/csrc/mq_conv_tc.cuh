@@ -71,6 +71,8 @@ struct ConvTcParams {
 cudaError_t launch_pack6(const uint8_t* in, uint8_t* out, size_t nbytes, cudaStream_t s);
 // one-code-per-byte E3M2 / E2M3 codes -> the E4M3 codes of the same values (every 6-bit value is an E4M3 value)
 cudaError_t launch_recode6_e4m3(const uint8_t* in, uint8_t* out, size_t nbytes, int fmt6, cudaStream_t s);
+// packed E2M1 codes (two per byte) -> the E4M3 codes of the same values, one per byte; n_out = elements = output bytes
+cudaError_t launch_recode4_e4m3(const uint8_t* in, uint8_t* out, size_t n_out, cudaStream_t s);
 cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_out, const CUtensorMap& map_sfa,
                            const CUtensorMap& map_sfb, cudaStream_t s);
 // Expands the compact tile scales into the per-stage scale-vector chunks the MMA reads (p.sfa_img, p.sfb_img).
