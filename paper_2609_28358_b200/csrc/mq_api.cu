@@ -243,6 +243,10 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
       }
     }
   }
+  // unit strides and one 128-byte chunk per stage: the activation-side scale chunk of (tile, kh) equals that of the tile one
+  // output row further with kh - 1, so chunks are stored per source row - Kh times fewer to expand
+  p.sfa_dedup = (!p.halo && !p.cta2 && p.KB == 128 && g.sh == 1 && g.sw == 1 && !env_int("MQ_TC_NO_SFA_DEDUP", 0)) ? 1 : 0;
+  p.sfa_hk = p.tiles_h + g.Kh - 1;
   out->p = p;
   size_t o = 0;
   out->off_wt_scales = 0;

@@ -71,6 +71,12 @@ __device__ __forceinline__ Tile decode_tile(const ConvTcParams& p, unsigned t) {
   q.n0 = (int)u * p.TN;
   return q;
 }
+// number of A-side scale chunks of a launch
+__host__ __device__ __forceinline__ unsigned conv_tc_sfa_chunks(const ConvTcParams& p) {
+  const unsigned tiles_m = (unsigned)(p.total_tiles / p.tiles_c);
+  if (p.sfa_dedup) return tiles_m / (unsigned)(p.tiles_h * p.classes) * (unsigned)p.sfa_hk * (unsigned)(p.Kw * p.cpt);
+  return tiles_m * (unsigned)p.max_stages;
+}
 // index of a tile among the tiles that differ in anything but the channel tile (A-side scale chunks)
 __device__ __forceinline__ unsigned tile_m_index(const ConvTcParams& p, const Tile& q) {
   return (((unsigned)(q.n0 >> p.lgTN) * p.tiles_h + q.h) * p.tiles_w + (q.w0 >> p.lgTW)) * p.classes + q.cls;
@@ -436,9 +442,15 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         pos.reset();
         const uint8_t* sfa_src = p.sfa_img + (size_t)tile_m_index(p, tile) * p.max_stages * (512 * SPA);
         const uint8_t* sfb_src = p.sfb_img + ((size_t)tile.cls * p.tiles_c + tile.ct) * p.max_stages * (512 * SPA * atoms_b);
+        // shared A-side chunks: keyed by the source row (output row + kh, or + Kh-1-kh for the input gradient)
+        const int dd_row = p.tiles_w * tw.nkw * p.cpt;
+        const uint8_t* sfa_dd = p.sfa_img + ((size_t)(((tile.n0 >> p.lgTN) * p.sfa_hk + tile.h + (MODE == MQ_OP_FWD ? 0 : p.Kh - 1)) * p.tiles_w +
+                                                      (tile.w0 >> p.lgTW)) * (tw.nkw * p.cpt)) * (512 * SPA);
         for (int q0 = 0; q0 < Q; q0 += G, ++gi) {
           const int nch = min(G, Q - q0);
           const bool mine = (gi & 1u) == (uint32_t)lhalf;
+          if (G == 1 && p.sfa_dedup)
+            sfa_src = sfa_dd + (long long)((MODE == MQ_OP_FWD ? pos.ia : -pos.ia) * dd_row + pos.ib * p.cpt + pos.cc) * (512 * SPA);
           // coordinates of the stage's boxes, before the wait
           int c0[G], c1[G], c2[G];
 #pragma unroll
@@ -1154,7 +1166,7 @@ __global__ void __launch_bounds__(256) expand_conv_scales_kernel(const ConvTcPar
   constexpr int G = 128 / KB, APC = KB / 32, SPA = FP4 ? 2 : 1, BPC = APC * SPA;
   const int lane = threadIdx.x & 31;
   const unsigned wid = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
-  const unsigned nA = n_tile_m * (unsigned)p.max_stages;
+  const unsigned nA = conv_tc_sfa_chunks(p);
   const unsigned nB = (unsigned)(p.classes * p.tiles_c * p.max_stages);
   const int atoms_b = (p.BN + 127) / 128;
   if (p.halo && wid >= nA + nB) {
@@ -1175,7 +1187,37 @@ __global__ void __launch_bounds__(256) expand_conv_scales_kernel(const ConvTcPar
     }
     return;
   }
-  if (wid < nA) {
+  if (G == 1 && p.sfa_dedup && wid < nA) {
+    // shared chunks: wid = (((sample tile * row keys + row key) * column tiles + column tile) * Kw + kw) * cpt + chunk
+    unsigned u = wid;
+    ChunkPos pos;
+    pos.ia = 0;
+    pos.cc = (int)(u % (unsigned)p.cpt); u /= (unsigned)p.cpt;
+    pos.ib = (int)(u % (unsigned)p.Kw); u /= (unsigned)p.Kw;
+    Tile tile;
+    tile.w0 = (int)(u % (unsigned)p.tiles_w) * p.TW; u /= (unsigned)p.tiles_w;
+    const int hk = (int)(u % (unsigned)p.sfa_hk);
+    tile.n0 = (int)(u / (unsigned)p.sfa_hk) * p.TN;
+    tile.h = 0; tile.cls = 0; tile.c0 = 0; tile.ct = 0;
+    TapWalk<MODE> tw;
+    tw.init(p, tile);
+    const int hs = hk + tw.hs0 - (MODE == MQ_OP_FWD ? 0 : p.Kh - 1);   // hs0 of output row 0: -ph, or +ph for the input gradient
+    const int ws0 = src_w0(tw, pos);
+    unsigned long long acc[4] = {0ull, 0ull, 0ull, 0ull};
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const int r = 32 * j + lane;
+      const int tw_ = r & (p.TW - 1), tn = r >> p.lgTW;
+      const int n = tile.n0 + tn, ws = ws0 + tw_;
+      if (n < p.N && hs >= 0 && hs < p.Hs && ws >= 0 && ws < p.Ws)
+        acc[j] = load_scale_bytes<BPC>(p.a_scales + (((long long)hs * p.Ws + ws) * p.Nt + (n >> 5)) * p.Kblocks + pos.cc * BPC);
+    }
+    uint8_t* dst = p.sfa_img + (size_t)wid * (512 * SPA) + lane * 16;
+#pragma unroll
+    for (int g = 0; g < SPA; ++g)
+      *reinterpret_cast<uint4*>(dst + g * 512) = make_uint4((uint32_t)(acc[0] >> (32 * g)), (uint32_t)(acc[1] >> (32 * g)), (uint32_t)(acc[2] >> (32 * g)),
+                                                          (uint32_t)(acc[3] >> (32 * g)));
+  } else if (wid < nA) {
     const unsigned tm = wid / (unsigned)p.max_stages;
     const int st = (int)(wid - tm * p.max_stages);
     const Tile tile = tile_of_m_index(p, tm);
@@ -1371,7 +1413,7 @@ cudaError_t launch_conv_tc_inst(const ConvTcParams& p, const CUtensorMap& map_a,
 }
 
 size_t conv_tc_sfa_bytes(const ConvTcParams& p) {
-  return (size_t)(p.total_tiles / p.tiles_c) * p.max_stages * 512 * (p.kind_fp4 ? 2 : 1);
+  return (size_t)conv_tc_sfa_chunks(p) * 512 * (p.kind_fp4 ? 2 : 1);
 }
 size_t conv_tc_sfb_bytes(const ConvTcParams& p) {
   return (size_t)p.classes * p.tiles_c * p.max_stages * 512 * (p.kind_fp4 ? 2 : 1) * ((p.BN + 127) / 128);
@@ -1380,7 +1422,7 @@ size_t conv_tc_sfb_bytes(const ConvTcParams& p) {
 template <int MODE, int KB, bool FP4>
 cudaError_t launch_expand_inst(const ConvTcParams& p, cudaStream_t s) {
   const unsigned n_tile_m = (unsigned)(p.total_tiles / p.tiles_c);
-  unsigned long long warps = (unsigned long long)n_tile_m * p.max_stages + (unsigned long long)p.classes * p.tiles_c * p.max_stages;
+  unsigned long long warps = (unsigned long long)conv_tc_sfa_chunks(p) + (unsigned long long)p.classes * p.tiles_c * p.max_stages;
   if (p.halo) warps += ((unsigned long long)p.tiles_c * p.Kh * p.Kw * p.BN * (KB / 16) + 31) / 32;
   const unsigned blocks = (unsigned)((warps + 7) / 8);
   count_launches(1);

@@ -42,6 +42,9 @@ struct ConvTcParams {
   uint8_t* sfa_img;         // [tile without the channel index][max_stages][512 * SPA]
   uint8_t* sfb_img;         // [class][channel tile][max_stages][512 * SPA * atoms_b]
   int max_stages;           // stages of the longest tile
+  int sfa_dedup;            // 1: A-side chunks are stored once per (sample tile, source row, column tile, kw, chunk) - unit strides, one
+                            // chunk per stage: tiles on neighbouring output rows read the same source row through different kh
+  int sfa_hk;               // source-row keys per sample tile = output rows + Kh - 1
   // whole-tile-per-stage variant (small channel counts, stride 1): see conv_tc_halo_kernel
   int halo;                 // 1: use it
   int WH;                   // columns of the activation halo box = TW + Kw - 1
