@@ -53,6 +53,12 @@ def _l():
         lib.orc_encode_elem.argtypes = [ctypes.c_int, ctypes.c_double]
         lib.orc_scale_code.restype = ctypes.c_int
         lib.orc_scale_code.argtypes = [ctypes.c_int, ctypes.c_double]
+        lib.orc_encode_elem_sr.restype = ctypes.c_int
+        lib.orc_encode_elem_sr.argtypes = [ctypes.c_int, ctypes.c_double, ctypes.c_uint32]
+        lib.orc_sr_bits.restype = ctypes.c_uint32
+        lib.orc_sr_bits.argtypes = [ctypes.c_uint64, ctypes.c_uint64]
+        lib.orc_quantize_sr.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_uint64,
+                                        ctypes.c_void_p, ctypes.c_void_p]
         _lib = lib
     return _lib
 
@@ -75,6 +81,16 @@ def decode_elem(fmt: int, code: int) -> float:
 
 def encode_elem(fmt: int, v: float) -> int:
     return int(_l().orc_encode_elem(fmt, float(v)))
+
+
+def encode_elem_sr(fmt: int, v: float, bits: int) -> int:
+    """Stochastic Round(.) of Eq. 6 for one scaled value, given the element's 32 random bits."""
+    return int(_l().orc_encode_elem_sr(fmt, float(v), int(bits) & 0xFFFFFFFF))
+
+
+def sr_bits(seed: int, index: int) -> int:
+    """The 32 random bits of element `index` (position in the logical NCHW / OIHW tensor) under `seed`."""
+    return int(_l().orc_sr_bits(int(seed), int(index)))
 
 
 def scale_code(fmt: int, amax: float) -> int:
@@ -111,6 +127,19 @@ def quantize(desc, role, fmt, src, block=(32, 32)):
     codes = np.zeros(cb, dtype=np.uint8)
     scales = np.zeros(sb, dtype=np.uint8)
     rc = _l().orc_quantize(_p(_desc(desc)), role, fmt, block[0], block[1], _p(src), _p(codes), _p(scales))
+    assert rc == 0
+    return codes, scales
+
+
+def quantize_sr(desc, role, fmt, src, seed, block=(32, 32)):
+    """As quantize(), with the stochastic Round(.) of Eq. 6 (Sec. III-A: the gradient's rounding)."""
+    src = np.ascontiguousarray(src, dtype=np.float32)
+    assert src.shape == logical_shape(desc, role), (src.shape, logical_shape(desc, role))
+    assert np.isfinite(src).all(), "non-finite inputs are outside the contract"
+    cb, sb = qtensor_sizes(desc, role, fmt, block)
+    codes = np.zeros(cb, dtype=np.uint8)
+    scales = np.zeros(sb, dtype=np.uint8)
+    rc = _l().orc_quantize_sr(_p(_desc(desc)), role, fmt, block[0], block[1], _p(src), int(seed), _p(codes), _p(scales))
     assert rc == 0
     return codes, scales
 

@@ -102,6 +102,39 @@ int encode_elem(int fmt, double v) {
   return (sign << (f.bits - 1)) | best;
 }
 
+// ---- stochastic Round(.) of Eq. 6 (Sec. III-A: used for the gradient) ----------------------------
+// The paper names the rounding but no generator.  Reading taken: one draw per element from a counter-based
+// generator keyed by (seed, index of the element in the logical NCHW / OIHW tensor), so the result does not
+// depend on the order in which elements are visited; u = (top 23 bits + 1/2) / 2^23 lies strictly inside
+// (0, 1).  With lo <= |v| < hi the neighbouring grid magnitudes, the element becomes hi when
+// u < (|v| - lo) / (hi - lo) and lo otherwise: the expectation is |v| up to 2^-24 of a grid step, grid
+// values never move, and magnitudes at or beyond the largest finite one saturate as in round-to-nearest.
+uint32_t mix32(uint32_t x) {  // an invertible 32-bit finalizer: xor-shift, odd multiply, twice, xor-shift
+  x ^= x >> 16;
+  x *= 0x7FEB352Du;
+  x ^= x >> 15;
+  x *= 0x846CA68Bu;
+  x ^= x >> 16;
+  return x;
+}
+uint32_t sr_bits(uint64_t seed, uint64_t index) {
+  uint32_t key = mix32((uint32_t)seed ^ mix32((uint32_t)(seed >> 32) ^ mix32((uint32_t)(index >> 32))));
+  return mix32((uint32_t)index ^ key);
+}
+int encode_elem_sr(int fmt, double v, uint32_t bits) {
+  FmtInfo f = fmt_info(fmt);
+  int sign = std::signbit(v) ? 1 : 0;
+  double a = std::fabs(v);
+  if (a >= decode_mag(fmt, f.max_code)) return (sign << (f.bits - 1)) | f.max_code;  // saturation
+  int lo = 0;  // magnitudes grow with the code: the last code whose value does not exceed a
+  for (int m = 0; m <= f.max_code; ++m)
+    if (decode_mag(fmt, m) <= a) lo = m;
+  double vlo = decode_mag(fmt, lo), vhi = decode_mag(fmt, lo + 1);
+  double frac = (a - vlo) / (vhi - vlo);
+  double u = ((double)(bits >> 9) + 0.5) / 8388608.0;
+  return (sign << (f.bits - 1)) | (u < frac ? lo + 1 : lo);
+}
+
 // E8M0 code of a block: the role of Eq. 5 in the power-of-two form of the original MX format,
 // shared exponent = floor(log2(amax)) - emax_elem, biased by 127 and clamped to [0, 254].
 int scale_code(int fmt, double amax) {
@@ -174,6 +207,8 @@ int orc_num_threads() {
 double orc_decode_elem(int fmt, int code) { return decode_elem(fmt, code); }
 int orc_encode_elem(int fmt, double v) { return encode_elem(fmt, v); }
 int orc_scale_code(int fmt, double amax) { return scale_code(fmt, amax); }
+int orc_encode_elem_sr(int fmt, double v, uint32_t bits) { return encode_elem_sr(fmt, v, bits); }
+uint32_t orc_sr_bits(uint64_t seed, uint64_t index) { return sr_bits(seed, index); }
 
 int orc_out_hw(const int* d, int* ho, int* wo) {
   Conv c = conv_from(d);
@@ -194,7 +229,8 @@ int orc_qtensor_sizes(const int* d, int role, int fmt, int br, int bc, int64_t* 
 
 // Microscaling quantization (Sec. III-A, Eq. 5-6 in the E8M0 form), applied once to a tensor in
 // the 2-D view of Sec. IV-B.  src: fp32, NCHW (X, G_Y) or OIHW (W).  Padded channels get code 0.
-int orc_quantize(const int* d, int role, int fmt, int br, int bc, const float* src, uint8_t* codes, uint8_t* scales) {
+static int quantize_impl(const int* d, int role, int fmt, int br, int bc, const float* src, uint8_t* codes, uint8_t* scales, bool stochastic,
+                         uint64_t seed) {
   Conv cv = conv_from(d);
   View v = view_of(cv, role);
   if (bc <= 0 || br <= 0 || v.Cp % bc != 0) return 1;
@@ -221,12 +257,20 @@ int orc_quantize(const int* d, int role, int fmt, int br, int bc, const float* s
           for (int c = cb * bc; c < (cb + 1) * bc && c < v.C; ++c) {
             double x = (double)src[src_index(v, p, r, c)];
             double scaled = std::ldexp(x, 127 - sc);  // X_i / B_scale of Eq. 6, exact
-            put_code(codes, fmt, code_index(v, p, r, c), encode_elem(fmt, scaled));
+            int code = stochastic ? encode_elem_sr(fmt, scaled, sr_bits(seed, (uint64_t)src_index(v, p, r, c))) : encode_elem(fmt, scaled);
+            put_code(codes, fmt, code_index(v, p, r, c), code);
           }
       }
     }
   }
   return 0;
+}
+int orc_quantize(const int* d, int role, int fmt, int br, int bc, const float* src, uint8_t* codes, uint8_t* scales) {
+  return quantize_impl(d, role, fmt, br, bc, src, codes, scales, false, 0);
+}
+// The same with the stochastic Round(.) of Eq. 6; block scales are those of the deterministic quantizer.
+int orc_quantize_sr(const int* d, int role, int fmt, int br, int bc, const float* src, uint64_t seed, uint8_t* codes, uint8_t* scales) {
+  return quantize_impl(d, role, fmt, br, bc, src, codes, scales, true, seed);
 }
 
 // Fake quantization of Sec. III-A: element value times its block scale.  out: double, logical order.
