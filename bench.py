@@ -153,7 +153,8 @@ def run_ours(args):
     calls = [
         ("quantize_x", lambda: mq.quantize(d, roles[0], fmts[0], src[0], out=q[0])),
         ("quantize_w", lambda: mq.quantize(d, roles[1], fmts[1], src[1], out=q[1])),
-        ("quantize_dy", lambda: mq.quantize(d, roles[2], fmts[2], src[2], out=q[2])),
+        ("quantize_dy", (lambda: mq.quantize_sr(d, roles[2], fmts[2], src[2], 1234, out=q[2])) if args.dy_rounding == "stochastic" else
+         (lambda: mq.quantize(d, roles[2], fmts[2], src[2], out=q[2]))),
         ("cbf_im2col", lambda: mq.cbf_im2col(d, q[0], ic, isc)),
         ("conv_fwd", lambda: mq.conv_fwd(d, q[0], q[1], y=y, workspace=ws)),
         ("conv_bwd_data", lambda: mq.conv_bwd_data(d, q[1], q[2], dx=dx, workspace=ws)),
@@ -223,7 +224,8 @@ def run_ours(args):
     calls_cl = [
         ("quantize_x", lambda: mq.quantize(d, roles[0], fmts[0], src_cl[0], out=q[0], src_layout=mq.HWNC)),
         ("quantize_w", lambda: mq.quantize(d, roles[1], fmts[1], src_cl[1], out=q[1], src_layout=mq.HWNC)),
-        ("quantize_dy", lambda: mq.quantize(d, roles[2], fmts[2], src_cl[2], out=q[2], src_layout=mq.HWNC)),
+        ("quantize_dy", (lambda: mq.quantize_sr(d, roles[2], fmts[2], src_cl[2], 1234, out=q[2], src_layout=mq.HWNC)) if args.dy_rounding == "stochastic"
+         else (lambda: mq.quantize(d, roles[2], fmts[2], src_cl[2], out=q[2], src_layout=mq.HWNC))),
         ("cbf_im2col", lambda: mq.cbf_im2col(d, q[0], ic, isc)),
         ("conv_fwd", lambda: mq.conv_fwd(d, q[0], q[1], y=y_cl, layout=mq.HWNC, workspace=ws)),
         ("conv_bwd_data", lambda: mq.conv_bwd_data(d, q[1], q[2], dx=dx_cl, layout=mq.HWNC, workspace=ws)),
@@ -334,7 +336,7 @@ def run_ours(args):
         "value": value, "unit": "TFLOPS", "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "+".join(FMT_NAME[f] for f in fmts) + " (fp32 accumulate)", "data": "synthetic",
-        "config": {"workload": args.workload, "layer": dict(d._asdict()), "formats": [FMT_NAME[f] for f in fmts],
+        "config": {"workload": args.workload, "layer": dict(d._asdict()), "formats": [FMT_NAME[f] for f in fmts], "dy_rounding": args.dy_rounding,
                    "global_batch": d.N * world, "parallelism": "dp%d" % world if world > 1 else "single", "l2": "flushed between steps (512 MiB write)"},
         "clocks": clocks,
         "e2e": {"value": flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOPS", "ms_per_step": e2e_ms,
@@ -456,6 +458,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--dy-rounding", default="nearest", choices=["nearest", "stochastic"],
+                    help="rounding of the gradient's quantizer in the device-timed step (the host-buffer call keeps nearest)")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
     if args.impl == "reference":

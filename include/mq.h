@@ -101,6 +101,18 @@ mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt
  * Non-finite inputs are outside the contract (result unspecified, no fault). */
 mq_status mq_quantize(const mq_conv_desc* desc, const void* src, int src_layout, mq_qtensor* dst, void* stream);
 
+/* mq_quantize_sr -- the same quantizer with the STOCHASTIC Round(.) of Eq. 6, which Sec. III-A assigns to the
+ * gradient (activations and weights keep round-to-nearest); any role is accepted.  Tile scales are those of
+ * mq_quantize.  Per element: with lo <= |x * 2^(127 - code)| < hi the neighbouring magnitudes of the element
+ * format, the result is hi when u < (|x * 2^(127 - code)| - lo) / (hi - lo) and lo otherwise, sign kept; values on
+ * the grid never move and magnitudes at or beyond the largest finite one saturate.  The paper names no generator;
+ * here u = (top 23 bits of r + 1/2) / 2^23 with r = mix(low32(i) ^ key), key = mix(low32(seed) ^ mix(high32(seed) ^
+ * mix(high32(i)))), i the element's index in the logical tensor ([N][C][H][W] / [C_out][C_in][Kh][Kw] order, for
+ * either src_layout) and mix(x): x ^= x >> 16; x *= 0x7FEB352D; x ^= x >> 15; x *= 0x846CA68B; x ^= x >> 16 on
+ * 32 bits.  The stored tensor is therefore a pure function of (src, seed): the same for both source layouts, on
+ * every launch and on any number of GPUs.  Arguments, layouts and errors as for mq_quantize. */
+mq_status mq_quantize_sr(const mq_conv_desc* desc, const void* src, int src_layout, mq_qtensor* dst, unsigned long long seed, void* stream);
+
 /* mq_cbf_im2col -- channel-batch-first im2col (Sec. IV-A) of the quantized activation `xq` (role X):
  * row (kh,kw,c), column (ho,wo,n) of X' is the stored code at pixel (ho*stride+kh-pad,
  * wo*stride+kw-pad); tile scales are gathered alongside; out-of-image taps are zero bytes (codes

@@ -654,7 +654,8 @@ mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt
   return MQ_OK;
 }
 
-mq_status mq_quantize(const mq_conv_desc* desc, const void* src, int src_layout, mq_qtensor* dst, void* stream) {
+static mq_status quantize_impl(const mq_conv_desc* desc, const void* src, int src_layout, mq_qtensor* dst, int sr, unsigned long long seed,
+                               void* stream) {
   mq_status st = check_desc(desc);
   if (st != MQ_OK) return st;
   if (!src || !dst || !valid_role(dst->role)) return MQ_ERR_INVALID_ARG;
@@ -682,8 +683,19 @@ mq_status mq_quantize(const mq_conv_desc* desc, const void* src, int src_layout,
     if (dst->role == MQ_ROLE_W) { a.src_stride_p = v.C; a.src_stride_r = v.P * v.C; }
     else { a.src_stride_p = v.R * v.C; a.src_stride_r = v.C; }
   }
+  a.sr = sr;
+  a.sr_seed_lo = (unsigned)seed; a.sr_seed_hi = (unsigned)(seed >> 32);
+  a.sr_key0 = sr_mix32(a.sr_seed_lo ^ sr_mix32(a.sr_seed_hi ^ sr_mix32(0u)));
   cudaError_t e = launch_quantize(a, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
+}
+
+mq_status mq_quantize(const mq_conv_desc* desc, const void* src, int src_layout, mq_qtensor* dst, void* stream) {
+  return quantize_impl(desc, src, src_layout, dst, 0, 0ull, stream);
+}
+
+mq_status mq_quantize_sr(const mq_conv_desc* desc, const void* src, int src_layout, mq_qtensor* dst, unsigned long long seed, void* stream) {
+  return quantize_impl(desc, src, src_layout, dst, 1, seed, stream);
 }
 
 mq_status mq_cbf_im2col(const mq_conv_desc* desc, const mq_qtensor* xq, void* cols_codes, uint8_t* cols_scales, void* stream) {

@@ -56,7 +56,16 @@ struct QuantArgs {
   // source strides in floats when the source has the channel axis fastest (fp32 [H][W][N][C] / [Cout][Kh][Kw][Cin]):
   // element (p, r, c) at p * src_stride_p + r * src_stride_r + c; both zero for the NCHW / OIHW source
   long long src_stride_p, src_stride_r;
+  // stochastic rounding (Eq. 6 with the stochastic Round(.), Sec. III-A): 0 = round to nearest even
+  int sr;
+  unsigned sr_seed_lo, sr_seed_hi;   // the 64-bit seed
+  unsigned sr_key0;                  // stream key of elements whose index is below 2^32 (computed on the host)
 };
+// invertible 32-bit mixer (xor-shift, odd multiply, twice, xor-shift) behind the per-element draws
+__host__ __device__ __forceinline__ unsigned sr_mix32(unsigned x) {
+  x ^= x >> 16; x *= 0x7FEB352Du; x ^= x >> 15; x *= 0x846CA68Bu; x ^= x >> 16;
+  return x;
+}
 cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s);
 
 struct Im2colArgs {

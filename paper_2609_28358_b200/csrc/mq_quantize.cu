@@ -39,6 +39,31 @@ __device__ __forceinline__ unsigned encode2(float lo, float hi) {
   }
 }
 
+// Stochastic Round(.) of Eq. 6 (Sec. III-A: the gradient's rounding).  x is the scaled element, idx its index in the
+// logical NCHW / OIHW tensor.  The element's draw is 32 bits of a counter-based generator keyed by (seed, idx);
+// u = (top 23 bits + 1/2) / 2^23.  With lo <= |x| < hi neighbours on the format's grid, the result is hi when
+// u < (|x| - lo) / (hi - lo), else lo -- returned as a float that lies on the grid, so the round-to-nearest
+// conversion that follows is exact.  Everything below is exact in fp32: |x| / step has at most 24 significant bits,
+// its fractional part and (23-bit draw + 1/2) likewise.  Magnitudes at or beyond the largest one are left to the
+// conversion's saturation.
+template <int FMT>
+__device__ __forceinline__ float sr_value(float x, unsigned long long idx, const QuantArgs& a) {
+  constexpr int M = (FMT == MQ_E4M3 || FMT == MQ_E2M3) ? 3 : (FMT == MQ_E2M1 ? 1 : 2);                      // mantissa bits
+  constexpr int EMIN = FMT == MQ_E4M3 ? -6 : (FMT == MQ_E5M2 ? -14 : (FMT == MQ_E3M2 ? -2 : 0));           // smallest normal exponent
+  const float maxv = FMT == MQ_E4M3 ? 448.f : (FMT == MQ_E5M2 ? 57344.f : (FMT == MQ_E2M1 ? 6.f : (FMT == MQ_E3M2 ? 28.f : 7.5f)));
+  const float ax = fabsf(x);
+  if (!(ax < maxv)) return x;
+  const int ex = max((int)(__float_as_uint(ax) >> 23) - 127, EMIN);
+  const float inv_step = __uint_as_float((unsigned)(127 - ex + M) << 23), step = __uint_as_float((unsigned)(127 + ex - M) << 23);
+  const float t = ax * inv_step;       // < 2^(M + 1)
+  const float fl = floorf(t);
+  const unsigned hi = (unsigned)(idx >> 32);
+  const unsigned key = hi == 0 ? a.sr_key0 : sr_mix32(a.sr_seed_lo ^ sr_mix32(a.sr_seed_hi ^ sr_mix32(hi)));
+  const unsigned r = sr_mix32((unsigned)idx ^ key);
+  const bool up = (t - fl) * 8388608.f > (float)(r >> 9) + 0.5f;
+  return copysignf((fl + (up ? 1.f : 0.f)) * step, x);
+}
+
 __device__ __forceinline__ int scale_code_of(unsigned amax_bits, int emax) {
   // floor(log2 amax) = biased exponent - 127 for normal amax; subnormal / zero amax clamps to 0
   const int e = (int)(amax_bits >> 23) - emax;
@@ -72,7 +97,7 @@ __device__ __forceinline__ Item item_of(unsigned it, int n_pstrips, int Ct) {
   return q;
 }
 
-template <int FMT, int NT>   // NT threads per block: 256 (two tile rows per thread) or 512 (one)
+template <int FMT, int NT, bool SR>   // NT threads per block: 256 (two tile rows per thread) or 512 (one); SR: stochastic rounding
 __global__ void __launch_bounds__(NT) quantize_pipe_kernel(QuantArgs a, int n_pstrips, int Ct, unsigned n_items) {
   constexpr int RI = 512 / NT;      // tile rows per thread
   constexpr int NW = NT / 32;       // warps
@@ -166,13 +191,21 @@ __global__ void __launch_bounds__(NT) quantize_pipe_kernel(QuantArgs a, int n_ps
       if (q.p0 + t < a.P)
         a.scales[(long long)(q.p0 + t) * a.sc_stride_p + (long long)q.rt * a.sc_stride_r + q.ct] = (uint8_t)scale_code_of(mm, fmt_emax(FMT));
     }
+    // index of element (row rs, channel 4 cq, position 4 quad) of this item in the logical tensor
+    const long long e_base = ((long long)(q.r0 + rs) * a.C + q.c0 + 4 * cq) * a.P + q.p0 + 4 * quad;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
       const float f = scale_factor(code[j]);
 #pragma unroll
       for (int i = 0; i < RI; ++i) {
-        const unsigned lo = encode2<FMT>(v[i][0][j] * f, v[i][1][j] * f);
-        const unsigned hi = encode2<FMT>(v[i][2][j] * f, v[i][3][j] * f);
+        float x[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          x[k] = v[i][k][j] * f;
+          if (SR) x[k] = sr_value<FMT>(x[k], (unsigned long long)(e_base + ((long long)(16 * i) * a.C + k) * a.P + j), a);
+        }
+        const unsigned lo = encode2<FMT>(x[0], x[1]);
+        const unsigned hi = encode2<FMT>(x[2], x[3]);
         uint8_t* dst = stage + ((4 * quad + j) * 32 + rs + 16 * i) * RB;
         if (FMT == MQ_E2M1) *reinterpret_cast<unsigned short*>(dst + 2 * cq) = (unsigned short)(lo | (hi << 8));
         else *reinterpret_cast<unsigned*>(dst + 4 * cq) = lo | (hi << 16);
@@ -204,7 +237,7 @@ __global__ void __launch_bounds__(NT) quantize_pipe_kernel(QuantArgs a, int n_ps
 }
 
 // Fallback for sources whose position axis is not a multiple of 4 elements (no 16-byte rows): one block per item.
-template <int FMT>
+template <int FMT, bool SR>
 __global__ void __launch_bounds__(QT_THREADS) quantize_simple_kernel(QuantArgs a, int n_pstrips, int Ct) {
   __shared__ __align__(16) unsigned red[8][2][4];
   __shared__ __align__(16) uint8_t stage[PS][32][32];   // one code per byte
@@ -258,7 +291,13 @@ __global__ void __launch_bounds__(QT_THREADS) quantize_simple_kernel(QuantArgs a
     const float f = scale_factor(code[j]);
 #pragma unroll
     for (int i = 0; i < 8; i += 2) {
-      const unsigned two = encode2<FMT>(v[i][j] * f, v[i + 1][j] * f);
+      float x0 = v[i][j] * f, x1 = v[i + 1][j] * f;
+      if (SR) {
+        const long long e0 = ((long long)(q.r0 + 4 * i + rsub) * a.C + (q.c0 + c)) * a.P + pq + j;
+        x0 = sr_value<FMT>(x0, (unsigned long long)e0, a);
+        x1 = sr_value<FMT>(x1, (unsigned long long)(e0 + 4ll * a.C * a.P), a);
+      }
+      const unsigned two = encode2<FMT>(x0, x1);
       unsigned lo, hi;
       if (FMT == MQ_E2M1) { lo = two & 0xF; hi = (two >> 4) & 0xF; }
       else { lo = two & 0xFF; hi = (two >> 8) & 0xFF; }
@@ -304,7 +343,7 @@ __global__ void __launch_bounds__(QT_THREADS) quantize_simple_kernel(QuantArgs a
 // (cq, rq) = (lane & 7, lane >> 3) loads 4 adjacent channels of rows rq, rq + 4, ... as one 128-bit load each (8 in
 // flight), the amax is a per-lane max plus one redux.sync, and the codes leave as 32-bit words (FP8) or, pairing
 // neighbouring lanes, 32-bit words of 8 E2M1 codes.  VEC = false takes any C and alignment with scalar loads.
-template <int FMT, bool VEC>
+template <int FMT, bool VEC, bool SR>
 __global__ void __launch_bounds__(256) quantize_cfast_kernel(QuantArgs a, unsigned Rt, unsigned Ct, unsigned n_items) {
   pdl_wait();
   const int lane = threadIdx.x & 31;
@@ -341,7 +380,13 @@ __global__ void __launch_bounds__(256) quantize_cfast_kernel(QuantArgs a, unsign
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int r = r0 + 4 * i;
-      const unsigned lo = encode2<FMT>(v[i].x * f, v[i].y * f), hi = encode2<FMT>(v[i].z * f, v[i].w * f);
+      float x[4] = {v[i].x * f, v[i].y * f, v[i].z * f, v[i].w * f};
+      if (SR) {
+        const long long e0 = ((long long)r * a.C + c0) * a.P + pos;    // index in the logical tensor, whatever the source order
+#pragma unroll
+        for (int k = 0; k < 4; ++k) x[k] = sr_value<FMT>(x[k], (unsigned long long)(e0 + (long long)k * a.P), a);
+      }
+      const unsigned lo = encode2<FMT>(x[0], x[1]), hi = encode2<FMT>(x[2], x[3]);
       const long long e = pbase + (long long)r * a.out_stride_r;
       if (FMT == MQ_E2M1) {
         const unsigned mine = lo | (hi << 8);                       // 4 codes; the odd lane's go above the even lane's
@@ -362,8 +407,12 @@ cudaError_t launch_q_cfast(const QuantArgs& a, int Ct, cudaStream_t s) {
   const bool vec = a.C % 4 == 0 && a.src_stride_p % 4 == 0 && a.src_stride_r % 4 == 0 && (reinterpret_cast<uintptr_t>(a.src) & 15) == 0;
   long long blocks = (items + 7) / 8;
   if (blocks > 148LL * 64) blocks = 148LL * 64;
-  if (vec) return launch_pdl(quantize_cfast_kernel<FMT, true>, dim3((unsigned)blocks), dim3(256), 0, s, a, (unsigned)Rt, (unsigned)Ct, (unsigned)items);
-  return launch_pdl(quantize_cfast_kernel<FMT, false>, dim3((unsigned)blocks), dim3(256), 0, s, a, (unsigned)Rt, (unsigned)Ct, (unsigned)items);
+  if (a.sr) {
+    if (vec) return launch_pdl(quantize_cfast_kernel<FMT, true, true>, dim3((unsigned)blocks), dim3(256), 0, s, a, (unsigned)Rt, (unsigned)Ct, (unsigned)items);
+    return launch_pdl(quantize_cfast_kernel<FMT, false, true>, dim3((unsigned)blocks), dim3(256), 0, s, a, (unsigned)Rt, (unsigned)Ct, (unsigned)items);
+  }
+  if (vec) return launch_pdl(quantize_cfast_kernel<FMT, true, false>, dim3((unsigned)blocks), dim3(256), 0, s, a, (unsigned)Rt, (unsigned)Ct, (unsigned)items);
+  return launch_pdl(quantize_cfast_kernel<FMT, false, false>, dim3((unsigned)blocks), dim3(256), 0, s, a, (unsigned)Rt, (unsigned)Ct, (unsigned)items);
 }
 
 constexpr size_t QPIPE_SMEM = 2 * QBUF_BYTES + PS * 32 * 32 + 16 * 2 * 4 * sizeof(unsigned);
@@ -371,15 +420,18 @@ constexpr size_t QPIPE_SMEM = 2 * QBUF_BYTES + PS * 32 * 32 + 16 * 2 * 4 * sizeo
 template <int FMT>
 cudaError_t launch_q(const QuantArgs& a, int n_pstrips, int Ct, long long n_items, bool vec, cudaStream_t s) {
   if (!vec) {
-    return launch_pdl(quantize_simple_kernel<FMT>, dim3((unsigned)n_items), dim3(QT_THREADS), 0, s, a, n_pstrips, Ct);
+    if (a.sr) return launch_pdl(quantize_simple_kernel<FMT, true>, dim3((unsigned)n_items), dim3(QT_THREADS), 0, s, a, n_pstrips, Ct);
+    return launch_pdl(quantize_simple_kernel<FMT, false>, dim3((unsigned)n_items), dim3(QT_THREADS), 0, s, a, n_pstrips, Ct);
   }
   static bool attr_set = false;
   static int ctas_per_sm = 2;   // 80 KB of shared memory per block
   static int nt = 256;   // 512-thread blocks measured slower: the kernel is bound by instruction issue
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(quantize_pipe_kernel<FMT, 256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QPIPE_SMEM);
+    cudaError_t e = cudaFuncSetAttribute(quantize_pipe_kernel<FMT, 256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QPIPE_SMEM);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(quantize_pipe_kernel<FMT, 512>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QPIPE_SMEM);
+    e = cudaFuncSetAttribute(quantize_pipe_kernel<FMT, 512, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QPIPE_SMEM);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(quantize_pipe_kernel<FMT, 256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QPIPE_SMEM);
     if (e != cudaSuccess) return e;
     const char* tv = std::getenv("MQ_QUANT_THREADS");
     if (tv && std::atoi(tv) == 512) nt = 512;
@@ -392,8 +444,9 @@ cudaError_t launch_q(const QuantArgs& a, int n_pstrips, int Ct, long long n_item
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   long long grid = (long long)sms * ctas_per_sm;
   if (grid > n_items) grid = n_items;
-  if (nt == 512) return launch_pdl(quantize_pipe_kernel<FMT, 512>, dim3((unsigned)grid), dim3(512), QPIPE_SMEM, s, a, n_pstrips, Ct, (unsigned)n_items);
-  return launch_pdl(quantize_pipe_kernel<FMT, 256>, dim3((unsigned)grid), dim3(256), QPIPE_SMEM, s, a, n_pstrips, Ct, (unsigned)n_items);
+  if (a.sr) return launch_pdl(quantize_pipe_kernel<FMT, 256, true>, dim3((unsigned)grid), dim3(256), QPIPE_SMEM, s, a, n_pstrips, Ct, (unsigned)n_items);
+  if (nt == 512) return launch_pdl(quantize_pipe_kernel<FMT, 512, false>, dim3((unsigned)grid), dim3(512), QPIPE_SMEM, s, a, n_pstrips, Ct, (unsigned)n_items);
+  return launch_pdl(quantize_pipe_kernel<FMT, 256, false>, dim3((unsigned)grid), dim3(256), QPIPE_SMEM, s, a, n_pstrips, Ct, (unsigned)n_items);
 }
 
 }  // namespace

@@ -114,6 +114,17 @@ def quantize(desc, role, fmt, src, out=None, src_layout=NCHW, stream=None):
     return out
 
 
+def quantize_sr(desc, role, fmt, src, seed, out=None, src_layout=NCHW, stream=None):
+    """mq_quantize_sr: as quantize(), with stochastic rounding of the elements (the gradient's rounding); `seed` is a 64-bit integer."""
+    assert src.is_cuda and src.dtype == torch.float32 and src.is_contiguous()
+    if out is None:
+        out = empty_qtensor(desc, role, fmt, src.device)
+    q = out._c()
+    _check("mq_quantize_sr", lib().mq_quantize_sr(ctypes.byref(_d(desc)), ctypes.c_void_p(src.data_ptr()), src_layout, ctypes.byref(q),
+                                                 ctypes.c_uint64(int(seed) & 0xFFFFFFFFFFFFFFFF), _stream(stream)))
+    return out
+
+
 def cbf_im2col(desc, xq, out_codes=None, out_scales=None, stream=None):
     """mq_cbf_im2col: stored quantized activation -> (codes, scales) of X'."""
     cb, sb = im2col_sizes(desc, xq.fmt)
