@@ -686,6 +686,7 @@ static mq_status quantize_impl(const mq_conv_desc* desc, const void* src, int sr
   a.sr = sr;
   a.sr_seed_lo = (unsigned)seed; a.sr_seed_hi = (unsigned)(seed >> 32);
   a.sr_key0 = sr_mix32(a.sr_seed_lo ^ sr_mix32(a.sr_seed_hi ^ sr_mix32(0u)));
+  a.sr_wide = ((unsigned long long)v.P * (unsigned long long)v.R * (unsigned long long)v.C >= (1ull << 32) || env_int("MQ_SR_WIDE", 0)) ? 1 : 0;
   cudaError_t e = launch_quantize(a, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }

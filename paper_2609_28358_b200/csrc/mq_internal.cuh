@@ -60,6 +60,7 @@ struct QuantArgs {
   int sr;
   unsigned sr_seed_lo, sr_seed_hi;   // the 64-bit seed
   unsigned sr_key0;                  // stream key of elements whose index is below 2^32 (computed on the host)
+  int sr_wide;                       // 1: the tensor has 2^32 elements or more (keys are derived per element)
 };
 // invertible 32-bit mixer (xor-shift, odd multiply, twice, xor-shift) behind the per-element draws
 __host__ __device__ __forceinline__ unsigned sr_mix32(unsigned x) {

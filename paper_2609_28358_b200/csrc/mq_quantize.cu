@@ -46,22 +46,37 @@ __device__ __forceinline__ unsigned encode2(float lo, float hi) {
 // conversion that follows is exact.  Everything below is exact in fp32: |x| / step has at most 24 significant bits,
 // its fractional part and (23-bit draw + 1/2) likewise.  Magnitudes at or beyond the largest one are left to the
 // conversion's saturation.
+// lo: low word of the element's index; key: the stream key of its high word (sr_key)
 template <int FMT>
-__device__ __forceinline__ float sr_value(float x, unsigned long long idx, const QuantArgs& a) {
+__device__ __forceinline__ float sr_value(float x, unsigned lo, unsigned key) {
   constexpr int M = (FMT == MQ_E4M3 || FMT == MQ_E2M3) ? 3 : (FMT == MQ_E2M1 ? 1 : 2);                      // mantissa bits
   constexpr int EMIN = FMT == MQ_E4M3 ? -6 : (FMT == MQ_E5M2 ? -14 : (FMT == MQ_E3M2 ? -2 : 0));           // smallest normal exponent
-  const float maxv = FMT == MQ_E4M3 ? 448.f : (FMT == MQ_E5M2 ? 57344.f : (FMT == MQ_E2M1 ? 6.f : (FMT == MQ_E3M2 ? 28.f : 7.5f)));
-  const float ax = fabsf(x);
-  if (!(ax < maxv)) return x;
-  const int ex = max((int)(__float_as_uint(ax) >> 23) - 127, EMIN);
-  const float inv_step = __uint_as_float((unsigned)(127 - ex + M) << 23), step = __uint_as_float((unsigned)(127 + ex - M) << 23);
-  const float t = ax * inv_step;       // < 2^(M + 1)
-  const float fl = floorf(t);
-  const unsigned hi = (unsigned)(idx >> 32);
-  const unsigned key = hi == 0 ? a.sr_key0 : sr_mix32(a.sr_seed_lo ^ sr_mix32(a.sr_seed_hi ^ sr_mix32(hi)));
-  const unsigned r = sr_mix32((unsigned)idx ^ key);
-  const bool up = (t - fl) * 8388608.f > (float)(r >> 9) + 0.5f;
-  return copysignf((fl + (up ? 1.f : 0.f)) * step, x);
+  // fp32 pattern of the largest magnitude: 448, 57344, 6, 28, 7.5
+  constexpr unsigned MAXBITS = FMT == MQ_E4M3 ? 0x43E00000u : (FMT == MQ_E5M2 ? 0x47600000u : (FMT == MQ_E2M1 ? 0x40C00000u : (FMT == MQ_E3M2 ? 0x41E00000u : 0x40F00000u)));
+  const unsigned b = __float_as_uint(x) & 0x7fffffffu;       // |x|; patterns of non-negative floats order like their values
+  const unsigned r23 = sr_mix32(lo ^ key) >> 9;
+  // normal range of the format: the grid keeps M mantissa bits of the fp32 pattern.  The dropped field f (23 - M bits)
+  // is the fraction of a step in units of 2^-(23 - M): f * 2^M > draw + 1/2 is an integer comparison, and stepping up
+  // is an integer addition on the pattern (the carry walks into the exponent at a binade's end).
+  constexpr unsigned MASK = (1u << (23 - M)) - 1u;
+  const unsigned f = b & MASK;
+  const unsigned q_norm = (b - f) + (((f << M) > r23) ? MASK + 1u : 0u);
+  // below it the step is the constant 2^(EMIN - M): t = |x| / step < 2^M, floor through a round-down addition of 2^23,
+  // draw + 1/2 as (2^23 + draw) - (2^23 - 1/2); all exact
+  const float t = __uint_as_float(b) * __uint_as_float((unsigned)(127 + M - EMIN) << 23);
+  const float fl = __fadd_rd(t, 8388608.f) - 8388608.f;
+  const float u = __uint_as_float(0x4B000000u | r23) - 8388607.5f;
+  const float up = (t - fl) * 8388608.f > u ? 1.f : 0.f;
+  const unsigned q_sub = __float_as_uint((fl + up) * __uint_as_float((unsigned)(127 + EMIN - M) << 23));
+  unsigned q = b >= ((unsigned)(127 + EMIN) << 23) ? q_norm : q_sub;
+  q = b < MAXBITS ? q : b;      // at or beyond the largest magnitude: left to the conversion's saturation
+  return __uint_as_float(q | (__float_as_uint(x) & 0x80000000u));
+}
+// Stream key of an element from the high word of its index; tensors below 2^32 elements (a.sr_wide == 0, uniform)
+// take the key computed on the host.
+__device__ __forceinline__ unsigned sr_key(const QuantArgs& a, long long idx) {
+  if (!a.sr_wide) return a.sr_key0;
+  return sr_mix32(a.sr_seed_lo ^ sr_mix32(a.sr_seed_hi ^ sr_mix32((unsigned)((unsigned long long)idx >> 32))));
 }
 
 __device__ __forceinline__ int scale_code_of(unsigned amax_bits, int emax) {
@@ -202,7 +217,10 @@ __global__ void __launch_bounds__(NT) quantize_pipe_kernel(QuantArgs a, int n_ps
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           x[k] = v[i][k][j] * f;
-          if (SR) x[k] = sr_value<FMT>(x[k], (unsigned long long)(e_base + ((long long)(16 * i) * a.C + k) * a.P + j), a);
+          if (SR) {
+            const unsigned e_lo = (unsigned)e_base + ((unsigned)(16 * i) * (unsigned)a.C + k) * (unsigned)a.P + j;   // low word, modular
+            x[k] = sr_value<FMT>(x[k], e_lo, sr_key(a, e_base + ((long long)(16 * i) * a.C + k) * a.P + j));
+          }
         }
         const unsigned lo = encode2<FMT>(x[0], x[1]);
         const unsigned hi = encode2<FMT>(x[2], x[3]);
@@ -294,8 +312,9 @@ __global__ void __launch_bounds__(QT_THREADS) quantize_simple_kernel(QuantArgs a
       float x0 = v[i][j] * f, x1 = v[i + 1][j] * f;
       if (SR) {
         const long long e0 = ((long long)(q.r0 + 4 * i + rsub) * a.C + (q.c0 + c)) * a.P + pq + j;
-        x0 = sr_value<FMT>(x0, (unsigned long long)e0, a);
-        x1 = sr_value<FMT>(x1, (unsigned long long)(e0 + 4ll * a.C * a.P), a);
+        const long long e1 = e0 + 4ll * a.C * a.P;
+        x0 = sr_value<FMT>(x0, (unsigned)e0, sr_key(a, e0));
+        x1 = sr_value<FMT>(x1, (unsigned)e1, sr_key(a, e1));
       }
       const unsigned two = encode2<FMT>(x0, x1);
       unsigned lo, hi;
@@ -384,7 +403,7 @@ __global__ void __launch_bounds__(256) quantize_cfast_kernel(QuantArgs a, unsign
       if (SR) {
         const long long e0 = ((long long)r * a.C + c0) * a.P + pos;    // index in the logical tensor, whatever the source order
 #pragma unroll
-        for (int k = 0; k < 4; ++k) x[k] = sr_value<FMT>(x[k], (unsigned long long)(e0 + (long long)k * a.P), a);
+        for (int k = 0; k < 4; ++k) x[k] = sr_value<FMT>(x[k], (unsigned)e0 + (unsigned)k * (unsigned)a.P, sr_key(a, e0 + (long long)k * a.P));
       }
       const unsigned lo = encode2<FMT>(x[0], x[1]), hi = encode2<FMT>(x[2], x[3]);
       const long long e = pbase + (long long)r * a.out_stride_r;

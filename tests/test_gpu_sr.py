@@ -37,6 +37,20 @@ def test_gradient_codes_match_the_oracle(name, shape, fmt):
 
 
 @pytest.mark.parametrize("fmt", [E4M3, E2M1])
+def test_per_element_key_path(fmt, monkeypatch):
+    """Tensors of 2^32 elements or more derive the stream key from the index's high word per element; forced here on a
+    small tensor (high word 0), where it must give the same bytes."""
+    monkeypatch.setenv("MQ_SR_WIDE", "1")
+    d = inputs.conv_desc(64, 96, 8, 8, 64, 3, 1, 1)
+    g = inputs.make_dy(d, 8, "gauss")
+    oc, osc = oracle.quantize_sr(d, oracle.ROLE_DY, fmt, g, 77)
+    for src, layout in ((g, mq.NCHW), (np.ascontiguousarray(g.transpose(2, 3, 0, 1)), mq.HWNC)):
+        q = mq.quantize_sr(d, mq.ROLE_DY, fmt, dev(src), 77, src_layout=layout)
+        assert_same_bytes(q.codes, oc, "codes")
+        assert_same_bytes(q.scales, osc, "scales")
+
+
+@pytest.mark.parametrize("fmt", [E4M3, E2M1])
 def test_every_role_accepts_it(fmt):
     d = inputs.conv_desc(36, 40, 6, 6, 72, 3, 1, 1)
     x, w, g = inputs.make_x(d, 3, "gauss"), inputs.make_w(d, 3), inputs.make_dy(d, 3, "small")
