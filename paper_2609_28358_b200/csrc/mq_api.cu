@@ -188,7 +188,9 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   // staging only in the whole-tile kernel, whose pipeline is short; the per-tap kernel keeps its stages
   const bool tma_store_ok = (op == MQ_OP_FWD || (g.sh == 1 && g.sw == 1)) && p.TW >= 4 && p.TW <= 32 &&
                             (layout == MQ_NCHW ? p.Wd % 4 == 0 : (p.Cd % 4 == 0 && p.BN % 64 == 0));   // [H][W][N][C]: whole 32-channel groups per column half
-  p.tma_store = tma_store_ok && env_int("MQ_TC_TMA_STORE", 0) ? 1 : 0;
+  // ... and for 1x1 layers, whose main loop is a handful of stages: the tile's time is its store (measured 4-12 % faster, 28x28 and
+  // 56x56 images, 256 and 512 channels)
+  p.tma_store = tma_store_ok && (env_int("MQ_TC_TMA_STORE", 0) || (taps == 1 && !env_int("MQ_TC_NO_TMA_STORE", 0))) ? 1 : 0;
   const size_t stage_bytes = 128 * 128 + (size_t)p.BN * 128 + 3072;
   int stages = (int)((227 * 1024 - 2048 - (p.tma_store ? 65536 : 0)) / stage_bytes);
   if (stages > 8) stages = 8;

@@ -30,6 +30,7 @@ SMALL_SHAPES = [
     ("stride2", (33, 64, 9, 11, 40, 3, 2, 1)),     # odd image, stride 2
     ("k1", (36, 40, 6, 6, 72, 1, 1, 0)),           # 1x1
     ("k1s2", (32, 32, 8, 8, 32, 1, 2, 0)),         # 1x1 stride 2
+    ("k1_w8", (40, 128, 6, 8, 160, 1, 1, 0)),      # 1x1 with rows of whole 16-byte units: staged stores, clipped channel tile and samples
     ("k5", (8, 16, 12, 12, 24, 5, 2, 2)),          # 5x5, C < 32
     ("nopad", (16, 32, 7, 7, 32, 3, 1, 0)),        # no padding
     ("rect", (4, 35, 6, 10, 33, 3, 1, 1)),
@@ -151,7 +152,7 @@ def test_config3_layers_full_size(li):
 
 CFG5_POINTS = ["cfg5_e4m3_k3s1_c64_hw14", "cfg5_e4m3_k3s2_c128_hw28", "cfg5_e4m3_k1s1_c256_hw14", "cfg5_e2m1_k3s1_c128_hw14",
                "cfg5_e2m1_k1s2_c64_hw28", "cfg5_e2m1_k3s2_c256_hw14", "cfg5_e4m3_k3s1_c512_hw14", "cfg5_e4m3_k3s1_c64_hw56",
-               "cfg5_e2m1_k3s1_c256_hw14"]
+               "cfg5_e2m1_k3s1_c256_hw14", "cfg5_e4m3_k1s1_c256_hw28"]
 
 
 @pytest.mark.parametrize("name", CFG5_POINTS)
