@@ -112,6 +112,8 @@ struct WgradTcParams {
   int mma_cp;           // E2M1: 1 = the MMA lane issues the scale copies itself (no copier warp)
   int cta2;             // 1: pairs of blocks (clusters of 2) compute 256 x 256 tiles with cta_group::2 MMAs
   int TG;               // taps per block: 1, or Kw (flat mode: the taps of a kernel row share the stage's pixels)
+  int grp8;             // 8-bit operands, 32 or 64 bytes of input channels, unit strides: the Kw taps of a kernel row are one wide B operand
+                        // (TG = Kw, b_rows = Cp) whose panels are views of one loaded strip of KPX + Kw - 1 pixels, one pixel apart
   int NB;               // 128-row chunks of the group's B rows = ceil(TG * b_rows / 128)
   int n0, n1;           // MMA widths per K slice: n0 = min(TG * b_rows, 256) and the rest (0: one MMA)
   int b_tile_bytes;     // bytes of X loaded per stage: b_rows * 128, flat mode (KPX + TG - 1) * b_rows * KBn

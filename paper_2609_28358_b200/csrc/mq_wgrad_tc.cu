@@ -85,10 +85,14 @@ __device__ __forceinline__ void expand_wgrad_scales_body(const WgradTcParams& p,
       const int nc = (int)(idx % p.nchunks); idx /= p.nchunks;
       const int wp = (int)(idx % p.Wp); idx /= p.Wp;
       const int hp = (int)(idx % p.Hp); const int cb = (int)(idx / p.Hp);
-      const int cib = (cb * p.b_rows + c * 128 + 32 * j) / 32;
-      if (b < NBS && cib < p.Ct) {
+      // rows of the chunk: input channels of one tap, or (grouped thin mode) tap-in-row major, input channel minor - tap tj
+      // reads the pixel tj further along the row
+      const int row0 = c * 128 + 32 * j;
+      const int tj = p.grp8 ? row0 / p.b_rows : 0;
+      const int cib = p.grp8 ? (row0 - tj * p.b_rows) / 32 : (cb * p.b_rows + row0) / 32;
+      if (b < NBS && cib < p.Ct && tj < p.TG) {
         const int px = b / p.BPP, nb = nc * p.BPP + (b - px * p.BPP);
-        const int h = hp - p.ph, w = wp - p.pw + px * p.sw;
+        const int h = hp - p.ph, w = wp - p.pw + px * p.sw + tj;
         if (nb < p.Nt && h >= 0 && h < p.H && w >= 0 && w < p.W) v = __ldg(p.x_scales + (((long long)h * p.W + w) * p.Nt + nb) * p.Ct + cib);
       }
     } else {
@@ -223,7 +227,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const uint32_t sfb_bytes = (uint32_t)p.NB * 512 * SPA;
     const uint8_t* sfb_src = p.sfb_img + (((size_t)cb * (taps / TG) + tgi) * p.stages_total + st_begin) * sfb_bytes;
     const uint32_t a_bytes = 128 * 128, b_step = (uint32_t)p.b_rows * 128;
-    const uint32_t b_bytes = p.mode == MQ_WG_FP8 ? 128u * 128u : (uint32_t)p.b_tile_bytes;   // per loader
+    const uint32_t b_bytes = (p.mode == MQ_WG_FP8 && !p.grp8) ? 128u * 128u : (uint32_t)p.b_tile_bytes;   // per loader
     const uint8_t* ga = nullptr; const uint8_t* gb = nullptr;
     if (p.mode == MQ_WG_FP4_FLAT) {
       ga = p.gt + (size_t)mt * p.gt_block_bytes + (size_t)st_begin * a_bytes;
@@ -301,7 +305,11 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const uint32_t fp4_layout = p.KBn == 128 ? 2u : (p.KBn == 64 ? 4u : (p.KBn == 32 ? 6u : 0u));
       const uint32_t a_piece = 128 * p.KBn, b_piece = (uint32_t)p.b_rows * p.KBn;
       const uint64_t a_desc0 = smem_desc(FP4 ? smem_desc_base(a_piece, 8 * p.KBn, fp4_layout) : smem_desc_base(128 * 128, 1024, 2), smem_u32(smem));
-      const uint64_t b_desc0 = smem_desc(FP4 ? smem_desc_base(b_piece, 8 * p.KBn, fp4_layout) : smem_desc_base(128 * 128, 1024, 2), smem_u32(smem + b_off));
+      // grouped thin mode: MN-major panels of Cp bytes (swizzle span Cp), a tap's panel one pixel (32 BPP rows) after the
+      // previous tap's, 8-row groups 8 Cp bytes apart
+      const uint64_t b_desc0 = smem_desc(FP4 ? smem_desc_base(b_piece, 8 * p.KBn, fp4_layout)
+                                             : (p.grp8 ? smem_desc_base(32 * p.BPP * p.Cp, 8 * p.Cp, p.Cp == 64 ? 4u : 6u) : smem_desc_base(128 * 128, 1024, 2)),
+                                         smem_u32(smem + b_off));
       const uint32_t stage16 = (uint32_t)stage_bytes >> 4;
       // The taps of a group are ONE wide B operand: tap j's view starts j pieces (= b_rows / 8 row groups) further,
       // which is exactly where rows [j * b_rows, (j + 1) * b_rows) of a (TG * b_rows)-row operand lie.  At most two
@@ -315,7 +323,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (FP4) {
           const int piece = (32 * a) / p.KBn, off = (32 * a) % p.KBn;
           ka16[a] = (piece * a_piece + off) >> 4; kb16[a] = (piece * b_piece + off) >> 4;
-        } else { ka16[a] = 256u * a; kb16[a] = 256u * a; }
+        } else { ka16[a] = 256u * a; kb16[a] = p.grp8 ? (uint32_t)(a * 32 * p.Cp) >> 4 : 256u * a; }   // 32 K rows per MMA
       }
       const uint32_t sf_base = tmem + acc_cols;
       const uint64_t sf_desc0 = smem_desc(smem_desc_base(0, 128, 0), smem_u32(smem + sf_off));
@@ -374,7 +382,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
               const uint32_t accu = a > 0 ? 1u : accumulate;
               const uint32_t id = idesc_n[0] | ((uint32_t)a << 4) | ((uint32_t)a << 29);
               if (CTA2) mma_mxf8f6f4_2(tmem, ad + 256u * a, bd + 256u * a, id, sf_t, sf_t + 8, accu);
-              else mma_mxf8f6f4(tmem, ad + 256u * a, bd + 256u * a, id, sf_t, sf_t + 8, accu);
+              else mma_mxf8f6f4(tmem, ad + 256u * a, bd + kb16[a], id, sf_t, sf_t + 8, accu);
             }
             if (CTA2) tc_commit_2_multicast(&empty[s], 3); else tc_commit(&empty[s]);
             WTRACE(3, i);
