@@ -433,8 +433,9 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   // fill.  Instead the Kw taps of a kernel row form one B operand of Kw * Cp rows: a stage loads a strip of
   // KPX + Kw - 1 pixels once ([pixel][sample][Cp bytes], swizzle span = Cp) and tap kw's panel is that strip one pixel
   // further - Kw times fewer stages, G_Y loads and MMA instructions.
-  p.grp8 = (fp8 && !p.cta2 && g.sh == 1 && g.sw == 1 && g.Kw > 1 && (g.Cp == 32 || g.Cp == 64) && g.Kw * g.Cp <= 256 &&
-            !env_int("MQ_WGRAD_NO_GROUP8", 0)) ? 1 : 0;
+  // (With a column stride the strip is the contiguous run of (KPX - 1) sw + Kw input pixels: output pixel a's tap kw is
+  // input pixel a sw + kw of the strip, so panels stay one pixel apart and K slices sw pixels apart.)
+  p.grp8 = (fp8 && !p.cta2 && g.Kw > 1 && (g.Cp == 32 || g.Cp == 64) && g.Kw * g.Cp <= 256 && !env_int("MQ_WGRAD_NO_GROUP8", 0)) ? 1 : 0;
   if (p.grp8) p.b_rows = g.Cp;
   p.cb_tiles = (g.Cp + p.b_rows - 1) / p.b_rows;
   // taps per block: a whole kernel row in the flat mode when its accumulators fit in tensor memory
@@ -452,7 +453,7 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   if (splits < 1) splits = 1;
   p.splits = splits;
   p.b_tile_bytes = flat ? (p.KPX + p.TG - 1) * p.b_rows * p.KBn : (p.cta2 ? 128 : p.b_rows) * 128;   // a pair's blocks load half of X each
-  if (p.grp8) p.b_tile_bytes = (p.KPX + p.TG - 1) * 32 * p.BPP * g.Cp;
+  if (p.grp8) p.b_tile_bytes = ((p.KPX - 1) * g.sw + p.TG) * 32 * p.BPP * g.Cp;
   p.stage_bytes = (128 * 128 + p.b_tile_bytes + (1 + p.NB) * 1024 + 1023) / 1024 * 1024;
   {
     int st = (227 * 1024 - 2048) / p.stage_bytes;
@@ -544,8 +545,8 @@ mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const 
       const uint64_t dims[4] = {rb, (uint64_t)g.N, (uint64_t)g.W, (uint64_t)g.H};
       const uint64_t strides[3] = {rb, (uint64_t)g.N * rb, (uint64_t)g.W * g.N * rb};
       uint32_t box[4] = {128u, (uint32_t)(p.BPP * 32), (uint32_t)((p.KPX - 1) * g.sw + 1), 1u};
-      const uint32_t es[4] = {1u, 1u, (uint32_t)g.sw, 1u};
-      if (p.grp8) { box[0] = (uint32_t)g.Cp; box[2] = (uint32_t)(p.KPX + p.TG - 1); }   // the strip of a kernel row's taps, rows of Cp bytes
+      uint32_t es[4] = {1u, 1u, (uint32_t)g.sw, 1u};
+      if (p.grp8) { box[0] = (uint32_t)g.Cp; box[2] = (uint32_t)((p.KPX - 1) * g.sw + p.TG); es[2] = 1u; }   // the contiguous strip of a kernel row's taps, rows of Cp bytes
       if (!encode_tensor_map_u8(&map_b, x_codes, 4, dims, strides, box, es, p.grp8 ? g.Cp : 128)) return MQ_ERR_CUDA;
     }
   }

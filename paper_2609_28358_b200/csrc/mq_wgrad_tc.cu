@@ -323,7 +323,11 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
         if (FP4) {
           const int piece = (32 * a) / p.KBn, off = (32 * a) % p.KBn;
           ka16[a] = (piece * a_piece + off) >> 4; kb16[a] = (piece * b_piece + off) >> 4;
-        } else { ka16[a] = 256u * a; kb16[a] = p.grp8 ? (uint32_t)(a * 32 * p.Cp) >> 4 : 256u * a; }   // 32 K rows per MMA
+        } else {
+          ka16[a] = 256u * a;      // 32 K rows of 128 bytes per MMA
+          // grouped thin mode: K slice a = (output pixel a / BPP, sample block a % BPP); its first tap's pixel lies sw strip pixels per output pixel on
+          kb16[a] = p.grp8 ? (uint32_t)(((a / p.BPP) * p.sw * p.BPP + (a % p.BPP)) * 32 * p.Cp) >> 4 : 256u * a;
+        }
       }
       const uint32_t sf_base = tmem + acc_cols;
       const uint64_t sf_desc0 = smem_desc(smem_desc_base(0, 128, 0), smem_u32(smem + sf_off));
