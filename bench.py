@@ -178,6 +178,32 @@ def run_ours(args):
     sampler = ClockSampler(local)
     sampler.start()
 
+    # Optionally the step's launches are captured once into a CUDA graph and replayed: the same kernels with the same
+    # arguments, without the per-call host work (small layers are bound by it).  Single GPU only; any failure to
+    # capture falls back to plain launches and is reported.
+    run_step, graph_note, launches_per_step = step, "off", None
+    if args.cuda_graph and world == 1:
+        try:
+            c0 = mq.kernel_launch_count()
+            side = torch.cuda.Stream()
+            side.wait_stream(torch.cuda.current_stream())
+            with torch.cuda.stream(side):
+                step()
+            torch.cuda.current_stream().wait_stream(side)
+            torch.cuda.synchronize()
+            launches_per_step = mq.kernel_launch_count() - c0
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(graph):
+                step()
+            graph.replay()
+            torch.cuda.synchronize()
+            if mq.last_device_status() != 0:
+                raise RuntimeError("device status after replay")
+            run_step, graph_note = graph.replay, "on"
+        except Exception as exc:  # noqa: BLE001
+            torch.cuda.synchronize()
+            run_step, graph_note, launches_per_step = step, f"capture failed ({type(exc).__name__}), plain launches", None
+
     # ---- timed region: K steps, L2 flushed between steps (flush outside the event pairs)
     K = args.steps
     ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
@@ -186,10 +212,12 @@ def run_ours(args):
     for s, e in ev:
         flush.zero_()
         s.record()
-        step()
+        run_step()
         e.record()
     barrier()
     launches = mq.kernel_launch_count() - launches0   # kernels of this library inside the timed region
+    if launches_per_step is not None:
+        launches = launches_per_step * K               # replayed launches are not counted by the library's host-side counter
     ms_total = sum(s.elapsed_time(e) for s, e in ev)
 
     # ---- per-call durations over K more steps (same stream, same flush), for the roofline
@@ -336,7 +364,7 @@ def run_ours(args):
         "value": value, "unit": "TFLOPS", "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "+".join(FMT_NAME[f] for f in fmts) + " (fp32 accumulate)", "data": "synthetic",
-        "config": {"workload": args.workload, "layer": dict(d._asdict()), "formats": [FMT_NAME[f] for f in fmts], "dy_rounding": args.dy_rounding,
+        "config": {"workload": args.workload, "layer": dict(d._asdict()), "formats": [FMT_NAME[f] for f in fmts], "dy_rounding": args.dy_rounding, "cuda_graph": graph_note,
                    "global_batch": d.N * world, "parallelism": "dp%d" % world if world > 1 else "single", "l2": "flushed between steps (512 MiB write)"},
         "clocks": clocks,
         "e2e": {"value": flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOPS", "ms_per_step": e2e_ms,
@@ -458,6 +486,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="config2")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--cuda-graph", action="store_true", help="replay the step's launches from a CUDA graph (single GPU)")
     ap.add_argument("--dy-rounding", default="nearest", choices=["nearest", "stochastic"],
                     help="rounding of the gradient's quantizer in the device-timed step (the host-buffer call keeps nearest)")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
