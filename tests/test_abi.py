@@ -77,6 +77,13 @@ def test_bad_arguments_are_rejected_on_the_host(mq):
     assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), 0, ctypes.byref(q), None) == 3  # alignment
     q = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 0)
     assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), 7, ctypes.byref(q), None) == 1  # no such source layout
+    # the stochastic-rounding entry point validates the same way (the seed is any 64-bit value)
+    seed = ctypes.c_uint64(0xFFFFFFFFFFFFFFFF)
+    assert L.mq_quantize_sr(ctypes.byref(good), None, 0, ctypes.byref(q), seed, None) == 1
+    assert L.mq_quantize_sr(ctypes.byref(good), ctypes.c_void_p(0x3000), 7, ctypes.byref(q), seed, None) == 1
+    assert L.mq_quantize_sr(ctypes.byref(good), ctypes.c_void_p(0x3004), 0, ctypes.byref(q), seed, None) == 3
+    small = mq._QTensor(0x1000, 0x2000, 16, 16, 0, 2)
+    assert L.mq_quantize_sr(ctypes.byref(good), ctypes.c_void_p(0x3000), 0, ctypes.byref(small), seed, None) == 4
     assert L.mq_cbf_im2col(ctypes.byref(good), ctypes.byref(q), None, None, None) == 1
     qw = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 1)
     assert L.mq_conv_fwd(ctypes.byref(good), ctypes.byref(qw), ctypes.byref(qw), ctypes.c_void_p(0x4000), 0, None, 0, None) == 1  # wrong role
