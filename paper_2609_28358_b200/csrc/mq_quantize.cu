@@ -100,7 +100,7 @@ template <int N>
 __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory"); }
 
 struct Item { int p0, r0, c0, rt, ct; };
-__device__ __forceinline__ Item item_of(unsigned it, int n_pstrips, int Ct) {
+__device__ __forceinline__ Item item_of(unsigned it, int n_pstrips, int Ct, int psi = PS) {
   // channel tile fastest: the tiles that share an output line ([n][c] rows are c-contiguous) are produced
   // together, so full 128-byte lines reach L2 at about the same time; then position strip, then row tile
   Item q;
@@ -108,11 +108,14 @@ __device__ __forceinline__ Item item_of(unsigned it, int n_pstrips, int Ct) {
   q.ct = (int)(it - u * (unsigned)Ct);
   q.rt = (int)(u / (unsigned)n_pstrips);
   const int ps = (int)(u - (unsigned)q.rt * (unsigned)n_pstrips);
-  q.p0 = ps * PS; q.r0 = q.rt * 32; q.c0 = q.ct * 32;
+  q.p0 = ps * psi; q.r0 = q.rt * 32; q.c0 = q.ct * 32;
   return q;
 }
 
-template <int FMT, int NT, bool SR>   // NT threads per block: 256 (two tile rows per thread) or 512 (one); SR: stochastic rounding
+// R16 (tensors of at most 16 rows, e.g. a batch of 16 samples; NT = 256): the upper half of the 32-row tile would be
+// padding, so an item takes 16 positions instead - buffer rows 16..31 hold rows 0..15 of the next eight positions - and
+// every amax, scale and slab below is per (half, position).
+template <int FMT, int NT, bool SR, bool R16 = false>   // NT threads per block: 256 (two tile rows per thread) or 512 (one); SR: stochastic rounding
 __global__ void __launch_bounds__(NT) quantize_pipe_kernel(QuantArgs a, int n_pstrips, int Ct, unsigned n_items) {
   constexpr int RI = 512 / NT;      // tile rows per thread
   constexpr int NW = NT / 32;       // warps
@@ -137,15 +140,21 @@ __global__ void __launch_bounds__(NT) quantize_pipe_kernel(QuantArgs a, int n_ps
   const unsigned ld_dst = (unsigned)(ld_row * 32 + (ld_row >> 2) * 16 + ld_qd * 16);   // + m * RSTEP * (32 * 32 + 8 * 16)
   const long long row_step = (long long)RSTEP * a.C * a.P;   // floats between a thread's consecutive chunks
   auto issue = [&](unsigned it, uint8_t* buf) -> Item {
-    const Item q = item_of(it, n_pstrips, Ct);
+    const Item q = item_of(it, n_pstrips, Ct, R16 ? 2 * PS : PS);
     const int pq = q.p0 + 4 * ld_qd;
     const bool col_ok = (q.c0 + ld_cc) < a.C && pq < a.P;
     const float* src = a.src + ((long long)(q.r0 + ld_rr) * a.C + (q.c0 + ld_cc)) * a.P + pq;
     const int rows_left = a.R - q.r0 - ld_rr;     // tile row 4 m is valid while 4 m < rows_left
 #pragma unroll
     for (int m = 0; m < CPT; ++m) {
-      const bool ok = col_ok && RSTEP * m < rows_left;
-      cp_async16(buf + ld_dst + m * RSTEP * (32 * 32 + 8 * 16), ok ? src + m * row_step : a.src, ok);
+      if (R16) {
+        // buffer row ld_rr + 4 m: tensor row (ld_rr + 4 m) & 15 at the positions of half m >> 2
+        const bool ok = (q.c0 + ld_cc) < a.C && pq + PS * (m >> 2) < a.P && RSTEP * (m & 3) < rows_left;
+        cp_async16(buf + ld_dst + m * RSTEP * (32 * 32 + 8 * 16), ok ? src + (m & 3) * row_step + PS * (m >> 2) : a.src, ok);
+      } else {
+        const bool ok = col_ok && RSTEP * m < rows_left;
+        cp_async16(buf + ld_dst + m * RSTEP * (32 * 32 + 8 * 16), ok ? src + m * row_step : a.src, ok);
+      }
     }
     cp_async_commit();
     return q;
@@ -175,34 +184,44 @@ __global__ void __launch_bounds__(NT) quantize_pipe_kernel(QuantArgs a, int n_ps
       }
     // amax per position on the bit patterns of |x| (order-preserving): thread, then the 16 lanes that share
     // this position quad (lane bits 0,1,2,4), then the 8 warps
-    unsigned m4[4];
+    // HV = 1: one amax per position over both of the thread's rows; R16: one per (half, position)
+    constexpr int HV = R16 ? RI : 1;
+    unsigned m4[HV][4];
 #pragma unroll
-    for (int j = 0; j < 4; ++j) {
-      float fm = 0.f;
+    for (int h = 0; h < HV; ++h)
 #pragma unroll
-      for (int i = 0; i < RI; ++i)
+      for (int j = 0; j < 4; ++j) {
+        float fm = 0.f;
 #pragma unroll
-        for (int k = 0; k < 4; ++k) fm = fmaxf(fm, fabsf(v[i][k][j]));
-      m4[j] = __reduce_max_sync(quad_mask, __float_as_uint(fm));
+        for (int i = 0; i < RI; ++i)
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            if (!R16 || i == h) fm = fmaxf(fm, fabsf(v[i][k][j]));
+        m4[h][j] = __reduce_max_sync(quad_mask, __float_as_uint(fm));
+      }
+    if ((lane & 23) == 0) {   // lanes 0 (quad 0) and 8 (quad 1)
+#pragma unroll
+      for (int h = 0; h < HV; ++h)
+        *reinterpret_cast<uint4*>(&red[((warp * 2 + quad) * HV + h) * 4]) = make_uint4(m4[h][0], m4[h][1], m4[h][2], m4[h][3]);
     }
-    if ((lane & 23) == 0)   // lanes 0 (quad 0) and 8 (quad 1)
-      *reinterpret_cast<uint4*>(&red[(warp * 2 + quad) * 4]) = make_uint4(m4[0], m4[1], m4[2], m4[3]);
     __syncthreads();
-    int code[4];
-    {
+    int code[HV][4];
+#pragma unroll
+    for (int h = 0; h < HV; ++h) {
       uint4 mx = make_uint4(0, 0, 0, 0);
 #pragma unroll
       for (int w = 0; w < NW; ++w) {
-        const uint4 r4 = *reinterpret_cast<const uint4*>(&red[(w * 2 + quad) * 4]);
+        const uint4 r4 = *reinterpret_cast<const uint4*>(&red[((w * 2 + quad) * HV + h) * 4]);
         mx.x = max(mx.x, r4.x); mx.y = max(mx.y, r4.y); mx.z = max(mx.z, r4.z); mx.w = max(mx.w, r4.w);
       }
-      code[0] = scale_code_of(mx.x, fmt_emax(FMT)); code[1] = scale_code_of(mx.y, fmt_emax(FMT));
-      code[2] = scale_code_of(mx.z, fmt_emax(FMT)); code[3] = scale_code_of(mx.w, fmt_emax(FMT));
+      code[h][0] = scale_code_of(mx.x, fmt_emax(FMT)); code[h][1] = scale_code_of(mx.y, fmt_emax(FMT));
+      code[h][2] = scale_code_of(mx.z, fmt_emax(FMT)); code[h][3] = scale_code_of(mx.w, fmt_emax(FMT));
     }
-    if (t < PS) {
+    if (t < PS * HV) {       // position t of the item: half t >> 3 (R16), quad (t >> 2) & 1, j = t & 3
+      const int h = t >> 3, qd = (t >> 2) & 1;
       unsigned mm = 0;
 #pragma unroll
-      for (int w = 0; w < NW; ++w) mm = max(mm, red[(w * 2 + (t >> 2)) * 4 + (t & 3)]);
+      for (int w = 0; w < NW; ++w) mm = max(mm, red[((w * 2 + qd) * HV + h) * 4 + (t & 3)]);
       if (q.p0 + t < a.P)
         a.scales[(long long)(q.p0 + t) * a.sc_stride_p + (long long)q.rt * a.sc_stride_r + q.ct] = (uint8_t)scale_code_of(mm, fmt_emax(FMT));
     }
@@ -210,21 +229,22 @@ __global__ void __launch_bounds__(NT) quantize_pipe_kernel(QuantArgs a, int n_ps
     const long long e_base = ((long long)(q.r0 + rs) * a.C + q.c0 + 4 * cq) * a.P + q.p0 + 4 * quad;
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
-      const float f = scale_factor(code[j]);
 #pragma unroll
       for (int i = 0; i < RI; ++i) {
+        const float f = scale_factor(code[R16 ? i : 0][j]);
         float x[4];
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           x[k] = v[i][k][j] * f;
           if (SR) {
-            const unsigned e_lo = (unsigned)e_base + ((unsigned)(16 * i) * (unsigned)a.C + k) * (unsigned)a.P + j;   // low word, modular
-            x[k] = sr_value<FMT>(x[k], e_lo, sr_key(a, e_base + ((long long)(16 * i) * a.C + k) * a.P + j));
+            // the thread's second row: 16 tensor rows on, or (R16) the same row eight positions on
+            const long long e_off = R16 ? (long long)k * a.P + j + PS * i : ((long long)(16 * i) * a.C + k) * a.P + j;
+            x[k] = sr_value<FMT>(x[k], (unsigned)e_base + (unsigned)e_off, sr_key(a, e_base + e_off));   // low word: modular arithmetic
           }
         }
         const unsigned lo = encode2<FMT>(x[0], x[1]);
         const unsigned hi = encode2<FMT>(x[2], x[3]);
-        uint8_t* dst = stage + ((4 * quad + j) * 32 + rs + 16 * i) * RB;
+        uint8_t* dst = R16 ? stage + ((PS * i + 4 * quad + j) * 16 + rs) * RB : stage + ((4 * quad + j) * 32 + rs + 16 * i) * RB;
         if (FMT == MQ_E2M1) *reinterpret_cast<unsigned short*>(dst + 2 * cq) = (unsigned short)(lo | (hi << 8));
         else *reinterpret_cast<unsigned*>(dst + 4 * cq) = lo | (hi << 16);
       }
@@ -232,19 +252,19 @@ __global__ void __launch_bounds__(NT) quantize_pipe_kernel(QuantArgs a, int n_ps
     __syncthreads();
     // copy out: per position a 32(r) x 32(c) slab; rows are contiguous runs of the stored tensor
     if (FMT == MQ_E2M1) {
-      const int p = t >> 5, r = t & 31;   // 256 rows of 16 bytes
+      const int p = R16 ? t >> 4 : t >> 5, r = R16 ? t & 15 : t & 31;   // 256 rows of 16 bytes: [position][row]
       if (t < 256 && q.p0 + p < a.P && q.r0 + r < a.R) {
-        const uint4 val = *reinterpret_cast<const uint4*>(stage + (p * 32 + r) * 16);
+        const uint4 val = *reinterpret_cast<const uint4*>(stage + t * 16);
         const long long e = (long long)(q.p0 + p) * a.out_stride_p + (long long)(q.r0 + r) * a.out_stride_r + q.c0;
         *reinterpret_cast<uint4*>(a.codes + (e >> 1)) = val;
       }
     } else {
 #pragma unroll
       for (int k = 0; k < 512 / NT; ++k) {
-        const int id = t + NT * k;  // 512 chunks of 16 bytes
-        const int p = id >> 6, r = (id >> 1) & 31, half = id & 1;
+        const int id = t + NT * k;  // 512 chunks of 16 bytes: [position][row][half]
+        const int p = R16 ? id >> 5 : id >> 6, r = R16 ? (id >> 1) & 15 : (id >> 1) & 31, half = id & 1;
         if (q.p0 + p < a.P && q.r0 + r < a.R) {
-          const uint4 val = *reinterpret_cast<const uint4*>(stage + (p * 32 + r) * 32 + 16 * half);
+          const uint4 val = *reinterpret_cast<const uint4*>(stage + id * 16);
           const long long e = (long long)(q.p0 + p) * a.out_stride_p + (long long)(q.r0 + r) * a.out_stride_r + q.c0 + 16 * half;
           *reinterpret_cast<uint4*>(a.codes + e) = val;
         }
@@ -437,7 +457,7 @@ cudaError_t launch_q_cfast(const QuantArgs& a, int Ct, cudaStream_t s) {
 constexpr size_t QPIPE_SMEM = 2 * QBUF_BYTES + PS * 32 * 32 + 16 * 2 * 4 * sizeof(unsigned);
 
 template <int FMT>
-cudaError_t launch_q(const QuantArgs& a, int n_pstrips, int Ct, long long n_items, bool vec, cudaStream_t s) {
+cudaError_t launch_q(const QuantArgs& a, int n_pstrips, int Ct, long long n_items, bool vec, bool r16, cudaStream_t s) {
   if (!vec) {
     if (a.sr) return launch_pdl(quantize_simple_kernel<FMT, true>, dim3((unsigned)n_items), dim3(QT_THREADS), 0, s, a, n_pstrips, Ct);
     return launch_pdl(quantize_simple_kernel<FMT, false>, dim3((unsigned)n_items), dim3(QT_THREADS), 0, s, a, n_pstrips, Ct);
@@ -452,6 +472,10 @@ cudaError_t launch_q(const QuantArgs& a, int n_pstrips, int Ct, long long n_item
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(quantize_pipe_kernel<FMT, 256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QPIPE_SMEM);
     if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(quantize_pipe_kernel<FMT, 256, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QPIPE_SMEM);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(quantize_pipe_kernel<FMT, 256, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QPIPE_SMEM);
+    if (e != cudaSuccess) return e;
     const char* tv = std::getenv("MQ_QUANT_THREADS");
     if (tv && std::atoi(tv) == 512) nt = 512;
     const char* v = std::getenv("MQ_QUANT_CTAS");
@@ -463,6 +487,8 @@ cudaError_t launch_q(const QuantArgs& a, int n_pstrips, int Ct, long long n_item
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   long long grid = (long long)sms * ctas_per_sm;
   if (grid > n_items) grid = n_items;
+  if (r16 && a.sr) return launch_pdl(quantize_pipe_kernel<FMT, 256, true, true>, dim3((unsigned)grid), dim3(256), QPIPE_SMEM, s, a, n_pstrips, Ct, (unsigned)n_items);
+  if (r16) return launch_pdl(quantize_pipe_kernel<FMT, 256, false, true>, dim3((unsigned)grid), dim3(256), QPIPE_SMEM, s, a, n_pstrips, Ct, (unsigned)n_items);
   if (a.sr) return launch_pdl(quantize_pipe_kernel<FMT, 256, true>, dim3((unsigned)grid), dim3(256), QPIPE_SMEM, s, a, n_pstrips, Ct, (unsigned)n_items);
   if (nt == 512) return launch_pdl(quantize_pipe_kernel<FMT, 512, false>, dim3((unsigned)grid), dim3(512), QPIPE_SMEM, s, a, n_pstrips, Ct, (unsigned)n_items);
   return launch_pdl(quantize_pipe_kernel<FMT, 256, false>, dim3((unsigned)grid), dim3(256), QPIPE_SMEM, s, a, n_pstrips, Ct, (unsigned)n_items);
@@ -471,11 +497,14 @@ cudaError_t launch_q(const QuantArgs& a, int n_pstrips, int Ct, long long n_item
 }  // namespace
 
 cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s) {
-  const int n_pstrips = (a.P + PS - 1) / PS;
+  const bool vec = (a.P % 4 == 0) && ((reinterpret_cast<uintptr_t>(a.src) & 15) == 0);
+  // at most 16 rows (e.g. a batch of 16 samples): items of 16 positions, see quantize_pipe_kernel
+  const bool r16 = vec && a.src_stride_r == 0 && a.R <= 16 && !std::getenv("MQ_QUANT_NO_R16");
+  const int psi = r16 ? 2 * PS : PS;
+  const int n_pstrips = (a.P + psi - 1) / psi;
   const int Rt = (a.R + 31) / 32, Ct = a.Cp / 32;
   const long long n_items = (long long)n_pstrips * Rt * Ct;
   if (n_items <= 0 || n_items > 0x7fffffffLL) return cudaErrorInvalidValue;
-  const bool vec = (a.P % 4 == 0) && ((reinterpret_cast<uintptr_t>(a.src) & 15) == 0);
   cudaError_t e;
   if (a.src_stride_r != 0) {   // channel-fastest source
     switch (a.fmt) {
@@ -490,11 +519,11 @@ cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s) {
     return e;
   }
   switch (a.fmt) {
-    case MQ_E4M3: e = launch_q<MQ_E4M3>(a, n_pstrips, Ct, n_items, vec, s); break;
-    case MQ_E5M2: e = launch_q<MQ_E5M2>(a, n_pstrips, Ct, n_items, vec, s); break;
-    case MQ_E2M1: e = launch_q<MQ_E2M1>(a, n_pstrips, Ct, n_items, vec, s); break;
-    case MQ_E3M2: e = launch_q<MQ_E3M2>(a, n_pstrips, Ct, n_items, vec, s); break;
-    case MQ_E2M3: e = launch_q<MQ_E2M3>(a, n_pstrips, Ct, n_items, vec, s); break;
+    case MQ_E4M3: e = launch_q<MQ_E4M3>(a, n_pstrips, Ct, n_items, vec, r16, s); break;
+    case MQ_E5M2: e = launch_q<MQ_E5M2>(a, n_pstrips, Ct, n_items, vec, r16, s); break;
+    case MQ_E2M1: e = launch_q<MQ_E2M1>(a, n_pstrips, Ct, n_items, vec, r16, s); break;
+    case MQ_E3M2: e = launch_q<MQ_E3M2>(a, n_pstrips, Ct, n_items, vec, r16, s); break;
+    case MQ_E2M3: e = launch_q<MQ_E2M3>(a, n_pstrips, Ct, n_items, vec, r16, s); break;
     default: return cudaErrorInvalidValue;
   }
   count_launches(1);

@@ -17,6 +17,8 @@ SHAPES = [
     ("ragged", (40, 48, 5, 6, 70, 3, 1, 1)),       # 30 positions: scalar-load kernel
     ("aligned", (64, 96, 8, 8, 64, 3, 1, 1)),      # 64 positions: the pipelined kernel, several tiles
     ("stride2", (33, 64, 9, 11, 40, 3, 2, 1)),     # ragged N and C_out
+    ("small_batch", (16, 48, 6, 8, 40, 3, 1, 1)),  # at most 16 samples: the 16-positions-per-item variant of the pipelined kernel
+    ("tiny_batch", (5, 20, 8, 8, 24, 3, 1, 1)),    # the same with ragged rows, channels and a partial last item
 ]
 
 
