@@ -38,6 +38,7 @@ SMALL_SHAPES = [
     ("wide_thin", (16, 160, 6, 8, 32, 3, 1, 1)),   # the same situation in the input gradient
     ("wide", (32, 256, 4, 8, 288, 3, 1, 1)),       # 256-channel MMAs (8-bit) and a remainder channel tile
     ("deep_batch", (250, 320, 3, 4, 288, 3, 1, 1)),  # 8 sample tiles (ragged): E2M1 whole-line re-layout with partial channel groups, block pairs
+    ("thin_n70", (70, 48, 5, 6, 40, 3, 1, 1)),       # thin layer, three sample tiles in one four-block K stage (one pixel per stage)
     ("stem7", (8, 3, 20, 20, 24, 7, 2, 3)),          # 7x7 stride-2 stem on 3 channels: seven taps of 32 bytes as one weight-gradient operand
     ("batch16", (16, 40, 10, 12, 72, 3, 1, 1)),      # at most 16 samples: quantizer items of 16 positions (120 positions: partial last item)
     ("shared_rows", (70, 128, 5, 6, 256, 3, 1, 1)),  # 128-byte K chunks, unit strides: activation-side scale chunks shared across output rows (ragged N, W)
