@@ -287,8 +287,14 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
     p.b_scales = qw->scales;
   } else {
     uint8_t* wt_scales = base + pl.off_wt_scales;
-    if (launch_weight_transpose(static_cast<const uint8_t*>(qw->codes), qw->scales, base, wt_scales, g, qw->fmt, stream) != cudaSuccess)
+    // per-tap kernel, operands that need no repacking: the re-layout rides in the scale-expansion launch
+    p.wt_fused = (!p.halo && !fmt_is_6bit(qw->fmt) && !env_int("MQ_TC_NO_WT_FUSED", 0)) ? 1 : 0;
+    if (p.wt_fused) {
+      p.wt_in = static_cast<const uint8_t*>(qw->codes); p.wt_out = base; p.wt_sc_in = qw->scales;
+      p.wt_Cout = g.Cout; p.wt_Cop = g.Cop; p.wt_Cp = g.Cp; p.wt_bx = g.Cp / 32; p.wt_by = g.Cop / 32;
+    } else if (launch_weight_transpose(static_cast<const uint8_t*>(qw->codes), qw->scales, base, wt_scales, g, qw->fmt, stream) != cudaSuccess) {
       return MQ_ERR_CUDA;
+    }
     b_codes = base;
     p.b_scales = wt_scales;
   }

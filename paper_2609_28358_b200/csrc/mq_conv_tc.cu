@@ -1163,6 +1163,40 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 template <int MODE, int KB, bool FP4>
 __global__ void __launch_bounds__(256) expand_conv_scales_kernel(const ConvTcParams p, unsigned n_tile_m) {
   pdl_wait();
+  if (p.wt_fused && blockIdx.x >= p.expand_blocks) {
+    // W -> W^T codes, one 32 x 32 (c_in, c_out) block of one tap per thread block (the work of weight_transpose_kernel)
+    __shared__ uint8_t tile[32][33];  // [ci][co]
+    unsigned b = blockIdx.x - p.expand_blocks;
+    const int bx = (int)(b % (unsigned)p.wt_bx); b /= (unsigned)p.wt_bx;
+    const int by = (int)(b % (unsigned)p.wt_by);
+    const int tap = (int)(b / (unsigned)p.wt_by);
+    const int taps = p.Kh * p.Kw, fp4 = FP4 ? 1 : 0;
+    const int co0 = by * 32, ci0 = bx * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;  // 32 x 8
+    for (int r = ty; r < 32; r += 8) {
+      const int co = co0 + r, ci = ci0 + tx;
+      uint8_t v = 0;
+      if (co < p.wt_Cout) {
+        const long long e = ((long long)co * taps + tap) * p.wt_Cp + ci;
+        v = fp4 ? (uint8_t)((p.wt_in[e >> 1] >> ((e & 1) * 4)) & 0xF) : p.wt_in[e];
+      }
+      tile[tx][r] = v;
+    }
+    __syncthreads();
+    if (!fp4) {
+      for (int r = ty; r < 32; r += 8) {
+        const int ci = ci0 + r, co = co0 + tx;
+        p.wt_out[((long long)ci * taps + tap) * p.wt_Cop + co] = tile[r][tx];
+      }
+    } else {
+      for (int idx = ty * 32 + tx; idx < 32 * 16; idx += 256) {
+        const int rr = idx >> 4, bb = idx & 15;
+        const int ci = ci0 + rr, co = co0 + 2 * bb;
+        p.wt_out[(((long long)ci * taps + tap) * p.wt_Cop + co) >> 1] = (uint8_t)(tile[rr][2 * bb] | (tile[rr][2 * bb + 1] << 4));
+      }
+    }
+    return;
+  }
   constexpr int G = 128 / KB, APC = KB / 32, SPA = FP4 ? 2 : 1, BPC = APC * SPA;
   const int lane = threadIdx.x & 31;
   const unsigned wid = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
@@ -1278,8 +1312,19 @@ __global__ void __launch_bounds__(256) expand_conv_scales_kernel(const ConvTcPar
         const int tap = tap_index(tw, pos);
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
-          if (j < 4 * atoms_b && 32 * j < p.BN && tile.c0 + 32 * j < p.Cd)
-            acc[j] |= load_scale_bytes<BPC>(p.b_scales + ((long long)((tile.c0 >> 5) + j) * taps_all + tap) * p.Kblocks + pos.cc * BPC) << (8 * c * BPC);
+          if (j < 4 * atoms_b && 32 * j < p.BN && tile.c0 + 32 * j < p.Cd) {
+            if (p.wt_fused) {
+              // from the stored (not re-laid) weight scales: K-block kb is output-channel block kb of [C_out/32][taps][C_in_p/32]
+              const int cib = (tile.c0 >> 5) + j, Ct_w = p.wt_Cp >> 5;
+              unsigned long long bytes = 0;
+#pragma unroll
+              for (int kb = 0; kb < BPC; ++kb)
+                bytes |= (unsigned long long)__ldg(p.wt_sc_in + ((long long)(pos.cc * BPC + kb) * taps_all + tap) * Ct_w + cib) << (8 * kb);
+              acc[j] |= bytes << (8 * c * BPC);
+            } else {
+              acc[j] |= load_scale_bytes<BPC>(p.b_scales + ((long long)((tile.c0 >> 5) + j) * taps_all + tap) * p.Kblocks + pos.cc * BPC) << (8 * c * BPC);
+            }
+          }
         }
       }
     }
@@ -1426,6 +1471,12 @@ cudaError_t launch_expand_inst(const ConvTcParams& p, cudaStream_t s) {
   if (p.halo) warps += ((unsigned long long)p.tiles_c * p.Kh * p.Kw * p.BN * (KB / 16) + 31) / 32;
   const unsigned blocks = (unsigned)((warps + 7) / 8);
   count_launches(1);
+  if (p.wt_fused) {
+    ConvTcParams q = p;
+    q.expand_blocks = blocks;
+    const unsigned extra = (unsigned)(p.wt_bx * p.wt_by * p.Kh * p.Kw);
+    return launch_pdl(expand_conv_scales_kernel<MODE, KB, FP4>, dim3(blocks + extra), dim3(256), 0, s, q, n_tile_m);
+  }
   return launch_pdl(expand_conv_scales_kernel<MODE, KB, FP4>, dim3(blocks), dim3(256), 0, s, p, n_tile_m);
 }
 

@@ -61,6 +61,14 @@ struct ConvTcParams {
   const uint8_t* b_codes;   // weight-like codes [rows][taps][b_rowbytes] (source of the images below)
   int b_rows_total, b_rowbytes;
   uint8_t* b_img;           // [channel tile][tap][BN rows][KB], each row stored with the KB-byte swizzle applied
+  // input gradient, per-tap kernel: the weight re-layout W -> W^T rides in the scale-expansion launch (extra blocks) and the
+  // B-side chunks are gathered from the ORIGINAL tile scales, so the call needs one preparation launch instead of two
+  int wt_fused;             // 1: on
+  const uint8_t* wt_in;     // stored W codes [C_out][taps][C_in_p]
+  uint8_t* wt_out;          // re-laid codes [C_in_p][taps][C_out_p]
+  const uint8_t* wt_sc_in;  // stored W tile scales [C_out/32][taps][C_in_p/32]
+  int wt_Cout, wt_Cop, wt_Cp, wt_bx, wt_by;   // channel counts; 32 x 32 blocks along C_in_p and C_out_p
+  unsigned expand_blocks;   // blocks of the launch that expand scale chunks (the re-layout blocks follow)
   // output
   float* out;
   int out_layout;
