@@ -148,8 +148,10 @@ mq_status mq_conv_bwd_data(const mq_conv_desc* desc, const mq_qtensor* wq, const
  * is launched (for scale: N=32, 128->64 channels, 80x80, 3x3 needs about 6 MB).
  * The call performs no cudaMalloc / cudaFree and calls no allocating library routine.
  *
- * First use on a device: the first call made while a given device is current looks up the array's device
- * address (once per device, kept for later calls).  Make that first call outside of any stream capture.
+ * Arguments are checked exactly as by mq_conv_bwd_data (same codes), then the size limit.
+ * First use on a device: every call looks up the array's device address for the current device (nothing is
+ * cached, so a cudaDeviceReset between calls is harmless); the first such lookup on a device may load the
+ * library's device code, so make the first call outside of any stream capture.
  * Sharing: all calls on a device use the same array and it keeps whatever the previous call left in it;
  * each call overwrites every byte it later reads, so nothing needs clearing, but two calls whose kernels
  * overlap on the GPU (different streams, no ordering between them) race on the array -- order them. */

@@ -582,28 +582,33 @@ mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const 
   return launch_bwd_weight_reduce(partial, out, g, p.splits, layout, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }
 
-// address of the current device's status word (a __device__ variable has one instance per device)
+// address of the current device's status word (a __device__ variable has one instance per device and per context:
+// looked up on every call, a host-side table lookup, so that no address outlives a cudaDeviceReset)
 unsigned int* device_status_ptr() {
-  static unsigned int* ptrs[64] = {nullptr};
-  int dev = 0;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
-  if (!ptrs[dev]) {
-    void* q = nullptr;
-    if (cudaGetSymbolAddress(&q, g_device_status) == cudaSuccess) ptrs[dev] = static_cast<unsigned int*>(q);
-  }
-  return ptrs[dev];
+  void* q = nullptr;
+  if (cudaGetSymbolAddress(&q, g_device_status) != cudaSuccess) return nullptr;
+  return static_cast<unsigned int*>(q);
 }
 
-mq_status run_conv(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int role_a, const mq_qtensor* qb, int role_b,
-                   void* out, int layout, void* ws, size_t ws_bytes, void* stream) {
+// argument checks common to the three convolution entry points (everything but the workspace)
+mq_status check_conv_args(const mq_conv_desc* desc, const mq_qtensor* qa, int role_a, const mq_qtensor* qb, int role_b, const void* out, int layout) {
   mq_status st = check_desc(desc);
   if (st != MQ_OK) return st;
-  Geom g = make_geom(*desc);
+  const Geom g = make_geom(*desc);
   if ((st = check_qtensor(g, qa, role_a)) != MQ_OK) return st;
   if ((st = check_qtensor(g, qb, role_b)) != MQ_OK) return st;
   if (!out) return MQ_ERR_INVALID_ARG;
   if (layout != MQ_NCHW && layout != MQ_HWNC) return MQ_ERR_INVALID_ARG;
-  if (!aligned16(out) || (ws && !aligned16(ws))) return MQ_ERR_ALIGNMENT;
+  if (!aligned16(out)) return MQ_ERR_ALIGNMENT;
+  return MQ_OK;
+}
+
+mq_status run_conv(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int role_a, const mq_qtensor* qb, int role_b,
+                   void* out, int layout, void* ws, size_t ws_bytes, void* stream) {
+  mq_status st = check_conv_args(desc, qa, role_a, qb, role_b, out, layout);
+  if (st != MQ_OK) return st;
+  Geom g = make_geom(*desc);
+  if (ws && !aligned16(ws)) return MQ_ERR_ALIGNMENT;
   size_t need = 0;
   mq_workspace_size(desc, op, qa->fmt, qb->fmt, &need);
   if (need > 0 && (!ws || ws_bytes < need)) return MQ_ERR_BUFFER_TOO_SMALL;
@@ -752,29 +757,23 @@ mq_status mq_conv_bwd_weight(const mq_conv_desc* desc, const mq_qtensor* xq, con
 
 // ---- allocation-free variant of mq_conv_bwd_data ---------------------------------------------------
 // Scratch for callers that cannot allocate: a static array in the device image.  In host code the name
-// below is only a handle for the runtime, not a device address; the address is looked up once per device
-// with cudaGetSymbolAddress (with that device current) and that pointer is what the kernels receive.
+// below is only a handle for the runtime, not a device address; the address is looked up with
+// cudaGetSymbolAddress (with the caller's device current) and that pointer is what the kernels receive.
+// The lookup is repeated on every call - after the first one on a device, which may load the module, it is a
+// host-side table lookup - so no cached address can outlive a cudaDeviceReset of its context.
 static __device__ __align__(256) unsigned char g_static_scratch[MQ_STATIC_SCRATCH_BYTES];
-static void* g_static_scratch_addr[64] = {};
 
 mq_status mq_conv_bwd_data_static(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, void* dx, int dx_layout,
                                   void* stream) {
-  mq_status st = check_desc(desc);
+  // the ordinary call's argument checks first, so that a bad argument is reported as such whatever the layer's size
+  mq_status st = check_conv_args(desc, wq, MQ_ROLE_W, dyq, MQ_ROLE_DY, dx, dx_layout);
   if (st != MQ_OK) return st;
-  if (!wq || !dyq) return MQ_ERR_INVALID_ARG;
-  if (!valid_fmt(wq->fmt) || !valid_fmt(dyq->fmt)) return MQ_ERR_INVALID_ARG;
   size_t need = 0;
   if ((st = mq_workspace_size(desc, MQ_OP_BWD_DATA, wq->fmt, dyq->fmt, &need)) != MQ_OK) return st;
   if (need > MQ_STATIC_SCRATCH_BYTES) return MQ_ERR_STATIC_SCRATCH;
-  int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess) return MQ_ERR_CUDA;
-  if (dev < 0 || dev >= 64) return MQ_ERR_UNSUPPORTED;
-  if (!g_static_scratch_addr[dev]) {
-    void* addr = nullptr;
-    if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || !addr) return MQ_ERR_CUDA;
-    g_static_scratch_addr[dev] = addr;
-  }
-  return run_conv(MQ_OP_BWD_DATA, desc, wq, MQ_ROLE_W, dyq, MQ_ROLE_DY, dx, dx_layout, g_static_scratch_addr[dev], MQ_STATIC_SCRATCH_BYTES, stream);
+  void* addr = nullptr;
+  if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || !addr) return MQ_ERR_CUDA;
+  return run_conv(MQ_OP_BWD_DATA, desc, wq, MQ_ROLE_W, dyq, MQ_ROLE_DY, dx, dx_layout, addr, MQ_STATIC_SCRATCH_BYTES, stream);
 }
 
 namespace {

@@ -36,27 +36,53 @@ def out_hw(d):
     return ((d.H + 2 * d.pad_h - d.Kh) // d.stride_h + 1, (d.W + 2 * d.pad_w - d.Kw) // d.stride_w + 1)
 
 
-def _rng(seed, name):
-    return np.random.Generator(np.random.Philox(key=[int(seed), _TENSOR_IDS[name]]))
+def _rng(seed, name, part=0):
+    return np.random.Generator(np.random.Philox(key=[int(seed), _TENSOR_IDS[name] + 16 * int(part)]))
+
+
+_BIG = 1 << 26   # tensors of this many elements or more are drawn slice by slice along their first axis, in parallel
+
+
+def _draw(seed, name, shape, fn):
+    """`fn(generator, shape)` over the whole tensor from one stream, or - for big tensors - over each slice of the
+    first axis from a stream of its own (key: seed, tensor name, slice index), drawn by a thread pool.  Either way
+    the tensor is a pure function of (seed, name, shape)."""
+    n = int(np.prod(shape))
+    if n < _BIG or shape[0] < 2:
+        return fn(_rng(seed, name), shape)
+    from concurrent.futures import ThreadPoolExecutor
+    import os
+
+    out = np.empty(shape, dtype=np.float32)
+
+    def one(i):
+        out[i] = fn(_rng(seed, name, i + 1), shape[1:])
+
+    with ThreadPoolExecutor(max_workers=min(32, os.cpu_count() or 1)) as ex:
+        list(ex.map(one, range(shape[0])))
+    return out
 
 
 def make_x(d, seed, kind="relu"):
     """Activations, fp32 NCHW.  kind: 'relu' = max(N(0,1),0); 'relu_outliers' = the same with each
     element independently multiplied by 50 with probability 0.01; 'gauss' = N(0,1);
-    'uniform' = U[0,1); 'smallint' = integers in {-2..2}."""
+    'uniform' = U[0,1); 'silu' = z*sigmoid(z) with z ~ N(0,1); 'smallint' = integers in {-2..2}."""
     d = ConvDesc(*d)
     shape = (d.N, d.C_in, d.H, d.W)
-    g = _rng(seed, "x")
     if kind == "uniform":
-        return g.random(shape, dtype=np.float32)
+        return _draw(seed, "x", shape, lambda g, s: g.random(s, dtype=np.float32))
     if kind == "smallint":
-        return g.integers(-2, 3, size=shape).astype(np.float32)
-    x = g.standard_normal(shape, dtype=np.float32)
+        return _rng(seed, "x").integers(-2, 3, size=shape).astype(np.float32)
+    x = _draw(seed, "x", shape, lambda g, s: g.standard_normal(s, dtype=np.float32))
     if kind == "gauss":
         return x
+    if kind == "silu":
+        # post-SiLU activations: z * sigmoid(z) of a standard normal pre-activation (small negatives down to -0.278)
+        x64 = x.astype(np.float64)
+        return (x64 / (1.0 + np.exp(-x64))).astype(np.float32)
     np.maximum(x, 0.0, out=x)
     if kind == "relu_outliers":
-        mask = _rng(seed, "outlier").random(shape, dtype=np.float32) < 0.01
+        mask = _draw(seed, "outlier", shape, lambda g, s: g.random(s, dtype=np.float32)) < 0.01
         x[mask] *= 50.0
     elif kind != "relu":
         raise ValueError(kind)
@@ -81,10 +107,9 @@ def make_dy(d, seed, kind="small", sigma=1e-3):
     d = ConvDesc(*d)
     ho, wo = out_hw(d)
     shape = (d.N, d.C_out, ho, wo)
-    g = _rng(seed, "dy")
     if kind == "smallint":
-        return g.integers(-2, 3, size=shape).astype(np.float32)
-    y = g.standard_normal(shape, dtype=np.float32)
+        return _rng(seed, "dy").integers(-2, 3, size=shape).astype(np.float32)
+    y = _draw(seed, "dy", shape, lambda g, s: g.standard_normal(s, dtype=np.float32))
     if kind == "small":
         y *= np.float32(sigma)
     return y
@@ -110,15 +135,15 @@ def config3(batch=16, image=640):
     """Backbone-shaped conv stack (nano-width detector backbone: stride-2 3x3 convs widening
     16->32->64->128->256, each followed by a split/bottleneck/concat stage of 1x1 and 3x3
     stride-1 convs).  The 3->16 stem is not an MX layer; the 24 convs after it are.  Each layer
-    is exercised with its own synthetic input of the right shape (post-activation values are
-    modelled as max(N(0,1),0)); MXFP8 E4M3 forward tensors, E5M2 gradients."""
+    is exercised with its own synthetic input of the right shape (post-SiLU activations: z*sigmoid(z) of a
+    standard normal z, which keeps the small negatives down to -0.278); MXFP8 E4M3 forward tensors, E5M2 gradients."""
     layers = []
     res = image // 2  # after the stem
     seed = 200
 
     def add(name, cin, cout, k, s, r):
         nonlocal seed
-        layers.append(Layer(name, conv_desc(batch, cin, r, r, cout, k, s), E4M3, E4M3, E5M2, "relu", "kaiming", "small", seed))
+        layers.append(Layer(name, conv_desc(batch, cin, r, r, cout, k, s), E4M3, E4M3, E5M2, "silu", "kaiming", "small", seed))
         seed += 1
 
     c = 16

@@ -19,6 +19,10 @@ NCHW, HWNC = 0, 1
 OP_FWD, OP_BWD_DATA, OP_BWD_WEIGHT = 0, 1, 2
 OK = 0
 
+# When true, every output buffer this module creates is pre-filled (fp32 with NaN, bytes with 0xA5) instead of left
+# uninitialised, so that an element a kernel fails to write cannot pass a comparison by holding an earlier result.
+DEBUG_FILL = False
+
 _LIB_PATH = os.path.join(os.path.dirname(os.path.abspath(__file__)), "libmq.so")
 _lib = None
 
@@ -81,6 +85,13 @@ class QTensor:
         return _QTensor(self.codes.data_ptr(), self.scales.data_ptr(), self.codes.numel(), self.scales.numel(), self.fmt, self.role)
 
 
+def _new(shape, dtype, device):
+    t = torch.empty(shape, dtype=dtype, device=device)
+    if DEBUG_FILL:
+        t.fill_(float("nan") if dtype.is_floating_point else 0xA5)
+    return t
+
+
 def qtensor_sizes(desc, role, fmt):
     cb, sb = ctypes.c_size_t(), ctypes.c_size_t()
     _check("mq_qtensor_sizes", lib().mq_qtensor_sizes(ctypes.byref(_d(desc)), role, fmt, ctypes.byref(cb), ctypes.byref(sb)))
@@ -101,7 +112,7 @@ def workspace_size(desc, op, fmt_a, fmt_b):
 
 def empty_qtensor(desc, role, fmt, device="cuda"):
     cb, sb = qtensor_sizes(desc, role, fmt)
-    return QTensor(torch.empty(cb, dtype=torch.uint8, device=device), torch.empty(sb, dtype=torch.uint8, device=device), fmt, role)
+    return QTensor(_new(cb, torch.uint8, device), _new(sb, torch.uint8, device), fmt, role)
 
 
 def quantize(desc, role, fmt, src, out=None, src_layout=NCHW, stream=None):
@@ -129,9 +140,9 @@ def cbf_im2col(desc, xq, out_codes=None, out_scales=None, stream=None):
     """mq_cbf_im2col: stored quantized activation -> (codes, scales) of X'."""
     cb, sb = im2col_sizes(desc, xq.fmt)
     if out_codes is None:
-        out_codes = torch.empty(cb, dtype=torch.uint8, device=xq.codes.device)
+        out_codes = _new(cb, torch.uint8, xq.codes.device)
     if out_scales is None:
-        out_scales = torch.empty(sb, dtype=torch.uint8, device=xq.codes.device)
+        out_scales = _new(sb, torch.uint8, xq.codes.device)
     q = xq._c()
     _check("mq_cbf_im2col", lib().mq_cbf_im2col(ctypes.byref(_d(desc)), ctypes.byref(q), ctypes.c_void_p(out_codes.data_ptr()),
                                                ctypes.c_void_p(out_scales.data_ptr()), _stream(stream)))
@@ -146,10 +157,10 @@ def _out_hw(desc):
 def _conv(name, op, desc, qa, qb, out, shape_nchw, shape_hwnc, layout, workspace, stream):
     dev = qa.codes.device
     if out is None:
-        out = torch.empty(shape_nchw if layout == NCHW else shape_hwnc, dtype=torch.float32, device=dev)
+        out = _new(shape_nchw if layout == NCHW else shape_hwnc, torch.float32, dev)
     need = workspace_size(desc, op, qa.fmt, qb.fmt)
     if workspace is None and need > 0:
-        workspace = torch.empty(need, dtype=torch.uint8, device=dev)
+        workspace = _new(need, torch.uint8, dev)
     wp = ctypes.c_void_p(workspace.data_ptr()) if workspace is not None else None
     wn = workspace.numel() * workspace.element_size() if workspace is not None else 0
     a, b = qa._c(), qb._c()
@@ -180,7 +191,7 @@ def conv_bwd_data_static(desc, wq, dyq, dx=None, layout=NCHW, stream=None):
     `dx` should be passed in by such callers; it is only created here for convenience when omitted."""
     d = ConvDesc(*desc)
     if dx is None:
-        dx = torch.empty((d.N, d.C_in, d.H, d.W) if layout == NCHW else (d.H, d.W, d.N, d.C_in), dtype=torch.float32, device=wq.codes.device)
+        dx = _new((d.N, d.C_in, d.H, d.W) if layout == NCHW else (d.H, d.W, d.N, d.C_in), torch.float32, wq.codes.device)
     a, b = wq._c(), dyq._c()
     _check("mq_conv_bwd_data_static", lib().mq_conv_bwd_data_static(ctypes.byref(_d(desc)), ctypes.byref(a), ctypes.byref(b),
                                                                   ctypes.c_void_p(dx.data_ptr()), layout, _stream(stream)))

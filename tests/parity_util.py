@@ -11,6 +11,10 @@ from paper_2609_28358_b200 import inputs, mq
 GEMM_TOL = 1e-4
 ROLES = (mq.ROLE_X, mq.ROLE_W, mq.ROLE_DY)
 
+# every output buffer the binding creates for these tests starts as NaN (fp32) / 0xA5 (bytes): an element a kernel
+# fails to write cannot pass by holding what an earlier call left in recycled memory
+mq.DEBUG_FILL = True
+
 
 def dev(a):
     return torch.from_numpy(np.ascontiguousarray(a)).cuda()
@@ -135,4 +139,114 @@ def check_convs(ol, qs, samples=None, layouts=(mq.NCHW,), seed=0, ops=("fwd", "d
             ref, ab = oracle.conv_bwd_weight(d, gh, xh, idx)
             got = host(dwn.contiguous()).reshape(-1)
             worst["dw"] = assert_gemm_close(torch.from_numpy(got if idx is None else got[idx]), ref, ab, f"{ol.layer.name} bwd_weight layout {layout}")
+    assert mq.last_device_status() == 0, "a bounded device-side wait gave up"
+    return worst
+
+
+def _pick_blocks(nblocks, want, rng):
+    """`want` of the `nblocks` 32-channel blocks: the first, the last and random ones in between."""
+    if nblocks <= want:
+        return list(range(nblocks))
+    mid = rng.choice(np.arange(1, nblocks - 1), want - 2, replace=False)
+    return sorted({0, nblocks - 1, *map(int, mid)})
+
+
+def check_large_layer(layer, samples=3000, dw_mac_budget=3e10, seed=0):
+    """Parity of a layer too large for the oracle to process whole.  The GPU runs the whole layer at full size; the
+    oracle checks it on pieces that are independent of the rest of the tensor:
+      * the first and the last 32-sample slab (tiles never span slabs; Y and G_X of a sample depend on that sample
+        only): every quantized byte and scale of X and G_Y, the im2col of the slab, sampled Y and G_X outputs with the
+        image border included;
+      * a subset of 32-channel blocks over ALL samples (tiles never span channel blocks; G_W[co, ci] depends on channels
+        co and ci only): every quantized byte of those blocks - which reaches the far end of tensors beyond 2^31
+        bytes - and the weight gradient of (chosen output blocks) x (chosen input blocks), every tap: in full while
+        that fits `dw_mac_budget` multiply-adds of the oracle, else samples stratified over (output block, tap, input block);
+      * W in full."""
+    d = layer.desc
+    fx, fw, fg = layer.fmt_x, layer.fmt_w, layer.fmt_dy
+    name = layer.name
+    rng = np.random.default_rng(seed)
+    x, w, g = inputs.layer_tensors(layer)
+    ho, wo = inputs.out_hw(d)
+    N, Nt = d.N, (d.N + 31) // 32
+    cp, cop = (d.C_in + 31) // 32 * 32, (d.C_out + 31) // 32 * 32
+    bpe = lambda f: 0.5 if f == mq.E2M1 else 1.0
+    xq, wq, gq = [mq.quantize(d, r, f, dev(t)) for r, f, t in zip(ROLES, (fx, fw, fg), (x, w, g))]
+    wc, wsc = oracle.quantize(d, oracle.ROLE_W, fw, w)
+    assert_same_bytes(wq.scales, wsc, f"{name} W scales")
+    assert_same_bytes(wq.codes, wc, f"{name} W codes")
+    wh = oracle.dequant(d, oracle.ROLE_W, fw, wc, wsc)
+    ic, isc = mq.cbf_im2col(d, xq)
+    y = mq.conv_fwd(d, xq, wq)
+    dx = mq.conv_bwd_data(d, wq, gq)
+    dw = mq.conv_bwd_weight(d, xq, gq)
+    P, Po, taps = d.H * d.W, ho * wo, d.Kh * d.Kw
+    xcodes = xq.codes.view(P, N, int(cp * bpe(fx)))
+    gcodes = gq.codes.view(Po, N, int(cop * bpe(fg)))
+    xscales = xq.scales.view(P, Nt, cp // 32)
+    gscales = gq.scales.view(Po, Nt, cop // 32)
+    icodes = ic.view(Po, N, int(taps * cp * bpe(fx)))
+    iscales = isc.view(Po, Nt, taps * (cp // 32))
+    worst = {}
+    for slab in sorted({0, Nt - 1}):
+        n0, n1 = 32 * slab, min(N, 32 * slab + 32)
+        ds = d._replace(N=n1 - n0)
+        xc, xsc = oracle.quantize(ds, oracle.ROLE_X, fx, x[n0:n1])
+        gc, gsc = oracle.quantize(ds, oracle.ROLE_DY, fg, g[n0:n1])
+        assert_same_bytes(xscales[:, slab].contiguous(), xsc, f"{name} X scales, samples {n0}..{n1}")
+        assert_same_bytes(xcodes[:, n0:n1].contiguous(), xc, f"{name} X codes, samples {n0}..{n1}")
+        assert_same_bytes(gscales[:, slab].contiguous(), gsc, f"{name} dY scales, samples {n0}..{n1}")
+        assert_same_bytes(gcodes[:, n0:n1].contiguous(), gc, f"{name} dY codes, samples {n0}..{n1}")
+        oc, osc = oracle.cbf_im2col(ds, fx, xc, xsc)
+        assert_same_bytes(iscales[:, slab].contiguous(), osc, f"{name} im2col scales, samples {n0}..{n1}")
+        assert_same_bytes(icodes[:, n0:n1].contiguous(), oc, f"{name} im2col codes, samples {n0}..{n1}")
+        del oc, osc
+        xh = oracle.dequant(ds, oracle.ROLE_X, fx, xc, xsc)
+        gh = oracle.dequant(ds, oracle.ROLE_DY, fg, gc, gsc)
+        shape = (n1 - n0, d.C_out, ho, wo)
+        idx = _sample(int(np.prod(shape)), samples, rng, border_indices(shape, rng=rng))
+        ref, ab = oracle.conv_fwd(ds, xh, wh, idx)
+        got = host(y[n0:n1].contiguous()).reshape(-1)[idx]
+        worst["fwd"] = max(worst.get("fwd", 0.0), assert_gemm_close(torch.from_numpy(got), ref, ab, f"{name} fwd, samples {n0}..{n1}"))
+        shape = (n1 - n0, d.C_in, d.H, d.W)
+        idx = _sample(int(np.prod(shape)), samples, rng, border_indices(shape, rng=rng))
+        ref, ab = oracle.conv_bwd_data(ds, wh, gh, idx)
+        got = host(dx[n0:n1].contiguous()).reshape(-1)[idx]
+        worst["dx"] = max(worst.get("dx", 0.0), assert_gemm_close(torch.from_numpy(got), ref, ab, f"{name} bwd_data, samples {n0}..{n1}"))
+        del xh, gh
+    del ic, isc, icodes, iscales, y, dx
+    # channel blocks over all samples
+    assert d.C_in % 32 == 0 and d.C_out % 32 == 0
+    bi, bo = _pick_blocks(cp // 32, 4, rng), _pick_blocks(cop // 32, 4, rng)
+    if cop // 32 >= 16:   # one output block in each 128-row tile of the weight gradient, at a different place in each
+        bo = [4 * t + (t % 4) for t in range(4)] if cop // 32 == 16 else bo
+    ci = np.concatenate([np.arange(32 * b, 32 * b + 32) for b in bi])
+    co = np.concatenate([np.arange(32 * b, 32 * b + 32) for b in bo])
+    dsel = d._replace(C_in=ci.size, C_out=co.size)
+    xs = np.ascontiguousarray(x[:, ci])
+    gs = np.ascontiguousarray(g[:, co])
+    del x, g
+    xc, xsc = oracle.quantize(dsel, oracle.ROLE_X, fx, xs)
+    gc, gsc = oracle.quantize(dsel, oracle.ROLE_DY, fg, gs)
+    del xs, gs
+    bx, bg = int(32 * bpe(fx)), int(32 * bpe(fg))
+    tb = lambda blocks: torch.as_tensor(blocks, device="cuda")
+    assert_same_bytes(xscales[:, :, tb(bi)].contiguous(), xsc, f"{name} X scales, channel blocks {bi}")
+    assert_same_bytes(xcodes.view(P, N, cp // 32, bx)[:, :, tb(bi)].contiguous(), xc, f"{name} X codes, channel blocks {bi}")
+    assert_same_bytes(gscales[:, :, tb(bo)].contiguous(), gsc, f"{name} dY scales, channel blocks {bo}")
+    assert_same_bytes(gcodes.view(Po, N, cop // 32, bg)[:, :, tb(bo)].contiguous(), gc, f"{name} dY codes, channel blocks {bo}")
+    xh = oracle.dequant(dsel, oracle.ROLE_X, fx, xc, xsc)
+    gh = oracle.dequant(dsel, oracle.ROLE_DY, fg, gc, gsc)
+    got = host(dw[tb(co)][:, tb(ci)].contiguous()).reshape(-1)
+    per_out = float(N) * ho * wo
+    if co.size * ci.size * taps * per_out <= dw_mac_budget:
+        idx = None
+    else:
+        per = max(1, int(dw_mac_budget / per_out / (len(bo) * taps * len(bi))))
+        o, i, t = np.meshgrid(np.arange(len(bo)), np.arange(len(bi)), np.arange(taps), indexing="ij")
+        o, i, t = [np.repeat(a.reshape(-1), per) for a in (o, i, t)]
+        idx = np.unique(((32 * o + rng.integers(0, 32, o.size)) * ci.size + 32 * i + rng.integers(0, 32, o.size)) * taps + t).astype(np.int64)
+    ref, ab = oracle.conv_bwd_weight(dsel, gh, xh, idx)
+    worst["dw"] = assert_gemm_close(torch.from_numpy(got if idx is None else got[idx]), ref, ab, f"{name} bwd_weight, blocks {bo} x {bi}")
+    assert mq.last_device_status() == 0, "a bounded device-side wait gave up"
     return worst

@@ -9,7 +9,7 @@ import torch
 
 import oracle
 from paper_2609_28358_b200 import inputs, mq
-from parity_util import (OracleLayer, assert_same_bytes, check_convs, check_im2col, check_quantize, dev,
+from parity_util import (OracleLayer, assert_same_bytes, check_convs, check_im2col, check_large_layer, check_quantize, dev,
                          gpu_quantize_layer)
 
 pytestmark = pytest.mark.gpu
@@ -144,7 +144,7 @@ def _cfg3_layers():
     return inputs.config3()
 
 
-@pytest.mark.parametrize("li", [0, 1, 2, 5, 11, 17, 18, 23])
+@pytest.mark.parametrize("li", range(24))
 def test_config3_layers_full_size(li):
     layer = _cfg3_layers()[li]
     ol = OracleLayer(layer)
@@ -165,6 +165,25 @@ def test_config5_points_full_size(name):
     qs = check_quantize(ol)
     check_im2col(ol, qs[0])
     check_convs(ol, qs, samples=4000)
+
+
+# The large points of the sweep: every (format, kernel, stride) family at 512 channels on 56x56 and 28x28 images, the
+# 3x3 families at 256 channels on 56x56.  Tensors reach 1.6 GB of fp32 and 3.7 GB of X' (offsets beyond 2^31 bytes).
+CFG5_LARGE = [f"cfg5_{f}_k{k}s{s}_c512_hw{hw}" for f in ("e4m3", "e2m1") for k in (3, 1) for s in (1, 2) for hw in (56, 28)] + \
+             [f"cfg5_{f}_k3s{s}_c256_hw56" for f in ("e4m3", "e2m1") for s in (1, 2)]
+
+
+@pytest.mark.parametrize("name", CFG5_LARGE)
+def test_config5_large_points_full_size(name):
+    """The GPU runs the point at full size; the oracle checks sample slabs, channel blocks and W (see check_large_layer)."""
+    layer = {l.name: l for l in inputs.config5()}[name]
+    check_large_layer(layer)
+
+
+@pytest.mark.parametrize("idx", [0, 1], ids=["e3m2-act", "e2m3"])
+def test_fp6_layers_full_size(idx):
+    """The two 6-bit layers the benchmark reports (256 channels, 28x28, N = 256)."""
+    check_large_layer(inputs.fp6_layers()[idx])
 
 
 @pytest.mark.parametrize("fmts", [(E4M3, E4M3, E5M2), (E2M1, E2M1, E2M1)], ids=["fp8", "fp4"])

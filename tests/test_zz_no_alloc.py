@@ -43,6 +43,9 @@ def test_static_scratch_variant_matches_workspace_variant_on_two_calls_in_a_row(
         _, ab = oracle.conv_bwd_data(d, ol.hat[1], ol.hat[2])
         err = np.abs(got.cpu().numpy().astype(np.float64) - ref.cpu().numpy().astype(np.float64))
         assert (err <= GEMM_TOL * ab).all()
+        # the same deterministic kernels ran on the same inputs: nothing of the previous call's leftovers in the
+        # shared array may leak, so the two results are the same bits
+        assert torch.equal(got, ref)
         # and against the oracle itself, like every other GEMM test
         gx, _ = oracle.conv_bwd_data(d, ol.hat[1], ol.hat[2])
         assert (np.abs(got.cpu().numpy().astype(np.float64) - gx) <= GEMM_TOL * ab).all()
@@ -58,3 +61,8 @@ def test_static_scratch_variant_rejects_layers_beyond_its_limit():
         mq.conv_bwd_data_static(d, wq, gq, dx=dx)
     assert e.value.status == 7 and "STATIC_SCRATCH" in str(e.value)
     assert not dx.any()      # nothing was launched
+    # a bad argument is reported as such even on a layer beyond the limit
+    lib = mq.lib()
+    a, b = wq._c(), gq._c()
+    st = lib.mq_conv_bwd_data_static(ctypes.byref(mq._d(d)), ctypes.byref(a), ctypes.byref(b), None, mq.NCHW, None)
+    assert st == 1   # MQ_ERR_INVALID_ARG: null dx
