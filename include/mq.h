@@ -184,6 +184,15 @@ mq_status mq_conv_layer_host(const mq_conv_desc* desc, int fmt_x, int fmt_w, int
 /* Diagnostic: how many kernels this library has launched so far in this process (all entry points). */
 unsigned long long mq_kernel_launch_count(void);
 
+/* Diagnostic self-test of the give-up path of the library's bounded device-side waits (the paper has no counterpart).
+ * Launches the quantizer's TMA pipeline for role X or DY (dst->role; H*W resp. Ho*Wo a multiple of 4, else
+ * MQ_ERR_UNSUPPORTED) on `src` (fp32 NCHW) with its loader issuing NO copies and every barrier wait limited to `polls`
+ * polls (1 .. 2^20): nothing ever arrives, each wait runs out, the kernel records MQ_ERR_TIMEOUT in the device status
+ * word, leaves its loops, and returns normally - nothing hangs, traps or faults, the context stays usable.  dst's buffers
+ * (sizes as for mq_quantize) are left with unspecified contents.  Afterwards mq_last_device_status() reports
+ * MQ_ERR_TIMEOUT once and clears the word. */
+mq_status mq_selftest_wait_timeout(const mq_conv_desc* desc, const void* src, mq_qtensor* dst, unsigned polls, void* stream);
+
 /* Human-readable name of a status code (static storage). */
 const char* mq_status_string(int status);
 

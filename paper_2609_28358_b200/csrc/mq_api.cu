@@ -678,7 +678,7 @@ mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt
 }
 
 static mq_status quantize_impl(const mq_conv_desc* desc, const void* src, int src_layout, mq_qtensor* dst, int sr, unsigned long long seed,
-                               void* stream) {
+                               void* stream, unsigned wait_limit = 0, int skip_loads = 0) {
   mq_status st = check_desc(desc);
   if (st != MQ_OK) return st;
   if (!src || !dst || !valid_role(dst->role)) return MQ_ERR_INVALID_ARG;
@@ -706,6 +706,8 @@ static mq_status quantize_impl(const mq_conv_desc* desc, const void* src, int sr
     if (dst->role == MQ_ROLE_W) { a.src_stride_p = v.C; a.src_stride_r = v.P * v.C; }
     else { a.src_stride_p = v.R * v.C; a.src_stride_r = v.C; }
   }
+  a.status = device_status_ptr();
+  a.wait_limit = wait_limit; a.debug_skip_loads = skip_loads;
   a.sr = sr;
   a.sr_seed_lo = (unsigned)seed; a.sr_seed_hi = (unsigned)(seed >> 32);
   a.sr_key0 = sr_mix32(a.sr_seed_lo ^ sr_mix32(a.sr_seed_hi ^ sr_mix32(0u)));
@@ -720,6 +722,13 @@ mq_status mq_quantize(const mq_conv_desc* desc, const void* src, int src_layout,
 
 mq_status mq_quantize_sr(const mq_conv_desc* desc, const void* src, int src_layout, mq_qtensor* dst, unsigned long long seed, void* stream) {
   return quantize_impl(desc, src, src_layout, dst, 1, seed, stream);
+}
+
+mq_status mq_selftest_wait_timeout(const mq_conv_desc* desc, const void* src, mq_qtensor* dst, unsigned polls, void* stream) {
+  if (polls == 0 || polls > (1u << 20)) return MQ_ERR_INVALID_ARG;
+  if (dst && dst->role == MQ_ROLE_W) return MQ_ERR_UNSUPPORTED;
+  if (desc && dst && (long long)(dst->role == MQ_ROLE_X ? desc->H * desc->W : 0) % 4 != 0) return MQ_ERR_UNSUPPORTED;
+  return quantize_impl(desc, src, MQ_NCHW, dst, 0, 0ull, stream, polls, 1);
 }
 
 mq_status mq_cbf_im2col(const mq_conv_desc* desc, const mq_qtensor* xq, void* cols_codes, uint8_t* cols_scales, void* stream) {

@@ -1419,7 +1419,7 @@ static CUtensorMapL2promotion l2promo() {
   return v == 0 ? CU_TENSOR_MAP_L2_PROMOTION_NONE : v == 1 ? CU_TENSOR_MAP_L2_PROMOTION_L2_64B : v == 2 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
 }
 bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes, const uint32_t* box,
-                          const uint32_t* elem_strides, int swizzle_bytes, bool f32) {
+                          const uint32_t* elem_strides, int swizzle_bytes, bool f32, int l2_promotion_bytes) {
   EncodeTiledFn fn = get_encoder();
   if (!fn) return false;
   cuuint64_t d[5], st[4];
@@ -1430,7 +1430,8 @@ bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const ui
                         : swizzle_bytes == 64  ? CU_TENSOR_MAP_SWIZZLE_64B
                         : swizzle_bytes == 32  ? CU_TENSOR_MAP_SWIZZLE_32B : CU_TENSOR_MAP_SWIZZLE_NONE;
   CUresult r = fn(map, f32 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_UINT8, (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es, CU_TENSOR_MAP_INTERLEAVE_NONE, sw,
-                  l2promo(), CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+                  l2_promotion_bytes < 0 ? l2promo() : l2_promotion_bytes == 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : l2_promotion_bytes == 256 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B
+                  : l2_promotion_bytes == 64 ? CU_TENSOR_MAP_L2_PROMOTION_L2_64B : CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
 }
 

@@ -154,8 +154,9 @@ cudaError_t launch_wgrad_flat_prep(const WgradTcParams& p, const uint8_t* x_code
 cudaError_t launch_bwd_weight_reduce(const float* partial, float* out, const Geom& g, int splits, int layout, cudaStream_t s);
 
 // Host: encode a tiled tensor map over bytes (or over fp32 elements when f32 is set: dims and box then count
-// elements).  Strides in bytes (stride[0] implied contiguous), fastest dimension first.
+// elements).  Strides in bytes (stride[0] implied contiguous), fastest dimension first.  l2_promotion_bytes: 0, 64, 128, 256,
+// or -1 for the library's default.
 bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
-                          const uint32_t* box, const uint32_t* elem_strides, int swizzle_bytes, bool f32 = false);
+                          const uint32_t* box, const uint32_t* elem_strides, int swizzle_bytes, bool f32 = false, int l2_promotion_bytes = -1);
 
 }  // namespace mq

@@ -61,6 +61,11 @@ struct QuantArgs {
   unsigned sr_seed_lo, sr_seed_hi;   // the 64-bit seed
   unsigned sr_key0;                  // stream key of elements whose index is below 2^32 (computed on the host)
   int sr_wide;                       // 1: the tensor has 2^32 elements or more (keys are derived per element)
+  unsigned int* status;              // device status word: set when a bounded wait gives up
+  // test hooks of the TMA kernel's abort path: polls a barrier wait may take (0: the default limit), and 1 = the loader
+  // issues no copies, so that every wait on them runs out
+  unsigned wait_limit;
+  int debug_skip_loads;
 };
 // invertible 32-bit mixer (xor-shift, odd multiply, twice, xor-shift) behind the per-element draws
 __host__ __device__ __forceinline__ unsigned sr_mix32(unsigned x) {

@@ -136,6 +136,16 @@ def quantize_sr(desc, role, fmt, src, seed, out=None, src_layout=NCHW, stream=No
     return out
 
 
+def selftest_wait_timeout(desc, role, fmt, src, polls=2000, stream=None):
+    """mq_selftest_wait_timeout: runs the quantizer's TMA pipeline with its loader off and short wait limits, so every
+    bounded wait gives up; the kernel must return normally with the device status word set."""
+    out = empty_qtensor(desc, role, fmt, src.device)
+    q = out._c()
+    _check("mq_selftest_wait_timeout", lib().mq_selftest_wait_timeout(ctypes.byref(_d(desc)), ctypes.c_void_p(src.data_ptr()), ctypes.byref(q),
+                                                                    ctypes.c_uint(polls), _stream(stream)))
+    return out
+
+
 def cbf_im2col(desc, xq, out_codes=None, out_scales=None, stream=None):
     """mq_cbf_im2col: stored quantized activation -> (codes, scales) of X'."""
     cb, sb = im2col_sizes(desc, xq.fmt)

@@ -237,3 +237,47 @@ def test_alternate_kernel_paths(knob, monkeypatch):
             ol = OracleLayer(make_layer(name, d, fmts, seed=23, kinds=("relu", "kaiming", "gauss")))
             qs = check_quantize(ol)
             check_convs(ol, qs, samples=20000, layouts=(mq.NCHW, mq.HWNC))
+
+
+TMA_Q_SHAPES = [
+    ("aligned", (64, 96, 8, 8, 64, 3, 1, 1)),          # whole tiles, two strips of 32 positions
+    ("ragged_n_c", (40, 48, 6, 6, 70, 3, 1, 1)),       # 36 positions: a partial second strip; ragged rows and channels
+    ("few_positions", (250, 320, 3, 4, 288, 3, 1, 1)),  # 12 positions: a box wider than the tensor; 8 row tiles, the last ragged
+    ("batch16", (16, 40, 10, 12, 72, 3, 1, 1)),        # two boxes per item
+    ("batch5", (5, 16, 10, 10, 24, 3, 1, 1)),          # one box per item, 16 channels, 100 positions
+    ("odd_rows", (77, 35, 8, 8, 34, 3, 1, 1)),         # three row tiles, the last of 13 rows (two boxes)
+]
+
+
+@pytest.mark.parametrize("fmt", [E4M3, E5M2, E2M1, E3M2, E2M3])
+@pytest.mark.parametrize("order", ["0", "1"], ids=["tile-fastest", "strip-fastest"])
+@pytest.mark.parametrize("name,shape", TMA_Q_SHAPES, ids=[s[0] for s in TMA_Q_SHAPES])
+def test_quantize_whole_line_kernel_on_small_shapes(name, shape, order, fmt, monkeypatch):
+    """The whole-line (TMA) quantizer that large NCHW tensors take, forced onto small ragged ones: the oracle's bytes,
+    with round-to-nearest and with the stochastic rounding."""
+    monkeypatch.setenv("MQ_QUANT_TMA", "1")
+    monkeypatch.setenv("MQ_QUANT_STRIP_FASTEST", order)
+    d = inputs.conv_desc(*shape)
+    ol = OracleLayer(make_layer(name, d, (fmt, fmt, fmt), seed=41, kinds=("relu", "kaiming", "gauss")))
+    check_quantize(ol)
+    g = ol.src[2]
+    oc, osc = oracle.quantize_sr(d, oracle.ROLE_DY, fmt, g, 99)
+    q = mq.quantize_sr(d, mq.ROLE_DY, fmt, dev(g), 99)
+    assert_same_bytes(q.scales, osc, f"{name} stochastic scales")
+    assert_same_bytes(q.codes, oc, f"{name} stochastic codes")
+    assert mq.last_device_status() == 0
+
+
+def test_bounded_waits_give_up_and_the_context_stays_usable():
+    """Every device-side wait of the library is bounded.  Here the quantizer's TMA pipeline runs with its loader switched
+    off and a limit of a few thousand polls, so each wait runs out: the kernel must return normally with
+    MQ_ERR_TIMEOUT in the device status word (read once, then cleared), and the next ordinary call must be correct."""
+    d = inputs.conv_desc(64, 96, 8, 8, 64, 3, 1, 1)
+    ol = OracleLayer(make_layer("timeout", d, (E4M3, E4M3, E5M2), seed=43, kinds=("relu", "kaiming", "gauss")))
+    assert mq.last_device_status() == 0
+    mq.selftest_wait_timeout(d, mq.ROLE_X, E4M3, dev(ol.src[0]), polls=2000)
+    torch.cuda.synchronize()                      # the kernel has returned: nothing hangs
+    assert mq.last_device_status() == 6           # MQ_ERR_TIMEOUT
+    assert mq.last_device_status() == 0           # reading it cleared it
+    qs = check_quantize(ol)                       # the context is intact
+    check_convs(ol, qs, samples=None)
