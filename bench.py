@@ -387,12 +387,77 @@ def run_ours(args):
                 "device_status": mq.last_device_status()}
             del w2
             torch.cuda.empty_cache()
+    if rank == 0 and world == 1 and not args.no_accounting:
+        out["quantization_accounting"] = quantization_accounting(all_wl[args.workload], flush)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(all_wl[args.workload], budget_s=args.cpu_budget)
     if rank == 0:
         print(json.dumps(out))
     if world > 1:
         dist.destroy_process_group()
+
+
+def quantization_accounting(layer, flush, reps=5):
+    """Measured counterpart of the paper's Table I (Sec. IV-C) on one layer: elements that pass through a quantizer per
+    forward + backward step, bytes those quantizer calls move, their time, and the bytes of activation kept for the
+    backward pass - for this library's path and for two stand-ins built from the library's own kernels:
+      square_blocks_once          X, W, G_Y quantized once each in 32 x 32 blocks (usable by both of their GEMMs); Q(X) kept;
+      line_blocks_expanded_twice  the scheme the paper compares with first: one-directional (line) blocks on the im2col-EXPANDED
+                                  activation, quantized for the forward pass and again, in the other direction, for the
+                                  backward pass (the library's line quantizer stands in for that second direction at the same
+                                  element count), W and G_Y likewise twice; the fp32 activation is what is kept;
+      square_blocks_on_expanded   the second comparison: the expanded activation quantized once in square blocks and kept.
+    The expanded fp32 matrix X' is produced by torch's unfold (glue, not timed).  Every count is the numel of a tensor
+    actually handed to mq_quantize; bytes are the sizes of the buffers those calls read and wrote."""
+    import torch
+    import torch.nn.functional as F
+
+    from paper_2609_28358_b200 import mq
+
+    d = layer.desc
+    fmts = (layer.fmt_x, layer.fmt_w, layer.fmt_dy)
+    ho, wo = inputs.out_hw(d)
+    x, w, g = [torch.from_numpy(t).cuda() for t in (inputs.make_x(d, layer.seed, layer.x_kind), inputs.make_w(d, layer.seed, layer.w_kind),
+                                                     inputs.make_dy(d, layer.seed, layer.dy_kind))]
+    xe = F.unfold(x, (d.Kh, d.Kw), padding=(d.pad_h, d.pad_w), stride=(d.stride_h, d.stride_w)).reshape(d.N, d.C_in * d.Kh * d.Kw, ho, wo).contiguous()
+    de = d._replace(C_in=d.C_in * d.Kh * d.Kw, H=ho, W=wo, Kh=1, Kw=1, stride_h=1, stride_w=1, pad_h=0, pad_w=0)   # X' as a 1x1 layer's input
+
+    def run(calls):
+        """calls: (desc, role, fmt, tensor, block); returns elements, bytes moved, ms per pass, size of the first call's stored tensor."""
+        outs = [mq.empty_qtensor(dd, r, f, block=b) for dd, r, f, t, b in calls]
+        fns = [lambda dd=dd, r=r, f=f, t=t, o=o, b=b: mq.quantize(dd, r, f, t, out=o, block=b) for (dd, r, f, t, b), o in zip(calls, outs)]
+        for fn in fns:
+            fn()
+        torch.cuda.synchronize()
+        ms = []
+        for _ in range(reps):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for fn in fns:
+                fn()
+            e1.record()
+            torch.cuda.synchronize()
+            ms.append(e0.elapsed_time(e1))
+        elems = sum(t.numel() for _, _, _, t, _ in calls)
+        moved = sum(4 * t.numel() for _, _, _, t, _ in calls) + sum(o.codes.numel() + o.scales.numel() for o in outs)
+        return elems, moved, float(np.median(ms)), outs[0].codes.numel() + outs[0].scales.numel()
+
+    T, L = mq.TILE32, mq.LINE32
+    ours = run([(d, 0, fmts[0], x, T), (d, 1, fmts[1], w, T), (d, 2, fmts[2], g, T)])
+    line2 = run([(de, 0, fmts[0], xe, L), (d, 1, fmts[1], w, L), (d, 2, fmts[2], g, L)] * 2)
+    sq_e = run([(de, 0, fmts[0], xe, T), (d, 1, fmts[1], w, T), (d, 2, fmts[2], g, T)])
+    res = {
+        "layer": dict(d._asdict()), "formats": [FMT_NAME[f] for f in fmts],
+        "square_blocks_once": {"quantized_elements": ours[0], "quantizer_bytes_moved": ours[1], "quantizer_ms": ours[2], "activation_kept_bytes": ours[3]},
+        "line_blocks_expanded_twice": {"quantized_elements": line2[0], "quantizer_bytes_moved": line2[1], "quantizer_ms": line2[2],
+                                       "activation_kept_bytes": 4 * x.numel()},
+        "square_blocks_on_expanded": {"quantized_elements": sq_e[0], "quantizer_bytes_moved": sq_e[1], "quantizer_ms": sq_e[2],
+                                      "activation_kept_bytes": sq_e[3]},
+    }
+    res["activation_elements_ratio"] = {"line_blocks_expanded_twice": 2.0 * xe.numel() / x.numel(), "square_blocks_on_expanded": xe.numel() / x.numel()}
+    res["activation_kept_ratio"] = {"line_blocks_expanded_twice": 4.0 * x.numel() / ours[3], "square_blocks_on_expanded": sq_e[3] / ours[3]}
+    return res
 
 
 # ----------------------------------------------------------------------------------- CPU oracle
@@ -480,6 +545,7 @@ def main():
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--more", default=",".join(MORE_WORKLOADS), help="further workloads timed after the main one (comma-separated, or 'none')")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-accounting", action="store_true", help="skip the measured Table-I style quantization accounting")
     ap.add_argument("--dy-rounding", default="nearest", choices=["nearest", "stochastic"],
                     help="rounding of the gradient's quantizer in the device-timed step (the host-buffer call keeps nearest)")
     ap.add_argument("--cpu-budget", type=float, default=15.0)

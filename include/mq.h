@@ -27,6 +27,14 @@
  *   byte (value 2^(code-127)) shared by a 32 x 32 tile: 32 channels x 32 samples (X, DY) or
  *   32 input x 32 output channels (W) at one spatial / tap position, so that every 32-element
  *   line of a tile, in either contraction direction, is a standard MX block (Sec. IV-B).
+ *
+ * Line blocks (MQ_BLOCK_LINE32): the one-directional block of Sec. III-A (Eq. 5-6) - 32 consecutive channels of ONE
+ *   row (sample / output channel) share the scale, amax over those 32 elements.  Codes are laid out as above; scales
+ *   have one entry per row instead of one per 32 rows:
+ *   role X : scales [H][W][N][C_in_p/32]     role W : scales [C_out][Kh][Kw][C_in_p/32]     role DY: scales [Ho][Wo][N][C_out_p/32]
+ *   Such a tensor can feed the GEMM that contracts over its channel axis (the forward GEMM for X and W) and no
+ *   other: that is the limitation Sec. III-B / III-C derive the square blocks from.  mq_quantize, mq_cbf_im2col
+ *   and mq_conv_fwd accept it; mq_conv_bwd_data and mq_conv_bwd_weight return MQ_ERR_UNSUPPORTED for it.
  */
 #ifndef MQ_H_
 #define MQ_H_
@@ -55,7 +63,10 @@ typedef enum { MQ_E4M3 = 0, MQ_E5M2 = 1, MQ_E2M1 = 2,
                                                         per byte, value in the low six bits, sign in bit 5 (the
                                                         convolution calls pack or re-encode them in their scratch) */
 typedef enum { MQ_ROLE_X = 0, MQ_ROLE_W = 1, MQ_ROLE_DY = 2 } mq_role; /* which tensor, Sec. IV-B   */
-typedef enum { MQ_NCHW = 0, MQ_HWNC = 1 } mq_layout;                   /* fp32 tensor layout        */
+typedef enum { MQ_NCHW = 0, MQ_HWNC = 1 } mq_layout;                   /* layout of an unquantized tensor */
+typedef enum { MQ_BLOCK_TILE32 = 0,      /* 32 x 32 square block (Sec. IV-B), the default           */
+               MQ_BLOCK_LINE32 = 1 } mq_block; /* 1 x 32 line block along the channel axis (Sec. III-A) */
+typedef enum { MQ_F32 = 0, MQ_BF16 = 1 } mq_dtype;                     /* element type of an unquantized tensor */
 typedef enum { MQ_OP_FWD = 0, MQ_OP_BWD_DATA = 1, MQ_OP_BWD_WEIGHT = 2 } mq_op;
 
 /* One convolution layer (Sec. II-A).  block_size must be 32 (the E8M0 block length). */
@@ -73,19 +84,21 @@ typedef struct {
   size_t scales_bytes; /* size of the scales buffer                   */
   int fmt;             /* mq_elem                                     */
   int role;            /* mq_role                                     */
+  int block;           /* mq_block                                    */
 } mq_qtensor;
 
 /* Size queries (host only, no GPU needed). */
 
-/* Bytes of codes and scales of the stored MX tensor of `role` (layouts above). */
-mq_status mq_qtensor_sizes(const mq_conv_desc* desc, int role, int fmt, size_t* codes_bytes, size_t* scales_bytes);
+/* Bytes of codes and scales of the stored MX tensor of `role` with blocks `block` (layouts above). */
+mq_status mq_qtensor_sizes(const mq_conv_desc* desc, int role, int fmt, int block, size_t* codes_bytes, size_t* scales_bytes);
 
-/* Bytes of X'_{Cin,N} (Sec. IV-A): codes [Ho][Wo][N][Kh][Kw][C_in_p], scales [Ho][Wo][ceil(N/32)][Kh][Kw][C_in_p/32]. */
-mq_status mq_im2col_sizes(const mq_conv_desc* desc, int fmt, size_t* codes_bytes, size_t* scales_bytes);
+/* Bytes of X'_{Cin,N} (Sec. IV-A): codes [Ho][Wo][N][Kh][Kw][C_in_p], scales [Ho][Wo][ceil(N/32)][Kh][Kw][C_in_p/32]
+ * (line blocks: [Ho][Wo][N][Kh][Kw][C_in_p/32]). */
+mq_status mq_im2col_sizes(const mq_conv_desc* desc, int fmt, int block, size_t* codes_bytes, size_t* scales_bytes);
 
 /* Bytes of scratch `op` (mq_op) needs for operand formats fmt_a, fmt_b (in the order of the call's
- * two mq_qtensor arguments).  May be 0. */
-mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt_b, size_t* bytes);
+ * two mq_qtensor arguments) quantized in blocks `block`.  May be 0. */
+mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt_b, int block, size_t* bytes);
 
 /* mq_quantize -- Sec. III-A (Eq. 5-6) in the E8M0 form of the original MX format (Sec. II-D), on the
  * square blocks and in the directions of Sec. IV-B; also re-lays the tensor into its stored order
@@ -93,13 +106,14 @@ mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt
  *   per tile: amax = max |x| over the valid elements; scale code = clamp(floor(log2 amax) - emax
  *   + 127, 0, 254) (0 if amax = 0); element = round-to-nearest-even(x * 2^(127 - code)) on the
  *   element format's grid, saturating at its largest finite magnitude, sign kept.
- * src: fp32 device memory, 16-byte aligned; `src_layout` = MQ_NCHW (X: [N][C_in][H][W], W: [C_out][C_in][Kh][Kw],
+ * src: device memory, 16-byte aligned, of element type `src_dtype` (MQ_F32; MQ_BF16 returns MQ_ERR_UNSUPPORTED in this
+ * build); `src_layout` = MQ_NCHW (X: [N][C_in][H][W], W: [C_out][C_in][Kh][Kw],
  * G_Y: [N][C_out][Ho][Wo]) or MQ_HWNC, the channel-fastest order the convolution entry points can emit
  * (X: [H][W][N][C_in], W: [C_out][Kh][Kw][C_in], G_Y: [Ho][Wo][N][C_out]); both give the same stored
- * tensor bit for bit.  dst->codes / dst->scales receive the stored tensor; dst->fmt and
- * dst->role select format and role; the *_bytes fields must be at least mq_qtensor_sizes().
+ * tensor bit for bit.  dst->codes / dst->scales receive the stored tensor; dst->fmt, dst->role and
+ * dst->block select format, role and block shape; the *_bytes fields must be at least mq_qtensor_sizes().
  * Non-finite inputs are outside the contract (result unspecified, no fault). */
-mq_status mq_quantize(const mq_conv_desc* desc, const void* src, int src_layout, mq_qtensor* dst, void* stream);
+mq_status mq_quantize(const mq_conv_desc* desc, const void* src, int src_dtype, int src_layout, mq_qtensor* dst, void* stream);
 
 /* mq_quantize_sr -- the same quantizer with the STOCHASTIC Round(.) of Eq. 6, which Sec. III-A assigns to the
  * gradient (activations and weights keep round-to-nearest); any role is accepted.  Tile scales are those of
@@ -111,26 +125,31 @@ mq_status mq_quantize(const mq_conv_desc* desc, const void* src, int src_layout,
  * either src_layout) and mix(x): x ^= x >> 16; x *= 0x7FEB352D; x ^= x >> 15; x *= 0x846CA68B; x ^= x >> 16 on
  * 32 bits.  The stored tensor is therefore a pure function of (src, seed): the same for both source layouts, on
  * every launch and on any number of GPUs.  Arguments, layouts and errors as for mq_quantize. */
-mq_status mq_quantize_sr(const mq_conv_desc* desc, const void* src, int src_layout, mq_qtensor* dst, unsigned long long seed, void* stream);
+mq_status mq_quantize_sr(const mq_conv_desc* desc, const void* src, int src_dtype, int src_layout, mq_qtensor* dst, unsigned long long seed,
+                         void* stream);
 
 /* mq_cbf_im2col -- channel-batch-first im2col (Sec. IV-A) of the quantized activation `xq` (role X):
  * row (kh,kw,c), column (ho,wo,n) of X' is the stored code at pixel (ho*stride+kh-pad,
  * wo*stride+kw-pad); tile scales are gathered alongside; out-of-image taps are zero bytes (codes
  * and scale).  No arithmetic on values: an element keeps its single quantized value everywhere.
- * cols_codes / cols_scales: sizes from mq_im2col_sizes(). */
+ * cols_codes / cols_scales: sizes from mq_im2col_sizes() for xq->fmt and xq->block. */
 mq_status mq_cbf_im2col(const mq_conv_desc* desc, const mq_qtensor* xq, void* cols_codes, uint8_t* cols_scales, void* stream);
 
 /* mq_conv_fwd -- Y_{f Cout,N} = W_{f Cout,Cin} . X'_{Cin,N} (Sec. II-C, IV-B; Eq. 1), block-scaled as
  * Eq. 7 with K-blocks of 32 input channels at one tap; X' is formed on the fly from `xq`.
- * y: fp32, `y_layout` MQ_NCHW ([N][C_out][Ho][Wo]) or MQ_HWNC ([Ho][Wo][N][C_out]); fp32 accumulation.
- * workspace: ws_bytes >= mq_workspace_size(desc, MQ_OP_FWD, xq->fmt, wq->fmt) (may be NULL if 0). */
-mq_status mq_conv_fwd(const mq_conv_desc* desc, const mq_qtensor* xq, const mq_qtensor* wq, void* y, int y_layout,
+ * y: `y_dtype` elements (MQ_F32; MQ_BF16 returns MQ_ERR_UNSUPPORTED in this build), `y_layout` MQ_NCHW
+ * ([N][C_out][Ho][Wo]) or MQ_HWNC ([Ho][Wo][N][C_out]); fp32 accumulation.
+ * xq and wq must have the same block shape; with line blocks the K-blocks carry one scale per row (Eq. 7 as written).
+ * workspace: ws_bytes >= mq_workspace_size(desc, MQ_OP_FWD, xq->fmt, wq->fmt, xq->block) (may be NULL if 0). */
+mq_status mq_conv_fwd(const mq_conv_desc* desc, const mq_qtensor* xq, const mq_qtensor* wq, void* y, int y_dtype, int y_layout,
                       void* workspace, size_t ws_bytes, void* stream);
 
 /* mq_conv_bwd_data -- G_X' = W_f^T . G_Yf followed by the col2im reordering (Sec. II-C, IV-B; Eq. 2):
  * the exact adjoint of mq_conv_fwd in X, K-blocks of 32 output channels at one tap.
- * dx: fp32, MQ_NCHW ([N][C_in][H][W]) or MQ_HWNC ([H][W][N][C_in]). */
-mq_status mq_conv_bwd_data(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, void* dx, int dx_layout,
+ * dx: `dx_dtype` elements (MQ_F32), MQ_NCHW ([N][C_in][H][W]) or MQ_HWNC ([H][W][N][C_in]).
+ * W is contracted along C_out, across its stored channel lines (the second direction of its blocks), which only
+ * square blocks allow: line-block operands give MQ_ERR_UNSUPPORTED. */
+mq_status mq_conv_bwd_data(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, void* dx, int dx_dtype, int dx_layout,
                            void* workspace, size_t ws_bytes, void* stream);
 
 /* mq_conv_bwd_data_static -- the same computation as mq_conv_bwd_data for callers that cannot hand the
@@ -156,15 +175,16 @@ mq_status mq_conv_bwd_data(const mq_conv_desc* desc, const mq_qtensor* wq, const
  * each call overwrites every byte it later reads, so nothing needs clearing, but two calls whose kernels
  * overlap on the GPU (different streams, no ordering between them) race on the array -- order them. */
 #define MQ_STATIC_SCRATCH_BYTES (16u << 20)
-mq_status mq_conv_bwd_data_static(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, void* dx, int dx_layout,
+mq_status mq_conv_bwd_data_static(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, void* dx, int dx_dtype, int dx_layout,
                                   void* stream);
 
 /* mq_conv_bwd_weight -- G_Wf = G_Yf . X'^T (Sec. II-C, IV-B; Eq. 3), K-blocks of 32 samples at one
  * output pixel: the stored X and G_Y are read along N, the other direction of their square blocks.
  * dw: fp32 OIHW ([C_out][C_in][Kh][Kw]) for MQ_NCHW, or [C_out][Kh][Kw][C_in] for MQ_HWNC.
  * The reduction over (ho,wo,n) is split across thread blocks through `workspace` and summed in a
- * fixed order (deterministic). */
-mq_status mq_conv_bwd_weight(const mq_conv_desc* desc, const mq_qtensor* xq, const mq_qtensor* dyq, void* dw, int dw_layout,
+ * fixed order (deterministic).  dw: `dw_dtype` elements (MQ_F32).  Line-block operands give MQ_ERR_UNSUPPORTED
+ * (the contraction runs along N, across the lines). */
+mq_status mq_conv_bwd_weight(const mq_conv_desc* desc, const mq_qtensor* xq, const mq_qtensor* dyq, void* dw, int dw_dtype, int dw_layout,
                              void* workspace, size_t ws_bytes, void* stream);
 
 /* mq_conv_layer_host -- one whole pass of the path for a layer whose tensors live in HOST memory:

@@ -16,6 +16,8 @@ namespace {
 
 bool valid_fmt(int f) { return f == MQ_E4M3 || f == MQ_E5M2 || f == MQ_E2M1 || f == MQ_E3M2 || f == MQ_E2M3; }
 bool valid_role(int r) { return r == MQ_ROLE_X || r == MQ_ROLE_W || r == MQ_ROLE_DY; }
+bool valid_block(int b) { return b == MQ_BLOCK_TILE32 || b == MQ_BLOCK_LINE32; }
+bool valid_dtype(int t) { return t == MQ_F32 || t == MQ_BF16; }
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 mq_status check_desc(const mq_conv_desc* d) {
@@ -36,18 +38,18 @@ View view_of(const Geom& g, int role) {
   return v;
 }
 
-void sizes_of(const Geom& g, int role, int fmt, size_t* cb, size_t* sb) {
+void sizes_of(const Geom& g, int role, int fmt, int block, size_t* cb, size_t* sb) {
   View v = view_of(g, role);
   *cb = (size_t)(v.P * v.R * v.Cp) * fmt_bits(fmt) / 8;
-  *sb = (size_t)(v.P * ((v.R + 31) / 32) * (v.Cp / 32));
+  *sb = (size_t)(v.P * (block == MQ_BLOCK_LINE32 ? v.R : (v.R + 31) / 32) * (v.Cp / 32));
 }
 
 mq_status check_qtensor(const Geom& g, const mq_qtensor* q, int role) {
   if (!q || !q->codes || !q->scales) return MQ_ERR_INVALID_ARG;
-  if (!valid_fmt(q->fmt) || q->role != role) return MQ_ERR_INVALID_ARG;
+  if (!valid_fmt(q->fmt) || q->role != role || !valid_block(q->block)) return MQ_ERR_INVALID_ARG;
   if (!aligned16(q->codes) || !aligned16(q->scales)) return MQ_ERR_ALIGNMENT;
   size_t cb, sb;
-  sizes_of(g, role, q->fmt, &cb, &sb);
+  sizes_of(g, role, q->fmt, q->block, &cb, &sb);
   if (q->codes_bytes < cb || q->scales_bytes < sb) return MQ_ERR_BUFFER_TOO_SMALL;
   return MQ_OK;
 }
@@ -115,7 +117,7 @@ struct ConvTcPlan {
   size_t off_wt_scales, off_sfa, off_sfb, off_bimg, off_pack_a, off_pack_b, total;   // off_pack_*: packed copies of 6-bit operands
 };
 
-bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, ConvTcPlan* out) {
+bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, ConvTcPlan* out, bool line = false) {
   const bool fp4 = fmt_w == MQ_E2M1;
   const int bits = fp4 ? 4 : 8;
   const int taps = g.Kh * g.Kw;
@@ -139,7 +141,9 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   p.G = 128 / p.KB;
   p.cpt = rowbytes / p.KB;
   const int w_eff = op == MQ_OP_FWD ? g.Wo : (g.W + g.sw - 1) / g.sw;
-  const bool thin = g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && !env_int("MQ_TC_NO_HALO", 0);
+  // line blocks (one scale per row): the per-tap kernel, whose preparation launch lays out the scale vectors row by row
+  const bool thin = !line && g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && !env_int("MQ_TC_NO_HALO", 0);
+  p.line = line ? 1 : 0;
   const int cd16 = (p.Cd + 15) / 16 * 16;
   p.BN = cd16 <= 128 ? cd16 : 128;
   // 256-channel tiles halve the re-reads of the activation tile but leave tensor memory for one accumulator only, so
@@ -223,7 +227,7 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   // whole-tile-per-stage variant: stride 1, one chunk per tap (<= 64 bytes of channels).  One box with the column
   // halo needs 8-column tiles; one box per column shift takes 8, 16 or 32 columns (longer NCHW store runs).
   p.halo = 0;
-  if (g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && taps <= 64 && !env_int("MQ_TC_NO_HALO", 0)) {
+  if (!line && g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && taps <= 64 && !env_int("MQ_TC_NO_HALO", 0)) {
     const int spa = fp4 ? 2 : 1, atoms_b = (p.BN + 127) / 128;
     if (p.TW == 8) {
       p.WH = p.TW + g.Kw - 1;
@@ -265,11 +269,11 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   return true;
 }
 
-size_t conv_tc_workspace(int op, const Geom& g, int fmt_x_like, int fmt_w) {
+size_t conv_tc_workspace(int op, const Geom& g, int fmt_x_like, int fmt_w, bool line) {
   size_t need = 0;
   for (int layout = 0; layout < 2; ++layout) {   // the tile shape, hence the scratch, depends on the output layout
     ConvTcPlan pl;
-    if (conv_tc_plan(op, g, fmt_x_like, fmt_w, layout, &pl) && pl.total > need) need = pl.total;
+    if (conv_tc_plan(op, g, fmt_x_like, fmt_w, layout, &pl, line) && pl.total > need) need = pl.total;
   }
   return need;
 }
@@ -277,7 +281,7 @@ size_t conv_tc_workspace(int op, const Geom& g, int fmt_x_like, int fmt_w) {
 mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq_qtensor* qw, float* out, int layout, void* ws,
                       unsigned int* status, cudaStream_t stream) {
   ConvTcPlan pl;
-  if (!conv_tc_plan(op, g, qx_like->fmt, qw->fmt, layout, &pl)) return MQ_ERR_UNSUPPORTED;
+  if (!conv_tc_plan(op, g, qx_like->fmt, qw->fmt, layout, &pl, qx_like->block == MQ_BLOCK_LINE32)) return MQ_ERR_UNSUPPORTED;
   ConvTcParams& p = pl.p;
   const int taps = g.Kh * g.Kw;
   uint8_t* base = static_cast<uint8_t*>(ws);
@@ -591,7 +595,8 @@ unsigned int* device_status_ptr() {
 }
 
 // argument checks common to the three convolution entry points (everything but the workspace)
-mq_status check_conv_args(const mq_conv_desc* desc, const mq_qtensor* qa, int role_a, const mq_qtensor* qb, int role_b, const void* out, int layout) {
+mq_status check_conv_args(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int role_a, const mq_qtensor* qb, int role_b, const void* out, int dtype,
+                          int layout) {
   mq_status st = check_desc(desc);
   if (st != MQ_OK) return st;
   const Geom g = make_geom(*desc);
@@ -599,18 +604,23 @@ mq_status check_conv_args(const mq_conv_desc* desc, const mq_qtensor* qa, int ro
   if ((st = check_qtensor(g, qb, role_b)) != MQ_OK) return st;
   if (!out) return MQ_ERR_INVALID_ARG;
   if (layout != MQ_NCHW && layout != MQ_HWNC) return MQ_ERR_INVALID_ARG;
+  if (!valid_dtype(dtype)) return MQ_ERR_INVALID_ARG;
   if (!aligned16(out)) return MQ_ERR_ALIGNMENT;
+  if (qa->block != qb->block) return MQ_ERR_UNSUPPORTED;
+  // a line-quantized tensor serves the GEMM that contracts along its lines and no other (Sec. III-B, III-C)
+  if (qa->block == MQ_BLOCK_LINE32 && op != MQ_OP_FWD) return MQ_ERR_UNSUPPORTED;
+  if (dtype != MQ_F32) return MQ_ERR_UNSUPPORTED;
   return MQ_OK;
 }
 
 mq_status run_conv(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int role_a, const mq_qtensor* qb, int role_b,
-                   void* out, int layout, void* ws, size_t ws_bytes, void* stream) {
-  mq_status st = check_conv_args(desc, qa, role_a, qb, role_b, out, layout);
+                   void* out, int dtype, int layout, void* ws, size_t ws_bytes, void* stream) {
+  mq_status st = check_conv_args(op, desc, qa, role_a, qb, role_b, out, dtype, layout);
   if (st != MQ_OK) return st;
   Geom g = make_geom(*desc);
   if (ws && !aligned16(ws)) return MQ_ERR_ALIGNMENT;
   size_t need = 0;
-  mq_workspace_size(desc, op, qa->fmt, qb->fmt, &need);
+  mq_workspace_size(desc, op, qa->fmt, qb->fmt, qa->block, &need);
   if (need > 0 && (!ws || ws_bytes < need)) return MQ_ERR_BUFFER_TOO_SMALL;
   if (op == MQ_OP_FWD && conv_tc_eligible(op, g, qa->fmt, qb->fmt))
     return run_conv_tc(op, g, qa, qb, static_cast<float*>(out), layout, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
@@ -625,6 +635,7 @@ mq_status run_conv(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int r
   a.a_codes = static_cast<const uint8_t*>(qa->codes); a.a_scales = qa->scales; a.fmt_a = qa->fmt;
   a.b_codes = static_cast<const uint8_t*>(qb->codes); a.b_scales = qb->scales; a.fmt_b = qb->fmt;
   a.out = static_cast<float*>(out); a.out_layout = layout; a.workspace = ws; a.ws_bytes = ws_bytes;
+  a.line = qa->block == MQ_BLOCK_LINE32 ? 1 : 0;
   cudaError_t e = launch_conv_generic(op, a, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }
@@ -643,33 +654,35 @@ using namespace mq;
 
 extern "C" {
 
-mq_status mq_qtensor_sizes(const mq_conv_desc* desc, int role, int fmt, size_t* codes_bytes, size_t* scales_bytes) {
+mq_status mq_qtensor_sizes(const mq_conv_desc* desc, int role, int fmt, int block, size_t* codes_bytes, size_t* scales_bytes) {
   mq_status st = check_desc(desc);
   if (st != MQ_OK) return st;
-  if (!valid_role(role) || !valid_fmt(fmt) || !codes_bytes || !scales_bytes) return MQ_ERR_INVALID_ARG;
-  sizes_of(make_geom(*desc), role, fmt, codes_bytes, scales_bytes);
+  if (!valid_role(role) || !valid_fmt(fmt) || !valid_block(block) || !codes_bytes || !scales_bytes) return MQ_ERR_INVALID_ARG;
+  sizes_of(make_geom(*desc), role, fmt, block, codes_bytes, scales_bytes);
   return MQ_OK;
 }
 
-mq_status mq_im2col_sizes(const mq_conv_desc* desc, int fmt, size_t* codes_bytes, size_t* scales_bytes) {
+mq_status mq_im2col_sizes(const mq_conv_desc* desc, int fmt, int block, size_t* codes_bytes, size_t* scales_bytes) {
   mq_status st = check_desc(desc);
   if (st != MQ_OK) return st;
-  if (!valid_fmt(fmt) || !codes_bytes || !scales_bytes) return MQ_ERR_INVALID_ARG;
+  if (!valid_fmt(fmt) || !valid_block(block) || !codes_bytes || !scales_bytes) return MQ_ERR_INVALID_ARG;
   Geom g = make_geom(*desc);
   *codes_bytes = (size_t)g.Ho * g.Wo * g.N * g.Kh * g.Kw * g.Cp * fmt_bits(fmt) / 8;
-  *scales_bytes = (size_t)g.Ho * g.Wo * g.Nt * g.Kh * g.Kw * g.Ct;
+  *scales_bytes = (size_t)g.Ho * g.Wo * (block == MQ_BLOCK_LINE32 ? g.N : g.Nt) * g.Kh * g.Kw * g.Ct;
   return MQ_OK;
 }
 
-mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt_b, size_t* bytes) {
+mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt_b, int block, size_t* bytes) {
   mq_status st = check_desc(desc);
   if (st != MQ_OK) return st;
-  if (!valid_fmt(fmt_a) || !valid_fmt(fmt_b) || !bytes) return MQ_ERR_INVALID_ARG;
+  if (!valid_fmt(fmt_a) || !valid_fmt(fmt_b) || !valid_block(block) || !bytes) return MQ_ERR_INVALID_ARG;
   if (op != MQ_OP_FWD && op != MQ_OP_BWD_DATA && op != MQ_OP_BWD_WEIGHT) return MQ_ERR_INVALID_ARG;
+  if (block == MQ_BLOCK_LINE32 && op != MQ_OP_FWD) return MQ_ERR_UNSUPPORTED;
   const Geom g = make_geom(*desc);
+  const bool line = block == MQ_BLOCK_LINE32;
   *bytes = conv_generic_workspace(op, g);
-  if (op == MQ_OP_FWD && conv_tc_eligible(op, g, fmt_a, fmt_b)) *bytes = conv_tc_workspace(op, g, fmt_a, fmt_b);
-  if (op == MQ_OP_BWD_DATA && conv_tc_eligible(op, g, fmt_b, fmt_a)) *bytes = conv_tc_workspace(op, g, fmt_b, fmt_a);
+  if (op == MQ_OP_FWD && conv_tc_eligible(op, g, fmt_a, fmt_b)) *bytes = conv_tc_workspace(op, g, fmt_a, fmt_b, line);
+  if (op == MQ_OP_BWD_DATA && conv_tc_eligible(op, g, fmt_b, fmt_a)) *bytes = conv_tc_workspace(op, g, fmt_b, fmt_a, false);
   if (op == MQ_OP_BWD_WEIGHT) {
     const WgradPlan w = wgrad_plan(g, fmt_a, fmt_b);
     if (w.ok) *bytes = w.total;
@@ -677,22 +690,25 @@ mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt
   return MQ_OK;
 }
 
-static mq_status quantize_impl(const mq_conv_desc* desc, const void* src, int src_layout, mq_qtensor* dst, int sr, unsigned long long seed,
+static mq_status quantize_impl(const mq_conv_desc* desc, const void* src, int src_dtype, int src_layout, mq_qtensor* dst, int sr, unsigned long long seed,
                                void* stream, unsigned wait_limit = 0, int skip_loads = 0) {
   mq_status st = check_desc(desc);
   if (st != MQ_OK) return st;
   if (!src || !dst || !valid_role(dst->role)) return MQ_ERR_INVALID_ARG;
   if (src_layout != MQ_NCHW && src_layout != MQ_HWNC) return MQ_ERR_INVALID_ARG;
+  if (!valid_dtype(src_dtype)) return MQ_ERR_INVALID_ARG;
   Geom g = make_geom(*desc);
   if ((st = check_qtensor(g, dst, dst->role)) != MQ_OK) return st;
   if (!aligned16(src)) return MQ_ERR_ALIGNMENT;
+  if (src_dtype != MQ_F32) return MQ_ERR_UNSUPPORTED;
   View v = view_of(g, dst->role);
   QuantArgs a;
   a.src = static_cast<const float*>(src);
   a.codes = static_cast<uint8_t*>(dst->codes);
   a.scales = dst->scales;
   a.P = (int)v.P; a.R = (int)v.R; a.C = (int)v.C; a.Cp = (int)v.Cp;
-  const long long Rt = (v.R + 31) / 32, Ct = v.Cp / 32;
+  a.line = dst->block == MQ_BLOCK_LINE32 ? 1 : 0;
+  const long long Rt = a.line ? v.R : (v.R + 31) / 32, Ct = v.Cp / 32;   // scale rows per position
   if (dst->role == MQ_ROLE_W) {  // [r][p][c]
     a.out_stride_p = v.Cp; a.out_stride_r = v.P * v.Cp;
     a.sc_stride_p = Ct; a.sc_stride_r = v.P * Ct;
@@ -716,19 +732,21 @@ static mq_status quantize_impl(const mq_conv_desc* desc, const void* src, int sr
   return e == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }
 
-mq_status mq_quantize(const mq_conv_desc* desc, const void* src, int src_layout, mq_qtensor* dst, void* stream) {
-  return quantize_impl(desc, src, src_layout, dst, 0, 0ull, stream);
+mq_status mq_quantize(const mq_conv_desc* desc, const void* src, int src_dtype, int src_layout, mq_qtensor* dst, void* stream) {
+  return quantize_impl(desc, src, src_dtype, src_layout, dst, 0, 0ull, stream);
 }
 
-mq_status mq_quantize_sr(const mq_conv_desc* desc, const void* src, int src_layout, mq_qtensor* dst, unsigned long long seed, void* stream) {
-  return quantize_impl(desc, src, src_layout, dst, 1, seed, stream);
+mq_status mq_quantize_sr(const mq_conv_desc* desc, const void* src, int src_dtype, int src_layout, mq_qtensor* dst, unsigned long long seed,
+                         void* stream) {
+  return quantize_impl(desc, src, src_dtype, src_layout, dst, 1, seed, stream);
 }
 
 mq_status mq_selftest_wait_timeout(const mq_conv_desc* desc, const void* src, mq_qtensor* dst, unsigned polls, void* stream) {
   if (polls == 0 || polls > (1u << 20)) return MQ_ERR_INVALID_ARG;
   if (dst && dst->role == MQ_ROLE_W) return MQ_ERR_UNSUPPORTED;
   if (desc && dst && (long long)(dst->role == MQ_ROLE_X ? desc->H * desc->W : 0) % 4 != 0) return MQ_ERR_UNSUPPORTED;
-  return quantize_impl(desc, src, MQ_NCHW, dst, 0, 0ull, stream, polls, 1);
+  if (dst && dst->block != MQ_BLOCK_TILE32) return MQ_ERR_UNSUPPORTED;
+  return quantize_impl(desc, src, MQ_F32, MQ_NCHW, dst, 0, 0ull, stream, polls, 1);
 }
 
 mq_status mq_cbf_im2col(const mq_conv_desc* desc, const mq_qtensor* xq, void* cols_codes, uint8_t* cols_scales, void* stream) {
@@ -745,23 +763,24 @@ mq_status mq_cbf_im2col(const mq_conv_desc* desc, const mq_qtensor* xq, void* co
   a.out_scales = cols_scales;
   a.g = g;
   a.fmt = xq->fmt;
+  a.line = xq->block == MQ_BLOCK_LINE32 ? 1 : 0;
   cudaError_t e = launch_im2col(a, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }
 
-mq_status mq_conv_fwd(const mq_conv_desc* desc, const mq_qtensor* xq, const mq_qtensor* wq, void* y, int y_layout,
+mq_status mq_conv_fwd(const mq_conv_desc* desc, const mq_qtensor* xq, const mq_qtensor* wq, void* y, int y_dtype, int y_layout,
                       void* workspace, size_t ws_bytes, void* stream) {
-  return run_conv(MQ_OP_FWD, desc, xq, MQ_ROLE_X, wq, MQ_ROLE_W, y, y_layout, workspace, ws_bytes, stream);
+  return run_conv(MQ_OP_FWD, desc, xq, MQ_ROLE_X, wq, MQ_ROLE_W, y, y_dtype, y_layout, workspace, ws_bytes, stream);
 }
 
-mq_status mq_conv_bwd_data(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, void* dx, int dx_layout,
+mq_status mq_conv_bwd_data(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, void* dx, int dx_dtype, int dx_layout,
                            void* workspace, size_t ws_bytes, void* stream) {
-  return run_conv(MQ_OP_BWD_DATA, desc, wq, MQ_ROLE_W, dyq, MQ_ROLE_DY, dx, dx_layout, workspace, ws_bytes, stream);
+  return run_conv(MQ_OP_BWD_DATA, desc, wq, MQ_ROLE_W, dyq, MQ_ROLE_DY, dx, dx_dtype, dx_layout, workspace, ws_bytes, stream);
 }
 
-mq_status mq_conv_bwd_weight(const mq_conv_desc* desc, const mq_qtensor* xq, const mq_qtensor* dyq, void* dw, int dw_layout,
+mq_status mq_conv_bwd_weight(const mq_conv_desc* desc, const mq_qtensor* xq, const mq_qtensor* dyq, void* dw, int dw_dtype, int dw_layout,
                              void* workspace, size_t ws_bytes, void* stream) {
-  return run_conv(MQ_OP_BWD_WEIGHT, desc, xq, MQ_ROLE_X, dyq, MQ_ROLE_DY, dw, dw_layout, workspace, ws_bytes, stream);
+  return run_conv(MQ_OP_BWD_WEIGHT, desc, xq, MQ_ROLE_X, dyq, MQ_ROLE_DY, dw, dw_dtype, dw_layout, workspace, ws_bytes, stream);
 }
 
 // ---- allocation-free variant of mq_conv_bwd_data ---------------------------------------------------
@@ -772,17 +791,17 @@ mq_status mq_conv_bwd_weight(const mq_conv_desc* desc, const mq_qtensor* xq, con
 // host-side table lookup - so no cached address can outlive a cudaDeviceReset of its context.
 static __device__ __align__(256) unsigned char g_static_scratch[MQ_STATIC_SCRATCH_BYTES];
 
-mq_status mq_conv_bwd_data_static(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, void* dx, int dx_layout,
+mq_status mq_conv_bwd_data_static(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, void* dx, int dx_dtype, int dx_layout,
                                   void* stream) {
   // the ordinary call's argument checks first, so that a bad argument is reported as such whatever the layer's size
-  mq_status st = check_conv_args(desc, wq, MQ_ROLE_W, dyq, MQ_ROLE_DY, dx, dx_layout);
+  mq_status st = check_conv_args(MQ_OP_BWD_DATA, desc, wq, MQ_ROLE_W, dyq, MQ_ROLE_DY, dx, dx_dtype, dx_layout);
   if (st != MQ_OK) return st;
   size_t need = 0;
-  if ((st = mq_workspace_size(desc, MQ_OP_BWD_DATA, wq->fmt, dyq->fmt, &need)) != MQ_OK) return st;
+  if ((st = mq_workspace_size(desc, MQ_OP_BWD_DATA, wq->fmt, dyq->fmt, wq->block, &need)) != MQ_OK) return st;
   if (need > MQ_STATIC_SCRATCH_BYTES) return MQ_ERR_STATIC_SCRATCH;
   void* addr = nullptr;
   if (cudaGetSymbolAddress(&addr, g_static_scratch) != cudaSuccess || !addr) return MQ_ERR_CUDA;
-  return run_conv(MQ_OP_BWD_DATA, desc, wq, MQ_ROLE_W, dyq, MQ_ROLE_DY, dx, dx_layout, addr, MQ_STATIC_SCRATCH_BYTES, stream);
+  return run_conv(MQ_OP_BWD_DATA, desc, wq, MQ_ROLE_W, dyq, MQ_ROLE_DY, dx, dx_dtype, dx_layout, addr, MQ_STATIC_SCRATCH_BYTES, stream);
 }
 
 namespace {
@@ -803,15 +822,15 @@ LayerArena layer_arena(const mq_conv_desc* desc, const int fmts[3]) {
   L.off_x = take(L.nx); L.off_w = take(L.nw); L.off_g = take(L.ng);
   L.off_y = take(L.ng); L.off_dx = take(L.nx); L.off_dw = take(L.nw);
   for (int r = 0; r < 3; ++r) {
-    sizes_of(g, r, fmts[r], &L.qc[r], &L.qs[r]);
+    sizes_of(g, r, fmts[r], MQ_BLOCK_TILE32, &L.qc[r], &L.qs[r]);
     L.off_qc[r] = take(L.qc[r]); L.off_qs[r] = take(L.qs[r]);
   }
-  mq_im2col_sizes(desc, fmts[0], &L.ic, &L.is);
+  mq_im2col_sizes(desc, fmts[0], MQ_BLOCK_TILE32, &L.ic, &L.is);
   L.off_ic = take(L.ic); L.off_is = take(L.is);
   L.ws = 0;
   const int ops[3] = {MQ_OP_FWD, MQ_OP_BWD_DATA, MQ_OP_BWD_WEIGHT};
   const int fa[3] = {fmts[0], fmts[1], fmts[0]}, fb[3] = {fmts[1], fmts[2], fmts[2]};
-  for (int i = 0; i < 3; ++i) { size_t b = 0; mq_workspace_size(desc, ops[i], fa[i], fb[i], &b); if (b > L.ws) L.ws = b; }
+  for (int i = 0; i < 3; ++i) { size_t b = 0; mq_workspace_size(desc, ops[i], fa[i], fb[i], MQ_BLOCK_TILE32, &b); if (b > L.ws) L.ws = b; }
   L.off_ws = take(L.ws);
   L.total = o;
   return L;
@@ -872,23 +891,23 @@ mq_status mq_conv_layer_host(const mq_conv_desc* desc, int fmt_x, int fmt_w, int
   const size_t src_off[3] = {L.off_x, L.off_w, L.off_g};
   for (int r = 0; r < 3; ++r) {
     q[r].codes = base + L.off_qc[r]; q[r].scales = base + L.off_qs[r];
-    q[r].codes_bytes = L.qc[r]; q[r].scales_bytes = L.qs[r]; q[r].fmt = fmts[r]; q[r].role = r;
+    q[r].codes_bytes = L.qc[r]; q[r].scales_bytes = L.qs[r]; q[r].fmt = fmts[r]; q[r].role = r; q[r].block = MQ_BLOCK_TILE32;
   }
   void* ws = L.ws ? base + L.off_ws : nullptr;
   if (!ok(cudaStreamWaitEvent(s, hp->ev[1], 0))) return MQ_ERR_CUDA;
-  if ((st = mq_quantize(desc, base + src_off[0], MQ_NCHW, &q[0], stream)) != MQ_OK) return st;
+  if ((st = mq_quantize(desc, base + src_off[0], MQ_F32, MQ_NCHW, &q[0], stream)) != MQ_OK) return st;
   if (!ok(cudaStreamWaitEvent(s, hp->ev[2], 0))) return MQ_ERR_CUDA;
-  if ((st = mq_quantize(desc, base + src_off[1], MQ_NCHW, &q[1], stream)) != MQ_OK) return st;
+  if ((st = mq_quantize(desc, base + src_off[1], MQ_F32, MQ_NCHW, &q[1], stream)) != MQ_OK) return st;
   if ((st = mq_cbf_im2col(desc, &q[0], base + L.off_ic, base + L.off_is, stream)) != MQ_OK) return st;
-  if ((st = mq_conv_fwd(desc, &q[0], &q[1], base + L.off_y, MQ_NCHW, ws, L.ws, stream)) != MQ_OK) return st;
+  if ((st = mq_conv_fwd(desc, &q[0], &q[1], base + L.off_y, MQ_F32, MQ_NCHW, ws, L.ws, stream)) != MQ_OK) return st;
   if (!ok(cudaEventRecord(hp->ev[4], s)) || !ok(cudaStreamWaitEvent(hp->d2h, hp->ev[4], 0))) return MQ_ERR_CUDA;
   if (!ok(cudaMemcpyAsync(y_host, base + L.off_y, L.ng, cudaMemcpyDeviceToHost, hp->d2h))) return MQ_ERR_CUDA;
   if (!ok(cudaStreamWaitEvent(s, hp->ev[3], 0))) return MQ_ERR_CUDA;
-  if ((st = mq_quantize(desc, base + src_off[2], MQ_NCHW, &q[2], stream)) != MQ_OK) return st;
-  if ((st = mq_conv_bwd_data(desc, &q[1], &q[2], base + L.off_dx, MQ_NCHW, ws, L.ws, stream)) != MQ_OK) return st;
+  if ((st = mq_quantize(desc, base + src_off[2], MQ_F32, MQ_NCHW, &q[2], stream)) != MQ_OK) return st;
+  if ((st = mq_conv_bwd_data(desc, &q[1], &q[2], base + L.off_dx, MQ_F32, MQ_NCHW, ws, L.ws, stream)) != MQ_OK) return st;
   if (!ok(cudaEventRecord(hp->ev[5], s)) || !ok(cudaStreamWaitEvent(hp->d2h, hp->ev[5], 0))) return MQ_ERR_CUDA;
   if (!ok(cudaMemcpyAsync(dx_host, base + L.off_dx, L.nx, cudaMemcpyDeviceToHost, hp->d2h))) return MQ_ERR_CUDA;
-  if ((st = mq_conv_bwd_weight(desc, &q[0], &q[2], base + L.off_dw, MQ_NCHW, ws, L.ws, stream)) != MQ_OK) return st;
+  if ((st = mq_conv_bwd_weight(desc, &q[0], &q[2], base + L.off_dw, MQ_F32, MQ_NCHW, ws, L.ws, stream)) != MQ_OK) return st;
   if (!ok(cudaEventRecord(hp->ev[6], s)) || !ok(cudaStreamWaitEvent(hp->d2h, hp->ev[6], 0))) return MQ_ERR_CUDA;
   if (!ok(cudaMemcpyAsync(dw_host, base + L.off_dw, L.nw, cudaMemcpyDeviceToHost, hp->d2h))) return MQ_ERR_CUDA;
   if (!ok(cudaEventRecord(hp->ev[7], hp->d2h)) || !ok(cudaStreamWaitEvent(s, hp->ev[7], 0))) return MQ_ERR_CUDA;

@@ -73,11 +73,11 @@ __global__ void __launch_bounds__(GT) fwd_generic(ConvArgs a) {
     for (int kb = 0; kb < g.Ct; ++kb) {
       float va[8], vb[8];
       if (pix_ok) {
-        float s = e8m0_to_float(a.a_scales[(pix * g.Nt + (n >> 5)) * g.Ct + kb]);
+        float s = e8m0_to_float(a.a_scales[(a.line ? pix * g.N + n : pix * g.Nt + (n >> 5)) * g.Ct + kb]);
         decode8<FX>(a.a_codes, (pix * g.N + n) * g.Cp + kb * 32 + kq * 8, s, va, a.fmt_a);
       } else zero8(va);
       if (co_ok) {
-        float s = e8m0_to_float(a.b_scales[((long long)(co >> 5) * taps + tap) * g.Ct + kb]);
+        float s = e8m0_to_float(a.b_scales[((long long)(a.line ? co : (co >> 5)) * taps + tap) * g.Ct + kb]);
         decode8<FW>(a.b_codes, ((long long)co * taps + tap) * g.Cp + kb * 32 + kq * 8, s, vb, a.fmt_b);
       } else zero8(vb);
       __syncthreads();

@@ -1244,7 +1244,7 @@ __global__ void __launch_bounds__(256) expand_conv_scales_kernel(const ConvTcPar
       const int tw_ = r & (p.TW - 1), tn = r >> p.lgTW;
       const int n = tile.n0 + tn, ws = ws0 + tw_;
       if (n < p.N && hs >= 0 && hs < p.Hs && ws >= 0 && ws < p.Ws)
-        acc[j] = load_scale_bytes<BPC>(p.a_scales + (((long long)hs * p.Ws + ws) * p.Nt + (n >> 5)) * p.Kblocks + pos.cc * BPC);
+        acc[j] = load_scale_bytes<BPC>(p.a_scales + (((long long)hs * p.Ws + ws) * (p.line ? p.N : p.Nt) + (p.line ? n : (n >> 5))) * p.Kblocks + pos.cc * BPC);
     }
     uint8_t* dst = p.sfa_img + (size_t)wid * (512 * SPA) + lane * 16;
 #pragma unroll
@@ -1278,7 +1278,7 @@ __global__ void __launch_bounds__(256) expand_conv_scales_kernel(const ConvTcPar
           const int tw_ = r & (p.TW - 1), tn = r >> p.lgTW;
           const int n = tile.n0 + tn, ws = ws0 + tw_ * wstep;
           if (n < p.N && hs >= 0 && hs < p.Hs && ws >= 0 && ws < p.Ws)
-            acc[j] |= load_scale_bytes<BPC>(p.a_scales + (((long long)hs * p.Ws + ws) * p.Nt + (n >> 5)) * p.Kblocks + pos.cc * BPC) << (8 * c * BPC);
+            acc[j] |= load_scale_bytes<BPC>(p.a_scales + (((long long)hs * p.Ws + ws) * (p.line ? p.N : p.Nt) + (p.line ? n : (n >> 5))) * p.Kblocks + pos.cc * BPC) << (8 * c * BPC);
         }
       }
     }
@@ -1321,6 +1321,10 @@ __global__ void __launch_bounds__(256) expand_conv_scales_kernel(const ConvTcPar
               for (int kb = 0; kb < BPC; ++kb)
                 bytes |= (unsigned long long)__ldg(p.wt_sc_in + ((long long)(pos.cc * BPC + kb) * taps_all + tap) * Ct_w + cib) << (8 * kb);
               acc[j] |= bytes << (8 * c * BPC);
+            } else if (p.line) {
+              // line blocks: every weight row has its own scale per K-block
+              const int row = tile.c0 + 32 * j + lane;
+              if (row < p.b_rows_total) acc[j] |= load_scale_bytes<BPC>(p.b_scales + ((long long)row * taps_all + tap) * p.Kblocks + pos.cc * BPC) << (8 * c * BPC);
             } else {
               acc[j] |= load_scale_bytes<BPC>(p.b_scales + ((long long)((tile.c0 >> 5) + j) * taps_all + tap) * p.Kblocks + pos.cc * BPC) << (8 * c * BPC);
             }

@@ -15,6 +15,7 @@ namespace mq {
 // bwd_data: W re-laid as [C_in_p][taps][C_out_p]).
 struct ConvTcParams {
   int mode;             // MQ_OP_FWD or MQ_OP_BWD_DATA
+  int line;             // 1: line-block scales (forward only): a_scales [Hs][Ws][N][Kblocks], b_scales [rows][taps][Kblocks]
   int kind_fp4;         // 1: both operands E2M1 (kind::mxf4), 0: 8-bit formats (kind::mxf8f6f4)
   uint32_t idesc;       // instruction descriptor without scale ids
   int KB;               // bytes of K per row per TMA box: 128, 64 or 32 (= swizzle span)

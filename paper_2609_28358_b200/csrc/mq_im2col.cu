@@ -69,19 +69,20 @@ __global__ void __launch_bounds__(IC_THREADS) im2col_kernel(Im2colArgs a, int rc
       if (j >= J) { j -= J; ++n; }
     }
   } else {
-    // scales [ho][wo][nt][kh][kw][ct]
-    const long long n_scales = (long long)g.Ho * g.Wo * g.Nt * taps * g.Ct;
+    // scales [ho][wo][nt][kh][kw][ct]; with line blocks one entry per sample: [ho][wo][n][kh][kw][ct]
+    const int Rt = a.line ? g.N : g.Nt;
+    const long long n_scales = (long long)g.Ho * g.Wo * Rt * taps * g.Ct;
     for (long long id = (long long)(blockIdx.x - n_main) * IC_THREADS + threadIdx.x; id < n_scales; id += (long long)(gridDim.x - n_main) * IC_THREADS) {
       long long q = id;
       const int ct = (int)(q % g.Ct); q /= g.Ct;
       const int tap = (int)(q % taps); q /= taps;
-      const int nt = (int)(q % g.Nt); q /= g.Nt;
+      const int nt = (int)(q % Rt); q /= Rt;
       const int wo = (int)(q % g.Wo);
       const int ho = (int)(q / g.Wo);
       const int kh = tap / g.Kw, kw = tap - kh * g.Kw;
       const int h = ho * g.sh + kh - g.ph, w = wo * g.sw + kw - g.pw;
       uint8_t sc = 0;
-      if (h >= 0 && h < g.H && w >= 0 && w < g.W) sc = a.scales[(((long long)h * g.W + w) * g.Nt + nt) * g.Ct + ct];
+      if (h >= 0 && h < g.H && w >= 0 && w < g.W) sc = a.scales[(((long long)h * g.W + w) * Rt + nt) * g.Ct + ct];
       a.out_scales[id] = sc;
     }
   }
@@ -109,13 +110,14 @@ __global__ void __launch_bounds__(IC_THREADS) im2col_generic_kernel(Im2colArgs a
       long long q = id - code_chunks;
       const int ct = (int)(q % g.Ct); q /= g.Ct;
       const int tap = (int)(q % taps); q /= taps;
-      const int nt = (int)(q % g.Nt); q /= g.Nt;
+      const int Rt = a.line ? g.N : g.Nt;
+      const int nt = (int)(q % Rt); q /= Rt;
       const int wo = (int)(q % g.Wo);
       const int ho = (int)(q / g.Wo);
       const int kh = tap / g.Kw, kw = tap - kh * g.Kw;
       const int h = ho * g.sh + kh - g.ph, w = wo * g.sw + kw - g.pw;
       uint8_t sc = 0;
-      if (h >= 0 && h < g.H && w >= 0 && w < g.W) sc = a.scales[(((long long)h * g.W + w) * g.Nt + nt) * g.Ct + ct];
+      if (h >= 0 && h < g.H && w >= 0 && w < g.W) sc = a.scales[(((long long)h * g.W + w) * Rt + nt) * g.Ct + ct];
       a.out_scales[id - code_chunks] = sc;
     }
   }
@@ -133,7 +135,7 @@ cudaError_t launch_im2col(const Im2colArgs& a, cudaStream_t s) {
   if (PX > 8) PX = 8;
   if (PX < 1) PX = 1;
   const long long n_main = (((long long)g.Ho * g.Wo + PX - 1) / PX) * g.Nt;
-  const long long n_scales = (long long)g.Ho * g.Wo * g.Nt * taps * g.Ct;
+  const long long n_scales = (long long)g.Ho * g.Wo * (a.line ? g.N : g.Nt) * taps * g.Ct;
   count_launches(1);
   if (J <= IC_MAX_J && src_chunks < 0x7fffffffLL && n_main < 0x7fff0000LL) {
     long long sc_blocks = (n_scales + IC_THREADS - 1) / IC_THREADS;

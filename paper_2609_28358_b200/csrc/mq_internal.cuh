@@ -61,6 +61,7 @@ struct QuantArgs {
   unsigned sr_seed_lo, sr_seed_hi;   // the 64-bit seed
   unsigned sr_key0;                  // stream key of elements whose index is below 2^32 (computed on the host)
   int sr_wide;                       // 1: the tensor has 2^32 elements or more (keys are derived per element)
+  int line;                          // 1: line blocks (one scale per row and 32 channels; the sc strides are per row), 0: 32 x 32 tiles
   unsigned int* status;              // device status word: set when a bounded wait gives up
   // test hooks of the TMA kernel's abort path: polls a barrier wait may take (0: the default limit), and 1 = the loader
   // issues no copies, so that every wait on them runs out
@@ -81,6 +82,7 @@ struct Im2colArgs {
   uint8_t* out_scales;
   Geom g;
   int fmt;
+  int line;   // 1: line blocks (scales per sample instead of per 32 samples)
 };
 cudaError_t launch_im2col(const Im2colArgs& a, cudaStream_t s);
 
@@ -95,6 +97,7 @@ struct ConvArgs {
   int out_layout;
   void* workspace;
   size_t ws_bytes;
+  int line;   // 1: both operands carry line-block scales (one per row), forward GEMM only
 };
 // CUDA-core implicit-GEMM kernels: every shape, every format pair.
 cudaError_t launch_conv_generic(int op, const ConvArgs& a, cudaStream_t s);

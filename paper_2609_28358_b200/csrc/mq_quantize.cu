@@ -277,9 +277,12 @@ __global__ void __launch_bounds__(NT) quantize_pipe_kernel(QuantArgs a, int n_ps
 }
 
 // Fallback for sources whose position axis is not a multiple of 4 elements (no 16-byte rows): one block per item.
-template <int FMT, bool SR>
+// LINE: line blocks - one scale per (position, row, 32 channels) instead of one per tile; the 32 channels of a line sit in
+// 16 lanes of each of two neighbouring warps (shuffles, then one exchange through shared memory).
+template <int FMT, bool SR, bool LINE = false>
 __global__ void __launch_bounds__(QT_THREADS) quantize_simple_kernel(QuantArgs a, int n_pstrips, int Ct) {
   __shared__ __align__(16) unsigned red[8][2][4];
+  __shared__ unsigned lred[LINE ? 8 : 1][2][8][4];
   __shared__ __align__(16) uint8_t stage[PS][32][32];   // one code per byte
   pdl_wait();
   const int t = threadIdx.x, lane = t & 31, warp = t >> 5;
@@ -296,42 +299,70 @@ __global__ void __launch_bounds__(QT_THREADS) quantize_simple_kernel(QuantArgs a
 #pragma unroll
     for (int j = 0; j < 4; ++j) v[i][j] = (ok && pq + j < a.P) ? __ldg(row + pq + j) : 0.f;
   }
-  unsigned m[4];
+  int code[LINE ? 8 : 1][4];
+  if (LINE) {
+    unsigned lm[8][4];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        unsigned mm = __float_as_uint(v[i][j]) & 0x7fffffffu;
+#pragma unroll
+        for (int off = 2; off < 32; off <<= 1) mm = max(mm, __shfl_xor_sync(0xffffffffu, mm, off));
+        lm[i][j] = mm;
+      }
+    if (lane < 2) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) lred[warp][lane][i][j] = lm[i][j];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        code[i][j] = scale_code_of(max(lm[i][j], lred[warp ^ 1][quad][i][j]), fmt_emax(FMT));
+        // the line's first channel sits in an even warp, lanes 0 (quad 0) and 1 (quad 1)
+        if (c == 0 && q.p0 + 4 * quad + j < a.P && q.r0 + 4 * i + rsub < a.R)
+          a.scales[(long long)(q.p0 + 4 * quad + j) * a.sc_stride_p + (long long)(q.r0 + 4 * i + rsub) * a.sc_stride_r + q.ct] = (uint8_t)code[i][j];
+      }
+  } else {
+    unsigned m[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      unsigned mm = 0;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) mm = max(mm, __float_as_uint(v[i][j]) & 0x7fffffffu);
+#pragma unroll
+      for (int off = 2; off < 32; off <<= 1) mm = max(mm, __shfl_xor_sync(0xffffffffu, mm, off));
+      m[j] = mm;
+    }
+    if (lane < 2) {
+#pragma unroll
+      for (int j = 0; j < 4; ++j) red[warp][lane][j] = m[j];
+    }
+    __syncthreads();
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      unsigned mm = 0;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) mm = max(mm, red[w][quad][j]);
+      code[0][j] = scale_code_of(mm, fmt_emax(FMT));
+    }
+    if (t < PS) {
+      unsigned mm = 0;
+#pragma unroll
+      for (int w = 0; w < 8; ++w) mm = max(mm, red[w][t >> 2][t & 3]);
+      if (q.p0 + t < a.P)
+        a.scales[(long long)(q.p0 + t) * a.sc_stride_p + (long long)q.rt * a.sc_stride_r + q.ct] = (uint8_t)scale_code_of(mm, fmt_emax(FMT));
+    }
+  }
 #pragma unroll
   for (int j = 0; j < 4; ++j) {
-    unsigned mm = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) mm = max(mm, __float_as_uint(v[i][j]) & 0x7fffffffu);
-#pragma unroll
-    for (int off = 2; off < 32; off <<= 1) mm = max(mm, __shfl_xor_sync(0xffffffffu, mm, off));
-    m[j] = mm;
-  }
-  if (lane < 2) {
-#pragma unroll
-    for (int j = 0; j < 4; ++j) red[warp][lane][j] = m[j];
-  }
-  __syncthreads();
-  int code[4];
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    unsigned mm = 0;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) mm = max(mm, red[w][quad][j]);
-    code[j] = scale_code_of(mm, fmt_emax(FMT));
-  }
-  if (t < PS) {
-    unsigned mm = 0;
-#pragma unroll
-    for (int w = 0; w < 8; ++w) mm = max(mm, red[w][t >> 2][t & 3]);
-    if (q.p0 + t < a.P)
-      a.scales[(long long)(q.p0 + t) * a.sc_stride_p + (long long)q.rt * a.sc_stride_r + q.ct] = (uint8_t)scale_code_of(mm, fmt_emax(FMT));
-  }
-#pragma unroll
-  for (int j = 0; j < 4; ++j) {
-    const float f = scale_factor(code[j]);
 #pragma unroll
     for (int i = 0; i < 8; i += 2) {
-      float x0 = v[i][j] * f, x1 = v[i + 1][j] * f;
+      float x0 = v[i][j] * scale_factor(code[LINE ? i : 0][j]), x1 = v[i + 1][j] * scale_factor(code[LINE ? i + 1 : 0][j]);
       if (SR) {
         const long long e0 = ((long long)(q.r0 + 4 * i + rsub) * a.C + (q.c0 + c)) * a.P + pq + j;
         const long long e1 = e0 + 4ll * a.C * a.P;
@@ -421,7 +452,9 @@ __device__ __forceinline__ Item tq_item_of(unsigned it, int n_pstrips, int Ct, i
   return item_of(it, n_pstrips, Ct, 32);
 }
 
-template <int FMT, bool SR>
+// LINE: line blocks.  A line (32 channels of one row at one position) is held by two threads of neighbouring warps; they
+// exchange their maxima through the (still unused) staging buffer and the one with the lower channels writes the scale.
+template <int FMT, bool SR, bool LINE>
 __global__ void __launch_bounds__(TQ_THREADS, 1)
 quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant__ CUtensorMap map_out, QuantArgs a, int n_pstrips, int Ct,
                     unsigned n_items, int strip_fastest) {
@@ -492,13 +525,18 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_con
       const int nb = min(4, (a.R - q.r0 + 7) >> 3);
       float v[4][16];
       float fm = 0.f;
+      float lm[LINE ? 4 : 1];
 #pragma unroll
       for (int b = 0; b < 4; ++b) {
+        if (LINE) { lm[b] = 0.f; }
         if (b < nb) {
           if (!dead && !mbar_wait_limit(&full[slot], phase, limit, a.status, MQ_ERR_TIMEOUT)) { dead = true; *abort_flag = 1; }
           const float* src = rd + (size_t)slot * TQ_BOX_FLOATS;
 #pragma unroll
-          for (int k = 0; k < 16; ++k) { v[b][k] = src[k * 32]; fm = fmaxf(fm, fabsf(v[b][k])); }
+          for (int k = 0; k < 16; ++k) {
+            v[b][k] = src[k * 32];
+            if (LINE) lm[b] = fmaxf(lm[b], fabsf(v[b][k])); else fm = fmaxf(fm, fabsf(v[b][k]));
+          }
           __syncwarp();
           if (lane == 0) tc::mbar_arrive(&empty[slot]);
           if (++slot == TQ_SLOTS) { slot = 0; phase ^= 1; }
@@ -507,20 +545,36 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_con
           for (int k = 0; k < 16; ++k) v[b][k] = 0.f;
         }
       }
-      red[warp * 32 + lane] = __float_as_uint(fm);
+      if (!LINE) red[warp * 32 + lane] = __float_as_uint(fm);
       if (t == 0) tc::bulk_wait_group_read<0>();    // the previous item's store has read the staging buffer
       consumer_sync();
       if (*abort_flag) break;    // uniform: written only between the previous item's last barrier and the one above
-      unsigned mx = 0;
+      int code[LINE ? 4 : 1];
+      if (LINE) {
+        unsigned* xch = reinterpret_cast<unsigned*>(stage);   // [box][warp][lane]
 #pragma unroll
-      for (int w = 0; w < 16; ++w) mx = max(mx, red[w * 32 + lane]);
-      const int code = scale_code_of(mx, fmt_emax(FMT));
-      if (warp == 0 && q.p0 + lane < a.P)
-        a.scales[(long long)(q.p0 + lane) * a.sc_stride_p + (long long)q.rt * a.sc_stride_r + q.ct] = (uint8_t)code;
-      const float f = scale_factor(code);
+        for (int b = 0; b < 4; ++b) xch[(b * 16 + warp) * 32 + lane] = __float_as_uint(lm[b]);
+        consumer_sync();
+#pragma unroll
+        for (int b = 0; b < 4; ++b) {
+          code[b] = scale_code_of(max(__float_as_uint(lm[b]), xch[(b * 16 + (warp ^ 1)) * 32 + lane]), fmt_emax(FMT));
+          const int n = 8 * b + n_sub;
+          if (b < nb && chalf == 0 && q.p0 + lane < a.P && q.r0 + n < a.R)
+            a.scales[(long long)(q.p0 + lane) * a.sc_stride_p + (long long)(q.r0 + n) * a.sc_stride_r + q.ct] = (uint8_t)code[b];
+        }
+        consumer_sync();    // every exchange word has been read before the codes overwrite the buffer
+      } else {
+        unsigned mx = 0;
+#pragma unroll
+        for (int w = 0; w < 16; ++w) mx = max(mx, red[w * 32 + lane]);
+        code[0] = scale_code_of(mx, fmt_emax(FMT));
+        if (warp == 0 && q.p0 + lane < a.P)
+          a.scales[(long long)(q.p0 + lane) * a.sc_stride_p + (long long)q.rt * a.sc_stride_r + q.ct] = (uint8_t)code[0];
+      }
 #pragma unroll
       for (int b = 0; b < 4; ++b) {
         if (b < nb) {
+          const float f = scale_factor(code[LINE ? b : 0]);
           const int n = 8 * b + n_sub;
           unsigned w4[4];
 #pragma unroll
@@ -560,7 +614,7 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_con
 // (cq, rq) = (lane & 7, lane >> 3) loads 4 adjacent channels of rows rq, rq + 4, ... as one 128-bit load each (8 in
 // flight), the amax is a per-lane max plus one redux.sync, and the codes leave as 32-bit words (FP8) or, pairing
 // neighbouring lanes, 32-bit words of 8 E2M1 codes.  VEC = false takes any C and alignment with scalar loads.
-template <int FMT, bool VEC, bool SR>
+template <int FMT, bool VEC, bool SR, bool LINE = false>   // LINE: one scale per row of the tile (line blocks), reduced over the 8 lanes of a row
 __global__ void __launch_bounds__(256) quantize_cfast_kernel(QuantArgs a, unsigned Rt, unsigned Ct, unsigned n_items) {
   pdl_wait();
   const int lane = threadIdx.x & 31;
@@ -587,16 +641,29 @@ __global__ void __launch_bounds__(256) quantize_cfast_kernel(QuantArgs a, unsign
         }
       }
     }
-    float m = 0.f;
+    int code[LINE ? 8 : 1];
+    if (LINE) {
 #pragma unroll
-    for (int i = 0; i < 8; ++i) m = fmaxf(fmaxf(m, fmaxf(fabsf(v[i].x), fabsf(v[i].y))), fmaxf(fabsf(v[i].z), fabsf(v[i].w)));
-    const int code = scale_code_of(__reduce_max_sync(0xffffffffu, __float_as_uint(m)), fmt_emax(FMT));
-    if (lane == 0) a.scales[(long long)pos * a.sc_stride_p + (long long)rt * a.sc_stride_r + ct] = (uint8_t)code;
-    const float f = scale_factor(code);
+      for (int i = 0; i < 8; ++i) {
+        unsigned mm = __float_as_uint(fmaxf(fmaxf(fabsf(v[i].x), fabsf(v[i].y)), fmaxf(fabsf(v[i].z), fabsf(v[i].w))));
+        mm = max(mm, __shfl_xor_sync(0xffffffffu, mm, 1));
+        mm = max(mm, __shfl_xor_sync(0xffffffffu, mm, 2));
+        mm = max(mm, __shfl_xor_sync(0xffffffffu, mm, 4));
+        code[i] = scale_code_of(mm, fmt_emax(FMT));
+        if (cq == 0 && r0 + 4 * i < a.R) a.scales[(long long)pos * a.sc_stride_p + (long long)(r0 + 4 * i) * a.sc_stride_r + ct] = (uint8_t)code[i];
+      }
+    } else {
+      float m = 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) m = fmaxf(fmaxf(m, fmaxf(fabsf(v[i].x), fabsf(v[i].y))), fmaxf(fabsf(v[i].z), fabsf(v[i].w)));
+      code[0] = scale_code_of(__reduce_max_sync(0xffffffffu, __float_as_uint(m)), fmt_emax(FMT));
+      if (lane == 0) a.scales[(long long)pos * a.sc_stride_p + (long long)rt * a.sc_stride_r + ct] = (uint8_t)code[0];
+    }
     const long long pbase = (long long)pos * a.out_stride_p + c0;
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       const int r = r0 + 4 * i;
+      const float f = scale_factor(code[LINE ? i : 0]);
       float x[4] = {v[i].x * f, v[i].y * f, v[i].z * f, v[i].w * f};
       if (SR) {
         const long long e0 = ((long long)r * a.C + c0) * a.P + pos;    // index in the logical tensor, whatever the source order
@@ -624,6 +691,14 @@ cudaError_t launch_q_cfast(const QuantArgs& a, int Ct, cudaStream_t s) {
   const bool vec = a.C % 4 == 0 && a.src_stride_p % 4 == 0 && a.src_stride_r % 4 == 0 && (reinterpret_cast<uintptr_t>(a.src) & 15) == 0;
   long long blocks = (items + 7) / 8;
   if (blocks > 148LL * 64) blocks = 148LL * 64;
+  if (a.line) {
+    if (a.sr) {
+      if (vec) return launch_pdl(quantize_cfast_kernel<FMT, true, true, true>, dim3((unsigned)blocks), dim3(256), 0, s, a, (unsigned)Rt, (unsigned)Ct, (unsigned)items);
+      return launch_pdl(quantize_cfast_kernel<FMT, false, true, true>, dim3((unsigned)blocks), dim3(256), 0, s, a, (unsigned)Rt, (unsigned)Ct, (unsigned)items);
+    }
+    if (vec) return launch_pdl(quantize_cfast_kernel<FMT, true, false, true>, dim3((unsigned)blocks), dim3(256), 0, s, a, (unsigned)Rt, (unsigned)Ct, (unsigned)items);
+    return launch_pdl(quantize_cfast_kernel<FMT, false, false, true>, dim3((unsigned)blocks), dim3(256), 0, s, a, (unsigned)Rt, (unsigned)Ct, (unsigned)items);
+  }
   if (a.sr) {
     if (vec) return launch_pdl(quantize_cfast_kernel<FMT, true, true>, dim3((unsigned)blocks), dim3(256), 0, s, a, (unsigned)Rt, (unsigned)Ct, (unsigned)items);
     return launch_pdl(quantize_cfast_kernel<FMT, false, true>, dim3((unsigned)blocks), dim3(256), 0, s, a, (unsigned)Rt, (unsigned)Ct, (unsigned)items);
@@ -653,9 +728,13 @@ cudaError_t launch_q_tma(const QuantArgs& a, cudaStream_t s) {
   static bool attr_set = false;
   static int strip_fastest = 0;
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(quantize_tma_kernel<FMT, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TQ_SMEM);
+    cudaError_t e = cudaFuncSetAttribute(quantize_tma_kernel<FMT, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TQ_SMEM);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(quantize_tma_kernel<FMT, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TQ_SMEM);
+    e = cudaFuncSetAttribute(quantize_tma_kernel<FMT, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TQ_SMEM);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(quantize_tma_kernel<FMT, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TQ_SMEM);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(quantize_tma_kernel<FMT, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TQ_SMEM);
     if (e != cudaSuccess) return e;
     const char* v = std::getenv("MQ_QUANT_STRIP_FASTEST");
     if (v) strip_fastest = std::atoi(v);
@@ -668,14 +747,22 @@ cudaError_t launch_q_tma(const QuantArgs& a, cudaStream_t s) {
   cudaGetDevice(&dev);
   cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
   const unsigned grid = (unsigned)(n_items < sms ? n_items : sms);
-  if (a.sr) return launch_pdl(quantize_tma_kernel<FMT, true>, dim3(grid), dim3(TQ_THREADS), TQ_SMEM, s, map_in, map_out, a, n_pstrips, Ct, (unsigned)n_items, strip_fastest);
-  return launch_pdl(quantize_tma_kernel<FMT, false>, dim3(grid), dim3(TQ_THREADS), TQ_SMEM, s, map_in, map_out, a, n_pstrips, Ct, (unsigned)n_items, strip_fastest);
+  if (a.line) {
+    if (a.sr) return launch_pdl(quantize_tma_kernel<FMT, true, true>, dim3(grid), dim3(TQ_THREADS), TQ_SMEM, s, map_in, map_out, a, n_pstrips, Ct, (unsigned)n_items, strip_fastest);
+    return launch_pdl(quantize_tma_kernel<FMT, false, true>, dim3(grid), dim3(TQ_THREADS), TQ_SMEM, s, map_in, map_out, a, n_pstrips, Ct, (unsigned)n_items, strip_fastest);
+  }
+  if (a.sr) return launch_pdl(quantize_tma_kernel<FMT, true, false>, dim3(grid), dim3(TQ_THREADS), TQ_SMEM, s, map_in, map_out, a, n_pstrips, Ct, (unsigned)n_items, strip_fastest);
+  return launch_pdl(quantize_tma_kernel<FMT, false, false>, dim3(grid), dim3(TQ_THREADS), TQ_SMEM, s, map_in, map_out, a, n_pstrips, Ct, (unsigned)n_items, strip_fastest);
 }
 
 constexpr size_t QPIPE_SMEM = 2 * QBUF_BYTES + PS * 32 * 32 + 16 * 2 * 4 * sizeof(unsigned);
 
 template <int FMT>
 cudaError_t launch_q(const QuantArgs& a, int n_pstrips, int Ct, long long n_items, bool vec, bool r16, cudaStream_t s) {
+  if (a.line) {   // line blocks without 16-byte rows (large aligned tensors take the whole-line kernel): the one-block-per-item kernel
+    if (a.sr) return launch_pdl(quantize_simple_kernel<FMT, true, true>, dim3((unsigned)n_items), dim3(QT_THREADS), 0, s, a, n_pstrips, Ct);
+    return launch_pdl(quantize_simple_kernel<FMT, false, true>, dim3((unsigned)n_items), dim3(QT_THREADS), 0, s, a, n_pstrips, Ct);
+  }
   if (!vec) {
     if (a.sr) return launch_pdl(quantize_simple_kernel<FMT, true>, dim3((unsigned)n_items), dim3(QT_THREADS), 0, s, a, n_pstrips, Ct);
     return launch_pdl(quantize_simple_kernel<FMT, false>, dim3((unsigned)n_items), dim3(QT_THREADS), 0, s, a, n_pstrips, Ct);
@@ -717,7 +804,7 @@ cudaError_t launch_q(const QuantArgs& a, int n_pstrips, int Ct, long long n_item
 cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s) {
   const bool vec = (a.P % 4 == 0) && ((reinterpret_cast<uintptr_t>(a.src) & 15) == 0);
   // at most 16 rows (e.g. a batch of 16 samples): items of 16 positions, see quantize_pipe_kernel
-  const bool r16 = vec && a.src_stride_r == 0 && a.R <= 16 && !std::getenv("MQ_QUANT_NO_R16");
+  const bool r16 = vec && !a.line && a.src_stride_r == 0 && a.R <= 16 && !std::getenv("MQ_QUANT_NO_R16");
   const int psi = r16 ? 2 * PS : PS;
   const int n_pstrips = (a.P + psi - 1) / psi;
   const int Rt = (a.R + 31) / 32, Ct = a.Cp / 32;
@@ -740,7 +827,7 @@ cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s) {
   // which give a small tensor more blocks to spread over
   const long long elems = (long long)a.P * a.R * a.C;
   const char* tv = std::getenv("MQ_QUANT_TMA");
-  const bool tma = vec && (a.debug_skip_loads || (tv ? std::atoi(tv) != 0 : elems >= (1ll << 22)));
+  const bool tma = vec && (a.debug_skip_loads || (tv ? std::atoi(tv) != 0 : (elems >= (1ll << 22) || (a.line && elems >= (1ll << 18)))));
   if (a.debug_skip_loads && !tma) return cudaErrorInvalidValue;
   if (tma) {
     switch (a.fmt) {

@@ -16,6 +16,8 @@ ConvDesc = namedtuple("ConvDesc", "N C_in H W C_out Kh Kw stride_h stride_w pad_
 E4M3, E5M2, E2M1, E3M2, E2M3 = 0, 1, 2, 3, 4
 ROLE_X, ROLE_W, ROLE_DY = 0, 1, 2
 NCHW, HWNC = 0, 1
+TILE32, LINE32 = 0, 1      # block shape: 32 x 32 squares (default) / 1 x 32 lines along the channel axis
+F32, BF16 = 0, 1
 OP_FWD, OP_BWD_DATA, OP_BWD_WEIGHT = 0, 1, 2
 OK = 0
 
@@ -40,7 +42,7 @@ class _Desc(ctypes.Structure):
 
 class _QTensor(ctypes.Structure):
     _fields_ = [("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("codes_bytes", ctypes.c_size_t),
-                ("scales_bytes", ctypes.c_size_t), ("fmt", ctypes.c_int), ("role", ctypes.c_int)]
+                ("scales_bytes", ctypes.c_size_t), ("fmt", ctypes.c_int), ("role", ctypes.c_int), ("block", ctypes.c_int)]
 
 
 def lib():
@@ -78,11 +80,11 @@ def _stream(stream):
 class QTensor:
     """A stored MX tensor: device uint8 buffers for codes and tile scales."""
 
-    def __init__(self, codes, scales, fmt, role):
-        self.codes, self.scales, self.fmt, self.role = codes, scales, fmt, role
+    def __init__(self, codes, scales, fmt, role, block=TILE32):
+        self.codes, self.scales, self.fmt, self.role, self.block = codes, scales, fmt, role, block
 
     def _c(self):
-        return _QTensor(self.codes.data_ptr(), self.scales.data_ptr(), self.codes.numel(), self.scales.numel(), self.fmt, self.role)
+        return _QTensor(self.codes.data_ptr(), self.scales.data_ptr(), self.codes.numel(), self.scales.numel(), self.fmt, self.role, self.block)
 
 
 def _new(shape, dtype, device):
@@ -92,46 +94,50 @@ def _new(shape, dtype, device):
     return t
 
 
-def qtensor_sizes(desc, role, fmt):
+def qtensor_sizes(desc, role, fmt, block=TILE32):
     cb, sb = ctypes.c_size_t(), ctypes.c_size_t()
-    _check("mq_qtensor_sizes", lib().mq_qtensor_sizes(ctypes.byref(_d(desc)), role, fmt, ctypes.byref(cb), ctypes.byref(sb)))
+    _check("mq_qtensor_sizes", lib().mq_qtensor_sizes(ctypes.byref(_d(desc)), role, fmt, block, ctypes.byref(cb), ctypes.byref(sb)))
     return cb.value, sb.value
 
 
-def im2col_sizes(desc, fmt):
+def im2col_sizes(desc, fmt, block=TILE32):
     cb, sb = ctypes.c_size_t(), ctypes.c_size_t()
-    _check("mq_im2col_sizes", lib().mq_im2col_sizes(ctypes.byref(_d(desc)), fmt, ctypes.byref(cb), ctypes.byref(sb)))
+    _check("mq_im2col_sizes", lib().mq_im2col_sizes(ctypes.byref(_d(desc)), fmt, block, ctypes.byref(cb), ctypes.byref(sb)))
     return cb.value, sb.value
 
 
-def workspace_size(desc, op, fmt_a, fmt_b):
+def workspace_size(desc, op, fmt_a, fmt_b, block=TILE32):
     b = ctypes.c_size_t()
-    _check("mq_workspace_size", lib().mq_workspace_size(ctypes.byref(_d(desc)), op, fmt_a, fmt_b, ctypes.byref(b)))
+    _check("mq_workspace_size", lib().mq_workspace_size(ctypes.byref(_d(desc)), op, fmt_a, fmt_b, block, ctypes.byref(b)))
     return b.value
 
 
-def empty_qtensor(desc, role, fmt, device="cuda"):
-    cb, sb = qtensor_sizes(desc, role, fmt)
-    return QTensor(_new(cb, torch.uint8, device), _new(sb, torch.uint8, device), fmt, role)
+def empty_qtensor(desc, role, fmt, device="cuda", block=TILE32):
+    cb, sb = qtensor_sizes(desc, role, fmt, block)
+    return QTensor(_new(cb, torch.uint8, device), _new(sb, torch.uint8, device), fmt, role, block)
 
 
-def quantize(desc, role, fmt, src, out=None, src_layout=NCHW, stream=None):
-    """mq_quantize: fp32 device tensor (NCHW / OIHW, or channel-fastest with src_layout=HWNC) -> stored MX tensor."""
-    assert src.is_cuda and src.dtype == torch.float32 and src.is_contiguous()
+_DTYPES = {torch.float32: F32, torch.bfloat16: BF16}
+
+
+def quantize(desc, role, fmt, src, out=None, src_layout=NCHW, stream=None, block=TILE32):
+    """mq_quantize: device tensor (NCHW / OIHW, or channel-fastest with src_layout=HWNC) -> stored MX tensor."""
+    assert src.is_cuda and src.dtype in _DTYPES and src.is_contiguous()
     if out is None:
-        out = empty_qtensor(desc, role, fmt, src.device)
+        out = empty_qtensor(desc, role, fmt, src.device, block)
     q = out._c()
-    _check("mq_quantize", lib().mq_quantize(ctypes.byref(_d(desc)), ctypes.c_void_p(src.data_ptr()), src_layout, ctypes.byref(q), _stream(stream)))
+    _check("mq_quantize", lib().mq_quantize(ctypes.byref(_d(desc)), ctypes.c_void_p(src.data_ptr()), _DTYPES[src.dtype], src_layout, ctypes.byref(q),
+                                           _stream(stream)))
     return out
 
 
-def quantize_sr(desc, role, fmt, src, seed, out=None, src_layout=NCHW, stream=None):
+def quantize_sr(desc, role, fmt, src, seed, out=None, src_layout=NCHW, stream=None, block=TILE32):
     """mq_quantize_sr: as quantize(), with stochastic rounding of the elements (the gradient's rounding); `seed` is a 64-bit integer."""
-    assert src.is_cuda and src.dtype == torch.float32 and src.is_contiguous()
+    assert src.is_cuda and src.dtype in _DTYPES and src.is_contiguous()
     if out is None:
-        out = empty_qtensor(desc, role, fmt, src.device)
+        out = empty_qtensor(desc, role, fmt, src.device, block)
     q = out._c()
-    _check("mq_quantize_sr", lib().mq_quantize_sr(ctypes.byref(_d(desc)), ctypes.c_void_p(src.data_ptr()), src_layout, ctypes.byref(q),
+    _check("mq_quantize_sr", lib().mq_quantize_sr(ctypes.byref(_d(desc)), ctypes.c_void_p(src.data_ptr()), _DTYPES[src.dtype], src_layout, ctypes.byref(q),
                                                  ctypes.c_uint64(int(seed) & 0xFFFFFFFFFFFFFFFF), _stream(stream)))
     return out
 
@@ -148,7 +154,7 @@ def selftest_wait_timeout(desc, role, fmt, src, polls=2000, stream=None):
 
 def cbf_im2col(desc, xq, out_codes=None, out_scales=None, stream=None):
     """mq_cbf_im2col: stored quantized activation -> (codes, scales) of X'."""
-    cb, sb = im2col_sizes(desc, xq.fmt)
+    cb, sb = im2col_sizes(desc, xq.fmt, xq.block)
     if out_codes is None:
         out_codes = _new(cb, torch.uint8, xq.codes.device)
     if out_scales is None:
@@ -164,31 +170,31 @@ def _out_hw(desc):
     return ((d.H + 2 * d.pad_h - d.Kh) // d.stride_h + 1, (d.W + 2 * d.pad_w - d.Kw) // d.stride_w + 1)
 
 
-def _conv(name, op, desc, qa, qb, out, shape_nchw, shape_hwnc, layout, workspace, stream):
+def _conv(name, op, desc, qa, qb, out, shape_nchw, shape_hwnc, layout, workspace, stream, dtype=torch.float32):
     dev = qa.codes.device
     if out is None:
-        out = _new(shape_nchw if layout == NCHW else shape_hwnc, torch.float32, dev)
-    need = workspace_size(desc, op, qa.fmt, qb.fmt)
+        out = _new(shape_nchw if layout == NCHW else shape_hwnc, dtype, dev)
+    need = workspace_size(desc, op, qa.fmt, qb.fmt, qa.block)
     if workspace is None and need > 0:
         workspace = _new(need, torch.uint8, dev)
     wp = ctypes.c_void_p(workspace.data_ptr()) if workspace is not None else None
     wn = workspace.numel() * workspace.element_size() if workspace is not None else 0
     a, b = qa._c(), qb._c()
     fn = getattr(lib(), name)
-    _check(name, fn(ctypes.byref(_d(desc)), ctypes.byref(a), ctypes.byref(b), ctypes.c_void_p(out.data_ptr()), layout, wp,
+    _check(name, fn(ctypes.byref(_d(desc)), ctypes.byref(a), ctypes.byref(b), ctypes.c_void_p(out.data_ptr()), _DTYPES[out.dtype], layout, wp,
                     ctypes.c_size_t(wn), _stream(stream)))
     return out
 
 
-def conv_fwd(desc, xq, wq, y=None, layout=NCHW, workspace=None, stream=None):
+def conv_fwd(desc, xq, wq, y=None, layout=NCHW, workspace=None, stream=None, dtype=torch.float32):
     d = ConvDesc(*desc)
     ho, wo = _out_hw(d)
-    return _conv("mq_conv_fwd", OP_FWD, desc, xq, wq, y, (d.N, d.C_out, ho, wo), (ho, wo, d.N, d.C_out), layout, workspace, stream)
+    return _conv("mq_conv_fwd", OP_FWD, desc, xq, wq, y, (d.N, d.C_out, ho, wo), (ho, wo, d.N, d.C_out), layout, workspace, stream, dtype)
 
 
-def conv_bwd_data(desc, wq, dyq, dx=None, layout=NCHW, workspace=None, stream=None):
+def conv_bwd_data(desc, wq, dyq, dx=None, layout=NCHW, workspace=None, stream=None, dtype=torch.float32):
     d = ConvDesc(*desc)
-    return _conv("mq_conv_bwd_data", OP_BWD_DATA, desc, wq, dyq, dx, (d.N, d.C_in, d.H, d.W), (d.H, d.W, d.N, d.C_in), layout, workspace, stream)
+    return _conv("mq_conv_bwd_data", OP_BWD_DATA, desc, wq, dyq, dx, (d.N, d.C_in, d.H, d.W), (d.H, d.W, d.N, d.C_in), layout, workspace, stream, dtype)
 
 
 STATIC_SCRATCH_BYTES = 16 << 20
@@ -204,7 +210,7 @@ def conv_bwd_data_static(desc, wq, dyq, dx=None, layout=NCHW, stream=None):
         dx = _new((d.N, d.C_in, d.H, d.W) if layout == NCHW else (d.H, d.W, d.N, d.C_in), torch.float32, wq.codes.device)
     a, b = wq._c(), dyq._c()
     _check("mq_conv_bwd_data_static", lib().mq_conv_bwd_data_static(ctypes.byref(_d(desc)), ctypes.byref(a), ctypes.byref(b),
-                                                                  ctypes.c_void_p(dx.data_ptr()), layout, _stream(stream)))
+                                                                  ctypes.c_void_p(dx.data_ptr()), _DTYPES[dx.dtype], layout, _stream(stream)))
     return dx
 
 

@@ -50,45 +50,68 @@ def test_size_queries_match_oracle(mq, desc):
     for fmt in (mq.E4M3, mq.E5M2, mq.E2M1, mq.E3M2, mq.E2M3):
         for role in (mq.ROLE_X, mq.ROLE_W, mq.ROLE_DY):
             assert mq.qtensor_sizes(desc, role, fmt) == oracle.qtensor_sizes(desc, role, fmt)
+            assert mq.qtensor_sizes(desc, role, fmt, mq.LINE32) == oracle.qtensor_sizes(desc, role, fmt, (1, 32))
         assert mq.im2col_sizes(desc, fmt) == oracle.im2col_sizes(desc, fmt)
+        assert mq.im2col_sizes(desc, fmt, mq.LINE32) == oracle.im2col_sizes(desc, fmt, (1, 32))
         for op in (mq.OP_FWD, mq.OP_BWD_DATA, mq.OP_BWD_WEIGHT):
             assert mq.workspace_size(desc, op, fmt, fmt) >= 0
+        assert mq.workspace_size(desc, mq.OP_FWD, fmt, fmt, mq.LINE32) >= 0
+        for op in (mq.OP_BWD_DATA, mq.OP_BWD_WEIGHT):      # a line-quantized tensor cannot feed the other contraction direction
+            with pytest.raises(mq.MqError) as e:
+                mq.workspace_size(desc, op, fmt, fmt, mq.LINE32)
+            assert e.value.status == 2
 
 
 def test_bad_arguments_are_rejected_on_the_host(mq):
     L = mq.lib()
     good = mq._d(inputs.conv_desc(8, 32, 8, 8, 32, 3))
     cb, sb = ctypes.c_size_t(), ctypes.c_size_t()
-    assert L.mq_qtensor_sizes(None, 0, 0, ctypes.byref(cb), ctypes.byref(sb)) == 1
-    assert L.mq_qtensor_sizes(ctypes.byref(good), 7, 0, ctypes.byref(cb), ctypes.byref(sb)) == 1
-    assert L.mq_qtensor_sizes(ctypes.byref(good), 0, 9, ctypes.byref(cb), ctypes.byref(sb)) == 1
+    assert L.mq_qtensor_sizes(None, 0, 0, 0, ctypes.byref(cb), ctypes.byref(sb)) == 1
+    assert L.mq_qtensor_sizes(ctypes.byref(good), 7, 0, 0, ctypes.byref(cb), ctypes.byref(sb)) == 1
+    assert L.mq_qtensor_sizes(ctypes.byref(good), 0, 9, 0, ctypes.byref(cb), ctypes.byref(sb)) == 1
+    assert L.mq_qtensor_sizes(ctypes.byref(good), 0, 0, 5, ctypes.byref(cb), ctypes.byref(sb)) == 1   # no such block shape
     bad = mq._d(inputs.conv_desc(8, 32, 8, 8, 32, 3), block_size=16)
-    assert L.mq_qtensor_sizes(ctypes.byref(bad), 0, 0, ctypes.byref(cb), ctypes.byref(sb)) == 2  # unsupported block
+    assert L.mq_qtensor_sizes(ctypes.byref(bad), 0, 0, 0, ctypes.byref(cb), ctypes.byref(sb)) == 2  # unsupported block length
     neg = mq._d(inputs.conv_desc(0, 32, 8, 8, 32, 3))
-    assert L.mq_qtensor_sizes(ctypes.byref(neg), 0, 0, ctypes.byref(cb), ctypes.byref(sb)) == 1
+    assert L.mq_qtensor_sizes(ctypes.byref(neg), 0, 0, 0, ctypes.byref(cb), ctypes.byref(sb)) == 1
     big_k = mq._d(inputs.conv_desc(1, 32, 2, 2, 32, 7, 1, 0))
-    assert L.mq_qtensor_sizes(ctypes.byref(big_k), 0, 0, ctypes.byref(cb), ctypes.byref(sb)) == 1
+    assert L.mq_qtensor_sizes(ctypes.byref(big_k), 0, 0, 0, ctypes.byref(cb), ctypes.byref(sb)) == 1
     # entry points: null / misaligned / undersized buffers never reach a launch
-    q = mq._QTensor(None, None, 0, 0, 0, 0)
-    assert L.mq_quantize(ctypes.byref(good), None, 0, ctypes.byref(q), None) == 1
-    q = mq._QTensor(0x1000, 0x2000, 16, 16, 0, 0)
-    assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), 0, ctypes.byref(q), None) == 4  # too small
-    q = mq._QTensor(0x1008, 0x2000, 1 << 30, 1 << 30, 0, 0)
-    assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), 0, ctypes.byref(q), None) == 3  # alignment
-    q = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 0)
-    assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), 7, ctypes.byref(q), None) == 1  # no such source layout
+    F32, BF16, NCHW = mq.F32, mq.BF16, mq.NCHW
+    q = mq._QTensor(None, None, 0, 0, 0, 0, 0)
+    assert L.mq_quantize(ctypes.byref(good), None, F32, NCHW, ctypes.byref(q), None) == 1
+    q = mq._QTensor(0x1000, 0x2000, 16, 16, 0, 0, 0)
+    assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), F32, NCHW, ctypes.byref(q), None) == 4  # too small
+    q = mq._QTensor(0x1008, 0x2000, 1 << 30, 1 << 30, 0, 0, 0)
+    assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), F32, NCHW, ctypes.byref(q), None) == 3  # alignment
+    q = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 0, 0)
+    assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), F32, 7, ctypes.byref(q), None) == 1  # no such source layout
+    assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), 9, NCHW, ctypes.byref(q), None) == 1  # no such element type
+    assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), BF16, NCHW, ctypes.byref(q), None) == 2  # bf16 source: not in this build
+    qbad = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 0, 3)
+    assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), F32, NCHW, ctypes.byref(qbad), None) == 1  # no such block shape
     # the stochastic-rounding entry point validates the same way (the seed is any 64-bit value)
     seed = ctypes.c_uint64(0xFFFFFFFFFFFFFFFF)
-    assert L.mq_quantize_sr(ctypes.byref(good), None, 0, ctypes.byref(q), seed, None) == 1
-    assert L.mq_quantize_sr(ctypes.byref(good), ctypes.c_void_p(0x3000), 7, ctypes.byref(q), seed, None) == 1
-    assert L.mq_quantize_sr(ctypes.byref(good), ctypes.c_void_p(0x3004), 0, ctypes.byref(q), seed, None) == 3
-    small = mq._QTensor(0x1000, 0x2000, 16, 16, 0, 2)
-    assert L.mq_quantize_sr(ctypes.byref(good), ctypes.c_void_p(0x3000), 0, ctypes.byref(small), seed, None) == 4
+    assert L.mq_quantize_sr(ctypes.byref(good), None, F32, NCHW, ctypes.byref(q), seed, None) == 1
+    assert L.mq_quantize_sr(ctypes.byref(good), ctypes.c_void_p(0x3000), F32, 7, ctypes.byref(q), seed, None) == 1
+    assert L.mq_quantize_sr(ctypes.byref(good), ctypes.c_void_p(0x3004), F32, NCHW, ctypes.byref(q), seed, None) == 3
+    small = mq._QTensor(0x1000, 0x2000, 16, 16, 0, 2, 0)
+    assert L.mq_quantize_sr(ctypes.byref(good), ctypes.c_void_p(0x3000), F32, NCHW, ctypes.byref(small), seed, None) == 4
     assert L.mq_cbf_im2col(ctypes.byref(good), ctypes.byref(q), None, None, None) == 1
-    qw = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 1)
-    assert L.mq_conv_fwd(ctypes.byref(good), ctypes.byref(qw), ctypes.byref(qw), ctypes.c_void_p(0x4000), 0, None, 0, None) == 1  # wrong role
-    assert L.mq_conv_fwd(ctypes.byref(good), ctypes.byref(q), ctypes.byref(qw), ctypes.c_void_p(0x4000), 5, None, 0, None) == 1  # layout
+    qw = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 1, 0)
+    out = ctypes.c_void_p(0x4000)
+    assert L.mq_conv_fwd(ctypes.byref(good), ctypes.byref(qw), ctypes.byref(qw), out, F32, NCHW, None, 0, None) == 1  # wrong role
+    assert L.mq_conv_fwd(ctypes.byref(good), ctypes.byref(q), ctypes.byref(qw), out, F32, 5, None, 0, None) == 1  # layout
+    assert L.mq_conv_fwd(ctypes.byref(good), ctypes.byref(q), ctypes.byref(qw), out, 9, NCHW, None, 0, None) == 1  # element type
+    assert L.mq_conv_fwd(ctypes.byref(good), ctypes.byref(q), ctypes.byref(qw), out, BF16, NCHW, None, 0, None) == 2  # bf16 output: not in this build
     need = mq.workspace_size(inputs.conv_desc(8, 32, 8, 8, 32, 3), mq.OP_BWD_WEIGHT, 0, 0)
-    qg = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 2)
+    qg = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 2, 0)
     if need:
-        assert L.mq_conv_bwd_weight(ctypes.byref(good), ctypes.byref(q), ctypes.byref(qg), ctypes.c_void_p(0x4000), 0, None, 0, None) == 4
+        assert L.mq_conv_bwd_weight(ctypes.byref(good), ctypes.byref(q), ctypes.byref(qg), out, F32, NCHW, None, 0, None) == 4
+    # line blocks: accepted by the forward GEMM only; operands must agree on the block shape
+    ql = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 0, 1)
+    qwl = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 1, 1)
+    qgl = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 2, 1)
+    assert L.mq_conv_fwd(ctypes.byref(good), ctypes.byref(ql), ctypes.byref(qw), out, F32, NCHW, None, 0, None) == 2  # mixed block shapes
+    assert L.mq_conv_bwd_data(ctypes.byref(good), ctypes.byref(qwl), ctypes.byref(qgl), out, F32, NCHW, None, 0, None) == 2
+    assert L.mq_conv_bwd_weight(ctypes.byref(good), ctypes.byref(ql), ctypes.byref(qgl), out, F32, NCHW, None, 0, None) == 2

@@ -64,5 +64,5 @@ def test_static_scratch_variant_rejects_layers_beyond_its_limit():
     # a bad argument is reported as such even on a layer beyond the limit
     lib = mq.lib()
     a, b = wq._c(), gq._c()
-    st = lib.mq_conv_bwd_data_static(ctypes.byref(mq._d(d)), ctypes.byref(a), ctypes.byref(b), None, mq.NCHW, None)
+    st = lib.mq_conv_bwd_data_static(ctypes.byref(mq._d(d)), ctypes.byref(a), ctypes.byref(b), None, mq.F32, mq.NCHW, None)
     assert st == 1   # MQ_ERR_INVALID_ARG: null dx
