@@ -68,6 +68,7 @@ typedef enum { MQ_BLOCK_TILE32 = 0,      /* 32 x 32 square block (Sec. IV-B), th
                MQ_BLOCK_LINE32 = 1 } mq_block; /* 1 x 32 line block along the channel axis (Sec. III-A) */
 typedef enum { MQ_F32 = 0, MQ_BF16 = 1 } mq_dtype;                     /* element type of an unquantized tensor */
 typedef enum { MQ_OP_FWD = 0, MQ_OP_BWD_DATA = 1, MQ_OP_BWD_WEIGHT = 2 } mq_op;
+typedef enum { MQ_ACT_NONE = 0, MQ_ACT_RELU = 1, MQ_ACT_SILU = 2 } mq_act;   /* activation of the quantizing producer epilogue */
 
 /* One convolution layer (Sec. II-A).  block_size must be 32 (the E8M0 block length). */
 typedef struct {
@@ -178,6 +179,29 @@ mq_status mq_conv_bwd_data(const mq_conv_desc* desc, const mq_qtensor* wq, const
 mq_status mq_conv_bwd_data_static(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, void* dx, int dx_dtype, int dx_layout,
                                   void* stream);
 
+/* Producer epilogue that quantizes.  The paper's cost model quantizes a tensor on chip, when its producer has it, and only
+ * then stores it (Sec. V, the DRAM model: activations leave the chip in their quantized form); these two calls are the
+ * GEMMs above with that order: the epilogue applies the activation and writes the NEXT tensor's stored MX form instead
+ * of fp32, so the fp32 tensor never exists in HBM and the separate mq_quantize pass over it disappears.
+ *
+ * mq_conv_fwd_mx:      Y = act(conv(X, W)), emitted as the stored activation of the next layer: yq has role MQ_ROLE_X
+ *                      and the layouts of a role-X tensor of N x C_out x Ho x Wo (codes [Ho][Wo][N][C_out_p], scales
+ *                      [Ho][Wo][ceil(N/32)][C_out_p/32]); yq->fmt selects its element format.
+ *                      act (mq_act): none, ReLU max(y, 0), or SiLU y / (1 + exp(-y)), evaluated in fp32.
+ * mq_conv_bwd_data_mx: G_X, emitted as the stored output gradient of the previous layer: dxq has role MQ_ROLE_DY and the
+ *                      layouts of N x C_in x H x W (codes [H][W][N][C_in_p], scales [H][W][ceil(N/32)][C_in_p/32]).
+ * Arithmetic of the emitted tensor: exactly mq_quantize's (tile amax over valid elements of the fp32 result, E8M0 floor
+ * rule, round-to-nearest-even, saturating, padded channels code 0) applied to the fp32-accumulated GEMM result.
+ * Square blocks only.  Layers the tensor-core kernels do not take (a tap's channel row not a multiple of 32 bytes, an
+ * E2M1 operand mixed with a one-byte format) give the same result in two launches inside the call: the CUDA-core GEMM
+ * writes fp32 into the workspace and the quantizer, applying the activation, reads it back.
+ * workspace: ws_bytes >= mq_conv_mx_workspace_size(desc, op, fmt of the first operand, fmt of the second). */
+mq_status mq_conv_mx_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt_b, size_t* bytes);
+mq_status mq_conv_fwd_mx(const mq_conv_desc* desc, const mq_qtensor* xq, const mq_qtensor* wq, int act, mq_qtensor* yq, void* workspace,
+                         size_t ws_bytes, void* stream);
+mq_status mq_conv_bwd_data_mx(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, mq_qtensor* dxq, void* workspace,
+                              size_t ws_bytes, void* stream);
+
 /* mq_conv_bwd_weight -- G_Wf = G_Yf . X'^T (Sec. II-C, IV-B; Eq. 3), K-blocks of 32 samples at one
  * output pixel: the stored X and G_Y are read along N, the other direction of their square blocks.
  * dw: fp32 OIHW ([C_out][C_in][Kh][Kw]) for MQ_NCHW, or [C_out][Kh][Kw][C_in] for MQ_HWNC.
@@ -203,6 +227,11 @@ mq_status mq_conv_layer_host(const mq_conv_desc* desc, int fmt_x, int fmt_w, int
 
 /* Diagnostic: how many kernels this library has launched so far in this process (all entry points). */
 unsigned long long mq_kernel_launch_count(void);
+
+/* Diagnostic: the library's MQ_* environment knobs (alternate kernel paths, kept for testing and measurement) are read
+ * once each, on first use, so that mq_workspace_size and the call it sizes always plan alike.  This call makes the next
+ * use of every knob read the environment again.  Not for use while another thread is inside the library. */
+void mq_reload_env(void);
 
 /* Diagnostic self-test of the give-up path of the library's bounded device-side waits (the paper has no counterpart).
  * Launches the quantizer's TMA pipeline for role X or DY (dst->role; H*W resp. Ho*Wo a multiple of 4, else

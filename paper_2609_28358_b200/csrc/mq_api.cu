@@ -1,6 +1,9 @@
 // extern "C" entry points: argument validation, size arithmetic, kernel selection.
 #include <atomic>
 #include <cstdlib>
+#include <map>
+#include <mutex>
+#include <string>
 
 #include "mq_internal.cuh"
 #include "mq_conv_tc.cuh"
@@ -11,6 +14,23 @@ __device__ unsigned int g_device_status = 0;  // set by kernels when a bounded w
 
 static std::atomic<unsigned long long> g_launches{0};
 void count_launches(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
+// environment knobs, read once each (see mq_internal.cuh)
+static std::mutex g_env_mutex;
+static std::map<std::string, std::pair<bool, int>> g_env;   // name -> (set in the environment, value)
+int env_int(const char* name, int dflt) {
+  std::lock_guard<std::mutex> lock(g_env_mutex);
+  auto it = g_env.find(name);
+  if (it == g_env.end()) {
+    const char* v = std::getenv(name);
+    it = g_env.emplace(name, std::make_pair(v != nullptr, v ? std::atoi(v) : 0)).first;
+  }
+  return it->second.first ? it->second.second : dflt;
+}
+static void env_forget() {
+  std::lock_guard<std::mutex> lock(g_env_mutex);
+  g_env.clear();
+}
 
 namespace {
 
@@ -56,10 +76,6 @@ mq_status check_qtensor(const Geom& g, const mq_qtensor* q, int role) {
 
 
 // ---- tensor-core path: eligibility, tile shape, tensor maps ------------------------------------
-int env_int(const char* name, int dflt) {
-  const char* v = std::getenv(name);
-  return v ? std::atoi(v) : dflt;
-}
 
 // fwd / bwd_data run on the tcgen05 kernel when both operands are 8-bit formats or both are E2M1 and a
 // tap's channel row is a whole number of 32-byte MMA K-atoms.
@@ -117,7 +133,9 @@ struct ConvTcPlan {
   size_t off_wt_scales, off_sfa, off_sfb, off_bimg, off_pack_a, off_pack_b, total;   // off_pack_*: packed copies of 6-bit operands
 };
 
-bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, ConvTcPlan* out, bool line = false) {
+// line: line-block operands (forward only).  mx: the quantizing epilogue (tiles of at most 4 output columns, channel tiles
+// of whole 32-channel blocks, per-tap kernel).
+bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, ConvTcPlan* out, bool line = false, bool mx = false) {
   const bool fp4 = fmt_w == MQ_E2M1;
   const int bits = fp4 ? 4 : 8;
   const int taps = g.Kh * g.Kw;
@@ -142,10 +160,11 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   p.cpt = rowbytes / p.KB;
   const int w_eff = op == MQ_OP_FWD ? g.Wo : (g.W + g.sw - 1) / g.sw;
   // line blocks (one scale per row): the per-tap kernel, whose preparation launch lays out the scale vectors row by row
-  const bool thin = !line && g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && !env_int("MQ_TC_NO_HALO", 0);
+  const bool thin = !line && !mx && g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && !env_int("MQ_TC_NO_HALO", 0);
   p.line = line ? 1 : 0;
-  const int cd16 = (p.Cd + 15) / 16 * 16;
+  const int cd16 = mx ? (p.Cd + 31) / 32 * 32 : (p.Cd + 15) / 16 * 16;
   p.BN = cd16 <= 128 ? cd16 : 128;
+  p.mx_out = mx ? 1 : 0;
   // 256-channel tiles halve the re-reads of the activation tile but leave tensor memory for one accumulator only, so
   // the epilogue no longer overlaps the next tile: worth it for 8-bit layers whose main loop is long (measured: +30 %
   // at 2304+ bytes of K per row)
@@ -161,8 +180,16 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
     // with a single accumulator the store time adds to the tile's time instead of hiding behind the next tile: wider
     // tiles (longer store runs) then win - as long as the activations stay in L2 (measured: 28x28 -11 %, 56x56 +11 %)
     const bool serial = bn_ > 128 && act_bytes <= 110e6;
-    const bool pair_hint = op == MQ_OP_BWD_DATA && g.sw == 2 && layout == MQ_NCHW && p.Wd % 2 == 0 && bn_ <= 128 && !env_int("MQ_TC_NO_PAIR", 0);
+    const bool pair_hint = !mx && op == MQ_OP_BWD_DATA && g.sw == 2 && layout == MQ_NCHW && p.Wd % 2 == 0 && bn_ <= 128 && !env_int("MQ_TC_NO_PAIR", 0);
     p.TW = choose_tw(w_eff, g.N, layout, (double)nkh_ * nkw_ * rowbytes, bn_ < 128 ? bn_ : (serial ? bn_ : 128), thin, serial, pair_hint);
+    if (mx) {   // a sample tile (32 samples) must lie inside a GEMM tile: 1, 2 or 4 columns; the least edge padding wins, then the widest
+      double best = 1e30;
+      for (int tw = 4; tw >= 1; tw >>= 1) {
+        const int tn = 128 / tw;
+        const double waste = (double)((w_eff + tw - 1) / tw * tw) / w_eff * (double)((g.N + tn - 1) / tn * tn) / g.N;
+        if (waste < best * (1.0 - 1e-9)) { best = waste; p.TW = tw; }
+      }
+    }
   }
   if (p.TW < 1 || p.TW > 32 || (p.TW & (p.TW - 1))) return false;
   p.TN = 128 / p.TW;
@@ -170,6 +197,7 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   while ((1 << p.lgTW) < p.TW) ++p.lgTW;
   const int forced_bn = env_int("MQ_TC_BN", 0);
   if (forced_bn >= 32 && forced_bn <= 256 && forced_bn % 32 == 0) p.BN = forced_bn < cd16 ? forced_bn : cd16;
+  if (mx && (p.BN % 32 != 0 || p.TW > 4)) return false;
   p.tiles_c = (p.Cd + p.BN - 1) / p.BN;
   p.tiles_w = (w_eff + p.TW - 1) / p.TW;
   p.tiles_n = (g.N + p.TN - 1) / p.TN;
@@ -194,7 +222,7 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
                             (layout == MQ_NCHW ? p.Wd % 4 == 0 : (p.Cd % 4 == 0 && p.BN % 64 == 0));   // [H][W][N][C]: whole 32-channel groups per column half
   // ... and for 1x1 layers, whose main loop is a handful of stages: the tile's time is its store (measured 4-12 % faster, 28x28 and
   // 56x56 images, 256 and 512 channels)
-  p.tma_store = tma_store_ok && (env_int("MQ_TC_TMA_STORE", 0) || (taps == 1 && !env_int("MQ_TC_NO_TMA_STORE", 0))) ? 1 : 0;
+  p.tma_store = !mx && tma_store_ok && (env_int("MQ_TC_TMA_STORE", 0) || (taps == 1 && !env_int("MQ_TC_NO_TMA_STORE", 0))) ? 1 : 0;
   const size_t stage_bytes = 128 * 128 + (size_t)p.BN * 128 + 3072;
   int stages = (int)((227 * 1024 - 2048 - (p.tma_store ? 65536 : 0)) / stage_bytes);
   if (stages > 8) stages = 8;
@@ -203,21 +231,8 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   // TMEM (512 columns): accumulators (BN columns each) + one 24-column scale buffer per pipeline stage
   p.n_acc = (2 * p.BN + 24 * stages <= 512) ? 2 : 1;
   if (p.n_acc * p.BN + 24 * stages > 512) return false;
-  // pairs of blocks (cta_group::2) on two neighbouring tiles that share the weight tile: 128-byte K chunks, 256-channel
-  // tiles, no stride classes, and an even number of tiles per channel tile so that a pair never straddles two of them
-  // Opt-in (MQ_TC_CTA2=1): measured within +-5 % of single blocks (512 channels 28x28 8-bit -2.5 %, E2M1 56x56 -5 %,
-  // 256 channels +2 %) - with one 256-column accumulator these kernels wait on their NCHW stores, not on loads or issue.
-  p.cta2 = (p.BN == 256 && p.KB == 128 && p.classes == 1 && ((long long)p.tiles_w * p.tiles_h) % 2 == 0 && p.total_tiles >= 2 &&
-            env_int("MQ_TC_CTA2", 0)) ? 1 : 0;
-  if (p.cta2) {
-    const size_t sb2 = 128 * 128 + 128 * 128 + 3072;
-    int st2 = (int)((227 * 1024 - 2048 - (p.tma_store ? 65536 : 0)) / sb2);
-    if (st2 > 8) st2 = 8;
-    if (st2 < 2 || 256 + 24 * st2 > 512) p.cta2 = 0;
-    else { p.stages = st2; p.n_acc = 1; }
-  }
   p.mma_cp = env_int("MQ_TC_NO_MMA_CP", 0) ? 0 : 1;   // E2M1 too: the bubble behind a copier warp costs more than the lane's extra issues
-  p.pair = op == MQ_OP_BWD_DATA && g.sw == 2 && layout == MQ_NCHW && p.Wd % 2 == 0 && p.n_acc == 2 && p.total_tiles % 2 == 0 &&
+  p.pair = !mx && op == MQ_OP_BWD_DATA && g.sw == 2 && layout == MQ_NCHW && p.Wd % 2 == 0 && p.n_acc == 2 && p.total_tiles % 2 == 0 &&
            !env_int("MQ_TC_NO_PAIR", 0);
   const int nkh = op == MQ_OP_FWD ? g.Kh : (g.Kh + g.sh - 1) / g.sh, nkw = op == MQ_OP_FWD ? g.Kw : (g.Kw + g.sw - 1) / g.sw;
   p.max_stages = (nkh * nkw * p.cpt + p.G - 1) / p.G;
@@ -227,7 +242,7 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   // whole-tile-per-stage variant: stride 1, one chunk per tap (<= 64 bytes of channels).  One box with the column
   // halo needs 8-column tiles; one box per column shift takes 8, 16 or 32 columns (longer NCHW store runs).
   p.halo = 0;
-  if (!line && g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && taps <= 64 && !env_int("MQ_TC_NO_HALO", 0)) {
+  if (!line && !mx && g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && taps <= 64 && !env_int("MQ_TC_NO_HALO", 0)) {
     const int spa = fp4 ? 2 : 1, atoms_b = (p.BN + 127) / 128;
     if (p.TW == 8) {
       p.WH = p.TW + g.Kw - 1;
@@ -251,7 +266,7 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   }
   // unit strides and one 128-byte chunk per stage: the activation-side scale chunk of (tile, kh) equals that of the tile one
   // output row further with kh - 1, so chunks are stored per source row - Kh times fewer to expand
-  p.sfa_dedup = (!p.halo && !p.cta2 && p.KB == 128 && g.sh == 1 && g.sw == 1 && !env_int("MQ_TC_NO_SFA_DEDUP", 0)) ? 1 : 0;
+  p.sfa_dedup = (!p.halo && p.KB == 128 && g.sh == 1 && g.sw == 1 && !env_int("MQ_TC_NO_SFA_DEDUP", 0)) ? 1 : 0;
   p.sfa_hk = p.tiles_h + g.Kh - 1;
   out->p = p;
   size_t o = 0;
@@ -269,8 +284,10 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   return true;
 }
 
+// Scratch of a forward / input-gradient call: the tensor-core plan's where one exists (it depends on the output layout: the
+// larger of the two), never less than what the CUDA-core kernels need, which take the layers a plan refuses.
 size_t conv_tc_workspace(int op, const Geom& g, int fmt_x_like, int fmt_w, bool line) {
-  size_t need = 0;
+  size_t need = conv_generic_workspace(op, g);
   for (int layout = 0; layout < 2; ++layout) {   // the tile shape, hence the scratch, depends on the output layout
     ConvTcPlan pl;
     if (conv_tc_plan(op, g, fmt_x_like, fmt_w, layout, &pl, line) && pl.total > need) need = pl.total;
@@ -278,49 +295,37 @@ size_t conv_tc_workspace(int op, const Geom& g, int fmt_x_like, int fmt_w, bool 
   return need;
 }
 
-mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq_qtensor* qw, float* out, int layout, void* ws,
+// Every tensor map of the call is encoded before its first launch, so a failing encode leaves nothing enqueued.
+mq_status run_conv_tc(int op, const Geom& g, ConvTcPlan& pl, const mq_qtensor* qx_like, const mq_qtensor* qw, float* out, int layout, void* ws,
                       unsigned int* status, cudaStream_t stream) {
-  ConvTcPlan pl;
-  if (!conv_tc_plan(op, g, qx_like->fmt, qw->fmt, layout, &pl, qx_like->block == MQ_BLOCK_LINE32)) return MQ_ERR_UNSUPPORTED;
   ConvTcParams& p = pl.p;
   const int taps = g.Kh * g.Kw;
   uint8_t* base = static_cast<uint8_t*>(ws);
-  const uint8_t* b_codes;
+  // where the kernels will find their operands: as stored, or in scratch (W re-laid for the input gradient; 6-bit operands
+  // repacked - 16 codes -> 12 packed bytes + 4 bytes of padding per 16-byte chunk, the container of the MMA's 6-bit types)
+  const uint8_t* w_stored = static_cast<const uint8_t*>(qw->codes);
+  const uint8_t* x_stored = static_cast<const uint8_t*>(qx_like->codes);
+  const uint8_t* b_unpacked = op == MQ_OP_FWD ? w_stored : base;
+  const uint8_t* b_codes = fmt_is_6bit(qw->fmt) ? base + pl.off_pack_b : b_unpacked;
+  const uint8_t* a_codes = fmt_is_6bit(qx_like->fmt) ? base + pl.off_pack_a : x_stored;
+  uint8_t* wt_scales = base + pl.off_wt_scales;
+  bool separate_transpose = false;
   if (op == MQ_OP_FWD) {
-    b_codes = static_cast<const uint8_t*>(qw->codes);
     p.b_scales = qw->scales;
   } else {
-    uint8_t* wt_scales = base + pl.off_wt_scales;
     // per-tap kernel, operands that need no repacking: the re-layout rides in the scale-expansion launch
     p.wt_fused = (!p.halo && !fmt_is_6bit(qw->fmt) && !env_int("MQ_TC_NO_WT_FUSED", 0)) ? 1 : 0;
     if (p.wt_fused) {
-      p.wt_in = static_cast<const uint8_t*>(qw->codes); p.wt_out = base; p.wt_sc_in = qw->scales;
+      p.wt_in = w_stored; p.wt_out = base; p.wt_sc_in = qw->scales;
       p.wt_Cout = g.Cout; p.wt_Cop = g.Cop; p.wt_Cp = g.Cp; p.wt_bx = g.Cp / 32; p.wt_by = g.Cop / 32;
-    } else if (launch_weight_transpose(static_cast<const uint8_t*>(qw->codes), qw->scales, base, wt_scales, g, qw->fmt, stream) != cudaSuccess) {
-      return MQ_ERR_CUDA;
-    }
-    b_codes = base;
+    } else separate_transpose = true;
     p.b_scales = wt_scales;
-  }
-  // 6-bit operands: 16 codes -> 12 packed bytes + 4 bytes of padding per 16-byte chunk (the container of the MMA's
-  // 6-bit types), written to scratch; every later step moves whole 16-byte chunks and is unchanged
-  const uint8_t* a_codes = static_cast<const uint8_t*>(qx_like->codes);
-  if (fmt_is_6bit(qx_like->fmt)) {
-    const size_t nbytes = (size_t)p.Hs * p.Ws * g.N * pl.rowbytes;
-    if (launch_pack6(a_codes, base + pl.off_pack_a, nbytes, stream) != cudaSuccess) return MQ_ERR_CUDA;
-    a_codes = base + pl.off_pack_a;
-  }
-  if (fmt_is_6bit(qw->fmt)) {
-    const size_t nbytes = (size_t)pl.rows_b * taps * pl.rowbytes;
-    if (launch_pack6(b_codes, base + pl.off_pack_b, nbytes, stream) != cudaSuccess) return MQ_ERR_CUDA;
-    b_codes = base + pl.off_pack_b;
   }
   p.a_scales = qx_like->scales;
   p.sfa_img = base + pl.off_sfa;
   p.sfb_img = base + pl.off_sfb;
   p.b_codes = b_codes; p.b_rows_total = pl.rows_b; p.b_rowbytes = pl.rowbytes; p.b_img = base + pl.off_bimg;
   p.out = out; p.out_layout = layout; p.status = status;
-  if (!(p.halo && p.fused) && launch_expand_conv_scales(p, stream) != cudaSuccess) return MQ_ERR_CUDA;
 
   CUtensorMap map_a, map_w;
   {
@@ -347,19 +352,8 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
     const uint64_t rb = (uint64_t)pl.rowbytes;
     const uint64_t dims[3] = {rb, (uint64_t)taps, (uint64_t)pl.rows_b};
     const uint64_t strides[2] = {rb, (uint64_t)taps * rb};
-    const uint32_t box[3] = {(uint32_t)p.KB, 1u, (uint32_t)(p.cta2 ? 128 : p.BN)};   // a pair's blocks load half of the weight rows each
+    const uint32_t box[3] = {(uint32_t)p.KB, 1u, (uint32_t)p.BN};
     if (!encode_tensor_map_u8(&map_w, b_codes, 3, dims, strides, box, nullptr, p.KB)) return MQ_ERR_CUDA;
-  }
-  CUtensorMap map_sfa = map_a, map_sfb = map_a;
-  if (p.cta2) {   // a pair's scale chunks travel as tiled copies (rows of 256 bytes), so that they can count on the leader's barrier
-    const int spa = p.kind_fp4 ? 2 : 1;
-    const uint64_t tiles_m = (uint64_t)p.tiles_n * p.tiles_h * p.tiles_w * p.classes;
-    const uint64_t rows_a = tiles_m * p.max_stages * 2 * spa;
-    const uint64_t rows_b = (uint64_t)p.classes * p.tiles_c * p.max_stages * 2 * spa * 2;
-    const uint64_t da[2] = {256, rows_a}, db[2] = {256, rows_b}, st[1] = {256};
-    const uint32_t ba[2] = {256u, (uint32_t)(2 * spa)}, bb[2] = {256u, (uint32_t)(2 * spa * 2)};
-    if (!encode_tensor_map_u8(&map_sfa, p.sfa_img, 2, da, st, ba, nullptr, 0)) return MQ_ERR_CUDA;
-    if (!encode_tensor_map_u8(&map_sfb, p.sfb_img, 2, db, st, bb, nullptr, 0)) return MQ_ERR_CUDA;
   }
   CUtensorMap map_out = map_a;
   if (p.tma_store) {
@@ -382,7 +376,12 @@ mq_status run_conv_tc(int op, const Geom& g, const mq_qtensor* qx_like, const mq
       }
     }
   }
-  return launch_conv_tc(p, map_a, map_w, map_out, map_sfa, map_sfb, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
+  // ---- launches
+  if (separate_transpose && launch_weight_transpose(w_stored, qw->scales, base, wt_scales, g, qw->fmt, stream) != cudaSuccess) return MQ_ERR_CUDA;
+  if (fmt_is_6bit(qx_like->fmt) && launch_pack6(x_stored, base + pl.off_pack_a, (size_t)p.Hs * p.Ws * g.N * pl.rowbytes, stream) != cudaSuccess) return MQ_ERR_CUDA;
+  if (fmt_is_6bit(qw->fmt) && launch_pack6(b_unpacked, base + pl.off_pack_b, (size_t)pl.rows_b * taps * pl.rowbytes, stream) != cudaSuccess) return MQ_ERR_CUDA;
+  if (!(p.halo && p.fused) && launch_expand_conv_scales(p, stream) != cudaSuccess) return MQ_ERR_CUDA;
+  return launch_conv_tc(p, map_a, map_w, map_out, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }
 
 // ---- weight gradient on tensor cores ---------------------------------------------------------------
@@ -457,7 +456,7 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   p.j_tiles = (g.Kh * g.Kw / p.TG) * p.cb_tiles;
   const int items = p.m_tiles * p.j_tiles;
   int splits = env_int("MQ_WGRAD_SPLITS", 0);
-  const int units = p.cta2 ? 74 : 148;   // blocks, or pairs of blocks, that run at once
+  const int units = p.cta2 ? sm_count() / 2 : sm_count();   // blocks, or pairs of blocks, that run at once
   if (splits <= 0) splits = items >= units ? 1 : units / items;
   if (splits > p.stages_total) splits = p.stages_total;
   if (splits < 1) splits = 1;
@@ -622,10 +621,15 @@ mq_status run_conv(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int r
   size_t need = 0;
   mq_workspace_size(desc, op, qa->fmt, qb->fmt, qa->block, &need);
   if (need > 0 && (!ws || ws_bytes < need)) return MQ_ERR_BUFFER_TOO_SMALL;
-  if (op == MQ_OP_FWD && conv_tc_eligible(op, g, qa->fmt, qb->fmt))
-    return run_conv_tc(op, g, qa, qb, static_cast<float*>(out), layout, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
-  if (op == MQ_OP_BWD_DATA && conv_tc_eligible(op, g, qb->fmt, qa->fmt))
-    return run_conv_tc(op, g, qb, qa, static_cast<float*>(out), layout, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
+  // tensor cores when the layer is eligible AND a plan exists for it; everything else runs on the CUDA-core kernels
+  {
+    const mq_qtensor* qx_like = op == MQ_OP_FWD ? qa : qb;
+    const mq_qtensor* qw = op == MQ_OP_FWD ? qb : qa;
+    ConvTcPlan pl;
+    if ((op == MQ_OP_FWD || op == MQ_OP_BWD_DATA) && conv_tc_eligible(op, g, qx_like->fmt, qw->fmt) &&
+        conv_tc_plan(op, g, qx_like->fmt, qw->fmt, layout, &pl, qx_like->block == MQ_BLOCK_LINE32))
+      return run_conv_tc(op, g, pl, qx_like, qw, static_cast<float*>(out), layout, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
+  }
   if (op == MQ_OP_BWD_WEIGHT) {
     WgradPlan w = wgrad_plan(g, qa->fmt, qb->fmt);
     if (w.ok) return run_wgrad_tc(g, w, qa, qb, static_cast<float*>(out), layout, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
@@ -642,11 +646,7 @@ mq_status run_conv(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int r
 
 }  // namespace
 
-bool pdl_enabled() {
-  static int v = -1;
-  if (v < 0) v = env_int("MQ_NO_PDL", 0) ? 0 : 1;
-  return v != 0;
-}
+bool pdl_enabled() { return env_int("MQ_NO_PDL", 0) == 0; }
 
 }  // namespace mq
 
@@ -723,6 +723,7 @@ static mq_status quantize_impl(const mq_conv_desc* desc, const void* src, int sr
     else { a.src_stride_p = v.R * v.C; a.src_stride_r = v.C; }
   }
   a.status = device_status_ptr();
+  a.act = 0;
   a.wait_limit = wait_limit; a.debug_skip_loads = skip_loads;
   a.sr = sr;
   a.sr_seed_lo = (unsigned)seed; a.sr_seed_hi = (unsigned)(seed >> 32);
@@ -781,6 +782,89 @@ mq_status mq_conv_bwd_data(const mq_conv_desc* desc, const mq_qtensor* wq, const
 mq_status mq_conv_bwd_weight(const mq_conv_desc* desc, const mq_qtensor* xq, const mq_qtensor* dyq, void* dw, int dw_dtype, int dw_layout,
                              void* workspace, size_t ws_bytes, void* stream) {
   return run_conv(MQ_OP_BWD_WEIGHT, desc, xq, MQ_ROLE_X, dyq, MQ_ROLE_DY, dw, dw_dtype, dw_layout, workspace, ws_bytes, stream);
+}
+
+// ---- producer epilogue that quantizes: forward / input-gradient GEMM emitting the next tensor's MX form ----------------
+namespace {
+// sizes of the emitted tensor: [Hd][Wd][N][Cd rounded up to 32] codes, one scale per (pixel, 32 samples, 32 channels)
+void mx_out_sizes(const Geom& g, int op, int fmt, size_t* cb, size_t* sb) {
+  const long long P = op == MQ_OP_FWD ? (long long)g.Ho * g.Wo : (long long)g.H * g.W;
+  const long long Cp = op == MQ_OP_FWD ? g.Cop : g.Cp;
+  *cb = (size_t)(P * g.N * Cp) * fmt_bits(fmt) / 8;
+  *sb = (size_t)(P * g.Nt * (Cp / 32));
+}
+mq_status run_conv_mx(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int role_a, const mq_qtensor* qb, int role_b, int act, mq_qtensor* out,
+                      int role_out, void* ws, size_t ws_bytes, void* stream, size_t* size_query) {
+  mq_status st = check_desc(desc);
+  if (st != MQ_OK) return st;
+  const Geom g = make_geom(*desc);
+  int fmt_x_like, fmt_w;
+  if (size_query) {   // formats only: qa / qb carry them in their fmt fields
+    fmt_x_like = op == MQ_OP_FWD ? qa->fmt : qb->fmt; fmt_w = op == MQ_OP_FWD ? qb->fmt : qa->fmt;
+  } else {
+    if ((st = check_qtensor(g, qa, role_a)) != MQ_OK) return st;
+    if ((st = check_qtensor(g, qb, role_b)) != MQ_OK) return st;
+    if (!out || !out->codes || !out->scales || !valid_fmt(out->fmt) || !valid_block(out->block) || out->role != role_out) return MQ_ERR_INVALID_ARG;
+    if (act != MQ_ACT_NONE && act != MQ_ACT_RELU && act != MQ_ACT_SILU) return MQ_ERR_INVALID_ARG;
+    if (!aligned16(out->codes) || !aligned16(out->scales) || (ws && !aligned16(ws))) return MQ_ERR_ALIGNMENT;
+    size_t cb, sb;
+    mx_out_sizes(g, op, out->fmt, &cb, &sb);
+    if (out->codes_bytes < cb || out->scales_bytes < sb) return MQ_ERR_BUFFER_TOO_SMALL;
+    if (qa->block != MQ_BLOCK_TILE32 || qb->block != MQ_BLOCK_TILE32 || out->block != MQ_BLOCK_TILE32) return MQ_ERR_UNSUPPORTED;
+    fmt_x_like = op == MQ_OP_FWD ? qa->fmt : qb->fmt; fmt_w = op == MQ_OP_FWD ? qb->fmt : qa->fmt;
+  }
+  ConvTcPlan pl;
+  if (!conv_tc_eligible(op, g, fmt_x_like, fmt_w) || !conv_tc_plan(op, g, fmt_x_like, fmt_w, MQ_HWNC, &pl, false, true)) {
+    // layers the tensor-core kernels do not take: the same result in two launches - the CUDA-core GEMM writes fp32
+    // [pixel][sample][channel] into scratch and the channel-fastest quantizer, which applies the activation, reads it back
+    const long long P = op == MQ_OP_FWD ? (long long)g.Ho * g.Wo : (long long)g.H * g.W;
+    const int Cd = op == MQ_OP_FWD ? g.Cout : g.Cin, Cdp = op == MQ_OP_FWD ? g.Cop : g.Cp;
+    const size_t y_bytes = up256((size_t)P * g.N * Cd * sizeof(float));
+    const size_t total = y_bytes + up256(conv_generic_workspace(op, g));
+    if (size_query) { *size_query = total; return MQ_OK; }
+    if (!ws || ws_bytes < total) return MQ_ERR_BUFFER_TOO_SMALL;
+    uint8_t* base = static_cast<uint8_t*>(ws);
+    ConvArgs a;
+    a.g = g;
+    a.a_codes = static_cast<const uint8_t*>(qa->codes); a.a_scales = qa->scales; a.fmt_a = qa->fmt;
+    a.b_codes = static_cast<const uint8_t*>(qb->codes); a.b_scales = qb->scales; a.fmt_b = qb->fmt;
+    a.out = reinterpret_cast<float*>(base); a.out_layout = MQ_HWNC; a.workspace = base + y_bytes; a.ws_bytes = ws_bytes - y_bytes; a.line = 0;
+    if (launch_conv_generic(op, a, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MQ_ERR_CUDA;
+    QuantArgs q{};
+    q.src = reinterpret_cast<const float*>(base); q.codes = static_cast<uint8_t*>(out->codes); q.scales = out->scales;
+    q.P = (int)P; q.R = g.N; q.C = Cd; q.Cp = Cdp;
+    q.out_stride_p = (long long)g.N * Cdp; q.out_stride_r = Cdp;
+    q.sc_stride_p = (long long)g.Nt * (Cdp / 32); q.sc_stride_r = Cdp / 32;
+    q.src_stride_p = (long long)g.N * Cd; q.src_stride_r = Cd;
+    q.fmt = out->fmt; q.act = act; q.status = device_status_ptr();
+    return launch_quantize(q, static_cast<cudaStream_t>(stream)) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
+  }
+  if (size_query) { *size_query = pl.total; return MQ_OK; }
+  if (pl.total > 0 && (!ws || ws_bytes < pl.total)) return MQ_ERR_BUFFER_TOO_SMALL;
+  pl.p.mx_fmt = out->fmt; pl.p.mx_act = act;
+  pl.p.mx_codes = static_cast<uint8_t*>(out->codes); pl.p.mx_scales = out->scales;
+  pl.p.mx_Cp = op == MQ_OP_FWD ? g.Cop : g.Cp;
+  const mq_qtensor* qx_like = op == MQ_OP_FWD ? qa : qb;
+  const mq_qtensor* qw = op == MQ_OP_FWD ? qb : qa;
+  return run_conv_tc(op, g, pl, qx_like, qw, nullptr, MQ_HWNC, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
+}
+}  // namespace
+
+mq_status mq_conv_mx_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt_b, size_t* bytes) {
+  if (!bytes || !valid_fmt(fmt_a) || !valid_fmt(fmt_b) || (op != MQ_OP_FWD && op != MQ_OP_BWD_DATA)) return MQ_ERR_INVALID_ARG;
+  mq_qtensor a{}, b{};
+  a.fmt = fmt_a; b.fmt = fmt_b;
+  return run_conv_mx(op, desc, &a, 0, &b, 0, 0, nullptr, 0, nullptr, 0, nullptr, bytes);
+}
+
+mq_status mq_conv_fwd_mx(const mq_conv_desc* desc, const mq_qtensor* xq, const mq_qtensor* wq, int act, mq_qtensor* yq, void* workspace, size_t ws_bytes,
+                         void* stream) {
+  return run_conv_mx(MQ_OP_FWD, desc, xq, MQ_ROLE_X, wq, MQ_ROLE_W, act, yq, MQ_ROLE_X, workspace, ws_bytes, stream, nullptr);
+}
+
+mq_status mq_conv_bwd_data_mx(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, mq_qtensor* dxq, void* workspace, size_t ws_bytes,
+                              void* stream) {
+  return run_conv_mx(MQ_OP_BWD_DATA, desc, wq, MQ_ROLE_W, dyq, MQ_ROLE_DY, MQ_ACT_NONE, dxq, MQ_ROLE_DY, workspace, ws_bytes, stream, nullptr);
 }
 
 // ---- allocation-free variant of mq_conv_bwd_data ---------------------------------------------------
@@ -915,6 +999,8 @@ mq_status mq_conv_layer_host(const mq_conv_desc* desc, int fmt_x, int fmt_w, int
 }
 
 unsigned long long mq_kernel_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
+
+void mq_reload_env(void) { env_forget(); }
 
 const char* mq_status_string(int status) {
   switch (status) {

@@ -274,7 +274,7 @@ __global__ void __launch_bounds__(256) bwd_weight_reduce(const float* __restrict
 int conv_generic_bwd_weight_splits(const Geom& g) {
   const int taps = g.Kh * g.Kw;
   const long long tiles = (long long)((g.Cop + TM - 1) / TM) * ((taps * g.Cp + TN - 1) / TN);
-  long long splits = (148LL * 4 + tiles - 1) / tiles;
+  long long splits = ((long long)sm_count() * 4 + tiles - 1) / tiles;
   const long long npix = (long long)g.Ho * g.Wo;
   if (splits > npix) splits = npix;
   if (splits > 256) splits = 256;
@@ -290,7 +290,7 @@ size_t conv_generic_workspace(int op, const Geom& g) {
 cudaError_t launch_bwd_weight_reduce(const float* partial, float* out, const Geom& g, int splits, int layout, cudaStream_t s) {
   const long long quads = (long long)g.Cout * g.Kh * g.Kw * (g.Cp / 4);
   unsigned blocks = (unsigned)((quads + 63) / 64);
-  if (blocks > 148u * 16) blocks = 148u * 16;
+  if (blocks > (unsigned)sm_count() * 16) blocks = (unsigned)sm_count() * 16;
   count_launches(1);
   return launch_pdl(bwd_weight_reduce, dim3(blocks), dim3(256), 0, s, partial, out, g, splits, layout);
 }
@@ -324,7 +324,7 @@ cudaError_t launch_conv_generic(int op, const ConvArgs& a, cudaStream_t s) {
     if (e != cudaSuccess) return e;
     const long long quads = (long long)g.Cout * g.Kh * g.Kw * (g.Cp / 4);
     unsigned blocks = (unsigned)((quads + 63) / 64);
-    if (blocks > 148u * 16) blocks = 148u * 16;
+    if (blocks > (unsigned)sm_count() * 16) blocks = (unsigned)sm_count() * 16;
     bwd_weight_reduce<<<blocks, 256, 0, s>>>(reinterpret_cast<const float*>(a.workspace), a.out, g, splits, a.out_layout);
     count_launches(1);
   }

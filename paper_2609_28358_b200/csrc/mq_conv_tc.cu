@@ -7,14 +7,15 @@
 // A small kernel first expands the compact tile scales (one E8M0 byte per 32x32 tile) into the per-row
 // scale-vector chunks the MMA reads, one chunk per (tile, pipeline stage), in scratch.
 //
-// One persistent thread block per SM, 12 warps:
-//   warp 0   TMA producer        one lane issues the A (gathered activation) and B (weight) boxes and the
-//                                bulk copies of the stage's two scale chunks
-//   warp 1   MMA issuer          one lane issues the stage's MMAs
-//   warp 2   scale copier        one lane copies the stage's scale chunks smem -> TMEM (tcgen05.cp), one stage
-//                                ahead of the MMA issuer and from its own thread so the copies overlap the MMAs
-//   warps 4-11 epilogue          TMEM -> registers -> global (fp32), overlapped with the next tile's main loop;
-//                                two warps per TMEM lane quadrant, each taking half of the tile's columns
+// One persistent thread block per SM, 16 warps, every role loop run by its whole warp with only the asynchronous
+// instruction itself under an elected lane:
+//   warps 0, 12   loaders of the activation boxes (even / odd stages)
+//   warps 3, 13   loaders of the weight boxes (even / odd stages)
+//   warps 14, 15  loaders of the stage's two scale-vector chunks (even / odd stages)
+//   warp 1        MMA issuer: the stage's scale copies smem -> TMEM (tcgen05.cp), then its MMAs
+//   warp 2        scale copier (E2M1 with the separate-copier option only)
+//   warps 4-11    epilogue: TMEM -> registers -> global (fp32) or a staged TMA store, overlapped with the next tile's
+//                 main loop when a second accumulator fits; two warps per TMEM lane quadrant, half of the columns each
 // A pipeline stage holds 128 bytes of K per row (four MMAs): one 128-byte box, or 128/KB boxes of KB
 // bytes when a tap has fewer than 128 bytes of channels (then several taps share a stage).
 // Every wait is bounded; on expiry the kernel records MQ_ERR_TIMEOUT in the status word and drains.
@@ -32,24 +33,6 @@ constexpr int SFA_BYTES = 1024;   // up to 2 groups of 4 scale bytes per row
 constexpr int SFB_BYTES = 2048;   // up to 2 groups x 2 atoms of 128 rows
 constexpr int SF_COLS = 24;       // TMEM columns of one scale buffer: 8 (A) + 16 (B)
 
-// Cycle counters of block 0's roles (debug aid): [role][0] = cycles in the role's loop, [role][1] = cycles waiting.
-#ifdef MQ_TC_PROFILE
-__device__ unsigned long long g_prof[8][2];
-__device__ unsigned long long g_blk[160][4];   // per block: SM id, start, body start, end (ns)
-__device__ unsigned long long g_role[160][4][2];   // per block and role: cycles in the loop, cycles waiting
-#define PROF_CLK() clock64()
-#define PROF_ADD(slot, idx, v) do { if (blockIdx.x == 0) g_prof[slot][idx] += (unsigned long long)(v); } while (0)
-#define PROF_BEGIN() const long long prof_t0 = clock64(); long long prof_wait = 0
-#define PROF_WAIT(expr) ([&]() { const long long w0_ = clock64(); const bool r_ = (expr); prof_wait += clock64() - w0_; return r_; }())
-#define PROF_END(role) do { if (blockIdx.x == 0) { g_prof[role][0] = clock64() - prof_t0; g_prof[role][1] = prof_wait; } \
-    if (blockIdx.x < 160) { g_role[blockIdx.x][role][0] = clock64() - prof_t0; g_role[blockIdx.x][role][1] = prof_wait; } } while (0)
-#else
-#define PROF_CLK() 0ll
-#define PROF_ADD(slot, idx, v) do { } while (0)
-#define PROF_BEGIN() do { } while (0)
-#define PROF_WAIT(expr) (expr)
-#define PROF_END(role) do { } while (0)
-#endif
 
 struct Tile { int c0, w0, n0, h, cls, ct; };
 
@@ -161,7 +144,6 @@ __device__ __forceinline__ void epilogue_role(const ConvTcParams& p, uint32_t tm
     const int cend = half == 0 ? ((p.BN / 2 + 15) & ~15) : p.BN;
     const long long cs = (long long)p.Hd * p.Wd;
     uint32_t tcount = 0;
-    PROF_BEGIN();
     for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
       const Tile tile = decode_tile(p, t);
       TapWalk<MODE> tw;
@@ -169,7 +151,7 @@ __device__ __forceinline__ void epilogue_role(const ConvTcParams& p, uint32_t tm
       const int Q = tw.chunks(p);
       const int acc = (int)(tcount & (uint32_t)(p.n_acc - 1));
       bool ok = true;
-      if (lane == 0) ok = PROF_WAIT(mbar_wait(&tfull[acc], (tcount >> (p.n_acc - 1)) & 1, p.status, MQ_ERR_TIMEOUT));
+      if (lane == 0) ok = mbar_wait(&tfull[acc], (tcount >> (p.n_acc - 1)) & 1, p.status, MQ_ERR_TIMEOUT);
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) { *abort_flag = 1; break; }
       tc_fence_after_sync();
@@ -220,7 +202,6 @@ __device__ __forceinline__ void epilogue_role(const ConvTcParams& p, uint32_t tm
       __syncwarp();
       if (lane == 0) release_acc(&tempty[acc], leader_remote);
     }
-    if (lane == 0 && warp == 4) PROF_END(3);
 }
 
 // Epilogue role of the pair mode (see tile_of_iter): both accumulators hold the same output rows and channels for the
@@ -283,6 +264,130 @@ __device__ __forceinline__ void epilogue_pair_role(const ConvTcParams& p, uint32
     }
 }
 
+// Quantizing epilogue (warps 4-11): the producer applies the activation and emits the NEXT tensor's stored MX form -
+// codes [Hd][Wd][N][Cp] and one E8M0 byte per 32-sample x 32-channel tile at a pixel - instead of fp32, i.e. the
+// tensor is quantized on chip before it is stored and the fp32 round trip through HBM disappears.  Tiles are TW <= 4
+// output columns x 128 / TW >= 32 samples, so a quantization tile (one pixel, 32 samples, 32 channels) lies inside one
+// GEMM tile: its 32 samples sit in TW consecutive TMEM lane quadrants (8, 16 or 32 lanes each), its channels in 32
+// accumulator columns.  Per 32-channel block a warp loads its 32 x 32 values, applies the activation, takes the
+// per-lane maximum, reduces it over the lanes of the same output column (shuffles), and the TW warps of a tile
+// combine their maxima through shared memory (one named barrier per block among the four warps of a column half);
+// scale and codes then follow exactly the quantizer's arithmetic.  A lane writes its row's 32 codes as one or two
+// 16-byte stores (a row of the emitted tensor is channel-contiguous).
+__device__ __forceinline__ void half_sync(int half) { asm volatile("bar.sync %0, 128;" ::"r"(2 + half) : "memory"); }
+__device__ __forceinline__ bool half_any(int half, bool pred) {
+  int r;
+  asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %2, 0;\n\tbar.red.or.pred q, %1, 128, p;\n\tselp.b32 %0, 1, 0, q;\n\t}\n" : "=r"(r) : "r"(2 + half), "r"(pred ? 1 : 0) : "memory");
+  return r != 0;
+}
+template <int FMT>
+__device__ __forceinline__ void mx_encode_row(const float* x, float f, uint8_t* dst) {
+  unsigned w[8];
+#pragma unroll
+  for (int k = 0; k < 32; k += 4) {
+    const unsigned lo = encode2<FMT>(x[k] * f, x[k + 1] * f), hi = encode2<FMT>(x[k + 2] * f, x[k + 3] * f);
+    w[k >> 2] = FMT == MQ_E2M1 ? (lo | (hi << 8)) : (lo | (hi << 16));
+  }
+  if (FMT == MQ_E2M1) {
+    *reinterpret_cast<uint4*>(dst) = make_uint4(w[0] | (w[1] << 16), w[2] | (w[3] << 16), w[4] | (w[5] << 16), w[6] | (w[7] << 16));
+  } else {
+    *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+    *reinterpret_cast<uint4*>(dst + 16) = make_uint4(w[4], w[5], w[6], w[7]);
+  }
+}
+template <int MODE>
+__device__ __forceinline__ void epilogue_mx_role(const ConvTcParams& p, unsigned* red, uint32_t tmem, uint64_t* tfull, uint64_t* tempty,
+                                                 volatile int* abort_flag, int warp, int lane, unsigned total) {
+    const int quad = warp & 3;
+    const int half = (warp - 4) >> 2;
+    const int r = 32 * quad + lane;
+    const int tw_ = r & (p.TW - 1), tn = r >> p.lgTW;
+    const int nblk = p.BN >> 5;                         // 32-channel blocks of a tile
+    const int bbeg = half == 0 ? 0 : (nblk + 1) >> 1, bend = half == 0 ? (nblk + 1) >> 1 : nblk;
+    const int grp0 = quad & ~(p.TW - 1);                // first quadrant of the TW quadrants that hold this sample tile
+    const int emax = fmt_emax(p.mx_fmt);
+    const int bpe4 = p.mx_fmt == MQ_E2M1 ? 1 : 2;       // bytes per element x 2
+    const int Ct = p.mx_Cp >> 5;
+    unsigned* my_red = red + half * 32;                 // [parity][quadrant][column]
+    uint32_t tcount = 0;
+    for (unsigned t = blockIdx.x; t < total; t += gridDim.x, ++tcount) {
+      const Tile tile = decode_tile(p, t);
+      TapWalk<MODE> tw;
+      tw.init(p, tile);
+      const int Q = tw.chunks(p);
+      const int acc = (int)(tcount & (uint32_t)(p.n_acc - 1));
+      bool ok = true;
+      if (lane == 0) ok = !*abort_flag && mbar_wait(&tfull[acc], (tcount >> (p.n_acc - 1)) & 1, p.status, MQ_ERR_TIMEOUT);
+      // the four warps of a half leave together or not at all: they meet at barriers inside the tile
+      if (half_any(half, !ok)) { *abort_flag = 1; break; }
+      tc_fence_after_sync();
+      int yo, xo;
+      if (MODE == MQ_OP_FWD) { yo = tile.h; xo = tile.w0 + tw_; }
+      else {
+        const int ch = (int)fdiv((unsigned)tile.cls, p.sw, p.m_sw);
+        yo = ch + p.sh * tile.h; xo = tile.cls - ch * p.sw + p.sw * (tile.w0 + tw_);
+      }
+      const int n = tile.n0 + tn;
+      const bool row_ok = yo < p.Hd && xo < p.Wd && n < p.N;
+      const uint32_t taddr = tmem + acc * p.BN + ((uint32_t)(32 * quad) << 16);
+      const long long pix = (long long)yo * p.Wd + xo;
+      uint8_t* o_codes = p.mx_codes + (((pix * p.N + n) * p.mx_Cp + tile.c0) * bpe4 >> 1);
+      uint8_t* o_scale = p.mx_scales + (pix * p.Nt + (n >> 5)) * Ct + (tile.c0 >> 5);
+#pragma unroll 1
+      for (int b = bbeg; b < bend; ++b) {
+        float x[32];
+        if (Q > 0) {
+          uint32_t v[32];
+          tmem_ld_32x32b_x16(taddr + 32 * b, v);
+          tmem_ld_32x32b_x16(taddr + 32 * b + 16, v + 16);
+          tmem_ld_wait();
+#pragma unroll
+          for (int k = 0; k < 32; ++k) x[k] = __uint_as_float(v[k]);
+        } else {
+#pragma unroll
+          for (int k = 0; k < 32; ++k) x[k] = 0.f;
+        }
+        if (b + 1 == bend) {      // the accumulator has been read: hand it back before the arithmetic and the stores
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&tempty[acc]);
+        }
+        float m = 0.f;
+#pragma unroll
+        for (int k = 0; k < 32; ++k) {
+          const float y = mx_activation(x[k], p.mx_act);
+          x[k] = y;
+          m = fmaxf(m, fabsf(y));
+        }
+        unsigned mb = row_ok ? __float_as_uint(m) : 0u;
+        for (int off = p.TW; off < 32; off <<= 1) mb = max(mb, __shfl_xor_sync(0xffffffffu, mb, off));
+        unsigned* rb = my_red + (b & 1) * 16;
+        if (lane < p.TW) rb[quad * 4 + lane] = mb;
+        half_sync(half);
+        unsigned mx = 0;
+        for (int g = 0; g < p.TW; ++g) mx = max(mx, rb[(grp0 + g) * 4 + tw_]);
+        const int code = scale_code_of(mx, emax);
+        if (quad == grp0 && lane < p.TW && row_ok && tile.c0 + 32 * b < p.mx_Cp) o_scale[b] = (uint8_t)code;
+        if (row_ok && tile.c0 + 32 * b < p.mx_Cp) {
+          const float f = scale_factor(code);
+          uint8_t* dst = o_codes + ((32 * b * bpe4) >> 1);
+          switch (p.mx_fmt) {
+            case MQ_E4M3: mx_encode_row<MQ_E4M3>(x, f, dst); break;
+            case MQ_E5M2: mx_encode_row<MQ_E5M2>(x, f, dst); break;
+            case MQ_E2M1: mx_encode_row<MQ_E2M1>(x, f, dst); break;
+            case MQ_E3M2: mx_encode_row<MQ_E3M2>(x, f, dst); break;
+            default: mx_encode_row<MQ_E2M3>(x, f, dst); break;
+          }
+        }
+      }
+      if (bbeg >= bend) {      // a tile of 32 channels leaves the second half without a block
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tempty[acc]);
+      }
+    }
+}
+
 // Epilogue role with TMA stores, NCHW output (warps 4-11).  Each warp moves its 32 rows x up to 64 channels on
 // its own: TMEM -> registers -> a private [channel][row] staging slice (row index fastest, so the writes are
 // conflict-free), then one lane stores the slice as a box of the output seen as (W, N, C, H): TW columns x
@@ -303,7 +408,6 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
     const bool hwnc = p.out_layout == MQ_HWNC;
     const int hrow = lane;   // the [H][W][N][C] store's box walks (sample, column) in the rows' own order
     uint32_t tcount = 0;
-    PROF_BEGIN();
     for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
       const Tile tile = decode_tile(p, t);
       TapWalk<MODE> tw;
@@ -311,7 +415,7 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
       const int Q = tw.chunks(p);
       const int acc = (int)(tcount & (uint32_t)(p.n_acc - 1));
       bool ok = true;
-      if (lane == 0) ok = PROF_WAIT(mbar_wait(&tfull[acc], (tcount >> (p.n_acc - 1)) & 1, p.status, MQ_ERR_TIMEOUT));
+      if (lane == 0) ok = mbar_wait(&tfull[acc], (tcount >> (p.n_acc - 1)) & 1, p.status, MQ_ERR_TIMEOUT);
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) { *abort_flag = 1; break; }
       tc_fence_after_sync();
@@ -369,7 +473,6 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
       }
     }
     if (lane == 0) bulk_wait_group_all();
-    if (lane == 0 && warp == 4) PROF_END(3);
 }
 
 template <int MODE, int KB, bool FP4>
@@ -394,6 +497,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   uint64_t* tempty = tfull + 2;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
   volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+  unsigned* mx_red = reinterpret_cast<unsigned*>((reinterpret_cast<uintptr_t>(tmem_slot + 2) + 15) & ~static_cast<uintptr_t>(15));   // quantizing epilogue only
 
   // The warp index goes through a shuffle so that the compiler knows it to be warp-uniform: the role loops below are
   // run by whole warps, their arithmetic stays in the uniform datapath, and only the copy / MMA / commit instructions
@@ -430,7 +534,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // (the walk is a few additions) but waits and issues only for its own; each kind arrives once per stage on the
     // stage's barrier with its own byte count.
     {
-      PROF_BEGIN();
       uint32_t s = 0, phase = 0, gi = 0;
       const uint32_t row_bytes = lkind == 1 ? (uint32_t)p.BN * KB : 128u * KB;
       for (unsigned i = 0, t; (t = tile_of_iter(p, i)) < total && !*abort_flag; ++i) {
@@ -465,7 +568,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (mine) {
             uint8_t* sa = smem + (size_t)s * stage_bytes;
             uint8_t* sb = sa + A_STAGE_BYTES;
-            if (!PROF_WAIT(mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+            if (!mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
             if (elect_one()) {
               if (lkind == 2) {
                 mbar_arrive_expect_tx(&full[s], 512u * SPA * (1 + atoms_b));
@@ -489,7 +592,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
         }
       }
-      if (warp == 0) PROF_END(0);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
@@ -508,14 +610,13 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       for (int i = 0; i < 4; ++i) idesc_id[i] = idesc_with_sf_ids(p.idesc, i, i);
       const bool self_cp = !FP4 || p.mma_cp;
       uint32_t s = 0, phase = 0, tcount = 0;
-      PROF_BEGIN();
       for (unsigned t; (t = tile_of_iter(p, tcount)) < total && !*abort_flag; ++tcount) {
         const Tile tile = decode_tile(p, t);
         TapWalk<MODE> tw;
         tw.init(p, tile);
         const int Q = tw.chunks(p);
         const int acc = (int)(tcount & (uint32_t)(p.n_acc - 1));
-        if (!PROF_WAIT(mbar_wait(&tempty[acc], ((tcount >> (p.n_acc - 1)) & 1) ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+        if (!mbar_wait(&tempty[acc], ((tcount >> (p.n_acc - 1)) & 1) ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem + acc * p.BN;
         uint32_t accumulate = 0;
@@ -524,7 +625,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           // E2M1: the scale copier signals sffull[s] once the stage's scale vectors are in TMEM.  8-bit operands: this
           // warp waits for the stage itself and its lane issues the (three) scale copies right before the MMAs that
           // read them - same thread, so the tensor pipe keeps the order, and no copy queues behind MMAs issued earlier.
-          if (!PROF_WAIT(mbar_wait(self_cp ? &full[s] : &sffull[s], phase, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+          if (!mbar_wait(self_cp ? &full[s] : &sffull[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
           tc_fence_after_sync();
           const uint32_t so = s * stage16;
           const uint32_t sfa_t = sf_base + s * SF_COLS, sfb_t = sfa_t + 8;
@@ -560,7 +661,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         if (elect_one()) { if (Q > 0) tc_commit(&tfull[acc]); else mbar_arrive(&tfull[acc]); }
         __syncwarp();
       }
-      PROF_END(1);
     }
   } else if (warp == 2) {
     // ------------------------------------------------------------------ scale copier
@@ -600,7 +700,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else if (warp >= 4 && warp < 12) {
-    if (p.pair) epilogue_pair_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
+    if (p.mx_out) epilogue_mx_role<MODE>(p, mx_red, tmem, tfull, tempty, abort_flag, warp, lane, total);
+    else if (p.pair) epilogue_pair_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else if (p.tma_store) epilogue_tma_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
   }
@@ -608,163 +709,6 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem, 512);
-}
-
-// ---- the per-tap kernel on PAIRS of blocks (clusters of two, tcgen05 cta_group::2) -------------------------------
-// Tiles 2k and 2k + 1 (neighbours in the tile order: same channel tile, same taps) form one 256-row x 256-channel MMA
-// tile: each block loads the activation boxes of ITS 128 rows and HALF of the weight rows (128 of the 256 channels)
-// plus its scale chunks, all with .cta_group::2 tiled loads that count their bytes on the LEADER's barrier.  The
-// leader's MMA lane issues the scale copies, the MMAs (M = 256) and multicast commits that free the stage and
-// publish the accumulator in both blocks; every block drains its own 128 rows.  Half the weight bytes per block
-// and stage buy six pipeline stages instead of four, and one issuing lane feeds two tensor cores.
-// KB = 128 only (>= 128 bytes of channels per tap), 256-channel tiles, one accumulator, no stride classes.
-template <int MODE, bool FP4>
-__global__ void __launch_bounds__(TC_THREADS, 1)
-conv_tc_pair_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_out,
-                    const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb, const ConvTcParams p) {
-  constexpr int KB = 128;
-  constexpr int SPA = FP4 ? 2 : 1;     // scale bytes per atom
-  constexpr int LAYOUT = 2;
-  constexpr int B_HALF_BYTES = 128 * 128;
-  extern __shared__ uint8_t smem_raw[];
-  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-  constexpr int stage_bytes = A_STAGE_BYTES + B_HALF_BYTES + SFA_BYTES + SFB_BYTES;
-  float* staging = reinterpret_cast<float*>(smem + (size_t)p.stages * stage_bytes);   // TMA-store epilogue only
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * stage_bytes + (p.tma_store ? EPI_STAGING_BYTES : 0));
-  uint64_t* empty = full + p.stages;
-  uint64_t* tfull = empty + p.stages;      // [2], one used
-  uint64_t* tempty = tfull + 2;            // [2], one used (the leader's: 16 epilogue warps arrive)
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(tempty + 2);
-  volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
-
-  const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;   // warp-uniform, see conv_tc_kernel
-  const uint32_t rank = __shfl_sync(0xffffffffu, cluster_ctarank(), 0);                            // 0: leader
-  const unsigned total = (unsigned)p.total_tiles;
-
-  if (threadIdx.x == 0) {
-    for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 3); mbar_init(&empty[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 16); }
-    *abort_flag = 0;
-    mbar_fence_init();
-    prefetch_tensormap(&map_a);
-    prefetch_tensormap(&map_b);
-    prefetch_tensormap(&map_sfa);
-    prefetch_tensormap(&map_sfb);
-    if (p.tma_store) prefetch_tensormap(&map_out);
-  }
-  if (warp == 1) { tmem_alloc_2(tmem_slot, 512); tmem_relinquish_2(); }
-  tc_fence_before_sync();
-  __syncthreads();
-  cluster_sync_all();   // both blocks' barriers and tensor memory exist before anything crosses over
-  tc_fence_after_sync();
-  const uint32_t tmem = *tmem_slot;
-  pdl_wait();
-
-  // loader warps: (kind, parity of the stages it serves), as in conv_tc_kernel
-  const int lkind = (warp == 0 || warp == 12) ? 0 : ((warp == 3 || warp == 13) ? 1 : (warp >= 14 ? 2 : -1));
-  const int lhalf = (warp == 12 || warp == 13 || warp == 15) ? 1 : 0;
-  if (lkind >= 0) {
-    uint32_t s = 0, phase = 0, gi = 0;
-    // the leader announces both blocks' bytes; the peer only issues
-    const uint32_t kind_bytes = 2u * (lkind == 2 ? 512u * SPA * 3u : 128u * KB);
-    for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x) {
-      const Tile tile = decode_tile(p, t);
-      TapWalk<MODE> tw;
-      tw.init(p, tile);
-      const int Q = tw.chunks(p);
-      ChunkPos pos;
-      pos.reset();
-      const int sfa_row0 = (int)(tile_m_index(p, tile) * (unsigned)p.max_stages) * (2 * SPA);                   // rows of 256 bytes
-      const int sfb_row0 = (int)((unsigned)(tile.cls * p.tiles_c + tile.ct) * (unsigned)p.max_stages) * (2 * SPA * 2);
-      for (int q = 0; q < Q; ++q, ++gi) {
-        const bool mine = (gi & 1u) == (uint32_t)lhalf;
-        const int c0 = pos.cc * KB;
-        const int c1 = lkind == 1 ? tap_index(tw, pos) : src_w0(tw, pos);
-        const int c2 = src_h(tw, pos);
-        pos.advance(tw, p.cpt);
-        if (mine) {
-          uint8_t* sa = smem + (size_t)s * stage_bytes;
-          uint8_t* sb = sa + A_STAGE_BYTES;
-          const uint32_t lbar = cluster_addr_of(&full[s], 0);
-          if (!mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
-          if (elect_one()) {
-            if (rank == 0) mbar_arrive_expect_tx(&full[s], kind_bytes);
-            if (lkind == 2) {
-              tma_load_2d_pair(sb + B_HALF_BYTES, &map_sfa, lbar, 0, sfa_row0 + q * (2 * SPA));
-              tma_load_2d_pair(sb + B_HALF_BYTES + SFA_BYTES, &map_sfb, lbar, 0, sfb_row0 + q * (2 * SPA * 2));
-            } else if (lkind == 1) {
-              tma_load_3d_pair(sb, &map_b, lbar, c0, c1, tile.c0 + 128 * (int)rank);
-            } else {
-              tma_load_4d_pair(sa, &map_a, lbar, c0, c1, tile.n0, c2);
-            }
-          }
-          __syncwarp();
-        }
-        if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
-      }
-    }
-  } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer (the leader's)
-    if (rank == 0) {
-      const uint64_t op_desc = smem_desc_base(16, 8 * KB, LAYOUT);
-      const uint32_t sf_base = tmem + (uint32_t)p.BN;
-      constexpr uint32_t stage16 = (uint32_t)stage_bytes >> 4;
-      const uint64_t a_desc0 = smem_desc(op_desc, smem_u32(smem));
-      const uint64_t b_desc0 = smem_desc(op_desc, smem_u32(smem + A_STAGE_BYTES));
-      const uint64_t sf_desc = smem_desc_base(0, 128, 0);
-      const uint64_t sfa_desc0 = smem_desc(sf_desc, smem_u32(smem + A_STAGE_BYTES + B_HALF_BYTES));
-      const uint64_t sfb_desc0 = smem_desc(sf_desc, smem_u32(smem + A_STAGE_BYTES + B_HALF_BYTES + SFA_BYTES));
-      const uint32_t idesc = (p.idesc & ~(0x1Fu << 24)) | ((256u >> 4) << 24);   // M = 256 over the pair
-      uint32_t s = 0, phase = 0, tcount = 0;
-      for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
-        const Tile tile = decode_tile(p, t);
-        TapWalk<MODE> tw;
-        tw.init(p, tile);
-        const int Q = tw.chunks(p);
-        if (!mbar_wait(&tempty[0], (tcount & 1) ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
-        tc_fence_after_sync();
-        uint32_t accumulate = 0;
-        for (int q = 0; q < Q; ++q) {
-          if (!mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
-          tc_fence_after_sync();
-          const uint32_t so = s * stage16;
-          const uint32_t sfa_t = sf_base + s * SF_COLS, sfb_t = sfa_t + 8;
-          if (elect_one()) {
-#pragma unroll
-            for (int g = 0; g < SPA; ++g) {
-              tmem_cp_32x128b_warpx4_2(sfa_t + 4 * g, sfa_desc0 + so + g * 32);
-              tmem_cp_32x128b_warpx4_2(sfb_t + 8 * g, sfb_desc0 + so + g * 64);
-              tmem_cp_32x128b_warpx4_2(sfb_t + 8 * g + 4, sfb_desc0 + so + g * 64 + 32);
-            }
-            uint32_t accu = accumulate;
-#pragma unroll
-            for (int a = 0; a < 4; ++a) {
-              const uint64_t ad = a_desc0 + so + a * 2;
-              const uint64_t bd = b_desc0 + so + a * 2;
-              const int g = (a * SPA) >> 2, id = (a * SPA) & 3;
-              const uint32_t idd = idesc_with_sf_ids(idesc, id, id);
-              if (FP4) mma_mxf4_2(tmem, ad, bd, idd, sfa_t + 4 * g, sfb_t + 8 * g, accu);
-              else mma_mxf8f6f4_2(tmem, ad, bd, idd, sfa_t + 4 * g, sfb_t + 8 * g, accu);
-              accu = 1;
-            }
-            tc_commit_2_multicast(&empty[s], 3);   // frees the stage in both blocks
-          }
-          __syncwarp();
-          accumulate = 1;
-          if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
-        }
-        if (elect_one()) { if (Q > 0) tc_commit_2_multicast(&tfull[0], 3); else { mbar_arrive(&tfull[0]); mbar_arrive_remote(&tfull[0], 1); } }
-        __syncwarp();
-      }
-    }
-  } else if (warp >= 4 && warp < 12) {
-    if (p.tma_store) epilogue_tma_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total, (int)rank);
-    else epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total, (int)rank);
-  }
-  tc_fence_before_sync();
-  __syncthreads();
-  cluster_sync_all();   // nothing of the peer block is touched after this point
-  if (warp == 1) tmem_dealloc_2(tmem, 512);
 }
 
 template <int BPC>
@@ -833,10 +777,6 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
                     const ConvTcParams p) {
   constexpr int G = 128 / KB, APC = KB / 32, SPA = FP4 ? 2 : 1;
   constexpr int LAYOUT = KB == 128 ? 2 : (KB == 64 ? 4 : 6);
-#ifdef MQ_TC_PROFILE
-  unsigned long long gt0 = 0;
-  if (threadIdx.x == 0) asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt0));
-#endif
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int taps = TAPS > 0 ? TAPS : p.Kh * p.Kw;
@@ -895,10 +835,6 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
-#ifdef MQ_TC_PROFILE
-  unsigned long long gt1 = 0;
-  if (threadIdx.x == 0) asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt1));
-#endif
   // TMEM columns: accumulators, the resident weight scale vectors (16 per chunk), then 8 per chunk per stage
   const uint32_t sfb_base = tmem + p.n_acc * p.BN;
   const uint32_t sfa_base = sfb_base + (uint32_t)nsf * 16;
@@ -909,13 +845,12 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
     {
       uint32_t s = 0, phase = 0, bcount = 0;
       int cur_ct = -1;
-      PROF_BEGIN();
       for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x) {
         const Tile tile = decode_tile(p, t);
         const int ct = tile.ct;
         if (!p.fused && ct != cur_ct) {
           // new weight tile: wait until the MMAs of the previous one have retired, then one copy of image + scales
-          if (bcount > 0 && !PROF_WAIT(mbar_wait(bempty, (bcount - 1) & 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+          if (bcount > 0 && !mbar_wait(bempty, (bcount - 1) & 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
           if (elect_one()) {
             mbar_arrive_expect_tx(bfull, (uint32_t)(b_bytes + sfb_bytes));
             bulk_load(smem, p.b_img + (size_t)ct * b_bytes, b_bytes, bfull);
@@ -924,7 +859,7 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
           __syncwarp();
           cur_ct = ct; ++bcount;
         }
-        if (!PROF_WAIT(mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+        if (!mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
         uint8_t* sa = stage0 + (size_t)s * stage_bytes;
         // first source pixel of the halo: forward (h - ph, w0 - pw); input gradient (h + ph - (Kh-1), w0 + pw - (Kw-1))
         const int hs = MODE == MQ_OP_FWD ? tile.h - p.ph : tile.h + p.ph - (p.Kh - 1);
@@ -937,7 +872,6 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         __syncwarp();
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
-      PROF_END(0);
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer: all taps of a tile per stage
@@ -955,22 +889,20 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 #pragma unroll
       for (int q = 0; q < TU; ++q) { ta[q] = tap_a[q]; tb[q] = tap_b[q]; }
       const uint32_t acc_mask = (uint32_t)p.n_acc - 1, acc_shift = (uint32_t)p.n_acc - 1;   // n_acc is 1 or 2
-      PROF_BEGIN();
       for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
         const int ct = p.tiles_c == 1 ? 0 : (int)((t / tiles_per_c) % (unsigned)p.tiles_c);
         const bool new_b = ct != cur_ct;
         if (new_b) {
-          if (!PROF_WAIT(mbar_wait(bfull, bcount & 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+          if (!mbar_wait(bfull, bcount & 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
           cur_ct = ct; ++bcount;
         }
         const int acc = (int)(tcount & acc_mask);
-        if (!PROF_WAIT(mbar_wait(&tempty[acc], ((tcount >> acc_shift) & 1) ^ 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
-        if (!PROF_WAIT(mbar_wait(p.mma_cp ? &full[s] : &sffull[s], phase, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+        if (!mbar_wait(&tempty[acc], ((tcount >> acc_shift) & 1) ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+        if (!mbar_wait(p.mma_cp ? &full[s] : &sffull[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem + acc * p.BN;
         const uint32_t sa16 = smem_u32(stage0 + (size_t)s * stage_bytes) >> 4;
         const uint32_t sfa_s = sfa_base + s * sfa_cols_stage;
-        const long long pc0 = PROF_CLK();
         if (elect_one()) {
         if (p.mma_cp) {   // this lane issues the scale copies itself, right before the MMAs that read them
           const uint64_t sf_desc = smem_desc_base(0, 128, 0);
@@ -1021,11 +953,8 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         }
         }
         __syncwarp();
-        const long long pc1 = PROF_CLK();
-        PROF_ADD(4, 1, pc1 - pc0);
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
-      PROF_END(1);
     }
   } else if (warp == 2) {
     // ------------------------------------------------------------------ scale copier: chunks smem -> TMEM
@@ -1033,15 +962,14 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
       const uint64_t sf_desc = smem_desc_base(0, 128, 0);
       uint32_t s = 0, phase = 0, bcount = 0;
       int cur_ct = -1;
-      PROF_BEGIN();
       for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x) {
         const int ct = p.tiles_c == 1 ? 0 : (int)((t / tiles_per_c) % (unsigned)p.tiles_c);
         const bool new_b = ct != cur_ct;
         if (new_b) {
-          if (!p.fused && !PROF_WAIT(mbar_wait(bfull, bcount & 1, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+          if (!p.fused && !mbar_wait(bfull, bcount & 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
           cur_ct = ct; ++bcount;
         }
-        if (!PROF_WAIT(mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT))) { *abort_flag = 1; break; }
+        if (!mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
         tc_fence_after_sync();
         if (elect_one()) {
         if (new_b) {
@@ -1066,7 +994,6 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
         __syncwarp();
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
       }
-      PROF_END(2);
     }
   } else if (warp == 3) {
     // ------------------------------------------------------------------ activation-scale expander (fused mode)
@@ -1144,15 +1071,6 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
   tc_fence_before_sync();
   __syncthreads();
   if (warp == 1) tmem_dealloc(tmem, 512);
-#ifdef MQ_TC_PROFILE
-  if (threadIdx.x == 0) {
-    unsigned long long gt2; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(gt2));
-    if (blockIdx.x < 160) {
-      unsigned smid; asm volatile("mov.u32 %0, %smid;" : "=r"(smid));
-      g_blk[blockIdx.x][0] = smid; g_blk[blockIdx.x][1] = gt0; g_blk[blockIdx.x][2] = gt1; g_blk[blockIdx.x][3] = gt2;
-    }
-  }
-#endif
 }
 
 // ---- scale expansion --------------------------------------------------------------------------------
@@ -1402,26 +1320,8 @@ EncodeTiledFn get_encoder() {
 
 }  // namespace
 
-#ifdef MQ_TC_PROFILE
-extern "C" int mqdbg_read_role(unsigned long long* out1280) {
-  return cudaMemcpyFromSymbol(out1280, g_role, sizeof(unsigned long long) * 1280) == cudaSuccess ? 0 : 1;
-}
-extern "C" int mqdbg_read_blk(unsigned long long* out640) {
-  return cudaMemcpyFromSymbol(out640, g_blk, sizeof(unsigned long long) * 640) == cudaSuccess ? 0 : 1;
-}
-extern "C" int mqdbg_read_prof(unsigned long long* out16) {
-  if (cudaMemcpyFromSymbol(out16, g_prof, sizeof(unsigned long long) * 16) != cudaSuccess) return 1;
-  unsigned long long z[16] = {0};
-  z[12] = ~0ull;
-  return cudaMemcpyToSymbol(g_prof, z, sizeof(z)) == cudaSuccess ? 0 : 1;
-}
-#endif
 
-static CUtensorMapL2promotion l2promo() {
-  const char* e = getenv("MQ_TMA_L2PROMO");
-  const int v = e ? atoi(e) : 3;
-  return v == 0 ? CU_TENSOR_MAP_L2_PROMOTION_NONE : v == 1 ? CU_TENSOR_MAP_L2_PROMOTION_L2_64B : v == 2 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : CU_TENSOR_MAP_L2_PROMOTION_L2_256B;
-}
+static CUtensorMapL2promotion l2promo() { return CU_TENSOR_MAP_L2_PROMOTION_L2_256B; }
 bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes, const uint32_t* box,
                           const uint32_t* elem_strides, int swizzle_bytes, bool f32, int l2_promotion_bytes) {
   EncodeTiledFn fn = get_encoder();
@@ -1441,7 +1341,7 @@ bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const ui
 
 size_t conv_tc_smem_bytes(const ConvTcParams& p) {
   const size_t stage = A_STAGE_BYTES + (size_t)p.BN * 128 + SFA_BYTES + SFB_BYTES;
-  return 1024 + (size_t)p.stages * stage + (p.tma_store ? EPI_STAGING_BYTES : 0) + (3 * (size_t)p.stages + 4) * 8 + 64;
+  return 1024 + (size_t)p.stages * stage + (p.tma_store ? EPI_STAGING_BYTES : 0) + (3 * (size_t)p.stages + 4) * 8 + 64 + (p.mx_out ? 288 : 0);
 }
 
 template <int MODE, int KB, bool FP4>
@@ -1453,9 +1353,7 @@ cudaError_t launch_conv_tc_inst(const ConvTcParams& p, const CUtensorMap& map_a,
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  int dev = 0, sms = 148;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = sm_count();
   const long long units = p.pair ? p.total_tiles / 2 : p.total_tiles;
   const unsigned grid = (unsigned)(units < sms ? units : sms);
   count_launches(1);
@@ -1505,9 +1403,7 @@ cudaError_t launch_conv_tc_halo_taps(const ConvTcParams& p, const CUtensorMap& m
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
-  int dev = 0, sms = 148;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = sm_count();
   const unsigned grid = (unsigned)(p.total_tiles < sms ? p.total_tiles : sms);
   count_launches(1);
   return launch_pdl(conv_tc_halo_kernel<MODE, KB, FP4, TAPS>, dim3(grid), dim3(TC_THREADS), smem, s, map_a, map_b, map_w, p);
@@ -1538,7 +1434,7 @@ cudaError_t launch_pack6(const uint8_t* in, uint8_t* out, size_t nbytes, cudaStr
   const size_t nchunks = nbytes / 16;
   if (nchunks == 0) return cudaSuccess;
   size_t blocks = (nchunks + 255) / 256;
-  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks > sm_count() * 16) blocks = sm_count() * 16;
   count_launches(1);
   return launch_pdl(pack6_kernel, dim3((unsigned)blocks), dim3(256), 0, s, reinterpret_cast<const uint4*>(in), reinterpret_cast<uint4*>(out), nchunks);
 }
@@ -1567,7 +1463,7 @@ cudaError_t launch_recode6_e4m3(const uint8_t* in, uint8_t* out, size_t nbytes, 
   const size_t nchunks = nbytes / 16;
   if (nchunks == 0) return cudaSuccess;
   size_t blocks = (nchunks + 255) / 256;
-  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks > sm_count() * 16) blocks = sm_count() * 16;
   count_launches(1);
   if (fmt6 == MQ_E3M2) return launch_pdl(recode6_kernel<true>, dim3((unsigned)blocks), dim3(256), 0, s, reinterpret_cast<const uint4*>(in), reinterpret_cast<uint4*>(out), nchunks);
   return launch_pdl(recode6_kernel<false>, dim3((unsigned)blocks), dim3(256), 0, s, reinterpret_cast<const uint4*>(in), reinterpret_cast<uint4*>(out), nchunks);
@@ -1598,45 +1494,13 @@ cudaError_t launch_recode4_e4m3(const uint8_t* in, uint8_t* out, size_t n_out, c
   const size_t nchunks = n_out / 16;
   if (nchunks == 0) return cudaSuccess;
   size_t blocks = (nchunks + 255) / 256;
-  if (blocks > 148 * 16) blocks = 148 * 16;
+  if (blocks > sm_count() * 16) blocks = sm_count() * 16;
   count_launches(1);
   return launch_pdl(recode4_kernel, dim3((unsigned)blocks), dim3(256), 0, s, reinterpret_cast<const uint2*>(in), reinterpret_cast<uint4*>(out), nchunks);
 }
 
-size_t conv_tc_pair_smem_bytes(const ConvTcParams& p) {
-  const size_t stage = A_STAGE_BYTES + 128 * 128 + SFA_BYTES + SFB_BYTES;
-  return 1024 + (size_t)p.stages * stage + (p.tma_store ? EPI_STAGING_BYTES : 0) + (2 * (size_t)p.stages + 4) * 8 + 64;
-}
-template <int MODE, bool FP4>
-cudaError_t launch_conv_tc_pair_inst(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_out, const CUtensorMap& map_sfa,
-                                     const CUtensorMap& map_sfb, cudaStream_t s) {
-  static bool attr_set = false;
-  const size_t smem = conv_tc_pair_smem_bytes(p);
-  if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(conv_tc_pair_kernel<MODE, FP4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
-    if (e != cudaSuccess) return e;
-    attr_set = true;
-  }
-  int dev = 0, sms = 148;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-  unsigned grid = (unsigned)(p.total_tiles < sms ? p.total_tiles : sms);
-  grid &= ~1u;   // whole pairs (the tile count is even in this mode)
-  if (grid < 2) return cudaErrorInvalidValue;
-  count_launches(1);
-  return launch_pdl_cluster(conv_tc_pair_kernel<MODE, FP4>, dim3(grid), dim3(TC_THREADS), smem, s, 2u, map_a, map_b, map_out, map_sfa, map_sfb, p);
-}
-
-cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_out, const CUtensorMap& map_sfa,
-                           const CUtensorMap& map_sfb, cudaStream_t s) {
+cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_out, cudaStream_t s) {
   if (p.total_tiles <= 0 || p.total_tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
-  if (p.cta2) {
-    const bool f4 = p.kind_fp4 != 0;
-    if (p.mode == MQ_OP_FWD) return f4 ? launch_conv_tc_pair_inst<MQ_OP_FWD, true>(p, map_a, map_w, map_out, map_sfa, map_sfb, s)
-                                       : launch_conv_tc_pair_inst<MQ_OP_FWD, false>(p, map_a, map_w, map_out, map_sfa, map_sfb, s);
-    return f4 ? launch_conv_tc_pair_inst<MQ_OP_BWD_DATA, true>(p, map_a, map_w, map_out, map_sfa, map_sfb, s)
-              : launch_conv_tc_pair_inst<MQ_OP_BWD_DATA, false>(p, map_a, map_w, map_out, map_sfa, map_sfb, s);
-  }
   if (p.halo) {
 #define MQ_TC_HCASE(M, K, F) if (p.mode == M && p.KB == K && (p.kind_fp4 != 0) == F) return launch_conv_tc_halo_inst<M, K, F>(p, map_a, map_out, map_w, s)
     MQ_TC_HCASE(MQ_OP_FWD, 64, false); MQ_TC_HCASE(MQ_OP_FWD, 32, false); MQ_TC_HCASE(MQ_OP_FWD, 64, true); MQ_TC_HCASE(MQ_OP_FWD, 32, true);

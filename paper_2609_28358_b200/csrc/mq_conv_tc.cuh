@@ -56,7 +56,6 @@ struct ConvTcParams {
   int fused;                // 1: single channel tile, stride 1: no preparation kernel (the blocks build the weight image, its
                             //    scale chunks and every tile's activation scale chunks themselves)
   int mma_cp;             // E2M1: 1 = the MMA lane issues the scale copies itself (no copier warp)
-  int cta2;               // 1: pairs of blocks (clusters of 2) on 256-row x 256-channel tiles, conv_tc_pair_kernel
   int pair;                 // per-tap kernel, input gradient with column stride 2, NCHW output: see tile_of_iter
   int tma_store;            // 1: NCHW output written by TMA stores from per-warp staging slices
   const uint8_t* b_codes;   // weight-like codes [rows][taps][b_rowbytes] (source of the images below)
@@ -74,6 +73,12 @@ struct ConvTcParams {
   float* out;
   int out_layout;
   unsigned int* status;
+  // quantizing epilogue (the producer emits the next tensor's MX tiles instead of fp32, see epilogue_mx_role)
+  int mx_out;               // 1: on
+  int mx_fmt, mx_act;       // element format of the emitted tensor; activation applied first (mq_act)
+  uint8_t* mx_codes;        // [Hd][Wd][N][mx_Cp] codes
+  uint8_t* mx_scales;       // [Hd][Wd][Nt][mx_Cp / 32] tile scales
+  int mx_Cp;                // Cd rounded up to 32
 };
 
 // map_a: gathered activation codes.  map_w: weight codes, one tap per box (per-tap kernel) or all taps of a tile in one
@@ -85,8 +90,7 @@ cudaError_t launch_pack6(const uint8_t* in, uint8_t* out, size_t nbytes, cudaStr
 cudaError_t launch_recode6_e4m3(const uint8_t* in, uint8_t* out, size_t nbytes, int fmt6, cudaStream_t s);
 // packed E2M1 codes (two per byte) -> the E4M3 codes of the same values, one per byte; n_out = elements = output bytes
 cudaError_t launch_recode4_e4m3(const uint8_t* in, uint8_t* out, size_t n_out, cudaStream_t s);
-cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_out, const CUtensorMap& map_sfa,
-                           const CUtensorMap& map_sfb, cudaStream_t s);
+cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_out, cudaStream_t s);
 // Expands the compact tile scales into the per-stage scale-vector chunks the MMA reads (p.sfa_img, p.sfb_img).
 cudaError_t launch_expand_conv_scales(const ConvTcParams& p, cudaStream_t s);
 size_t conv_tc_sfa_bytes(const ConvTcParams& p);

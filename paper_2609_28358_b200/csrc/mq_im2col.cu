@@ -139,14 +139,14 @@ cudaError_t launch_im2col(const Im2colArgs& a, cudaStream_t s) {
   count_launches(1);
   if (J <= IC_MAX_J && src_chunks < 0x7fffffffLL && n_main < 0x7fff0000LL) {
     long long sc_blocks = (n_scales + IC_THREADS - 1) / IC_THREADS;
-    if (sc_blocks > 148 * 4) sc_blocks = 148 * 4;
+    if (sc_blocks > sm_count() * 4) sc_blocks = sm_count() * 4;
     if (sc_blocks < 1) sc_blocks = 1;
     return launch_pdl(im2col_kernel, dim3((unsigned)(n_main + sc_blocks)), dim3(IC_THREADS), 0, s, a, rc, (int)J, PX, (unsigned)n_main);
   }
   const long long code_chunks = (long long)g.Ho * g.Wo * g.N * J;
   const long long total = code_chunks + n_scales;
   long long blocks = (total + IC_THREADS - 1) / IC_THREADS;
-  const long long cap = 148LL * 8 * 16;  // grid-stride beyond this
+  const long long cap = (long long)sm_count() * 8 * 16;  // grid-stride beyond this
   if (blocks > cap) blocks = cap;
   if (blocks <= 0) return cudaErrorInvalidValue;
   im2col_generic_kernel<<<(unsigned)blocks, IC_THREADS, 0, s>>>(a, rc, code_chunks, n_scales);

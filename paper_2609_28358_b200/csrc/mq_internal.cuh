@@ -44,6 +44,18 @@ __host__ __device__ inline unsigned fmt_mma_code(int fmt) { return fmt == MQ_E4M
 // Number of kernels the library has launched in this process (diagnostic; see mq_kernel_launch_count).
 void count_launches(int n);
 
+// Streaming multiprocessors of the current device (148 on a B200); grids are sized in multiples of it.
+inline int sm_count() {
+  int dev = 0, sms = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms <= 0) return 148;
+  return sms;
+}
+
+// Integer value of an MQ_* environment knob.  Each knob is read from the environment ONCE, on its first use in the
+// process, and answered from a table afterwards, so that a size query and the call it sizes always see the same plan;
+// mq_reload_env() (a diagnostic entry point) empties the table.
+int env_int(const char* name, int dflt);
+
 // ---- launchers (defined in the .cu files) ---------------------------------------------------
 struct QuantArgs {
   const float* src;
@@ -61,6 +73,7 @@ struct QuantArgs {
   unsigned sr_seed_lo, sr_seed_hi;   // the 64-bit seed
   unsigned sr_key0;                  // stream key of elements whose index is below 2^32 (computed on the host)
   int sr_wide;                       // 1: the tensor has 2^32 elements or more (keys are derived per element)
+  int act;                           // mq_act applied to every element before quantization (channel-fastest source only; 0: none)
   int line;                          // 1: line blocks (one scale per row and 32 channels; the sc strides are per row), 0: 32 x 32 tiles
   unsigned int* status;              // device status word: set when a bounded wait gives up
   // test hooks of the TMA kernel's abort path: polls a barrier wait may take (0: the default limit), and 1 = the loader
@@ -142,6 +155,38 @@ __device__ __forceinline__ void decode8(const uint8_t* codes_base, long long ele
     }
   }
 }
+
+// ---- quantization arithmetic shared by the quantizer kernels and the quantizing GEMM epilogue (Eq. 5-6, E8M0 form) ----
+template <int FMT>
+__device__ __forceinline__ unsigned encode2(float lo, float hi) {
+  // two elements -> two codes (lo in the low byte / nibble), round-to-nearest-even, saturating
+  if (FMT == MQ_E2M1) {
+    return (unsigned)__nv_cvt_float2_to_fp4x2(make_float2(lo, hi), __NV_E2M1, cudaRoundNearest);
+  } else if (FMT == MQ_E3M2 || FMT == MQ_E2M3) {
+    // two 6-bit codes, each in the low six bits of its byte (the container the tensor core reads)
+    return (unsigned)__nv_cvt_float2_to_fp6x2(make_float2(lo, hi), FMT == MQ_E3M2 ? __NV_E3M2 : __NV_E2M3, cudaRoundNearest);
+  } else {
+    return (unsigned)__nv_cvt_float2_to_fp8x2(make_float2(lo, hi), __NV_SATFINITE, FMT == MQ_E4M3 ? __NV_E4M3 : __NV_E5M2);
+  }
+}
+
+// activation of the quantizing producer epilogue (mq_act), evaluated in fp32
+__device__ __forceinline__ float mx_activation(float y, int act) {
+  if (act == MQ_ACT_RELU) return fmaxf(y, 0.f);
+  if (act == MQ_ACT_SILU) return __fdividef(y, 1.f + __expf(-y));
+  return y;
+}
+
+__device__ __forceinline__ int scale_code_of(unsigned amax_bits, int emax) {
+  // floor(log2 amax) = biased exponent - 127 for normal amax; subnormal / zero amax clamps to 0
+  const int e = (int)(amax_bits >> 23) - emax;
+  return min(max(e, 0), 254);
+}
+
+// 2^(127 - code) as a normal fp32 number: code = clamp(E - emax, 0, 254) with E <= 254 and emax >= 2, so
+// 127 - code lies in [-125, 127].  x * 2^(127 - code) is then exact (|result| < 2^(emax + 1)) except where it
+// underflows below 2^-126, far under half of the smallest element step, where it rounds to zero either way.
+__device__ __forceinline__ float scale_factor(int code) { return __uint_as_float((unsigned)(254 - code) << 23); }
 
 #endif  // __CUDACC__
 

@@ -28,19 +28,6 @@ constexpr int QT_THREADS = 256;
 // a quarter-warp (rows 4 apart) hit 8 different 16-byte bank groups
 constexpr int QBUF_BYTES = 1024 * 32 + 256 * 16;
 
-template <int FMT>
-__device__ __forceinline__ unsigned encode2(float lo, float hi) {
-  // two elements -> two codes (lo in the low byte / nibble), round-to-nearest-even, saturating
-  if (FMT == MQ_E2M1) {
-    return (unsigned)__nv_cvt_float2_to_fp4x2(make_float2(lo, hi), __NV_E2M1, cudaRoundNearest);
-  } else if (FMT == MQ_E3M2 || FMT == MQ_E2M3) {
-    // two 6-bit codes, each in the low six bits of its byte (the container the tensor core reads)
-    return (unsigned)__nv_cvt_float2_to_fp6x2(make_float2(lo, hi), FMT == MQ_E3M2 ? __NV_E3M2 : __NV_E2M3, cudaRoundNearest);
-  } else {
-    return (unsigned)__nv_cvt_float2_to_fp8x2(make_float2(lo, hi), __NV_SATFINITE, FMT == MQ_E4M3 ? __NV_E4M3 : __NV_E5M2);
-  }
-}
-
 // Stochastic Round(.) of Eq. 6 (Sec. III-A: the gradient's rounding).  x is the scaled element, idx its index in the
 // logical NCHW / OIHW tensor.  The element's draw is 32 bits of a counter-based generator keyed by (seed, idx);
 // u = (top 23 bits + 1/2) / 2^23.  With lo <= |x| < hi neighbours on the format's grid, the result is hi when
@@ -80,17 +67,6 @@ __device__ __forceinline__ unsigned sr_key(const QuantArgs& a, long long idx) {
   if (!a.sr_wide) return a.sr_key0;
   return sr_mix32(a.sr_seed_lo ^ sr_mix32(a.sr_seed_hi ^ sr_mix32((unsigned)((unsigned long long)idx >> 32))));
 }
-
-__device__ __forceinline__ int scale_code_of(unsigned amax_bits, int emax) {
-  // floor(log2 amax) = biased exponent - 127 for normal amax; subnormal / zero amax clamps to 0
-  const int e = (int)(amax_bits >> 23) - emax;
-  return min(max(e, 0), 254);
-}
-
-// 2^(127 - code) as a normal fp32 number: code = clamp(E - emax, 0, 254) with E <= 254 and emax >= 2, so
-// 127 - code lies in [-125, 127].  x * 2^(127 - code) is then exact (|result| < 2^(emax + 1)) except where it
-// underflows below 2^-126, far under half of the smallest element step, where it rounds to zero either way.
-__device__ __forceinline__ float scale_factor(int code) { return __uint_as_float((unsigned)(254 - code) << 23); }
 
 __device__ __forceinline__ void cp_async16(void* dst, const void* src, bool valid) {
   const unsigned d = (unsigned)__cvta_generic_to_shared(dst);
@@ -439,25 +415,17 @@ __device__ __forceinline__ bool mbar_wait_limit(uint64_t* bar, uint32_t parity, 
 }
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(TQ_CONSUMERS) : "memory"); }
 
-__device__ __forceinline__ Item tq_item_of(unsigned it, int n_pstrips, int Ct, int strip_fastest) {
-  Item q;
-  if (strip_fastest) {   // neighbouring strips of the same source rows are read at about the same time
-    const unsigned u = it / (unsigned)n_pstrips;
-    const int ps = (int)(it - u * (unsigned)n_pstrips);
-    q.rt = (int)(u / (unsigned)Ct);
-    q.ct = (int)(u - (unsigned)q.rt * (unsigned)Ct);
-    q.p0 = ps * 32; q.r0 = q.rt * 32; q.c0 = q.ct * 32;
-    return q;
-  }
-  return item_of(it, n_pstrips, Ct, 32);
-}
+// channel tile fastest (as item_of): the tiles that share an output line are produced together.  (Position strip fastest,
+// so that neighbouring strips of the same source rows are read together, measured 0.69 against 0.77 of the copy rate on a
+// 1.6 GB tensor and 0.78 against 0.72 on a 0.4 GB one: not kept.)
+__device__ __forceinline__ Item tq_item_of(unsigned it, int n_pstrips, int Ct) { return item_of(it, n_pstrips, Ct, 32); }
 
 // LINE: line blocks.  A line (32 channels of one row at one position) is held by two threads of neighbouring warps; they
 // exchange their maxima through the (still unused) staging buffer and the one with the lower channels writes the scale.
 template <int FMT, bool SR, bool LINE>
 __global__ void __launch_bounds__(TQ_THREADS, 1)
 quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant__ CUtensorMap map_out, QuantArgs a, int n_pstrips, int Ct,
-                    unsigned n_items, int strip_fastest) {
+                    unsigned n_items) {
   extern __shared__ uint8_t tq_raw[];
   uint8_t* base = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(tq_raw) + 127) & ~(uintptr_t)127);
   float* ring = reinterpret_cast<float*>(base);
@@ -485,7 +453,7 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_con
       bool ok = true;
 #pragma unroll 1
       for (unsigned it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
-        const Item q = tq_item_of(it, n_pstrips, Ct, strip_fastest);
+        const Item q = tq_item_of(it, n_pstrips, Ct);
         const int nb = min(4, (a.R - q.r0 + 7) >> 3);
 #pragma unroll 1
         for (int b = 0; b < nb; ++b) {
@@ -521,7 +489,7 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_con
     bool dead = false;
 #pragma unroll 1
     for (unsigned it = blockIdx.x; it < n_items; it += gridDim.x) {
-      const Item q = tq_item_of(it, n_pstrips, Ct, strip_fastest);
+      const Item q = tq_item_of(it, n_pstrips, Ct);
       const int nb = min(4, (a.R - q.r0 + 7) >> 3);
       float v[4][16];
       float fm = 0.f;
@@ -641,6 +609,11 @@ __global__ void __launch_bounds__(256) quantize_cfast_kernel(QuantArgs a, unsign
         }
       }
     }
+    if (a.act) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i)
+        v[i] = make_float4(mx_activation(v[i].x, a.act), mx_activation(v[i].y, a.act), mx_activation(v[i].z, a.act), mx_activation(v[i].w, a.act));
+    }
     int code[LINE ? 8 : 1];
     if (LINE) {
 #pragma unroll
@@ -690,7 +663,7 @@ cudaError_t launch_q_cfast(const QuantArgs& a, int Ct, cudaStream_t s) {
   if (items <= 0 || items > 0xffffffffLL) return cudaErrorInvalidValue;
   const bool vec = a.C % 4 == 0 && a.src_stride_p % 4 == 0 && a.src_stride_r % 4 == 0 && (reinterpret_cast<uintptr_t>(a.src) & 15) == 0;
   long long blocks = (items + 7) / 8;
-  if (blocks > 148LL * 64) blocks = 148LL * 64;
+  if (blocks > (long long)sm_count() * 64) blocks = (long long)sm_count() * 64;
   if (a.line) {
     if (a.sr) {
       if (vec) return launch_pdl(quantize_cfast_kernel<FMT, true, true, true>, dim3((unsigned)blocks), dim3(256), 0, s, a, (unsigned)Rt, (unsigned)Ct, (unsigned)items);
@@ -726,7 +699,6 @@ cudaError_t launch_q_tma(const QuantArgs& a, cudaStream_t s) {
     if (!encode_tensor_map_u8(&map_out, a.codes, 3, dims, strides, box, nullptr, 0)) return cudaErrorInvalidValue;
   }
   static bool attr_set = false;
-  static int strip_fastest = 0;
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(quantize_tma_kernel<FMT, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TQ_SMEM);
     if (e != cudaSuccess) return e;
@@ -736,23 +708,19 @@ cudaError_t launch_q_tma(const QuantArgs& a, cudaStream_t s) {
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(quantize_tma_kernel<FMT, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TQ_SMEM);
     if (e != cudaSuccess) return e;
-    const char* v = std::getenv("MQ_QUANT_STRIP_FASTEST");
-    if (v) strip_fastest = std::atoi(v);
     attr_set = true;
   }
   const int n_pstrips = (a.P + 31) / 32, Rt = (a.R + 31) / 32, Ct = a.Cp / 32;
   const long long n_items = (long long)n_pstrips * Rt * Ct;
   if (n_items <= 0 || n_items > 0x7fffffffLL) return cudaErrorInvalidValue;
-  int dev = 0, sms = 148;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = sm_count();
   const unsigned grid = (unsigned)(n_items < sms ? n_items : sms);
   if (a.line) {
-    if (a.sr) return launch_pdl(quantize_tma_kernel<FMT, true, true>, dim3(grid), dim3(TQ_THREADS), TQ_SMEM, s, map_in, map_out, a, n_pstrips, Ct, (unsigned)n_items, strip_fastest);
-    return launch_pdl(quantize_tma_kernel<FMT, false, true>, dim3(grid), dim3(TQ_THREADS), TQ_SMEM, s, map_in, map_out, a, n_pstrips, Ct, (unsigned)n_items, strip_fastest);
+    if (a.sr) return launch_pdl(quantize_tma_kernel<FMT, true, true>, dim3(grid), dim3(TQ_THREADS), TQ_SMEM, s, map_in, map_out, a, n_pstrips, Ct, (unsigned)n_items);
+    return launch_pdl(quantize_tma_kernel<FMT, false, true>, dim3(grid), dim3(TQ_THREADS), TQ_SMEM, s, map_in, map_out, a, n_pstrips, Ct, (unsigned)n_items);
   }
-  if (a.sr) return launch_pdl(quantize_tma_kernel<FMT, true, false>, dim3(grid), dim3(TQ_THREADS), TQ_SMEM, s, map_in, map_out, a, n_pstrips, Ct, (unsigned)n_items, strip_fastest);
-  return launch_pdl(quantize_tma_kernel<FMT, false, false>, dim3(grid), dim3(TQ_THREADS), TQ_SMEM, s, map_in, map_out, a, n_pstrips, Ct, (unsigned)n_items, strip_fastest);
+  if (a.sr) return launch_pdl(quantize_tma_kernel<FMT, true, false>, dim3(grid), dim3(TQ_THREADS), TQ_SMEM, s, map_in, map_out, a, n_pstrips, Ct, (unsigned)n_items);
+  return launch_pdl(quantize_tma_kernel<FMT, false, false>, dim3(grid), dim3(TQ_THREADS), TQ_SMEM, s, map_in, map_out, a, n_pstrips, Ct, (unsigned)n_items);
 }
 
 constexpr size_t QPIPE_SMEM = 2 * QBUF_BYTES + PS * 32 * 32 + 16 * 2 * 4 * sizeof(unsigned);
@@ -768,12 +736,9 @@ cudaError_t launch_q(const QuantArgs& a, int n_pstrips, int Ct, long long n_item
     return launch_pdl(quantize_simple_kernel<FMT, false>, dim3((unsigned)n_items), dim3(QT_THREADS), 0, s, a, n_pstrips, Ct);
   }
   static bool attr_set = false;
-  static int ctas_per_sm = 2;   // 80 KB of shared memory per block
-  static int nt = 256;   // 512-thread blocks measured slower: the kernel is bound by instruction issue
+  const int ctas_per_sm = 2;   // 80 KB of shared memory per block; 256 threads (512-thread blocks measured slower: bound by instruction issue)
   if (!attr_set) {
     cudaError_t e = cudaFuncSetAttribute(quantize_pipe_kernel<FMT, 256, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QPIPE_SMEM);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(quantize_pipe_kernel<FMT, 512, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QPIPE_SMEM);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(quantize_pipe_kernel<FMT, 256, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QPIPE_SMEM);
     if (e != cudaSuccess) return e;
@@ -781,21 +746,14 @@ cudaError_t launch_q(const QuantArgs& a, int n_pstrips, int Ct, long long n_item
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(quantize_pipe_kernel<FMT, 256, true, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)QPIPE_SMEM);
     if (e != cudaSuccess) return e;
-    const char* tv = std::getenv("MQ_QUANT_THREADS");
-    if (tv && std::atoi(tv) == 512) nt = 512;
-    const char* v = std::getenv("MQ_QUANT_CTAS");
-    if (v && std::atoi(v) > 0) ctas_per_sm = std::atoi(v);
     attr_set = true;
   }
-  int dev = 0, sms = 148;
-  cudaGetDevice(&dev);
-  cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+  const int sms = sm_count();
   long long grid = (long long)sms * ctas_per_sm;
   if (grid > n_items) grid = n_items;
   if (r16 && a.sr) return launch_pdl(quantize_pipe_kernel<FMT, 256, true, true>, dim3((unsigned)grid), dim3(256), QPIPE_SMEM, s, a, n_pstrips, Ct, (unsigned)n_items);
   if (r16) return launch_pdl(quantize_pipe_kernel<FMT, 256, false, true>, dim3((unsigned)grid), dim3(256), QPIPE_SMEM, s, a, n_pstrips, Ct, (unsigned)n_items);
   if (a.sr) return launch_pdl(quantize_pipe_kernel<FMT, 256, true>, dim3((unsigned)grid), dim3(256), QPIPE_SMEM, s, a, n_pstrips, Ct, (unsigned)n_items);
-  if (nt == 512) return launch_pdl(quantize_pipe_kernel<FMT, 512, false>, dim3((unsigned)grid), dim3(512), QPIPE_SMEM, s, a, n_pstrips, Ct, (unsigned)n_items);
   return launch_pdl(quantize_pipe_kernel<FMT, 256, false>, dim3((unsigned)grid), dim3(256), QPIPE_SMEM, s, a, n_pstrips, Ct, (unsigned)n_items);
 }
 
@@ -804,7 +762,7 @@ cudaError_t launch_q(const QuantArgs& a, int n_pstrips, int Ct, long long n_item
 cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s) {
   const bool vec = (a.P % 4 == 0) && ((reinterpret_cast<uintptr_t>(a.src) & 15) == 0);
   // at most 16 rows (e.g. a batch of 16 samples): items of 16 positions, see quantize_pipe_kernel
-  const bool r16 = vec && !a.line && a.src_stride_r == 0 && a.R <= 16 && !std::getenv("MQ_QUANT_NO_R16");
+  const bool r16 = vec && !a.line && a.src_stride_r == 0 && a.R <= 16 && !env_int("MQ_QUANT_NO_R16", 0);
   const int psi = r16 ? 2 * PS : PS;
   const int n_pstrips = (a.P + psi - 1) / psi;
   const int Rt = (a.R + 31) / 32, Ct = a.Cp / 32;
@@ -826,8 +784,8 @@ cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s) {
   // large tensors with 16-byte rows: whole-line TMA boxes (items of 32 positions); small ones keep the 8-position items,
   // which give a small tensor more blocks to spread over
   const long long elems = (long long)a.P * a.R * a.C;
-  const char* tv = std::getenv("MQ_QUANT_TMA");
-  const bool tma = vec && (a.debug_skip_loads || (tv ? std::atoi(tv) != 0 : (elems >= (1ll << 22) || (a.line && elems >= (1ll << 18)))));
+  const int tv = env_int("MQ_QUANT_TMA", -1);   // 1 / 0 force the choice
+  const bool tma = vec && (a.debug_skip_loads || (tv >= 0 ? tv != 0 : (elems >= (1ll << 22) || (a.line && elems >= (1ll << 18)))));
   if (a.debug_skip_loads && !tma) return cudaErrorInvalidValue;
   if (tma) {
     switch (a.fmt) {

@@ -25,16 +25,6 @@
 namespace mq {
 namespace {
 using namespace tc;
-#ifdef MQ_TC_PROFILE
-__device__ unsigned long long g_wblk[160][6];   // per block: start, after setup, producer done, MMA done, epilogue done, SM id
-__device__ __forceinline__ unsigned long long gtime() { unsigned long long t; asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t)); return t; }
-#define WPROF(slot) do { if (blockIdx.x < 160) g_wblk[blockIdx.x][slot] = gtime(); } while (0)
-__device__ unsigned long long g_wtrace[2][4][256];   // blocks 0 and 1: per stage TMA issue, landed, scales copied, MMAs issued
-#define WTRACE(k, i) do { if (blockIdx.x < 2 && (i) < 256) g_wtrace[blockIdx.x][k][i] = gtime(); } while (0)
-#else
-#define WPROF(slot) do { } while (0)
-#define WTRACE(k, i) do { } while (0)
-#endif
 
 constexpr int WG_THREADS = 320;   // MMA warp, scale copier / loader, eight more loader warps (four of them the epilogue)
 
@@ -147,7 +137,6 @@ __global__ void __launch_bounds__(WG_THREADS, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_p,
                 const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb, const WgradTcParams p) {
   constexpr int SPA = FP4 ? 2 : 1;     // scale bytes per MMA per row
-  if (threadIdx.x == 0) WPROF(0);
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int TG = p.TG;
@@ -206,7 +195,6 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
   pdl_wait();   // set-up above touched only shared memory, tensor memory and the kernel parameters
-  if (threadIdx.x == 0) WPROF(1);
 
   // ------------------------------------------------------------------ loaders
   // A warp gets one bulk copy accepted per ~170 cycles whatever its size, and its loop around that copy (barrier
@@ -256,7 +244,6 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       if (*abort_flag) break;
       if (!mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
       if (elect_one()) {
-        if (kind == 0) WTRACE(0, i);
         if (rank == 0) mbar_arrive_expect_tx(bar, my_bytes);
         // 8-bit mode: the X-side chunk of (padded pixel, sample chunk); E2M1: of (tap group, stage)
         const long long xchunk = !FP4 ? ((((long long)cb * p.Hp + (xh + p.ph)) * p.Wp + (xw + p.pw)) * p.nchunks + nc) : 0;
@@ -293,7 +280,6 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       for (int r = 0; r < 2; ++r)
         if (++nc == p.nchunks) { nc = 0; if (++wg == p.groups_w) { wg = 0; ++ho; } }
     }
-    if (kind == 0 && half == 0 && lane == 0) WPROF(2);
   }
   __syncwarp();
   if (warp == 1) {
@@ -346,20 +332,9 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       }
       const uint32_t d1 = tmem + (uint32_t)p.n0;
       uint32_t s = 0, phase = 0, accumulate = 0;
-#ifdef MQ_TC_PROFILE
-      long long cw = 0, ci = 0, cc = 0;
-      const long long loop_c0 = clock64(); const unsigned long long loop_g0 = gtime();
-#endif
 #pragma unroll 1
       for (int i = 0; i < nst; ++i) {   // another role's abort shows here as this thread's own bounded wait running out
-#ifdef MQ_TC_PROFILE
-        const long long q0 = clock64();
-#endif
         if (!mbar_wait((FP4 && !p.mma_cp) ? &sffull[s] : &full[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
-#ifdef MQ_TC_PROFILE
-        const long long q1 = clock64();
-        if (!FP4 && lane == 0) WTRACE(1, i);
-#endif
         tc_fence_after_sync();
         const uint32_t so = s * stage16;
         const uint32_t sf_t = sf_base + s * sf_cols;
@@ -380,7 +355,6 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
               tmem_cp_32x128b_warpx4(sf_t + 8, sfd + 64);
               if (p.NB > 1) tmem_cp_32x128b_warpx4(sf_t + 12, sfd + 96);
             }
-            WTRACE(2, i);
 #pragma unroll
             for (int a = 0; a < 4; ++a) {
               const uint32_t accu = a > 0 ? 1u : accumulate;
@@ -389,7 +363,6 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
               else mma_mxf8f6f4(tmem, ad + 256u * a, bd + kb16[a], id, sf_t, sf_t + 8, accu);
             }
             if (CTA2) tc_commit_2_multicast(&empty[s], 3); else tc_commit(&empty[s]);
-            WTRACE(3, i);
           }
         } else
         if (elect_one()) {
@@ -413,31 +386,18 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             else mma_mxf8f6f4(d1, ad + ka16[a], bd + row16_1 + kb16[a], idesc_a[1][a], sf_t + sfa_off[a], sf_t + sfb_off[1][a], accu);
           }
         }
-        WTRACE(3, i);
         if (CTA2) tc_commit_2_multicast(&empty[s], 3); else tc_commit(&empty[s]);   // frees the stage in both blocks
         }
         __syncwarp();
         accumulate = 1;
-#ifdef MQ_TC_PROFILE
-        const long long q2 = clock64();
-#endif
         if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
-#ifdef MQ_TC_PROFILE
-        const long long q3 = clock64();
-        cw += q1 - q0; ci += q2 - q1; cc += q3 - q2;
-#endif
       }
-#ifdef MQ_TC_PROFILE
-      if (blockIdx.x < 2 && lane == 0) { g_wtrace[blockIdx.x][1][254] = (unsigned long long)(clock64() - loop_c0); g_wtrace[blockIdx.x][1][255] = gtime() - loop_g0; }
-      if (blockIdx.x < 2 && lane == 0) { g_wtrace[blockIdx.x][0][253] = (unsigned long long)cw; g_wtrace[blockIdx.x][0][254] = (unsigned long long)ci; g_wtrace[blockIdx.x][0][255] = (unsigned long long)cc; }
-#endif
       if (elect_one()) {
         if (CTA2) {
           if (nst > 0) tc_commit_2_multicast(tfull, 3); else { mbar_arrive(tfull); mbar_arrive_remote(tfull, 1); }
         } else {
           if (nst > 0) tc_commit(tfull); else mbar_arrive(tfull);
         }
-        WPROF(3);
       }
       __syncwarp();
     }
@@ -453,7 +413,6 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 #pragma unroll 1
       for (int i = 0; i < nst && !*abort_flag; ++i) {
         if (!mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
-        if (lane == 0) WTRACE(1, i);
         tc_fence_after_sync();
         const uint32_t so = s * stage16;
         const uint32_t sf_t = sf_base + s * sf_cols;
@@ -476,7 +435,6 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
             }
           }
           }
-          WTRACE(2, i);
           if (CTA2) tc_commit_2(&sffull[s]); else tc_commit(&sffull[s]);
         }
         __syncwarp();
@@ -536,9 +494,6 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   __syncthreads();
   if (CTA2) cluster_sync_all();   // nothing of the peer block is touched after this point
   if (warp == 1) { if (CTA2) tmem_dealloc_2(tmem, p.tmem_cols); else tmem_dealloc(tmem, p.tmem_cols); }
-#ifdef MQ_TC_PROFILE
-  if (threadIdx.x == 0) { WPROF(4); unsigned smid; asm volatile("mov.u32 %0, %smid;" : "=r"(smid)); if (blockIdx.x < 160) g_wblk[blockIdx.x][5] = smid; }
-#endif
 }
 
 // ---- E2M1 re-layout: stored [pixel][n][Cp] nibbles -> [pixel][Cp][Npad] nibbles (n fastest, zero for n >= N) ----
@@ -705,10 +660,6 @@ __global__ void __launch_bounds__(256) wgrad_flat_prep_kernel(const FlatArgs x, 
 
 }  // namespace
 
-#ifdef MQ_TC_PROFILE
-extern "C" int mqdbg_read_wtrace(unsigned long long* out2048) { return cudaMemcpyFromSymbol(out2048, g_wtrace, sizeof(unsigned long long) * 2048) == cudaSuccess ? 0 : 1; }
-extern "C" int mqdbg_read_wblk(unsigned long long* out960) { return cudaMemcpyFromSymbol(out960, g_wblk, sizeof(unsigned long long) * 960) == cudaSuccess ? 0 : 1; }
-#endif
 size_t wgrad_tc_smem_bytes(const WgradTcParams& p) { return 1024 + (size_t)p.stages * p.stage_bytes + (4 * (size_t)p.stages + 2) * 8 + 64; }
 
 cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_p, const CUtensorMap& map_sfa,
@@ -750,13 +701,13 @@ static bool make_flat_args(FlatArgs* fa, const uint8_t* in, uint8_t* out, int Hs
                            int nblocks, int KBn) {
   fa->in = in; fa->out = out; fa->Hs = Hs; fa->Ws = Ws; fa->N = N; fa->Cs_p = Cs_p; fa->P_out = P_out; fa->Wp = Wp; fa->off_h = off_h; fa->off_w = off_w;
   fa->rows = rows; fa->nblocks = nblocks; fa->KBn = KBn;
-  fa->wide = (KBn == 128 && nblocks * rows >= 256 && N <= 256 && !getenv("MQ_WGRAD_NO_WIDE_PREP")) ? 1 : 0;
+  fa->wide = (KBn == 128 && nblocks * rows >= 256 && N <= 256 && !env_int("MQ_WGRAD_NO_WIDE_PREP", 0)) ? 1 : 0;
   if (fa->wide) {
     fa->ncg = (nblocks * rows + 255) / 256;
     const long long units = (long long)P_out * fa->ncg;
     if (units >= 0xffffffffLL) return false;
     fa->units = (unsigned)units;
-    fa->blocks = (unsigned)(units < 148LL * 3 ? (units < 1 ? 1 : units) : 148LL * 3);
+    fa->blocks = (unsigned)(units < (long long)sm_count() * 3 ? (units < 1 ? 1 : units) : (long long)sm_count() * 3);
     return true;
   }
   fa->ncg = (nblocks * rows + 63) / 64;
@@ -764,7 +715,7 @@ static bool make_flat_args(FlatArgs* fa, const uint8_t* in, uint8_t* out, int Hs
   if (units >= 0xffffffffLL) return false;
   fa->units = (unsigned)units;
   long long blocks = (units + 7) / 8;
-  if (blocks > 148LL * 32) blocks = 148LL * 32;
+  if (blocks > (long long)sm_count() * 32) blocks = (long long)sm_count() * 32;
   if (blocks < 1) blocks = 1;
   fa->blocks = (unsigned)blocks;
   return true;

@@ -55,6 +55,7 @@ def lib():
         _lib = ctypes.CDLL(_LIB_PATH)
         _lib.mq_status_string.restype = ctypes.c_char_p
         _lib.mq_kernel_launch_count.restype = ctypes.c_ulonglong
+        _lib.mq_reload_env.restype = None
     return _lib
 
 
@@ -197,6 +198,52 @@ def conv_bwd_data(desc, wq, dyq, dx=None, layout=NCHW, workspace=None, stream=No
     return _conv("mq_conv_bwd_data", OP_BWD_DATA, desc, wq, dyq, dx, (d.N, d.C_in, d.H, d.W), (d.H, d.W, d.N, d.C_in), layout, workspace, stream, dtype)
 
 
+ACT_NONE, ACT_RELU, ACT_SILU = 0, 1, 2
+
+
+def conv_mx_workspace_size(desc, op, fmt_a, fmt_b):
+    b = ctypes.c_size_t()
+    _check("mq_conv_mx_workspace_size", lib().mq_conv_mx_workspace_size(ctypes.byref(_d(desc)), op, fmt_a, fmt_b, ctypes.byref(b)))
+    return b.value
+
+
+def _mx_out(desc, op, fmt, role, device):
+    """An empty stored tensor of what the quantizing epilogue emits: the forward result as a role-X tensor of
+    N x C_out x Ho x Wo, the input gradient as a role-DY tensor of N x C_in x H x W."""
+    d = ConvDesc(*desc)
+    ho, wo = _out_hw(d)
+    c, h, w = (d.C_out, ho, wo) if op == OP_FWD else (d.C_in, d.H, d.W)
+    cp = (c + 31) // 32 * 32
+    cb = h * w * d.N * cp * (4 if fmt == E2M1 else 8) // 8
+    sb = h * w * ((d.N + 31) // 32) * (cp // 32)
+    return QTensor(_new(cb, torch.uint8, device), _new(sb, torch.uint8, device), fmt, role)
+
+
+def _conv_mx(name, op, desc, qa, qb, out, extra, workspace, stream):
+    need = conv_mx_workspace_size(desc, op, qa.fmt, qb.fmt)
+    if workspace is None and need > 0:
+        workspace = _new(need, torch.uint8, qa.codes.device)
+    wp = ctypes.c_void_p(workspace.data_ptr()) if workspace is not None else None
+    wn = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    a, b, o = qa._c(), qb._c(), out._c()
+    _check(name, getattr(lib(), name)(ctypes.byref(_d(desc)), ctypes.byref(a), ctypes.byref(b), *extra, ctypes.byref(o), wp, ctypes.c_size_t(wn), _stream(stream)))
+    return out
+
+
+def conv_fwd_mx(desc, xq, wq, fmt, act=ACT_NONE, yq=None, workspace=None, stream=None):
+    """mq_conv_fwd_mx: act(conv(X, W)) emitted as the next layer's stored activation (element format `fmt`)."""
+    if yq is None:
+        yq = _mx_out(desc, OP_FWD, fmt, ROLE_X, xq.codes.device)
+    return _conv_mx("mq_conv_fwd_mx", OP_FWD, desc, xq, wq, yq, (ctypes.c_int(act),), workspace, stream)
+
+
+def conv_bwd_data_mx(desc, wq, dyq, fmt, dxq=None, workspace=None, stream=None):
+    """mq_conv_bwd_data_mx: the input gradient emitted as the previous layer's stored output gradient."""
+    if dxq is None:
+        dxq = _mx_out(desc, OP_BWD_DATA, fmt, ROLE_DY, wq.codes.device)
+    return _conv_mx("mq_conv_bwd_data_mx", OP_BWD_DATA, desc, wq, dyq, dxq, (), workspace, stream)
+
+
 STATIC_SCRATCH_BYTES = 16 << 20
 
 
@@ -217,6 +264,11 @@ def conv_bwd_data_static(desc, wq, dyq, dx=None, layout=NCHW, stream=None):
 def conv_bwd_weight(desc, xq, dyq, dw=None, layout=NCHW, workspace=None, stream=None):
     d = ConvDesc(*desc)
     return _conv("mq_conv_bwd_weight", OP_BWD_WEIGHT, desc, xq, dyq, dw, (d.C_out, d.C_in, d.Kh, d.Kw), (d.C_out, d.Kh, d.Kw, d.C_in), layout, workspace, stream)
+
+
+def reload_env():
+    """mq_reload_env: the MQ_* environment knobs are read once each; call this after changing one."""
+    lib().mq_reload_env()
 
 
 def kernel_launch_count():

@@ -52,11 +52,11 @@ def check_fwd(d, fmts, oq, gq, samples=None, seed=0):
 @pytest.mark.parametrize("route", ["tensor-cores", "cuda-cores", "whole-line-quantizer"])
 @pytest.mark.parametrize("fmts", [(E4M3, E4M3), (E2M1, E2M1), (E5M2, E4M3), (E3M2, E2M3)], ids=lambda f: "-".join(map(str, f)))
 @pytest.mark.parametrize("name,shape", SHAPES, ids=[s[0] for s in SHAPES])
-def test_line_blocks_quantize_im2col_forward(name, shape, fmts, route, monkeypatch):
+def test_line_blocks_quantize_im2col_forward(name, shape, fmts, route, knobs):
     if route == "cuda-cores":
-        monkeypatch.setenv("MQ_DISABLE_TC", "1")
+        knobs(MQ_DISABLE_TC="1")
     if route == "whole-line-quantizer":
-        monkeypatch.setenv("MQ_QUANT_TMA", "1")
+        knobs(MQ_QUANT_TMA="1")
     d, x, w, oq = line_case(name, shape, fmts)
     gq = [mq.quantize(d, r, f, dev(t), block=mq.LINE32) for r, f, t in zip((mq.ROLE_X, mq.ROLE_W), fmts, (x, w))]
     for what, g, (c, s) in zip(("X", "W"), gq, oq):

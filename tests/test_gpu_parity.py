@@ -208,10 +208,10 @@ def test_layer_from_host_buffers_matches_the_device_calls(fmts):
     assert mq.last_device_status() == 0
 
 
-def test_6bit_gemms_on_cuda_cores(monkeypatch):
+def test_6bit_gemms_on_cuda_cores(knobs):
     """The CUDA-core route of 6-bit operands (the default packs them for the tensor cores; the weight gradient always
     takes this route)."""
-    monkeypatch.setenv("MQ_TC_NO_FP6", "1")
+    knobs(MQ_TC_NO_FP6="1")
     d = inputs.conv_desc(64, 96, 8, 8, 64, 3, 1, 1)
     for fmts in ((E3M2, E4M3, E5M2), (E2M3, E2M3, E2M3)):
         ol = OracleLayer(make_layer("fp6_cuda_cores", d, fmts, seed=31, kinds=("relu", "kaiming", "gauss")))
@@ -221,17 +221,21 @@ def test_6bit_gemms_on_cuda_cores(monkeypatch):
 
 ALT_PATHS = [("MQ_TC_NO_HALO", "1"), ("MQ_TC_NO_FUSED", "1"), ("MQ_TC_NO_TMA_STORE", "1"), ("MQ_TC_TMA_STORE", "1"), ("MQ_TC_NO_PAIR", "1"),
              ("MQ_TC_BN", "256"), ("MQ_TC_TW", "4"), ("MQ_TC_TW", "16"), ("MQ_TC_TW", "32"), ("MQ_WGRAD_NO_FLAT", "1"),
-             ("MQ_WGRAD_NO_GROUP", "1"), ("MQ_WGRAD_NO_GROUP8", "1"), ("MQ_WGRAD_N128", "1"), ("MQ_WGRAD_NO_CTA2", "1"), ("MQ_TC_NO_MMA_CP", "1"), ("MQ_WGRAD_MMA_CP", "1"), ("MQ_TC_FP4_BN128", "1"), ("MQ_TC_CTA2", "1"), ("MQ_TC_NO_SFA_DEDUP", "1"), ("MQ_TC_NO_WT_FUSED", "1"), ("MQ_WGRAD_FP4_PIXEL", "1"), ("MQ_WGRAD_SPLITS", "3"), ("MQ_DISABLE_TC_WGRAD", "1"), ("MQ_DISABLE_TC", "1")]
+             ("MQ_WGRAD_NO_GROUP", "1"), ("MQ_WGRAD_NO_GROUP8", "1"), ("MQ_WGRAD_N128", "1"), ("MQ_WGRAD_NO_CTA2", "1"), ("MQ_TC_NO_MMA_CP", "1"), ("MQ_WGRAD_MMA_CP", "1"), ("MQ_TC_FP4_BN128", "1"), ("MQ_TC_NO_SFA_DEDUP", "1"), ("MQ_TC_NO_WT_FUSED", "1"), ("MQ_WGRAD_FP4_PIXEL", "1"), ("MQ_WGRAD_SPLITS", "3"), ("MQ_DISABLE_TC_WGRAD", "1"), ("MQ_DISABLE_TC", "1"),
+             ("MQ_NO_PDL", "1"), ("MQ_QUANT_NO_R16", "1"), ("MQ_QUANT_TMA", "0"), ("MQ_WGRAD_NO_WIDE_PREP", "1")]
 ALT_SHAPES = [("thin", (32, 64, 8, 16, 96, 3, 1, 1)), ("wide_s2", (32, 256, 8, 12, 288, 3, 2, 1)), ("wide_s1", (32, 256, 4, 8, 288, 3, 1, 1)),
               ("thin32_s2", (40, 20, 9, 10, 48, 3, 2, 1))]
+# knobs that act on other shapes: at most 16 samples (quantizer items of 16 positions), 256 samples x 256 channels (the wide E2M1
+# weight-gradient preparation)
+ALT_EXTRA = {"MQ_QUANT_NO_R16": [("batch16", (16, 40, 10, 12, 72, 3, 1, 1))], "MQ_WGRAD_NO_WIDE_PREP": [("n256_c256", (256, 256, 4, 4, 256, 3, 1, 1))]}
 
 
 @pytest.mark.parametrize("knob", ALT_PATHS, ids=[f"{k}={v}" for k, v in ALT_PATHS])
-def test_alternate_kernel_paths(knob, monkeypatch):
+def test_alternate_kernel_paths(knob, knobs):
     """Every switchable kernel path (per-tap instead of whole-tile, unfused preparation, plain stores, other tile
     shapes, the other weight-gradient modes incl. single blocks where pairs are the default, the CUDA-core kernels) meets the same parity bar."""
-    monkeypatch.setenv(knob[0], knob[1])
-    for name, shape in ALT_SHAPES:
+    knobs(**{knob[0]: knob[1]})
+    for name, shape in ALT_SHAPES + ALT_EXTRA.get(knob[0], []):
         d = inputs.conv_desc(*shape)
         for fmts in ((E4M3, E4M3, E5M2), (E2M1, E2M1, E2M1)):
             ol = OracleLayer(make_layer(name, d, fmts, seed=23, kinds=("relu", "kaiming", "gauss")))
@@ -250,13 +254,11 @@ TMA_Q_SHAPES = [
 
 
 @pytest.mark.parametrize("fmt", [E4M3, E5M2, E2M1, E3M2, E2M3])
-@pytest.mark.parametrize("order", ["0", "1"], ids=["tile-fastest", "strip-fastest"])
 @pytest.mark.parametrize("name,shape", TMA_Q_SHAPES, ids=[s[0] for s in TMA_Q_SHAPES])
-def test_quantize_whole_line_kernel_on_small_shapes(name, shape, order, fmt, monkeypatch):
+def test_quantize_whole_line_kernel_on_small_shapes(name, shape, fmt, knobs):
     """The whole-line (TMA) quantizer that large NCHW tensors take, forced onto small ragged ones: the oracle's bytes,
     with round-to-nearest and with the stochastic rounding."""
-    monkeypatch.setenv("MQ_QUANT_TMA", "1")
-    monkeypatch.setenv("MQ_QUANT_STRIP_FASTEST", order)
+    knobs(MQ_QUANT_TMA="1")
     d = inputs.conv_desc(*shape)
     ol = OracleLayer(make_layer(name, d, (fmt, fmt, fmt), seed=41, kinds=("relu", "kaiming", "gauss")))
     check_quantize(ol)

@@ -39,10 +39,10 @@ def test_gradient_codes_match_the_oracle(name, shape, fmt):
 
 
 @pytest.mark.parametrize("fmt", [E4M3, E2M1])
-def test_per_element_key_path(fmt, monkeypatch):
+def test_per_element_key_path(fmt, knobs):
     """Tensors of 2^32 elements or more derive the stream key from the index's high word per element; forced here on a
     small tensor (high word 0), where it must give the same bytes."""
-    monkeypatch.setenv("MQ_SR_WIDE", "1")
+    knobs(MQ_SR_WIDE="1")
     d = inputs.conv_desc(64, 96, 8, 8, 64, 3, 1, 1)
     g = inputs.make_dy(d, 8, "gauss")
     oc, osc = oracle.quantize_sr(d, oracle.ROLE_DY, fmt, g, 77)
