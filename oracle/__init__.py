@@ -59,6 +59,11 @@ def _l():
         lib.orc_sr_bits.argtypes = [ctypes.c_uint64, ctypes.c_uint64]
         lib.orc_quantize_sr.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_uint64,
                                         ctypes.c_void_p, ctypes.c_void_p]
+        lib.orc_quantize_ts.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_float, ctypes.c_int, ctypes.c_uint64,
+                                        ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_void_p]
+        lib.orc_dequant_ts.argtypes = [ctypes.c_void_p, ctypes.c_int, ctypes.c_int, ctypes.c_int, ctypes.c_void_p, ctypes.c_void_p, ctypes.c_float, ctypes.c_void_p]
+        lib.orc_block_scale_code.argtypes = [ctypes.c_float, ctypes.c_float]
+        lib.orc_ts_elem_code.argtypes = [ctypes.c_float, ctypes.c_float, ctypes.c_float]
         _lib = lib
     return _lib
 
@@ -142,6 +147,42 @@ def quantize_sr(desc, role, fmt, src, seed, block=(32, 32)):
     rc = _l().orc_quantize_sr(_p(_desc(desc)), role, fmt, block[0], block[1], _p(src), int(seed), _p(codes), _p(scales))
     assert rc == 0
     return codes, scales
+
+
+def quantize_ts(desc, role, src, block=(16, 16), amax=None, seed=None):
+    """The paper's own number format (Sec. III-A, Eq. 4-6): fp32 scale per tensor, E4M3 scale per block, E2M1 elements.
+    Returns (codes, block scales as E4M3 bytes, T_scale, max|X|).  amax: take T_scale from this value instead of the
+    tensor's own maximum (statistics of earlier batches, Sec. VII-B).  seed: stochastic Round(.) with that seed."""
+    src = np.ascontiguousarray(src, dtype=np.float32)
+    assert src.shape == logical_shape(desc, role), (src.shape, logical_shape(desc, role))
+    assert np.isfinite(src).all(), "non-finite inputs are outside the contract"
+    cb, sb = qtensor_sizes(desc, role, E2M1, block)
+    codes = np.zeros(cb, dtype=np.uint8)
+    scales = np.zeros(sb, dtype=np.uint8)
+    ts, am = np.zeros(1, dtype=np.float32), np.zeros(1, dtype=np.float32)
+    rc = _l().orc_quantize_ts(_p(_desc(desc)), role, block[0], block[1], _p(src), ctypes.c_float(-1.0 if amax is None else float(amax)),
+                              0 if seed is None else 1, 0 if seed is None else int(seed), _p(codes), _p(scales), _p(ts), _p(am))
+    assert rc == 0
+    return codes, scales, float(ts[0]), float(am[0])
+
+
+def dequant_ts(desc, role, codes, scales, tensor_scale, block=(16, 16)):
+    """Fake quantization of the paper's own format: element x block scale x tensor scale, float64, logical order."""
+    out = np.zeros(logical_shape(desc, role), dtype=np.float64)
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    scales = np.ascontiguousarray(scales, dtype=np.uint8)
+    _l().orc_dequant_ts(_p(_desc(desc)), role, block[0], block[1], _p(codes), _p(scales), ctypes.c_float(tensor_scale), _p(out))
+    return out
+
+
+def block_scale_code(block_amax, tensor_scale):
+    """Eq. 5 for one block: the E4M3 code of max|X_i| / (T_scale * 6)."""
+    return int(_l().orc_block_scale_code(ctypes.c_float(block_amax), ctypes.c_float(tensor_scale)))
+
+
+def ts_elem_code(x, block_scale, tensor_scale):
+    """Eq. 6 for one element (round to nearest): the E2M1 code of x / (B_scale * T_scale)."""
+    return int(_l().orc_ts_elem_code(ctypes.c_float(x), ctypes.c_float(block_scale), ctypes.c_float(tensor_scale)))
 
 
 def dequant(desc, role, fmt, codes, scales, block=(32, 32)):

@@ -22,7 +22,11 @@
 //  * a quantization block is a br x bc rectangle over the two axes Sec. IV-B names for each
 //    tensor (X: N x Cin, W: Cout x Cin, G_Y: N x Cout) at one spatial / tap position;
 //    32 x 32 is the square of Sec. IV-B with sqrt(B) = 32, 1 x 32 is the line block of Sec. III-A;
-//  * stored order inside a spatial position is [n][c] with c fastest ("channel-batch-first").
+//  * stored order inside a spatial position is [n][c] with c fastest ("channel-batch-first");
+//  * the paper's own number format (Sec. III-A, Eq. 4-6: an fp32 scale per tensor, an E4M3 scale per block, E2M1
+//    elements) is provided beside the E8M0 one (orc_quantize_ts and friends).  The paper does not say in which precision
+//    Eq. 4-6 are evaluated; since their roundings decide integer codes, they are evaluated here in IEEE single precision,
+//    one rounding per written operation, in the order the equations are written - the precision of the tensors they act on.
 
 #include <cmath>
 #include <cstdint>
@@ -148,6 +152,28 @@ int scale_code(int fmt, double amax) {
 }
 
 double scale_value(int code) { return std::ldexp(1.0, code - 127); }
+
+// ---- the paper's own number format: per-tensor scale + E4M3 block scale + E2M1 elements (Sec. III-A, Eq. 4-6) ------
+// Eq. 4:  T_scale = max|X| / (max B_sf * max B_ef)                with max B_sf = 448 (E4M3), max B_ef = 6 (E2M1)
+// Eq. 5:  B_scale = CastE4M3( max|X_i| / (T_scale * max B_ef) )   round to nearest E4M3 value
+// Eq. 6:  X_i^q   = Round( X_i / (B_scale * T_scale) )            round to nearest E2M1 value
+// Each written operation is one IEEE single-precision operation (see the header).  Readings where the paper is silent:
+// ties go to the even code and magnitudes beyond the largest finite value saturate, in both roundings (as for the E8M0
+// format); a block or tensor of zeros has scale 0 and codes +-0 (no division takes place); when the tensor's maximum
+// is supplied from outside (statistics of earlier batches, Sec. VII-B) values may exceed it and saturate likewise.
+float tensor_scale_of(float amax) { return amax / (448.0f * 6.0f); }                       // Eq. 4
+int block_scale_code(float block_amax, float tscale) {                                     // Eq. 5
+  if (!(block_amax > 0.0f) || !(tscale > 0.0f)) return 0;
+  float arg = block_amax / (tscale * 6.0f);
+  return encode_elem(E4M3, (double)arg) & 0x7F;
+}
+int ts_elem_code(float x, float bscale, float tscale, bool stochastic, uint32_t bits) {    // Eq. 6
+  int sign = std::signbit(x) ? 8 : 0;
+  if (!(bscale > 0.0f) || !(tscale > 0.0f)) return sign;
+  float scaled = x / (bscale * tscale);
+  return stochastic ? encode_elem_sr(E2M1, (double)scaled, bits) : encode_elem(E2M1, (double)scaled);
+}
+
 
 // ---- the 2-D views of Sec. IV-B -------------------------------------------------------------
 // Each tensor is seen, at every position p (a pixel (h,w) for X, (ho,wo) for G_Y, a tap (kh,kw)
@@ -287,6 +313,69 @@ int orc_dequant(const int* d, int role, int fmt, int br, int bc, const uint8_t* 
       }
   return 0;
 }
+
+
+// ---- the paper's own format (Eq. 4-6) on br x bc blocks --------------------------------------------------------------
+// codes: E2M1, packed as in orc_quantize; scales: one E4M3 byte per block, in the order of orc_quantize's scales;
+// tensor_scale: T_scale; tensor_amax: max|X| of this tensor.  amax_in < 0: T_scale from this tensor's own maximum
+// (two passes over the data); amax_in >= 0: T_scale from that value instead (statistics of earlier batches).
+int orc_quantize_ts(const int* d, int role, int br, int bc, const float* src, float amax_in, int stochastic, uint64_t seed, uint8_t* codes,
+                    uint8_t* scales, float* tensor_scale, float* tensor_amax) {
+  Conv cv = conv_from(d);
+  View v = view_of(cv, role);
+  if (bc <= 0 || br <= 0 || v.Cp % bc != 0 || (bc & 1)) return 1;
+  int64_t cb_bytes, sb_bytes;
+  orc_qtensor_sizes(d, role, E2M1, br, bc, &cb_bytes, &sb_bytes);
+  std::memset(codes, 0, (size_t)cb_bytes);
+  std::memset(scales, 0, (size_t)sb_bytes);
+  float amax = 0.0f;
+  size_t total = (size_t)v.P * v.R * v.C;
+  for (size_t i = 0; i < total; ++i) { float a = std::fabs(src[i]); if (a > amax) amax = a; }
+  *tensor_amax = amax;
+  const float tscale = tensor_scale_of(amax_in >= 0.0f ? amax_in : amax);
+  *tensor_scale = tscale;
+  int Rb = (v.R + br - 1) / br, Cb = v.Cp / bc;
+#pragma omp parallel for schedule(static)
+  for (int p = 0; p < v.P; ++p) {
+    for (int rb = 0; rb < Rb; ++rb) {
+      for (int cb = 0; cb < Cb; ++cb) {
+        float bmax = 0.0f;
+        for (int r = rb * br; r < (rb + 1) * br && r < v.R; ++r)
+          for (int c = cb * bc; c < (cb + 1) * bc && c < v.C; ++c) {
+            float a = std::fabs(src[src_index(v, p, r, c)]);
+            if (a > bmax) bmax = a;
+          }
+        int sc = block_scale_code(bmax, tscale);
+        scales[scale_index(v, br, bc, p, rb, cb)] = (uint8_t)sc;
+        float bscale = (float)decode_elem(E4M3, sc);
+        for (int r = rb * br; r < (rb + 1) * br && r < v.R; ++r)
+          for (int c = cb * bc; c < (cb + 1) * bc && c < v.C; ++c) {
+            size_t si = src_index(v, p, r, c);
+            int code = ts_elem_code(src[si], bscale, tscale, stochastic != 0, stochastic ? sr_bits(seed, (uint64_t)si) : 0u);
+            put_code(codes, E2M1, code_index(v, p, r, c), code);
+          }
+      }
+    }
+  }
+  return 0;
+}
+
+// Fake quantization of that format: element value x block scale x tensor scale (Sec. III-A).
+int orc_dequant_ts(const int* d, int role, int br, int bc, const uint8_t* codes, const uint8_t* scales, float tensor_scale, double* out) {
+  Conv cv = conv_from(d);
+  View v = view_of(cv, role);
+#pragma omp parallel for schedule(static)
+  for (int p = 0; p < v.P; ++p)
+    for (int r = 0; r < v.R; ++r)
+      for (int c = 0; c < v.C; ++c) {
+        int code = get_code(codes, E2M1, code_index(v, p, r, c));
+        int sc = scales[scale_index(v, br, bc, p, r / br, c / bc)];
+        out[src_index(v, p, r, c)] = decode_elem(E2M1, code) * decode_elem(E4M3, sc) * (double)tensor_scale;
+      }
+  return 0;
+}
+int orc_block_scale_code(float block_amax, float tscale) { return block_scale_code(block_amax, tscale); }
+int orc_ts_elem_code(float x, float bscale, float tscale) { return ts_elem_code(x, bscale, tscale, false, 0u); }
 
 // sizes of X'_{Cin,N} built from the stored quantized activation
 int orc_im2col_sizes(const int* d, int fmt, int br, int bc, int64_t* codes_bytes, int64_t* scales_bytes) {
