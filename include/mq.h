@@ -35,6 +35,19 @@
  *   Such a tensor can feed the GEMM that contracts over its channel axis (the forward GEMM for X and W) and no
  *   other: that is the limitation Sec. III-B / III-C derive the square blocks from.  mq_quantize, mq_cbf_im2col
  *   and mq_conv_fwd accept it; mq_conv_bwd_data and mq_conv_bwd_weight return MQ_ERR_UNSUPPORTED for it.
+ *
+ * The paper's own number format (MQ_BLOCK_TS16): Sec. III-A as written - an fp32 scale per TENSOR (Eq. 4:
+ *   T_scale = max|X| / (448 * 6)), an E4M3 scale per block (Eq. 5: B_scale = CastE4M3(max|X_i| / (6 T_scale))) and E2M1
+ *   elements (Eq. 6: Round(X_i / (B_scale T_scale))) - on the square blocks of Sec. IV-B with a side of 16, the finest
+ *   scale granularity of the tensor cores' block-scaled E2M1 path (the paper's experiments use a side of 8).  Element
+ *   format is MQ_E2M1; codes are laid out as above; scales hold one E4M3 byte per 16 x 16 block, in the order of the
+ *   32 x 32 case with 16 in place of 32:
+ *   role X : scales [H][W][ceil(N/16)][C_in_p/16]     role W : scales [ceil(C_out/16)][Kh][Kw][C_in_p/16]
+ *   role DY: scales [Ho][Wo][ceil(N/16)][C_out_p/16]
+ *   and mq_qtensor.tensor_scale points at two device floats: T_scale, and the tensor's own max|X| (kept so that a later
+ *   step can use it as its estimate, Sec. VII-B).  Eq. 4-6 are evaluated in IEEE single precision, one rounding per
+ *   written operation; both roundings go to nearest, ties to even, and saturate; a block of zeros has scale 0.
+ *   All calls accept it (both operands of a GEMM must use it); the GEMMs run on the CUDA-core kernels in this build.
  */
 #ifndef MQ_H_
 #define MQ_H_
@@ -65,7 +78,8 @@ typedef enum { MQ_E4M3 = 0, MQ_E5M2 = 1, MQ_E2M1 = 2,
 typedef enum { MQ_ROLE_X = 0, MQ_ROLE_W = 1, MQ_ROLE_DY = 2 } mq_role; /* which tensor, Sec. IV-B   */
 typedef enum { MQ_NCHW = 0, MQ_HWNC = 1 } mq_layout;                   /* layout of an unquantized tensor */
 typedef enum { MQ_BLOCK_TILE32 = 0,      /* 32 x 32 square block (Sec. IV-B), the default           */
-               MQ_BLOCK_LINE32 = 1 } mq_block; /* 1 x 32 line block along the channel axis (Sec. III-A) */
+               MQ_BLOCK_LINE32 = 1,      /* 1 x 32 line block along the channel axis (Sec. III-A)   */
+               MQ_BLOCK_TS16 = 2 } mq_block; /* 16 x 16 square block, E4M3 block scale + fp32 tensor scale (Eq. 4-6) */
 typedef enum { MQ_F32 = 0, MQ_BF16 = 1 } mq_dtype;                     /* element type of an unquantized tensor */
 typedef enum { MQ_OP_FWD = 0, MQ_OP_BWD_DATA = 1, MQ_OP_BWD_WEIGHT = 2 } mq_op;
 typedef enum { MQ_ACT_NONE = 0, MQ_ACT_RELU = 1, MQ_ACT_SILU = 2 } mq_act;   /* activation of the quantizing producer epilogue */
@@ -86,6 +100,7 @@ typedef struct {
   int fmt;             /* mq_elem                                     */
   int role;            /* mq_role                                     */
   int block;           /* mq_block                                    */
+  float* tensor_scale; /* MQ_BLOCK_TS16: two device floats (T_scale, max|X|), 8-byte aligned; else unused */
 } mq_qtensor;
 
 /* Size queries (host only, no GPU needed). */
@@ -128,6 +143,17 @@ mq_status mq_quantize(const mq_conv_desc* desc, const void* src, int src_dtype, 
  * every launch and on any number of GPUs.  Arguments, layouts and errors as for mq_quantize. */
 mq_status mq_quantize_sr(const mq_conv_desc* desc, const void* src, int src_dtype, int src_layout, mq_qtensor* dst, unsigned long long seed,
                          void* stream);
+
+/* mq_quantize_ts -- quantizer of the paper's own format (dst->block = MQ_BLOCK_TS16, dst->fmt = MQ_E2M1) with control over
+ * where Eq. 4 takes the tensor's maximum from.  amax_in = NULL: from this tensor (two passes over `src`: a reduction,
+ * then the quantizer); mq_quantize on such a dst does exactly this.  amax_in = a device fp32: from that value - e.g.
+ * the max|X| an earlier step left in its tensor_scale[1] (statistics of previous batches, Sec. VII-B), so that the
+ * quantizer needs no result of a reduction over this tensor; elements beyond the estimate saturate.  Either way
+ * dst->tensor_scale[0] receives T_scale and dst->tensor_scale[1] this tensor's own max|X|.
+ * seed_or_null: NULL = round to nearest; else a host pointer to the 64-bit seed of the stochastic Round(.) of Eq. 6 (the
+ * gradient's rounding; draws as in mq_quantize_sr). */
+mq_status mq_quantize_ts(const mq_conv_desc* desc, const void* src, int src_dtype, int src_layout, mq_qtensor* dst, const float* amax_in,
+                         const unsigned long long* seed_or_null, void* stream);
 
 /* mq_cbf_im2col -- channel-batch-first im2col (Sec. IV-A) of the quantized activation `xq` (role X):
  * row (kh,kw,c), column (ho,wo,n) of X' is the stored code at pixel (ho*stride+kh-pad,

@@ -36,7 +36,7 @@ namespace {
 
 bool valid_fmt(int f) { return f == MQ_E4M3 || f == MQ_E5M2 || f == MQ_E2M1 || f == MQ_E3M2 || f == MQ_E2M3; }
 bool valid_role(int r) { return r == MQ_ROLE_X || r == MQ_ROLE_W || r == MQ_ROLE_DY; }
-bool valid_block(int b) { return b == MQ_BLOCK_TILE32 || b == MQ_BLOCK_LINE32; }
+bool valid_block(int b) { return b == MQ_BLOCK_TILE32 || b == MQ_BLOCK_LINE32 || b == MQ_BLOCK_TS16; }
 bool valid_dtype(int t) { return t == MQ_F32 || t == MQ_BF16; }
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
@@ -61,12 +61,17 @@ View view_of(const Geom& g, int role) {
 void sizes_of(const Geom& g, int role, int fmt, int block, size_t* cb, size_t* sb) {
   View v = view_of(g, role);
   *cb = (size_t)(v.P * v.R * v.Cp) * fmt_bits(fmt) / 8;
-  *sb = (size_t)(v.P * (block == MQ_BLOCK_LINE32 ? v.R : (v.R + 31) / 32) * (v.Cp / 32));
+  if (block == MQ_BLOCK_TS16) *sb = (size_t)(v.P * ((v.R + 15) / 16) * (v.Cp / 16));
+  else *sb = (size_t)(v.P * (block == MQ_BLOCK_LINE32 ? v.R : (v.R + 31) / 32) * (v.Cp / 32));
 }
 
 mq_status check_qtensor(const Geom& g, const mq_qtensor* q, int role) {
   if (!q || !q->codes || !q->scales) return MQ_ERR_INVALID_ARG;
   if (!valid_fmt(q->fmt) || q->role != role || !valid_block(q->block)) return MQ_ERR_INVALID_ARG;
+  if (q->block == MQ_BLOCK_TS16) {   // the paper's own format: E2M1 elements and a tensor-scale buffer
+    if (q->fmt != MQ_E2M1 || !q->tensor_scale) return MQ_ERR_INVALID_ARG;
+    if (reinterpret_cast<uintptr_t>(q->tensor_scale) & 7u) return MQ_ERR_ALIGNMENT;
+  }
   if (!aligned16(q->codes) || !aligned16(q->scales)) return MQ_ERR_ALIGNMENT;
   size_t cb, sb;
   sizes_of(g, role, q->fmt, q->block, &cb, &sb);
@@ -626,11 +631,11 @@ mq_status run_conv(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int r
     const mq_qtensor* qx_like = op == MQ_OP_FWD ? qa : qb;
     const mq_qtensor* qw = op == MQ_OP_FWD ? qb : qa;
     ConvTcPlan pl;
-    if ((op == MQ_OP_FWD || op == MQ_OP_BWD_DATA) && conv_tc_eligible(op, g, qx_like->fmt, qw->fmt) &&
+    if (qa->block != MQ_BLOCK_TS16 && (op == MQ_OP_FWD || op == MQ_OP_BWD_DATA) && conv_tc_eligible(op, g, qx_like->fmt, qw->fmt) &&
         conv_tc_plan(op, g, qx_like->fmt, qw->fmt, layout, &pl, qx_like->block == MQ_BLOCK_LINE32))
       return run_conv_tc(op, g, pl, qx_like, qw, static_cast<float*>(out), layout, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
   }
-  if (op == MQ_OP_BWD_WEIGHT) {
+  if (op == MQ_OP_BWD_WEIGHT && qa->block != MQ_BLOCK_TS16) {
     WgradPlan w = wgrad_plan(g, qa->fmt, qb->fmt);
     if (w.ok) return run_wgrad_tc(g, w, qa, qb, static_cast<float*>(out), layout, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
   }
@@ -640,6 +645,8 @@ mq_status run_conv(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int r
   a.b_codes = static_cast<const uint8_t*>(qb->codes); a.b_scales = qb->scales; a.fmt_b = qb->fmt;
   a.out = static_cast<float*>(out); a.out_layout = layout; a.workspace = ws; a.ws_bytes = ws_bytes;
   a.line = qa->block == MQ_BLOCK_LINE32 ? 1 : 0;
+  a.ts16 = qa->block == MQ_BLOCK_TS16 ? 1 : 0;
+  a.a_tscale = qa->tensor_scale; a.b_tscale = qb->tensor_scale;
   cudaError_t e = launch_conv_generic(op, a, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }
@@ -668,7 +675,8 @@ mq_status mq_im2col_sizes(const mq_conv_desc* desc, int fmt, int block, size_t* 
   if (!valid_fmt(fmt) || !valid_block(block) || !codes_bytes || !scales_bytes) return MQ_ERR_INVALID_ARG;
   Geom g = make_geom(*desc);
   *codes_bytes = (size_t)g.Ho * g.Wo * g.N * g.Kh * g.Kw * g.Cp * fmt_bits(fmt) / 8;
-  *scales_bytes = (size_t)g.Ho * g.Wo * (block == MQ_BLOCK_LINE32 ? g.N : g.Nt) * g.Kh * g.Kw * g.Ct;
+  if (block == MQ_BLOCK_TS16) *scales_bytes = (size_t)g.Ho * g.Wo * ((g.N + 15) / 16) * g.Kh * g.Kw * (g.Cp / 16);
+  else *scales_bytes = (size_t)g.Ho * g.Wo * (block == MQ_BLOCK_LINE32 ? g.N : g.Nt) * g.Kh * g.Kw * g.Ct;
   return MQ_OK;
 }
 
@@ -681,6 +689,7 @@ mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt
   const Geom g = make_geom(*desc);
   const bool line = block == MQ_BLOCK_LINE32;
   *bytes = conv_generic_workspace(op, g);
+  if (block == MQ_BLOCK_TS16) return (fmt_a == MQ_E2M1 && fmt_b == MQ_E2M1) ? MQ_OK : MQ_ERR_INVALID_ARG;   // CUDA-core kernels in this build
   if (op == MQ_OP_FWD && conv_tc_eligible(op, g, fmt_a, fmt_b)) *bytes = conv_tc_workspace(op, g, fmt_a, fmt_b, line);
   if (op == MQ_OP_BWD_DATA && conv_tc_eligible(op, g, fmt_b, fmt_a)) *bytes = conv_tc_workspace(op, g, fmt_b, fmt_a, false);
   if (op == MQ_OP_BWD_WEIGHT) {
@@ -691,7 +700,7 @@ mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt
 }
 
 static mq_status quantize_impl(const mq_conv_desc* desc, const void* src, int src_dtype, int src_layout, mq_qtensor* dst, int sr, unsigned long long seed,
-                               void* stream, unsigned wait_limit = 0, int skip_loads = 0) {
+                               void* stream, unsigned wait_limit = 0, int skip_loads = 0, const float* amax_in = nullptr) {
   mq_status st = check_desc(desc);
   if (st != MQ_OK) return st;
   if (!src || !dst || !valid_role(dst->role)) return MQ_ERR_INVALID_ARG;
@@ -708,7 +717,8 @@ static mq_status quantize_impl(const mq_conv_desc* desc, const void* src, int sr
   a.scales = dst->scales;
   a.P = (int)v.P; a.R = (int)v.R; a.C = (int)v.C; a.Cp = (int)v.Cp;
   a.line = dst->block == MQ_BLOCK_LINE32 ? 1 : 0;
-  const long long Rt = a.line ? v.R : (v.R + 31) / 32, Ct = v.Cp / 32;   // scale rows per position
+  const bool ts16 = dst->block == MQ_BLOCK_TS16;
+  const long long Rt = ts16 ? (v.R + 15) / 16 : (a.line ? v.R : (v.R + 31) / 32), Ct = ts16 ? v.Cp / 16 : v.Cp / 32;   // scale blocks per position
   if (dst->role == MQ_ROLE_W) {  // [r][p][c]
     a.out_stride_p = v.Cp; a.out_stride_r = v.P * v.Cp;
     a.sc_stride_p = Ct; a.sc_stride_r = v.P * Ct;
@@ -729,8 +739,15 @@ static mq_status quantize_impl(const mq_conv_desc* desc, const void* src, int sr
   a.sr_seed_lo = (unsigned)seed; a.sr_seed_hi = (unsigned)(seed >> 32);
   a.sr_key0 = sr_mix32(a.sr_seed_lo ^ sr_mix32(a.sr_seed_hi ^ sr_mix32(0u)));
   a.sr_wide = ((unsigned long long)v.P * (unsigned long long)v.R * (unsigned long long)v.C >= (1ull << 32) || env_int("MQ_SR_WIDE", 0)) ? 1 : 0;
-  cudaError_t e = launch_quantize(a, static_cast<cudaStream_t>(stream));
+  cudaError_t e = ts16 ? launch_quantize_ts(a, amax_in, dst->tensor_scale, static_cast<cudaStream_t>(stream)) : launch_quantize(a, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
+}
+
+mq_status mq_quantize_ts(const mq_conv_desc* desc, const void* src, int src_dtype, int src_layout, mq_qtensor* dst, const float* amax_in,
+                         const unsigned long long* seed_or_null, void* stream) {
+  if (dst && dst->block != MQ_BLOCK_TS16) return MQ_ERR_INVALID_ARG;
+  if (amax_in && (reinterpret_cast<uintptr_t>(amax_in) & 3u)) return MQ_ERR_ALIGNMENT;
+  return quantize_impl(desc, src, src_dtype, src_layout, dst, seed_or_null ? 1 : 0, seed_or_null ? *seed_or_null : 0ull, stream, 0, 0, amax_in);
 }
 
 mq_status mq_quantize(const mq_conv_desc* desc, const void* src, int src_dtype, int src_layout, mq_qtensor* dst, void* stream) {
@@ -765,6 +782,7 @@ mq_status mq_cbf_im2col(const mq_conv_desc* desc, const mq_qtensor* xq, void* co
   a.g = g;
   a.fmt = xq->fmt;
   a.line = xq->block == MQ_BLOCK_LINE32 ? 1 : 0;
+  a.ts16 = xq->block == MQ_BLOCK_TS16 ? 1 : 0;
   cudaError_t e = launch_im2col(a, static_cast<cudaStream_t>(stream));
   return e == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }
@@ -828,7 +846,7 @@ mq_status run_conv_mx(int op, const mq_conv_desc* desc, const mq_qtensor* qa, in
     a.g = g;
     a.a_codes = static_cast<const uint8_t*>(qa->codes); a.a_scales = qa->scales; a.fmt_a = qa->fmt;
     a.b_codes = static_cast<const uint8_t*>(qb->codes); a.b_scales = qb->scales; a.fmt_b = qb->fmt;
-    a.out = reinterpret_cast<float*>(base); a.out_layout = MQ_HWNC; a.workspace = base + y_bytes; a.ws_bytes = ws_bytes - y_bytes; a.line = 0;
+    a.out = reinterpret_cast<float*>(base); a.out_layout = MQ_HWNC; a.workspace = base + y_bytes; a.ws_bytes = ws_bytes - y_bytes; a.line = 0; a.ts16 = 0; a.a_tscale = nullptr; a.b_tscale = nullptr;
     if (launch_conv_generic(op, a, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MQ_ERR_CUDA;
     QuantArgs q{};
     q.src = reinterpret_cast<const float*>(base); q.codes = static_cast<uint8_t*>(out->codes); q.scales = out->scales;
@@ -975,7 +993,7 @@ mq_status mq_conv_layer_host(const mq_conv_desc* desc, int fmt_x, int fmt_w, int
   const size_t src_off[3] = {L.off_x, L.off_w, L.off_g};
   for (int r = 0; r < 3; ++r) {
     q[r].codes = base + L.off_qc[r]; q[r].scales = base + L.off_qs[r];
-    q[r].codes_bytes = L.qc[r]; q[r].scales_bytes = L.qs[r]; q[r].fmt = fmts[r]; q[r].role = r; q[r].block = MQ_BLOCK_TILE32;
+    q[r].codes_bytes = L.qc[r]; q[r].scales_bytes = L.qs[r]; q[r].fmt = fmts[r]; q[r].role = r; q[r].block = MQ_BLOCK_TILE32; q[r].tensor_scale = nullptr;
   }
   void* ws = L.ws ? base + L.off_ws : nullptr;
   if (!ok(cudaStreamWaitEvent(s, hp->ev[1], 0))) return MQ_ERR_CUDA;

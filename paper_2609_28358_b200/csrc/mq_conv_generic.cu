@@ -32,6 +32,26 @@ __device__ __forceinline__ void zero8(float* v) {
   for (int j = 0; j < 8; ++j) v[j] = 0.f;
 }
 
+// Scale of the 8 consecutive channels starting at channel c of row `row` at position `pos` of a stored tensor:
+//   activation-like tensors ([pos][row][c], R rows): sc[(pos * RB + row_block) * CB + channel_block]
+//   weights ([row][pos][c], P positions):            sc[(row_block * P + pos) * CB + channel_block]
+// with 32 x 32 tiles (E8M0), line blocks (one row per block) or, ts16, 16 x 16 blocks whose E4M3 scale is multiplied by the
+// tensor's fp32 scale t.
+__device__ __forceinline__ float e4m3_to_float(unsigned code) {
+  const __half_raw h = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)code, __NV_E4M3);
+  return __half2float(*reinterpret_cast<const __half*>(&h));
+}
+__device__ __forceinline__ float act_scale(const ConvArgs& a, const uint8_t* sc, float t, long long pos, int row, int c, int R, int Cp) {
+  if (a.ts16) return e4m3_to_float(sc[(pos * ((R + 15) >> 4) + (row >> 4)) * (Cp >> 4) + (c >> 4)]) * t;
+  if (a.line) return e8m0_to_float(sc[(pos * R + row) * (Cp >> 5) + (c >> 5)]);
+  return e8m0_to_float(sc[(pos * ((R + 31) >> 5) + (row >> 5)) * (Cp >> 5) + (c >> 5)]);
+}
+__device__ __forceinline__ float w_scale(const ConvArgs& a, const uint8_t* sc, float t, int row, int taps, int tap, int c, int Cp) {
+  if (a.ts16) return e4m3_to_float(sc[((long long)(row >> 4) * taps + tap) * (Cp >> 4) + (c >> 4)]) * t;
+  if (a.line) return e8m0_to_float(sc[((long long)row * taps + tap) * (Cp >> 5) + (c >> 5)]);
+  return e8m0_to_float(sc[((long long)(row >> 5) * taps + tap) * (Cp >> 5) + (c >> 5)]);
+}
+
 __device__ __forceinline__ void mma_tile(const Tiles& sm, int ty, int tx, float acc[4][4]) {
 #pragma unroll
   for (int k = 0; k < TK; ++k) {
@@ -63,6 +83,7 @@ __global__ void __launch_bounds__(GT) fwd_generic(ConvArgs a) {
   if (m_ok) { n = (int)(m % g.N); long long q = m / g.N; wo = (int)(q % g.Wo); ho = (int)(q / g.Wo); }
   const int co = n0 + row_l;
   const bool co_ok = co < g.Cout;
+  const float ta = a.ts16 ? *a.a_tscale : 1.f, tb = a.ts16 ? *a.b_tscale : 1.f;
 
   float acc[4][4] = {};
   for (int tap = 0; tap < taps; ++tap) {
@@ -73,11 +94,11 @@ __global__ void __launch_bounds__(GT) fwd_generic(ConvArgs a) {
     for (int kb = 0; kb < g.Ct; ++kb) {
       float va[8], vb[8];
       if (pix_ok) {
-        float s = e8m0_to_float(a.a_scales[(a.line ? pix * g.N + n : pix * g.Nt + (n >> 5)) * g.Ct + kb]);
+        const float s = act_scale(a, a.a_scales, ta, pix, n, kb * 32 + kq * 8, g.N, g.Cp);
         decode8<FX>(a.a_codes, (pix * g.N + n) * g.Cp + kb * 32 + kq * 8, s, va, a.fmt_a);
       } else zero8(va);
       if (co_ok) {
-        float s = e8m0_to_float(a.b_scales[((long long)(a.line ? co : (co >> 5)) * taps + tap) * g.Ct + kb]);
+        const float s = w_scale(a, a.b_scales, tb, co, taps, tap, kb * 32 + kq * 8, g.Cp);
         decode8<FW>(a.b_codes, ((long long)co * taps + tap) * g.Cp + kb * 32 + kq * 8, s, vb, a.fmt_b);
       } else zero8(vb);
       __syncthreads();
@@ -122,6 +143,7 @@ __global__ void __launch_bounds__(GT) bwd_data_generic(ConvArgs a) {
   if (m_ok) { n = (int)(m % g.N); long long q = m / g.N; w = (int)(q % g.W); h = (int)(q / g.W); }
   const int ci0 = n0 + nq * 8;
   const bool ci_ok = ci0 < g.Cp;
+  const float ta = a.ts16 ? *a.a_tscale : 1.f, tb = a.ts16 ? *a.b_tscale : 1.f;
 
   float acc[4][4] = {};
   for (int tap = 0; tap < taps; ++tap) {
@@ -134,12 +156,12 @@ __global__ void __launch_bounds__(GT) bwd_data_generic(ConvArgs a) {
     for (int kb = 0; kb < g.Cot; ++kb) {
       float va[8], vb[8];
       if (pix_ok) {
-        float s = e8m0_to_float(a.b_scales[(pix * g.Nt + (n >> 5)) * g.Cot + kb]);
+        const float s = act_scale(a, a.b_scales, tb, pix, n, kb * 32 + kq * 8, g.N, g.Cop);
         decode8<FG>(a.b_codes, (pix * g.N + n) * g.Cop + kb * 32 + kq * 8, s, va, a.fmt_b);
       } else zero8(va);
       const int co = kb * 32 + k_l;
       if (ci_ok && co < g.Cout) {
-        float s = e8m0_to_float(a.a_scales[((long long)kb * taps + tap) * g.Ct + (ci0 >> 5)]);
+        const float s = w_scale(a, a.a_scales, ta, co, taps, tap, ci0, g.Cp);
         decode8<FW>(a.a_codes, ((long long)co * taps + tap) * g.Cp + ci0, s, vb, a.fmt_a);
       } else zero8(vb);
       __syncthreads();
@@ -187,6 +209,7 @@ __global__ void __launch_bounds__(GT) bwd_weight_generic(ConvArgs a, int splits)
   const bool j_ok = j0 < J;
   const int tap = j_ok ? j0 / g.Cp : 0, ci0 = j_ok ? j0 - tap * g.Cp : 0;
   const int kh = tap / g.Kw, kw = tap - kh * g.Kw;
+  const float ta = a.ts16 ? *a.a_tscale : 1.f, tb = a.ts16 ? *a.b_tscale : 1.f;
 
   float acc[4][4] = {};
   for (int pix = pix_begin; pix < pix_end; ++pix) {
@@ -198,11 +221,11 @@ __global__ void __launch_bounds__(GT) bwd_weight_generic(ConvArgs a, int splits)
       const int n = kb * 32 + k_l;
       float va[8], vb[8];
       if (co_ok && n < g.N) {
-        float s = e8m0_to_float(a.b_scales[((long long)pix * g.Nt + kb) * g.Cot + (co0 >> 5)]);
+        const float s = act_scale(a, a.b_scales, tb, pix, n, co0, g.N, g.Cop);
         decode8<FG>(a.b_codes, ((long long)pix * g.N + n) * g.Cop + co0, s, va, a.fmt_b);
       } else zero8(va);
       if (x_ok && n < g.N) {
-        float s = e8m0_to_float(a.a_scales[(xpix * g.Nt + kb) * g.Ct + (ci0 >> 5)]);
+        const float s = act_scale(a, a.a_scales, ta, xpix, n, ci0, g.N, g.Cp);
         decode8<FX>(a.a_codes, (xpix * g.N + n) * g.Cp + ci0, s, vb, a.fmt_a);
       } else zero8(vb);
       __syncthreads();

@@ -70,11 +70,11 @@ __global__ void __launch_bounds__(IC_THREADS) im2col_kernel(Im2colArgs a, int rc
     }
   } else {
     // scales [ho][wo][nt][kh][kw][ct]; with line blocks one entry per sample: [ho][wo][n][kh][kw][ct]
-    const int Rt = a.line ? g.N : g.Nt;
-    const long long n_scales = (long long)g.Ho * g.Wo * Rt * taps * g.Ct;
+    const int Rt = a.line ? g.N : (a.ts16 ? (g.N + 15) / 16 : g.Nt), Cb = a.ts16 ? g.Cp / 16 : g.Ct;
+    const long long n_scales = (long long)g.Ho * g.Wo * Rt * taps * Cb;
     for (long long id = (long long)(blockIdx.x - n_main) * IC_THREADS + threadIdx.x; id < n_scales; id += (long long)(gridDim.x - n_main) * IC_THREADS) {
       long long q = id;
-      const int ct = (int)(q % g.Ct); q /= g.Ct;
+      const int ct = (int)(q % Cb); q /= Cb;
       const int tap = (int)(q % taps); q /= taps;
       const int nt = (int)(q % Rt); q /= Rt;
       const int wo = (int)(q % g.Wo);
@@ -82,7 +82,7 @@ __global__ void __launch_bounds__(IC_THREADS) im2col_kernel(Im2colArgs a, int rc
       const int kh = tap / g.Kw, kw = tap - kh * g.Kw;
       const int h = ho * g.sh + kh - g.ph, w = wo * g.sw + kw - g.pw;
       uint8_t sc = 0;
-      if (h >= 0 && h < g.H && w >= 0 && w < g.W) sc = a.scales[(((long long)h * g.W + w) * Rt + nt) * g.Ct + ct];
+      if (h >= 0 && h < g.H && w >= 0 && w < g.W) sc = a.scales[(((long long)h * g.W + w) * Rt + nt) * Cb + ct];
       a.out_scales[id] = sc;
     }
   }
@@ -108,16 +108,16 @@ __global__ void __launch_bounds__(IC_THREADS) im2col_generic_kernel(Im2colArgs a
       __stcs(reinterpret_cast<uint4*>(a.out_codes) + id, v);
     } else {
       long long q = id - code_chunks;
-      const int ct = (int)(q % g.Ct); q /= g.Ct;
+      const int Rt = a.line ? g.N : (a.ts16 ? (g.N + 15) / 16 : g.Nt), Cb = a.ts16 ? g.Cp / 16 : g.Ct;
+      const int ct = (int)(q % Cb); q /= Cb;
       const int tap = (int)(q % taps); q /= taps;
-      const int Rt = a.line ? g.N : g.Nt;
       const int nt = (int)(q % Rt); q /= Rt;
       const int wo = (int)(q % g.Wo);
       const int ho = (int)(q / g.Wo);
       const int kh = tap / g.Kw, kw = tap - kh * g.Kw;
       const int h = ho * g.sh + kh - g.ph, w = wo * g.sw + kw - g.pw;
       uint8_t sc = 0;
-      if (h >= 0 && h < g.H && w >= 0 && w < g.W) sc = a.scales[(((long long)h * g.W + w) * Rt + nt) * g.Ct + ct];
+      if (h >= 0 && h < g.H && w >= 0 && w < g.W) sc = a.scales[(((long long)h * g.W + w) * Rt + nt) * Cb + ct];
       a.out_scales[id - code_chunks] = sc;
     }
   }
@@ -135,7 +135,7 @@ cudaError_t launch_im2col(const Im2colArgs& a, cudaStream_t s) {
   if (PX > 8) PX = 8;
   if (PX < 1) PX = 1;
   const long long n_main = (((long long)g.Ho * g.Wo + PX - 1) / PX) * g.Nt;
-  const long long n_scales = (long long)g.Ho * g.Wo * (a.line ? g.N : g.Nt) * taps * g.Ct;
+  const long long n_scales = (long long)g.Ho * g.Wo * (a.line ? g.N : (a.ts16 ? (g.N + 15) / 16 : g.Nt)) * taps * (a.ts16 ? g.Cp / 16 : g.Ct);
   count_launches(1);
   if (J <= IC_MAX_J && src_chunks < 0x7fffffffLL && n_main < 0x7fff0000LL) {
     long long sc_blocks = (n_scales + IC_THREADS - 1) / IC_THREADS;

@@ -28,46 +28,6 @@ constexpr int QT_THREADS = 256;
 // a quarter-warp (rows 4 apart) hit 8 different 16-byte bank groups
 constexpr int QBUF_BYTES = 1024 * 32 + 256 * 16;
 
-// Stochastic Round(.) of Eq. 6 (Sec. III-A: the gradient's rounding).  x is the scaled element, idx its index in the
-// logical NCHW / OIHW tensor.  The element's draw is 32 bits of a counter-based generator keyed by (seed, idx);
-// u = (top 23 bits + 1/2) / 2^23.  With lo <= |x| < hi neighbours on the format's grid, the result is hi when
-// u < (|x| - lo) / (hi - lo), else lo -- returned as a float that lies on the grid, so the round-to-nearest
-// conversion that follows is exact.  Everything below is exact in fp32: |x| / step has at most 24 significant bits,
-// its fractional part and (23-bit draw + 1/2) likewise.  Magnitudes at or beyond the largest one are left to the
-// conversion's saturation.
-// lo: low word of the element's index; key: the stream key of its high word (sr_key)
-template <int FMT>
-__device__ __forceinline__ float sr_value(float x, unsigned lo, unsigned key) {
-  constexpr int M = (FMT == MQ_E4M3 || FMT == MQ_E2M3) ? 3 : (FMT == MQ_E2M1 ? 1 : 2);                      // mantissa bits
-  constexpr int EMIN = FMT == MQ_E4M3 ? -6 : (FMT == MQ_E5M2 ? -14 : (FMT == MQ_E3M2 ? -2 : 0));           // smallest normal exponent
-  // fp32 pattern of the largest magnitude: 448, 57344, 6, 28, 7.5
-  constexpr unsigned MAXBITS = FMT == MQ_E4M3 ? 0x43E00000u : (FMT == MQ_E5M2 ? 0x47600000u : (FMT == MQ_E2M1 ? 0x40C00000u : (FMT == MQ_E3M2 ? 0x41E00000u : 0x40F00000u)));
-  const unsigned b = __float_as_uint(x) & 0x7fffffffu;       // |x|; patterns of non-negative floats order like their values
-  const unsigned r23 = sr_mix32(lo ^ key) >> 9;
-  // normal range of the format: the grid keeps M mantissa bits of the fp32 pattern.  The dropped field f (23 - M bits)
-  // is the fraction of a step in units of 2^-(23 - M): f * 2^M > draw + 1/2 is an integer comparison, and stepping up
-  // is an integer addition on the pattern (the carry walks into the exponent at a binade's end).
-  constexpr unsigned MASK = (1u << (23 - M)) - 1u;
-  const unsigned f = b & MASK;
-  const unsigned q_norm = (b - f) + (((f << M) > r23) ? MASK + 1u : 0u);
-  // below it the step is the constant 2^(EMIN - M): t = |x| / step < 2^M, floor through a round-down addition of 2^23,
-  // draw + 1/2 as (2^23 + draw) - (2^23 - 1/2); all exact
-  const float t = __uint_as_float(b) * __uint_as_float((unsigned)(127 + M - EMIN) << 23);
-  const float fl = __fadd_rd(t, 8388608.f) - 8388608.f;
-  const float u = __uint_as_float(0x4B000000u | r23) - 8388607.5f;
-  const float up = (t - fl) * 8388608.f > u ? 1.f : 0.f;
-  const unsigned q_sub = __float_as_uint((fl + up) * __uint_as_float((unsigned)(127 + EMIN - M) << 23));
-  unsigned q = b >= ((unsigned)(127 + EMIN) << 23) ? q_norm : q_sub;
-  q = b < MAXBITS ? q : b;      // at or beyond the largest magnitude: left to the conversion's saturation
-  return __uint_as_float(q | (__float_as_uint(x) & 0x80000000u));
-}
-// Stream key of an element from the high word of its index; tensors below 2^32 elements (a.sr_wide == 0, uniform)
-// take the key computed on the host.
-__device__ __forceinline__ unsigned sr_key(const QuantArgs& a, long long idx) {
-  if (!a.sr_wide) return a.sr_key0;
-  return sr_mix32(a.sr_seed_lo ^ sr_mix32(a.sr_seed_hi ^ sr_mix32((unsigned)((unsigned long long)idx >> 32))));
-}
-
 __device__ __forceinline__ void cp_async16(void* dst, const void* src, bool valid) {
   const unsigned d = (unsigned)__cvta_generic_to_shared(dst);
   const int bytes = valid ? 16 : 0;   // 0 source bytes: the 16 destination bytes are zero-filled

@@ -16,7 +16,8 @@ ConvDesc = namedtuple("ConvDesc", "N C_in H W C_out Kh Kw stride_h stride_w pad_
 E4M3, E5M2, E2M1, E3M2, E2M3 = 0, 1, 2, 3, 4
 ROLE_X, ROLE_W, ROLE_DY = 0, 1, 2
 NCHW, HWNC = 0, 1
-TILE32, LINE32 = 0, 1      # block shape: 32 x 32 squares (default) / 1 x 32 lines along the channel axis
+TILE32, LINE32, TS16 = 0, 1, 2   # 32 x 32 squares (default) / 1 x 32 lines along the channel axis / the paper's own format: 16 x 16
+                                 # squares with an E4M3 block scale and an fp32 tensor scale (E2M1 elements)
 F32, BF16 = 0, 1
 OP_FWD, OP_BWD_DATA, OP_BWD_WEIGHT = 0, 1, 2
 OK = 0
@@ -42,7 +43,7 @@ class _Desc(ctypes.Structure):
 
 class _QTensor(ctypes.Structure):
     _fields_ = [("codes", ctypes.c_void_p), ("scales", ctypes.c_void_p), ("codes_bytes", ctypes.c_size_t),
-                ("scales_bytes", ctypes.c_size_t), ("fmt", ctypes.c_int), ("role", ctypes.c_int), ("block", ctypes.c_int)]
+                ("scales_bytes", ctypes.c_size_t), ("fmt", ctypes.c_int), ("role", ctypes.c_int), ("block", ctypes.c_int), ("tensor_scale", ctypes.c_void_p)]
 
 
 def lib():
@@ -81,11 +82,13 @@ def _stream(stream):
 class QTensor:
     """A stored MX tensor: device uint8 buffers for codes and tile scales."""
 
-    def __init__(self, codes, scales, fmt, role, block=TILE32):
+    def __init__(self, codes, scales, fmt, role, block=TILE32, tensor_scale=None):
         self.codes, self.scales, self.fmt, self.role, self.block = codes, scales, fmt, role, block
+        self.tensor_scale = tensor_scale      # TS16: two device floats (T_scale, max|X|)
 
     def _c(self):
-        return _QTensor(self.codes.data_ptr(), self.scales.data_ptr(), self.codes.numel(), self.scales.numel(), self.fmt, self.role, self.block)
+        return _QTensor(self.codes.data_ptr(), self.scales.data_ptr(), self.codes.numel(), self.scales.numel(), self.fmt, self.role, self.block,
+                        self.tensor_scale.data_ptr() if self.tensor_scale is not None else None)
 
 
 def _new(shape, dtype, device):
@@ -115,7 +118,8 @@ def workspace_size(desc, op, fmt_a, fmt_b, block=TILE32):
 
 def empty_qtensor(desc, role, fmt, device="cuda", block=TILE32):
     cb, sb = qtensor_sizes(desc, role, fmt, block)
-    return QTensor(_new(cb, torch.uint8, device), _new(sb, torch.uint8, device), fmt, role, block)
+    ts = _new(2, torch.float32, device) if block == TS16 else None
+    return QTensor(_new(cb, torch.uint8, device), _new(sb, torch.uint8, device), fmt, role, block, ts)
 
 
 _DTYPES = {torch.float32: F32, torch.bfloat16: BF16}
@@ -140,6 +144,21 @@ def quantize_sr(desc, role, fmt, src, seed, out=None, src_layout=NCHW, stream=No
     q = out._c()
     _check("mq_quantize_sr", lib().mq_quantize_sr(ctypes.byref(_d(desc)), ctypes.c_void_p(src.data_ptr()), _DTYPES[src.dtype], src_layout, ctypes.byref(q),
                                                  ctypes.c_uint64(int(seed) & 0xFFFFFFFFFFFFFFFF), _stream(stream)))
+    return out
+
+
+def quantize_ts(desc, role, src, out=None, src_layout=NCHW, amax_in=None, seed=None, stream=None):
+    """mq_quantize_ts: the paper's own format (fp32 tensor scale, E4M3 scale per 16 x 16 block, E2M1 elements).  amax_in: a
+    device float tensor holding the maximum Eq. 4 should use (e.g. an earlier tensor's tensor_scale[1:2]); None = this
+    tensor's own (two passes).  seed: stochastic rounding with that 64-bit seed."""
+    assert src.is_cuda and src.dtype in _DTYPES and src.is_contiguous()
+    if out is None:
+        out = empty_qtensor(desc, role, E2M1, src.device, TS16)
+    q = out._c()
+    sd = ctypes.c_uint64(int(seed) & 0xFFFFFFFFFFFFFFFF) if seed is not None else None
+    _check("mq_quantize_ts", lib().mq_quantize_ts(ctypes.byref(_d(desc)), ctypes.c_void_p(src.data_ptr()), _DTYPES[src.dtype], src_layout, ctypes.byref(q),
+                                                 ctypes.c_void_p(amax_in.data_ptr()) if amax_in is not None else None,
+                                                 ctypes.byref(sd) if sd is not None else None, _stream(stream)))
     return out
 
 

@@ -78,40 +78,40 @@ def test_bad_arguments_are_rejected_on_the_host(mq):
     assert L.mq_qtensor_sizes(ctypes.byref(big_k), 0, 0, 0, ctypes.byref(cb), ctypes.byref(sb)) == 1
     # entry points: null / misaligned / undersized buffers never reach a launch
     F32, BF16, NCHW = mq.F32, mq.BF16, mq.NCHW
-    q = mq._QTensor(None, None, 0, 0, 0, 0, 0)
+    q = mq._QTensor(None, None, 0, 0, 0, 0, 0, None)
     assert L.mq_quantize(ctypes.byref(good), None, F32, NCHW, ctypes.byref(q), None) == 1
-    q = mq._QTensor(0x1000, 0x2000, 16, 16, 0, 0, 0)
+    q = mq._QTensor(0x1000, 0x2000, 16, 16, 0, 0, 0, None)
     assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), F32, NCHW, ctypes.byref(q), None) == 4  # too small
-    q = mq._QTensor(0x1008, 0x2000, 1 << 30, 1 << 30, 0, 0, 0)
+    q = mq._QTensor(0x1008, 0x2000, 1 << 30, 1 << 30, 0, 0, 0, None)
     assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), F32, NCHW, ctypes.byref(q), None) == 3  # alignment
-    q = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 0, 0)
+    q = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 0, 0, None)
     assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), F32, 7, ctypes.byref(q), None) == 1  # no such source layout
     assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), 9, NCHW, ctypes.byref(q), None) == 1  # no such element type
     assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), BF16, NCHW, ctypes.byref(q), None) == 2  # bf16 source: not in this build
-    qbad = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 0, 3)
+    qbad = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 0, 3, None)
     assert L.mq_quantize(ctypes.byref(good), ctypes.c_void_p(0x3000), F32, NCHW, ctypes.byref(qbad), None) == 1  # no such block shape
     # the stochastic-rounding entry point validates the same way (the seed is any 64-bit value)
     seed = ctypes.c_uint64(0xFFFFFFFFFFFFFFFF)
     assert L.mq_quantize_sr(ctypes.byref(good), None, F32, NCHW, ctypes.byref(q), seed, None) == 1
     assert L.mq_quantize_sr(ctypes.byref(good), ctypes.c_void_p(0x3000), F32, 7, ctypes.byref(q), seed, None) == 1
     assert L.mq_quantize_sr(ctypes.byref(good), ctypes.c_void_p(0x3004), F32, NCHW, ctypes.byref(q), seed, None) == 3
-    small = mq._QTensor(0x1000, 0x2000, 16, 16, 0, 2, 0)
+    small = mq._QTensor(0x1000, 0x2000, 16, 16, 0, 2, 0, None)
     assert L.mq_quantize_sr(ctypes.byref(good), ctypes.c_void_p(0x3000), F32, NCHW, ctypes.byref(small), seed, None) == 4
     assert L.mq_cbf_im2col(ctypes.byref(good), ctypes.byref(q), None, None, None) == 1
-    qw = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 1, 0)
+    qw = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 1, 0, None)
     out = ctypes.c_void_p(0x4000)
     assert L.mq_conv_fwd(ctypes.byref(good), ctypes.byref(qw), ctypes.byref(qw), out, F32, NCHW, None, 0, None) == 1  # wrong role
     assert L.mq_conv_fwd(ctypes.byref(good), ctypes.byref(q), ctypes.byref(qw), out, F32, 5, None, 0, None) == 1  # layout
     assert L.mq_conv_fwd(ctypes.byref(good), ctypes.byref(q), ctypes.byref(qw), out, 9, NCHW, None, 0, None) == 1  # element type
     assert L.mq_conv_fwd(ctypes.byref(good), ctypes.byref(q), ctypes.byref(qw), out, BF16, NCHW, None, 0, None) == 2  # bf16 output: not in this build
     need = mq.workspace_size(inputs.conv_desc(8, 32, 8, 8, 32, 3), mq.OP_BWD_WEIGHT, 0, 0)
-    qg = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 2, 0)
+    qg = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 2, 0, None)
     if need:
         assert L.mq_conv_bwd_weight(ctypes.byref(good), ctypes.byref(q), ctypes.byref(qg), out, F32, NCHW, None, 0, None) == 4
     # line blocks: accepted by the forward GEMM only; operands must agree on the block shape
-    ql = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 0, 1)
-    qwl = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 1, 1)
-    qgl = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 2, 1)
+    ql = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 0, 1, None)
+    qwl = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 1, 1, None)
+    qgl = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, 0, 2, 1, None)
     assert L.mq_conv_fwd(ctypes.byref(good), ctypes.byref(ql), ctypes.byref(qw), out, F32, NCHW, None, 0, None) == 2  # mixed block shapes
     assert L.mq_conv_bwd_data(ctypes.byref(good), ctypes.byref(qwl), ctypes.byref(qgl), out, F32, NCHW, None, 0, None) == 2
     assert L.mq_conv_bwd_weight(ctypes.byref(good), ctypes.byref(ql), ctypes.byref(qgl), out, F32, NCHW, None, 0, None) == 2
