@@ -48,6 +48,11 @@ CALLS = ("quantize_x", "quantize_w", "quantize_dy", "cbf_im2col", "conv_fwd", "c
 # of the captured one, traffic being proportional to the units processed).
 NCU_TRAFFIC = {
     # (bench workload, call): (captured workload, bytes per launch there, scale)
+    ("cfg5_e4m3_k3s1_c512_hw56", "conv_fwd"): ("cfg5_e4m3_k3s1_c512_hw28", 119497984 + 357722112, 4.0),       # conv_tc_kernel<fwd>
+    ("cfg5_e4m3_k3s1_c512_hw56", "conv_bwd_data"): ("cfg5_e4m3_k3s1_c512_hw28", 119599104 + 359816192, 4.0),  # conv_tc_kernel<bwd_data>
+    ("cfg5_e4m3_k3s1_c512_hw56", "quantize_x"): ("cfg5_e4m3_k3s1_c512_hw28", 420059648 + 81590016, 4.0),      # quantize_tma_kernel
+    ("cfg5_e4m3_k3s1_c512_hw56", "quantize_dy"): ("cfg5_e4m3_k3s1_c512_hw28", 423871488 + 81877248, 4.0),
+    ("cfg5_e4m3_k3s1_c512_hw28", "conv_fwd"): ("cfg5_e4m3_k3s1_c512_hw28", 119497984 + 357722112, 1.0),
 }
 
 
@@ -130,7 +135,7 @@ class ClockSampler(threading.Thread):
 class Workload:
     """Device buffers and the seven calls of one layer step."""
 
-    def __init__(self, name, layer, rank, dy_rounding="nearest"):
+    def __init__(self, name, layer, rank, dy_rounding="nearest", fp32_layout="nchw"):
         import torch
 
         from paper_2609_28358_b200 import mq
@@ -142,26 +147,30 @@ class Workload:
         seed = layer.seed + 1000 * rank
         self.host = (inputs.make_x(d, seed, layer.x_kind), inputs.make_w(d, layer.seed, layer.w_kind), inputs.make_dy(d, seed, layer.dy_kind))
         src = self.src = [torch.from_numpy(t).cuda() for t in self.host]
+        hwnc = fp32_layout == "hwnc"     # fp32 tensors in the channel-fastest order the convolution calls can emit when layers chain
+        sl = ol = mq.HWNC if hwnc else mq.NCHW
+        if hwnc:
+            src = self.src = [src[0].permute(2, 3, 0, 1).contiguous(), src[1].permute(0, 2, 3, 1).contiguous(), src[2].permute(2, 3, 0, 1).contiguous()]
         q = self.q = [mq.empty_qtensor(d, r, f) for r, f in zip(roles, fmts)]
         self.icb, self.isb = mq.im2col_sizes(d, fmts[0])
         ic = torch.empty(self.icb, dtype=torch.uint8, device="cuda")
         isc = torch.empty(self.isb, dtype=torch.uint8, device="cuda")
         ho, wo = inputs.out_hw(d)
-        self.y = y = torch.empty((d.N, d.C_out, ho, wo), dtype=torch.float32, device="cuda")
-        self.dx = dx = torch.empty((d.N, d.C_in, d.H, d.W), dtype=torch.float32, device="cuda")
-        self.dw = dw = torch.empty((d.C_out, d.C_in, d.Kh, d.Kw), dtype=torch.float32, device="cuda")
+        self.y = y = torch.empty((ho, wo, d.N, d.C_out) if hwnc else (d.N, d.C_out, ho, wo), dtype=torch.float32, device="cuda")
+        self.dx = dx = torch.empty((d.H, d.W, d.N, d.C_in) if hwnc else (d.N, d.C_in, d.H, d.W), dtype=torch.float32, device="cuda")
+        self.dw = dw = torch.empty((d.C_out, d.Kh, d.Kw, d.C_in) if hwnc else (d.C_out, d.C_in, d.Kh, d.Kw), dtype=torch.float32, device="cuda")
         ws_bytes = max(mq.workspace_size(d, op, a, b) for op, a, b in
                        ((mq.OP_FWD, fmts[0], fmts[1]), (mq.OP_BWD_DATA, fmts[1], fmts[2]), (mq.OP_BWD_WEIGHT, fmts[0], fmts[2])))
         self.ws = ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device="cuda")
         self.calls = [
-            ("quantize_x", lambda: mq.quantize(d, roles[0], fmts[0], src[0], out=q[0])),
-            ("quantize_w", lambda: mq.quantize(d, roles[1], fmts[1], src[1], out=q[1])),
-            ("quantize_dy", (lambda: mq.quantize_sr(d, roles[2], fmts[2], src[2], 1234, out=q[2])) if dy_rounding == "stochastic" else
-             (lambda: mq.quantize(d, roles[2], fmts[2], src[2], out=q[2]))),
+            ("quantize_x", lambda: mq.quantize(d, roles[0], fmts[0], src[0], out=q[0], src_layout=sl)),
+            ("quantize_w", lambda: mq.quantize(d, roles[1], fmts[1], src[1], out=q[1], src_layout=sl)),
+            ("quantize_dy", (lambda: mq.quantize_sr(d, roles[2], fmts[2], src[2], 1234, out=q[2], src_layout=sl)) if dy_rounding == "stochastic" else
+             (lambda: mq.quantize(d, roles[2], fmts[2], src[2], out=q[2], src_layout=sl))),
             ("cbf_im2col", lambda: mq.cbf_im2col(d, q[0], ic, isc)),
-            ("conv_fwd", lambda: mq.conv_fwd(d, q[0], q[1], y=y, workspace=ws)),
-            ("conv_bwd_data", lambda: mq.conv_bwd_data(d, q[1], q[2], dx=dx, workspace=ws)),
-            ("conv_bwd_weight", lambda: mq.conv_bwd_weight(d, q[0], q[2], dw=dw, workspace=ws)),
+            ("conv_fwd", lambda: mq.conv_fwd(d, q[0], q[1], y=y, layout=ol, workspace=ws)),
+            ("conv_bwd_data", lambda: mq.conv_bwd_data(d, q[1], q[2], dx=dx, layout=ol, workspace=ws)),
+            ("conv_bwd_weight", lambda: mq.conv_bwd_weight(d, q[0], q[2], dw=dw, layout=ol, workspace=ws)),
         ]
 
     def step(self):
@@ -262,7 +271,7 @@ def run_ours(args):
     mq.lib()  # fail loudly if the CUDA library is missing
 
     all_wl = workloads()
-    wl = Workload(args.workload, all_wl[args.workload], rank, args.dy_rounding)
+    wl = Workload(args.workload, all_wl[args.workload], rank, args.dy_rounding, args.fp32_layout)
     d, fmts = wl.d, wl.fmts
     flush = torch.empty(512 << 20, dtype=torch.uint8, device="cuda")  # > 126 MB L2
 
@@ -346,7 +355,7 @@ def run_ours(args):
         "value": value, "unit": "TFLOPS", "n_gpus": world, "steps": K, "warmup": max(args.warmup, 3), "ms_per_step": ms_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "+".join(FMT_NAME[f] for f in fmts) + " (fp32 accumulate)", "data": "synthetic",
-        "config": {"workload": args.workload, "layer": dict(d._asdict()), "formats": [FMT_NAME[f] for f in fmts], "dy_rounding": args.dy_rounding,
+        "config": {"workload": args.workload, "layer": dict(d._asdict()), "formats": [FMT_NAME[f] for f in fmts], "dy_rounding": args.dy_rounding, "fp32_layout": args.fp32_layout,
                    "global_batch": d.N * world, "parallelism": "dp%d" % world if world > 1 else "single", "l2": "flushed between steps (512 MiB write)"},
         "clocks": clocks,
         "e2e": {"value": flops / (e2e_ms * 1e-3) / 1e12, "unit": "TFLOPS", "ms_per_step": e2e_ms,
@@ -366,7 +375,7 @@ def run_ours(args):
         out["more_workloads"] = {}
         Km = max(3, min(K, 20))
         for name in more:
-            w2 = Workload(name, all_wl[name], rank, args.dy_rounding)
+            w2 = Workload(name, all_wl[name], rank, args.dy_rounding, args.fp32_layout)
             for _ in range(3):
                 w2.step()
             torch.cuda.synchronize()
@@ -548,6 +557,8 @@ def main():
     ap.add_argument("--no-accounting", action="store_true", help="skip the measured Table-I style quantization accounting")
     ap.add_argument("--dy-rounding", default="nearest", choices=["nearest", "stochastic"],
                     help="rounding of the gradient's quantizer in the device-timed step (the host-buffer call keeps nearest)")
+    ap.add_argument("--fp32-layout", default="nchw", choices=["nchw", "hwnc"],
+                    help="order of the fp32 tensors in the device-timed step: NCHW / OIHW (the layout of record) or channel-fastest [H][W][N][C] / [Cout][Kh][Kw][Cin]")
     ap.add_argument("--cpu-budget", type=float, default=15.0)
     args = ap.parse_args()
     if args.impl == "reference":
