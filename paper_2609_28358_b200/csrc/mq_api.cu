@@ -174,6 +174,10 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   // the epilogue no longer overlaps the next tile: worth it for 8-bit layers whose main loop is long (measured: +30 %
   // at 2304+ bytes of K per row)
   if (!fp4 && p.Cd >= 256 && (double)taps * rowbytes >= 2048.0 && (op == MQ_OP_FWD || (g.sh == 1 && g.sw == 1))) p.BN = 256;
+  // 1x1 layers: the activation tile is the whole of a tile's loads, so halving its re-reads pays although the main loop is short
+  // (measured, N = 256, 8-bit, fp32 / quantized output: 256 channels 56x56 324 -> 207 us / 217 -> 196 us; 512 channels 56x56
+  // 531 -> 528 / 464 -> 410 us; 512 channels 28x28 181 -> 175 / 133 -> 127 us)
+  if (!fp4 && p.Cd >= 256 && taps == 1 && g.sh == 1 && g.sw == 1 && !env_int("MQ_TC_1X1_BN128", 0)) p.BN = 256;
   // E2M1: the same trade (measured with the tile widths chosen below: 256 channels 28x28 -13 %, 512 channels 14x14 -6 %,
   // 56x56 -10 %)
   const double act_bytes = (double)p.Hs * p.Ws * g.N * rowbytes;

@@ -127,6 +127,10 @@ __device__ __forceinline__ int tap_index(const TapWalk<MODE>& w, const ChunkPos&
 
 // An epilogue warp hands its accumulator back: to this block's barrier, or (a pair of blocks: the peer's warps) to the
 // leader's, whose MMA warp waits for the epilogues of both blocks.
+// Accumulator buffer of a block's tcount-th tile and the parity of that buffer's barriers (1 or 2 buffers; a third
+// buffer of 128 columns was measured on stride-2 and 1x1 layers: no change)
+__device__ __forceinline__ int acc_index(const ConvTcParams& p, uint32_t tcount) { return (int)(tcount & (uint32_t)(p.n_acc - 1)); }
+__device__ __forceinline__ uint32_t acc_phase(const ConvTcParams& p, uint32_t tcount) { return (tcount >> (p.n_acc - 1)) & 1u; }
 __device__ __forceinline__ void release_acc(uint64_t* bar, int leader_remote) {
   if (leader_remote) mbar_arrive_remote(bar, 0); else mbar_arrive(bar);
 }
@@ -149,9 +153,9 @@ __device__ __forceinline__ void epilogue_role(const ConvTcParams& p, uint32_t tm
       TapWalk<MODE> tw;
       tw.init(p, tile);
       const int Q = tw.chunks(p);
-      const int acc = (int)(tcount & (uint32_t)(p.n_acc - 1));
+      const int acc = acc_index(p, tcount);
       bool ok = true;
-      if (lane == 0) ok = mbar_wait(&tfull[acc], (tcount >> (p.n_acc - 1)) & 1, p.status, MQ_ERR_TIMEOUT);
+      if (lane == 0) ok = mbar_wait(&tfull[acc], acc_phase(p, tcount), p.status, MQ_ERR_TIMEOUT);
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) { *abort_flag = 1; break; }
       tc_fence_after_sync();
@@ -300,7 +304,11 @@ __device__ __forceinline__ void mx_encode_row(const float* x, float f, uint8_t* 
     *reinterpret_cast<uint4*>(dst + 16) = make_uint4(w[4], w[5], w[6], w[7]);
   }
 }
-template <int MODE>
+// FMT: element format of the emitted tensor.  The role is compiled into kernel instances of its own (conv_tc_kernel's EPI
+// parameter), one per format, and the activation is chosen outside the element loops: a format switch per block inside
+// one kernel measured 602 us on a 1x1 layer (N = 256, 512 channels, 56 x 56) against 461 us for a single-format kernel, and
+// a non-inlined role per format 785 us.
+template <int MODE, int FMT>
 __device__ __forceinline__ void epilogue_mx_role(const ConvTcParams& p, unsigned* red, uint32_t tmem, uint64_t* tfull, uint64_t* tempty,
                                                  volatile int* abort_flag, int warp, int lane, unsigned total) {
     const int quad = warp & 3;
@@ -310,8 +318,8 @@ __device__ __forceinline__ void epilogue_mx_role(const ConvTcParams& p, unsigned
     const int nblk = p.BN >> 5;                         // 32-channel blocks of a tile
     const int bbeg = half == 0 ? 0 : (nblk + 1) >> 1, bend = half == 0 ? (nblk + 1) >> 1 : nblk;
     const int grp0 = quad & ~(p.TW - 1);                // first quadrant of the TW quadrants that hold this sample tile
-    const int emax = fmt_emax(p.mx_fmt);
-    const int bpe4 = p.mx_fmt == MQ_E2M1 ? 1 : 2;       // bytes per element x 2
+    constexpr int emax = FMT == MQ_E4M3 ? 8 : (FMT == MQ_E5M2 ? 15 : (FMT == MQ_E3M2 ? 4 : 2));
+    constexpr int bpe4 = FMT == MQ_E2M1 ? 1 : 2;        // bytes per element x 2
     const int Ct = p.mx_Cp >> 5;
     unsigned* my_red = red + half * 32;                 // [parity][quadrant][column]
     uint32_t tcount = 0;
@@ -320,9 +328,9 @@ __device__ __forceinline__ void epilogue_mx_role(const ConvTcParams& p, unsigned
       TapWalk<MODE> tw;
       tw.init(p, tile);
       const int Q = tw.chunks(p);
-      const int acc = (int)(tcount & (uint32_t)(p.n_acc - 1));
+      const int acc = acc_index(p, tcount);
       bool ok = true;
-      if (lane == 0) ok = !*abort_flag && mbar_wait(&tfull[acc], (tcount >> (p.n_acc - 1)) & 1, p.status, MQ_ERR_TIMEOUT);
+      if (lane == 0) ok = !*abort_flag && mbar_wait(&tfull[acc], acc_phase(p, tcount), p.status, MQ_ERR_TIMEOUT);
       // the four warps of a half leave together or not at all: they meet at barriers inside the tile
       if (half_any(half, !ok)) { *abort_flag = 1; break; }
       tc_fence_after_sync();
@@ -338,16 +346,33 @@ __device__ __forceinline__ void epilogue_mx_role(const ConvTcParams& p, unsigned
       const long long pix = (long long)yo * p.Wd + xo;
       uint8_t* o_codes = p.mx_codes + (((pix * p.N + n) * p.mx_Cp + tile.c0) * bpe4 >> 1);
       uint8_t* o_scale = p.mx_scales + (pix * p.Nt + (n >> 5)) * Ct + (tile.c0 >> 5);
+      // the TMEM load of block b + 1 is in flight while block b is reduced, converted and stored
+      uint32_t v[32];
+      if (Q > 0 && bbeg < bend) {
+        tmem_ld_32x32b_x16(taddr + 32 * bbeg, v);
+        tmem_ld_32x32b_x16(taddr + 32 * bbeg + 16, v + 16);
+      }
 #pragma unroll 1
       for (int b = bbeg; b < bend; ++b) {
         float x[32];
+        float m = 0.f;
         if (Q > 0) {
-          uint32_t v[32];
-          tmem_ld_32x32b_x16(taddr + 32 * b, v);
-          tmem_ld_32x32b_x16(taddr + 32 * b + 16, v + 16);
           tmem_ld_wait();
+          // the activation is chosen outside the element loop: three straight-line copies instead of a test per element
+          if (p.mx_act == MQ_ACT_RELU) {
 #pragma unroll
-          for (int k = 0; k < 32; ++k) x[k] = __uint_as_float(v[k]);
+            for (int k = 0; k < 32; ++k) { x[k] = fmaxf(__uint_as_float(v[k]), 0.f); m = fmaxf(m, x[k]); }
+          } else if (p.mx_act == MQ_ACT_SILU) {
+#pragma unroll
+            for (int k = 0; k < 32; ++k) { x[k] = mx_activation(__uint_as_float(v[k]), MQ_ACT_SILU); m = fmaxf(m, fabsf(x[k])); }
+          } else {
+#pragma unroll
+            for (int k = 0; k < 32; ++k) { x[k] = __uint_as_float(v[k]); m = fmaxf(m, fabsf(x[k])); }
+          }
+          if (b + 1 < bend) {
+            tmem_ld_32x32b_x16(taddr + 32 * (b + 1), v);
+            tmem_ld_32x32b_x16(taddr + 32 * (b + 1) + 16, v + 16);
+          }
         } else {
 #pragma unroll
           for (int k = 0; k < 32; ++k) x[k] = 0.f;
@@ -356,13 +381,6 @@ __device__ __forceinline__ void epilogue_mx_role(const ConvTcParams& p, unsigned
           tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) mbar_arrive(&tempty[acc]);
-        }
-        float m = 0.f;
-#pragma unroll
-        for (int k = 0; k < 32; ++k) {
-          const float y = mx_activation(x[k], p.mx_act);
-          x[k] = y;
-          m = fmaxf(m, fabsf(y));
         }
         unsigned mb = row_ok ? __float_as_uint(m) : 0u;
         for (int off = p.TW; off < 32; off <<= 1) mb = max(mb, __shfl_xor_sync(0xffffffffu, mb, off));
@@ -376,13 +394,7 @@ __device__ __forceinline__ void epilogue_mx_role(const ConvTcParams& p, unsigned
         if (row_ok && tile.c0 + 32 * b < p.mx_Cp) {
           const float f = scale_factor(code);
           uint8_t* dst = o_codes + ((32 * b * bpe4) >> 1);
-          switch (p.mx_fmt) {
-            case MQ_E4M3: mx_encode_row<MQ_E4M3>(x, f, dst); break;
-            case MQ_E5M2: mx_encode_row<MQ_E5M2>(x, f, dst); break;
-            case MQ_E2M1: mx_encode_row<MQ_E2M1>(x, f, dst); break;
-            case MQ_E3M2: mx_encode_row<MQ_E3M2>(x, f, dst); break;
-            default: mx_encode_row<MQ_E2M3>(x, f, dst); break;
-          }
+          mx_encode_row<FMT>(x, f, dst);
         }
       }
       if (bbeg >= bend) {      // a tile of 32 channels leaves the second half without a block
@@ -418,9 +430,9 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
       TapWalk<MODE> tw;
       tw.init(p, tile);
       const int Q = tw.chunks(p);
-      const int acc = (int)(tcount & (uint32_t)(p.n_acc - 1));
+      const int acc = acc_index(p, tcount);
       bool ok = true;
-      if (lane == 0) ok = mbar_wait(&tfull[acc], (tcount >> (p.n_acc - 1)) & 1, p.status, MQ_ERR_TIMEOUT);
+      if (lane == 0) ok = mbar_wait(&tfull[acc], acc_phase(p, tcount), p.status, MQ_ERR_TIMEOUT);
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) { *abort_flag = 1; break; }
       tc_fence_after_sync();
@@ -480,7 +492,9 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
     if (lane == 0) bulk_wait_group_all();
 }
 
-template <int MODE, int KB, bool FP4>
+// EPI: -1 = fp32 output (the three fp32 epilogue roles, chosen at run time: an instance per role was measured, no
+// change); 0..4 = quantizing epilogue emitting element format EPI
+template <int MODE, int KB, bool FP4, int EPI = -1>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_out,
                const ConvTcParams p) {
@@ -620,8 +634,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         TapWalk<MODE> tw;
         tw.init(p, tile);
         const int Q = tw.chunks(p);
-        const int acc = (int)(tcount & (uint32_t)(p.n_acc - 1));
-        if (!mbar_wait(&tempty[acc], ((tcount >> (p.n_acc - 1)) & 1) ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+        const int acc = acc_index(p, tcount);
+        if (!mbar_wait(&tempty[acc], acc_phase(p, tcount) ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem + acc * p.BN;
         uint32_t accumulate = 0;
@@ -705,7 +719,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else if (warp >= 4 && warp < 12) {
-    if (p.mx_out) epilogue_mx_role<MODE>(p, mx_red, tmem, tfull, tempty, abort_flag, warp, lane, total);
+    if (EPI >= 0) epilogue_mx_role<MODE, EPI < 0 ? 0 : EPI>(p, mx_red, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else if (p.pair) epilogue_pair_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else if (p.tma_store) epilogue_tma_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
@@ -1349,12 +1363,12 @@ size_t conv_tc_smem_bytes(const ConvTcParams& p) {
   return 1024 + (size_t)p.stages * stage + (p.tma_store ? EPI_STAGING_BYTES : 0) + (3 * (size_t)p.stages + 4) * 8 + 64 + (p.mx_out ? 288 : 0);
 }
 
-template <int MODE, int KB, bool FP4>
+template <int MODE, int KB, bool FP4, int EPI = -1>
 cudaError_t launch_conv_tc_inst(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_out, cudaStream_t s) {
   static bool attr_set = false;
   const size_t smem = conv_tc_smem_bytes(p);
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(conv_tc_kernel<MODE, KB, FP4>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(conv_tc_kernel<MODE, KB, FP4, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
@@ -1362,7 +1376,7 @@ cudaError_t launch_conv_tc_inst(const ConvTcParams& p, const CUtensorMap& map_a,
   const long long units = p.pair ? p.total_tiles / 2 : p.total_tiles;
   const unsigned grid = (unsigned)(units < sms ? units : sms);
   count_launches(1);
-  return launch_pdl(conv_tc_kernel<MODE, KB, FP4>, dim3(grid), dim3(TC_THREADS), smem, s, map_a, map_b, map_out, p);
+  return launch_pdl(conv_tc_kernel<MODE, KB, FP4, EPI>, dim3(grid), dim3(TC_THREADS), smem, s, map_a, map_b, map_out, p);
 }
 
 size_t conv_tc_sfa_bytes(const ConvTcParams& p) {
@@ -1511,6 +1525,17 @@ cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, cons
     MQ_TC_HCASE(MQ_OP_FWD, 64, false); MQ_TC_HCASE(MQ_OP_FWD, 32, false); MQ_TC_HCASE(MQ_OP_FWD, 64, true); MQ_TC_HCASE(MQ_OP_FWD, 32, true);
     MQ_TC_HCASE(MQ_OP_BWD_DATA, 64, false); MQ_TC_HCASE(MQ_OP_BWD_DATA, 32, false); MQ_TC_HCASE(MQ_OP_BWD_DATA, 64, true); MQ_TC_HCASE(MQ_OP_BWD_DATA, 32, true);
 #undef MQ_TC_HCASE
+    return cudaErrorInvalidValue;
+  }
+  if (p.mx_out) {   // the quantizing epilogue: one kernel instance per emitted format
+#define MQ_TC_MX(M, K, F, E) if (p.mode == M && p.KB == K && (p.kind_fp4 != 0) == F && p.mx_fmt == E) return launch_conv_tc_inst<M, K, F, E>(p, map_a, map_w, map_out, s)
+#define MQ_TC_MX5(M, K, F) MQ_TC_MX(M, K, F, MQ_E4M3); MQ_TC_MX(M, K, F, MQ_E5M2); MQ_TC_MX(M, K, F, MQ_E2M1); MQ_TC_MX(M, K, F, MQ_E3M2); MQ_TC_MX(M, K, F, MQ_E2M3)
+    MQ_TC_MX5(MQ_OP_FWD, 128, false); MQ_TC_MX5(MQ_OP_FWD, 64, false); MQ_TC_MX5(MQ_OP_FWD, 32, false);
+    MQ_TC_MX5(MQ_OP_FWD, 128, true);  MQ_TC_MX5(MQ_OP_FWD, 64, true);  MQ_TC_MX5(MQ_OP_FWD, 32, true);
+    MQ_TC_MX5(MQ_OP_BWD_DATA, 128, false); MQ_TC_MX5(MQ_OP_BWD_DATA, 64, false); MQ_TC_MX5(MQ_OP_BWD_DATA, 32, false);
+    MQ_TC_MX5(MQ_OP_BWD_DATA, 128, true);  MQ_TC_MX5(MQ_OP_BWD_DATA, 64, true);  MQ_TC_MX5(MQ_OP_BWD_DATA, 32, true);
+#undef MQ_TC_MX5
+#undef MQ_TC_MX
     return cudaErrorInvalidValue;
   }
 #define MQ_TC_CASE(M, K, F) if (p.mode == M && p.KB == K && (p.kind_fp4 != 0) == F) return launch_conv_tc_inst<M, K, F>(p, map_a, map_w, map_out, s)
