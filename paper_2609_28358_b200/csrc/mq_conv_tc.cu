@@ -274,40 +274,130 @@ __device__ __forceinline__ void epilogue_pair_role(const ConvTcParams& p, uint32
 // output columns x 128 / TW >= 32 samples, so a quantization tile (one pixel, 32 samples, 32 channels) lies inside one
 // GEMM tile: its 32 samples sit in TW consecutive TMEM lane quadrants (8, 16 or 32 lanes each), its channels in 32
 // accumulator columns.  Per 32-channel block a warp loads its 32 x 32 values, applies the activation, takes the
-// per-lane maximum, reduces it over the lanes of the same output column (shuffles), and the TW warps of a tile
-// combine their maxima through shared memory (one named barrier per block among the four warps of a column half);
-// scale and codes then follow exactly the quantizer's arithmetic.  A lane writes its row's 32 codes as one or two
-// 16-byte stores (a row of the emitted tensor is channel-contiguous), and the accumulator goes back to the MMA warp right
-// after the warp's last TMEM load.
-// Measured and dropped (N = 256, 512 channels, 56 x 56, E4M3; this version: 3x3 1611 us, 1x1 654 us): staging the codes
-// in shared memory so that four lanes cover a row's 64-byte run (8 store requests per instruction instead of 32): 1660 /
-// 704 us - the stores are not what the epilogue waits for; two passes over the columns (all maxima first, one barrier
-// per tile instead of one per block), which read tensor memory twice and return the accumulator late: 1804 / 904 us.
+// per-lane maximum and reduces it over the lanes of the same output column (one integer warp reduction).  With
+// one-column tiles (the host's choice whenever the batch fills them) a warp's 32 rows ARE a sample tile and that is
+// the tile's maximum; with 2 or 4 columns the TW warps of a tile combine their maxima through shared memory (one
+// named barrier per block among the four warps of a column half).  Scale and codes then follow exactly the
+// quantizer's arithmetic.  A lane writes its row's 32 codes as two stores (a row of the emitted tensor is
+// channel-contiguous), and the accumulator goes back to the MMA warp right after the warp's last TMEM load.
+// Measured (N = 256, 512 channels, 56 x 56, 1x1, E4M3 -> E4M3 with ReLU, us): one kernel for all formats with a switch per
+// block 602; an instance per format 461 (a non-inlined role per format: 785); 256-channel tiles 410; one-column tiles
+// 368, without the exchange 323.  Fewer ALU instructions (three-input maxima, ReLU by clearing negative codes after
+// packing instead of a maximum per element) or the warp reduction left out: no change - a block takes about 1100
+// cycles of its warp for some 150 instructions, i.e. the epilogue waits on latencies (TMEM load, reduction,
+// conversion chains) that two warps per scheduler cannot hide, and a second register buffer to overlap two blocks
+// does not fit in 128 registers (spills: 538).  Dropped earlier: staging the codes in shared memory for 64-byte
+// store runs (slower: the stores are not what the epilogue waits for); two passes over the columns (all maxima
+// first, one barrier per tile), which read tensor memory twice and return the accumulator late (slower).
 __device__ __forceinline__ void half_sync(int half) { asm volatile("bar.sync %0, 128;" ::"r"(2 + half) : "memory"); }
 __device__ __forceinline__ bool half_any(int half, bool pred) {
   int r;
   asm volatile("{\n\t.reg .pred p, q;\n\tsetp.ne.b32 p, %2, 0;\n\tbar.red.or.pred q, %1, 128, p;\n\tselp.b32 %0, 1, 0, q;\n\t}\n" : "=r"(r) : "r"(2 + half), "r"(pred ? 1 : 0) : "memory");
   return r != 0;
 }
-template <int FMT>
-__device__ __forceinline__ void mx_encode_row(const float* x, float f, uint8_t* dst) {
-  unsigned w[8];
+__device__ __forceinline__ float fmax3(float a, float b, float c) {
+  float r;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+  return r;
+}
+// 16 values of a row x f -> 16 codes, stored as one 16-byte (E2M1: 8-byte) word.  RELU: the codes of negative values
+// are cleared afterwards, four (E2M1: eight) codes per 32-bit operation - quantize(max(x, 0)) = quantize(x) with the
+// negative codes set to zero, and the clearing costs a fifth of a maximum per element.
+template <int FMT, bool RELU>
+__device__ __forceinline__ void mx_encode_half(const uint32_t* v, float f, uint8_t* dst) {
+  unsigned w[4];
 #pragma unroll
-  for (int k = 0; k < 32; k += 4) {
-    const unsigned lo = encode2<FMT>(x[k] * f, x[k + 1] * f), hi = encode2<FMT>(x[k + 2] * f, x[k + 3] * f);
+  for (int k = 0; k < 16; k += 4) {
+    const unsigned lo = encode2<FMT>(__uint_as_float(v[k]) * f, __uint_as_float(v[k + 1]) * f);
+    const unsigned hi = encode2<FMT>(__uint_as_float(v[k + 2]) * f, __uint_as_float(v[k + 3]) * f);
     w[k >> 2] = FMT == MQ_E2M1 ? (lo | (hi << 8)) : (lo | (hi << 16));
   }
   if (FMT == MQ_E2M1) {
-    *reinterpret_cast<uint4*>(dst) = make_uint4(w[0] | (w[1] << 16), w[2] | (w[3] << 16), w[4] | (w[5] << 16), w[6] | (w[7] << 16));
+    unsigned q0 = w[0] | (w[1] << 16), q1 = w[2] | (w[3] << 16);
+    if (RELU) {
+      q0 &= ~(((q0 >> 3) & 0x11111111u) * 0xFu);
+      q1 &= ~(((q1 >> 3) & 0x11111111u) * 0xFu);
+    }
+    *reinterpret_cast<uint2*>(dst) = make_uint2(q0, q1);
   } else {
+    if (RELU) {
+      constexpr int S = (FMT == MQ_E4M3 || FMT == MQ_E5M2) ? 7 : 5;   // sign bit of a code in its byte
+#pragma unroll
+      for (int j = 0; j < 4; ++j) w[j] &= ~(((w[j] >> S) & 0x01010101u) * 0xFFu);
+    }
     *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
-    *reinterpret_cast<uint4*>(dst + 16) = make_uint4(w[4], w[5], w[6], w[7]);
   }
 }
+struct MxBlockCtx {
+  int Q, bend, half, quad, grp0, tw_, lane, c0;
+  uint32_t taddr;
+  bool row_ok;
+  unsigned col_mask;
+  unsigned* my_red;
+  uint8_t* o_codes;
+  uint8_t* o_scale;
+  uint64_t* tempty_acc;
+};
+// One 32-channel block of a warp's 32 rows.  v holds (or is about to hold) the block's accumulator values; each half of
+// the next block's load is issued as soon as its 16 registers have been converted, so it is in flight during the rest of
+// the conversion, the stores and the loop's bookkeeping (a second register buffer, which would put the whole of the next
+// load behind this block's arithmetic, does not fit in 128 registers: measured with spills, 1.6x slower).
+template <int FMT, int ACT>
+__device__ __forceinline__ void mx_block(const ConvTcParams& p, const MxBlockCtx& c, int b, uint32_t* v) {
+  constexpr int emax = FMT == MQ_E4M3 ? 8 : (FMT == MQ_E5M2 ? 15 : (FMT == MQ_E3M2 ? 4 : 2));
+  constexpr int bpe4 = FMT == MQ_E2M1 ? 1 : 2;
+  float m = 0.f;
+  if (c.Q > 0) {
+    tmem_ld_wait();
+    float m0 = 0.f, m1 = 0.f;
+    if (ACT == MQ_ACT_SILU) {
+#pragma unroll
+      for (int k = 0; k < 32; ++k) v[k] = __float_as_uint(mx_activation(__uint_as_float(v[k]), MQ_ACT_SILU));
+    }
+#pragma unroll
+    for (int k = 0; k < 32; k += 4) {
+      if (ACT == MQ_ACT_RELU) {
+        m0 = fmax3(m0, __uint_as_float(v[k]), __uint_as_float(v[k + 1]));
+        m1 = fmax3(m1, __uint_as_float(v[k + 2]), __uint_as_float(v[k + 3]));
+      } else {
+        m0 = fmax3(m0, fabsf(__uint_as_float(v[k])), fabsf(__uint_as_float(v[k + 1])));
+        m1 = fmax3(m1, fabsf(__uint_as_float(v[k + 2])), fabsf(__uint_as_float(v[k + 3])));
+      }
+    }
+    m = fmaxf(m0, m1);
+  } else {
+#pragma unroll
+    for (int k = 0; k < 32; ++k) v[k] = 0u;
+  }
+  const bool more = c.Q > 0 && b + 1 < c.bend;
+  if (b + 1 == c.bend) {      // the accumulator has been read: hand it back before the arithmetic and the stores
+    tc_fence_before_sync();
+    __syncwarp();
+    if (c.lane == 0) mbar_arrive(c.tempty_acc);
+  }
+  // maximum over the lanes of the same output column: non-negative floats order like their bit patterns, so one
+  // integer warp reduction per column group replaces a chain of shuffles
+  const unsigned mb = __reduce_max_sync(c.col_mask, c.row_ok ? __float_as_uint(m) : 0u);
+  unsigned mx = mb;
+  if (p.TW > 1) {     // the sample tile spans TW warps: exchange the maxima through shared memory
+    unsigned* rb = c.my_red + (b & 1) * 16;
+    if (c.lane < p.TW) rb[c.quad * 4 + c.lane] = mb;
+    half_sync(c.half);
+    mx = 0;
+    for (int g = 0; g < p.TW; ++g) mx = max(mx, rb[(c.grp0 + g) * 4 + c.tw_]);
+  }
+  const int code = scale_code_of(mx, emax);
+  const bool blk_ok = c.row_ok && c.c0 + 32 * b < p.mx_Cp;
+  if (c.quad == c.grp0 && c.lane < p.TW && blk_ok) c.o_scale[b] = (uint8_t)code;
+  const float f = scale_factor(code);
+  uint8_t* dst = c.o_codes + ((32 * b * bpe4) >> 1);
+  if (blk_ok) mx_encode_half<FMT, ACT == MQ_ACT_RELU>(v, f, dst);
+  if (more) tmem_ld_32x32b_x16(c.taddr + 32 * (b + 1), v);
+  if (blk_ok) mx_encode_half<FMT, ACT == MQ_ACT_RELU>(v + 16, f, dst + 8 * bpe4);   // 16 codes further: 16 bytes (E2M1: 8)
+  if (more) tmem_ld_32x32b_x16(c.taddr + 32 * (b + 1) + 16, v + 16);
+}
 // FMT: element format of the emitted tensor.  The role is compiled into kernel instances of its own (conv_tc_kernel's EPI
-// parameter), one per format, and the activation is chosen outside the element loops: a format switch per block inside
-// one kernel measured 602 us on a 1x1 layer (N = 256, 512 channels, 56 x 56) against 461 us for a single-format kernel, and
-// a non-inlined role per format 785 us.
+// parameter), one per format, and the activation is chosen outside the block loop.
 template <int MODE, int FMT>
 __device__ __forceinline__ void epilogue_mx_role(const ConvTcParams& p, unsigned* red, uint32_t tmem, uint64_t* tfull, uint64_t* tempty,
                                                  volatile int* abort_flag, int warp, int lane, unsigned total) {
@@ -322,6 +412,7 @@ __device__ __forceinline__ void epilogue_mx_role(const ConvTcParams& p, unsigned
     constexpr int bpe4 = FMT == MQ_E2M1 ? 1 : 2;        // bytes per element x 2
     const int Ct = p.mx_Cp >> 5;
     unsigned* my_red = red + half * 32;                 // [parity][quadrant][column]
+    const unsigned col_mask = (p.TW == 1 ? 0xffffffffu : (p.TW == 2 ? 0x55555555u : 0x11111111u)) << (lane & (p.TW - 1));   // lanes of this lane's column
     uint32_t tcount = 0;
     for (unsigned t = blockIdx.x; t < total; t += gridDim.x, ++tcount) {
       const Tile tile = decode_tile(p, t);
@@ -332,7 +423,8 @@ __device__ __forceinline__ void epilogue_mx_role(const ConvTcParams& p, unsigned
       bool ok = true;
       if (lane == 0) ok = !*abort_flag && mbar_wait(&tfull[acc], acc_phase(p, tcount), p.status, MQ_ERR_TIMEOUT);
       // the four warps of a half leave together or not at all: they meet at barriers inside the tile
-      if (half_any(half, !ok)) { *abort_flag = 1; break; }
+      // (one-column tiles have no barriers inside: each warp decides for itself)
+      if (p.TW > 1 ? half_any(half, !ok) : __shfl_sync(0xffffffffu, ok ? 0 : 1, 0) != 0) { *abort_flag = 1; break; }
       tc_fence_after_sync();
       int yo, xo;
       if (MODE == MQ_OP_FWD) { yo = tile.h; xo = tile.w0 + tw_; }
@@ -346,56 +438,26 @@ __device__ __forceinline__ void epilogue_mx_role(const ConvTcParams& p, unsigned
       const long long pix = (long long)yo * p.Wd + xo;
       uint8_t* o_codes = p.mx_codes + (((pix * p.N + n) * p.mx_Cp + tile.c0) * bpe4 >> 1);
       uint8_t* o_scale = p.mx_scales + (pix * p.Nt + (n >> 5)) * Ct + (tile.c0 >> 5);
-      // the TMEM load of block b + 1 is in flight while block b is reduced, converted and stored
+      // no separate activation pass for none / ReLU: the maximum of max(x, 0) is the maximum of x and 0, and negative
+      // codes are cleared after packing
+      MxBlockCtx c;
+      c.Q = Q; c.bend = bend; c.taddr = taddr; c.row_ok = row_ok; c.col_mask = col_mask; c.my_red = my_red; c.half = half; c.quad = quad;
+      c.grp0 = grp0; c.tw_ = tw_; c.lane = lane; c.o_codes = o_codes; c.o_scale = o_scale; c.c0 = tile.c0; c.tempty_acc = &tempty[acc];
       uint32_t v[32];
       if (Q > 0 && bbeg < bend) {
         tmem_ld_32x32b_x16(taddr + 32 * bbeg, v);
         tmem_ld_32x32b_x16(taddr + 32 * bbeg + 16, v + 16);
       }
+      // the activation is chosen outside the block loop: three straight-line copies instead of a test per element
+      if (p.mx_act == MQ_ACT_RELU) {
 #pragma unroll 1
-      for (int b = bbeg; b < bend; ++b) {
-        float x[32];
-        float m = 0.f;
-        if (Q > 0) {
-          tmem_ld_wait();
-          // the activation is chosen outside the element loop: three straight-line copies instead of a test per element
-          if (p.mx_act == MQ_ACT_RELU) {
-#pragma unroll
-            for (int k = 0; k < 32; ++k) { x[k] = fmaxf(__uint_as_float(v[k]), 0.f); m = fmaxf(m, x[k]); }
-          } else if (p.mx_act == MQ_ACT_SILU) {
-#pragma unroll
-            for (int k = 0; k < 32; ++k) { x[k] = mx_activation(__uint_as_float(v[k]), MQ_ACT_SILU); m = fmaxf(m, fabsf(x[k])); }
-          } else {
-#pragma unroll
-            for (int k = 0; k < 32; ++k) { x[k] = __uint_as_float(v[k]); m = fmaxf(m, fabsf(x[k])); }
-          }
-          if (b + 1 < bend) {
-            tmem_ld_32x32b_x16(taddr + 32 * (b + 1), v);
-            tmem_ld_32x32b_x16(taddr + 32 * (b + 1) + 16, v + 16);
-          }
-        } else {
-#pragma unroll
-          for (int k = 0; k < 32; ++k) x[k] = 0.f;
-        }
-        if (b + 1 == bend) {      // the accumulator has been read: hand it back before the arithmetic and the stores
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&tempty[acc]);
-        }
-        unsigned mb = row_ok ? __float_as_uint(m) : 0u;
-        for (int off = p.TW; off < 32; off <<= 1) mb = max(mb, __shfl_xor_sync(0xffffffffu, mb, off));
-        unsigned* rb = my_red + (b & 1) * 16;
-        if (lane < p.TW) rb[quad * 4 + lane] = mb;
-        half_sync(half);
-        unsigned mx = 0;
-        for (int g = 0; g < p.TW; ++g) mx = max(mx, rb[(grp0 + g) * 4 + tw_]);
-        const int code = scale_code_of(mx, emax);
-        if (quad == grp0 && lane < p.TW && row_ok && tile.c0 + 32 * b < p.mx_Cp) o_scale[b] = (uint8_t)code;
-        if (row_ok && tile.c0 + 32 * b < p.mx_Cp) {
-          const float f = scale_factor(code);
-          uint8_t* dst = o_codes + ((32 * b * bpe4) >> 1);
-          mx_encode_row<FMT>(x, f, dst);
-        }
+        for (int b = bbeg; b < bend; ++b) mx_block<FMT, MQ_ACT_RELU>(p, c, b, v);
+      } else if (p.mx_act == MQ_ACT_SILU) {
+#pragma unroll 1
+        for (int b = bbeg; b < bend; ++b) mx_block<FMT, MQ_ACT_SILU>(p, c, b, v);
+      } else {
+#pragma unroll 1
+        for (int b = bbeg; b < bend; ++b) mx_block<FMT, MQ_ACT_NONE>(p, c, b, v);
       }
       if (bbeg >= bend) {      // a tile of 32 channels leaves the second half without a block
         tc_fence_before_sync();

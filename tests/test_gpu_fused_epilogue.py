@@ -145,6 +145,29 @@ def test_input_gradient_emits_previous_layers_gradient(name, shape, fmts, out_fm
     check_emitted(f"{name} bwd_data", d_prev, oracle.ROLE_DY, out_fmt, gx64, GEMM_TOL * ab, mq.ACT_NONE, dxq)
 
 
+@pytest.mark.parametrize("tw", [1, 2, 4])
+@pytest.mark.parametrize("fmts,out_fmt", [((E4M3, E4M3, E5M2), E4M3), ((E2M1, E2M1, E2M1), E2M1)], ids=["fp8", "fp4"])
+def test_every_tile_width(knobs, fmts, out_fmt, tw):
+    """The epilogue's tiles are 1, 2 or 4 output columns wide (one column: a warp's rows are a whole sample tile; more: the
+    warps of a tile exchange their maxima).  The library picks one per layer; here each is forced on the same ragged layer."""
+    knobs(MQ_TC_MX_TW=tw)
+    d = inputs.conv_desc(140, 64, 5, 6, 96, 3, 1, 1)
+    x, w, g = inputs.make_x(d, 71, "gauss"), inputs.make_w(d, 71), inputs.make_dy(d, 71, "gauss")
+    oq = [oracle.quantize(d, r, f, t) for r, f, t in zip((oracle.ROLE_X, oracle.ROLE_W, oracle.ROLE_DY), fmts, (x, w, g))]
+    xh, wh, gh = [oracle.dequant(d, r, f, *q) for r, f, q in zip((oracle.ROLE_X, oracle.ROLE_W, oracle.ROLE_DY), fmts, oq)]
+    gq = [mq.quantize(d, r, f, dev(t)) for r, f, t in zip((mq.ROLE_X, mq.ROLE_W, mq.ROLE_DY), fmts, (x, w, g))]
+    y64, ab = oracle.conv_fwd(d, xh, wh)
+    yq = mq.conv_fwd_mx(d, gq[0], gq[1], out_fmt, mq.ACT_RELU)
+    assert mq.last_device_status() == 0
+    ho, wo = inputs.out_hw(d)
+    check_emitted(f"tw{tw} fwd", d._replace(C_in=d.C_out, H=ho, W=wo), oracle.ROLE_X, out_fmt, y64, GEMM_TOL * ab, mq.ACT_RELU, yq)
+    gx64, ab = oracle.conv_bwd_data(d, wh, gh)
+    dxq = mq.conv_bwd_data_mx(d, gq[1], gq[2], fmts[2])
+    assert mq.last_device_status() == 0
+    check_emitted(f"tw{tw} bwd_data", inputs.conv_desc(d.N, 32, d.H, d.W, d.C_in, 1, 1, 0), oracle.ROLE_DY, fmts[2], gx64, GEMM_TOL * ab,
+                  mq.ACT_NONE, dxq)
+
+
 def test_bad_arguments():
     d = inputs.conv_desc(32, 64, 6, 6, 64, 3, 1, 1)
     xq, wq = mq.quantize(d, mq.ROLE_X, E4M3, dev(inputs.make_x(d, 1))), mq.quantize(d, mq.ROLE_W, E4M3, dev(inputs.make_w(d, 1)))
