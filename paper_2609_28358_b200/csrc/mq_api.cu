@@ -140,13 +140,15 @@ struct ConvTcPlan {
 
 // line: line-block operands (forward only).  mx: the quantizing epilogue (tiles of at most 4 output columns, channel tiles
 // of whole 32-channel blocks, per-tap kernel).
-bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, ConvTcPlan* out, bool line = false, bool mx = false) {
+// ts16: the paper's own format (E2M1 elements, one E4M3 scale per 16 x 16 block, an fp32 scale per tensor): kind::mxf4nvf4, per-tap kernel.
+bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, ConvTcPlan* out, bool line = false, bool mx = false, bool ts16 = false) {
   const bool fp4 = fmt_w == MQ_E2M1;
+  if (ts16 && (!fp4 || fmt_x_like != MQ_E2M1 || mx || line)) return false;
   const int bits = fp4 ? 4 : 8;
   const int taps = g.Kh * g.Kw;
   ConvTcParams p{};
   p.mode = op;
-  p.kind_fp4 = fp4 ? 1 : 0;
+  p.kind_fp4 = ts16 ? 2 : (fp4 ? 1 : 0);
   p.N = g.N; p.Nt = g.Nt;
   p.Kh = g.Kh; p.Kw = g.Kw; p.sh = g.sh; p.sw = g.sw; p.ph = g.ph; p.pw = g.pw;
   int Kp;
@@ -165,7 +167,7 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   p.cpt = rowbytes / p.KB;
   const int w_eff = op == MQ_OP_FWD ? g.Wo : (g.W + g.sw - 1) / g.sw;
   // line blocks (one scale per row): the per-tap kernel, whose preparation launch lays out the scale vectors row by row
-  const bool thin = !line && !mx && g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && !env_int("MQ_TC_NO_HALO", 0);
+  const bool thin = !line && !mx && !ts16 && g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && !env_int("MQ_TC_NO_HALO", 0);
   p.line = line ? 1 : 0;
   const int cd16 = mx ? (p.Cd + 31) / 32 * 32 : (p.Cd + 15) / 16 * 16;
   p.BN = cd16 <= 128 ? cd16 : 128;
@@ -236,14 +238,17 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   // ... and for 1x1 layers, whose main loop is a handful of stages: the tile's time is its store (measured 4-12 % faster, 28x28 and
   // 56x56 images, 256 and 512 channels)
   p.tma_store = !mx && tma_store_ok && (env_int("MQ_TC_TMA_STORE", 0) || (taps == 1 && !env_int("MQ_TC_NO_TMA_STORE", 0))) ? 1 : 0;
-  const size_t stage_bytes = 128 * 128 + (size_t)p.BN * 128 + 3072;
+  const size_t stage_bytes = 128 * 128 + (size_t)p.BN * 128 + (ts16 ? 6144 : 3072);
+  const int sf_cols = ts16 ? 48 : 24;
   int stages = (int)((227 * 1024 - 2048 - (p.tma_store ? 65536 : 0)) / stage_bytes);
   if (stages > 8) stages = 8;
   if (stages < 2) return false;
   p.stages = stages;
-  // TMEM (512 columns): accumulators (BN columns each) + one 24-column scale buffer per pipeline stage
-  p.n_acc = (2 * p.BN + 24 * stages <= 512) ? 2 : 1;
-  if (p.n_acc * p.BN + 24 * stages > 512) return false;
+  // TMEM (512 columns): accumulators (BN columns each) + one 24-column (E4M3 scales per 16: 48-column) scale buffer per pipeline stage
+  while (stages > 2 && p.BN + sf_cols * stages > 512) --stages;
+  p.stages = stages;
+  p.n_acc = (2 * p.BN + sf_cols * stages <= 512) ? 2 : 1;
+  if (p.n_acc * p.BN + sf_cols * stages > 512) return false;
   p.mma_cp = env_int("MQ_TC_NO_MMA_CP", 0) ? 0 : 1;   // E2M1 too: the bubble behind a copier warp costs more than the lane's extra issues
   p.pair = !mx && op == MQ_OP_BWD_DATA && g.sw == 2 && layout == MQ_NCHW && p.Wd % 2 == 0 && p.n_acc == 2 && p.total_tiles % 2 == 0 &&
            !env_int("MQ_TC_NO_PAIR", 0);
@@ -251,11 +256,12 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   p.max_stages = (nkh * nkw * p.cpt + p.G - 1) / p.G;
   const uint32_t fa = fp4 ? 1u : fmt_mma_code(fmt_x_like);   // kind::mxf4: 1 = E2M1; kind::mxf8f6f4: E4M3 0, E5M2 1, E2M3 3, E3M2 4
   const uint32_t fb = fp4 ? 1u : fmt_mma_code(fmt_w);
-  p.idesc = (fa << 7) | (fb << 10) | ((uint32_t)(p.BN >> 3) << 17) | (1u << 23) | ((128u >> 4) << 24);
+  // bit 23: scale type, 1 = E8M0, 0 = E4M3 (kind::mxf4nvf4)
+  p.idesc = (fa << 7) | (fb << 10) | ((uint32_t)(p.BN >> 3) << 17) | (ts16 ? 0u : (1u << 23)) | ((128u >> 4) << 24);
   // whole-tile-per-stage variant: stride 1, one chunk per tap (<= 64 bytes of channels).  One box with the column
   // halo needs 8-column tiles; one box per column shift takes 8, 16 or 32 columns (longer NCHW store runs).
   p.halo = 0;
-  if (!line && !mx && g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && taps <= 64 && !env_int("MQ_TC_NO_HALO", 0)) {
+  if (!line && !mx && !ts16 && g.sh == 1 && g.sw == 1 && p.cpt == 1 && p.KB <= 64 && taps <= 64 && !env_int("MQ_TC_NO_HALO", 0)) {
     const int spa = fp4 ? 2 : 1, atoms_b = (p.BN + 127) / 128;
     if (p.TW == 8) {
       p.WH = p.TW + g.Kw - 1;
@@ -279,12 +285,12 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   }
   // unit strides and one 128-byte chunk per stage: the activation-side scale chunk of (tile, kh) equals that of the tile one
   // output row further with kh - 1, so chunks are stored per source row - Kh times fewer to expand
-  p.sfa_dedup = (!p.halo && p.KB == 128 && g.sh == 1 && g.sw == 1 && !env_int("MQ_TC_NO_SFA_DEDUP", 0)) ? 1 : 0;
+  p.sfa_dedup = (!p.halo && !ts16 && p.KB == 128 && g.sh == 1 && g.sw == 1 && !env_int("MQ_TC_NO_SFA_DEDUP", 0)) ? 1 : 0;
   p.sfa_hk = p.tiles_h + g.Kh - 1;
   out->p = p;
   size_t o = 0;
   out->off_wt_scales = 0;
-  if (op == MQ_OP_BWD_DATA) { o = wt_codes_bytes(g, fmt_w); out->off_wt_scales = o; o += up256((size_t)g.Ct * taps * g.Cot); }
+  if (op == MQ_OP_BWD_DATA) { o = wt_codes_bytes(g, fmt_w); out->off_wt_scales = o; o += up256((size_t)g.Ct * taps * g.Cot * (ts16 ? 4 : 1)); }
   out->off_sfa = o; o += up256(conv_tc_sfa_bytes(p));
   out->off_sfb = o; o += up256(conv_tc_sfb_bytes(p));
   out->off_bimg = o;
@@ -299,11 +305,11 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
 
 // Scratch of a forward / input-gradient call: the tensor-core plan's where one exists (it depends on the output layout: the
 // larger of the two), never less than what the CUDA-core kernels need, which take the layers a plan refuses.
-size_t conv_tc_workspace(int op, const Geom& g, int fmt_x_like, int fmt_w, bool line) {
+size_t conv_tc_workspace(int op, const Geom& g, int fmt_x_like, int fmt_w, bool line, bool ts16 = false) {
   size_t need = conv_generic_workspace(op, g);
   for (int layout = 0; layout < 2; ++layout) {   // the tile shape, hence the scratch, depends on the output layout
     ConvTcPlan pl;
-    if (conv_tc_plan(op, g, fmt_x_like, fmt_w, layout, &pl, line) && pl.total > need) need = pl.total;
+    if (conv_tc_plan(op, g, fmt_x_like, fmt_w, layout, &pl, line, false, ts16) && pl.total > need) need = pl.total;
   }
   return need;
 }
@@ -327,7 +333,7 @@ mq_status run_conv_tc(int op, const Geom& g, ConvTcPlan& pl, const mq_qtensor* q
     p.b_scales = qw->scales;
   } else {
     // per-tap kernel, operands that need no repacking: the re-layout rides in the scale-expansion launch
-    p.wt_fused = (!p.halo && !fmt_is_6bit(qw->fmt) && !env_int("MQ_TC_NO_WT_FUSED", 0)) ? 1 : 0;
+    p.wt_fused = (!p.halo && !fmt_is_6bit(qw->fmt) && (p.kind_fp4 == 2 || !env_int("MQ_TC_NO_WT_FUSED", 0))) ? 1 : 0;   // kind 2: this route only
     if (p.wt_fused) {
       p.wt_in = w_stored; p.wt_out = base; p.wt_sc_in = qw->scales;
       p.wt_Cout = g.Cout; p.wt_Cop = g.Cop; p.wt_Cp = g.Cp; p.wt_bx = g.Cp / 32; p.wt_by = g.Cop / 32;
@@ -335,6 +341,7 @@ mq_status run_conv_tc(int op, const Geom& g, ConvTcPlan& pl, const mq_qtensor* q
     p.b_scales = wt_scales;
   }
   p.a_scales = qx_like->scales;
+  p.a_tscale = qx_like->tensor_scale; p.b_tscale = qw->tensor_scale;
   p.sfa_img = base + pl.off_sfa;
   p.sfb_img = base + pl.off_sfb;
   p.b_codes = b_codes; p.b_rows_total = pl.rows_b; p.b_rowbytes = pl.rowbytes; p.b_img = base + pl.off_bimg;
@@ -407,8 +414,10 @@ struct WgradPlan {
   bool recode4;   // E2M1 operands re-encoded as E4M3 bytes for the 8-bit path
 };
 
-WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
+// ts16: the paper's own format (E4M3 scales per 16 x 16 block): the two E2M1 modes with kind::mxf4nvf4
+WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g, bool ts16 = false) {
   WgradPlan w{};
+  if (ts16 && (fmt_x != MQ_E2M1 || fmt_g != MQ_E2M1 || env_int("MQ_TC_NO_TS16", 0))) return w;
   if (env_int("MQ_DISABLE_TC", 0) || env_int("MQ_DISABLE_TC_WGRAD", 0)) return w;
   const bool fp4_in = fmt_x == MQ_E2M1 && fmt_g == MQ_E2M1;
   const bool fp8_in = fmt_x != MQ_E2M1 && fmt_g != MQ_E2M1;
@@ -417,7 +426,7 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   // E2M1 value is an E4M3 value, so the codes are re-encoded exactly as E4M3 bytes in scratch and the 8-bit path (stored
   // order read MN-major, block pairs) runs - faster than the per-pixel E2M1 mode (MQ_WGRAD_FP4_PIXEL=1 keeps that mode)
   const bool flat_ok = fp4_in && g.sh == 1 && g.sw == 1 && (g.Nt == 1 || g.Nt == 2 || g.Nt == 4 || g.Nt == 8) && !env_int("MQ_WGRAD_NO_FLAT", 0);
-  const bool recode4 = fp4_in && !flat_ok && !env_int("MQ_WGRAD_FP4_PIXEL", 0);
+  const bool recode4 = fp4_in && !flat_ok && !ts16 && !env_int("MQ_WGRAD_FP4_PIXEL", 0);   // (E4M3 block scales are no E8M0 scales: not for ts16)
   const bool fp4 = fp4_in && !recode4;
   const bool fp8 = fp8_in || recode4;
   w.recode4 = recode4;
@@ -430,6 +439,9 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   p.Kh = g.Kh; p.Kw = g.Kw; p.sh = g.sh; p.sw = g.sw; p.ph = g.ph; p.pw = g.pw;
   const bool flat = fp4 && g.sh == 1 && g.sw == 1 && (g.Nt == 1 || g.Nt == 2 || g.Nt == 4 || g.Nt == 8) && !env_int("MQ_WGRAD_NO_FLAT", 0);
   p.mode = fp8 ? MQ_WG_FP8 : (flat ? MQ_WG_FP4_FLAT : MQ_WG_FP4_PIXEL);
+  p.kind = ts16 ? 2 : (fp4 ? 1 : 0);
+  const int sf_cols1 = ts16 ? 16 : 8;       // TMEM columns and shared-memory bytes of one 128-row scale chunk
+  const int sf_bytes1 = ts16 ? 2048 : 1024;
   if (fp4) p.BPP = flat ? g.Nt : (g.Nt >= 5 ? 8 : (g.Nt >= 3 ? 4 : g.Nt));
   else p.BPP = g.Nt >= 3 ? 4 : g.Nt;
   p.KPX = (fp4 ? 8 : 4) / p.BPP;
@@ -462,7 +474,7 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   p.cb_tiles = (g.Cp + p.b_rows - 1) / p.b_rows;
   // taps per block: a whole kernel row in the flat mode when its accumulators fit in tensor memory
   p.TG = p.grp8 ? g.Kw : 1;
-  if (flat && g.Kw > 1 && g.Kw * p.b_rows + 2 * (8 + 8 * ((g.Kw * p.b_rows + 127) / 128)) <= 512 && !env_int("MQ_WGRAD_NO_GROUP", 0)) p.TG = g.Kw;
+  if (flat && g.Kw > 1 && g.Kw * p.b_rows + 2 * sf_cols1 * (1 + (g.Kw * p.b_rows + 127) / 128) <= 512 && !env_int("MQ_WGRAD_NO_GROUP", 0)) p.TG = g.Kw;
   p.NB = (p.TG * p.b_rows + 127) / 128;
   p.n0 = p.TG * p.b_rows < 256 ? p.TG * p.b_rows : 256;
   p.n1 = p.TG * p.b_rows - p.n0;
@@ -476,17 +488,17 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g) {
   p.splits = splits;
   p.b_tile_bytes = flat ? (p.KPX + p.TG - 1) * p.b_rows * p.KBn : (p.cta2 ? 128 : p.b_rows) * 128;   // a pair's blocks load half of X each
   if (p.grp8) p.b_tile_bytes = ((p.KPX - 1) * g.sw + p.TG) * 32 * p.BPP * g.Cp;
-  p.stage_bytes = (128 * 128 + p.b_tile_bytes + (1 + p.NB) * 1024 + 1023) / 1024 * 1024;
+  p.stage_bytes = (128 * 128 + p.b_tile_bytes + (1 + p.NB) * sf_bytes1 + 1023) / 1024 * 1024;
   {
     int st = (227 * 1024 - 2048) / p.stage_bytes;
     if (st > 6) st = 6;
-    while (st > 2 && p.TG * p.b_rows + st * (8 + 8 * p.NB) > 512) --st;
+    while (st > 2 && p.TG * p.b_rows + st * sf_cols1 * (1 + p.NB) > 512) --st;
     p.stages = st;
-    const int cols = p.TG * p.b_rows + st * (8 + 8 * p.NB);
+    const int cols = p.TG * p.b_rows + st * sf_cols1 * (1 + p.NB);
     p.tmem_cols = cols <= 256 ? 256 : 512;
     if (st < 2 || cols > 512) return w;
   }
-  const int spa = fp4 ? 2 : 1;
+  const int spa = ts16 ? 4 : (fp4 ? 2 : 1);
   w.P_a = p.stages_total * p.KPX;
   w.P_b = (w.P_a + (g.Kh - 1) * p.Wp + g.Kw - 1 + 7) / 8 * 8;
   size_t o = up256((size_t)splits * g.Cout * g.Kh * g.Kw * g.Cp * sizeof(float));
@@ -515,13 +527,14 @@ mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const 
   uint8_t* xt = base + w.off_xt;
   uint8_t* gt = base + w.off_gt;
   CUtensorMap map_a{}, map_b{};
+  const uint32_t sf_type = p.kind == 2 ? 0u : (1u << 23);   // instruction descriptor bit 23: E8M0 scales (0: E4M3)
   if (p.mode == MQ_WG_FP4_FLAT) {
     p.xt = xt; p.gt = gt;
-    p.idesc = (1u << 7) | (1u << 10) | (1u << 23) | ((128u >> 4) << 24);
+    p.idesc = (1u << 7) | (1u << 10) | sf_type | ((128u >> 4) << 24);
   } else if (p.mode == MQ_WG_FP4_PIXEL) {
     if (launch_fp4_to_n_major(static_cast<const uint8_t*>(qx->codes), xt, g.H * g.W, g.N, g.Cp, w.Npad, stream) != cudaSuccess) return MQ_ERR_CUDA;
     if (launch_fp4_to_n_major(static_cast<const uint8_t*>(qg->codes), gt, g.Ho * g.Wo, g.N, g.Cop, w.Npad, stream) != cudaSuccess) return MQ_ERR_CUDA;
-    p.idesc = (1u << 7) | (1u << 10) | (1u << 23) | ((128u >> 4) << 24);
+    p.idesc = (1u << 7) | (1u << 10) | sf_type | ((128u >> 4) << 24);
     const uint64_t nb = (uint64_t)w.Npad / 2;
     const int swz = p.KBn >= 32 ? p.KBn : 0;
     {
@@ -595,7 +608,9 @@ mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const 
     if (!encode_tensor_map_u8(&map_sfb, p.sfb_img, 2, db, st, bb, nullptr, 0)) return MQ_ERR_CUDA;
   }
   if (launch_wgrad_tc(p, map_a, map_b, map_p, map_sfa, map_sfb, stream) != cudaSuccess) return MQ_ERR_CUDA;
-  return launch_bwd_weight_reduce(partial, out, g, p.splits, layout, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
+  const bool tsc = p.kind == 2;
+  return launch_bwd_weight_reduce(partial, out, g, p.splits, layout, stream, tsc ? qx->tensor_scale : nullptr, tsc ? qg->tensor_scale : nullptr) == cudaSuccess
+             ? MQ_OK : MQ_ERR_CUDA;
 }
 
 // address of the current device's status word (a __device__ variable has one instance per device and per context:
@@ -639,12 +654,13 @@ mq_status run_conv(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int r
     const mq_qtensor* qx_like = op == MQ_OP_FWD ? qa : qb;
     const mq_qtensor* qw = op == MQ_OP_FWD ? qb : qa;
     ConvTcPlan pl;
-    if (qa->block != MQ_BLOCK_TS16 && (op == MQ_OP_FWD || op == MQ_OP_BWD_DATA) && conv_tc_eligible(op, g, qx_like->fmt, qw->fmt) &&
-        conv_tc_plan(op, g, qx_like->fmt, qw->fmt, layout, &pl, qx_like->block == MQ_BLOCK_LINE32))
+    const bool ts16 = qa->block == MQ_BLOCK_TS16;
+    if ((!ts16 || !env_int("MQ_TC_NO_TS16", 0)) && (op == MQ_OP_FWD || op == MQ_OP_BWD_DATA) && conv_tc_eligible(op, g, qx_like->fmt, qw->fmt) &&
+        conv_tc_plan(op, g, qx_like->fmt, qw->fmt, layout, &pl, qx_like->block == MQ_BLOCK_LINE32, false, ts16))
       return run_conv_tc(op, g, pl, qx_like, qw, static_cast<float*>(out), layout, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
   }
-  if (op == MQ_OP_BWD_WEIGHT && qa->block != MQ_BLOCK_TS16) {
-    WgradPlan w = wgrad_plan(g, qa->fmt, qb->fmt);
+  if (op == MQ_OP_BWD_WEIGHT) {
+    WgradPlan w = wgrad_plan(g, qa->fmt, qb->fmt, qa->block == MQ_BLOCK_TS16);
     if (w.ok) return run_wgrad_tc(g, w, qa, qb, static_cast<float*>(out), layout, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
   }
   ConvArgs a;
@@ -697,11 +713,12 @@ mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt
   const Geom g = make_geom(*desc);
   const bool line = block == MQ_BLOCK_LINE32;
   *bytes = conv_generic_workspace(op, g);
-  if (block == MQ_BLOCK_TS16) return (fmt_a == MQ_E2M1 && fmt_b == MQ_E2M1) ? MQ_OK : MQ_ERR_INVALID_ARG;   // CUDA-core kernels in this build
-  if (op == MQ_OP_FWD && conv_tc_eligible(op, g, fmt_a, fmt_b)) *bytes = conv_tc_workspace(op, g, fmt_a, fmt_b, line);
-  if (op == MQ_OP_BWD_DATA && conv_tc_eligible(op, g, fmt_b, fmt_a)) *bytes = conv_tc_workspace(op, g, fmt_b, fmt_a, false);
+  const bool ts16 = block == MQ_BLOCK_TS16;
+  if (ts16 && (fmt_a != MQ_E2M1 || fmt_b != MQ_E2M1)) return MQ_ERR_INVALID_ARG;
+  if (op == MQ_OP_FWD && conv_tc_eligible(op, g, fmt_a, fmt_b)) *bytes = conv_tc_workspace(op, g, fmt_a, fmt_b, line, ts16);
+  if (op == MQ_OP_BWD_DATA && conv_tc_eligible(op, g, fmt_b, fmt_a)) *bytes = conv_tc_workspace(op, g, fmt_b, fmt_a, false, ts16);
   if (op == MQ_OP_BWD_WEIGHT) {
-    const WgradPlan w = wgrad_plan(g, fmt_a, fmt_b);
+    const WgradPlan w = wgrad_plan(g, fmt_a, fmt_b, ts16);
     if (w.ok) *bytes = w.total;
   }
   return MQ_OK;

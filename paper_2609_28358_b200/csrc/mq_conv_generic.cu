@@ -252,8 +252,11 @@ __global__ void __launch_bounds__(GT) bwd_weight_generic(ConvArgs a, int splits)
 // The reads are `splits` times the writes, so threads follow the partials' own order (4 consecutive input
 // channels per thread, 16-byte loads); a block's four thread groups take every fourth split each and are
 // combined through shared memory in group order, so the result does not depend on scheduling.
-__global__ void __launch_bounds__(256) bwd_weight_reduce(const float* __restrict__ part, float* __restrict__ out, Geom g, int splits, int layout) {
+// ta, tb: the two tensors' fp32 scales when the partial sums still lack them (tensor-core GEMM on E4M3-scaled blocks, Eq. 4), else null
+__global__ void __launch_bounds__(256) bwd_weight_reduce(const float* __restrict__ part, float* __restrict__ out, Geom g, int splits, int layout,
+                                                         const float* __restrict__ ta, const float* __restrict__ tb) {
   pdl_wait();
+  const float os = ta ? __ldg(ta) * __ldg(tb) : 1.f;
   __shared__ float4 sh[3][64];
   const int taps = g.Kh * g.Kw;
   const int cq = g.Cp >> 2;                                   // float4 columns per (co, tap)
@@ -278,7 +281,7 @@ __global__ void __launch_bounds__(256) bwd_weight_reduce(const float* __restrict
       for (int q = 0; q < 3; ++q) { const float4 v = sh[q][col]; s.x += v.x; s.y += v.y; s.z += v.z; s.w += v.w; }
       const int c4 = (int)(qd % cq); const long long r = qd / cq;
       const int tap = (int)(r % taps), co = (int)(r / taps);
-      const float vals[4] = {s.x, s.y, s.z, s.w};
+      const float vals[4] = {s.x * os, s.y * os, s.z * os, s.w * os};
 #pragma unroll
       for (int e = 0; e < 4; ++e) {
         const int ci = 4 * c4 + e;
@@ -310,12 +313,13 @@ size_t conv_generic_workspace(int op, const Geom& g) {
   return (size_t)conv_generic_bwd_weight_splits(g) * g.Cout * g.Kh * g.Kw * g.Cp * sizeof(float);
 }
 
-cudaError_t launch_bwd_weight_reduce(const float* partial, float* out, const Geom& g, int splits, int layout, cudaStream_t s) {
+cudaError_t launch_bwd_weight_reduce(const float* partial, float* out, const Geom& g, int splits, int layout, cudaStream_t s, const float* ta,
+                                     const float* tb) {
   const long long quads = (long long)g.Cout * g.Kh * g.Kw * (g.Cp / 4);
   unsigned blocks = (unsigned)((quads + 63) / 64);
   if (blocks > (unsigned)sm_count() * 16) blocks = (unsigned)sm_count() * 16;
   count_launches(1);
-  return launch_pdl(bwd_weight_reduce, dim3(blocks), dim3(256), 0, s, partial, out, g, splits, layout);
+  return launch_pdl(bwd_weight_reduce, dim3(blocks), dim3(256), 0, s, partial, out, g, splits, layout, ta, tb);
 }
 
 // Two template classes per operand: packed E2M1 (2) or one byte per code (0; the format itself is read at run time)
@@ -348,7 +352,7 @@ cudaError_t launch_conv_generic(int op, const ConvArgs& a, cudaStream_t s) {
     const long long quads = (long long)g.Cout * g.Kh * g.Kw * (g.Cp / 4);
     unsigned blocks = (unsigned)((quads + 63) / 64);
     if (blocks > (unsigned)sm_count() * 16) blocks = (unsigned)sm_count() * 16;
-    bwd_weight_reduce<<<blocks, 256, 0, s>>>(reinterpret_cast<const float*>(a.workspace), a.out, g, splits, a.out_layout);
+    bwd_weight_reduce<<<blocks, 256, 0, s>>>(reinterpret_cast<const float*>(a.workspace), a.out, g, splits, a.out_layout, nullptr, nullptr);
     count_launches(1);
   }
   count_launches(1);

@@ -32,6 +32,9 @@ constexpr int A_STAGE_BYTES = 128 * 128;
 constexpr int SFA_BYTES = 1024;   // up to 2 groups of 4 scale bytes per row
 constexpr int SFB_BYTES = 2048;   // up to 2 groups x 2 atoms of 128 rows
 constexpr int SF_COLS = 24;       // TMEM columns of one scale buffer: 8 (A) + 16 (B)
+// The same three for kind 2 (four scale bytes per row and MMA instead of at most two)
+constexpr int SFA_BYTES_NV = 2048, SFB_BYTES_NV = 4096, SF_COLS_NV = 48;
+__host__ __device__ constexpr int spa_of_kind(int kind) { return kind == 2 ? 4 : (kind == 1 ? 2 : 1); }
 
 
 struct Tile { int c0, w0, n0, h, cls, ct; };
@@ -125,6 +128,12 @@ __device__ __forceinline__ int src_w0(const TapWalk<MODE>& w, const ChunkPos& c)
 template <int MODE>
 __device__ __forceinline__ int tap_index(const TapWalk<MODE>& w, const ChunkPos& c) { return w.tap0 + c.ia * w.tap_dh + c.ib * w.tap_dw; }
 
+// Product of the two tensors' fp32 scales (Eq. 4) that the accumulator of kind 2 is multiplied by; 1 for the other kinds
+__device__ __forceinline__ float out_scale_of(const ConvTcParams& p) { return p.kind_fp4 == 2 ? __ldg(p.a_tscale) * __ldg(p.b_tscale) : 1.f; }
+__device__ __forceinline__ void scale16(uint32_t* v, float os) {
+#pragma unroll
+  for (int j = 0; j < 16; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * os);
+}
 // An epilogue warp hands its accumulator back: to this block's barrier, or (a pair of blocks: the peer's warps) to the
 // leader's, whose MMA warp waits for the epilogues of both blocks.
 // Accumulator buffer of a block's tcount-th tile and the parity of that buffer's barriers (1 or 2 buffers; a third
@@ -147,6 +156,7 @@ __device__ __forceinline__ void epilogue_role(const ConvTcParams& p, uint32_t tm
     const int cbeg = half == 0 ? 0 : ((p.BN / 2 + 15) & ~15);
     const int cend = half == 0 ? ((p.BN / 2 + 15) & ~15) : p.BN;
     const long long cs = (long long)p.Hd * p.Wd;
+    const float os = out_scale_of(p);
     uint32_t tcount = 0;
     for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
       const Tile tile = decode_tile(p, t);
@@ -180,6 +190,7 @@ __device__ __forceinline__ void epilogue_role(const ConvTcParams& p, uint32_t tm
         if (Q > 0) {
           tmem_ld_32x32b_x16(taddr + c, v);
           tmem_ld_wait();
+          if (p.kind_fp4 == 2) scale16(v, os);
         } else {
 #pragma unroll
           for (int j = 0; j < 16; ++j) v[j] = 0u;
@@ -221,6 +232,7 @@ __device__ __forceinline__ void epilogue_pair_role(const ConvTcParams& p, uint32
     const int cbeg = half == 0 ? 0 : ((p.BN / 2 + 15) & ~15);
     const int cend = half == 0 ? ((p.BN / 2 + 15) & ~15) : p.BN;
     const long long cs = (long long)p.Hd * p.Wd;
+    const float os = out_scale_of(p);
 #pragma unroll 1
     for (unsigned j = 0, t; (t = tile_of_iter(p, 2 * j)) < total && !*abort_flag; ++j) {
       const Tile t0 = decode_tile(p, t), t1 = decode_tile(p, t + 1);
@@ -244,6 +256,7 @@ __device__ __forceinline__ void epilogue_pair_role(const ConvTcParams& p, uint32
         if (Q0 > 0) tmem_ld_32x32b_x16(taddr + c, v0);
         if (Q1 > 0) tmem_ld_32x32b_x16(taddr + p.BN + c, v1);
         tmem_ld_wait();
+        if (p.kind_fp4 == 2) { scale16(v0, os); scale16(v1, os); }   // (accumulators without taps are zeroed below)
         if (Q0 == 0) {
 #pragma unroll
           for (int q = 0; q < 16; ++q) v0[q] = 0u;
@@ -486,6 +499,7 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
     const int n_off = quad * (32 >> p.lgTW);          // first sample of this warp's rows inside the tile
     const bool hwnc = p.out_layout == MQ_HWNC;
     const int hrow = lane;   // the [H][W][N][C] store's box walks (sample, column) in the rows' own order
+    const float os = out_scale_of(p);
     uint32_t tcount = 0;
     for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
       const Tile tile = decode_tile(p, t);
@@ -517,6 +531,7 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
           if (Q > 0) {
             tmem_ld_32x32b_x16(taddr + c0 + 16 * i, v);
             tmem_ld_wait();
+            if (p.kind_fp4 == 2) scale16(v, os);
           } else {
 #pragma unroll
             for (int j = 0; j < 16; ++j) v[j] = 0u;
@@ -556,20 +571,23 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
 
 // EPI: -1 = fp32 output (the three fp32 epilogue roles, chosen at run time: an instance per role was measured, no
 // change); 0..4 = quantizing epilogue emitting element format EPI
-template <int MODE, int KB, bool FP4, int EPI = -1>
+template <int MODE, int KB, int KIND, int EPI = -1>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_out,
                const ConvTcParams p) {
   constexpr int G = 128 / KB;          // chunks per stage
   constexpr int APC = KB / 32;         // MMA K-atoms (32 bytes) per chunk
-  constexpr int SPA = FP4 ? 2 : 1;     // scale bytes per atom
+  constexpr bool FP4 = KIND != 0;
+  constexpr int SPA = spa_of_kind(KIND);     // scale bytes per atom
+  constexpr int SFA_B = KIND == 2 ? SFA_BYTES_NV : SFA_BYTES, SFB_B = KIND == 2 ? SFB_BYTES_NV : SFB_BYTES;
+  constexpr int SFC = KIND == 2 ? SF_COLS_NV : SF_COLS, SFB_OFF = KIND == 2 ? 16 : 8;   // TMEM columns per stage; B-side offset in them
   constexpr int BPC = APC * SPA;       // scale bytes per chunk: 1, 2, 4 or 8
   constexpr int LAYOUT = KB == 128 ? 2 : (KB == 64 ? 4 : 6);
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int b_stage_bytes = p.BN * 128;
-  const int stage_bytes = A_STAGE_BYTES + b_stage_bytes + SFA_BYTES + SFB_BYTES;
+  const int stage_bytes = A_STAGE_BYTES + b_stage_bytes + SFA_B + SFB_B;
   float* staging = reinterpret_cast<float*>(smem + (size_t)p.stages * stage_bytes);   // TMA-store epilogue only
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * stage_bytes + (p.tma_store ? EPI_STAGING_BYTES : 0));
   uint64_t* empty = full + p.stages;
@@ -654,7 +672,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
               if (lkind == 2) {
                 mbar_arrive_expect_tx(&full[s], 512u * SPA * (1 + atoms_b));
                 bulk_load(sb + b_stage_bytes, sfa_src, 512 * SPA, &full[s]);
-                bulk_load(sb + b_stage_bytes + SFA_BYTES, sfb_src, 512 * SPA * atoms_b, &full[s]);
+                bulk_load(sb + b_stage_bytes + SFA_B, sfb_src, 512 * SPA * atoms_b, &full[s]);
               } else {
                 mbar_arrive_expect_tx(&full[s], (uint32_t)nch * row_bytes);
 #pragma unroll
@@ -685,7 +703,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const uint32_t b_chunk16 = (uint32_t)(p.BN * KB) >> 4;
       const uint64_t sf_desc = smem_desc_base(0, 128, 0);
       const uint64_t sfa_desc0 = smem_desc(sf_desc, smem_u32(smem + A_STAGE_BYTES + b_stage_bytes));
-      const uint64_t sfb_desc0 = smem_desc(sf_desc, smem_u32(smem + A_STAGE_BYTES + b_stage_bytes + SFA_BYTES));
+      const uint64_t sfb_desc0 = smem_desc(sf_desc, smem_u32(smem + A_STAGE_BYTES + b_stage_bytes + SFA_B));
       uint32_t idesc_id[4];
 #pragma unroll
       for (int i = 0; i < 4; ++i) idesc_id[i] = idesc_with_sf_ids(p.idesc, i, i);
@@ -709,7 +727,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (!mbar_wait(self_cp ? &full[s] : &sffull[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
           tc_fence_after_sync();
           const uint32_t so = s * stage16;
-          const uint32_t sfa_t = sf_base + s * SF_COLS, sfb_t = sfa_t + 8;
+          const uint32_t sfa_t = sf_base + s * SFC, sfb_t = sfa_t + SFB_OFF;
           const int natoms = min(G, Q - q0) * APC;
           if (elect_one()) {
             if (self_cp) {
@@ -728,7 +746,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const uint64_t ad = a_desc0 + so + c * ((128 * KB) >> 4) + ja * 2;
                 const uint64_t bd = b_desc0 + so + c * b_chunk16 + ja * 2;
                 const int g = (a * SPA) >> 2, id = (a * SPA) & 3;
-                if (FP4) mma_mxf4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accu);
+                if (KIND == 2) mma_nvf4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accu);
+                else if (KIND == 1) mma_mxf4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accu);
                 else mma_mxf8f6f4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accu);
                 accu = 1;
               }
@@ -754,7 +773,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       const uint32_t sf_base = tmem + p.n_acc * p.BN;
       const uint32_t stage16 = (uint32_t)stage_bytes >> 4;
       const uint64_t sfa_desc0 = smem_desc(sf_desc, smem_u32(smem + A_STAGE_BYTES + b_stage_bytes));
-      const uint64_t sfb_desc0 = smem_desc(sf_desc, smem_u32(smem + A_STAGE_BYTES + b_stage_bytes + SFA_BYTES));
+      const uint64_t sfb_desc0 = smem_desc(sf_desc, smem_u32(smem + A_STAGE_BYTES + b_stage_bytes + SFA_B));
       uint32_t s = 0, phase = 0;
       bool alive = true;
       for (unsigned i = 0, t; (t = tile_of_iter(p, i)) < total && alive && !*abort_flag; ++i) {
@@ -766,7 +785,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           if (!mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; alive = false; break; }
           tc_fence_after_sync();
           const uint32_t so = s * stage16;
-          const uint32_t sfa_t = sf_base + s * SF_COLS, sfb_t = sfa_t + 8;
+          const uint32_t sfa_t = sf_base + s * SFC, sfb_t = sfa_t + SFB_OFF;
           if (elect_one()) {
 #pragma unroll
             for (int g = 0; g < SPA; ++g) {
@@ -1159,8 +1178,9 @@ conv_tc_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_cons
 // row r of the tile at byte (r % 32) * 16 + (r / 32) * 4, four consecutive K-blocks per 32-bit word --
 // from the compact tile scales.  A-side chunks exist per tile (without its channel index), B-side
 // chunks per (stride class, channel tile).
-template <int MODE, int KB, bool FP4>
+template <int MODE, int KB, int KIND>
 __global__ void __launch_bounds__(256) expand_conv_scales_kernel(const ConvTcParams p, unsigned n_tile_m) {
+  constexpr bool FP4 = KIND != 0;
   pdl_wait();
   if (p.wt_fused && blockIdx.x >= p.expand_blocks) {
     // W -> W^T codes, one 32 x 32 (c_in, c_out) block of one tap per thread block (the work of weight_transpose_kernel)
@@ -1196,12 +1216,119 @@ __global__ void __launch_bounds__(256) expand_conv_scales_kernel(const ConvTcPar
     }
     return;
   }
-  constexpr int G = 128 / KB, APC = KB / 32, SPA = FP4 ? 2 : 1, BPC = APC * SPA;
+  constexpr int G = 128 / KB, APC = KB / 32, SPA = KIND == 1 ? 2 : 1, BPC = APC * SPA;
   const int lane = threadIdx.x & 31;
   const unsigned wid = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const unsigned nA = conv_tc_sfa_chunks(p);
   const unsigned nB = (unsigned)(p.classes * p.tiles_c * p.max_stages);
   const int atoms_b = (p.BN + 127) / 128;
+  if (KIND == 2) {
+    // One E4M3 scale per 16 x 16 block (Eq. 5): a row's four scale bytes of an MMA (64 elements of K) are four consecutive
+    // bytes of its 16-row block's scale line, and each MMA of a stage (group ga = chunk * APC + atom) gets a 512-byte
+    // chunk of its own ([32 rows][row quarter][4 bytes]).  A: [Hs][Ws][ceil(N/16)][K/16]; B: [ceil(rows/16)][taps][K/16],
+    // or, for the input gradient, gathered from the stored W scales [ceil(C_out/16)][taps][C_in_p/16] with K = C_out.
+    const int Kb16 = p.Kblocks * 2, Nt16 = (p.N + 15) >> 4;
+    if (wid < nA) {
+      const unsigned tm = wid / (unsigned)p.max_stages;
+      const int st = (int)(wid - tm * p.max_stages);
+      const Tile tile = tile_of_m_index(p, tm);
+      TapWalk<MODE> tw;
+      tw.init(p, tile);
+      const int Q = tw.chunks(p);
+      if (st * G >= Q) return;
+      const int wstep = MODE == MQ_OP_FWD ? p.sw : 1;
+      uint32_t val[4][4];
+#pragma unroll
+      for (int ga = 0; ga < 4; ++ga)
+#pragma unroll
+        for (int j = 0; j < 4; ++j) val[ga][j] = 0u;
+#pragma unroll
+      for (int c = 0; c < G; ++c) {
+        const int q = st * G + c;
+        if (q < Q) {
+          ChunkPos pos;
+          const int per_row = tw.nkw * p.cpt;
+          pos.ia = q / per_row;
+          const int rem = q - pos.ia * per_row;
+          pos.ib = rem / p.cpt;
+          pos.cc = rem - pos.ib * p.cpt;
+          const int hs = src_h(tw, pos), ws0 = src_w0(tw, pos);
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const int r = 32 * j + lane;
+            const int tw_ = r & (p.TW - 1), tn = r >> p.lgTW;
+            const int n = tile.n0 + tn, ws = ws0 + tw_ * wstep;
+            if (n < p.N && hs >= 0 && hs < p.Hs && ws >= 0 && ws < p.Ws) {
+              const uint8_t* rowp = p.a_scales + (((long long)hs * p.Ws + ws) * Nt16 + (n >> 4)) * Kb16 + pos.cc * (4 * APC);
+#pragma unroll
+              for (int ja = 0; ja < APC; ++ja) val[c * APC + ja][j] = __ldg(reinterpret_cast<const unsigned int*>(rowp + 4 * ja));
+            }
+          }
+        }
+      }
+      uint8_t* dst = p.sfa_img + (size_t)wid * (512 * 4) + lane * 16;
+#pragma unroll
+      for (int ga = 0; ga < 4; ++ga) *reinterpret_cast<uint4*>(dst + ga * 512) = make_uint4(val[ga][0], val[ga][1], val[ga][2], val[ga][3]);
+    } else if (wid < nA + nB) {
+      unsigned idx = wid - nA;
+      const int st = (int)(idx % (unsigned)p.max_stages); idx /= (unsigned)p.max_stages;
+      const int ct = (int)(idx % (unsigned)p.tiles_c);
+      Tile tile;
+      tile.cls = (int)(idx / (unsigned)p.tiles_c); tile.ct = ct; tile.c0 = ct * p.BN; tile.w0 = 0; tile.n0 = 0; tile.h = 0;
+      TapWalk<MODE> tw;
+      tw.init(p, tile);
+      const int Q = tw.chunks(p);
+      if (st * G >= Q) return;
+      const int taps_all = p.Kh * p.Kw;
+      uint32_t val[4][8];
+#pragma unroll
+      for (int ga = 0; ga < 4; ++ga)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) val[ga][j] = 0u;
+#pragma unroll
+      for (int c = 0; c < G; ++c) {
+        const int q = st * G + c;
+        if (q < Q) {
+          ChunkPos pos;
+          const int per_row = tw.nkw * p.cpt;
+          pos.ia = q / per_row;
+          const int rem = q - pos.ia * per_row;
+          pos.ib = rem / p.cpt;
+          pos.cc = rem - pos.ib * p.cpt;
+          const int tap = tap_index(tw, pos);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            const int row = tile.c0 + 32 * j + lane;
+            if (j < 4 * atoms_b && 32 * j < p.BN) {
+              if (p.wt_fused) {
+                if (row < p.wt_Cp) {
+                  const int Cb_w = p.wt_Cp >> 4;
+#pragma unroll
+                  for (int ja = 0; ja < APC; ++ja) {
+                    unsigned w = 0;
+#pragma unroll
+                    for (int kb = 0; kb < 4; ++kb)
+                      w |= (unsigned)__ldg(p.wt_sc_in + ((long long)(pos.cc * (4 * APC) + 4 * ja + kb) * taps_all + tap) * Cb_w + (row >> 4)) << (8 * kb);
+                    val[c * APC + ja][j] = w;
+                  }
+                }
+              } else if (row < p.b_rows_total) {
+                const uint8_t* rowp = p.b_scales + ((long long)(row >> 4) * taps_all + tap) * Kb16 + pos.cc * (4 * APC);
+#pragma unroll
+                for (int ja = 0; ja < APC; ++ja) val[c * APC + ja][j] = __ldg(reinterpret_cast<const unsigned int*>(rowp + 4 * ja));
+              }
+            }
+          }
+        }
+      }
+      uint8_t* dst = p.sfb_img + (size_t)(wid - nA) * (512 * 4 * atoms_b) + lane * 16;
+#pragma unroll
+      for (int ga = 0; ga < 4; ++ga)
+        for (int a = 0; a < atoms_b; ++a)
+          *reinterpret_cast<uint4*>(dst + (ga * atoms_b + a) * 512) = make_uint4(val[ga][4 * a], val[ga][4 * a + 1], val[ga][4 * a + 2], val[ga][4 * a + 3]);
+    }
+    return;
+  }
   if (p.halo && wid >= nA + nB) {
     // weight tile images for the whole-tile variant: one 16-byte chunk per thread
     const int taps_all = p.Kh * p.Kw;
@@ -1421,11 +1548,11 @@ bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const ui
 }
 
 size_t conv_tc_smem_bytes(const ConvTcParams& p) {
-  const size_t stage = A_STAGE_BYTES + (size_t)p.BN * 128 + SFA_BYTES + SFB_BYTES;
+  const size_t stage = A_STAGE_BYTES + (size_t)p.BN * 128 + (p.kind_fp4 == 2 ? SFA_BYTES_NV + SFB_BYTES_NV : SFA_BYTES + SFB_BYTES);
   return 1024 + (size_t)p.stages * stage + (p.tma_store ? EPI_STAGING_BYTES : 0) + (3 * (size_t)p.stages + 4) * 8 + 64 + (p.mx_out ? 288 : 0);
 }
 
-template <int MODE, int KB, bool FP4, int EPI = -1>
+template <int MODE, int KB, int FP4, int EPI = -1>
 cudaError_t launch_conv_tc_inst(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_out, cudaStream_t s) {
   static bool attr_set = false;
   const size_t smem = conv_tc_smem_bytes(p);
@@ -1442,13 +1569,13 @@ cudaError_t launch_conv_tc_inst(const ConvTcParams& p, const CUtensorMap& map_a,
 }
 
 size_t conv_tc_sfa_bytes(const ConvTcParams& p) {
-  return (size_t)conv_tc_sfa_chunks(p) * 512 * (p.kind_fp4 ? 2 : 1);
+  return (size_t)conv_tc_sfa_chunks(p) * 512 * spa_of_kind(p.kind_fp4);
 }
 size_t conv_tc_sfb_bytes(const ConvTcParams& p) {
-  return (size_t)p.classes * p.tiles_c * p.max_stages * 512 * (p.kind_fp4 ? 2 : 1) * ((p.BN + 127) / 128);
+  return (size_t)p.classes * p.tiles_c * p.max_stages * 512 * spa_of_kind(p.kind_fp4) * ((p.BN + 127) / 128);
 }
 
-template <int MODE, int KB, bool FP4>
+template <int MODE, int KB, int FP4>
 cudaError_t launch_expand_inst(const ConvTcParams& p, cudaStream_t s) {
   const unsigned n_tile_m = (unsigned)(p.total_tiles / p.tiles_c);
   unsigned long long warps = (unsigned long long)conv_tc_sfa_chunks(p) + (unsigned long long)p.classes * p.tiles_c * p.max_stages;
@@ -1465,11 +1592,13 @@ cudaError_t launch_expand_inst(const ConvTcParams& p, cudaStream_t s) {
 }
 
 cudaError_t launch_expand_conv_scales(const ConvTcParams& p, cudaStream_t s) {
-#define MQ_TC_CASE(M, K, F) if (p.mode == M && p.KB == K && (p.kind_fp4 != 0) == F) return launch_expand_inst<M, K, F>(p, s)
-  MQ_TC_CASE(MQ_OP_FWD, 128, false); MQ_TC_CASE(MQ_OP_FWD, 64, false); MQ_TC_CASE(MQ_OP_FWD, 32, false);
-  MQ_TC_CASE(MQ_OP_FWD, 128, true);  MQ_TC_CASE(MQ_OP_FWD, 64, true);  MQ_TC_CASE(MQ_OP_FWD, 32, true);
-  MQ_TC_CASE(MQ_OP_BWD_DATA, 128, false); MQ_TC_CASE(MQ_OP_BWD_DATA, 64, false); MQ_TC_CASE(MQ_OP_BWD_DATA, 32, false);
-  MQ_TC_CASE(MQ_OP_BWD_DATA, 128, true);  MQ_TC_CASE(MQ_OP_BWD_DATA, 64, true);  MQ_TC_CASE(MQ_OP_BWD_DATA, 32, true);
+#define MQ_TC_CASE(M, K, F) if (p.mode == M && p.KB == K && p.kind_fp4 == F) return launch_expand_inst<M, K, F>(p, s)
+  MQ_TC_CASE(MQ_OP_FWD, 128, 0); MQ_TC_CASE(MQ_OP_FWD, 64, 0); MQ_TC_CASE(MQ_OP_FWD, 32, 0);
+  MQ_TC_CASE(MQ_OP_FWD, 128, 1); MQ_TC_CASE(MQ_OP_FWD, 64, 1); MQ_TC_CASE(MQ_OP_FWD, 32, 1);
+  MQ_TC_CASE(MQ_OP_FWD, 128, 2); MQ_TC_CASE(MQ_OP_FWD, 64, 2); MQ_TC_CASE(MQ_OP_FWD, 32, 2);
+  MQ_TC_CASE(MQ_OP_BWD_DATA, 128, 0); MQ_TC_CASE(MQ_OP_BWD_DATA, 64, 0); MQ_TC_CASE(MQ_OP_BWD_DATA, 32, 0);
+  MQ_TC_CASE(MQ_OP_BWD_DATA, 128, 1); MQ_TC_CASE(MQ_OP_BWD_DATA, 64, 1); MQ_TC_CASE(MQ_OP_BWD_DATA, 32, 1);
+  MQ_TC_CASE(MQ_OP_BWD_DATA, 128, 2); MQ_TC_CASE(MQ_OP_BWD_DATA, 64, 2); MQ_TC_CASE(MQ_OP_BWD_DATA, 32, 2);
 #undef MQ_TC_CASE
   return cudaErrorInvalidValue;
 }
@@ -1583,14 +1712,14 @@ cudaError_t launch_recode4_e4m3(const uint8_t* in, uint8_t* out, size_t n_out, c
 cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_out, cudaStream_t s) {
   if (p.total_tiles <= 0 || p.total_tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
   if (p.halo) {
-#define MQ_TC_HCASE(M, K, F) if (p.mode == M && p.KB == K && (p.kind_fp4 != 0) == F) return launch_conv_tc_halo_inst<M, K, F>(p, map_a, map_out, map_w, s)
+#define MQ_TC_HCASE(M, K, F) if (p.mode == M && p.KB == K && p.kind_fp4 == (F ? 1 : 0)) return launch_conv_tc_halo_inst<M, K, F>(p, map_a, map_out, map_w, s)
     MQ_TC_HCASE(MQ_OP_FWD, 64, false); MQ_TC_HCASE(MQ_OP_FWD, 32, false); MQ_TC_HCASE(MQ_OP_FWD, 64, true); MQ_TC_HCASE(MQ_OP_FWD, 32, true);
     MQ_TC_HCASE(MQ_OP_BWD_DATA, 64, false); MQ_TC_HCASE(MQ_OP_BWD_DATA, 32, false); MQ_TC_HCASE(MQ_OP_BWD_DATA, 64, true); MQ_TC_HCASE(MQ_OP_BWD_DATA, 32, true);
 #undef MQ_TC_HCASE
     return cudaErrorInvalidValue;
   }
   if (p.mx_out) {   // the quantizing epilogue: one kernel instance per emitted format
-#define MQ_TC_MX(M, K, F, E) if (p.mode == M && p.KB == K && (p.kind_fp4 != 0) == F && p.mx_fmt == E) return launch_conv_tc_inst<M, K, F, E>(p, map_a, map_w, map_out, s)
+#define MQ_TC_MX(M, K, F, E) if (p.mode == M && p.KB == K && p.kind_fp4 == (F ? 1 : 0) && p.mx_fmt == E) return launch_conv_tc_inst<M, K, F, E>(p, map_a, map_w, map_out, s)
 #define MQ_TC_MX5(M, K, F) MQ_TC_MX(M, K, F, MQ_E4M3); MQ_TC_MX(M, K, F, MQ_E5M2); MQ_TC_MX(M, K, F, MQ_E2M1); MQ_TC_MX(M, K, F, MQ_E3M2); MQ_TC_MX(M, K, F, MQ_E2M3)
     MQ_TC_MX5(MQ_OP_FWD, 128, false); MQ_TC_MX5(MQ_OP_FWD, 64, false); MQ_TC_MX5(MQ_OP_FWD, 32, false);
     MQ_TC_MX5(MQ_OP_FWD, 128, true);  MQ_TC_MX5(MQ_OP_FWD, 64, true);  MQ_TC_MX5(MQ_OP_FWD, 32, true);
@@ -1600,11 +1729,13 @@ cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, cons
 #undef MQ_TC_MX
     return cudaErrorInvalidValue;
   }
-#define MQ_TC_CASE(M, K, F) if (p.mode == M && p.KB == K && (p.kind_fp4 != 0) == F) return launch_conv_tc_inst<M, K, F>(p, map_a, map_w, map_out, s)
-  MQ_TC_CASE(MQ_OP_FWD, 128, false); MQ_TC_CASE(MQ_OP_FWD, 64, false); MQ_TC_CASE(MQ_OP_FWD, 32, false);
-  MQ_TC_CASE(MQ_OP_FWD, 128, true);  MQ_TC_CASE(MQ_OP_FWD, 64, true);  MQ_TC_CASE(MQ_OP_FWD, 32, true);
-  MQ_TC_CASE(MQ_OP_BWD_DATA, 128, false); MQ_TC_CASE(MQ_OP_BWD_DATA, 64, false); MQ_TC_CASE(MQ_OP_BWD_DATA, 32, false);
-  MQ_TC_CASE(MQ_OP_BWD_DATA, 128, true);  MQ_TC_CASE(MQ_OP_BWD_DATA, 64, true);  MQ_TC_CASE(MQ_OP_BWD_DATA, 32, true);
+#define MQ_TC_CASE(M, K, F) if (p.mode == M && p.KB == K && p.kind_fp4 == F) return launch_conv_tc_inst<M, K, F>(p, map_a, map_w, map_out, s)
+  MQ_TC_CASE(MQ_OP_FWD, 128, 0); MQ_TC_CASE(MQ_OP_FWD, 64, 0); MQ_TC_CASE(MQ_OP_FWD, 32, 0);
+  MQ_TC_CASE(MQ_OP_FWD, 128, 1); MQ_TC_CASE(MQ_OP_FWD, 64, 1); MQ_TC_CASE(MQ_OP_FWD, 32, 1);
+  MQ_TC_CASE(MQ_OP_FWD, 128, 2); MQ_TC_CASE(MQ_OP_FWD, 64, 2); MQ_TC_CASE(MQ_OP_FWD, 32, 2);
+  MQ_TC_CASE(MQ_OP_BWD_DATA, 128, 0); MQ_TC_CASE(MQ_OP_BWD_DATA, 64, 0); MQ_TC_CASE(MQ_OP_BWD_DATA, 32, 0);
+  MQ_TC_CASE(MQ_OP_BWD_DATA, 128, 1); MQ_TC_CASE(MQ_OP_BWD_DATA, 64, 1); MQ_TC_CASE(MQ_OP_BWD_DATA, 32, 1);
+  MQ_TC_CASE(MQ_OP_BWD_DATA, 128, 2); MQ_TC_CASE(MQ_OP_BWD_DATA, 64, 2); MQ_TC_CASE(MQ_OP_BWD_DATA, 32, 2);
 #undef MQ_TC_CASE
   return cudaErrorInvalidValue;
 }

@@ -16,7 +16,10 @@ namespace mq {
 struct ConvTcParams {
   int mode;             // MQ_OP_FWD or MQ_OP_BWD_DATA
   int line;             // 1: line-block scales (forward only): a_scales [Hs][Ws][N][Kblocks], b_scales [rows][taps][Kblocks]
-  int kind_fp4;         // 1: both operands E2M1 (kind::mxf4), 0: 8-bit formats (kind::mxf8f6f4)
+  int kind_fp4;         // 0: 8-bit formats (kind::mxf8f6f4, one E8M0 scale per 32 elements); 1: both operands E2M1 (kind::mxf4, E8M0 per 32);
+                        // 2: both E2M1 with one E4M3 scale per 16 x 16 block and an fp32 scale per tensor (kind::mxf4nvf4, Eq. 4-6)
+  const float* a_tscale;    // kind 2: the two tensors' fp32 scales (device); the epilogue multiplies the accumulator by their product
+  const float* b_tscale;
   uint32_t idesc;       // instruction descriptor without scale ids
   int KB;               // bytes of K per row per TMA box: 128, 64 or 32 (= swizzle span)
   int G;                // boxes (chunks) per pipeline stage = 128 / KB
@@ -105,6 +108,8 @@ cudaError_t launch_weight_transpose(const uint8_t* w_codes, const uint8_t* w_sca
 // Parameters of the tensor-core weight-gradient kernel (see mq_wgrad_tc.cu).
 enum { MQ_WG_FP8 = 0, MQ_WG_FP4_PIXEL = 1, MQ_WG_FP4_FLAT = 2 };
 struct WgradTcParams {
+  int kind;             // 0: 8-bit operands (kind::mxf8f6f4); 1: E2M1 with E8M0 tile scales (kind::mxf4); 2: E2M1 with E4M3 scales per 16 x 16
+                        // block (kind::mxf4nvf4; the tensors' fp32 scales are applied by bwd_weight_reduce) - modes FP4_PIXEL / FP4_FLAT
   int mode;             // MQ_WG_FP8: 8-bit operands as stored (MN-major TMA boxes); MQ_WG_FP4_PIXEL: E2M1 re-laid
                         // [pixel][c][n], one TMA box per pixel; MQ_WG_FP4_FLAT: stride 1, E2M1 re-laid as contiguous
                         // pre-swizzled pieces over the zero-padded, flattened pixel axis (bulk copies)
@@ -156,7 +161,9 @@ cudaError_t launch_fp4_to_n_major(const uint8_t* in, uint8_t* out, int P, int N,
 cudaError_t launch_wgrad_flat_prep(const WgradTcParams& p, const uint8_t* x_codes, uint8_t* xt, int P_b, const uint8_t* g_codes, uint8_t* gt, int P_a,
                                    cudaStream_t s);
 // Adds the split partial sums in a fixed order and writes G_W in its final layout.
-cudaError_t launch_bwd_weight_reduce(const float* partial, float* out, const Geom& g, int splits, int layout, cudaStream_t s);
+// ta, tb (device, may be null): fp32 tensor scales whose product the sums are multiplied by
+cudaError_t launch_bwd_weight_reduce(const float* partial, float* out, const Geom& g, int splits, int layout, cudaStream_t s, const float* ta = nullptr,
+                                     const float* tb = nullptr);
 
 // Host: encode a tiled tensor map over bytes (or over fp32 elements when f32 is set: dims and box then count
 // elements).  Strides in bytes (stride[0] implied contiguous), fastest dimension first.  l2_promotion_bytes: 0, 64, 128, 256,

@@ -41,6 +41,73 @@ __device__ __forceinline__ void stage_block(const WgradTcParams& p, int st, int 
   }
 }
 
+// ---- scale expansion, E4M3 scales per 16 x 16 block (kind 2): one warp per 2048-byte chunk of 128 rows --------------
+// A stage is 16 K-blocks of 16 samples; MMA ga of the stage reads K-blocks 4 ga .. 4 ga + 3, four bytes per row, from
+// its own 512-byte group [32 rows][row quarter][4 bytes].  Row r of quarter jj is channel 128 tile + 32 jj + r, whose
+// scale line is that of its 16-channel block.  G_Y scales [Ho][Wo][ceil(N/16)][C_out_p/16], X scales [H][W][ceil(N/16)][C_in_p/16].
+__device__ __forceinline__ void expand_wgrad_scales_nv_body(const WgradTcParams& p, unsigned block) {
+  const int lane = threadIdx.x & 31;
+  const long long wid = (long long)block * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  const int taps = p.Kh * p.Kw;
+  const long long nA = (long long)p.m_tiles128 * p.stages_total;
+  const int groups = taps / p.TG;
+  const long long nB = (long long)p.cb_tiles * groups * p.stages_total * p.NB;
+  if (wid >= nA + nB) return;
+  const int Nt16 = (p.N + 15) >> 4, Cot16 = p.Cot * 2, Ct16 = p.Ct * 2;
+  uint32_t val[4][4];   // [MMA of the stage][row quarter]
+#pragma unroll
+  for (int ga = 0; ga < 4; ++ga)
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) val[ga][jj] = 0u;
+  uint8_t* dst;
+  if (wid < nA) {
+    const int mt = (int)(wid / p.stages_total), st = (int)(wid - (long long)mt * p.stages_total);
+#pragma unroll 1
+    for (int b16 = 0; b16 < 16; ++b16) {
+      int ho, wo, nb;
+      stage_block(p, st, b16 >> 1, ho, wo, nb);
+      const int nb16 = 2 * nb + (b16 & 1);
+      if (ho < p.Ho && wo < p.Wo && nb16 < Nt16) {
+        const uint8_t* line = p.g_scales + (((long long)ho * p.Wo + wo) * Nt16 + nb16) * Cot16;
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+          const int cob16 = (mt * 128 + 32 * jj + lane) >> 4;
+          if (cob16 < Cot16) val[b16 >> 2][jj] |= (uint32_t)__ldg(line + cob16) << (8 * (b16 & 3));
+        }
+      }
+    }
+    dst = p.sfa_img + wid * 2048;
+  } else {
+    long long idx = wid - nA;
+    const int c = (int)(idx % p.NB); idx /= p.NB;
+    const int st = (int)(idx % p.stages_total); idx /= p.stages_total;
+    const int tg = (int)(idx % groups); const int cb = (int)(idx / groups);
+#pragma unroll 1
+    for (int b16 = 0; b16 < 16; ++b16) {
+      int ho, wo, nb;
+      stage_block(p, st, b16 >> 1, ho, wo, nb);
+      const int nb16 = 2 * nb + (b16 & 1);
+      if (ho < p.Ho && wo < p.Wo && nb16 < Nt16) {
+#pragma unroll
+        for (int jj = 0; jj < 4; ++jj) {
+          // B rows of a tap group: tap-in-group major, input channel minor; chunk c holds rows [128c, 128c + 128)
+          const int row = c * 128 + 32 * jj + lane;
+          const int tj = row / p.b_rows, rj = row - tj * p.b_rows;
+          const int tap = tg * p.TG + tj;
+          const int kh = tap / p.Kw, kw = tap - kh * p.Kw;
+          const int cib16 = (cb * p.b_rows + rj) >> 4;
+          const int h = ho * p.sh + kh - p.ph, w = wo * p.sw + kw - p.pw;
+          if (tj < p.TG && cib16 < Ct16 && h >= 0 && h < p.H && w >= 0 && w < p.W)
+            val[b16 >> 2][jj] |= (uint32_t)__ldg(p.x_scales + (((long long)h * p.W + w) * Nt16 + nb16) * Ct16 + cib16) << (8 * (b16 & 3));
+        }
+      }
+    }
+    dst = p.sfb_img + (wid - nA) * 2048;
+  }
+#pragma unroll
+  for (int ga = 0; ga < 4; ++ga) *reinterpret_cast<uint4*>(dst + ga * 512 + lane * 16) = make_uint4(val[ga][0], val[ga][1], val[ga][2], val[ga][3]);
+}
+
 // ---- scale expansion: one warp per 512*SPA-byte chunk ----------------------------------------------------
 template <bool FP4>
 __device__ __forceinline__ void expand_wgrad_scales_body(const WgradTcParams& p, unsigned block) {
@@ -124,6 +191,7 @@ __device__ __forceinline__ void expand_wgrad_scales_body(const WgradTcParams& p,
 // tile feeds Kw accumulators (Kw times less shared-memory traffic per FLOP than one tap per block).
 template <bool FP4>
 __global__ void __launch_bounds__(256) expand_wgrad_scales_kernel(const WgradTcParams p) { pdl_wait(); expand_wgrad_scales_body<FP4>(p, blockIdx.x); }
+__global__ void __launch_bounds__(256) expand_wgrad_scales_nv_kernel(const WgradTcParams p) { pdl_wait(); expand_wgrad_scales_nv_body(p, blockIdx.x); }
 
 //
 // CTA2 (8-bit operands, C_out and C_in >= 256): the two blocks of a cluster compute a 256 x 256 tile with
@@ -132,11 +200,14 @@ __global__ void __launch_bounds__(256) expand_wgrad_scales_kernel(const WgradTcP
 // 128 x 256 tile -- and the shared-memory operand path is what bounds these kernels.  The leader block's threads issue
 // the scale copies, MMAs and commits for the pair; the other block only loads, relays "my stage has landed" to the
 // leader's barrier, and stores its half of the result.
-template <bool FP4, bool CTA2>
+template <int KIND, bool CTA2>
 __global__ void __launch_bounds__(WG_THREADS, 1)
 wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_p,
                 const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb, const WgradTcParams p) {
-  constexpr int SPA = FP4 ? 2 : 1;     // scale bytes per MMA per row
+  constexpr bool FP4 = KIND != 0;
+  constexpr int SPA = KIND == 2 ? 4 : (KIND == 1 ? 2 : 1);     // scale bytes per MMA per row
+  constexpr int SFC_BYTES = KIND == 2 ? 2048 : 1024;           // shared-memory bytes of a 128-row scale chunk
+  constexpr uint32_t SFA_COLS = KIND == 2 ? 16u : 8u;          // TMEM columns of a 128-row scale chunk
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
   const int TG = p.TG;
@@ -172,7 +243,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
   const int st_end = (int)((long long)p.stages_total * (split + 1) / p.splits);
   const int nst = st_end - st_begin;
   const uint32_t acc_cols = (uint32_t)(TG * p.b_rows);  // accumulators first, then the per-stage scale buffers
-  const uint32_t sf_cols = 8u + 8u * (uint32_t)p.NB;
+  const uint32_t sf_cols = SFA_COLS * (1u + (uint32_t)p.NB);
   const bool has_b1 = p.mode == MQ_WG_FP8 && !CTA2 && p.b_rows > 128;   // a fifth loader: second X panel
 
   if (threadIdx.x == 0) {
@@ -252,11 +323,11 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           else if (kind == 1) tma_load_4d_pair(sb, &map_b, lbar, ci_ld, nrow, xw, xh);
           else {
             tma_load_2d_pair(ssf, &map_sfa, lbar, 0, sfa_row0 + i * (2 * SPA));
-            tma_load_2d_pair(ssf + 1024, &map_sfb, lbar, 0, (int)(xchunk * (2 * SPA * p.NB)));
+            tma_load_2d_pair(ssf + SFC_BYTES, &map_sfb, lbar, 0, (int)(xchunk * (2 * SPA * p.NB)));
           }
         } else if (kind == 3) {
           bulk_load(ssf, sfa_src + (size_t)i * (512 * SPA), 512 * SPA, bar);
-          bulk_load(ssf + 1024, FP4 ? sfb_src + (size_t)i * sfb_bytes : p.sfb_img + (size_t)xchunk * sfb_bytes, sfb_bytes, bar);
+          bulk_load(ssf + SFC_BYTES, FP4 ? sfb_src + (size_t)i * sfb_bytes : p.sfb_img + (size_t)xchunk * sfb_bytes, sfb_bytes, bar);
         } else if (p.mode == MQ_WG_FP4_FLAT) {
           if (kind == 0) bulk_load(sa, ga + (size_t)i * a_bytes, a_bytes, bar);
           else bulk_load(sb, gb + (size_t)i * b_step, b_bytes, bar);          // KPX + TG - 1 consecutive pixels
@@ -327,7 +398,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 #pragma unroll
         for (int m = 0; m < 2; ++m) {
           idesc_a[m][a] = idesc_with_sf_ids(idesc_n[m], id, id);
-          sfb_off[m][a] = 8 + 4 * (g * (uint32_t)p.NB + (m ? (uint32_t)(p.n0 >> 7) : 0u));
+          sfb_off[m][a] = SFA_COLS + 4 * (g * (uint32_t)p.NB + (m ? (uint32_t)(p.n0 >> 7) : 0u));
         }
       }
       const uint32_t d1 = tmem + (uint32_t)p.n0;
@@ -373,16 +444,18 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
 #pragma unroll 1
           for (int c = 0; c < p.NB; ++c)
 #pragma unroll
-            for (int g = 0; g < SPA; ++g) tmem_cp_32x128b_warpx4(sf_t + 8 + 4 * (g * p.NB + c), sfd + 64 + (c * SPA + g) * 32);
+            for (int g = 0; g < SPA; ++g) tmem_cp_32x128b_warpx4(sf_t + SFA_COLS + 4 * (g * p.NB + c), sfd + (SFC_BYTES >> 4) + (c * SPA + g) * 32);
         }
 #pragma unroll
         for (int a = 0; a < 4; ++a) {
           const uint32_t accu = a > 0 ? 1u : accumulate;
-          if (FP4) mma_mxf4(tmem, ad + ka16[a], bd + kb16[a], idesc_a[0][a], sf_t + sfa_off[a], sf_t + sfb_off[0][a], accu);
+          if (KIND == 2) mma_nvf4(tmem, ad + ka16[a], bd + kb16[a], idesc_a[0][a], sf_t + sfa_off[a], sf_t + sfb_off[0][a], accu);
+          else if (FP4) mma_mxf4(tmem, ad + ka16[a], bd + kb16[a], idesc_a[0][a], sf_t + sfa_off[a], sf_t + sfb_off[0][a], accu);
           else if (CTA2) mma_mxf8f6f4_2(tmem, ad + ka16[a], bd + kb16[a], idesc_a[0][a], sf_t + sfa_off[a], sf_t + sfb_off[0][a], accu);
           else mma_mxf8f6f4(tmem, ad + ka16[a], bd + kb16[a], idesc_a[0][a], sf_t + sfa_off[a], sf_t + sfb_off[0][a], accu);
           if (nm == 2) {   // the remaining n1 rows of a tap group's operand (flat mode only)
-            if (FP4) mma_mxf4(d1, ad + ka16[a], bd + row16_1 + kb16[a], idesc_a[1][a], sf_t + sfa_off[a], sf_t + sfb_off[1][a], accu);
+            if (KIND == 2) mma_nvf4(d1, ad + ka16[a], bd + row16_1 + kb16[a], idesc_a[1][a], sf_t + sfa_off[a], sf_t + sfb_off[1][a], accu);
+            else if (FP4) mma_mxf4(d1, ad + ka16[a], bd + row16_1 + kb16[a], idesc_a[1][a], sf_t + sfa_off[a], sf_t + sfb_off[1][a], accu);
             else mma_mxf8f6f4(d1, ad + ka16[a], bd + row16_1 + kb16[a], idesc_a[1][a], sf_t + sfa_off[a], sf_t + sfb_off[1][a], accu);
           }
         }
@@ -430,8 +503,8 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           for (int c = 0; c < p.NB; ++c) {     // B-side chunk c: rows [128c, 128c + 128) of the group's operand
 #pragma unroll
             for (int g = 0; g < SPA; ++g) {
-              if (CTA2) tmem_cp_32x128b_warpx4_2(sf_t + 8 + 4 * (g * p.NB + c), sf_desc0 + so + 64 + (c * SPA + g) * 32);
-              else tmem_cp_32x128b_warpx4(sf_t + 8 + 4 * (g * p.NB + c), sf_desc0 + so + 64 + (c * SPA + g) * 32);
+              if (CTA2) tmem_cp_32x128b_warpx4_2(sf_t + SFA_COLS + 4 * (g * p.NB + c), sf_desc0 + so + (SFC_BYTES >> 4) + (c * SPA + g) * 32);
+              else tmem_cp_32x128b_warpx4(sf_t + SFA_COLS + 4 * (g * p.NB + c), sf_desc0 + so + (SFC_BYTES >> 4) + (c * SPA + g) * 32);
             }
           }
           }
@@ -655,7 +728,8 @@ __global__ void __launch_bounds__(256) wgrad_flat_prep_kernel(const FlatArgs x, 
   if (blockIdx.x < x.blocks) { if (x.wide) fp4_to_flat_wide_body(x, blockIdx.x, x.blocks, flat_sm); else fp4_to_flat_body(x, blockIdx.x, x.blocks); }
   else if (blockIdx.x < x.blocks + gy.blocks) {
     if (gy.wide) fp4_to_flat_wide_body(gy, blockIdx.x - x.blocks, gy.blocks, flat_sm); else fp4_to_flat_body(gy, blockIdx.x - x.blocks, gy.blocks);
-  } else expand_wgrad_scales_body<true>(p, blockIdx.x - x.blocks - gy.blocks);
+  } else if (p.kind == 2) expand_wgrad_scales_nv_body(p, blockIdx.x - x.blocks - gy.blocks);
+  else expand_wgrad_scales_body<true>(p, blockIdx.x - x.blocks - gy.blocks);
 }
 
 }  // namespace
@@ -664,21 +738,23 @@ size_t wgrad_tc_smem_bytes(const WgradTcParams& p) { return 1024 + (size_t)p.sta
 
 cudaError_t launch_wgrad_tc(const WgradTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_p, const CUtensorMap& map_sfa,
                             const CUtensorMap& map_sfb, cudaStream_t s) {
-  static bool attr_set[3] = {false, false, false};
+  static bool attr_set[4] = {false, false, false, false};
   const size_t smem = wgrad_tc_smem_bytes(p);
-  const int f = p.cta2 ? 2 : (p.mode == MQ_WG_FP8 ? 0 : 1);
+  const int f = p.cta2 ? 2 : (p.mode == MQ_WG_FP8 ? 0 : (p.kind == 2 ? 3 : 1));
   if (!attr_set[f]) {
-    cudaError_t e = f == 2 ? cudaFuncSetAttribute(wgrad_tc_kernel<false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)
-                  : f == 1 ? cudaFuncSetAttribute(wgrad_tc_kernel<true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)
-                           : cudaFuncSetAttribute(wgrad_tc_kernel<false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = f == 2 ? cudaFuncSetAttribute(wgrad_tc_kernel<0, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)
+                  : f == 1 ? cudaFuncSetAttribute(wgrad_tc_kernel<1, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)
+                  : f == 3 ? cudaFuncSetAttribute(wgrad_tc_kernel<2, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024)
+                           : cudaFuncSetAttribute(wgrad_tc_kernel<0, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_set[f] = true;
   }
   const unsigned grid = (unsigned)(p.m_tiles * p.j_tiles * p.splits) * (p.cta2 ? 2u : 1u);
   count_launches(1);
-  if (f == 2) return launch_pdl_cluster(wgrad_tc_kernel<false, true>, dim3(grid), dim3(WG_THREADS), smem, s, 2u, map_a, map_b, map_p, map_sfa, map_sfb, p);
-  if (f == 1) return launch_pdl(wgrad_tc_kernel<true, false>, dim3(grid), dim3(WG_THREADS), smem, s, map_a, map_b, map_p, map_sfa, map_sfb, p);
-  return launch_pdl(wgrad_tc_kernel<false, false>, dim3(grid), dim3(WG_THREADS), smem, s, map_a, map_b, map_p, map_sfa, map_sfb, p);
+  if (f == 2) return launch_pdl_cluster(wgrad_tc_kernel<0, true>, dim3(grid), dim3(WG_THREADS), smem, s, 2u, map_a, map_b, map_p, map_sfa, map_sfb, p);
+  if (f == 1) return launch_pdl(wgrad_tc_kernel<1, false>, dim3(grid), dim3(WG_THREADS), smem, s, map_a, map_b, map_p, map_sfa, map_sfb, p);
+  if (f == 3) return launch_pdl(wgrad_tc_kernel<2, false>, dim3(grid), dim3(WG_THREADS), smem, s, map_a, map_b, map_p, map_sfa, map_sfb, p);
+  return launch_pdl(wgrad_tc_kernel<0, false>, dim3(grid), dim3(WG_THREADS), smem, s, map_a, map_b, map_p, map_sfa, map_sfb, p);
 }
 
 cudaError_t launch_expand_wgrad_scales(const WgradTcParams& p, cudaStream_t s) {
@@ -687,6 +763,7 @@ cudaError_t launch_expand_wgrad_scales(const WgradTcParams& p, cudaStream_t s) {
   const unsigned blocks = (unsigned)((warps + 7) / 8);
   count_launches(1);
   if (p.mode == MQ_WG_FP8) return launch_pdl(expand_wgrad_scales_kernel<false>, dim3(blocks), dim3(256), 0, s, p);
+  if (p.kind == 2) return launch_pdl(expand_wgrad_scales_nv_kernel, dim3(blocks), dim3(256), 0, s, p);
   return launch_pdl(expand_wgrad_scales_kernel<true>, dim3(blocks), dim3(256), 0, s, p);
 }
 

@@ -20,6 +20,13 @@ SHAPES = [
     ("k1", (36, 40, 6, 8, 72, 1, 1, 0)),
     ("few_samples", (5, 20, 8, 8, 24, 3, 1, 1)),
     ("wide", (32, 256, 4, 8, 288, 3, 1, 1)),
+    # layers whose forward and input-gradient GEMMs run on the tensor cores (K a multiple of 64 elements)
+    ("tc_c256", (48, 256, 6, 7, 256, 3, 1, 1)),       # 128-byte chunks, 256-channel tiles, three 16-sample blocks
+    ("tc_c128_s2", (40, 128, 9, 10, 128, 3, 2, 1)),   # 64-byte chunks, stride 2 (parity classes of the input gradient)
+    ("tc_c64_k1", (150, 64, 5, 4, 192, 1, 1, 0)),     # 32-byte chunks (four per stage), 1x1, ragged sample tile
+    ("tc_c512_k1", (32, 512, 3, 4, 512, 1, 1, 0)),    # two 128-byte chunks per tap
+    ("tc_n96", (96, 64, 6, 5, 128, 3, 1, 1)),         # three 32-sample tiles: the weight gradient's per-pixel mode (four K-blocks per pixel)
+    ("tc_n24", (24, 128, 5, 5, 64, 3, 1, 1)),         # fewer than 32 samples: a half-empty sample tile
 ]
 
 
@@ -65,6 +72,45 @@ def test_quantizer_im2col_and_gemms(name, shape, kinds):
         ref, ab = oracle.conv_bwd_weight(d, gh, xh)
         assert_gemm_close((dw if layout == mq.NCHW else dw.permute(0, 3, 1, 2)).contiguous(), ref, ab, f"{name} bwd_weight layout {layout}", GEMM_TOL)
     assert mq.last_device_status() == 0
+
+
+def test_tensor_core_and_cuda_core_routes_agree(knobs):
+    """The forward and input-gradient GEMMs of this format run on the tensor cores where the layer allows it
+    (kind::mxf4nvf4: E4M3 scales per 16 elements in tensor memory, the tensors' fp32 scales applied to the accumulator)
+    and on the CUDA-core kernels elsewhere; the same layer through both routes."""
+    d = inputs.conv_desc(48, 128, 7, 6, 192, 3, 1, 1)
+    src = (inputs.make_x(d, 75, "gauss"), inputs.make_w(d, 75), inputs.make_dy(d, 75, "gauss"))
+    gq = [mq.quantize_ts(d, r, dev(t)) for r, t in zip(ROLES, src)]
+    n0 = mq.kernel_launch_count()
+    y_tc, dx_tc = mq.conv_fwd(d, gq[0], gq[1]), mq.conv_bwd_data(d, gq[1], gq[2])
+    n_tc = mq.kernel_launch_count() - n0
+    knobs(MQ_TC_NO_TS16=1)
+    n0 = mq.kernel_launch_count()
+    y_cc, dx_cc = mq.conv_fwd(d, gq[0], gq[1]), mq.conv_bwd_data(d, gq[1], gq[2])
+    n_cc = mq.kernel_launch_count() - n0
+    assert mq.last_device_status() == 0
+    assert n_tc == 4 and n_cc == 2, (n_tc, n_cc)      # scale expansion + GEMM per call against one CUDA-core kernel per call
+    oq = [oracle.quantize_ts(d, r, t, B16) for r, t in zip(ROLES, src)]
+    xh, wh, gh = [oracle.dequant_ts(d, r, o[0], o[1], o[2], B16) for r, o in zip(ROLES, oq)]
+    ref, ab = oracle.conv_fwd(d, xh, wh)
+    assert_gemm_close(y_tc, ref, ab, "fwd tensor cores", GEMM_TOL)
+    assert_gemm_close(y_cc, ref, ab, "fwd CUDA cores", GEMM_TOL)
+    ref, ab = oracle.conv_bwd_data(d, wh, gh)
+    assert_gemm_close(dx_tc, ref, ab, "bwd_data tensor cores", GEMM_TOL)
+    assert_gemm_close(dx_cc, ref, ab, "bwd_data CUDA cores", GEMM_TOL)
+    # the weight gradient: contraction over the samples, the second direction of the same 16 x 16 blocks
+    n0 = mq.kernel_launch_count()
+    dw_cc = mq.conv_bwd_weight(d, gq[0], gq[2])
+    n_cc = mq.kernel_launch_count() - n0
+    knobs(MQ_TC_NO_TS16=0)
+    n0 = mq.kernel_launch_count()
+    dw_tc = mq.conv_bwd_weight(d, gq[0], gq[2])
+    n_tc = mq.kernel_launch_count() - n0
+    assert mq.last_device_status() == 0
+    assert n_cc == 2 and n_tc > 2, (n_cc, n_tc)       # CUDA cores: GEMM + reduction; tensor cores: re-layout / scale expansion launches as well
+    ref, ab = oracle.conv_bwd_weight(d, gh, xh)
+    assert_gemm_close(dw_tc, ref, ab, "bwd_weight tensor cores", GEMM_TOL)
+    assert_gemm_close(dw_cc, ref, ab, "bwd_weight CUDA cores", GEMM_TOL)
 
 
 def test_tensor_maximum_from_an_earlier_step_and_stochastic_rounding():
