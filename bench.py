@@ -33,7 +33,8 @@ import numpy as np  # noqa: E402
 from paper_2609_28358_b200 import inputs  # noqa: E402
 
 DEFAULT_WORKLOAD = "cfg5_e4m3_k3s1_c512_hw56"
-MORE_WORKLOADS = ("cfg5_e2m1_k3s1_c512_hw56", "cfg4_3x3", "config2")
+# a name + "+ts16": the same layer in the paper's own number format (fp32 tensor scale, E4M3 scale per 16 x 16 block, E2M1; Eq. 4-6)
+MORE_WORKLOADS = ("cfg5_e2m1_k3s1_c512_hw56", "cfg5_e2m1_k3s1_c512_hw56+ts16", "cfg4_3x3", "config2")
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # published dense figures (NVIDIA's B200 / HGX B200 data sheet, per GPU, without sparsity): context beside the measured roofs
 PUBLISHED = {"hbm_gbs": 7700.0, "tensor_tflops": {8: 4500.0, 4: 9000.0}}
@@ -56,8 +57,17 @@ NCU_TRAFFIC = {
 }
 
 
+class _WorkloadTable(dict):
+    """name -> layer; a "+ts16" suffix selects the number format, not the layer"""
+
+    def __missing__(self, name):
+        if name.endswith("+ts16") and name[:-5] in self:
+            return self[name[:-5]]
+        raise KeyError(name)
+
+
 def workloads():
-    w = {}
+    w = _WorkloadTable()
     for cfg in ("config1", "config2", "config4"):
         for l in inputs.CONFIGS[cfg]():
             w[l.name] = l
@@ -143,6 +153,8 @@ class Workload:
         self.name, self.layer = name, layer
         d = self.d = layer.desc
         self.fmts = fmts = (layer.fmt_x, layer.fmt_w, layer.fmt_dy)
+        blk = self.block = mq.TS16 if name.endswith("+ts16") else mq.TILE32
+        assert blk == mq.TILE32 or all(f == mq.E2M1 for f in fmts), "the paper's own format has E2M1 elements"
         roles = (mq.ROLE_X, mq.ROLE_W, mq.ROLE_DY)
         seed = layer.seed + 1000 * rank
         self.host = (inputs.make_x(d, seed, layer.x_kind), inputs.make_w(d, layer.seed, layer.w_kind), inputs.make_dy(d, seed, layer.dy_kind))
@@ -151,22 +163,22 @@ class Workload:
         sl = ol = mq.HWNC if hwnc else mq.NCHW
         if hwnc:
             src = self.src = [src[0].permute(2, 3, 0, 1).contiguous(), src[1].permute(0, 2, 3, 1).contiguous(), src[2].permute(2, 3, 0, 1).contiguous()]
-        q = self.q = [mq.empty_qtensor(d, r, f) for r, f in zip(roles, fmts)]
-        self.icb, self.isb = mq.im2col_sizes(d, fmts[0])
+        q = self.q = [mq.empty_qtensor(d, r, f, block=blk) for r, f in zip(roles, fmts)]
+        self.icb, self.isb = mq.im2col_sizes(d, fmts[0], blk)
         ic = torch.empty(self.icb, dtype=torch.uint8, device="cuda")
         isc = torch.empty(self.isb, dtype=torch.uint8, device="cuda")
         ho, wo = inputs.out_hw(d)
         self.y = y = torch.empty((ho, wo, d.N, d.C_out) if hwnc else (d.N, d.C_out, ho, wo), dtype=torch.float32, device="cuda")
         self.dx = dx = torch.empty((d.H, d.W, d.N, d.C_in) if hwnc else (d.N, d.C_in, d.H, d.W), dtype=torch.float32, device="cuda")
         self.dw = dw = torch.empty((d.C_out, d.Kh, d.Kw, d.C_in) if hwnc else (d.C_out, d.C_in, d.Kh, d.Kw), dtype=torch.float32, device="cuda")
-        ws_bytes = max(mq.workspace_size(d, op, a, b) for op, a, b in
+        ws_bytes = max(mq.workspace_size(d, op, a, b, blk) for op, a, b in
                        ((mq.OP_FWD, fmts[0], fmts[1]), (mq.OP_BWD_DATA, fmts[1], fmts[2]), (mq.OP_BWD_WEIGHT, fmts[0], fmts[2])))
         self.ws = ws = torch.empty(max(ws_bytes, 16), dtype=torch.uint8, device="cuda")
         self.calls = [
-            ("quantize_x", lambda: mq.quantize(d, roles[0], fmts[0], src[0], out=q[0], src_layout=sl)),
-            ("quantize_w", lambda: mq.quantize(d, roles[1], fmts[1], src[1], out=q[1], src_layout=sl)),
-            ("quantize_dy", (lambda: mq.quantize_sr(d, roles[2], fmts[2], src[2], 1234, out=q[2], src_layout=sl)) if dy_rounding == "stochastic" else
-             (lambda: mq.quantize(d, roles[2], fmts[2], src[2], out=q[2], src_layout=sl))),
+            ("quantize_x", lambda: mq.quantize(d, roles[0], fmts[0], src[0], out=q[0], src_layout=sl, block=blk)),
+            ("quantize_w", lambda: mq.quantize(d, roles[1], fmts[1], src[1], out=q[1], src_layout=sl, block=blk)),
+            ("quantize_dy", (lambda: mq.quantize_sr(d, roles[2], fmts[2], src[2], 1234, out=q[2], src_layout=sl, block=blk)) if dy_rounding == "stochastic" else
+             (lambda: mq.quantize(d, roles[2], fmts[2], src[2], out=q[2], src_layout=sl, block=blk))),
             ("cbf_im2col", lambda: mq.cbf_im2col(d, q[0], ic, isc)),
             ("conv_fwd", lambda: mq.conv_fwd(d, q[0], q[1], y=y, layout=ol, workspace=ws)),
             ("conv_bwd_data", lambda: mq.conv_bwd_data(d, q[1], q[2], dx=dx, layout=ol, workspace=ws)),
@@ -390,7 +402,8 @@ def run_ours(args):
             per2, nl2 = time_per_call(w2, flush, Km)
             k2, qi2 = roofline_table(w2, per2, nl2, pk)
             out["more_workloads"][name] = {
-                "layer": dict(w2.d._asdict()), "formats": [FMT_NAME[f] for f in w2.fmts], "steps": Km, "ms_per_step": ms2,
+                "layer": dict(w2.d._asdict()), "formats": [FMT_NAME[f] for f in w2.fmts],
+                "blocks": "16x16, E4M3 block scale, fp32 tensor scale" if name.endswith("+ts16") else "32x32, E8M0 scale", "steps": Km, "ms_per_step": ms2,
                 "value": 3.0 * layer_flops(w2.d) / (ms2 * 1e-3) / 1e12, "unit": "TFLOPS", "quantize_im2col_gbs": qi2,
                 "kernels": {n: {k: v for k, v in k2[n].items() if k != "algorithmic_bytes"} for n in CALLS},
                 "device_status": mq.last_device_status()}

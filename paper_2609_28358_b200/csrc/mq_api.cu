@@ -736,7 +736,7 @@ static mq_status quantize_impl(const mq_conv_desc* desc, const void* src, int sr
   if (!aligned16(src)) return MQ_ERR_ALIGNMENT;
   if (src_dtype != MQ_F32) return MQ_ERR_UNSUPPORTED;
   View v = view_of(g, dst->role);
-  QuantArgs a;
+  QuantArgs a{};
   a.src = static_cast<const float*>(src);
   a.codes = static_cast<uint8_t*>(dst->codes);
   a.scales = dst->scales;

@@ -80,6 +80,10 @@ struct QuantArgs {
   // issues no copies, so that every wait on them runs out
   unsigned wait_limit;
   int debug_skip_loads;
+  // the paper's own format on the whole-line kernel (launch_quantize_ts_tma): where Eq. 4 takes max|X| from, and the
+  // tensor's statistics buffer (T_scale is written to [0])
+  const float* ts_amax;
+  float* ts_stats;
 };
 // invertible 32-bit mixer (xor-shift, odd multiply, twice, xor-shift) behind the per-element draws
 __host__ __device__ __forceinline__ unsigned sr_mix32(unsigned x) {
@@ -90,6 +94,9 @@ cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s);
 // The paper's own format (fp32 tensor scale, E4M3 scale per 16 x 16 block, E2M1 elements; mq_quantize_ts.cu).  stats: device, two
 // floats (T_scale, max|X|); amax_in: device fp32 that Eq. 4 takes its maximum from, or null for the tensor's own.
 cudaError_t launch_quantize_ts(const QuantArgs& a, const float* amax_in, float* stats, cudaStream_t s);
+// Second pass of that quantizer on the whole-line TMA kernel (NCHW / OIHW source with 16-byte rows): true if the tensor qualifies
+bool quantize_ts_tma_eligible(const QuantArgs& a);
+cudaError_t launch_quantize_ts_tma(const QuantArgs& a, const float* amax_src, float* stats, cudaStream_t s);
 
 struct Im2colArgs {
   const uint8_t* codes;

@@ -382,7 +382,11 @@ __device__ __forceinline__ Item tq_item_of(unsigned it, int n_pstrips, int Ct) {
 
 // LINE: line blocks.  A line (32 channels of one row at one position) is held by two threads of neighbouring warps; they
 // exchange their maxima through the (still unused) staging buffer and the one with the lower channels writes the scale.
-template <int FMT, bool SR, bool LINE>
+// TS: the paper's own format (Eq. 4-6) - E2M1 elements, one E4M3 scale per 16 samples x 16 channels at a position, an
+// fp32 scale per tensor.  A thread's 4 x 16 values are 2 x 16 of the block (samples 0-15, its channel half) and 2 x 16
+// of the block 16 samples further; the 8 warps that hold the other samples of the same channel half are those of
+// this warp's parity.  Every operation of Eq. 4-6 is one IEEE single-precision operation in the order written.
+template <int FMT, bool SR, bool LINE, bool TS = false>
 __global__ void __launch_bounds__(TQ_THREADS, 1)
 quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_constant__ CUtensorMap map_out, QuantArgs a, int n_pstrips, int Ct,
                     unsigned n_items) {
@@ -447,23 +451,29 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_con
     int slot = 0;
     unsigned phase = 0;
     bool dead = false;
+    float tscale = 0.f, t6 = 0.f;
+    if (TS) {
+      tscale = __fdiv_rn(*a.ts_amax, __fmul_rn(448.0f, 6.0f));                                  // Eq. 4
+      t6 = __fmul_rn(tscale, 6.0f);
+      if (blockIdx.x == 0 && t == 0) a.ts_stats[0] = tscale;
+    }
 #pragma unroll 1
     for (unsigned it = blockIdx.x; it < n_items; it += gridDim.x) {
       const Item q = tq_item_of(it, n_pstrips, Ct);
       const int nb = min(4, (a.R - q.r0 + 7) >> 3);
       float v[4][16];
       float fm = 0.f;
-      float lm[LINE ? 4 : 1];
+      float lm[(LINE || TS) ? 4 : 1];
 #pragma unroll
       for (int b = 0; b < 4; ++b) {
-        if (LINE) { lm[b] = 0.f; }
+        if (LINE || TS) { lm[b] = 0.f; }
         if (b < nb) {
           if (!dead && !mbar_wait_limit(&full[slot], phase, limit, a.status, MQ_ERR_TIMEOUT)) { dead = true; *abort_flag = 1; }
           const float* src = rd + (size_t)slot * TQ_BOX_FLOATS;
 #pragma unroll
           for (int k = 0; k < 16; ++k) {
             v[b][k] = src[k * 32];
-            if (LINE) lm[b] = fmaxf(lm[b], fabsf(v[b][k])); else fm = fmaxf(fm, fabsf(v[b][k]));
+            if (LINE || TS) lm[b] = fmaxf(lm[b], fabsf(v[b][k])); else fm = fmaxf(fm, fabsf(v[b][k]));
           }
           __syncwarp();
           if (lane == 0) tc::mbar_arrive(&empty[slot]);
@@ -473,12 +483,34 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_con
           for (int k = 0; k < 16; ++k) v[b][k] = 0.f;
         }
       }
-      if (!LINE) red[warp * 32 + lane] = __float_as_uint(fm);
+      if (!LINE && !TS) red[warp * 32 + lane] = __float_as_uint(fm);
       if (t == 0) tc::bulk_wait_group_read<0>();    // the previous item's store has read the staging buffer
       consumer_sync();
       if (*abort_flag) break;    // uniform: written only between the previous item's last barrier and the one above
       int code[LINE ? 4 : 1];
-      if (LINE) {
+      float den[2] = {0.f, 0.f};   // TS: Scale_b * T_scale of the thread's two blocks (0: the block encodes to signed zeros)
+      if (TS) {
+        unsigned* xch = reinterpret_cast<unsigned*>(stage);   // [sample half][warp][lane]
+        xch[warp * 32 + lane] = __float_as_uint(fmaxf(lm[0], lm[1]));
+        xch[(16 + warp) * 32 + lane] = __float_as_uint(fmaxf(lm[2], lm[3]));
+        consumer_sync();
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+          unsigned mx = 0;
+#pragma unroll
+          for (int k = 0; k < 8; ++k) mx = max(mx, xch[(16 * hf + (warp & 1) + 2 * k) * 32 + lane]);
+          const float bmax = __uint_as_float(mx);
+          unsigned sc = 0;
+          if (bmax > 0.f && tscale > 0.f) sc = (unsigned)__nv_cvt_float_to_fp8(__fdiv_rn(bmax, t6), __NV_SATFINITE, __NV_E4M3) & 0x7Fu;   // Eq. 5
+          const __half_raw hr = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)sc, __NV_E4M3);
+          const float bscale = __half2float(*reinterpret_cast<const __half*>(&hr));
+          den[hf] = (bscale > 0.f && tscale > 0.f) ? __fmul_rn(bscale, tscale) : 0.f;
+          // one thread per (position, sample half, channel half): warps 0 and 1 hold both channel halves of every position
+          if ((warp >> 1) == 0 && q.p0 + lane < a.P && q.r0 + 16 * hf < a.R)
+            a.scales[(long long)(q.p0 + lane) * a.sc_stride_p + (long long)(2 * q.rt + hf) * a.sc_stride_r + 2 * q.ct + chalf] = (uint8_t)sc;
+        }
+        consumer_sync();    // every exchange word has been read before the codes overwrite the buffer
+      } else if (LINE) {
         unsigned* xch = reinterpret_cast<unsigned*>(stage);   // [box][warp][lane]
 #pragma unroll
         for (int b = 0; b < 4; ++b) xch[(b * 16 + warp) * 32 + lane] = __float_as_uint(lm[b]);
@@ -502,7 +534,8 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_con
 #pragma unroll
       for (int b = 0; b < 4; ++b) {
         if (b < nb) {
-          const float f = scale_factor(code[LINE ? b : 0]);
+          const float f = TS ? 0.f : scale_factor(code[LINE ? b : 0]);
+          const float dn = den[b >> 1];
           const int n = 8 * b + n_sub;
           unsigned w4[4];
 #pragma unroll
@@ -510,8 +543,9 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_con
             float x[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-              x[j] = v[b][k + j] * f;
-              if (SR) {
+              if (TS) x[j] = dn > 0.f ? __fdiv_rn(v[b][k + j], dn) : copysignf(0.f, v[b][k + j]);   // Eq. 6
+              else x[j] = v[b][k + j] * f;
+              if (SR && (!TS || dn > 0.f)) {
                 const long long e = ((long long)(q.r0 + n) * a.C + q.c0 + chalf * 16 + k + j) * a.P + q.p0 + lane;
                 x[j] = sr_value<FMT>(x[j], (unsigned)e, sr_key(a, e));
               }
@@ -718,6 +752,46 @@ cudaError_t launch_q(const QuantArgs& a, int n_pstrips, int Ct, long long n_item
 }
 
 }  // namespace
+
+bool quantize_ts_tma_eligible(const QuantArgs& a) {
+  const bool vec = (a.P % 4 == 0) && ((reinterpret_cast<uintptr_t>(a.src) & 15) == 0);
+  const long long elems = (long long)a.P * a.R * a.C;
+  const int tv = env_int("MQ_QUANT_TMA", -1);   // 1 / 0 force the choice
+  return vec && a.src_stride_r == 0 && a.fmt == MQ_E2M1 && (tv >= 0 ? tv != 0 : elems >= (1ll << 22));
+}
+
+cudaError_t launch_quantize_ts_tma(const QuantArgs& a0, const float* amax_src, float* stats, cudaStream_t s) {
+  QuantArgs a = a0;
+  a.ts_amax = amax_src; a.ts_stats = stats;
+  CUtensorMap map_in, map_out;
+  {
+    const uint64_t dims[3] = {(uint64_t)a.P, (uint64_t)a.C, (uint64_t)a.R};
+    const uint64_t strides[2] = {(uint64_t)a.P * 4, (uint64_t)a.C * a.P * 4};
+    const uint32_t box[3] = {32u, 32u, 8u};
+    if (!encode_tensor_map_u8(&map_in, a.src, 3, dims, strides, box, nullptr, 0, true, 128)) return cudaErrorInvalidValue;
+  }
+  {
+    const uint64_t dims[3] = {(uint64_t)a.Cp / 2, (uint64_t)a.R, (uint64_t)a.P};
+    const uint64_t strides[2] = {(uint64_t)a.out_stride_r / 2, (uint64_t)a.out_stride_p / 2};
+    const uint32_t box[3] = {16u, 32u, 32u};
+    if (!encode_tensor_map_u8(&map_out, a.codes, 3, dims, strides, box, nullptr, 0)) return cudaErrorInvalidValue;
+  }
+  static bool attr_set = false;
+  if (!attr_set) {
+    cudaError_t e = cudaFuncSetAttribute(quantize_tma_kernel<MQ_E2M1, false, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TQ_SMEM);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(quantize_tma_kernel<MQ_E2M1, true, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TQ_SMEM);
+    if (e != cudaSuccess) return e;
+    attr_set = true;
+  }
+  const int n_pstrips = (a.P + 31) / 32, Rt = (a.R + 31) / 32, Ct = a.Cp / 32;
+  const long long n_items = (long long)n_pstrips * Rt * Ct;
+  if (n_items <= 0 || n_items > 0x7fffffffLL) return cudaErrorInvalidValue;
+  const int sms = sm_count();
+  const unsigned grid = (unsigned)(n_items < sms ? n_items : sms);
+  if (a.sr) return launch_pdl(quantize_tma_kernel<MQ_E2M1, true, false, true>, dim3(grid), dim3(TQ_THREADS), TQ_SMEM, s, map_in, map_out, a, n_pstrips, Ct, (unsigned)n_items);
+  return launch_pdl(quantize_tma_kernel<MQ_E2M1, false, false, true>, dim3(grid), dim3(TQ_THREADS), TQ_SMEM, s, map_in, map_out, a, n_pstrips, Ct, (unsigned)n_items);
+}
 
 cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s) {
   const bool vec = (a.P % 4 == 0) && ((reinterpret_cast<uintptr_t>(a.src) & 15) == 0);

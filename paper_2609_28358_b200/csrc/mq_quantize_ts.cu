@@ -143,6 +143,8 @@ cudaError_t launch_quantize_ts(const QuantArgs& a, const float* amax_in, float* 
   const int vec = (a.P % 4 == 0 && (reinterpret_cast<uintptr_t>(a.src) & 15) == 0) ? 1 : 0;
   const float* amax_src = amax_in ? amax_in : stats + 1;
   count_launches(2);
+  // large NCHW / OIHW tensors with 16-byte rows: the whole-line TMA kernel (items of 32 positions x 32 rows x 32 channels = 4 blocks per position)
+  if (quantize_ts_tma_eligible(a)) return launch_quantize_ts_tma(a, amax_src, stats, s);
   if (a.sr) return launch_pdl(quantize_ts_kernel<true>, dim3((unsigned)qb), dim3(256), 0, s, a, amax_src, stats, Rb, Cb, (unsigned)n_pstrips, (unsigned)n_items, vec);
   return launch_pdl(quantize_ts_kernel<false>, dim3((unsigned)qb), dim3(256), 0, s, a, amax_src, stats, Rb, Cb, (unsigned)n_pstrips, (unsigned)n_items, vec);
 }

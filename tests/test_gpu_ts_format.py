@@ -74,6 +74,31 @@ def test_quantizer_im2col_and_gemms(name, shape, kinds):
     assert mq.last_device_status() == 0
 
 
+@pytest.mark.parametrize("name,shape", [("aligned", (64, 96, 8, 8, 64, 3, 1, 1)), ("ragged", (40, 48, 6, 6, 70, 3, 1, 1)),
+                                        ("few_samples", (5, 20, 8, 8, 24, 3, 1, 1)), ("wide", (33, 256, 4, 8, 288, 3, 1, 1))],
+                         ids=["aligned", "ragged", "few_samples", "wide"])
+def test_whole_line_quantizer(knobs, name, shape):
+    """Large NCHW tensors take the second pass on the whole-line TMA kernel (items of 32 positions x 32 samples x 32
+    channels, four 16 x 16 blocks per position); forced here on small shapes: same bytes as the oracle, own and
+    supplied maximum, stochastic rounding."""
+    knobs(MQ_QUANT_TMA=1)
+    d = inputs.conv_desc(*shape)
+    src = (inputs.make_x(d, 81, "relu"), inputs.make_dy(d, 81, "small"))
+    for what, r, t in zip(("X", "dY"), (mq.ROLE_X, mq.ROLE_DY), src):
+        o = oracle.quantize_ts(d, r, t, B16)
+        assert_ts_equal(f"{name} {what}", mq.quantize_ts(d, r, dev(t)), o)
+        amax = np.float32(1.7) * np.abs(t).max()
+        o2 = oracle.quantize_ts(d, r, t, B16, amax=float(amax))
+        g2 = mq.quantize_ts(d, r, dev(t), amax_in=torch.tensor([amax], dtype=torch.float32, device="cuda"))
+        assert_same_bytes(g2.scales, o2[1], f"{name} {what} supplied maximum: block scales")
+        assert_same_bytes(g2.codes, o2[0], f"{name} {what} supplied maximum: codes")
+        o3 = oracle.quantize_ts(d, r, t, B16, seed=99)
+        g3 = mq.quantize_ts(d, r, dev(t), seed=99)
+        assert_same_bytes(g3.scales, o3[1], f"{name} {what} stochastic: block scales")
+        assert_same_bytes(g3.codes, o3[0], f"{name} {what} stochastic: codes")
+    assert mq.last_device_status() == 0
+
+
 def test_tensor_core_and_cuda_core_routes_agree(knobs):
     """The forward and input-gradient GEMMs of this format run on the tensor cores where the layer allows it
     (kind::mxf4nvf4: E4M3 scales per 16 elements in tensor memory, the tensors' fp32 scales applied to the accumulator)
