@@ -209,6 +209,42 @@ class Workload:
                 "conv_bwd_weight": max(FMT_BITS[f[0]], FMT_BITS[f[2]])}
 
 
+def fused_epilogue_times(wl, flush, K, kern, pk):
+    """mq_conv_fwd_mx (ReLU, emitting the next layer's activation tensor in X's format) and mq_conv_bwd_data_mx (emitting the
+    previous layer's gradient tensor in dY's format) on the workload's quantized operands."""
+    import torch
+
+    from paper_2609_28358_b200 import mq
+
+    d, q, f = wl.d, wl.q, wl.fmts
+    ws = torch.empty(max(mq.conv_mx_workspace_size(d, mq.OP_FWD, f[0], f[1]), mq.conv_mx_workspace_size(d, mq.OP_BWD_DATA, f[1], f[2]), 16), dtype=torch.uint8,
+                     device="cuda")
+    yq = mq.conv_fwd_mx(d, q[0], q[1], f[0], mq.ACT_RELU, workspace=ws)
+    dxq = mq.conv_bwd_data_mx(d, q[1], q[2], f[2], workspace=ws)
+    calls = {"conv_fwd_mx": (lambda: mq.conv_fwd_mx(d, q[0], q[1], f[0], mq.ACT_RELU, yq=yq, workspace=ws), "conv_fwd", max(FMT_BITS[f[0]], FMT_BITS[f[1]])),
+             "conv_bwd_data_mx": (lambda: mq.conv_bwd_data_mx(d, q[1], q[2], f[2], dxq=dxq, workspace=ws), "conv_bwd_data", max(FMT_BITS[f[1]], FMT_BITS[f[2]]))}
+    res = {}
+    for name, (fn, plain, bits) in calls.items():
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        for s, e in ev:
+            flush.zero_()
+            s.record()
+            fn()
+            e.record()
+        torch.cuda.synchronize()
+        ms = sum(s.elapsed_time(e) for s, e in ev) / K
+        tf = layer_flops(d) / (ms * 1e-3) / 1e12
+        peak = pk["bf16_tflops"] * TENSOR_RATIO[bits]
+        res[name] = {"ms": ms, "tflops": tf, "frac": tf / peak, "frac_of_published": tf / PUBLISHED["tensor_tflops"][bits],
+                     "fp32_output_call_ms": kern[plain]["ms"], "activation": "relu" if name == "conv_fwd_mx" else "none",
+                     "emits": FMT_NAME[f[0] if name == "conv_fwd_mx" else f[2]]}
+    res["device_status"] = mq.last_device_status()
+    return res
+
+
 def time_per_call(wl, flush, K):
     """Mean duration of each call over K steps (CUDA events on the launching stream, L2 flushed before each step) and
     the number of kernels each call launches (the library's own count)."""
@@ -378,6 +414,11 @@ def run_ours(args):
         "kernels": kern,
         "device_status": dev_status,
     }
+
+    # ---- the two GEMMs with the quantizing producer epilogue (the next tensor leaves the chip in its stored MX form instead of
+    # fp32): per-call times beside the fp32-output calls and the quantizer call they replace
+    if world == 1 and wl.block == mq.TILE32:
+        out["fused_epilogue"] = fused_epilogue_times(wl, flush, max(3, min(K, 10)), kern, pk)
 
     # ---- the same step on further workloads (device-timed step and per-call roofline only)
     more = [] if args.more == "none" else [m for m in args.more.split(",") if m and m != args.workload]

@@ -47,7 +47,9 @@
  *   and mq_qtensor.tensor_scale points at two device floats: T_scale, and the tensor's own max|X| (kept so that a later
  *   step can use it as its estimate, Sec. VII-B).  Eq. 4-6 are evaluated in IEEE single precision, one rounding per
  *   written operation; both roundings go to nearest, ties to even, and saturate; a block of zeros has scale 0.
- *   All calls accept it (both operands of a GEMM must use it); the GEMMs run on the CUDA-core kernels in this build.
+ *   All calls accept it (both operands of a GEMM must use it).  The three GEMMs run on the tensor cores (E4M3 scale per 16
+ *   elements of the contraction axis, the tensors' fp32 scales applied to the accumulator) for the layers the MX E2M1
+ *   path takes, on the CUDA-core kernels otherwise; mq_conv_fwd_mx / mq_conv_bwd_data_mx do not take it.
  */
 #ifndef MQ_H_
 #define MQ_H_

@@ -492,9 +492,13 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g, bool ts16 = false) {
   {
     int st = (227 * 1024 - 2048) / p.stage_bytes;
     if (st > 6) st = 6;
-    while (st > 2 && p.TG * p.b_rows + st * sf_cols1 * (1 + p.NB) > 512) --st;
+    int slots = st;
+    // kind 2: the scale buffers are twice as wide; rather than giving up pipeline stages, fewer buffers are used in turn
+    if (ts16 && !env_int("MQ_WGRAD_TS_NO_SLOTS", 0)) { while (slots > 2 && p.TG * p.b_rows + slots * sf_cols1 * (1 + p.NB) > 512) --slots; }
+    else { while (st > 2 && p.TG * p.b_rows + st * sf_cols1 * (1 + p.NB) > 512) --st; slots = st; }
     p.stages = st;
-    const int cols = p.TG * p.b_rows + st * sf_cols1 * (1 + p.NB);
+    p.sf_slots = slots;
+    const int cols = p.TG * p.b_rows + slots * sf_cols1 * (1 + p.NB);
     p.tmem_cols = cols <= 256 ? 256 : 512;
     if (st < 2 || cols > 512) return w;
   }

@@ -136,6 +136,7 @@ struct WgradTcParams {
   int n0, n1;           // MMA widths per K slice: n0 = min(TG * b_rows, 256) and the rest (0: one MMA)
   int b_tile_bytes;     // bytes of X loaded per stage: b_rows * 128, flat mode (KPX + TG - 1) * b_rows * KBn
   int stage_bytes;      // A tile + B tile + (1 + NB) scale chunks of 1024 bytes, rounded up to 1024
+  int sf_slots;         // scale buffers in tensor memory: = stages, or fewer (kind 2), used in turn
   int tmem_cols;        // TMEM allocation: accumulators (TG * b_rows) + stages * (8 + 8 * NB), a power of two
   const uint8_t* g_scales;  // [Ho][Wo][Nt][Cot]
   const uint8_t* x_scales;  // [H][W][Nt][Ct]

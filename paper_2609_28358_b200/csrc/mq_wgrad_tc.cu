@@ -403,12 +403,21 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       }
       const uint32_t d1 = tmem + (uint32_t)p.n0;
       uint32_t s = 0, phase = 0, accumulate = 0;
+      // Scale buffers in tensor memory: one per pipeline stage, or (sf_slots < stages: the wide scale vectors of kind 2 next to
+      // a tap group's accumulators) fewer, taken in turn - a buffer is rewritten only after the MMAs that read it have
+      // completed, which is what the stage's `empty` barrier reports.
+      uint32_t ss = 0, es = 0, ephase = 0;   // scale slot of this stage; stage (and its parity) whose MMAs used that slot last
 #pragma unroll 1
       for (int i = 0; i < nst; ++i) {   // another role's abort shows here as this thread's own bounded wait running out
         if (!mbar_wait((FP4 && !p.mma_cp) ? &sffull[s] : &full[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+        if (FP4 && p.mma_cp && p.sf_slots < p.stages && i >= p.sf_slots) {
+          if (!mbar_wait(&empty[es], ephase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+          if (++es == (uint32_t)p.stages) { es = 0; ephase ^= 1; }
+        }
         tc_fence_after_sync();
         const uint32_t so = s * stage16;
-        const uint32_t sf_t = sf_base + s * sf_cols;
+        const uint32_t sf_t = sf_base + ss * sf_cols;
+        if (++ss == (uint32_t)p.sf_slots) ss = 0;
         const uint64_t ad = a_desc0 + so, bd = b_desc0 + so;
         if (!FP4 && nm == 1) {
           // 8-bit operands: this lane also issues the stage's three scale copies, right before the MMAs that read
@@ -483,12 +492,18 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
       const uint32_t stage16 = (uint32_t)stage_bytes >> 4;
       const uint32_t sf_base = tmem + acc_cols;
       uint32_t s = 0, phase = 0;
+      uint32_t ss = 0, es = 0, ephase = 0;   // see the MMA issuer
 #pragma unroll 1
       for (int i = 0; i < nst && !*abort_flag; ++i) {
         if (!mbar_wait(&full[s], phase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+        if (p.sf_slots < p.stages && i >= p.sf_slots) {
+          if (!mbar_wait(&empty[es], ephase, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+          if (++es == (uint32_t)p.stages) { es = 0; ephase ^= 1; }
+        }
         tc_fence_after_sync();
         const uint32_t so = s * stage16;
-        const uint32_t sf_t = sf_base + s * sf_cols;
+        const uint32_t sf_t = sf_base + ss * sf_cols;
+        if (++ss == (uint32_t)p.sf_slots) ss = 0;
         if (elect_one()) {
 #ifdef MQ_WG_SKIPCP
           if (i < p.stages)
