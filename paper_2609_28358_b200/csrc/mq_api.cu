@@ -179,7 +179,8 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   // 1x1 layers: the activation tile is the whole of a tile's loads, so halving its re-reads pays although the main loop is short
   // (measured, N = 256, 8-bit, fp32 / quantized output: 256 channels 56x56 324 -> 207 us / 217 -> 196 us; 512 channels 56x56
   // 531 -> 528 / 464 -> 410 us; 512 channels 28x28 181 -> 175 / 133 -> 127 us)
-  if (!fp4 && p.Cd >= 256 && taps == 1 && g.sh == 1 && g.sw == 1 && !env_int("MQ_TC_1X1_BN128", 0)) p.BN = 256;
+  // E2M1 likewise: 512 channels 56x56 550 -> 364 us, 256 channels 56x56 290 -> 173 us
+  if (p.Cd >= 256 && taps == 1 && g.sh == 1 && g.sw == 1 && !env_int("MQ_TC_1X1_BN128", 0)) p.BN = 256;
   // E2M1: the same trade (measured with the tile widths chosen below: 256 channels 28x28 -13 %, 512 channels 14x14 -6 %,
   // 56x56 -10 %)
   const double act_bytes = (double)p.Hs * p.Ws * g.N * rowbytes;
@@ -285,7 +286,7 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   }
   // unit strides and one 128-byte chunk per stage: the activation-side scale chunk of (tile, kh) equals that of the tile one
   // output row further with kh - 1, so chunks are stored per source row - Kh times fewer to expand
-  p.sfa_dedup = (!p.halo && !ts16 && p.KB == 128 && g.sh == 1 && g.sw == 1 && !env_int("MQ_TC_NO_SFA_DEDUP", 0)) ? 1 : 0;
+  p.sfa_dedup = (!p.halo && p.KB == 128 && g.sh == 1 && g.sw == 1 && !env_int("MQ_TC_NO_SFA_DEDUP", 0)) ? 1 : 0;
   p.sfa_hk = p.tiles_h + g.Kh - 1;
   out->p = p;
   size_t o = 0;

@@ -1228,7 +1228,38 @@ __global__ void __launch_bounds__(256) expand_conv_scales_kernel(const ConvTcPar
     // chunk of its own ([32 rows][row quarter][4 bytes]).  A: [Hs][Ws][ceil(N/16)][K/16]; B: [ceil(rows/16)][taps][K/16],
     // or, for the input gradient, gathered from the stored W scales [ceil(C_out/16)][taps][C_in_p/16] with K = C_out.
     const int Kb16 = p.Kblocks * 2, Nt16 = (p.N + 15) >> 4;
-    if (wid < nA) {
+    if (G == 1 && p.sfa_dedup && wid < nA) {
+      // shared chunks (unit strides, one chunk per stage), keyed as in the branch for the E8M0 kinds below:
+      // wid = (((sample tile * row keys + row key) * column tiles + column tile) * Kw + kw) * cpt + chunk
+      unsigned u = wid;
+      ChunkPos pos;
+      pos.ia = 0;
+      pos.cc = (int)(u % (unsigned)p.cpt); u /= (unsigned)p.cpt;
+      pos.ib = (int)(u % (unsigned)p.Kw); u /= (unsigned)p.Kw;
+      Tile tile;
+      tile.w0 = (int)(u % (unsigned)p.tiles_w) * p.TW; u /= (unsigned)p.tiles_w;
+      const int hk = (int)(u % (unsigned)p.sfa_hk);
+      tile.n0 = (int)(u / (unsigned)p.sfa_hk) * p.TN;
+      tile.h = 0; tile.cls = 0; tile.c0 = 0; tile.ct = 0;
+      TapWalk<MODE> tw;
+      tw.init(p, tile);
+      const int hs = hk + tw.hs0 - (MODE == MQ_OP_FWD ? 0 : p.Kh - 1);
+      const int ws0 = src_w0(tw, pos);
+      uint32_t val[4][4];
+#pragma unroll
+      for (int j = 0; j < 4; ++j) {
+        const int r = 32 * j + lane;
+        const int tw_ = r & (p.TW - 1), tn = r >> p.lgTW;
+        const int n = tile.n0 + tn, ws = ws0 + tw_;
+        const bool ok = n < p.N && hs >= 0 && hs < p.Hs && ws >= 0 && ws < p.Ws;
+        const uint8_t* rowp = p.a_scales + (((long long)hs * p.Ws + ws) * Nt16 + (n >> 4)) * Kb16 + pos.cc * (4 * APC);
+#pragma unroll
+        for (int ja = 0; ja < 4; ++ja) val[ja][j] = (ok && ja < APC) ? __ldg(reinterpret_cast<const unsigned int*>(rowp + 4 * ja)) : 0u;
+      }
+      uint8_t* dst = p.sfa_img + (size_t)wid * (512 * 4) + lane * 16;
+#pragma unroll
+      for (int ga = 0; ga < 4; ++ga) *reinterpret_cast<uint4*>(dst + ga * 512) = make_uint4(val[ga][0], val[ga][1], val[ga][2], val[ga][3]);
+    } else if (wid < nA) {
       const unsigned tm = wid / (unsigned)p.max_stages;
       const int st = (int)(wid - tm * p.max_stages);
       const Tile tile = tile_of_m_index(p, tm);

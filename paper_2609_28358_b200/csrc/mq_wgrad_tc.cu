@@ -54,58 +54,67 @@ __device__ __forceinline__ void expand_wgrad_scales_nv_body(const WgradTcParams&
   const long long nB = (long long)p.cb_tiles * groups * p.stages_total * p.NB;
   if (wid >= nA + nB) return;
   const int Nt16 = (p.N + 15) >> 4, Cot16 = p.Cot * 2, Ct16 = p.Ct * 2;
-  uint32_t val[4][4];   // [MMA of the stage][row quarter]
-#pragma unroll
-  for (int ga = 0; ga < 4; ++ga)
-#pragma unroll
-    for (int jj = 0; jj < 4; ++jj) val[ga][jj] = 0u;
+  // A chunk holds 16 K-blocks x 8 row blocks (16 rows each) = 128 distinct scale bytes: lane (b16, jh) = (lane >> 1, lane & 1)
+  // loads the four of K-block b16 and row blocks 4 jh .. 4 jh + 3; the words of the chunk are then assembled by shuffles
+  // (a lane loading its own 64 bytes, two distinct addresses per warp-wide load, took 2.5 times as long).
+  const int b16 = lane >> 1, jh = lane & 1;
+  uint32_t mine = 0;
   uint8_t* dst;
+  const int st = wid < nA ? (int)(wid % p.stages_total) : (int)(((wid - nA) / p.NB) % p.stages_total);
+  int ho, wo, nb;
+  stage_block(p, st, b16 >> 1, ho, wo, nb);
+  const int nb16 = 2 * nb + (b16 & 1);
+  const bool kok = ho < p.Ho && wo < p.Wo && nb16 < Nt16;
   if (wid < nA) {
-    const int mt = (int)(wid / p.stages_total), st = (int)(wid - (long long)mt * p.stages_total);
-#pragma unroll 1
-    for (int b16 = 0; b16 < 16; ++b16) {
-      int ho, wo, nb;
-      stage_block(p, st, b16 >> 1, ho, wo, nb);
-      const int nb16 = 2 * nb + (b16 & 1);
-      if (ho < p.Ho && wo < p.Wo && nb16 < Nt16) {
-        const uint8_t* line = p.g_scales + (((long long)ho * p.Wo + wo) * Nt16 + nb16) * Cot16;
+    const int mt = (int)(wid / p.stages_total);
+    if (kok) {
+      const uint8_t* line = p.g_scales + (((long long)ho * p.Wo + wo) * Nt16 + nb16) * Cot16;
 #pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-          const int cob16 = (mt * 128 + 32 * jj + lane) >> 4;
-          if (cob16 < Cot16) val[b16 >> 2][jj] |= (uint32_t)__ldg(line + cob16) << (8 * (b16 & 3));
-        }
+      for (int k = 0; k < 4; ++k) {
+        const int cob16 = mt * 8 + 4 * jh + k;
+        if (cob16 < Cot16) mine |= (uint32_t)__ldg(line + cob16) << (8 * k);
       }
     }
     dst = p.sfa_img + wid * 2048;
   } else {
     long long idx = wid - nA;
     const int c = (int)(idx % p.NB); idx /= p.NB;
-    const int st = (int)(idx % p.stages_total); idx /= p.stages_total;
+    idx /= p.stages_total;
     const int tg = (int)(idx % groups); const int cb = (int)(idx / groups);
-#pragma unroll 1
-    for (int b16 = 0; b16 < 16; ++b16) {
-      int ho, wo, nb;
-      stage_block(p, st, b16 >> 1, ho, wo, nb);
-      const int nb16 = 2 * nb + (b16 & 1);
-      if (ho < p.Ho && wo < p.Wo && nb16 < Nt16) {
+    if (kok) {
 #pragma unroll
-        for (int jj = 0; jj < 4; ++jj) {
-          // B rows of a tap group: tap-in-group major, input channel minor; chunk c holds rows [128c, 128c + 128)
-          const int row = c * 128 + 32 * jj + lane;
-          const int tj = row / p.b_rows, rj = row - tj * p.b_rows;
-          const int tap = tg * p.TG + tj;
-          const int kh = tap / p.Kw, kw = tap - kh * p.Kw;
-          const int cib16 = (cb * p.b_rows + rj) >> 4;
-          const int h = ho * p.sh + kh - p.ph, w = wo * p.sw + kw - p.pw;
-          if (tj < p.TG && cib16 < Ct16 && h >= 0 && h < p.H && w >= 0 && w < p.W)
-            val[b16 >> 2][jj] |= (uint32_t)__ldg(p.x_scales + (((long long)h * p.W + w) * Nt16 + nb16) * Ct16 + cib16) << (8 * (b16 & 3));
-        }
+      for (int k = 0; k < 4; ++k) {
+        // B rows of a tap group: tap-in-group major, input channel minor; chunk c holds rows [128c, 128c + 128); a 16-row
+        // block lies inside one tap (b_rows is a multiple of 32)
+        const int row = c * 128 + 16 * (4 * jh + k);
+        const int tj = row / p.b_rows, rj = row - tj * p.b_rows;
+        const int tap = tg * p.TG + tj;
+        const int kh = tap / p.Kw, kw = tap - kh * p.Kw;
+        const int cib16 = (cb * p.b_rows + rj) >> 4;
+        const int h = ho * p.sh + kh - p.ph, w = wo * p.sw + kw - p.pw;
+        if (tj < p.TG && cib16 < Ct16 && h >= 0 && h < p.H && w >= 0 && w < p.W)
+          mine |= (uint32_t)__ldg(p.x_scales + (((long long)h * p.W + w) * Nt16 + nb16) * Ct16 + cib16) << (8 * k);
       }
     }
     dst = p.sfb_img + (wid - nA) * 2048;
   }
+  // word (MMA ga, row quarter jj) of row `lane`: K-blocks 4 ga .. 4 ga + 3 of row block 2 jj + (lane >> 4)
+  const int sh8 = 8 * (lane >> 4);
 #pragma unroll
-  for (int ga = 0; ga < 4; ++ga) *reinterpret_cast<uint4*>(dst + ga * 512 + lane * 16) = make_uint4(val[ga][0], val[ga][1], val[ga][2], val[ga][3]);
+  for (int ga = 0; ga < 4; ++ga) {
+    uint32_t w4[4];
+#pragma unroll
+    for (int jj = 0; jj < 4; ++jj) {
+      uint32_t word = 0;
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const uint32_t src = __shfl_sync(0xffffffffu, mine, ((4 * ga + k) << 1) | (jj >> 1));
+        word |= ((src >> (16 * (jj & 1) + sh8)) & 0xffu) << (8 * k);
+      }
+      w4[jj] = word;
+    }
+    *reinterpret_cast<uint4*>(dst + ga * 512 + lane * 16) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+  }
 }
 
 // ---- scale expansion: one warp per 512*SPA-byte chunk ----------------------------------------------------
