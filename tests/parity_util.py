@@ -151,7 +151,7 @@ def _pick_blocks(nblocks, want, rng):
     return sorted({0, nblocks - 1, *map(int, mid)})
 
 
-def check_large_layer(layer, samples=3000, dw_mac_budget=3e10, seed=0):
+def check_large_layer(layer, samples=3000, dw_mac_budget=3e10, seed=0, block=None):
     """Parity of a layer too large for the oracle to process whole.  The GPU runs the whole layer at full size; the
     oracle checks it on pieces that are independent of the rest of the tensor:
       * the first and the last 32-sample slab (tiles never span slabs; Y and G_X of a sample depend on that sample
@@ -161,21 +161,44 @@ def check_large_layer(layer, samples=3000, dw_mac_budget=3e10, seed=0):
         co and ci only): every quantized byte of those blocks - which reaches the far end of tensors beyond 2^31
         bytes - and the weight gradient of (chosen output blocks) x (chosen input blocks), every tap: in full while
         that fits `dw_mac_budget` multiply-adds of the oracle, else samples stratified over (output block, tap, input block);
-      * W in full."""
+      * W in full.
+    block=mq.TS16: the paper's own format (E2M1 elements whatever the layer names).  Its blocks are 16 x 16, so the same
+    pieces are independent once the oracle is given the whole tensor's maximum (Eq. 4), which is computed here with numpy
+    and also compared with what the GPU's first pass found."""
     d = layer.desc
-    fx, fw, fg = layer.fmt_x, layer.fmt_w, layer.fmt_dy
-    name = layer.name
+    ts = block == mq.TS16
+    fx, fw, fg = (mq.E2M1,) * 3 if ts else (layer.fmt_x, layer.fmt_w, layer.fmt_dy)
+    bs = 16 if ts else 32                       # side of a scale block
+    name = layer.name + (" (paper's format)" if ts else "")
     rng = np.random.default_rng(seed)
     x, w, g = inputs.layer_tensors(layer)
     ho, wo = inputs.out_hw(d)
-    N, Nt = d.N, (d.N + 31) // 32
+    N, Nt = d.N, (d.N + bs - 1) // bs
     cp, cop = (d.C_in + 31) // 32 * 32, (d.C_out + 31) // 32 * 32
     bpe = lambda f: 0.5 if f == mq.E2M1 else 1.0
-    xq, wq, gq = [mq.quantize(d, r, f, dev(t)) for r, f, t in zip(ROLES, (fx, fw, fg), (x, w, g))]
-    wc, wsc = oracle.quantize(d, oracle.ROLE_W, fw, w)
+    OR = (oracle.ROLE_X, oracle.ROLE_W, oracle.ROLE_DY)
+    amax = [float(np.abs(t).max()) for t in (x, w, g)] if ts else None
+
+    def oq(dsub, r, f, t):          # oracle: (codes, scales, tensor scale)
+        if ts:
+            o = oracle.quantize_ts(dsub, OR[r], t, (16, 16), amax=amax[r])
+            return o[0], o[1], o[2]
+        return oracle.quantize(dsub, OR[r], f, t) + (None,)
+
+    def odq(dsub, r, f, c, sc, t):
+        return oracle.dequant_ts(dsub, OR[r], c, sc, t, (16, 16)) if ts else oracle.dequant(dsub, OR[r], f, c, sc)
+
+    if ts:
+        xq, wq, gq = [mq.quantize_ts(d, r, dev(t)) for r, t in zip(ROLES, (x, w, g))]
+        for q, a in zip((xq, wq, gq), amax):
+            st = host(q.tensor_scale)
+            assert st[1] == np.float32(a) and st[0] == np.float32(a) / (np.float32(448.0) * np.float32(6.0)), (name, st, a)
+    else:
+        xq, wq, gq = [mq.quantize(d, r, f, dev(t)) for r, f, t in zip(ROLES, (fx, fw, fg), (x, w, g))]
+    wc, wsc, wt = oq(d, 1, fw, w)
     assert_same_bytes(wq.scales, wsc, f"{name} W scales")
     assert_same_bytes(wq.codes, wc, f"{name} W codes")
-    wh = oracle.dequant(d, oracle.ROLE_W, fw, wc, wsc)
+    wh = odq(d, 1, fw, wc, wsc, wt)
     ic, isc = mq.cbf_im2col(d, xq)
     y = mq.conv_fwd(d, xq, wq)
     dx = mq.conv_bwd_data(d, wq, gq)
@@ -183,26 +206,27 @@ def check_large_layer(layer, samples=3000, dw_mac_budget=3e10, seed=0):
     P, Po, taps = d.H * d.W, ho * wo, d.Kh * d.Kw
     xcodes = xq.codes.view(P, N, int(cp * bpe(fx)))
     gcodes = gq.codes.view(Po, N, int(cop * bpe(fg)))
-    xscales = xq.scales.view(P, Nt, cp // 32)
-    gscales = gq.scales.view(Po, Nt, cop // 32)
+    xscales = xq.scales.view(P, Nt, cp // bs)
+    gscales = gq.scales.view(Po, Nt, cop // bs)
     icodes = ic.view(Po, N, int(taps * cp * bpe(fx)))
-    iscales = isc.view(Po, Nt, taps * (cp // 32))
+    iscales = isc.view(Po, Nt, taps * (cp // bs))
     worst = {}
-    for slab in sorted({0, Nt - 1}):
+    for slab in sorted({0, (N + 31) // 32 - 1}):
         n0, n1 = 32 * slab, min(N, 32 * slab + 32)
+        b0, b1 = n0 // bs, (n1 + bs - 1) // bs          # scale rows of the slab
         ds = d._replace(N=n1 - n0)
-        xc, xsc = oracle.quantize(ds, oracle.ROLE_X, fx, x[n0:n1])
-        gc, gsc = oracle.quantize(ds, oracle.ROLE_DY, fg, g[n0:n1])
-        assert_same_bytes(xscales[:, slab].contiguous(), xsc, f"{name} X scales, samples {n0}..{n1}")
+        xc, xsc, xt = oq(ds, 0, fx, x[n0:n1])
+        gc, gsc, gt = oq(ds, 2, fg, g[n0:n1])
+        assert_same_bytes(xscales[:, b0:b1].contiguous(), xsc, f"{name} X scales, samples {n0}..{n1}")
         assert_same_bytes(xcodes[:, n0:n1].contiguous(), xc, f"{name} X codes, samples {n0}..{n1}")
-        assert_same_bytes(gscales[:, slab].contiguous(), gsc, f"{name} dY scales, samples {n0}..{n1}")
+        assert_same_bytes(gscales[:, b0:b1].contiguous(), gsc, f"{name} dY scales, samples {n0}..{n1}")
         assert_same_bytes(gcodes[:, n0:n1].contiguous(), gc, f"{name} dY codes, samples {n0}..{n1}")
-        oc, osc = oracle.cbf_im2col(ds, fx, xc, xsc)
-        assert_same_bytes(iscales[:, slab].contiguous(), osc, f"{name} im2col scales, samples {n0}..{n1}")
+        oc, osc = oracle.cbf_im2col(ds, fx, xc, xsc, (16, 16)) if ts else oracle.cbf_im2col(ds, fx, xc, xsc)
+        assert_same_bytes(iscales[:, b0:b1].contiguous(), osc, f"{name} im2col scales, samples {n0}..{n1}")
         assert_same_bytes(icodes[:, n0:n1].contiguous(), oc, f"{name} im2col codes, samples {n0}..{n1}")
         del oc, osc
-        xh = oracle.dequant(ds, oracle.ROLE_X, fx, xc, xsc)
-        gh = oracle.dequant(ds, oracle.ROLE_DY, fg, gc, gsc)
+        xh = odq(ds, 0, fx, xc, xsc, xt)
+        gh = odq(ds, 2, fg, gc, gsc, gt)
         shape = (n1 - n0, d.C_out, ho, wo)
         idx = _sample(int(np.prod(shape)), samples, rng, border_indices(shape, rng=rng))
         ref, ab = oracle.conv_fwd(ds, xh, wh, idx)
@@ -226,17 +250,18 @@ def check_large_layer(layer, samples=3000, dw_mac_budget=3e10, seed=0):
     xs = np.ascontiguousarray(x[:, ci])
     gs = np.ascontiguousarray(g[:, co])
     del x, g
-    xc, xsc = oracle.quantize(dsel, oracle.ROLE_X, fx, xs)
-    gc, gsc = oracle.quantize(dsel, oracle.ROLE_DY, fg, gs)
+    xc, xsc, xt = oq(dsel, 0, fx, xs)
+    gc, gsc, gt = oq(dsel, 2, fg, gs)
     del xs, gs
     bx, bg = int(32 * bpe(fx)), int(32 * bpe(fg))
     tb = lambda blocks: torch.as_tensor(blocks, device="cuda")
-    assert_same_bytes(xscales[:, :, tb(bi)].contiguous(), xsc, f"{name} X scales, channel blocks {bi}")
+    sb = lambda blocks: tb([(32 // bs) * b + k for b in blocks for k in range(32 // bs)])      # scale columns of 32-channel blocks
+    assert_same_bytes(xscales[:, :, sb(bi)].contiguous(), xsc, f"{name} X scales, channel blocks {bi}")
     assert_same_bytes(xcodes.view(P, N, cp // 32, bx)[:, :, tb(bi)].contiguous(), xc, f"{name} X codes, channel blocks {bi}")
-    assert_same_bytes(gscales[:, :, tb(bo)].contiguous(), gsc, f"{name} dY scales, channel blocks {bo}")
+    assert_same_bytes(gscales[:, :, sb(bo)].contiguous(), gsc, f"{name} dY scales, channel blocks {bo}")
     assert_same_bytes(gcodes.view(Po, N, cop // 32, bg)[:, :, tb(bo)].contiguous(), gc, f"{name} dY codes, channel blocks {bo}")
-    xh = oracle.dequant(dsel, oracle.ROLE_X, fx, xc, xsc)
-    gh = oracle.dequant(dsel, oracle.ROLE_DY, fg, gc, gsc)
+    xh = odq(dsel, 0, fx, xc, xsc, xt)
+    gh = odq(dsel, 2, fg, gc, gsc, gt)
     got = host(dw[tb(co)][:, tb(ci)].contiguous()).reshape(-1)
     per_out = float(N) * ho * wo
     if co.size * ci.size * taps * per_out <= dw_mac_budget:

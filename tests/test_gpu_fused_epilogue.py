@@ -168,6 +168,68 @@ def test_every_tile_width(knobs, fmts, out_fmt, tw):
                   mq.ACT_NONE, dxq)
 
 
+def _tiles_of_slab(rng, n_pix, n_cb, border, count):
+    """(pixel, channel block) pairs: the image's corner / edge pixels first, then random ones"""
+    pix = list(border) + list(rng.integers(0, n_pix, count))
+    return [(int(p), int(rng.integers(0, n_cb))) for p in pix[:count]]
+
+
+@pytest.mark.parametrize("name,act", [("cfg5_e4m3_k3s1_c512_hw28", mq.ACT_RELU), ("cfg5_e4m3_k3s1_c512_hw56", mq.ACT_SILU),
+                                      ("cfg5_e4m3_k1s1_c512_hw56", mq.ACT_RELU), ("cfg5_e4m3_k3s2_c512_hw28", mq.ACT_NONE),
+                                      ("cfg5_e2m1_k3s1_c512_hw28", mq.ACT_RELU)],
+                         ids=["3x3_hw28_relu", "3x3_hw56_silu", "1x1_hw56_relu", "3x3s2_hw28_none", "e2m1_hw28_relu"])
+def test_bench_layers_full_size(name, act):
+    """The layers `bench.py` times with the quantizing epilogue, on the GPU at full size (one-column tiles, 256-channel tiles,
+    tensors beyond 2^31 elements).  The oracle checks whole sample tiles - (pixel, 32 samples, 32 channels), corner and edge
+    pixels included, in the first and the last 32-sample slab - of the emitted activation tensor and of the emitted
+    gradient tensor: the tile's 1024 sums in float64, then the bracket rule of check_emitted on the tiles laid side by side."""
+    import types
+    layer = {l.name: l for l in inputs.config5()}[name]
+    d, (fx, fw, fg) = layer.desc, (layer.fmt_x, layer.fmt_w, layer.fmt_dy)
+    x, w, g = inputs.layer_tensors(layer)
+    ho, wo = inputs.out_hw(d)
+    xq, wq, gq = [mq.quantize(d, r, f, dev(t)) for r, f, t in zip((mq.ROLE_X, mq.ROLE_W, mq.ROLE_DY), (fx, fw, fg), (x, w, g))]
+    yq = mq.conv_fwd_mx(d, xq, wq, fx, act)
+    dxq = mq.conv_bwd_data_mx(d, wq, gq, fg)
+    assert mq.last_device_status() == 0
+    wc, wsc = oracle.quantize(d, oracle.ROLE_W, fw, w)
+    wh = oracle.dequant(d, oracle.ROLE_W, fw, wc, wsc)
+    rng = np.random.default_rng(5)
+    T = 24
+    bpe = lambda f: 0.5 if f == E2M1 else 1.0
+    for what, q_out, fmt_out, C, Hh, Ww, a in (("fwd", yq, fx, d.C_out, ho, wo, act), ("bwd_data", dxq, fg, d.C_in, d.H, d.W, mq.ACT_NONE)):
+        Cp, Nt = (C + 31) // 32 * 32, (d.N + 31) // 32
+        codes = q_out.codes.view(Hh * Ww, d.N, int(Cp * bpe(fmt_out)))
+        scales = q_out.scales.view(Hh * Ww, Nt, Cp // 32)
+        for slab in sorted({0, Nt - 1}):
+            n0, n1 = 32 * slab, min(d.N, 32 * slab + 32)
+            assert n1 - n0 == 32
+            ds = d._replace(N=32)
+            if what == "fwd":
+                oc, osc = oracle.quantize(ds, oracle.ROLE_X, fx, x[n0:n1])
+                ah = oracle.dequant(ds, oracle.ROLE_X, fx, oc, osc)
+            else:
+                oc, osc = oracle.quantize(ds, oracle.ROLE_DY, fg, g[n0:n1])
+                ah = oracle.dequant(ds, oracle.ROLE_DY, fg, oc, osc)
+            border = [0, Ww - 1, (Hh - 1) * Ww, Hh * Ww - 1, Ww // 2, (Hh // 2) * Ww]
+            tiles = _tiles_of_slab(rng, Hh * Ww, Cp // 32, border, T)
+            nn, cc = np.meshgrid(np.arange(32), np.arange(32), indexing="ij")
+            idx = np.concatenate([((nn * C + 32 * cb + cc) * (Hh * Ww) + p).reshape(-1) for p, cb in tiles]).astype(np.int64)
+            ref, ab = oracle.conv_fwd(ds, ah, wh, idx) if what == "fwd" else oracle.conv_bwd_data(ds, wh, ah, idx)
+            # the tiles side by side as one pixel of a 32-sample tensor with 32 T channels
+            y64 = ref.reshape(T, 32, 32).transpose(1, 0, 2).reshape(32, 32 * T, 1, 1)
+            bnd = (GEMM_TOL * ab).reshape(T, 32, 32).transpose(1, 0, 2).reshape(32, 32 * T, 1, 1)
+            bb = int(32 * bpe(fmt_out))
+            got = types.SimpleNamespace(
+                codes=torch.cat([codes[p, n0:n1, cb * bb:(cb + 1) * bb] for p, cb in tiles], dim=1).contiguous().reshape(-1),
+                scales=torch.stack([scales[p, slab, cb] for p, cb in tiles]).contiguous())
+            if what == "fwd":
+                d_out, role = inputs.conv_desc(32, 32 * T, 1, 1, 32, 1, 1, 0), oracle.ROLE_X
+            else:
+                d_out, role = inputs.conv_desc(32, 32, 1, 1, 32 * T, 1, 1, 0), oracle.ROLE_DY
+            check_emitted(f"{name} {what} slab {slab}", d_out, role, fmt_out, y64, bnd, a, got)
+
+
 def test_bad_arguments():
     d = inputs.conv_desc(32, 64, 6, 6, 64, 3, 1, 1)
     xq, wq = mq.quantize(d, mq.ROLE_X, E4M3, dev(inputs.make_x(d, 1))), mq.quantize(d, mq.ROLE_W, E4M3, dev(inputs.make_w(d, 1)))

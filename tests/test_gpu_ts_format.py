@@ -7,7 +7,7 @@ import torch
 
 import oracle
 from paper_2609_28358_b200 import inputs, mq
-from parity_util import GEMM_TOL, assert_gemm_close, assert_same_bytes, dev, host
+from parity_util import GEMM_TOL, assert_gemm_close, assert_same_bytes, check_large_layer, dev, host
 
 pytestmark = pytest.mark.gpu
 
@@ -97,6 +97,14 @@ def test_whole_line_quantizer(knobs, name, shape):
         assert_same_bytes(g3.scales, o3[1], f"{name} {what} stochastic: block scales")
         assert_same_bytes(g3.codes, o3[0], f"{name} {what} stochastic: codes")
     assert mq.last_device_status() == 0
+
+
+@pytest.mark.parametrize("name", ["cfg5_e2m1_k3s1_c512_hw28", "cfg5_e2m1_k3s2_c512_hw28", "cfg5_e2m1_k1s1_c512_hw28", "cfg5_e2m1_k3s1_c256_hw56",
+                                  "cfg5_e2m1_k3s1_c512_hw56"])
+def test_config5_points_full_size(name):
+    """The points `bench.py` times in this format ('<layer>+ts16'), on the GPU at full size; the oracle checks sample slabs,
+    channel blocks and W with the whole tensor's maximum supplied (see check_large_layer)."""
+    check_large_layer({l.name: l for l in inputs.config5()}[name], block=mq.TS16)
 
 
 def test_tensor_core_and_cuda_core_routes_agree(knobs):
