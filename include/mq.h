@@ -49,7 +49,8 @@
  *   written operation; both roundings go to nearest, ties to even, and saturate; a block of zeros has scale 0.
  *   All calls accept it (both operands of a GEMM must use it).  The three GEMMs run on the tensor cores (E4M3 scale per 16
  *   elements of the contraction axis, the tensors' fp32 scales applied to the accumulator) for the layers the MX E2M1
- *   path takes, on the CUDA-core kernels otherwise; mq_conv_fwd_mx / mq_conv_bwd_data_mx do not take it.
+ *   path takes, on the CUDA-core kernels otherwise; the quantizing producer epilogue of this format is
+ *   mq_conv_fwd_ts / mq_conv_bwd_data_ts (mq_conv_fwd_mx / mq_conv_bwd_data_mx do not take it).
  */
 #ifndef MQ_H_
 #define MQ_H_
@@ -229,6 +230,26 @@ mq_status mq_conv_fwd_mx(const mq_conv_desc* desc, const mq_qtensor* xq, const m
                          size_t ws_bytes, void* stream);
 mq_status mq_conv_bwd_data_mx(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, mq_qtensor* dxq, void* workspace,
                               size_t ws_bytes, void* stream);
+
+/* The same producer epilogue in the paper's own number format (Sec. III-A, Eq. 4-6; MQ_BLOCK_TS16 operands AND emitted tensor).
+ * Eq. 4 needs the emitted tensor's maximum before its first element can be scaled, which a single pass over the
+ * accumulators cannot know: the maximum is SUPPLIED, from statistics of earlier batches (Sec. VII-B), as for mq_quantize_ts.
+ *   amax_in: device pointer to one fp32, the maximum Eq. 4 uses (4-byte aligned; e.g. the previous step's
+ *            tensor_scale[1] of the same tensor).  Values beyond it saturate (block scale at 448, elements at 6).
+ *   yq / dxq: caller-allocated MQ_BLOCK_TS16 / MQ_E2M1 tensor with the sizes of mq_qtensor_sizes for the NEXT layer's
+ *            role-X tensor (N x C_out x Ho x Wo), resp. the previous layer's role-DY tensor (N x C_in x H x W): codes
+ *            [pixel][N][C_p / 2], scales [pixel][ceil(N/16)][C_p/16] E4M3 bytes; on return tensor_scale[0] =
+ *            amax_in / (448 x 6) and tensor_scale[1] = the emitted tensor's own max|value| (for the next step).
+ * Arithmetic: mq_quantize_ts's, one IEEE single-precision operation per written operation of Eq. 4-6, applied to the
+ * fp32-accumulated GEMM result times the two operands' tensor scales, after the activation.  Round-to-nearest-even.
+ * Layers the tensor-core kernels do not take run as two launches inside the call, as above.
+ * workspace: ws_bytes >= mq_conv_ts_workspace_size(desc, op).  Errors as mq_conv_fwd_mx; operands or output that are not
+ * MQ_BLOCK_TS16 give MQ_ERR_UNSUPPORTED, a null amax_in MQ_ERR_INVALID_ARG. */
+mq_status mq_conv_ts_workspace_size(const mq_conv_desc* desc, int op, size_t* bytes);
+mq_status mq_conv_fwd_ts(const mq_conv_desc* desc, const mq_qtensor* xq, const mq_qtensor* wq, int act, const float* amax_in, mq_qtensor* yq,
+                         void* workspace, size_t ws_bytes, void* stream);
+mq_status mq_conv_bwd_data_ts(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, const float* amax_in, mq_qtensor* dxq,
+                              void* workspace, size_t ws_bytes, void* stream);
 
 /* mq_conv_bwd_weight -- G_Wf = G_Yf . X'^T (Sec. II-C, IV-B; Eq. 3), K-blocks of 32 samples at one
  * output pixel: the stored X and G_Y are read along N, the other direction of their square blocks.

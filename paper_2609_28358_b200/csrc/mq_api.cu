@@ -143,7 +143,7 @@ struct ConvTcPlan {
 // ts16: the paper's own format (E2M1 elements, one E4M3 scale per 16 x 16 block, an fp32 scale per tensor): kind::mxf4nvf4, per-tap kernel.
 bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, ConvTcPlan* out, bool line = false, bool mx = false, bool ts16 = false) {
   const bool fp4 = fmt_w == MQ_E2M1;
-  if (ts16 && (!fp4 || fmt_x_like != MQ_E2M1 || mx || line)) return false;
+  if (ts16 && (!fp4 || fmt_x_like != MQ_E2M1 || line)) return false;
   const int bits = fp4 ? 4 : 8;
   const int taps = g.Kh * g.Kw;
   ConvTcParams p{};
@@ -198,13 +198,13 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
                 // narrowest: with one column a warp's 32 rows ARE a sample tile, and the epilogue needs no exchange between warps
                 // (measured, N = 256, 4 -> 1 columns: 1x1 512 channels 56x56 417 -> 368 us, 3x3 stride 2 input gradient 267 -> 234 us)
       double best = 1e30;
-      for (int tw = 1; tw <= 4; tw <<= 1) {
+      for (int tw = 1; tw <= (ts16 ? 2 : 4); tw <<= 1) {   // emitting 16-sample blocks: a warp's rows must hold whole blocks (1 or 2 columns)
         const int tn = 128 / tw;
         const double waste = (double)((w_eff + tw - 1) / tw * tw) / w_eff * (double)((g.N + tn - 1) / tn * tn) / g.N;
         if (waste < best * (1.0 - 1e-9)) { best = waste; p.TW = tw; }
       }
       const int ftw = env_int("MQ_TC_MX_TW", 0);
-      if (ftw == 1 || ftw == 2 || ftw == 4) p.TW = ftw;
+      if (ftw == 1 || ftw == 2 || (ftw == 4 && !ts16)) p.TW = ftw;
     }
   }
   if (p.TW < 1 || p.TW > 32 || (p.TW & (p.TW - 1))) return false;
@@ -213,7 +213,7 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   while ((1 << p.lgTW) < p.TW) ++p.lgTW;
   const int forced_bn = env_int("MQ_TC_BN", 0);
   if (forced_bn >= 32 && forced_bn <= 256 && forced_bn % 32 == 0) p.BN = forced_bn < cd16 ? forced_bn : cd16;
-  if (mx && (p.BN % 32 != 0 || p.TW > 4)) return false;
+  if (mx && (p.BN % 32 != 0 || p.TW > (ts16 ? 2 : 4))) return false;
   p.tiles_c = (p.Cd + p.BN - 1) / p.BN;
   p.tiles_w = (w_eff + p.TW - 1) / p.TW;
   p.tiles_n = (g.N + p.TN - 1) / p.TN;
@@ -841,14 +841,27 @@ void mx_out_sizes(const Geom& g, int op, int fmt, size_t* cb, size_t* sb) {
   *cb = (size_t)(P * g.N * Cp) * fmt_bits(fmt) / 8;
   *sb = (size_t)(P * g.Nt * (Cp / 32));
 }
+// ts: the paper's own format in and out (MQ_BLOCK_TS16 everywhere); ts_amax: the maximum Eq. 4 takes for the emitted tensor
 mq_status run_conv_mx(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int role_a, const mq_qtensor* qb, int role_b, int act, mq_qtensor* out,
-                      int role_out, void* ws, size_t ws_bytes, void* stream, size_t* size_query) {
+                      int role_out, void* ws, size_t ws_bytes, void* stream, size_t* size_query, bool ts = false, const float* ts_amax = nullptr) {
   mq_status st = check_desc(desc);
   if (st != MQ_OK) return st;
   const Geom g = make_geom(*desc);
   int fmt_x_like, fmt_w;
   if (size_query) {   // formats only: qa / qb carry them in their fmt fields
     fmt_x_like = op == MQ_OP_FWD ? qa->fmt : qb->fmt; fmt_w = op == MQ_OP_FWD ? qb->fmt : qa->fmt;
+  } else if (ts) {
+    if ((st = check_qtensor(g, qa, role_a)) != MQ_OK) return st;
+    if ((st = check_qtensor(g, qb, role_b)) != MQ_OK) return st;
+    if (!out || !out->codes || !out->scales || !out->tensor_scale || out->fmt != MQ_E2M1 || out->role != role_out || !ts_amax) return MQ_ERR_INVALID_ARG;
+    if (act != MQ_ACT_NONE && act != MQ_ACT_RELU && act != MQ_ACT_SILU) return MQ_ERR_INVALID_ARG;
+    if (qa->block != MQ_BLOCK_TS16 || qb->block != MQ_BLOCK_TS16 || out->block != MQ_BLOCK_TS16) return MQ_ERR_UNSUPPORTED;
+    if (!aligned16(out->codes) || !aligned16(out->scales) || (ws && !aligned16(ws)) || (reinterpret_cast<uintptr_t>(out->tensor_scale) & 7u) ||
+        (reinterpret_cast<uintptr_t>(ts_amax) & 3u)) return MQ_ERR_ALIGNMENT;
+    const long long P = op == MQ_OP_FWD ? (long long)g.Ho * g.Wo : (long long)g.H * g.W;
+    const long long Cdp = op == MQ_OP_FWD ? g.Cop : g.Cp;
+    if (out->codes_bytes < (size_t)(P * g.N * Cdp / 2) || out->scales_bytes < (size_t)(P * ((g.N + 15) / 16) * (Cdp / 16))) return MQ_ERR_BUFFER_TOO_SMALL;
+    fmt_x_like = fmt_w = MQ_E2M1;
   } else {
     if ((st = check_qtensor(g, qa, role_a)) != MQ_OK) return st;
     if ((st = check_qtensor(g, qb, role_b)) != MQ_OK) return st;
@@ -862,7 +875,7 @@ mq_status run_conv_mx(int op, const mq_conv_desc* desc, const mq_qtensor* qa, in
     fmt_x_like = op == MQ_OP_FWD ? qa->fmt : qb->fmt; fmt_w = op == MQ_OP_FWD ? qb->fmt : qa->fmt;
   }
   ConvTcPlan pl;
-  if (!conv_tc_eligible(op, g, fmt_x_like, fmt_w) || !conv_tc_plan(op, g, fmt_x_like, fmt_w, MQ_HWNC, &pl, false, true)) {
+  if (!conv_tc_eligible(op, g, fmt_x_like, fmt_w) || !conv_tc_plan(op, g, fmt_x_like, fmt_w, MQ_HWNC, &pl, false, true, ts)) {
     // layers the tensor-core kernels do not take: the same result in two launches - the CUDA-core GEMM writes fp32
     // [pixel][sample][channel] into scratch and the channel-fastest quantizer, which applies the activation, reads it back
     const long long P = op == MQ_OP_FWD ? (long long)g.Ho * g.Wo : (long long)g.H * g.W;
@@ -876,22 +889,29 @@ mq_status run_conv_mx(int op, const mq_conv_desc* desc, const mq_qtensor* qa, in
     a.g = g;
     a.a_codes = static_cast<const uint8_t*>(qa->codes); a.a_scales = qa->scales; a.fmt_a = qa->fmt;
     a.b_codes = static_cast<const uint8_t*>(qb->codes); a.b_scales = qb->scales; a.fmt_b = qb->fmt;
-    a.out = reinterpret_cast<float*>(base); a.out_layout = MQ_HWNC; a.workspace = base + y_bytes; a.ws_bytes = ws_bytes - y_bytes; a.line = 0; a.ts16 = 0; a.a_tscale = nullptr; a.b_tscale = nullptr;
+    a.out = reinterpret_cast<float*>(base); a.out_layout = MQ_HWNC; a.workspace = base + y_bytes; a.ws_bytes = ws_bytes - y_bytes; a.line = 0;
+    a.ts16 = ts ? 1 : 0; a.a_tscale = ts ? qa->tensor_scale : nullptr; a.b_tscale = ts ? qb->tensor_scale : nullptr;
     if (launch_conv_generic(op, a, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MQ_ERR_CUDA;
     QuantArgs q{};
     q.src = reinterpret_cast<const float*>(base); q.codes = static_cast<uint8_t*>(out->codes); q.scales = out->scales;
     q.P = (int)P; q.R = g.N; q.C = Cd; q.Cp = Cdp;
     q.out_stride_p = (long long)g.N * Cdp; q.out_stride_r = Cdp;
-    q.sc_stride_p = (long long)g.Nt * (Cdp / 32); q.sc_stride_r = Cdp / 32;
+    q.sc_stride_p = ts ? (long long)((g.N + 15) / 16) * (Cdp / 16) : (long long)g.Nt * (Cdp / 32); q.sc_stride_r = ts ? Cdp / 16 : Cdp / 32;
     q.src_stride_p = (long long)g.N * Cd; q.src_stride_r = Cd;
     q.fmt = out->fmt; q.act = act; q.status = device_status_ptr();
+    if (ts) return launch_quantize_ts(q, ts_amax, out->tensor_scale, static_cast<cudaStream_t>(stream)) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
     return launch_quantize(q, static_cast<cudaStream_t>(stream)) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
   }
   if (size_query) { *size_query = pl.total; return MQ_OK; }
   if (pl.total > 0 && (!ws || ws_bytes < pl.total)) return MQ_ERR_BUFFER_TOO_SMALL;
-  pl.p.mx_fmt = out->fmt; pl.p.mx_act = act;
+  pl.p.mx_fmt = ts ? 5 : out->fmt; pl.p.mx_act = act;   // 5: the emitted tensor is in the paper's own format
   pl.p.mx_codes = static_cast<uint8_t*>(out->codes); pl.p.mx_scales = out->scales;
   pl.p.mx_Cp = op == MQ_OP_FWD ? g.Cop : g.Cp;
+  if (ts) {
+    pl.p.mx_ts_amax = ts_amax; pl.p.mx_ts_stats = out->tensor_scale;
+    // the tensor's own maximum is collected with atomicMax on its bit pattern: start from zero
+    if (cudaMemsetAsync(out->tensor_scale + 1, 0, sizeof(float), static_cast<cudaStream_t>(stream)) != cudaSuccess) return MQ_ERR_CUDA;
+  }
   const mq_qtensor* qx_like = op == MQ_OP_FWD ? qa : qb;
   const mq_qtensor* qw = op == MQ_OP_FWD ? qb : qa;
   return run_conv_tc(op, g, pl, qx_like, qw, nullptr, MQ_HWNC, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
@@ -913,6 +933,25 @@ mq_status mq_conv_fwd_mx(const mq_conv_desc* desc, const mq_qtensor* xq, const m
 mq_status mq_conv_bwd_data_mx(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, mq_qtensor* dxq, void* workspace, size_t ws_bytes,
                               void* stream) {
   return run_conv_mx(MQ_OP_BWD_DATA, desc, wq, MQ_ROLE_W, dyq, MQ_ROLE_DY, MQ_ACT_NONE, dxq, MQ_ROLE_DY, workspace, ws_bytes, stream, nullptr);
+}
+
+mq_status mq_conv_ts_workspace_size(const mq_conv_desc* desc, int op, size_t* bytes) {
+  if (!bytes || (op != MQ_OP_FWD && op != MQ_OP_BWD_DATA)) return MQ_ERR_INVALID_ARG;
+  mq_qtensor a{}, b{};
+  a.fmt = MQ_E2M1; b.fmt = MQ_E2M1;
+  return run_conv_mx(op, desc, &a, 0, &b, 0, 0, nullptr, 0, nullptr, 0, nullptr, bytes, true, nullptr);
+}
+
+mq_status mq_conv_fwd_ts(const mq_conv_desc* desc, const mq_qtensor* xq, const mq_qtensor* wq, int act, const float* amax_in, mq_qtensor* yq, void* workspace,
+                         size_t ws_bytes, void* stream) {
+  if (!xq || !wq) return MQ_ERR_INVALID_ARG;
+  return run_conv_mx(MQ_OP_FWD, desc, xq, MQ_ROLE_X, wq, MQ_ROLE_W, act, yq, MQ_ROLE_X, workspace, ws_bytes, stream, nullptr, true, amax_in);
+}
+
+mq_status mq_conv_bwd_data_ts(const mq_conv_desc* desc, const mq_qtensor* wq, const mq_qtensor* dyq, const float* amax_in, mq_qtensor* dxq, void* workspace,
+                              size_t ws_bytes, void* stream) {
+  if (!wq || !dyq) return MQ_ERR_INVALID_ARG;
+  return run_conv_mx(MQ_OP_BWD_DATA, desc, wq, MQ_ROLE_W, dyq, MQ_ROLE_DY, MQ_ACT_NONE, dxq, MQ_ROLE_DY, workspace, ws_bytes, stream, nullptr, true, amax_in);
 }
 
 // ---- allocation-free variant of mq_conv_bwd_data ---------------------------------------------------

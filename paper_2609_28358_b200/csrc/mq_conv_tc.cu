@@ -350,7 +350,70 @@ struct MxBlockCtx {
   uint8_t* o_codes;
   uint8_t* o_scale;
   uint64_t* tempty_acc;
+  // the paper's own format (FMT 5): product of the operands' tensor scales (applied to the accumulator first), T_scale of the
+  // emitted tensor and 6 T_scale (Eq. 4-5), the running maximum of this warp's emitted values
+  float in_scale, tscale, t6;
+  unsigned* own_max;
 };
+// The paper's own format as the emitted one (FMT 5; Eq. 4-6 with the tensor maximum supplied from an earlier step, Sec. VII-B):
+// E2M1 elements, one E4M3 scale per 16 samples x 16 channels, written [pixel][ceil(N/16)][C_p/16].  A warp's 32 rows are
+// 32 samples of one pixel (one-column tiles: two 16-sample blocks, lanes 0-15 and 16-31) or 16 samples of each of two
+// pixels (two-column tiles: even and odd lanes); a 32-channel block of the accumulator is two 16-channel blocks.  Every
+// operation of Eq. 5-6 is one IEEE single-precision operation in the order written, as in the quantizer.
+template <int ACT>
+__device__ __forceinline__ void ts_block(const ConvTcParams& p, MxBlockCtx& c, int b, uint32_t* v) {
+  float m[2] = {0.f, 0.f};
+  if (c.Q > 0) {
+    tmem_ld_wait();
+#pragma unroll
+    for (int k = 0; k < 32; ++k) {
+      float x = __uint_as_float(v[k]) * c.in_scale;
+      if (ACT != MQ_ACT_NONE) x = mx_activation(x, ACT);
+      v[k] = __float_as_uint(x);
+      m[k >> 4] = fmaxf(m[k >> 4], fabsf(x));
+    }
+  } else {
+#pragma unroll
+    for (int k = 0; k < 32; ++k) v[k] = 0u;
+  }
+  const bool more = c.Q > 0 && b + 1 < c.bend;
+  if (b + 1 == c.bend) {      // the accumulator has been read: hand it back before the arithmetic and the stores
+    tc_fence_before_sync();
+    __syncwarp();
+    if (c.lane == 0) mbar_arrive(c.tempty_acc);
+  }
+  const bool blk_ok = c.row_ok && c.c0 + 32 * b < p.mx_Cp;
+  float den[2];
+  unsigned sc2 = 0;
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    const unsigned mb = __reduce_max_sync(c.col_mask, c.row_ok ? __float_as_uint(m[h]) : 0u);
+    const float bmax = __uint_as_float(mb);
+    *c.own_max = max(*c.own_max, mb);
+    unsigned sc = 0;
+    if (bmax > 0.f && c.tscale > 0.f) sc = (unsigned)__nv_cvt_float_to_fp8(__fdiv_rn(bmax, c.t6), __NV_SATFINITE, __NV_E4M3) & 0x7Fu;   // Eq. 5
+    const __half_raw hr = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)sc, __NV_E4M3);
+    const float bscale = __half2float(*reinterpret_cast<const __half*>(&hr));
+    den[h] = (bscale > 0.f && c.tscale > 0.f) ? __fmul_rn(bscale, c.tscale) : 0.f;
+    sc2 |= sc << (8 * h);
+  }
+  // the first lane of each 16-sample block writes the two scale bytes of its 32 channels
+  if (blk_ok && c.lane == __ffs(c.col_mask) - 1) *reinterpret_cast<unsigned short*>(c.o_scale + 2 * b) = (unsigned short)sc2;
+  uint8_t* dst = c.o_codes + 16 * b;
+#pragma unroll
+  for (int h = 0; h < 2; ++h) {
+    unsigned w[2] = {0u, 0u};
+#pragma unroll
+    for (int k = 0; k < 16; k += 2) {
+      const float x0 = __uint_as_float(v[16 * h + k]), x1 = __uint_as_float(v[16 * h + k + 1]);
+      const float q0 = ts_div(x0, den[h]), q1 = ts_div(x1, den[h]);                                   // Eq. 6
+      w[k >> 3] |= encode2<MQ_E2M1>(q0, q1) << (4 * (k & 7));
+    }
+    if (blk_ok) *reinterpret_cast<uint2*>(dst + 8 * h) = make_uint2(w[0], w[1]);
+    if (more) tmem_ld_32x32b_x16(c.taddr + 32 * (b + 1) + 16 * h, v + 16 * h);
+  }
+}
+
 // One 32-channel block of a warp's 32 rows.  v holds (or is about to hold) the block's accumulator values; each half of
 // the next block's load is issued as soon as its 16 registers have been converted, so it is in flight during the rest of
 // the conversion, the stores and the loop's bookkeeping (a second register buffer, which would put the whole of the next
@@ -421,11 +484,21 @@ __device__ __forceinline__ void epilogue_mx_role(const ConvTcParams& p, unsigned
     const int nblk = p.BN >> 5;                         // 32-channel blocks of a tile
     const int bbeg = half == 0 ? 0 : (nblk + 1) >> 1, bend = half == 0 ? (nblk + 1) >> 1 : nblk;
     const int grp0 = quad & ~(p.TW - 1);                // first quadrant of the TW quadrants that hold this sample tile
-    constexpr int emax = FMT == MQ_E4M3 ? 8 : (FMT == MQ_E5M2 ? 15 : (FMT == MQ_E3M2 ? 4 : 2));
-    constexpr int bpe4 = FMT == MQ_E2M1 ? 1 : 2;        // bytes per element x 2
-    const int Ct = p.mx_Cp >> 5;
+    constexpr bool TS = FMT == 5;                       // the paper's own format (16 x 16 blocks; TW is 1 or 2)
+    constexpr int bpe4 = (FMT == MQ_E2M1 || TS) ? 1 : 2;        // bytes per element x 2
+    const int Ct = TS ? p.mx_Cp >> 4 : p.mx_Cp >> 5;
     unsigned* my_red = red + half * 32;                 // [parity][quadrant][column]
-    const unsigned col_mask = (p.TW == 1 ? 0xffffffffu : (p.TW == 2 ? 0x55555555u : 0x11111111u)) << (lane & (p.TW - 1));   // lanes of this lane's column
+    // lanes of this lane's column (TS: of its 16-sample block - half a warp with one-column tiles)
+    const unsigned col_mask = TS ? (p.TW == 1 ? 0xffffu << (lane & 16) : 0x55555555u << (lane & 1))
+                                 : (p.TW == 1 ? 0xffffffffu : (p.TW == 2 ? 0x55555555u : 0x11111111u)) << (lane & (p.TW - 1));
+    unsigned own_max = 0;
+    float ts_in = 1.f, ts_t = 0.f, ts_t6 = 0.f;
+    if (TS) {
+      ts_in = out_scale_of(p);
+      ts_t = __fdiv_rn(__ldg(p.mx_ts_amax), __fmul_rn(448.0f, 6.0f));                       // Eq. 4
+      ts_t6 = __fmul_rn(ts_t, 6.0f);
+      if (blockIdx.x == 0 && warp == 4 && lane == 0) p.mx_ts_stats[0] = ts_t;
+    }
     uint32_t tcount = 0;
     for (unsigned t = blockIdx.x; t < total; t += gridDim.x, ++tcount) {
       const Tile tile = decode_tile(p, t);
@@ -450,33 +523,52 @@ __device__ __forceinline__ void epilogue_mx_role(const ConvTcParams& p, unsigned
       const uint32_t taddr = tmem + acc * p.BN + ((uint32_t)(32 * quad) << 16);
       const long long pix = (long long)yo * p.Wd + xo;
       uint8_t* o_codes = p.mx_codes + (((pix * p.N + n) * p.mx_Cp + tile.c0) * bpe4 >> 1);
-      uint8_t* o_scale = p.mx_scales + (pix * p.Nt + (n >> 5)) * Ct + (tile.c0 >> 5);
+      uint8_t* o_scale = TS ? p.mx_scales + (pix * ((p.N + 15) >> 4) + (n >> 4)) * Ct + (tile.c0 >> 4)
+                            : p.mx_scales + (pix * p.Nt + (n >> 5)) * Ct + (tile.c0 >> 5);
       // no separate activation pass for none / ReLU: the maximum of max(x, 0) is the maximum of x and 0, and negative
       // codes are cleared after packing
       MxBlockCtx c;
       c.Q = Q; c.bend = bend; c.taddr = taddr; c.row_ok = row_ok; c.col_mask = col_mask; c.my_red = my_red; c.half = half; c.quad = quad;
       c.grp0 = grp0; c.tw_ = tw_; c.lane = lane; c.o_codes = o_codes; c.o_scale = o_scale; c.c0 = tile.c0; c.tempty_acc = &tempty[acc];
+      c.in_scale = ts_in; c.tscale = ts_t; c.t6 = ts_t6; c.own_max = &own_max;
       uint32_t v[32];
       if (Q > 0 && bbeg < bend) {
         tmem_ld_32x32b_x16(taddr + 32 * bbeg, v);
         tmem_ld_32x32b_x16(taddr + 32 * bbeg + 16, v + 16);
       }
       // the activation is chosen outside the block loop: three straight-line copies instead of a test per element
-      if (p.mx_act == MQ_ACT_RELU) {
+      if constexpr (TS) {
+        if (p.mx_act == MQ_ACT_RELU) {
 #pragma unroll 1
-        for (int b = bbeg; b < bend; ++b) mx_block<FMT, MQ_ACT_RELU>(p, c, b, v);
-      } else if (p.mx_act == MQ_ACT_SILU) {
+          for (int b = bbeg; b < bend; ++b) ts_block<MQ_ACT_RELU>(p, c, b, v);
+        } else if (p.mx_act == MQ_ACT_SILU) {
 #pragma unroll 1
-        for (int b = bbeg; b < bend; ++b) mx_block<FMT, MQ_ACT_SILU>(p, c, b, v);
+          for (int b = bbeg; b < bend; ++b) ts_block<MQ_ACT_SILU>(p, c, b, v);
+        } else {
+#pragma unroll 1
+          for (int b = bbeg; b < bend; ++b) ts_block<MQ_ACT_NONE>(p, c, b, v);
+        }
       } else {
+        if (p.mx_act == MQ_ACT_RELU) {
 #pragma unroll 1
-        for (int b = bbeg; b < bend; ++b) mx_block<FMT, MQ_ACT_NONE>(p, c, b, v);
+          for (int b = bbeg; b < bend; ++b) mx_block<FMT, MQ_ACT_RELU>(p, c, b, v);
+        } else if (p.mx_act == MQ_ACT_SILU) {
+#pragma unroll 1
+          for (int b = bbeg; b < bend; ++b) mx_block<FMT, MQ_ACT_SILU>(p, c, b, v);
+        } else {
+#pragma unroll 1
+          for (int b = bbeg; b < bend; ++b) mx_block<FMT, MQ_ACT_NONE>(p, c, b, v);
+        }
       }
       if (bbeg >= bend) {      // a tile of 32 channels leaves the second half without a block
         tc_fence_before_sync();
         __syncwarp();
         if (lane == 0) mbar_arrive(&tempty[acc]);
       }
+    }
+    if (TS) {   // this tensor's own maximum, for the next step's Eq. 4: one atomic per warp
+      const unsigned wmax = __reduce_max_sync(0xffffffffu, own_max);
+      if (lane == 0 && wmax != 0) atomicMax(reinterpret_cast<unsigned*>(p.mx_ts_stats + 1), wmax);
     }
 }
 
@@ -1758,6 +1850,11 @@ cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, cons
     MQ_TC_MX5(MQ_OP_BWD_DATA, 128, true);  MQ_TC_MX5(MQ_OP_BWD_DATA, 64, true);  MQ_TC_MX5(MQ_OP_BWD_DATA, 32, true);
 #undef MQ_TC_MX5
 #undef MQ_TC_MX
+    // the paper's own format in and out: kind 2 operands, emitted format 5
+#define MQ_TC_TS(M, K) if (p.mode == M && p.KB == K && p.kind_fp4 == 2 && p.mx_fmt == 5) return launch_conv_tc_inst<M, K, 2, 5>(p, map_a, map_w, map_out, s)
+    MQ_TC_TS(MQ_OP_FWD, 128); MQ_TC_TS(MQ_OP_FWD, 64); MQ_TC_TS(MQ_OP_FWD, 32);
+    MQ_TC_TS(MQ_OP_BWD_DATA, 128); MQ_TC_TS(MQ_OP_BWD_DATA, 64); MQ_TC_TS(MQ_OP_BWD_DATA, 32);
+#undef MQ_TC_TS
     return cudaErrorInvalidValue;
   }
 #define MQ_TC_CASE(M, K, F) if (p.mode == M && p.KB == K && p.kind_fp4 == F) return launch_conv_tc_inst<M, K, F>(p, map_a, map_w, map_out, s)

@@ -78,7 +78,10 @@ struct ConvTcParams {
   unsigned int* status;
   // quantizing epilogue (the producer emits the next tensor's MX tiles instead of fp32, see epilogue_mx_role)
   int mx_out;               // 1: on
-  int mx_fmt, mx_act;       // element format of the emitted tensor; activation applied first (mq_act)
+  int mx_fmt, mx_act;       // element format of the emitted tensor (5: the paper's own format - E2M1, E4M3 scale per 16 x 16 block, fp32
+                            // tensor scale from mx_ts_amax); activation applied first (mq_act)
+  const float* mx_ts_amax;  // format 5: the maximum Eq. 4 takes (device; an earlier step's)
+  float* mx_ts_stats;       // format 5: [0] receives T_scale, [1] (zero on entry) this tensor's own maximum
   uint8_t* mx_codes;        // [Hd][Wd][N][mx_Cp] codes
   uint8_t* mx_scales;       // [Hd][Wd][Nt][mx_Cp / 32] tile scales
   int mx_Cp;                // Cd rounded up to 32

@@ -184,6 +184,16 @@ __device__ __forceinline__ unsigned encode2(float lo, float hi) {
   }
 }
 
+// x / den of Eq. 6 (den = Scale_b x T_scale, or 0 for an all-zero block / tensor: the element is then a signed zero).  A zero
+// numerator would send __fdiv_rn down its slow path (a call that the whole warp waits for - post-ReLU tensors are half
+// zeros: measured 2x on the quantizing epilogue), so zeros divide a stand-in and keep their sign; the quotient of every
+// other value is the IEEE one.
+__device__ __forceinline__ float ts_div(float x, float den) {
+  const bool z = x == 0.f || !(den > 0.f);
+  const float q = __fdiv_rn(z ? 1.f : x, z ? 1.f : den);
+  return z ? copysignf(0.f, x) : q;
+}
+
 // activation of the quantizing producer epilogue (mq_act), evaluated in fp32
 __device__ __forceinline__ float mx_activation(float y, int act) {
   if (act == MQ_ACT_RELU) return fmaxf(y, 0.f);

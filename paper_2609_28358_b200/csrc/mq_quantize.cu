@@ -543,7 +543,7 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_con
             float x[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-              if (TS) x[j] = dn > 0.f ? __fdiv_rn(v[b][k + j], dn) : copysignf(0.f, v[b][k + j]);   // Eq. 6
+              if (TS) x[j] = ts_div(v[b][k + j], dn);   // Eq. 6
               else x[j] = v[b][k + j] * f;
               if (SR && (!TS || dn > 0.f)) {
                 const long long e = ((long long)(q.r0 + n) * a.C + q.c0 + chalf * 16 + k + j) * a.P + q.p0 + lane;

@@ -21,16 +21,18 @@
 namespace mq {
 namespace {
 
-__global__ void __launch_bounds__(256) tensor_amax_kernel(const float* __restrict__ src, long long n, unsigned* __restrict__ amax_bits) {
+// act: mq_act applied to every element first (the two-launch route of the quantizing epilogue), 0 = none
+__global__ void __launch_bounds__(256) tensor_amax_kernel(const float* __restrict__ src, long long n, unsigned* __restrict__ amax_bits, int act) {
   pdl_wait();
   float m = 0.f;
   const long long n4 = (reinterpret_cast<uintptr_t>(src) & 15) == 0 ? n >> 2 : 0;
   const long long stride = (long long)gridDim.x * blockDim.x, t0 = (long long)blockIdx.x * blockDim.x + threadIdx.x;
   for (long long i = t0; i < n4; i += stride) {
-    const float4 v = __ldg(reinterpret_cast<const float4*>(src) + i);
+    float4 v = __ldg(reinterpret_cast<const float4*>(src) + i);
+    if (act) { v.x = mx_activation(v.x, act); v.y = mx_activation(v.y, act); v.z = mx_activation(v.z, act); v.w = mx_activation(v.w, act); }
     m = fmaxf(fmaxf(m, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
   }
-  for (long long i = 4 * n4 + t0; i < n; i += stride) m = fmaxf(m, fabsf(__ldg(src + i)));
+  for (long long i = 4 * n4 + t0; i < n; i += stride) m = fmaxf(m, fabsf(act ? mx_activation(__ldg(src + i), act) : __ldg(src + i)));
   const unsigned w = __reduce_max_sync(0xffffffffu, __float_as_uint(m));    // bit patterns of non-negative floats order like the values
   if ((threadIdx.x & 31) == 0 && w != 0) atomicMax(amax_bits, w);
 }
@@ -83,7 +85,7 @@ __global__ void __launch_bounds__(256) quantize_ts_kernel(QuantArgs a, const flo
           if (p0 + j < a.P) {
             const float* q = a.src + (long long)(p0 + j) * a.src_stride_p + (long long)r * a.src_stride_r + c0;
 #pragma unroll
-            for (int k = 0; k < 8; ++k) if (c0 + k < a.C) v[k][j] = __ldg(q + k);
+            for (int k = 0; k < 8; ++k) if (c0 + k < a.C) v[k][j] = a.act ? mx_activation(__ldg(q + k), a.act) : __ldg(q + k);
           }
         }
       }
@@ -104,8 +106,8 @@ __global__ void __launch_bounds__(256) quantize_ts_kernel(QuantArgs a, const flo
       unsigned word = 0;
 #pragma unroll
       for (int k = 0; k < 8; k += 2) {
-        float x0 = live ? __fdiv_rn(v[k][j], den) : copysignf(0.f, v[k][j]);                 // Eq. 6
-        float x1 = live ? __fdiv_rn(v[k + 1][j], den) : copysignf(0.f, v[k + 1][j]);
+        float x0 = ts_div(v[k][j], live ? den : 0.f);                                         // Eq. 6
+        float x1 = ts_div(v[k + 1][j], live ? den : 0.f);
         if (SR && live) {
           const long long e0 = ((long long)r * a.C + c0 + k) * a.P + p0 + j;
           x0 = sr_value<MQ_E2M1>(x0, (unsigned)e0, sr_key(a, e0));
@@ -133,7 +135,8 @@ cudaError_t launch_quantize_ts(const QuantArgs& a, const float* amax_in, float* 
   if (blocks > (long long)sm_count() * 8) blocks = (long long)sm_count() * 8;
   if (blocks < 1) blocks = 1;
   // the source of either layout is a dense array of n floats
-  e = launch_pdl(tensor_amax_kernel, dim3((unsigned)blocks), dim3(256), 0, s, a.src, n, reinterpret_cast<unsigned*>(stats + 1));
+  if (a.act && a.src_stride_r == 0) return cudaErrorInvalidValue;   // the activation rides on the channel-fastest source only
+  e = launch_pdl(tensor_amax_kernel, dim3((unsigned)blocks), dim3(256), 0, s, a.src, n, reinterpret_cast<unsigned*>(stats + 1), a.act);
   if (e != cudaSuccess) return e;
   const int Rb = (a.R + 15) / 16, Cb = a.Cp / 16;
   const long long n_pstrips = (a.P + 7) / 8, n_items = n_pstrips * Rb * Cb;

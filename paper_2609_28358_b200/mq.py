@@ -263,6 +263,50 @@ def conv_bwd_data_mx(desc, wq, dyq, fmt, dxq=None, workspace=None, stream=None):
     return _conv_mx("mq_conv_bwd_data_mx", OP_BWD_DATA, desc, wq, dyq, dxq, (), workspace, stream)
 
 
+def conv_ts_workspace_size(desc, op):
+    b = ctypes.c_size_t()
+    _check("mq_conv_ts_workspace_size", lib().mq_conv_ts_workspace_size(ctypes.byref(_d(desc)), op, ctypes.byref(b)))
+    return b.value
+
+
+def _ts_out(desc, op, role, device):
+    """An empty stored tensor in the paper's own format of what the quantizing epilogue emits (see _mx_out)."""
+    d = ConvDesc(*desc)
+    ho, wo = _out_hw(d)
+    c, h, w = (d.C_out, ho, wo) if op == OP_FWD else (d.C_in, d.H, d.W)
+    cp = (c + 31) // 32 * 32
+    return QTensor(_new(h * w * d.N * cp // 2, torch.uint8, device), _new(h * w * ((d.N + 15) // 16) * (cp // 16), torch.uint8, device), E2M1, role, TS16,
+                   _new(2, torch.float32, device))
+
+
+def _conv_ts(name, op, desc, qa, qb, out, extra, workspace, stream):
+    need = conv_ts_workspace_size(desc, op)
+    if workspace is None and need > 0:
+        workspace = _new(need, torch.uint8, qa.codes.device)
+    wp = ctypes.c_void_p(workspace.data_ptr()) if workspace is not None else None
+    wn = workspace.numel() * workspace.element_size() if workspace is not None else 0
+    a, b, o = qa._c(), qb._c(), out._c()
+    _check(name, getattr(lib(), name)(ctypes.byref(_d(desc)), ctypes.byref(a), ctypes.byref(b), *extra, ctypes.byref(o), wp, ctypes.c_size_t(wn), _stream(stream)))
+    return out
+
+
+def conv_fwd_ts(desc, xq, wq, amax_in, act=ACT_NONE, yq=None, workspace=None, stream=None):
+    """mq_conv_fwd_ts: act(conv(X, W)) emitted as the next layer's stored activation in the paper's own format; amax_in: a
+    device float tensor holding the maximum Eq. 4 uses (an earlier step's tensor_scale[1:2])."""
+    assert amax_in.is_cuda and amax_in.dtype == torch.float32 and amax_in.numel() >= 1
+    if yq is None:
+        yq = _ts_out(desc, OP_FWD, ROLE_X, xq.codes.device)
+    return _conv_ts("mq_conv_fwd_ts", OP_FWD, desc, xq, wq, yq, (ctypes.c_int(act), ctypes.c_void_p(amax_in.data_ptr())), workspace, stream)
+
+
+def conv_bwd_data_ts(desc, wq, dyq, amax_in, dxq=None, workspace=None, stream=None):
+    """mq_conv_bwd_data_ts: the input gradient emitted as the previous layer's stored output gradient in the paper's own format."""
+    assert amax_in.is_cuda and amax_in.dtype == torch.float32 and amax_in.numel() >= 1
+    if dxq is None:
+        dxq = _ts_out(desc, OP_BWD_DATA, ROLE_DY, wq.codes.device)
+    return _conv_ts("mq_conv_bwd_data_ts", OP_BWD_DATA, desc, wq, dyq, dxq, (ctypes.c_void_p(amax_in.data_ptr()),), workspace, stream)
+
+
 STATIC_SCRATCH_BYTES = 16 << 20
 
 

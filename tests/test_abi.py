@@ -115,3 +115,21 @@ def test_bad_arguments_are_rejected_on_the_host(mq):
     assert L.mq_conv_fwd(ctypes.byref(good), ctypes.byref(ql), ctypes.byref(qw), out, F32, NCHW, None, 0, None) == 2  # mixed block shapes
     assert L.mq_conv_bwd_data(ctypes.byref(good), ctypes.byref(qwl), ctypes.byref(qgl), out, F32, NCHW, None, 0, None) == 2
     assert L.mq_conv_bwd_weight(ctypes.byref(good), ctypes.byref(ql), ctypes.byref(qgl), out, F32, NCHW, None, 0, None) == 2
+    # the quantizing epilogue in the paper's own format: all three tensors in that format, a supplied maximum
+    E2M1, TS16 = mq.E2M1, mq.TS16
+    ts_x = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, E2M1, 0, TS16, 0x5000)
+    ts_w = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, E2M1, 1, TS16, 0x5000)
+    ts_y = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, E2M1, 0, TS16, 0x5000)
+    amax = ctypes.c_void_p(0x6000)
+    assert L.mq_conv_ts_workspace_size(ctypes.byref(good), 0, None) == 1
+    assert L.mq_conv_ts_workspace_size(ctypes.byref(good), 2, ctypes.byref(cb)) == 1           # no weight-gradient variant
+    assert L.mq_conv_fwd_ts(ctypes.byref(good), ctypes.byref(ts_x), ctypes.byref(ts_w), 0, None, ctypes.byref(ts_y), None, 0, None) == 1   # no maximum
+    assert L.mq_conv_fwd_ts(ctypes.byref(good), ctypes.byref(ts_x), ctypes.byref(ts_w), 7, amax, ctypes.byref(ts_y), None, 0, None) == 1   # no such activation
+    assert L.mq_conv_fwd_ts(ctypes.byref(good), ctypes.byref(q), ctypes.byref(qw), 0, amax, ctypes.byref(ts_y), None, 0, None) == 2        # MX operands
+    mx_y = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, E2M1, 0, 0, 0x5000)
+    assert L.mq_conv_fwd_ts(ctypes.byref(good), ctypes.byref(ts_x), ctypes.byref(ts_w), 0, amax, ctypes.byref(mx_y), None, 0, None) == 2   # MX output
+    small_y = mq._QTensor(0x1000, 0x2000, 16, 16, E2M1, 0, TS16, 0x5000)
+    assert L.mq_conv_fwd_ts(ctypes.byref(good), ctypes.byref(ts_x), ctypes.byref(ts_w), 0, amax, ctypes.byref(small_y), None, 0, None) == 4
+    assert L.mq_conv_fwd_ts(ctypes.byref(good), ctypes.byref(ts_x), ctypes.byref(ts_w), 0, ctypes.c_void_p(0x6002), ctypes.byref(ts_y), None, 0, None) == 3
+    ts_g = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, E2M1, 2, TS16, 0x5000)
+    assert L.mq_conv_bwd_data_ts(ctypes.byref(good), ctypes.byref(ts_w), ctypes.byref(ts_g), None, ctypes.byref(ts_g), None, 0, None) == 1

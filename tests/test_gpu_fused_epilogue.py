@@ -168,6 +168,91 @@ def test_every_tile_width(knobs, fmts, out_fmt, tw):
                   mq.ACT_NONE, dxq)
 
 
+def check_emitted_ts(name, d_out, role, y64, bound, act, amax_in, got):
+    """check_emitted for the paper's own format (16 x 16 blocks, E4M3 block scales, the tensor maximum supplied)."""
+    B16 = (16, 16)
+    lo, hi = _act_interval(y64, bound, act)
+    mid = _act(y64, act)
+    q_lo, q_hi, q_mid = [oracle.quantize_ts(d_out, role, a.astype(np.float32), B16, amax=float(amax_in)) for a in (lo, hi, mid)]
+    stats = host(got.tensor_scale)
+    assert stats[0] == np.float32(amax_in) / (np.float32(448.0) * np.float32(6.0)), (name, stats)
+    # the tensor's own maximum, left for the next step: that of the fp32 result, inside the bracket of the float64 one
+    assert np.abs(lo).max() * (1 - 1e-6) <= stats[1] <= np.abs(hi).max() * (1 + 1e-6) or abs(stats[1] - np.abs(mid).max()) <= bound.max(), (name, stats)
+    g_codes, g_scales = host(got.codes), host(got.scales)
+    assert g_scales.shape == q_mid[1].shape and g_codes.shape == q_mid[0].shape
+    N = d_out.N
+    C = d_out.C_in if role == oracle.ROLE_X else d_out.C_out
+    Cp, Nt = (C + 31) // 32 * 32, (N + 15) // 16
+    P = g_scales.size // (Nt * (Cp // 16))
+    s_lo, s_hi, s_g = [a.reshape(P, Nt, Cp // 16) for a in (q_lo[1], q_hi[1], g_scales)]
+    tile_fixed = s_lo == s_hi
+    assert (s_g[tile_fixed] == s_lo[tile_fixed]).all(), f"{name}: a determined block scale differs"
+    c_lo, c_hi, c_mid, c_g = [_unpack(c, E2M1).reshape(P, N, Cp) for c in (q_lo[0], q_hi[0], q_mid[0], g_codes)]
+    fixed_e = np.repeat(np.repeat(tile_fixed, 16, axis=2), 16, axis=1)[:, :N, :]
+    det = fixed_e & (c_lo == c_hi)
+    bad = det & (c_g != c_lo)
+    assert not bad.any(), f"{name}: {int(bad.sum())} determined codes differ; first at {np.argwhere(bad)[0]}"
+    tab = _decode_table(E2M1)
+    und = fixed_e & ~det
+    v_g, v_lo, v_hi = tab[c_g[und]], tab[c_lo[und]], tab[c_hi[und]]
+    assert ((v_g >= np.minimum(v_lo, v_hi)) & (v_g <= np.maximum(v_lo, v_hi))).all(), f"{name}: a code at a rounding threshold lies outside its interval"
+    frac_und = 1.0 - det.mean()
+    frac_diff = float((c_g != c_mid).mean())
+    assert frac_und < 0.45, (name, frac_und)
+    assert frac_diff < 0.02, (name, frac_diff)
+    return frac_und, frac_diff
+
+
+TS_SHAPES = [
+    ("c128", (140, 128, 6, 5, 128, 3, 1, 1)),          # one-column tiles (two sample tiles of 128, the second ragged), 64-byte chunks
+    ("c256_n48", (48, 256, 5, 6, 256, 3, 1, 1)),       # two-column tiles (64 samples per tile), 256-channel tiles, three 16-sample blocks
+    ("stride2", (64, 64, 9, 10, 192, 3, 2, 1)),        # 32-byte chunks; parity classes of the input gradient
+    ("k1", (32, 512, 3, 4, 320, 1, 1, 0)),
+    ("odd_channels", (36, 40, 6, 6, 72, 3, 1, 1)),     # not a tensor-core layer: the two-launch route
+]
+
+
+@pytest.mark.parametrize("act", [mq.ACT_NONE, mq.ACT_RELU, mq.ACT_SILU], ids=["none", "relu", "silu"])
+@pytest.mark.parametrize("name,shape", TS_SHAPES, ids=[s[0] for s in TS_SHAPES])
+def test_paper_format_in_and_out(name, shape, act):
+    """mq_conv_fwd_ts / mq_conv_bwd_data_ts: operands and emitted tensor in the paper's own format (Eq. 4-6), the emitted
+    tensor's maximum supplied (here: 0.8 x its true maximum, so the top saturates) - against conv in float64 ->
+    activation -> oracle.quantize_ts with that maximum."""
+    B16 = (16, 16)
+    d = inputs.conv_desc(*shape)
+    x, w, g = inputs.make_x(d, 91, "gauss"), inputs.make_w(d, 91), inputs.make_dy(d, 91, "gauss")
+    roles = (oracle.ROLE_X, oracle.ROLE_W, oracle.ROLE_DY)
+    oq = [oracle.quantize_ts(d, r, t, B16) for r, t in zip(roles, (x, w, g))]
+    xh, wh, gh = [oracle.dequant_ts(d, r, o[0], o[1], o[2], B16) for r, o in zip(roles, oq)]
+    gq = [mq.quantize_ts(d, r, dev(t)) for r, t in zip((mq.ROLE_X, mq.ROLE_W, mq.ROLE_DY), (x, w, g))]
+    ho, wo = inputs.out_hw(d)
+    y64, ab = oracle.conv_fwd(d, xh, wh)
+    amax = np.float32(0.8 * np.abs(_act(y64, act)).max())
+    amax_dev = torch.tensor([amax], dtype=torch.float32, device="cuda")
+    n0 = mq.kernel_launch_count()
+    yq = mq.conv_fwd_ts(d, gq[0], gq[1], amax_dev, act)
+    assert mq.last_device_status() == 0
+    assert mq.kernel_launch_count() - n0 == 2      # tensor cores: scale expansion + the GEMM with the quantizing epilogue
+    d_next = d._replace(C_in=d.C_out, H=ho, W=wo)
+    check_emitted_ts(f"{name} fwd", d_next, oracle.ROLE_X, y64, GEMM_TOL * ab, act, amax, yq)
+    # the emitted tensor feeds a following layer like any stored tensor of that format
+    d2 = inputs.conv_desc(d.N, d.C_out, ho, wo, 64, 1, 1, 0)
+    w2q = mq.quantize_ts(d2, mq.ROLE_W, dev(inputs.make_w(d2, 92)))
+    mq.conv_fwd(d2, yq, w2q)
+    assert mq.last_device_status() == 0
+    if act == mq.ACT_NONE:
+        gx64, ab = oracle.conv_bwd_data(d, wh, gh)
+        amax = np.float32(0.8 * np.abs(gx64).max())
+        amax_dev = torch.tensor([amax], dtype=torch.float32, device="cuda")
+        n0 = mq.kernel_launch_count()
+        dxq = mq.conv_bwd_data_ts(d, gq[1], gq[2], amax_dev)
+        assert mq.last_device_status() == 0
+        # 72 output channels are 48-byte rows of K: not a tensor-core layer - CUDA-core GEMM + the quantizer's two passes
+        assert mq.kernel_launch_count() - n0 == (3 if name == "odd_channels" else 2)
+        d_prev = inputs.conv_desc(d.N, 32, d.H, d.W, d.C_in, 1, 1, 0)
+        check_emitted_ts(f"{name} bwd_data", d_prev, oracle.ROLE_DY, gx64, GEMM_TOL * ab, mq.ACT_NONE, amax, dxq)
+
+
 def _tiles_of_slab(rng, n_pix, n_cb, border, count):
     """(pixel, channel block) pairs: the image's corner / edge pixels first, then random ones"""
     pix = list(border) + list(rng.integers(0, n_pix, count))
