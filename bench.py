@@ -217,12 +217,23 @@ def fused_epilogue_times(wl, flush, K, kern, pk):
     from paper_2609_28358_b200 import mq
 
     d, q, f = wl.d, wl.q, wl.fmts
-    ws = torch.empty(max(mq.conv_mx_workspace_size(d, mq.OP_FWD, f[0], f[1]), mq.conv_mx_workspace_size(d, mq.OP_BWD_DATA, f[1], f[2]), 16), dtype=torch.uint8,
-                     device="cuda")
-    yq = mq.conv_fwd_mx(d, q[0], q[1], f[0], mq.ACT_RELU, workspace=ws)
-    dxq = mq.conv_bwd_data_mx(d, q[1], q[2], f[2], workspace=ws)
-    calls = {"conv_fwd_mx": (lambda: mq.conv_fwd_mx(d, q[0], q[1], f[0], mq.ACT_RELU, yq=yq, workspace=ws), "conv_fwd", max(FMT_BITS[f[0]], FMT_BITS[f[1]])),
-             "conv_bwd_data_mx": (lambda: mq.conv_bwd_data_mx(d, q[1], q[2], f[2], dxq=dxq, workspace=ws), "conv_bwd_data", max(FMT_BITS[f[1]], FMT_BITS[f[2]]))}
+    if wl.block == mq.TS16:
+        # the paper's own format: mq_conv_fwd_ts / mq_conv_bwd_data_ts, the emitted tensors' maxima supplied (here: the true ones,
+        # taken from the fp32 outputs of the step that has just run, as an earlier step's statistics would be)
+        am_y = wl.y.abs().max().reshape(1).float()
+        am_dx = wl.dx.abs().max().reshape(1).float()
+        ws = torch.empty(max(mq.conv_ts_workspace_size(d, mq.OP_FWD), mq.conv_ts_workspace_size(d, mq.OP_BWD_DATA), 16), dtype=torch.uint8, device="cuda")
+        yq = mq.conv_fwd_ts(d, q[0], q[1], am_y, mq.ACT_RELU, workspace=ws)
+        dxq = mq.conv_bwd_data_ts(d, q[1], q[2], am_dx, workspace=ws)
+        calls = {"conv_fwd_ts": (lambda: mq.conv_fwd_ts(d, q[0], q[1], am_y, mq.ACT_RELU, yq=yq, workspace=ws), "conv_fwd", 4),
+                 "conv_bwd_data_ts": (lambda: mq.conv_bwd_data_ts(d, q[1], q[2], am_dx, dxq=dxq, workspace=ws), "conv_bwd_data", 4)}
+    else:
+        ws = torch.empty(max(mq.conv_mx_workspace_size(d, mq.OP_FWD, f[0], f[1]), mq.conv_mx_workspace_size(d, mq.OP_BWD_DATA, f[1], f[2]), 16),
+                         dtype=torch.uint8, device="cuda")
+        yq = mq.conv_fwd_mx(d, q[0], q[1], f[0], mq.ACT_RELU, workspace=ws)
+        dxq = mq.conv_bwd_data_mx(d, q[1], q[2], f[2], workspace=ws)
+        calls = {"conv_fwd_mx": (lambda: mq.conv_fwd_mx(d, q[0], q[1], f[0], mq.ACT_RELU, yq=yq, workspace=ws), "conv_fwd", max(FMT_BITS[f[0]], FMT_BITS[f[1]])),
+                 "conv_bwd_data_mx": (lambda: mq.conv_bwd_data_mx(d, q[1], q[2], f[2], dxq=dxq, workspace=ws), "conv_bwd_data", max(FMT_BITS[f[1]], FMT_BITS[f[2]]))}
     res = {}
     for name, (fn, plain, bits) in calls.items():
         for _ in range(3):
@@ -239,8 +250,8 @@ def fused_epilogue_times(wl, flush, K, kern, pk):
         tf = layer_flops(d) / (ms * 1e-3) / 1e12
         peak = pk["bf16_tflops"] * TENSOR_RATIO[bits]
         res[name] = {"ms": ms, "tflops": tf, "frac": tf / peak, "frac_of_published": tf / PUBLISHED["tensor_tflops"][bits],
-                     "fp32_output_call_ms": kern[plain]["ms"], "activation": "relu" if name == "conv_fwd_mx" else "none",
-                     "emits": FMT_NAME[f[0] if name == "conv_fwd_mx" else f[2]]}
+                     "fp32_output_call_ms": kern[plain]["ms"], "activation": "relu" if plain == "conv_fwd" else "none",
+                     "emits": FMT_NAME[f[0] if plain == "conv_fwd" else f[2]] + (" (16x16 blocks, E4M3 scales, supplied maximum)" if wl.block == mq.TS16 else "")}
     res["device_status"] = mq.last_device_status()
     return res
 
@@ -417,7 +428,7 @@ def run_ours(args):
 
     # ---- the two GEMMs with the quantizing producer epilogue (the next tensor leaves the chip in its stored MX form instead of
     # fp32): per-call times beside the fp32-output calls and the quantizer call they replace
-    if world == 1 and wl.block == mq.TILE32:
+    if world == 1:
         out["fused_epilogue"] = fused_epilogue_times(wl, flush, max(3, min(K, 10)), kern, pk)
 
     # ---- the same step on further workloads (device-timed step and per-call roofline only)
@@ -448,6 +459,8 @@ def run_ours(args):
                 "value": 3.0 * layer_flops(w2.d) / (ms2 * 1e-3) / 1e12, "unit": "TFLOPS", "quantize_im2col_gbs": qi2,
                 "kernels": {n: {k: v for k, v in k2[n].items() if k != "algorithmic_bytes"} for n in CALLS},
                 "device_status": mq.last_device_status()}
+            if name.endswith("+ts16"):
+                out["more_workloads"][name]["fused_epilogue"] = fused_epilogue_times(w2, flush, max(3, min(Km, 10)), k2, pk)
             del w2
             torch.cuda.empty_cache()
     if rank == 0 and world == 1 and not args.no_accounting:
