@@ -28,6 +28,12 @@ namespace {
 using namespace tc;
 
 constexpr int TC_THREADS = 512;   // 16 warps: MMA, scale copier, scale expander / loader, 8 epilogue, 5 more loaders
+// The quantizing epilogue of the paper's own format (emitted format 5) runs with 16 epilogue warps (8 more, warps 16-23): a block
+// of it is a chain of latencies (tensor-memory load, warp reductions, IEEE divisions, conversions, stores) that two warps
+// per scheduler do not hide; four do better, at 80 registers per thread (measured, 512 channels 28x28 3x3: 320 -> 278 us).
+// The MX formats' epilogue (multiplications instead of divisions) was measured the other way: 345 -> 384 us, 1x1 323 -> 404 us.
+constexpr int TC_THREADS_MX = 768;
+__host__ __device__ constexpr int tc_threads_of(int epi) { return epi == 5 ? TC_THREADS_MX : TC_THREADS; }
 constexpr int A_STAGE_BYTES = 128 * 128;
 constexpr int SFA_BYTES = 1024;   // up to 2 groups of 4 scale bytes per row
 constexpr int SFB_BYTES = 2048;   // up to 2 groups x 2 atoms of 128 rows
@@ -478,11 +484,13 @@ template <int MODE, int FMT>
 __device__ __forceinline__ void epilogue_mx_role(const ConvTcParams& p, unsigned* red, uint32_t tmem, uint64_t* tfull, uint64_t* tempty,
                                                  volatile int* abort_flag, int warp, int lane, unsigned total) {
     const int quad = warp & 3;
-    const int half = (warp - 4) >> 2;
+    const int half = warp < 12 ? (warp - 4) >> 2 : 2 + ((warp - 16) >> 2);   // column group 0..3 of this warp (four warps each, one per lane quadrant)
     const int r = 32 * quad + lane;
     const int tw_ = r & (p.TW - 1), tn = r >> p.lgTW;
     const int nblk = p.BN >> 5;                         // 32-channel blocks of a tile
-    const int bbeg = half == 0 ? 0 : (nblk + 1) >> 1, bend = half == 0 ? (nblk + 1) >> 1 : nblk;
+    constexpr int NG = FMT == 5 ? 4 : 2;                // column groups: 16 epilogue warps for the paper's format, else 8
+    const int per = (nblk + NG - 1) / NG;
+    const int bbeg = min(nblk, half * per), bend = min(nblk, bbeg + per);
     const int grp0 = quad & ~(p.TW - 1);                // first quadrant of the TW quadrants that hold this sample tile
     constexpr bool TS = FMT == 5;                       // the paper's own format (16 x 16 blocks; TW is 1 or 2)
     constexpr int bpe4 = (FMT == MQ_E2M1 || TS) ? 1 : 2;        // bytes per element x 2
@@ -664,7 +672,7 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
 // EPI: -1 = fp32 output (the three fp32 epilogue roles, chosen at run time: an instance per role was measured, no
 // change); 0..4 = quantizing epilogue emitting element format EPI
 template <int MODE, int KB, int KIND, int EPI = -1>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(tc_threads_of(EPI), 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_out,
                const ConvTcParams p) {
   constexpr int G = 128 / KB;          // chunks per stage
@@ -700,7 +708,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 3); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], 8); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], EPI == 5 ? 16 : 8); }
     *abort_flag = 0;
     mbar_fence_init();
     prefetch_tensormap(&map_a);
@@ -715,7 +723,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   pdl_wait();   // set-up above touched only shared memory, tensor memory and the kernel parameters
 
   // loader warps: (kind, parity of the stages it serves)
-  const int lkind = (warp == 0 || warp == 12) ? 0 : ((warp == 3 || warp == 13) ? 1 : (warp >= 14 ? 2 : -1));
+  const int lkind = (warp == 0 || warp == 12) ? 0 : ((warp == 3 || warp == 13) ? 1 : ((warp == 14 || warp == 15) ? 2 : -1));
   const int lhalf = (warp == 12 || warp == 13 || warp == 15) ? 1 : 0;
   if (lkind >= 0) {
     // ------------------------------------------------------------------ TMA loaders
@@ -891,7 +899,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
       }
     }
-  } else if (warp >= 4 && warp < 12) {
+  } else if ((warp >= 4 && warp < 12) || warp >= 16) {
     if (EPI >= 0) epilogue_mx_role<MODE, EPI < 0 ? 0 : EPI>(p, mx_red, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else if (p.pair) epilogue_pair_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else if (p.tma_store) epilogue_tma_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total);
@@ -1672,7 +1680,7 @@ bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const ui
 
 size_t conv_tc_smem_bytes(const ConvTcParams& p) {
   const size_t stage = A_STAGE_BYTES + (size_t)p.BN * 128 + (p.kind_fp4 == 2 ? SFA_BYTES_NV + SFB_BYTES_NV : SFA_BYTES + SFB_BYTES);
-  return 1024 + (size_t)p.stages * stage + (p.tma_store ? EPI_STAGING_BYTES : 0) + (3 * (size_t)p.stages + 4) * 8 + 64 + (p.mx_out ? 288 : 0);
+  return 1024 + (size_t)p.stages * stage + (p.tma_store ? EPI_STAGING_BYTES : 0) + (3 * (size_t)p.stages + 4) * 8 + 64 + (p.mx_out ? 544 : 0);
 }
 
 template <int MODE, int KB, int FP4, int EPI = -1>
@@ -1688,7 +1696,7 @@ cudaError_t launch_conv_tc_inst(const ConvTcParams& p, const CUtensorMap& map_a,
   const long long units = p.pair ? p.total_tiles / 2 : p.total_tiles;
   const unsigned grid = (unsigned)(units < sms ? units : sms);
   count_launches(1);
-  return launch_pdl(conv_tc_kernel<MODE, KB, FP4, EPI>, dim3(grid), dim3(TC_THREADS), smem, s, map_a, map_b, map_out, p);
+  return launch_pdl(conv_tc_kernel<MODE, KB, FP4, EPI>, dim3(grid), dim3(tc_threads_of(EPI)), smem, s, map_a, map_b, map_out, p);
 }
 
 size_t conv_tc_sfa_bytes(const ConvTcParams& p) {
