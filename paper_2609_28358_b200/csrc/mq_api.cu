@@ -236,14 +236,19 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   // staging only in the whole-tile kernel, whose pipeline is short; the per-tap kernel keeps its stages
   // (NCHW: rows of TW floats, at least 16 bytes; [H][W][N][C]: rows of 32 channels whatever the tile's width, whole 32-channel
   // groups per column half)
-  const bool tma_store_ok = (op == MQ_OP_FWD || (g.sh == 1 && g.sw == 1)) && p.TW <= 32 &&
+  // Strided input gradient, channel-fastest output: the staged epilogue writes a parity class through a tensor map that steps sw
+  // pixels along W.  Not for NCHW: there W is the innermost axis and a class's first column (x = 1 for the odd one) would be
+  // a TMA coordinate that is not on a 16-byte boundary, which the hardware refuses; NCHW keeps the paired direct stores.
+  const bool strided_out = op == MQ_OP_BWD_DATA && (g.sh != 1 || g.sw != 1);
+  const bool s2_tma_ok = strided_out && layout == MQ_HWNC && g.sw <= 8 && !env_int("MQ_TC_NO_S2_TMA", 0);
+  const bool tma_store_ok = (!strided_out || s2_tma_ok) && p.TW <= 32 &&
                             (layout == MQ_NCHW ? (p.TW >= 4 && p.Wd % 4 == 0) : (p.Cd % 4 == 0 && p.BN % 64 == 0));
   // ... and for 1x1 layers, whose main loop is a handful of stages: the tile's time is its store (measured 4-12 % faster, 28x28 and
   // 56x56 images, 256 and 512 channels)
   // ... and for the channel-fastest output order, where a direct store is one 16-byte request per row and instruction - the request
   // count, not the bytes, bounds the store path (measured, N = 256, 512 channels: 1x1 56x56 841 -> 443 us, 3x3 28x28 447 -> 396 us,
   // the latter 2.39 PFLOP/s against 2.15 for the NCHW order)
-  p.tma_store = !mx && tma_store_ok && (env_int("MQ_TC_TMA_STORE", 0) || ((taps == 1 || layout == MQ_HWNC) && !env_int("MQ_TC_NO_TMA_STORE", 0))) ? 1 : 0;
+  p.tma_store = !mx && tma_store_ok && (env_int("MQ_TC_TMA_STORE", 0) || ((taps == 1 || layout == MQ_HWNC || strided_out) && !env_int("MQ_TC_NO_TMA_STORE", 0))) ? 1 : 0;
   const size_t stage_bytes = 128 * 128 + (size_t)p.BN * 128 + (ts16 ? 6144 : 3072);
   const int sf_cols = ts16 ? 48 : 24;
   int stages = (int)((227 * 1024 - 2048 - (p.tma_store ? 65536 : 0)) / stage_bytes);
@@ -256,7 +261,7 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   p.n_acc = (2 * p.BN + sf_cols * stages <= 512) ? 2 : 1;
   if (p.n_acc * p.BN + sf_cols * stages > 512) return false;
   p.mma_cp = env_int("MQ_TC_NO_MMA_CP", 0) ? 0 : 1;   // E2M1 too: the bubble behind a copier warp costs more than the lane's extra issues
-  p.pair = !mx && op == MQ_OP_BWD_DATA && g.sw == 2 && layout == MQ_NCHW && p.Wd % 2 == 0 && p.n_acc == 2 && p.total_tiles % 2 == 0 &&
+  p.pair = !mx && !p.tma_store && op == MQ_OP_BWD_DATA && g.sw == 2 && layout == MQ_NCHW && p.Wd % 2 == 0 && p.n_acc == 2 && p.total_tiles % 2 == 0 &&
            !env_int("MQ_TC_NO_PAIR", 0);
   const int nkh = op == MQ_OP_FWD ? g.Kh : (g.Kh + g.sh - 1) / g.sh, nkw = op == MQ_OP_FWD ? g.Kw : (g.Kw + g.sw - 1) / g.sw;
   p.max_stages = (nkh * nkw * p.cpt + p.G - 1) / p.G;
@@ -397,8 +402,11 @@ mq_status run_conv_tc(int op, const Geom& g, ConvTcPlan& pl, const mq_qtensor* q
         // bytes with the 128-byte swizzle
         const uint64_t dims[4] = {(uint64_t)p.Cd, (uint64_t)p.Wd, (uint64_t)g.N, (uint64_t)p.Hd};
         const uint64_t strides[3] = {(uint64_t)g.N * p.Cd * 4, (uint64_t)p.Cd * 4, (uint64_t)p.Wd * g.N * p.Cd * 4};
-        const uint32_t box[4] = {32u, (uint32_t)p.TW, (uint32_t)(32 / p.TW), 1u};
-        if (!encode_tensor_map_u8(&map_out, out, 4, dims, strides, box, nullptr, 128, true)) return MQ_ERR_CUDA;
+        // strided input gradient: a parity class's columns are sw pixels apart - the box steps sw along W (TW of its pixels land)
+        const uint32_t esw = op == MQ_OP_BWD_DATA ? (uint32_t)g.sw : 1u;
+        const uint32_t box[4] = {32u, (uint32_t)p.TW * esw, (uint32_t)(32 / p.TW), 1u};
+        const uint32_t es[4] = {1u, esw, 1u, 1u};
+        if (!encode_tensor_map_u8(&map_out, out, 4, dims, strides, box, es, 128, true)) return MQ_ERR_CUDA;
       }
     }
   }

@@ -612,7 +612,9 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
       ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
       if (!ok) { *abort_flag = 1; break; }
       tc_fence_after_sync();
-      const int yo = MODE == MQ_OP_FWD ? tile.h : (int)fdiv((unsigned)tile.cls, p.sw, p.m_sw) + p.sh * tile.h;
+      const int cls_h = MODE == MQ_OP_FWD ? 0 : (int)fdiv((unsigned)tile.cls, p.sw, p.m_sw);
+      const int yo = MODE == MQ_OP_FWD ? tile.h : cls_h + p.sh * tile.h;
+      const int xo0 = MODE == MQ_OP_FWD ? tile.w0 : (tile.cls - cls_h * p.sw) + p.sw * tile.w0;   // first output column (a parity class's columns are sw apart)
       const uint32_t taddr = tmem + acc * p.BN + ((uint32_t)(32 * quad) << 16);
       if (cbeg >= cend) {      // a tile of 16 channels leaves the second half without columns
         tc_fence_before_sync();
@@ -657,10 +659,10 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
-          if (!hwnc) tma_store_4d(map_out, buf, tile.w0, tile.n0 + n_off, tile.c0 + c0, yo);
+          if (!hwnc) tma_store_4d(map_out, buf, xo0, tile.n0 + n_off, tile.c0 + c0, yo);
           else {
-            tma_store_4d(map_out, buf, tile.c0 + c0, tile.w0, tile.n0 + n_off, yo);
-            if (nch > 2) tma_store_4d(map_out, buf + 1024, tile.c0 + c0 + 32, tile.w0, tile.n0 + n_off, yo);
+            tma_store_4d(map_out, buf, tile.c0 + c0, xo0, tile.n0 + n_off, yo);
+            if (nch > 2) tma_store_4d(map_out, buf + 1024, tile.c0 + c0 + 32, xo0, tile.n0 + n_off, yo);
           }
           bulk_commit_group();
         }
