@@ -31,7 +31,8 @@ constexpr int TC_THREADS = 512;   // 16 warps: MMA, scale copier, scale expander
 // The quantizing epilogue of the paper's own format (emitted format 5) runs with 16 epilogue warps (8 more, warps 16-23): a block
 // of it is a chain of latencies (tensor-memory load, warp reductions, IEEE divisions, conversions, stores) that two warps
 // per scheduler do not hide; four do better, at 80 registers per thread (measured, 512 channels 28x28 3x3: 320 -> 278 us).
-// The MX formats' epilogue (multiplications instead of divisions) was measured the other way: 345 -> 384 us, 1x1 323 -> 404 us.
+// The MX formats' epilogue (multiplications instead of divisions) was measured the other way: 345 -> 384 us, 1x1 323 -> 404 us;
+// the fp32 direct-store epilogue does not change with 16 warps (445 -> 456 us: its stores are the bound).
 constexpr int TC_THREADS_MX = 768;
 __host__ __device__ constexpr int tc_threads_of(int epi) { return epi == 5 ? TC_THREADS_MX : TC_THREADS; }
 constexpr int A_STAGE_BYTES = 128 * 128;
