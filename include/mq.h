@@ -268,6 +268,9 @@ mq_status mq_conv_bwd_weight(const mq_conv_desc* desc, const mq_qtensor* xq, con
  * created on first use, no device memory involved) tied to `stream` by events, so uploads and downloads
  * overlap the kernels; `stream` waits for the last download, so the host results are valid after `stream`
  * is synchronised and successive calls on one stream stay ordered.
+ * The step runs slab by slab along the batch (slabs of whole 32-sample tiles, at most 8): every call above needs only the
+ * slab's own samples (and W), so slab k + 1 uploads and slab k's Y and G_X download while the kernels run.  Y and G_X
+ * are exactly the device calls' results; G_W is the sum of the slabs' weight gradients, added in slab order.
  * arena: device memory, arena_bytes >= mq_conv_layer_host_arena_size(); contents are scratch. */
 mq_status mq_conv_layer_host_arena_size(const mq_conv_desc* desc, int fmt_x, int fmt_w, int fmt_dy, size_t* bytes);
 mq_status mq_conv_layer_host(const mq_conv_desc* desc, int fmt_x, int fmt_w, int fmt_dy, const float* x_host, const float* w_host,

@@ -989,10 +989,15 @@ mq_status mq_conv_bwd_data_static(const mq_conv_desc* desc, const mq_qtensor* wq
 }
 
 namespace {
+// The step runs slab by slab along the batch (slabs of whole 32-sample tiles, at most 8 of them): the quantized tensors, the
+// im2col and the GEMMs of a slab need that slab's samples only (W in full), so the upload of slab k + 1 and the download of
+// slab k's Y and G_X overlap the computation, and both copy engines stay busy for the whole step.  G_W is the sum of the
+// slabs' weight gradients, added in slab order.
 struct LayerArena {
-  size_t off_x, off_w, off_g, off_y, off_dx, off_dw, off_ws, off_ic, off_is, total;
+  size_t off_x, off_w, off_g, off_y, off_dx, off_dw, off_dwp, off_ws, off_ic, off_is, total;
   size_t off_qc[3], off_qs[3];
   size_t nx, nw, ng, qc[3], qs[3], ic, is, ws;
+  int slab_n, slabs;        // samples per slab (the last may hold fewer), number of slabs
 };
 size_t up256(size_t v) { return (v + 255) / 256 * 256; }
 LayerArena layer_arena(const mq_conv_desc* desc, const int fmts[3]) {
@@ -1005,16 +1010,29 @@ LayerArena layer_arena(const mq_conv_desc* desc, const int fmts[3]) {
   auto take = [&](size_t n) { size_t r = o; o += up256(n); return r; };
   L.off_x = take(L.nx); L.off_w = take(L.nw); L.off_g = take(L.ng);
   L.off_y = take(L.ng); L.off_dx = take(L.nx); L.off_dw = take(L.nw);
-  for (int r = 0; r < 3; ++r) {
-    sizes_of(g, r, fmts[r], MQ_BLOCK_TILE32, &L.qc[r], &L.qs[r]);
-    L.off_qc[r] = take(L.qc[r]); L.off_qs[r] = take(L.qs[r]);
-  }
-  mq_im2col_sizes(desc, fmts[0], MQ_BLOCK_TILE32, &L.ic, &L.is);
+  int max_slabs = env_int("MQ_HOST_SLABS", 8);
+  max_slabs = max_slabs < 1 ? 1 : (max_slabs > 8 ? 8 : max_slabs);
+  const int tiles_per_slab = (g.Nt + max_slabs - 1) / max_slabs;
+  L.slab_n = 32 * tiles_per_slab;
+  L.slabs = (g.N + L.slab_n - 1) / L.slab_n;
+  L.off_dwp = L.slabs > 1 ? take((size_t)L.slabs * up256(L.nw)) : 0;
+  mq_conv_desc ds = *desc;
+  ds.N = L.slabs > 1 ? L.slab_n : g.N;     // the largest slab sizes the per-slab buffers
+  const Geom gs = make_geom(ds);
+  sizes_of(gs, 0, fmts[0], MQ_BLOCK_TILE32, &L.qc[0], &L.qs[0]);
+  sizes_of(g, 1, fmts[1], MQ_BLOCK_TILE32, &L.qc[1], &L.qs[1]);
+  sizes_of(gs, 2, fmts[2], MQ_BLOCK_TILE32, &L.qc[2], &L.qs[2]);
+  for (int r = 0; r < 3; ++r) { L.off_qc[r] = take(L.qc[r]); L.off_qs[r] = take(L.qs[r]); }
+  mq_im2col_sizes(&ds, fmts[0], MQ_BLOCK_TILE32, &L.ic, &L.is);
   L.off_ic = take(L.ic); L.off_is = take(L.is);
   L.ws = 0;
   const int ops[3] = {MQ_OP_FWD, MQ_OP_BWD_DATA, MQ_OP_BWD_WEIGHT};
   const int fa[3] = {fmts[0], fmts[1], fmts[0]}, fb[3] = {fmts[1], fmts[2], fmts[2]};
-  for (int i = 0; i < 3; ++i) { size_t b = 0; mq_workspace_size(desc, ops[i], fa[i], fb[i], MQ_BLOCK_TILE32, &b); if (b > L.ws) L.ws = b; }
+  for (int pass = 0; pass < 2; ++pass) {     // the full slab, and the ragged last one (its plans may need more scratch)
+    mq_conv_desc dq = ds;
+    if (pass == 1) { dq.N = g.N - (L.slabs - 1) * L.slab_n; if (L.slabs == 1 || dq.N == ds.N) break; }
+    for (int i = 0; i < 3; ++i) { size_t b = 0; mq_workspace_size(&dq, ops[i], fa[i], fb[i], MQ_BLOCK_TILE32, &b); if (b > L.ws) L.ws = b; }
+  }
   L.off_ws = take(L.ws);
   L.total = o;
   return L;
@@ -1022,7 +1040,24 @@ LayerArena layer_arena(const mq_conv_desc* desc, const int fmts[3]) {
 }  // namespace
 
 // Side streams and events of mq_conv_layer_host, created once per device (no device memory is allocated).
-struct HostPipe { cudaStream_t h2d, d2h; cudaEvent_t ev[8]; bool ready; };
+// G_W = sum over the slabs of their weight gradients, in slab order (float4 body, scalar tail)
+__global__ void __launch_bounds__(256) sum_slabs_kernel(const float4* __restrict__ part4, float4* __restrict__ out4, long long n4, long long stride4, int slabs,
+                                                        const float* __restrict__ part, float* __restrict__ out, long long n) {
+  const long long t0 = (long long)blockIdx.x * blockDim.x + threadIdx.x, step = (long long)gridDim.x * blockDim.x;
+  for (long long i = t0; i < n4; i += step) {
+    float4 a = __ldg(part4 + i);
+    for (int k = 1; k < slabs; ++k) { const float4 b = __ldg(part4 + (long long)k * stride4 + i); a.x += b.x; a.y += b.y; a.z += b.z; a.w += b.w; }
+    out4[i] = a;
+  }
+  for (long long i = 4 * n4 + t0; i < n; i += step) {
+    float a = __ldg(part + i);
+    for (int k = 1; k < slabs; ++k) a += __ldg(part + (long long)k * stride4 * 4 + i);
+    out[i] = a;
+  }
+}
+
+constexpr int HOST_EVENTS = 48;   // start, W, final, and four per slab (at most 8 slabs)
+struct HostPipe { cudaStream_t h2d, d2h; cudaEvent_t ev[HOST_EVENTS]; bool ready; };
 static HostPipe* host_pipe() {
   static HostPipe pipes[32];
   int dev = 0;
@@ -1031,7 +1066,7 @@ static HostPipe* host_pipe() {
   if (!hp->ready) {
     if (cudaStreamCreateWithFlags(&hp->h2d, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
     if (cudaStreamCreateWithFlags(&hp->d2h, cudaStreamNonBlocking) != cudaSuccess) return nullptr;
-    for (int i = 0; i < 8; ++i)
+    for (int i = 0; i < HOST_EVENTS; ++i)
       if (cudaEventCreateWithFlags(&hp->ev[i], cudaEventDisableTiming) != cudaSuccess) return nullptr;
     hp->ready = true;
   }
@@ -1061,40 +1096,68 @@ mq_status mq_conv_layer_host(const mq_conv_desc* desc, int fmt_x, int fmt_w, int
   uint8_t* base = static_cast<uint8_t*>(arena);
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   // Copies run on two side streams of their own (one per direction: the copy engines are full duplex) and are tied to
-  // the caller's stream by events, so the upload of G_Y overlaps the forward half of the step and the download of Y
-  // overlaps the backward half.  The caller's stream waits for the last download: synchronising it is enough.
+  // the caller's stream by events.  Slab by slab: upload X_k and G_Y_k; quantize, im2col, forward -> download Y_k;
+  // input gradient -> download G_X_k; weight gradient of the slab into its own buffer.  The caller's stream waits for
+  // the last download: synchronising it is enough.
   HostPipe* hp = host_pipe();
   if (!hp) return MQ_ERR_CUDA;
   auto ok = [](cudaError_t e) { return e == cudaSuccess; };
-  if (!ok(cudaEventRecord(hp->ev[0], s)) || !ok(cudaStreamWaitEvent(hp->h2d, hp->ev[0], 0)) || !ok(cudaStreamWaitEvent(hp->d2h, hp->ev[0], 0)))
-    return MQ_ERR_CUDA;
-  if (!ok(cudaMemcpyAsync(base + L.off_x, x_host, L.nx, cudaMemcpyHostToDevice, hp->h2d)) || !ok(cudaEventRecord(hp->ev[1], hp->h2d))) return MQ_ERR_CUDA;
-  if (!ok(cudaMemcpyAsync(base + L.off_w, w_host, L.nw, cudaMemcpyHostToDevice, hp->h2d)) || !ok(cudaEventRecord(hp->ev[2], hp->h2d))) return MQ_ERR_CUDA;
-  if (!ok(cudaMemcpyAsync(base + L.off_g, dy_host, L.ng, cudaMemcpyHostToDevice, hp->h2d)) || !ok(cudaEventRecord(hp->ev[3], hp->h2d))) return MQ_ERR_CUDA;
+  const Geom g = make_geom(*desc);
+  const int S = L.slabs;
+  cudaEvent_t* ev = hp->ev;     // 0 start, 1 W uploaded, 2 G_W ready, 3 last download; 4 + 4k .. : X_k, G_Y_k uploaded, Y_k, G_X_k ready
+  if (!ok(cudaEventRecord(ev[0], s)) || !ok(cudaStreamWaitEvent(hp->h2d, ev[0], 0)) || !ok(cudaStreamWaitEvent(hp->d2h, ev[0], 0))) return MQ_ERR_CUDA;
+  if (!ok(cudaMemcpyAsync(base + L.off_w, w_host, L.nw, cudaMemcpyHostToDevice, hp->h2d)) || !ok(cudaEventRecord(ev[1], hp->h2d))) return MQ_ERR_CUDA;
+  const size_t x_per_n = (size_t)g.Cin * g.H * g.W * 4, g_per_n = (size_t)g.Cout * g.Ho * g.Wo * 4;
+  for (int k = 0; k < S; ++k) {
+    const size_t n0 = (size_t)k * L.slab_n, nk = (size_t)(k == S - 1 ? g.N - (int)n0 : L.slab_n);
+    if (!ok(cudaMemcpyAsync(base + L.off_x + n0 * x_per_n, reinterpret_cast<const uint8_t*>(x_host) + n0 * x_per_n, nk * x_per_n, cudaMemcpyHostToDevice, hp->h2d)) ||
+        !ok(cudaEventRecord(ev[4 + 4 * k], hp->h2d))) return MQ_ERR_CUDA;
+    if (!ok(cudaMemcpyAsync(base + L.off_g + n0 * g_per_n, reinterpret_cast<const uint8_t*>(dy_host) + n0 * g_per_n, nk * g_per_n, cudaMemcpyHostToDevice, hp->h2d)) ||
+        !ok(cudaEventRecord(ev[5 + 4 * k], hp->h2d))) return MQ_ERR_CUDA;
+  }
   mq_qtensor q[3];
-  const size_t src_off[3] = {L.off_x, L.off_w, L.off_g};
   for (int r = 0; r < 3; ++r) {
     q[r].codes = base + L.off_qc[r]; q[r].scales = base + L.off_qs[r];
     q[r].codes_bytes = L.qc[r]; q[r].scales_bytes = L.qs[r]; q[r].fmt = fmts[r]; q[r].role = r; q[r].block = MQ_BLOCK_TILE32; q[r].tensor_scale = nullptr;
   }
   void* ws = L.ws ? base + L.off_ws : nullptr;
-  if (!ok(cudaStreamWaitEvent(s, hp->ev[1], 0))) return MQ_ERR_CUDA;
-  if ((st = mq_quantize(desc, base + src_off[0], MQ_F32, MQ_NCHW, &q[0], stream)) != MQ_OK) return st;
-  if (!ok(cudaStreamWaitEvent(s, hp->ev[2], 0))) return MQ_ERR_CUDA;
-  if ((st = mq_quantize(desc, base + src_off[1], MQ_F32, MQ_NCHW, &q[1], stream)) != MQ_OK) return st;
-  if ((st = mq_cbf_im2col(desc, &q[0], base + L.off_ic, base + L.off_is, stream)) != MQ_OK) return st;
-  if ((st = mq_conv_fwd(desc, &q[0], &q[1], base + L.off_y, MQ_F32, MQ_NCHW, ws, L.ws, stream)) != MQ_OK) return st;
-  if (!ok(cudaEventRecord(hp->ev[4], s)) || !ok(cudaStreamWaitEvent(hp->d2h, hp->ev[4], 0))) return MQ_ERR_CUDA;
-  if (!ok(cudaMemcpyAsync(y_host, base + L.off_y, L.ng, cudaMemcpyDeviceToHost, hp->d2h))) return MQ_ERR_CUDA;
-  if (!ok(cudaStreamWaitEvent(s, hp->ev[3], 0))) return MQ_ERR_CUDA;
-  if ((st = mq_quantize(desc, base + src_off[2], MQ_F32, MQ_NCHW, &q[2], stream)) != MQ_OK) return st;
-  if ((st = mq_conv_bwd_data(desc, &q[1], &q[2], base + L.off_dx, MQ_F32, MQ_NCHW, ws, L.ws, stream)) != MQ_OK) return st;
-  if (!ok(cudaEventRecord(hp->ev[5], s)) || !ok(cudaStreamWaitEvent(hp->d2h, hp->ev[5], 0))) return MQ_ERR_CUDA;
-  if (!ok(cudaMemcpyAsync(dx_host, base + L.off_dx, L.nx, cudaMemcpyDeviceToHost, hp->d2h))) return MQ_ERR_CUDA;
-  if ((st = mq_conv_bwd_weight(desc, &q[0], &q[2], base + L.off_dw, MQ_F32, MQ_NCHW, ws, L.ws, stream)) != MQ_OK) return st;
-  if (!ok(cudaEventRecord(hp->ev[6], s)) || !ok(cudaStreamWaitEvent(hp->d2h, hp->ev[6], 0))) return MQ_ERR_CUDA;
+  if (!ok(cudaStreamWaitEvent(s, ev[1], 0))) return MQ_ERR_CUDA;
+  if ((st = mq_quantize(desc, base + L.off_w, MQ_F32, MQ_NCHW, &q[1], stream)) != MQ_OK) return st;
+  for (int k = 0; k < S; ++k) {
+    const size_t n0 = (size_t)k * L.slab_n, nk = (size_t)(k == S - 1 ? g.N - (int)n0 : L.slab_n);
+    mq_conv_desc dk = *desc;
+    dk.N = (int)nk;
+    uint8_t* xk = base + L.off_x + n0 * x_per_n;
+    uint8_t* gk = base + L.off_g + n0 * g_per_n;
+    uint8_t* yk = base + L.off_y + n0 * g_per_n;
+    uint8_t* dxk = base + L.off_dx + n0 * x_per_n;
+    void* dwk = S > 1 ? static_cast<void*>(base + L.off_dwp + (size_t)k * ((L.nw + 255) / 256 * 256)) : static_cast<void*>(base + L.off_dw);
+    if (!ok(cudaStreamWaitEvent(s, ev[4 + 4 * k], 0))) return MQ_ERR_CUDA;
+    if ((st = mq_quantize(&dk, xk, MQ_F32, MQ_NCHW, &q[0], stream)) != MQ_OK) return st;
+    if ((st = mq_cbf_im2col(&dk, &q[0], base + L.off_ic, base + L.off_is, stream)) != MQ_OK) return st;
+    if ((st = mq_conv_fwd(&dk, &q[0], &q[1], yk, MQ_F32, MQ_NCHW, ws, L.ws, stream)) != MQ_OK) return st;
+    if (!ok(cudaEventRecord(ev[6 + 4 * k], s)) || !ok(cudaStreamWaitEvent(hp->d2h, ev[6 + 4 * k], 0))) return MQ_ERR_CUDA;
+    if (!ok(cudaMemcpyAsync(reinterpret_cast<uint8_t*>(y_host) + n0 * g_per_n, yk, nk * g_per_n, cudaMemcpyDeviceToHost, hp->d2h))) return MQ_ERR_CUDA;
+    if (!ok(cudaStreamWaitEvent(s, ev[5 + 4 * k], 0))) return MQ_ERR_CUDA;
+    if ((st = mq_quantize(&dk, gk, MQ_F32, MQ_NCHW, &q[2], stream)) != MQ_OK) return st;
+    if ((st = mq_conv_bwd_data(&dk, &q[1], &q[2], dxk, MQ_F32, MQ_NCHW, ws, L.ws, stream)) != MQ_OK) return st;
+    if (!ok(cudaEventRecord(ev[7 + 4 * k], s)) || !ok(cudaStreamWaitEvent(hp->d2h, ev[7 + 4 * k], 0))) return MQ_ERR_CUDA;
+    if (!ok(cudaMemcpyAsync(reinterpret_cast<uint8_t*>(dx_host) + n0 * x_per_n, dxk, nk * x_per_n, cudaMemcpyDeviceToHost, hp->d2h))) return MQ_ERR_CUDA;
+    if ((st = mq_conv_bwd_weight(&dk, &q[0], &q[2], dwk, MQ_F32, MQ_NCHW, ws, L.ws, stream)) != MQ_OK) return st;
+  }
+  if (S > 1) {
+    const long long n4 = (long long)(L.nw / 16), stride4 = (long long)((L.nw + 255) / 256 * 256 / 16);
+    unsigned blocks = (unsigned)((n4 + 255) / 256);
+    if (blocks > (unsigned)sm_count() * 8) blocks = (unsigned)sm_count() * 8;
+    if (blocks < 1) blocks = 1;
+    sum_slabs_kernel<<<blocks, 256, 0, s>>>(reinterpret_cast<const float4*>(base + L.off_dwp), reinterpret_cast<float4*>(base + L.off_dw), n4, stride4, S,
+                                          reinterpret_cast<const float*>(base + L.off_dwp), reinterpret_cast<float*>(base + L.off_dw), (long long)(L.nw / 4));
+    count_launches(1);
+    if (cudaGetLastError() != cudaSuccess) return MQ_ERR_CUDA;
+  }
+  if (!ok(cudaEventRecord(ev[2], s)) || !ok(cudaStreamWaitEvent(hp->d2h, ev[2], 0))) return MQ_ERR_CUDA;
   if (!ok(cudaMemcpyAsync(dw_host, base + L.off_dw, L.nw, cudaMemcpyDeviceToHost, hp->d2h))) return MQ_ERR_CUDA;
-  if (!ok(cudaEventRecord(hp->ev[7], hp->d2h)) || !ok(cudaStreamWaitEvent(s, hp->ev[7], 0))) return MQ_ERR_CUDA;
+  if (!ok(cudaEventRecord(ev[3], hp->d2h)) || !ok(cudaStreamWaitEvent(s, ev[3], 0))) return MQ_ERR_CUDA;
   return MQ_OK;
 }
 
