@@ -252,6 +252,26 @@ def fused_epilogue_times(wl, flush, K, kern, pk):
         res[name] = {"ms": ms, "tflops": tf, "frac": tf / peak, "frac_of_published": tf / PUBLISHED["tensor_tflops"][bits],
                      "fp32_output_call_ms": kern[plain]["ms"], "activation": "relu" if plain == "conv_fwd" else "none",
                      "emits": FMT_NAME[f[0] if plain == "conv_fwd" else f[2]] + (" (16x16 blocks, E4M3 scales, supplied maximum)" if wl.block == mq.TS16 else "")}
+    if wl.block == mq.TS16:
+        # the quantizer itself with the maximum supplied (Sec. VII-B): one pass that also records the tensor's own maximum
+        src = wl.src[0]
+        sl = mq.HWNC if tuple(src.shape) != (d.N, d.C_in, d.H, d.W) else mq.NCHW
+        am_x = src.abs().max().reshape(1).float()
+        fn = lambda: mq.quantize_ts(d, mq.ROLE_X, src, out=q[0], src_layout=sl, amax_in=am_x)
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(K)]
+        for s, e in ev:
+            flush.zero_()
+            s.record()
+            fn()
+            e.record()
+        torch.cuda.synchronize()
+        ms = sum(s.elapsed_time(e) for s, e in ev) / K
+        nbytes = wl.algorithmic_bytes()["quantize_x"]
+        res["quantize_x_supplied_maximum"] = {"ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9, "frac": nbytes / (ms * 1e-3) / 1e9 / pk["hbm_gbs"],
+                                              "own_maximum_call_ms": kern["quantize_x"]["ms"]}
     res["device_status"] = mq.last_device_status()
     return res
 

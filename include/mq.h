@@ -151,8 +151,10 @@ mq_status mq_quantize_sr(const mq_conv_desc* desc, const void* src, int src_dtyp
  * where Eq. 4 takes the tensor's maximum from.  amax_in = NULL: from this tensor (two passes over `src`: a reduction,
  * then the quantizer); mq_quantize on such a dst does exactly this.  amax_in = a device fp32: from that value - e.g.
  * the max|X| an earlier step left in its tensor_scale[1] (statistics of previous batches, Sec. VII-B), so that the
- * quantizer needs no result of a reduction over this tensor; elements beyond the estimate saturate.  Either way
- * dst->tensor_scale[0] receives T_scale and dst->tensor_scale[1] this tensor's own max|X|.
+ * quantizer needs no result of a reduction over this tensor (large NCHW / OIHW sources are then read ONCE, the quantizer
+ * collecting this tensor's maximum as it goes); elements beyond the estimate saturate.  amax_in must not point into
+ * dst->tensor_scale (the call rewrites both words).  Either way dst->tensor_scale[0] receives T_scale and
+ * dst->tensor_scale[1] this tensor's own max|X|.
  * seed_or_null: NULL = round to nearest; else a host pointer to the 64-bit seed of the stochastic Round(.) of Eq. 6 (the
  * gradient's rounding; draws as in mq_quantize_sr). */
 mq_status mq_quantize_ts(const mq_conv_desc* desc, const void* src, int src_dtype, int src_layout, mq_qtensor* dst, const float* amax_in,

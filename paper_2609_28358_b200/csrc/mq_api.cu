@@ -790,6 +790,8 @@ mq_status mq_quantize_ts(const mq_conv_desc* desc, const void* src, int src_dtyp
                          const unsigned long long* seed_or_null, void* stream) {
   if (dst && dst->block != MQ_BLOCK_TS16) return MQ_ERR_INVALID_ARG;
   if (amax_in && (reinterpret_cast<uintptr_t>(amax_in) & 3u)) return MQ_ERR_ALIGNMENT;
+  if (amax_in && dst && dst->tensor_scale && amax_in >= static_cast<const float*>(dst->tensor_scale) &&
+      amax_in < static_cast<const float*>(dst->tensor_scale) + 2) return MQ_ERR_INVALID_ARG;   // the call rewrites both words
   return quantize_impl(desc, src, src_dtype, src_layout, dst, seed_or_null ? 1 : 0, seed_or_null ? *seed_or_null : 0ull, stream, 0, 0, amax_in);
 }
 

@@ -84,6 +84,7 @@ struct QuantArgs {
   // tensor's statistics buffer (T_scale is written to [0])
   const float* ts_amax;
   float* ts_stats;
+  int ts_track_max;   // 1: the kernel also collects max|X| into ts_stats[1] (maximum supplied from outside: the tensor is read once)
 };
 // invertible 32-bit mixer (xor-shift, odd multiply, twice, xor-shift) behind the per-element draws
 __host__ __device__ __forceinline__ unsigned sr_mix32(unsigned x) {
@@ -96,7 +97,7 @@ cudaError_t launch_quantize(const QuantArgs& a, cudaStream_t s);
 cudaError_t launch_quantize_ts(const QuantArgs& a, const float* amax_in, float* stats, cudaStream_t s);
 // Second pass of that quantizer on the whole-line TMA kernel (NCHW / OIHW source with 16-byte rows): true if the tensor qualifies
 bool quantize_ts_tma_eligible(const QuantArgs& a);
-cudaError_t launch_quantize_ts_tma(const QuantArgs& a, const float* amax_src, float* stats, cudaStream_t s);
+cudaError_t launch_quantize_ts_tma(const QuantArgs& a, const float* amax_src, float* stats, cudaStream_t s, bool track_max = false);
 
 struct Im2colArgs {
   const uint8_t* codes;

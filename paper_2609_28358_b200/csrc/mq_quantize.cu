@@ -452,6 +452,7 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_con
     unsigned phase = 0;
     bool dead = false;
     float tscale = 0.f, t6 = 0.f;
+    unsigned own_max = 0;     // TS: bit pattern of the largest block maximum this thread has seen
     if (TS) {
       tscale = __fdiv_rn(*a.ts_amax, __fmul_rn(448.0f, 6.0f));                                  // Eq. 4
       t6 = __fmul_rn(tscale, 6.0f);
@@ -500,6 +501,7 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_con
 #pragma unroll
           for (int k = 0; k < 8; ++k) mx = max(mx, xch[(16 * hf + (warp & 1) + 2 * k) * 32 + lane]);
           const float bmax = __uint_as_float(mx);
+          own_max = max(own_max, mx);
           unsigned sc = 0;
           if (bmax > 0.f && tscale > 0.f) sc = (unsigned)__nv_cvt_float_to_fp8(__fdiv_rn(bmax, t6), __NV_SATFINITE, __NV_E4M3) & 0x7Fu;   // Eq. 5
           const __half_raw hr = __nv_cvt_fp8_to_halfraw((__nv_fp8_storage_t)sc, __NV_E4M3);
@@ -567,6 +569,10 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_con
       }
     }
     if (t == 0) tc::bulk_wait_group_all();
+    if (TS && a.ts_track_max) {   // the tensor's own maximum for the next step (Sec. VII-B): one atomic per warp
+      const unsigned wmax = __reduce_max_sync(0xffffffffu, own_max);
+      if (lane == 0 && wmax != 0) atomicMax(reinterpret_cast<unsigned*>(a.ts_stats + 1), wmax);
+    }
   }
   __syncthreads();
 }
@@ -760,9 +766,9 @@ bool quantize_ts_tma_eligible(const QuantArgs& a) {
   return vec && a.src_stride_r == 0 && a.fmt == MQ_E2M1 && (tv >= 0 ? tv != 0 : elems >= (1ll << 22));
 }
 
-cudaError_t launch_quantize_ts_tma(const QuantArgs& a0, const float* amax_src, float* stats, cudaStream_t s) {
+cudaError_t launch_quantize_ts_tma(const QuantArgs& a0, const float* amax_src, float* stats, cudaStream_t s, bool track_max) {
   QuantArgs a = a0;
-  a.ts_amax = amax_src; a.ts_stats = stats;
+  a.ts_amax = amax_src; a.ts_stats = stats; a.ts_track_max = track_max ? 1 : 0;
   CUtensorMap map_in, map_out;
   {
     const uint64_t dims[3] = {(uint64_t)a.P, (uint64_t)a.C, (uint64_t)a.R};

@@ -4,8 +4,9 @@
 //
 // Two passes when the tensor's own maximum is wanted (Eq. 4 needs max|X| before any element can be scaled):
 // tensor_amax_kernel reduces max|X| into the tensor's statistics buffer, quantize_ts_kernel then reads it.  With the
-// maximum supplied from outside (statistics of earlier batches, Sec. VII-B) the first pass only records this tensor's
-// maximum for the next step and the quantizer does not wait for it.
+// maximum supplied from outside (statistics of earlier batches, Sec. VII-B) nothing has to wait for this tensor's maximum:
+// large NCHW / OIHW tensors then take ONE pass, the whole-line quantizer collecting max|X| for the next step from the block
+// maxima it forms anyway; the others keep the separate reduction, which the quantizer does not wait for.
 //
 // Every operation of Eq. 4-6 is one IEEE single-precision operation, in the order written (division = __fdiv_rn,
 // products = __fmul_rn): the roundings decide integer codes, so nothing here may be contracted or approximated.
@@ -134,8 +135,14 @@ cudaError_t launch_quantize_ts(const QuantArgs& a, const float* amax_in, float* 
   long long blocks = (n / 4 + 255) / 256;
   if (blocks > (long long)sm_count() * 8) blocks = (long long)sm_count() * 8;
   if (blocks < 1) blocks = 1;
-  // the source of either layout is a dense array of n floats
   if (a.act && a.src_stride_r == 0) return cudaErrorInvalidValue;   // the activation rides on the channel-fastest source only
+  // maximum supplied from outside and the whole-line kernel applies: ONE pass - the quantizer collects this tensor's own
+  // maximum for the next step while it works (MQ_QUANT_TS_TWO_PASS=1 keeps the separate reduction)
+  if (amax_in && quantize_ts_tma_eligible(a) && !env_int("MQ_QUANT_TS_TWO_PASS", 0)) {
+    count_launches(1);
+    return launch_quantize_ts_tma(a, amax_in, stats, s, true);
+  }
+  // the source of either layout is a dense array of n floats
   e = launch_pdl(tensor_amax_kernel, dim3((unsigned)blocks), dim3(256), 0, s, a.src, n, reinterpret_cast<unsigned*>(stats + 1), a.act);
   if (e != cudaSuccess) return e;
   const int Rb = (a.R + 15) / 16, Cb = a.Cp / 16;

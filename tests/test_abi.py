@@ -133,3 +133,8 @@ def test_bad_arguments_are_rejected_on_the_host(mq):
     assert L.mq_conv_fwd_ts(ctypes.byref(good), ctypes.byref(ts_x), ctypes.byref(ts_w), 0, ctypes.c_void_p(0x6002), ctypes.byref(ts_y), None, 0, None) == 3
     ts_g = mq._QTensor(0x1000, 0x2000, 1 << 30, 1 << 30, E2M1, 2, TS16, 0x5000)
     assert L.mq_conv_bwd_data_ts(ctypes.byref(good), ctypes.byref(ts_w), ctypes.byref(ts_g), None, ctypes.byref(ts_g), None, 0, None) == 1
+    # the quantizer of that format: the supplied maximum may not live in the words the call rewrites, and must be 4-byte aligned
+    src = ctypes.c_void_p(0x7000)
+    assert L.mq_quantize_ts(ctypes.byref(good), src, F32, NCHW, ctypes.byref(ts_x), ctypes.c_void_p(0x5004), None, None) == 1
+    assert L.mq_quantize_ts(ctypes.byref(good), src, F32, NCHW, ctypes.byref(ts_x), ctypes.c_void_p(0x6002), None, None) == 3
+    assert L.mq_quantize_ts(ctypes.byref(good), src, F32, NCHW, ctypes.byref(mx_y), amax, None, None) == 1   # not that format

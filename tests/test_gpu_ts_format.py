@@ -89,9 +89,16 @@ def test_whole_line_quantizer(knobs, name, shape):
         assert_ts_equal(f"{name} {what}", mq.quantize_ts(d, r, dev(t)), o)
         amax = np.float32(1.7) * np.abs(t).max()
         o2 = oracle.quantize_ts(d, r, t, B16, amax=float(amax))
-        g2 = mq.quantize_ts(d, r, dev(t), amax_in=torch.tensor([amax], dtype=torch.float32, device="cuda"))
+        amax_dev, t_dev = torch.tensor([amax], dtype=torch.float32, device="cuda"), dev(t)
+        n0 = mq.kernel_launch_count()
+        g2 = mq.quantize_ts(d, r, t_dev, amax_in=amax_dev)
+        n1 = mq.kernel_launch_count()
         assert_same_bytes(g2.scales, o2[1], f"{name} {what} supplied maximum: block scales")
         assert_same_bytes(g2.codes, o2[0], f"{name} {what} supplied maximum: codes")
+        # a supplied maximum makes it ONE launch that still records the tensor's own maximum for the next step
+        assert n1 - n0 == 1, (name, what, n1 - n0)
+        st = host(g2.tensor_scale)
+        assert st[1] == np.abs(t).max() and st[0] == np.float32(o2[2]), (name, what, st)
         o3 = oracle.quantize_ts(d, r, t, B16, seed=99)
         g3 = mq.quantize_ts(d, r, dev(t), seed=99)
         assert_same_bytes(g3.scales, o3[1], f"{name} {what} stochastic: block scales")
