@@ -28,6 +28,14 @@
  *   32 input x 32 output channels (W) at one spatial / tap position, so that every 32-element
  *   line of a tile, in either contraction direction, is a standard MX block (Sec. IV-B).
  *
+ * Packed 6-bit storage (MQ_E3M2_P6, MQ_E2M3_P6): the 6-bit element formats at the six bits per element Sec. VI counts
+ *   for them.  Layouts as above; a group of 16 consecutive channels occupies 12 bytes, code k of the group in bits
+ *   6k .. 6k+5 of that 96-bit little-endian field (so a row of Cp channels takes 3 Cp / 4 bytes, and the tensor 3/4 of
+ *   the bytes of MQ_E3M2 / MQ_E2M3, which store one code per byte).  Scales are unchanged.  mq_qtensor_sizes,
+ *   mq_im2col_sizes, mq_workspace_size, mq_quantize, mq_quantize_sr, mq_cbf_im2col and the three mq_conv_* GEMMs accept
+ *   them and give the results of the one-code-per-byte format bit for bit; the quantizing producer epilogues,
+ *   mq_conv_bwd_data_static and mq_conv_layer_host return MQ_ERR_UNSUPPORTED for them.
+ *
  * Line blocks (MQ_BLOCK_LINE32): the one-directional block of Sec. III-A (Eq. 5-6) - 32 consecutive channels of ONE
  *   row (sample / output channel) share the scale, amax over those 32 elements.  Codes are laid out as above; scales
  *   have one entry per row instead of one per 32 rows:
@@ -74,10 +82,10 @@ typedef enum {
 } mq_status;
 
 typedef enum { MQ_E4M3 = 0, MQ_E5M2 = 1, MQ_E2M1 = 2,
-               MQ_E3M2 = 3, MQ_E2M3 = 4 } mq_elem;   /* element format, Sec. II-D; the 6-bit formats (Sec. V: the
+               MQ_E3M2 = 3, MQ_E2M3 = 4,             /* element format, Sec. II-D; the 6-bit formats (Sec. V: the
                                                         activations of MicroQonv+, the "-6" variant) are stored one code
-                                                        per byte, value in the low six bits, sign in bit 5 (the
-                                                        convolution calls pack or re-encode them in their scratch) */
+                                                        per byte, value in the low six bits, sign in bit 5 ...        */
+               MQ_E3M2_P6 = 5, MQ_E2M3_P6 = 6 } mq_elem; /* ... or packed, 16 codes in 12 bytes (see above)            */
 typedef enum { MQ_ROLE_X = 0, MQ_ROLE_W = 1, MQ_ROLE_DY = 2 } mq_role; /* which tensor, Sec. IV-B   */
 typedef enum { MQ_NCHW = 0, MQ_HWNC = 1 } mq_layout;                   /* layout of an unquantized tensor */
 typedef enum { MQ_BLOCK_TILE32 = 0,      /* 32 x 32 square block (Sec. IV-B), the default           */

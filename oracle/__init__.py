@@ -8,7 +8,7 @@ All arrays are host numpy arrays.  Conventions (Sec. II-A, IV-A, IV-B of the pap
   * ``desc`` = ConvDesc(N, C_in, H, W, C_out, Kh, Kw, stride_h, stride_w, pad_h, pad_w)
   * roles: X (activations, NCHW), W (weights, OIHW), DY (output gradient, N.Cout.Ho.Wo)
   * element formats: E4M3, E5M2, E3M2, E2M3 (one byte per code), E2M1 (two codes per byte, lower index in
-    the low nibble); block scale E8M0
+    the low nibble); block scale E8M0; pack6 / unpack6 give the packed storage of the 6-bit codes (16 in 12 bytes)
   * block shape (br, bc): br along N (X, DY) or Cout (W); bc along the channel axis that is
     stored fastest.  (32, 32) is the square block, (1, 32) the line block.
 """
@@ -192,6 +192,24 @@ def dequant(desc, role, fmt, codes, scales, block=(32, 32)):
     scales = np.ascontiguousarray(scales, dtype=np.uint8)
     _l().orc_dequant(_p(_desc(desc)), role, fmt, block[0], block[1], _p(codes), _p(scales), _p(out))
     return out
+
+
+def pack6(codes):
+    """Packed storage of a tensor of 6-bit codes (Sec. VI counts six bits per element for the 6-bit formats): the low six
+    bits of every code as one little-endian bit stream - code k of the flat array occupies bits 6k .. 6k+5 - so that 16
+    codes take 12 bytes.  Layout only: no arithmetic of the method."""
+    c = np.ascontiguousarray(codes, dtype=np.uint8).reshape(-1)
+    assert c.size % 4 == 0 and int(c.max(initial=0)) < 64
+    bits = np.unpackbits(c[:, None], axis=1, bitorder="little")[:, :6]
+    return np.packbits(bits.reshape(-1), bitorder="little")
+
+
+def unpack6(packed):
+    """Inverse of pack6: one code per byte."""
+    b = np.ascontiguousarray(packed, dtype=np.uint8).reshape(-1)
+    assert b.size % 3 == 0
+    bits = np.unpackbits(b, bitorder="little").reshape(-1, 6)
+    return np.packbits(np.pad(bits, ((0, 0), (0, 2))), axis=1, bitorder="little").reshape(-1)
 
 
 def im2col_sizes(desc, fmt, block=(32, 32)):

@@ -34,7 +34,8 @@ static void env_forget() {
 
 namespace {
 
-bool valid_fmt(int f) { return f == MQ_E4M3 || f == MQ_E5M2 || f == MQ_E2M1 || f == MQ_E3M2 || f == MQ_E2M3; }
+bool valid_fmt_unpacked(int f) { return f == MQ_E4M3 || f == MQ_E5M2 || f == MQ_E2M1 || f == MQ_E3M2 || f == MQ_E2M3; }
+bool valid_fmt(int f) { return valid_fmt_unpacked(f) || fmt_is_packed6(f); }
 bool valid_role(int r) { return r == MQ_ROLE_X || r == MQ_ROLE_W || r == MQ_ROLE_DY; }
 bool valid_block(int b) { return b == MQ_BLOCK_TILE32 || b == MQ_BLOCK_LINE32 || b == MQ_BLOCK_TS16; }
 bool valid_dtype(int t) { return t == MQ_F32 || t == MQ_BF16; }
@@ -60,7 +61,7 @@ View view_of(const Geom& g, int role) {
 
 void sizes_of(const Geom& g, int role, int fmt, int block, size_t* cb, size_t* sb) {
   View v = view_of(g, role);
-  *cb = (size_t)(v.P * v.R * v.Cp) * fmt_bits(fmt) / 8;
+  *cb = (size_t)(v.P * v.R * v.Cp) * fmt_store_bits(fmt) / 8;
   if (block == MQ_BLOCK_TS16) *sb = (size_t)(v.P * ((v.R + 15) / 16) * (v.Cp / 16));
   else *sb = (size_t)(v.P * (block == MQ_BLOCK_LINE32 ? v.R : (v.R + 31) / 32) * (v.Cp / 32));
 }
@@ -335,16 +336,21 @@ mq_status run_conv_tc(int op, const Geom& g, ConvTcPlan& pl, const mq_qtensor* q
   // repacked - 16 codes -> 12 packed bytes + 4 bytes of padding per 16-byte chunk, the container of the MMA's 6-bit types)
   const uint8_t* w_stored = static_cast<const uint8_t*>(qw->codes);
   const uint8_t* x_stored = static_cast<const uint8_t*>(qx_like->codes);
+  // (operands in packed 6-bit storage - 16 codes in 12 bytes - reach that container by a copy that pads each group; the
+  // weights of the input gradient arrive here one code per byte whatever their storage: their re-layout reads bytes)
+  const int fx = fmt_base(qx_like->fmt), fw = fmt_base(qw->fmt);
+  const bool pk_x = fmt_is_packed6(qx_like->fmt), pk_w = fmt_is_packed6(qw->fmt);
+  if (pk_w && op != MQ_OP_FWD) return MQ_ERR_INVALID_ARG;
   const uint8_t* b_unpacked = op == MQ_OP_FWD ? w_stored : base;
-  const uint8_t* b_codes = fmt_is_6bit(qw->fmt) ? base + pl.off_pack_b : b_unpacked;
-  const uint8_t* a_codes = fmt_is_6bit(qx_like->fmt) ? base + pl.off_pack_a : x_stored;
+  const uint8_t* b_codes = fmt_is_6bit(fw) ? base + pl.off_pack_b : b_unpacked;
+  const uint8_t* a_codes = fmt_is_6bit(fx) ? base + pl.off_pack_a : x_stored;
   uint8_t* wt_scales = base + pl.off_wt_scales;
   bool separate_transpose = false;
   if (op == MQ_OP_FWD) {
     p.b_scales = qw->scales;
   } else {
     // per-tap kernel, operands that need no repacking: the re-layout rides in the scale-expansion launch
-    p.wt_fused = (!p.halo && !fmt_is_6bit(qw->fmt) && (p.kind_fp4 == 2 || !env_int("MQ_TC_NO_WT_FUSED", 0))) ? 1 : 0;   // kind 2: this route only
+    p.wt_fused = (!p.halo && !fmt_is_6bit(fw) && (p.kind_fp4 == 2 || !env_int("MQ_TC_NO_WT_FUSED", 0))) ? 1 : 0;   // kind 2: this route only
     if (p.wt_fused) {
       p.wt_in = w_stored; p.wt_out = base; p.wt_sc_in = qw->scales;
       p.wt_Cout = g.Cout; p.wt_Cop = g.Cop; p.wt_Cp = g.Cp; p.wt_bx = g.Cp / 32; p.wt_by = g.Cop / 32;
@@ -411,9 +417,15 @@ mq_status run_conv_tc(int op, const Geom& g, ConvTcPlan& pl, const mq_qtensor* q
     }
   }
   // ---- launches
-  if (separate_transpose && launch_weight_transpose(w_stored, qw->scales, base, wt_scales, g, qw->fmt, stream) != cudaSuccess) return MQ_ERR_CUDA;
-  if (fmt_is_6bit(qx_like->fmt) && launch_pack6(x_stored, base + pl.off_pack_a, (size_t)p.Hs * p.Ws * g.N * pl.rowbytes, stream) != cudaSuccess) return MQ_ERR_CUDA;
-  if (fmt_is_6bit(qw->fmt) && launch_pack6(b_unpacked, base + pl.off_pack_b, (size_t)pl.rows_b * taps * pl.rowbytes, stream) != cudaSuccess) return MQ_ERR_CUDA;
+  if (separate_transpose && launch_weight_transpose(w_stored, qw->scales, base, wt_scales, g, fw, stream) != cudaSuccess) return MQ_ERR_CUDA;
+  if (fmt_is_6bit(fx)) {
+    const size_t n = (size_t)p.Hs * p.Ws * g.N * pl.rowbytes;
+    if ((pk_x ? launch_unpack6(x_stored, base + pl.off_pack_a, n, 0, fx, stream) : launch_pack6(x_stored, base + pl.off_pack_a, n, stream)) != cudaSuccess) return MQ_ERR_CUDA;
+  }
+  if (fmt_is_6bit(fw)) {
+    const size_t n = (size_t)pl.rows_b * taps * pl.rowbytes;
+    if ((pk_w ? launch_unpack6(b_unpacked, base + pl.off_pack_b, n, 0, fw, stream) : launch_pack6(b_unpacked, base + pl.off_pack_b, n, stream)) != cudaSuccess) return MQ_ERR_CUDA;
+  }
   if (!(p.halo && p.fused) && launch_expand_conv_scales(p, stream) != cudaSuccess) return MQ_ERR_CUDA;
   return launch_conv_tc(p, map_a, map_w, map_out, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }
@@ -570,13 +582,15 @@ mq_status run_wgrad_tc(const Geom& g, WgradPlan& w, const mq_qtensor* qx, const 
   } else {
     const uint8_t* g_codes = static_cast<const uint8_t*>(qg->codes);
     const uint8_t* x_codes = static_cast<const uint8_t*>(qx->codes);
-    int fmt_g_eff = qg->fmt, fmt_x_eff = qx->fmt;
-    if (fmt_is_6bit(qx->fmt)) {
-      if (launch_recode6_e4m3(x_codes, xt, (size_t)g.H * g.W * g.N * g.Cp, qx->fmt, stream) != cudaSuccess) return MQ_ERR_CUDA;
+    int fmt_g_eff = fmt_base(qg->fmt), fmt_x_eff = fmt_base(qx->fmt);
+    if (fmt_is_6bit(fmt_x_eff)) {   // (from either storage of the 6-bit codes)
+      const size_t n = (size_t)g.H * g.W * g.N * g.Cp;
+      if ((fmt_is_packed6(qx->fmt) ? launch_unpack6(x_codes, xt, n, 2, fmt_x_eff, stream) : launch_recode6_e4m3(x_codes, xt, n, fmt_x_eff, stream)) != cudaSuccess) return MQ_ERR_CUDA;
       x_codes = xt; fmt_x_eff = MQ_E4M3;
     }
-    if (fmt_is_6bit(qg->fmt)) {
-      if (launch_recode6_e4m3(g_codes, gt, (size_t)g.Ho * g.Wo * g.N * g.Cop, qg->fmt, stream) != cudaSuccess) return MQ_ERR_CUDA;
+    if (fmt_is_6bit(fmt_g_eff)) {
+      const size_t n = (size_t)g.Ho * g.Wo * g.N * g.Cop;
+      if ((fmt_is_packed6(qg->fmt) ? launch_unpack6(g_codes, gt, n, 2, fmt_g_eff, stream) : launch_recode6_e4m3(g_codes, gt, n, fmt_g_eff, stream)) != cudaSuccess) return MQ_ERR_CUDA;
       g_codes = gt; fmt_g_eff = MQ_E4M3;
     }
     if (w.recode4) {
@@ -658,29 +672,93 @@ mq_status check_conv_args(int op, const mq_conv_desc* desc, const mq_qtensor* qa
   return MQ_OK;
 }
 
-mq_status run_conv(int op, const mq_conv_desc* desc, const mq_qtensor* qa, int role_a, const mq_qtensor* qb, int role_b,
+// Does a forward / input-gradient call of this layer, formats and output layout run on the tensor cores?  (formats: one code per byte)
+bool conv_takes_tc(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, bool line, bool ts16, ConvTcPlan* pl) {
+  return (!ts16 || !env_int("MQ_TC_NO_TS16", 0)) && (op == MQ_OP_FWD || op == MQ_OP_BWD_DATA) && conv_tc_eligible(op, g, fmt_x_like, fmt_w) &&
+         conv_tc_plan(op, g, fmt_x_like, fmt_w, layout, pl, line, false, ts16);
+}
+
+// Operands in packed 6-bit storage: scratch, behind the call's own, for the one-code-per-byte copies of the operands no
+// kernel of the call's route reads packed - the weights of the input gradient (their re-layout reads bytes) and both
+// operands of a layer the CUDA-core kernels take.  (The tensor-core routes read a packed activation / gradient tensor
+// through the copy that builds the MMA's container, which a one-code-per-byte tensor needs as well.)
+struct PackedExtra { bool keep_a, keep_b; size_t bytes_a, bytes_b; };
+int operand_role(int op, int which) {
+  if (op == MQ_OP_FWD) return which == 0 ? MQ_ROLE_X : MQ_ROLE_W;
+  if (op == MQ_OP_BWD_DATA) return which == 0 ? MQ_ROLE_W : MQ_ROLE_DY;
+  return which == 0 ? MQ_ROLE_X : MQ_ROLE_DY;
+}
+PackedExtra packed_extra(int op, const Geom& g, int fmt_a, int fmt_b, int block) {
+  PackedExtra e{false, false, 0, 0};
+  const bool pa = fmt_is_packed6(fmt_a), pb = fmt_is_packed6(fmt_b);
+  if (!pa && !pb) return e;
+  const int fa = fmt_base(fmt_a), fb = fmt_base(fmt_b);
+  const bool line = block == MQ_BLOCK_LINE32, ts16 = block == MQ_BLOCK_TS16;
+  bool tc = true;    // on the tensor cores whatever the output layout
+  ConvTcPlan pl;
+  if (op == MQ_OP_BWD_WEIGHT) tc = wgrad_plan(g, fa, fb, ts16).ok;
+  else for (int layout = 0; layout < 2; ++layout) tc = tc && conv_takes_tc(op, g, op == MQ_OP_FWD ? fa : fb, op == MQ_OP_FWD ? fb : fa, layout, line, ts16, &pl);
+  e.keep_a = pa && (!tc || op == MQ_OP_BWD_DATA);
+  e.keep_b = pb && !tc;
+  const View va = view_of(g, operand_role(op, 0)), vb = view_of(g, operand_role(op, 1));
+  e.bytes_a = e.keep_a ? ((size_t)(va.P * va.R * va.Cp) + 255) / 256 * 256 : 0;
+  e.bytes_b = e.keep_b ? ((size_t)(vb.P * vb.R * vb.Cp) + 255) / 256 * 256 : 0;
+  return e;
+}
+size_t conv_workspace_unpacked(int op, const Geom& g, int fa, int fb, int block) {
+  const bool line = block == MQ_BLOCK_LINE32, ts16 = block == MQ_BLOCK_TS16;
+  size_t bytes = conv_generic_workspace(op, g);
+  if (op == MQ_OP_FWD && conv_tc_eligible(op, g, fa, fb)) bytes = conv_tc_workspace(op, g, fa, fb, line, ts16);
+  if (op == MQ_OP_BWD_DATA && conv_tc_eligible(op, g, fb, fa)) bytes = conv_tc_workspace(op, g, fb, fa, false, ts16);
+  if (op == MQ_OP_BWD_WEIGHT) {
+    const WgradPlan w = wgrad_plan(g, fa, fb, ts16);
+    if (w.ok) bytes = w.total;
+  }
+  return bytes;
+}
+
+mq_status run_conv(int op, const mq_conv_desc* desc, const mq_qtensor* qa_in, int role_a, const mq_qtensor* qb_in, int role_b,
                    void* out, int dtype, int layout, void* ws, size_t ws_bytes, void* stream) {
-  mq_status st = check_conv_args(op, desc, qa, role_a, qb, role_b, out, dtype, layout);
+  mq_status st = check_conv_args(op, desc, qa_in, role_a, qb_in, role_b, out, dtype, layout);
   if (st != MQ_OK) return st;
   Geom g = make_geom(*desc);
   if (ws && !aligned16(ws)) return MQ_ERR_ALIGNMENT;
   size_t need = 0;
-  mq_workspace_size(desc, op, qa->fmt, qb->fmt, qa->block, &need);
+  mq_workspace_size(desc, op, qa_in->fmt, qb_in->fmt, qa_in->block, &need);
   if (need > 0 && (!ws || ws_bytes < need)) return MQ_ERR_BUFFER_TOO_SMALL;
-  // tensor cores when the layer is eligible AND a plan exists for it; everything else runs on the CUDA-core kernels
-  {
+  const int fa = fmt_base(qa_in->fmt), fb = fmt_base(qb_in->fmt);
+  const bool ts16 = qa_in->block == MQ_BLOCK_TS16, line = qa_in->block == MQ_BLOCK_LINE32;
+  // which route: tensor cores when the layer is eligible AND a plan exists for it; everything else runs on the CUDA-core kernels
+  ConvTcPlan pl;
+  WgradPlan wp;
+  wp.ok = false;
+  const bool conv_tc = op != MQ_OP_BWD_WEIGHT && conv_takes_tc(op, g, op == MQ_OP_FWD ? fa : fb, op == MQ_OP_FWD ? fb : fa, layout, line, ts16, &pl);
+  if (op == MQ_OP_BWD_WEIGHT) wp = wgrad_plan(g, fa, fb, ts16);
+  const bool tc = conv_tc || wp.ok;
+  // operands in packed 6-bit storage that this route reads one code per byte: copies behind the call's own scratch
+  mq_qtensor qa_v = *qa_in, qb_v = *qb_in;
+  if (fmt_is_packed6(qa_in->fmt) || fmt_is_packed6(qb_in->fmt)) {
+    const PackedExtra pe = packed_extra(op, g, qa_in->fmt, qb_in->fmt, qa_in->block);
+    uint8_t* extra = static_cast<uint8_t*>(ws) + (conv_workspace_unpacked(op, g, fa, fb, qa_in->block) + 255) / 256 * 256;
+    if (fmt_is_packed6(qa_in->fmt) && (!tc || op == MQ_OP_BWD_DATA)) {
+      const View v = view_of(g, role_a);
+      if (launch_unpack6(static_cast<const uint8_t*>(qa_in->codes), extra, (size_t)(v.P * v.R * v.Cp), 1, fa, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MQ_ERR_CUDA;
+      qa_v.codes = extra; qa_v.fmt = fa; qa_v.codes_bytes = pe.bytes_a;
+    }
+    if (fmt_is_packed6(qb_in->fmt) && !tc) {
+      const View v = view_of(g, role_b);
+      if (launch_unpack6(static_cast<const uint8_t*>(qb_in->codes), extra + pe.bytes_a, (size_t)(v.P * v.R * v.Cp), 1, fb, static_cast<cudaStream_t>(stream)) != cudaSuccess) return MQ_ERR_CUDA;
+      qb_v.codes = extra + pe.bytes_a; qb_v.fmt = fb; qb_v.codes_bytes = pe.bytes_b;
+    }
+  }
+  const mq_qtensor* qa = &qa_v;
+  const mq_qtensor* qb = &qb_v;
+  if (conv_tc) {
     const mq_qtensor* qx_like = op == MQ_OP_FWD ? qa : qb;
     const mq_qtensor* qw = op == MQ_OP_FWD ? qb : qa;
-    ConvTcPlan pl;
-    const bool ts16 = qa->block == MQ_BLOCK_TS16;
-    if ((!ts16 || !env_int("MQ_TC_NO_TS16", 0)) && (op == MQ_OP_FWD || op == MQ_OP_BWD_DATA) && conv_tc_eligible(op, g, qx_like->fmt, qw->fmt) &&
-        conv_tc_plan(op, g, qx_like->fmt, qw->fmt, layout, &pl, qx_like->block == MQ_BLOCK_LINE32, false, ts16))
-      return run_conv_tc(op, g, pl, qx_like, qw, static_cast<float*>(out), layout, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
+    return run_conv_tc(op, g, pl, qx_like, qw, static_cast<float*>(out), layout, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
   }
-  if (op == MQ_OP_BWD_WEIGHT) {
-    WgradPlan w = wgrad_plan(g, qa->fmt, qb->fmt, qa->block == MQ_BLOCK_TS16);
-    if (w.ok) return run_wgrad_tc(g, w, qa, qb, static_cast<float*>(out), layout, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
-  }
+  if (wp.ok) return run_wgrad_tc(g, wp, qa, qb, static_cast<float*>(out), layout, ws, device_status_ptr(), static_cast<cudaStream_t>(stream));
   ConvArgs a;
   a.g = g;
   a.a_codes = static_cast<const uint8_t*>(qa->codes); a.a_scales = qa->scales; a.fmt_a = qa->fmt;
@@ -716,7 +794,7 @@ mq_status mq_im2col_sizes(const mq_conv_desc* desc, int fmt, int block, size_t* 
   if (st != MQ_OK) return st;
   if (!valid_fmt(fmt) || !valid_block(block) || !codes_bytes || !scales_bytes) return MQ_ERR_INVALID_ARG;
   Geom g = make_geom(*desc);
-  *codes_bytes = (size_t)g.Ho * g.Wo * g.N * g.Kh * g.Kw * g.Cp * fmt_bits(fmt) / 8;
+  *codes_bytes = (size_t)g.Ho * g.Wo * g.N * g.Kh * g.Kw * g.Cp * fmt_store_bits(fmt) / 8;
   if (block == MQ_BLOCK_TS16) *scales_bytes = (size_t)g.Ho * g.Wo * ((g.N + 15) / 16) * g.Kh * g.Kw * (g.Cp / 16);
   else *scales_bytes = (size_t)g.Ho * g.Wo * (block == MQ_BLOCK_LINE32 ? g.N : g.Nt) * g.Kh * g.Kw * g.Ct;
   return MQ_OK;
@@ -729,15 +807,11 @@ mq_status mq_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt
   if (op != MQ_OP_FWD && op != MQ_OP_BWD_DATA && op != MQ_OP_BWD_WEIGHT) return MQ_ERR_INVALID_ARG;
   if (block == MQ_BLOCK_LINE32 && op != MQ_OP_FWD) return MQ_ERR_UNSUPPORTED;
   const Geom g = make_geom(*desc);
-  const bool line = block == MQ_BLOCK_LINE32;
-  *bytes = conv_generic_workspace(op, g);
-  const bool ts16 = block == MQ_BLOCK_TS16;
-  if (ts16 && (fmt_a != MQ_E2M1 || fmt_b != MQ_E2M1)) return MQ_ERR_INVALID_ARG;
-  if (op == MQ_OP_FWD && conv_tc_eligible(op, g, fmt_a, fmt_b)) *bytes = conv_tc_workspace(op, g, fmt_a, fmt_b, line, ts16);
-  if (op == MQ_OP_BWD_DATA && conv_tc_eligible(op, g, fmt_b, fmt_a)) *bytes = conv_tc_workspace(op, g, fmt_b, fmt_a, false, ts16);
-  if (op == MQ_OP_BWD_WEIGHT) {
-    const WgradPlan w = wgrad_plan(g, fmt_a, fmt_b, ts16);
-    if (w.ok) *bytes = w.total;
+  if (block == MQ_BLOCK_TS16 && (fmt_a != MQ_E2M1 || fmt_b != MQ_E2M1)) return MQ_ERR_INVALID_ARG;
+  *bytes = conv_workspace_unpacked(op, g, fmt_base(fmt_a), fmt_base(fmt_b), block);
+  if (fmt_is_packed6(fmt_a) || fmt_is_packed6(fmt_b)) {
+    const PackedExtra pe = packed_extra(op, g, fmt_a, fmt_b, block);
+    *bytes = (*bytes + 255) / 256 * 256 + pe.bytes_a + pe.bytes_b;
   }
   return MQ_OK;
 }
@@ -769,7 +843,8 @@ static mq_status quantize_impl(const mq_conv_desc* desc, const void* src, int sr
     a.out_stride_p = v.R * v.Cp; a.out_stride_r = v.Cp;
     a.sc_stride_p = Rt * Ct; a.sc_stride_r = Ct;
   }
-  a.fmt = dst->fmt;
+  a.fmt = fmt_base(dst->fmt);
+  a.packed6 = fmt_is_packed6(dst->fmt) ? 1 : 0;
   a.src_stride_p = 0; a.src_stride_r = 0;
   if (src_layout == MQ_HWNC) {   // channel-fastest source: activations / gradients [pixel][n][c], weights [cout][tap][cin]
     if (dst->role == MQ_ROLE_W) { a.src_stride_p = v.C; a.src_stride_r = v.P * v.C; }
@@ -887,6 +962,7 @@ mq_status run_conv_mx(int op, const mq_conv_desc* desc, const mq_qtensor* qa, in
     mx_out_sizes(g, op, out->fmt, &cb, &sb);
     if (out->codes_bytes < cb || out->scales_bytes < sb) return MQ_ERR_BUFFER_TOO_SMALL;
     if (qa->block != MQ_BLOCK_TILE32 || qb->block != MQ_BLOCK_TILE32 || out->block != MQ_BLOCK_TILE32) return MQ_ERR_UNSUPPORTED;
+    if (fmt_is_packed6(qa->fmt) || fmt_is_packed6(qb->fmt) || fmt_is_packed6(out->fmt)) return MQ_ERR_UNSUPPORTED;   // packed 6-bit storage: not here
     fmt_x_like = op == MQ_OP_FWD ? qa->fmt : qb->fmt; fmt_w = op == MQ_OP_FWD ? qb->fmt : qa->fmt;
   }
   ConvTcPlan pl;
@@ -935,6 +1011,7 @@ mq_status run_conv_mx(int op, const mq_conv_desc* desc, const mq_qtensor* qa, in
 
 mq_status mq_conv_mx_workspace_size(const mq_conv_desc* desc, int op, int fmt_a, int fmt_b, size_t* bytes) {
   if (!bytes || !valid_fmt(fmt_a) || !valid_fmt(fmt_b) || (op != MQ_OP_FWD && op != MQ_OP_BWD_DATA)) return MQ_ERR_INVALID_ARG;
+  if (fmt_is_packed6(fmt_a) || fmt_is_packed6(fmt_b)) return MQ_ERR_UNSUPPORTED;
   mq_qtensor a{}, b{};
   a.fmt = fmt_a; b.fmt = fmt_b;
   return run_conv_mx(op, desc, &a, 0, &b, 0, 0, nullptr, 0, nullptr, 0, nullptr, bytes);

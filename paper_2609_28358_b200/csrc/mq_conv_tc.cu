@@ -1783,6 +1783,46 @@ cudaError_t launch_pack6(const uint8_t* in, uint8_t* out, size_t nbytes, cudaStr
   return launch_pdl(pack6_kernel, dim3((unsigned)blocks), dim3(256), 0, s, reinterpret_cast<const uint4*>(in), reinterpret_cast<uint4*>(out), nchunks);
 }
 
+// Packed 6-bit storage (16 codes in 12 bytes) -> what a kernel reads.  MODE 0: the MMA's container (the 12 bytes + 4 bytes of
+// padding); 1: one code per byte; 2: E4M3 bytes of the same values (the weight gradient's 8-bit path).
+template <int MODE, bool IS_E3M2>
+__global__ void __launch_bounds__(256) unpack6_kernel(const uint32_t* __restrict__ in, uint4* __restrict__ out, size_t ngroups) {
+  pdl_wait();
+  for (size_t i = (size_t)blockIdx.x * 256 + threadIdx.x; i < ngroups; i += (size_t)gridDim.x * 256) {
+    const uint32_t f[3] = {__ldg(in + 3 * i), __ldg(in + 3 * i + 1), __ldg(in + 3 * i + 2)};
+    if (MODE == 0) { out[i] = make_uint4(f[0], f[1], f[2], 0u); continue; }
+    uint32_t w[4];
+    unpack6x16(f, w);
+    if (MODE == 2) {
+#pragma unroll
+      for (int q = 0; q < 4; ++q) {
+        uint32_t r = 0;
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          const unsigned short pair = (unsigned short)((w[q] >> (16 * h)) & 0xFFFF);
+          const __half2_raw hr = __nv_cvt_fp6x2_to_halfraw2((__nv_fp6x2_storage_t)pair, IS_E3M2 ? __NV_E3M2 : __NV_E2M3);
+          r |= (uint32_t)__nv_cvt_halfraw2_to_fp8x2(hr, __NV_SATFINITE, __NV_E4M3) << (16 * h);   // exact: the value is representable
+        }
+        w[q] = r;
+      }
+    }
+    out[i] = make_uint4(w[0], w[1], w[2], w[3]);
+  }
+}
+cudaError_t launch_unpack6(const uint8_t* in, uint8_t* out, size_t n_codes, int mode, int fmt6, cudaStream_t s) {
+  const size_t ngroups = n_codes / 16;
+  if (ngroups == 0) return cudaSuccess;
+  size_t blocks = (ngroups + 255) / 256;
+  if (blocks > sm_count() * 16) blocks = sm_count() * 16;
+  count_launches(1);
+  const uint32_t* src = reinterpret_cast<const uint32_t*>(in);
+  uint4* dst = reinterpret_cast<uint4*>(out);
+  if (mode == 0) return launch_pdl(unpack6_kernel<0, false>, dim3((unsigned)blocks), dim3(256), 0, s, src, dst, ngroups);
+  if (mode == 1) return launch_pdl(unpack6_kernel<1, false>, dim3((unsigned)blocks), dim3(256), 0, s, src, dst, ngroups);
+  if (fmt_base(fmt6) == MQ_E3M2) return launch_pdl(unpack6_kernel<2, true>, dim3((unsigned)blocks), dim3(256), 0, s, src, dst, ngroups);
+  return launch_pdl(unpack6_kernel<2, false>, dim3((unsigned)blocks), dim3(256), 0, s, src, dst, ngroups);
+}
+
 template <bool IS_E3M2>
 __global__ void __launch_bounds__(256) recode6_kernel(const uint4* __restrict__ in, uint4* __restrict__ out, size_t nchunks) {
   pdl_wait();

@@ -92,6 +92,9 @@ struct ConvTcParams {
 // p.tma_store is set.
 // 16-byte chunks of one-code-per-byte 6-bit codes -> 12 packed bytes (code i at bit 6 i) + 4 zero bytes
 cudaError_t launch_pack6(const uint8_t* in, uint8_t* out, size_t nbytes, cudaStream_t s);
+// packed 6-bit storage (16 codes in 12 bytes, n_codes a multiple of 16) -> mode 0: that container; 1: one code per byte;
+// 2: E4M3 bytes of the same values (fmt6 says which 6-bit format)
+cudaError_t launch_unpack6(const uint8_t* in, uint8_t* out, size_t n_codes, int mode, int fmt6, cudaStream_t s);
 // one-code-per-byte E3M2 / E2M3 codes -> the E4M3 codes of the same values (every 6-bit value is an E4M3 value)
 cudaError_t launch_recode6_e4m3(const uint8_t* in, uint8_t* out, size_t nbytes, int fmt6, cudaStream_t s);
 // packed E2M1 codes (two per byte) -> the E4M3 codes of the same values, one per byte; n_out = elements = output bytes

@@ -11,11 +11,16 @@ namespace mq {
 namespace {
 
 constexpr int IC_THREADS = 256;
-constexpr int IC_MAX_J = 1024;   // chunks of 16 bytes per X' row held in the offset table
+constexpr int IC_MAX_J = 1024;   // chunks per X' row held in the offset table
 constexpr int IC_TABLE = 2048;   // table entries per block: PX pixels x J chunks
 
+__device__ __forceinline__ void zero_chunk(uint4& v) { v = make_uint4(0, 0, 0, 0); }
+__device__ __forceinline__ void zero_chunk(uint2& v) { v = make_uint2(0, 0); }
+
 // PX consecutive output pixels per block amortise the block's fixed cost (launch, offset table, barrier) over
-// PX * 32 rows of X'.
+// PX * 32 rows of X'.  V: the chunk - 16 bytes, or 8 where a row is no multiple of 16 bytes (packed 6-bit codes, 24 bytes per
+// 32 channels, with an odd number of channel tiles).
+template <typename V>
 __global__ void __launch_bounds__(IC_THREADS) im2col_kernel(Im2colArgs a, int rc, int J, int PX, unsigned n_main) {
   pdl_wait();
   const Geom& g = a.g;
@@ -40,22 +45,22 @@ __global__ void __launch_bounds__(IC_THREADS) im2col_kernel(Im2colArgs a, int rc
     const int n0 = nt * 32;
     const int rows = min(32, g.N - n0);
     const int total = rows * J;
-    const uint4* src = reinterpret_cast<const uint4*>(a.codes) + (long long)n0 * rc;
+    const V* src = reinterpret_cast<const V*>(a.codes) + (long long)n0 * rc;
     const int dn = IC_THREADS / J, dj = IC_THREADS - dn * J;
-    uint4* dst0 = reinterpret_cast<uint4*>(a.out_codes) + ((long long)pix0 * g.N + n0) * J;
+    V* dst0 = reinterpret_cast<V*>(a.out_codes) + ((long long)pix0 * g.N + n0) * J;
     const long long px_stride = (long long)g.N * J;      // chunks between the rows of consecutive pixels
     // chunk i = n * J + j of every pixel of the block, advanced by IC_THREADS per step without divisions; the loads of
     // four pixels are issued before their stores (the kernel waits on L2 latency, not on bandwidth)
     int n = threadIdx.x / J, j = threadIdx.x - n * J;
 #pragma unroll 1
     for (int i = threadIdx.x; i < total; i += IC_THREADS) {
-      const uint4* s_n = src + n * rc;
+      const V* s_n = src + n * rc;
 #pragma unroll 1
       for (int px0 = 0; px0 < px_n; px0 += 4) {
-        uint4 v[4];
+        V v[4];
 #pragma unroll
         for (int q = 0; q < 4; ++q) {
-          v[q] = make_uint4(0, 0, 0, 0);
+          zero_chunk(v[q]);
           if (px0 + q < px_n) {
             const int so = soff[(px0 + q) * J + j];
             if (so >= 0) v[q] = __ldg(s_n + so);
@@ -89,6 +94,7 @@ __global__ void __launch_bounds__(IC_THREADS) im2col_kernel(Im2colArgs a, int rc
 }
 
 // General fallback (rows longer than the offset table, or tensors beyond 2^31 chunks): one thread per chunk.
+template <typename V>
 __global__ void __launch_bounds__(IC_THREADS) im2col_generic_kernel(Im2colArgs a, int row_chunks, long long code_chunks, long long n_scales) {
   const Geom& g = a.g;
   const long long stride = (long long)gridDim.x * IC_THREADS;
@@ -103,9 +109,10 @@ __global__ void __launch_bounds__(IC_THREADS) im2col_generic_kernel(Im2colArgs a
       const int ho = (int)(q / g.Wo);
       const int kh = tap / g.Kw, kw = tap - kh * g.Kw;
       const int h = ho * g.sh + kh - g.ph, w = wo * g.sw + kw - g.pw;
-      uint4 v = make_uint4(0, 0, 0, 0);
-      if (h >= 0 && h < g.H && w >= 0 && w < g.W) v = __ldg(reinterpret_cast<const uint4*>(a.codes) + (((long long)h * g.W + w) * g.N + n) * row_chunks + ch);
-      __stcs(reinterpret_cast<uint4*>(a.out_codes) + id, v);
+      V v;
+      zero_chunk(v);
+      if (h >= 0 && h < g.H && w >= 0 && w < g.W) v = __ldg(reinterpret_cast<const V*>(a.codes) + (((long long)h * g.W + w) * g.N + n) * row_chunks + ch);
+      __stcs(reinterpret_cast<V*>(a.out_codes) + id, v);
     } else {
       long long q = id - code_chunks;
       const int Rt = a.line ? g.N : (a.ts16 ? (g.N + 15) / 16 : g.Nt), Cb = a.ts16 ? g.Cp / 16 : g.Ct;
@@ -125,9 +132,10 @@ __global__ void __launch_bounds__(IC_THREADS) im2col_generic_kernel(Im2colArgs a
 
 }  // namespace
 
-cudaError_t launch_im2col(const Im2colArgs& a, cudaStream_t s) {
+template <typename V>
+cudaError_t launch_im2col_v(const Im2colArgs& a, cudaStream_t s) {
   const Geom& g = a.g;
-  const int rc = g.Cp * fmt_bits(a.fmt) / 8 / 16;  // 16-byte chunks per (pixel, sample) row
+  const int rc = g.Cp * fmt_store_bits(a.fmt) / 8 / (int)sizeof(V);  // chunks per (pixel, sample) row
   const int taps = g.Kh * g.Kw;
   const long long J = (long long)taps * rc;
   const long long src_chunks = (long long)g.H * g.W * g.N * rc;
@@ -141,7 +149,7 @@ cudaError_t launch_im2col(const Im2colArgs& a, cudaStream_t s) {
     long long sc_blocks = (n_scales + IC_THREADS - 1) / IC_THREADS;
     if (sc_blocks > sm_count() * 4) sc_blocks = sm_count() * 4;
     if (sc_blocks < 1) sc_blocks = 1;
-    return launch_pdl(im2col_kernel, dim3((unsigned)(n_main + sc_blocks)), dim3(IC_THREADS), 0, s, a, rc, (int)J, PX, (unsigned)n_main);
+    return launch_pdl(im2col_kernel<V>, dim3((unsigned)(n_main + sc_blocks)), dim3(IC_THREADS), 0, s, a, rc, (int)J, PX, (unsigned)n_main);
   }
   const long long code_chunks = (long long)g.Ho * g.Wo * g.N * J;
   const long long total = code_chunks + n_scales;
@@ -149,8 +157,13 @@ cudaError_t launch_im2col(const Im2colArgs& a, cudaStream_t s) {
   const long long cap = (long long)sm_count() * 8 * 16;  // grid-stride beyond this
   if (blocks > cap) blocks = cap;
   if (blocks <= 0) return cudaErrorInvalidValue;
-  im2col_generic_kernel<<<(unsigned)blocks, IC_THREADS, 0, s>>>(a, rc, code_chunks, n_scales);
+  im2col_generic_kernel<V><<<(unsigned)blocks, IC_THREADS, 0, s>>>(a, rc, code_chunks, n_scales);
   return cudaGetLastError();
+}
+
+cudaError_t launch_im2col(const Im2colArgs& a, cudaStream_t s) {
+  if ((a.g.Cp * fmt_store_bits(a.fmt) / 8) % 16 != 0) return launch_im2col_v<uint2>(a, s);
+  return launch_im2col_v<uint4>(a, s);
 }
 
 }  // namespace mq

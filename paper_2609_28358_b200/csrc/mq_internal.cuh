@@ -38,6 +38,27 @@ inline Geom make_geom(const mq_conv_desc& d) {
 __host__ __device__ inline int fmt_bits(int fmt) { return fmt == MQ_E2M1 ? 4 : 8; }
 __host__ __device__ inline int fmt_emax(int fmt) { return fmt == MQ_E4M3 ? 8 : (fmt == MQ_E5M2 ? 15 : (fmt == MQ_E3M2 ? 4 : 2)); }
 __host__ __device__ inline bool fmt_is_6bit(int fmt) { return fmt == MQ_E3M2 || fmt == MQ_E2M3; }
+// packed 6-bit storage: the same element formats, 16 codes in 12 bytes
+__host__ __device__ inline bool fmt_is_packed6(int fmt) { return fmt == MQ_E3M2_P6 || fmt == MQ_E2M3_P6; }
+__host__ __device__ inline int fmt_base(int fmt) { return fmt == MQ_E3M2_P6 ? MQ_E3M2 : (fmt == MQ_E2M3_P6 ? MQ_E2M3 : fmt); }
+__host__ __device__ inline int fmt_store_bits(int fmt) { return fmt_is_packed6(fmt) ? 6 : fmt_bits(fmt); }
+// 16 one-byte 6-bit codes (four words) -> the 96-bit field of the packed storage: code k in bits 6k .. 6k+5
+__host__ __device__ inline void pack6x16(const uint32_t w[4], uint32_t out[3]) {
+  uint32_t t[4];
+  for (int i = 0; i < 4; ++i) t[i] = (w[i] & 0x3Fu) | ((w[i] >> 2) & 0xFC0u) | ((w[i] >> 4) & 0x3F000u) | ((w[i] >> 6) & 0xFC0000u);
+  out[0] = t[0] | (t[1] << 24);
+  out[1] = (t[1] >> 8) | (t[2] << 16);
+  out[2] = (t[2] >> 16) | (t[3] << 8);
+}
+// and back: the field's three words -> 16 one-byte codes
+__host__ __device__ inline void unpack6x16(const uint32_t in[3], uint32_t w[4]) {
+  uint32_t t[4];
+  t[0] = in[0] & 0xFFFFFFu;
+  t[1] = ((in[0] >> 24) | (in[1] << 8)) & 0xFFFFFFu;
+  t[2] = ((in[1] >> 16) | (in[2] << 16)) & 0xFFFFFFu;
+  t[3] = in[2] >> 8;
+  for (int i = 0; i < 4; ++i) w[i] = (t[i] & 0x3Fu) | ((t[i] & 0xFC0u) << 2) | ((t[i] & 0x3F000u) << 4) | ((t[i] & 0xFC0000u) << 6);
+}
 // format field of the tcgen05 instruction descriptor (kind::mxf8f6f4)
 __host__ __device__ inline unsigned fmt_mma_code(int fmt) { return fmt == MQ_E4M3 ? 0u : (fmt == MQ_E5M2 ? 1u : (fmt == MQ_E2M3 ? 3u : (fmt == MQ_E3M2 ? 4u : 5u))); }
 
@@ -84,6 +105,7 @@ struct QuantArgs {
   // tensor's statistics buffer (T_scale is written to [0])
   const float* ts_amax;
   float* ts_stats;
+  int packed6;        // 1: 6-bit codes leave packed, 16 codes in 12 bytes (out strides stay in elements)
   int ts_track_max;   // 1: the kernel also collects max|X| into ts_stats[1] (maximum supplied from outside: the tensor is read once)
 };
 // invertible 32-bit mixer (xor-shift, odd multiply, twice, xor-shift) behind the per-element draws

@@ -53,6 +53,20 @@ __device__ __forceinline__ Item item_of(unsigned it, int n_pstrips, int Ct, int 
 // R16 (tensors of at most 16 rows, e.g. a batch of 16 samples; NT = 256): the upper half of the 32-row tile would be
 // padding, so an item takes 16 positions instead - buffer rows 16..31 hold rows 0..15 of the next eight positions - and
 // every amax, scale and slab below is per (half, position).
+// 16 consecutive one-byte codes at element index e (a multiple of 16): stored as they are, or - packed 6-bit storage - as
+// the 12-byte field of their group
+__device__ __forceinline__ void store_codes16(const QuantArgs& a, long long e, const uint4 val) {
+  if (a.packed6) {
+    const uint32_t w[4] = {val.x, val.y, val.z, val.w};
+    uint32_t o[3];
+    pack6x16(w, o);
+    uint32_t* d = reinterpret_cast<uint32_t*>(a.codes + (e >> 4) * 12);
+    d[0] = o[0]; d[1] = o[1]; d[2] = o[2];
+  } else {
+    *reinterpret_cast<uint4*>(a.codes + e) = val;
+  }
+}
+
 template <int FMT, int NT, bool SR, bool R16 = false>   // NT threads per block: 256 (two tile rows per thread) or 512 (one); SR: stochastic rounding
 __global__ void __launch_bounds__(NT) quantize_pipe_kernel(QuantArgs a, int n_pstrips, int Ct, unsigned n_items) {
   constexpr int RI = 512 / NT;      // tile rows per thread
@@ -204,7 +218,7 @@ __global__ void __launch_bounds__(NT) quantize_pipe_kernel(QuantArgs a, int n_ps
         if (q.p0 + p < a.P && q.r0 + r < a.R) {
           const uint4 val = *reinterpret_cast<const uint4*>(stage + id * 16);
           const long long e = (long long)(q.p0 + p) * a.out_stride_p + (long long)(q.r0 + r) * a.out_stride_r + q.c0 + 16 * half;
-          *reinterpret_cast<uint4*>(a.codes + e) = val;
+          store_codes16(a, e, val);
         }
       }
     }
@@ -340,7 +354,7 @@ __global__ void __launch_bounds__(QT_THREADS) quantize_simple_kernel(QuantArgs a
       if (q.p0 + p < a.P && q.r0 + r < a.R) {
         const uint4 val = *reinterpret_cast<const uint4*>(&stage[p][r][16 * half]);
         const long long e = (long long)(q.p0 + p) * a.out_stride_p + (long long)(q.r0 + r) * a.out_stride_r + q.c0 + 16 * half;
-        *reinterpret_cast<uint4*>(a.codes + e) = val;
+        store_codes16(a, e, val);
       }
     }
   }
@@ -562,7 +576,20 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_con
       }
       tc::fence_proxy_async_smem();
       consumer_sync();
-      if (t == 0) {
+      if ((FMT == MQ_E3M2 || FMT == MQ_E2M3) && a.packed6) {
+        // packed 6-bit storage: a row of the tile is 24 bytes, no TMA box - two rows per thread, packed on the way out (the
+        // next item's first barrier orders these reads before the buffer is written again)
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+          const int id = t + TQ_CONSUMERS * k, p = id >> 5, n = id & 31;
+          if (q.p0 + p < a.P && q.r0 + n < a.R) {
+            const uint4* sp = reinterpret_cast<const uint4*>(stage + id * 32);
+            const long long e = (long long)(q.p0 + p) * a.out_stride_p + (long long)(q.r0 + n) * a.out_stride_r + q.c0;
+            store_codes16(a, e, sp[0]);
+            store_codes16(a, e + 16, sp[1]);
+          }
+        }
+      } else if (t == 0) {
         // codes of the tile at 32 positions: box (32 channels, 32 rows, 32 positions), clipped to the tensor
         tc::tma_store_3d(&map_out, stage, q.c0 * (FMT == MQ_E2M1 ? 4 : 8) / 8, q.r0, q.p0);
         tc::bulk_commit_group();
@@ -649,6 +676,17 @@ __global__ void __launch_bounds__(256) quantize_cfast_kernel(QuantArgs a, unsign
         const unsigned mine = lo | (hi << 8);                       // 4 codes; the odd lane's go above the even lane's
         const unsigned other = __shfl_xor_sync(0xffffffffu, mine, 1);
         if ((lane & 1) == 0 && r < a.R) *reinterpret_cast<unsigned*>(a.codes + (e >> 1)) = mine | (other << 16);
+      } else if ((FMT == MQ_E3M2 || FMT == MQ_E2M3) && a.packed6) {
+        // packed 6-bit storage: a lane's four codes are 24 bits; lanes 4j .. 4j+3 hold a 12-byte group, its word k written by
+        // lane 4j + k from its own bits and the next lane's
+        const unsigned w = lo | (hi << 16);
+        const unsigned t24 = (w & 0x3Fu) | ((w >> 2) & 0xFC0u) | ((w >> 4) & 0x3F000u) | ((w >> 6) & 0xFC0000u);
+        const unsigned nxt = __shfl_down_sync(0xffffffffu, t24, 1);
+        const int k = lane & 3;
+        if (k < 3 && r < a.R) {
+          const long long e16 = (e - 4 * k) >> 4;    // the group's index
+          *reinterpret_cast<unsigned*>(a.codes + e16 * 12 + 4 * k) = (t24 >> (8 * k)) | (nxt << (24 - 8 * k));
+        }
       } else {
         if (r < a.R) *reinterpret_cast<unsigned*>(a.codes + e) = lo | (hi << 16);
       }

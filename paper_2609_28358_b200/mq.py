@@ -14,6 +14,7 @@ import torch
 ConvDesc = namedtuple("ConvDesc", "N C_in H W C_out Kh Kw stride_h stride_w pad_h pad_w")
 
 E4M3, E5M2, E2M1, E3M2, E2M3 = 0, 1, 2, 3, 4
+E3M2_P6, E2M3_P6 = 5, 6          # the 6-bit formats in packed storage: 16 codes in 12 bytes instead of one code per byte
 ROLE_X, ROLE_W, ROLE_DY = 0, 1, 2
 NCHW, HWNC = 0, 1
 TILE32, LINE32, TS16 = 0, 1, 2   # 32 x 32 squares (default) / 1 x 32 lines along the channel axis / the paper's own format: 16 x 16

@@ -60,6 +60,20 @@ def test_size_queries_match_oracle(mq, desc):
             with pytest.raises(mq.MqError) as e:
                 mq.workspace_size(desc, op, fmt, fmt, mq.LINE32)
             assert e.value.status == 2
+    # packed 6-bit storage: three quarters of the one-code-per-byte tensor, the same scales; never less scratch
+    for fmt, pf in ((mq.E3M2, mq.E3M2_P6), (mq.E2M3, mq.E2M3_P6)):
+        for role in (mq.ROLE_X, mq.ROLE_W, mq.ROLE_DY):
+            cb, sb = mq.qtensor_sizes(desc, role, fmt)
+            assert mq.qtensor_sizes(desc, role, pf) == (cb * 3 // 4, sb)
+        cb, sb = mq.im2col_sizes(desc, fmt)
+        assert mq.im2col_sizes(desc, pf) == (cb * 3 // 4, sb)
+        for op in (mq.OP_FWD, mq.OP_BWD_DATA, mq.OP_BWD_WEIGHT):
+            assert mq.workspace_size(desc, op, pf, pf) >= mq.workspace_size(desc, op, fmt, fmt)
+            assert mq.workspace_size(desc, op, pf, mq.E4M3 if op != mq.OP_BWD_DATA else mq.E5M2) >= 0
+        for op in (mq.OP_FWD, mq.OP_BWD_DATA):             # the quantizing epilogue does not take it
+            with pytest.raises(mq.MqError) as e:
+                mq.conv_mx_workspace_size(desc, op, pf, mq.E4M3)
+            assert e.value.status == 2
 
 
 def test_bad_arguments_are_rejected_on_the_host(mq):

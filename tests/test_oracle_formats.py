@@ -194,3 +194,26 @@ def test_paper_format_arithmetic():
     # storing the quantized im2col-expanded tensor instead costs Kh*Kw times more (stride 1, same-size output)
     icb, isb = oracle.im2col_sizes(d, E2M1, (8, 8))
     assert icb / cb == gold["act_quantizations_im2col_k3"] and isb / sb == gold["act_quantizations_im2col_k3"]
+
+
+def test_packed_6bit_storage_layout():
+    """pack6: code k of the array in bits 6k .. 6k+5 of one little-endian bit stream (16 codes in 12 bytes).  Checked against
+    the same definition written with Python's unbounded integers, on explicit vectors and on random codes, and inverted by
+    unpack6."""
+    assert oracle.pack6(np.array([1, 0, 0, 0], dtype=np.uint8)).tolist() == [0x01, 0x00, 0x00]
+    assert oracle.pack6(np.array([0, 1, 0, 0], dtype=np.uint8)).tolist() == [0x40, 0x00, 0x00]      # bit 6
+    assert oracle.pack6(np.array([0, 0, 1, 0], dtype=np.uint8)).tolist() == [0x00, 0x10, 0x00]      # bit 12
+    assert oracle.pack6(np.array([0, 0, 0, 63], dtype=np.uint8)).tolist() == [0x00, 0x00, 0xFC]     # bits 18 .. 23
+    assert oracle.pack6(np.array([63, 63, 63, 63], dtype=np.uint8)).tolist() == [0xFF, 0xFF, 0xFF]
+    rng = np.random.default_rng(5)
+    codes = rng.integers(0, 64, size=16 * 37, dtype=np.uint8)
+    stream = 0
+    for k, c in enumerate(codes.tolist()):
+        stream |= c << (6 * k)
+    want = np.frombuffer(stream.to_bytes(codes.size * 3 // 4, "little"), dtype=np.uint8)
+    got = oracle.pack6(codes)
+    assert got.size == codes.size * 3 // 4 and np.array_equal(got, want)
+    assert np.array_equal(oracle.unpack6(got), codes)
+    # a group of 16 codes is a 12-byte field of its own: packing commutes with any regrouping by 16
+    perm = rng.permutation(37)
+    assert np.array_equal(oracle.pack6(codes.reshape(37, 16)[perm]), got.reshape(37, 12)[perm].reshape(-1))
