@@ -365,6 +365,7 @@ mq_status run_conv_tc(int op, const Geom& g, ConvTcPlan& pl, const mq_qtensor* q
   p.out = out; p.out_layout = layout; p.status = status;
 
   CUtensorMap map_a, map_w;
+  bool direct_x = false;
   {
     const uint64_t rb = (uint64_t)pl.rowbytes;
     const uint64_t dims[4] = {rb, (uint64_t)p.Ws, (uint64_t)g.N, (uint64_t)p.Hs};
@@ -373,7 +374,15 @@ mq_status run_conv_tc(int op, const Geom& g, ConvTcPlan& pl, const mq_qtensor* q
     uint32_t box[4] = {(uint32_t)p.KB, (uint32_t)((p.TW - 1) * wst + 1), (uint32_t)p.TN, 1u};
     if (p.halo) { box[1] = (uint32_t)p.WH; box[3] = (uint32_t)g.Kh; }   // the whole halo of a tile in one box
     const uint32_t es[4] = {1u, wst, 1u, 1u};
-    if (!encode_tensor_map_u8(&map_a, a_codes, 4, dims, strides, box, es, p.KB)) return MQ_ERR_CUDA;
+    // a packed activation / gradient tensor with rows of whole 128-code boxes is read where it is stored (the copy engine pads
+    // each 12-byte group on its way into shared memory): no scratch copy, no pass over the tensor before the GEMM
+    if (pk_x && p.KB == 128 && rb % 128 == 0 && !env_int("MQ_TC_NO_P6_DIRECT", 0)) {
+      const uint64_t ps[3] = {strides[0] * 3 / 4, strides[1] * 3 / 4, strides[2] * 3 / 4};
+      direct_x = encode_tensor_map_p6(&map_a, x_stored, 4, dims, ps, box, es);
+    }
+    if (!direct_x && !encode_tensor_map_u8(&map_a, a_codes, 4, dims, strides, box, es, p.KB)) return MQ_ERR_CUDA;
+    p.a_tx34 = direct_x ? 1 : 0;
+    if (direct_x && p.halo) p.halo_box_bytes = p.halo_box_bytes * 3 / 4;
   }
   map_w = map_a;
   if (p.halo) {
@@ -418,7 +427,7 @@ mq_status run_conv_tc(int op, const Geom& g, ConvTcPlan& pl, const mq_qtensor* q
   }
   // ---- launches
   if (separate_transpose && launch_weight_transpose(w_stored, qw->scales, base, wt_scales, g, fw, stream) != cudaSuccess) return MQ_ERR_CUDA;
-  if (fmt_is_6bit(fx)) {
+  if (fmt_is_6bit(fx) && !direct_x) {
     const size_t n = (size_t)p.Hs * p.Ws * g.N * pl.rowbytes;
     if ((pk_x ? launch_unpack6(x_stored, base + pl.off_pack_a, n, 0, fx, stream) : launch_pack6(x_stored, base + pl.off_pack_a, n, stream)) != cudaSuccess) return MQ_ERR_CUDA;
   }

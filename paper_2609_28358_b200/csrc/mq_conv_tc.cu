@@ -737,7 +737,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // stage's barrier with its own byte count.
     {
       uint32_t s = 0, phase = 0, gi = 0;
-      const uint32_t row_bytes = lkind == 1 ? (uint32_t)p.BN * KB : 128u * KB;
+      const uint32_t row_bytes = lkind == 1 ? (uint32_t)p.BN * KB : (p.a_tx34 ? 96u * KB : 128u * KB);
       for (unsigned i = 0, t; (t = tile_of_iter(p, i)) < total && !*abort_flag; ++i) {
         const Tile tile = decode_tile(p, t);
         TapWalk<MODE> tw;
@@ -1679,6 +1679,21 @@ bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const ui
                   l2_promotion_bytes < 0 ? l2promo() : l2_promotion_bytes == 128 ? CU_TENSOR_MAP_L2_PROMOTION_L2_128B : l2_promotion_bytes == 256 ? CU_TENSOR_MAP_L2_PROMOTION_L2_256B
                   : l2_promotion_bytes == 64 ? CU_TENSOR_MAP_L2_PROMOTION_L2_64B : CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
   return r == CUDA_SUCCESS;
+}
+
+// A tiled map over packed 6-bit codes (16 in 12 bytes in global memory; in shared memory each group lands as the 12 bytes +
+// 4 bytes of padding the MMA's 6-bit operand types want): dims, box and coordinates count codes, strides bytes.  The
+// innermost extent must be a multiple of 128 codes, the box 128 codes wide, base 32-byte aligned, strides multiples of 32.
+bool encode_tensor_map_p6(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes, const uint32_t* box,
+                          const uint32_t* elem_strides) {
+  EncodeTiledFn fn = get_encoder();
+  if (!fn || (reinterpret_cast<uintptr_t>(base) & 31u) || dims[0] % 128 != 0 || box[0] != 128) return false;
+  cuuint64_t d[5], st[4];
+  cuuint32_t b[5], es[5];
+  for (int i = 0; i < rank; ++i) { d[i] = dims[i]; b[i] = box[i]; es[i] = elem_strides ? elem_strides[i] : 1; }
+  for (int i = 0; i + 1 < rank; ++i) { st[i] = strides_bytes[i]; if (st[i] % 32 != 0) return false; }
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_16U6_ALIGN16B, (cuuint32_t)rank, const_cast<void*>(base), d, st, b, es, CU_TENSOR_MAP_INTERLEAVE_NONE,
+            CU_TENSOR_MAP_SWIZZLE_128B, l2promo(), CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 size_t conv_tc_smem_bytes(const ConvTcParams& p) {

@@ -52,6 +52,7 @@ struct ConvTcParams {
   // whole-tile-per-stage variant (small channel counts, stride 1): see conv_tc_halo_kernel
   int halo;                 // 1: use it
   int WH;                   // columns of the activation halo box = TW + Kw - 1
+  int a_tx34;               // 1: the activation boxes come from packed 6-bit storage - a box counts 3/4 of its shared-memory bytes on the barrier
   int halo_box_bytes;       // bytes of one activation box = Kh * TN * WH * KB
   int halo_a_bytes;         // bytes of a tile's activation boxes (rounded up to 1024)
   int halo_stage_bytes;     // bytes of one pipeline stage (activation boxes + A-side scale chunks)
@@ -177,5 +178,9 @@ cudaError_t launch_bwd_weight_reduce(const float* partial, float* out, const Geo
 // or -1 for the library's default.
 bool encode_tensor_map_u8(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes,
                           const uint32_t* box, const uint32_t* elem_strides, int swizzle_bytes, bool f32 = false, int l2_promotion_bytes = -1);
+
+// The same over a tensor in packed 6-bit storage, 128-byte swizzle: dims, box and coordinates count codes (box[0] = 128).
+bool encode_tensor_map_p6(CUtensorMap* map, const void* base, int rank, const uint64_t* dims, const uint64_t* strides_bytes, const uint32_t* box,
+                          const uint32_t* elem_strides);
 
 }  // namespace mq

@@ -577,16 +577,27 @@ quantize_tma_kernel(const __grid_constant__ CUtensorMap map_in, const __grid_con
       tc::fence_proxy_async_smem();
       consumer_sync();
       if ((FMT == MQ_E3M2 || FMT == MQ_E2M3) && a.packed6) {
-        // packed 6-bit storage: a row of the tile is 24 bytes, no TMA box - two rows per thread, packed on the way out (the
-        // next item's first barrier orders these reads before the buffer is written again)
+        // packed 6-bit storage: a row of the tile is 24 bytes - no TMA box.  Each thread packs two rows in place (32 -> 24
+        // bytes of their slot), then the rows leave as 8-byte pieces, three neighbouring lanes per row, so that a row is one
+        // request (the next item's first barrier orders these reads before the buffer is written again)
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
-          const int id = t + TQ_CONSUMERS * k, p = id >> 5, n = id & 31;
+          uint4* sp = reinterpret_cast<uint4*>(stage + (t + TQ_CONSUMERS * k) * 32);
+          const uint4 v0 = sp[0], v1 = sp[1];
+          const uint32_t w0[4] = {v0.x, v0.y, v0.z, v0.w}, w1[4] = {v1.x, v1.y, v1.z, v1.w};
+          uint32_t o0[3], o1[3];
+          pack6x16(w0, o0);
+          pack6x16(w1, o1);
+          sp[0] = make_uint4(o0[0], o0[1], o0[2], o1[0]);
+          *reinterpret_cast<uint2*>(sp + 1) = make_uint2(o1[1], o1[2]);
+        }
+        consumer_sync();
+#pragma unroll
+        for (int k = 0; k < 6; ++k) {
+          const int id = t + TQ_CONSUMERS * k, row = id / 3, piece = id - 3 * row, p = row >> 5, n = row & 31;
           if (q.p0 + p < a.P && q.r0 + n < a.R) {
-            const uint4* sp = reinterpret_cast<const uint4*>(stage + id * 32);
             const long long e = (long long)(q.p0 + p) * a.out_stride_p + (long long)(q.r0 + n) * a.out_stride_r + q.c0;
-            store_codes16(a, e, sp[0]);
-            store_codes16(a, e + 16, sp[1]);
+            *reinterpret_cast<uint2*>(a.codes + (e >> 4) * 12 + 8 * piece) = *reinterpret_cast<const uint2*>(stage + row * 32 + 8 * piece);
           }
         }
       } else if (t == 0) {
