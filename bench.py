@@ -38,8 +38,9 @@ MORE_WORKLOADS = ("cfg5_e2m1_k3s1_c512_hw56", "cfg5_e2m1_k3s1_c512_hw56+ts16", "
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0}
 # published dense figures (NVIDIA's B200 / HGX B200 data sheet, per GPU, without sparsity): context beside the measured roofs
 PUBLISHED = {"hbm_gbs": 7700.0, "tensor_tflops": {8: 4500.0, 4: 9000.0}}
-FMT_NAME = {0: "e4m3", 1: "e5m2", 2: "e2m1", 3: "e3m2", 4: "e2m3"}
-FMT_BITS = {0: 8, 1: 8, 2: 4, 3: 8, 4: 8}   # stored bits per code (the 6-bit formats sit one per byte and run at the 8-bit tensor rate)
+FMT_NAME = {0: "e4m3", 1: "e5m2", 2: "e2m1", 3: "e3m2", 4: "e2m3", 5: "e3m2_p6", 6: "e2m3_p6"}
+FMT_BITS = {0: 8, 1: 8, 2: 4, 3: 8, 4: 8, 5: 8, 6: 8}   # tensor-core rate class of a code (the 6-bit formats run at the 8-bit rate, one per byte or packed)
+PACKED6 = {3: 5, 4: 6}                       # name + "+p6": the layer's 6-bit tensors in packed storage (16 codes in 12 bytes)
 # nominal dense tensor-core ratio to bf16 for the operand formats of a GEMM
 TENSOR_RATIO = {8: 2.0, 4: 4.0}
 CALLS = ("quantize_x", "quantize_w", "quantize_dy", "cbf_im2col", "conv_fwd", "conv_bwd_data", "conv_bwd_weight")
@@ -58,11 +59,13 @@ NCU_TRAFFIC = {
 
 
 class _WorkloadTable(dict):
-    """name -> layer; a "+ts16" suffix selects the number format, not the layer"""
+    """name -> layer; a "+ts16" / "+p6" suffix selects the number format / the storage, not the layer"""
 
     def __missing__(self, name):
         if name.endswith("+ts16") and name[:-5] in self:
             return self[name[:-5]]
+        if name.endswith("+p6") and name[:-3] in self:
+            return self[name[:-3]]
         raise KeyError(name)
 
 
@@ -152,7 +155,7 @@ class Workload:
 
         self.name, self.layer = name, layer
         d = self.d = layer.desc
-        self.fmts = fmts = (layer.fmt_x, layer.fmt_w, layer.fmt_dy)
+        self.fmts = fmts = tuple(PACKED6.get(f, f) if name.endswith("+p6") else f for f in (layer.fmt_x, layer.fmt_w, layer.fmt_dy))
         blk = self.block = mq.TS16 if name.endswith("+ts16") else mq.TILE32
         assert blk == mq.TILE32 or all(f == mq.E2M1 for f in fmts), "the paper's own format has E2M1 elements"
         roles = (mq.ROLE_X, mq.ROLE_W, mq.ROLE_DY)
@@ -448,7 +451,7 @@ def run_ours(args):
 
     # ---- the two GEMMs with the quantizing producer epilogue (the next tensor leaves the chip in its stored MX form instead of
     # fp32): per-call times beside the fp32-output calls and the quantizer call they replace
-    if world == 1:
+    if world == 1 and not any(f in PACKED6.values() for f in fmts):   # (the quantizing epilogue does not emit packed 6-bit storage)
         out["fused_epilogue"] = fused_epilogue_times(wl, flush, max(3, min(K, 10)), kern, pk)
 
     # ---- the same step on further workloads (device-timed step and per-call roofline only)

@@ -32,9 +32,11 @@
  *   for them.  Layouts as above; a group of 16 consecutive channels occupies 12 bytes, code k of the group in bits
  *   6k .. 6k+5 of that 96-bit little-endian field (so a row of Cp channels takes 3 Cp / 4 bytes, and the tensor 3/4 of
  *   the bytes of MQ_E3M2 / MQ_E2M3, which store one code per byte).  Scales are unchanged.  mq_qtensor_sizes,
- *   mq_im2col_sizes, mq_workspace_size, mq_quantize, mq_quantize_sr, mq_cbf_im2col and the three mq_conv_* GEMMs accept
- *   them and give the results of the one-code-per-byte format bit for bit; the quantizing producer epilogues,
- *   mq_conv_bwd_data_static and mq_conv_layer_host return MQ_ERR_UNSUPPORTED for them.
+ *   mq_im2col_sizes, mq_workspace_size, mq_quantize, mq_quantize_sr, mq_cbf_im2col, the three mq_conv_* GEMMs,
+ *   mq_conv_bwd_data_static and mq_conv_layer_host accept them and give the results of the one-code-per-byte format bit
+ *   for bit; the quantizing producer epilogues (mq_conv_*_mx) return MQ_ERR_UNSUPPORTED for them.  Activation and
+ *   gradient tensors whose padded channel count is a multiple of 128 are read by the tensor-core GEMMs where they
+ *   are stored; other operands pass through a copy in the call's scratch.
  *
  * Line blocks (MQ_BLOCK_LINE32): the one-directional block of Sec. III-A (Eq. 5-6) - 32 consecutive channels of ONE
  *   row (sample / output channel) share the scale, amax over those 32 elements.  Codes are laid out as above; scales

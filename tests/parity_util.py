@@ -151,7 +151,7 @@ def _pick_blocks(nblocks, want, rng):
     return sorted({0, nblocks - 1, *map(int, mid)})
 
 
-def check_large_layer(layer, samples=3000, dw_mac_budget=3e10, seed=0, block=None):
+def check_large_layer(layer, samples=3000, dw_mac_budget=3e10, seed=0, block=None, packed6=False):
     """Parity of a layer too large for the oracle to process whole.  The GPU runs the whole layer at full size; the
     oracle checks it on pieces that are independent of the rest of the tensor:
       * the first and the last 32-sample slab (tiles never span slabs; Y and G_X of a sample depend on that sample
@@ -164,10 +164,15 @@ def check_large_layer(layer, samples=3000, dw_mac_budget=3e10, seed=0, block=Non
       * W in full.
     block=mq.TS16: the paper's own format (E2M1 elements whatever the layer names).  Its blocks are 16 x 16, so the same
     pieces are independent once the oracle is given the whole tensor's maximum (Eq. 4), which is computed here with numpy
-    and also compared with what the GPU's first pass found."""
+    and also compared with what the GPU's first pass found.
+    packed6: the GPU keeps the layer's 6-bit tensors in packed storage (16 codes in 12 bytes); the oracle's one-code-per-byte
+    pieces are packed (oracle.pack6) before the comparison - every piece is whole 32-channel rows, hence whole groups."""
     d = layer.desc
     ts = block == mq.TS16
     fx, fw, fg = (mq.E2M1,) * 3 if ts else (layer.fmt_x, layer.fmt_w, layer.fmt_dy)
+    P6 = {mq.E3M2: mq.E3M2_P6, mq.E2M3: mq.E2M3_P6}
+    gx, gw, gg = [P6.get(f, f) if packed6 else f for f in (fx, fw, fg)]        # the GPU's storage of each tensor
+    enc = lambda f, c: oracle.pack6(c) if f in P6.values() else c
     bs = 16 if ts else 32                       # side of a scale block
     name = layer.name + (" (paper's format)" if ts else "")
     rng = np.random.default_rng(seed)
@@ -175,7 +180,7 @@ def check_large_layer(layer, samples=3000, dw_mac_budget=3e10, seed=0, block=Non
     ho, wo = inputs.out_hw(d)
     N, Nt = d.N, (d.N + bs - 1) // bs
     cp, cop = (d.C_in + 31) // 32 * 32, (d.C_out + 31) // 32 * 32
-    bpe = lambda f: 0.5 if f == mq.E2M1 else 1.0
+    bpe = lambda f: 0.5 if f == mq.E2M1 else (0.75 if f in P6.values() else 1.0)
     OR = (oracle.ROLE_X, oracle.ROLE_W, oracle.ROLE_DY)
     amax = [float(np.abs(t).max()) for t in (x, w, g)] if ts else None
 
@@ -194,21 +199,21 @@ def check_large_layer(layer, samples=3000, dw_mac_budget=3e10, seed=0, block=Non
             st = host(q.tensor_scale)
             assert st[1] == np.float32(a) and st[0] == np.float32(a) / (np.float32(448.0) * np.float32(6.0)), (name, st, a)
     else:
-        xq, wq, gq = [mq.quantize(d, r, f, dev(t)) for r, f, t in zip(ROLES, (fx, fw, fg), (x, w, g))]
+        xq, wq, gq = [mq.quantize(d, r, f, dev(t)) for r, f, t in zip(ROLES, (gx, gw, gg), (x, w, g))]
     wc, wsc, wt = oq(d, 1, fw, w)
     assert_same_bytes(wq.scales, wsc, f"{name} W scales")
-    assert_same_bytes(wq.codes, wc, f"{name} W codes")
+    assert_same_bytes(wq.codes, enc(gw, wc), f"{name} W codes")
     wh = odq(d, 1, fw, wc, wsc, wt)
     ic, isc = mq.cbf_im2col(d, xq)
     y = mq.conv_fwd(d, xq, wq)
     dx = mq.conv_bwd_data(d, wq, gq)
     dw = mq.conv_bwd_weight(d, xq, gq)
     P, Po, taps = d.H * d.W, ho * wo, d.Kh * d.Kw
-    xcodes = xq.codes.view(P, N, int(cp * bpe(fx)))
-    gcodes = gq.codes.view(Po, N, int(cop * bpe(fg)))
+    xcodes = xq.codes.view(P, N, int(cp * bpe(gx)))
+    gcodes = gq.codes.view(Po, N, int(cop * bpe(gg)))
     xscales = xq.scales.view(P, Nt, cp // bs)
     gscales = gq.scales.view(Po, Nt, cop // bs)
-    icodes = ic.view(Po, N, int(taps * cp * bpe(fx)))
+    icodes = ic.view(Po, N, int(taps * cp * bpe(gx)))
     iscales = isc.view(Po, Nt, taps * (cp // bs))
     worst = {}
     for slab in sorted({0, (N + 31) // 32 - 1}):
@@ -218,12 +223,12 @@ def check_large_layer(layer, samples=3000, dw_mac_budget=3e10, seed=0, block=Non
         xc, xsc, xt = oq(ds, 0, fx, x[n0:n1])
         gc, gsc, gt = oq(ds, 2, fg, g[n0:n1])
         assert_same_bytes(xscales[:, b0:b1].contiguous(), xsc, f"{name} X scales, samples {n0}..{n1}")
-        assert_same_bytes(xcodes[:, n0:n1].contiguous(), xc, f"{name} X codes, samples {n0}..{n1}")
+        assert_same_bytes(xcodes[:, n0:n1].contiguous(), enc(gx, xc), f"{name} X codes, samples {n0}..{n1}")
         assert_same_bytes(gscales[:, b0:b1].contiguous(), gsc, f"{name} dY scales, samples {n0}..{n1}")
-        assert_same_bytes(gcodes[:, n0:n1].contiguous(), gc, f"{name} dY codes, samples {n0}..{n1}")
+        assert_same_bytes(gcodes[:, n0:n1].contiguous(), enc(gg, gc), f"{name} dY codes, samples {n0}..{n1}")
         oc, osc = oracle.cbf_im2col(ds, fx, xc, xsc, (16, 16)) if ts else oracle.cbf_im2col(ds, fx, xc, xsc)
         assert_same_bytes(iscales[:, b0:b1].contiguous(), osc, f"{name} im2col scales, samples {n0}..{n1}")
-        assert_same_bytes(icodes[:, n0:n1].contiguous(), oc, f"{name} im2col codes, samples {n0}..{n1}")
+        assert_same_bytes(icodes[:, n0:n1].contiguous(), enc(gx, oc), f"{name} im2col codes, samples {n0}..{n1}")
         del oc, osc
         xh = odq(ds, 0, fx, xc, xsc, xt)
         gh = odq(ds, 2, fg, gc, gsc, gt)
@@ -253,13 +258,13 @@ def check_large_layer(layer, samples=3000, dw_mac_budget=3e10, seed=0, block=Non
     xc, xsc, xt = oq(dsel, 0, fx, xs)
     gc, gsc, gt = oq(dsel, 2, fg, gs)
     del xs, gs
-    bx, bg = int(32 * bpe(fx)), int(32 * bpe(fg))
+    bx, bg = int(32 * bpe(gx)), int(32 * bpe(gg))
     tb = lambda blocks: torch.as_tensor(blocks, device="cuda")
     sb = lambda blocks: tb([(32 // bs) * b + k for b in blocks for k in range(32 // bs)])      # scale columns of 32-channel blocks
     assert_same_bytes(xscales[:, :, sb(bi)].contiguous(), xsc, f"{name} X scales, channel blocks {bi}")
-    assert_same_bytes(xcodes.view(P, N, cp // 32, bx)[:, :, tb(bi)].contiguous(), xc, f"{name} X codes, channel blocks {bi}")
+    assert_same_bytes(xcodes.view(P, N, cp // 32, bx)[:, :, tb(bi)].contiguous(), enc(gx, xc), f"{name} X codes, channel blocks {bi}")
     assert_same_bytes(gscales[:, :, sb(bo)].contiguous(), gsc, f"{name} dY scales, channel blocks {bo}")
-    assert_same_bytes(gcodes.view(Po, N, cop // 32, bg)[:, :, tb(bo)].contiguous(), gc, f"{name} dY codes, channel blocks {bo}")
+    assert_same_bytes(gcodes.view(Po, N, cop // 32, bg)[:, :, tb(bo)].contiguous(), enc(gg, gc), f"{name} dY codes, channel blocks {bo}")
     xh = odq(dsel, 0, fx, xc, xsc, xt)
     gh = odq(dsel, 2, fg, gc, gsc, gt)
     got = host(dw[tb(co)][:, tb(ci)].contiguous()).reshape(-1)

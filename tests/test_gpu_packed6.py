@@ -87,6 +87,27 @@ def test_gemms_match_the_one_code_per_byte_tensors(name, shape, fmts):
     assert mq.last_device_status() == 0
 
 
+def test_cuda_core_routes_and_static_scratch(knobs):
+    """Layers the tensor-core kernels do not take (forced here) read one-byte copies of packed operands from the call's scratch;
+    the call on the library's static scratch accepts packed tensors like the ordinary one."""
+    d = inputs.conv_desc(40, 48, 6, 6, 70, 3, 1, 1)
+    src = (inputs.make_x(d, 94, "relu"), inputs.make_w(d, 94), inputs.make_dy(d, 94, "gauss"))
+    fmts = (mq.E3M2, mq.E2M3, mq.E2M3)
+    qu = [mq.quantize(d, r, f, dev(t)) for r, f, t in zip(ROLES, fmts, src)]
+    qp = [mq.quantize(d, r, PACKED[f], dev(t)) for r, f, t in zip(ROLES, fmts, src)]
+    assert torch.equal(mq.conv_bwd_data_static(d, qp[1], qp[2]), mq.conv_bwd_data(d, qu[1], qu[2]))
+    knobs(MQ_TC_NO_FP6=1)
+    for what, fn, a, b in (("fwd", mq.conv_fwd, 0, 1), ("bwd_data", mq.conv_bwd_data, 1, 2), ("bwd_weight", mq.conv_bwd_weight, 0, 2)):
+        n0 = mq.kernel_launch_count()
+        want = fn(d, qu[a], qu[b])
+        n1 = mq.kernel_launch_count()
+        got = fn(d, qp[a], qp[b])
+        n2 = mq.kernel_launch_count()
+        assert torch.equal(got, want), (what, float((got - want).abs().max()))
+        assert n2 - n1 == n1 - n0 + 2, (what, n1 - n0, n2 - n1)     # the two one-byte copies
+    assert mq.last_device_status() == 0
+
+
 def test_calls_that_do_not_take_packed_storage():
     d = inputs.conv_desc(32, 64, 6, 6, 64, 3, 1, 1)
     x, w = dev(inputs.make_x(d, 93, "relu")), dev(inputs.make_w(d, 93))

@@ -180,14 +180,15 @@ def test_config5_large_points_full_size(name):
     check_large_layer(layer)
 
 
+@pytest.mark.parametrize("packed6", [False, True], ids=["one-per-byte", "packed"])
 @pytest.mark.parametrize("idx", [0, 1], ids=["e3m2-act", "e2m3"])
-def test_fp6_layers_full_size(idx):
-    """The two 6-bit layers the benchmark reports (256 channels, 28x28, N = 256)."""
-    check_large_layer(inputs.fp6_layers()[idx])
+def test_fp6_layers_full_size(idx, packed6):
+    """The two 6-bit layers the benchmark reports (256 channels, 28x28, N = 256), in both storages of the 6-bit codes."""
+    check_large_layer(inputs.fp6_layers()[idx], packed6=packed6)
 
 
 @pytest.mark.parametrize("slabs", [8, 1, 3], ids=["slabs8", "one_slab", "slabs3"])
-@pytest.mark.parametrize("fmts", [(E4M3, E4M3, E5M2), (E2M1, E2M1, E2M1)], ids=["fp8", "fp4"])
+@pytest.mark.parametrize("fmts", [(E4M3, E4M3, E5M2), (E2M1, E2M1, E2M1), (mq.E3M2_P6, E4M3, mq.E2M3_P6)], ids=["fp8", "fp4", "fp6-packed"])
 def test_layer_from_host_buffers_matches_the_device_calls(fmts, slabs, knobs):
     """mq_conv_layer_host (pinned host tensors in, host results out, copies overlapped with the kernels, the step run slab by
     slab along the batch) gives, twice in a row, exactly the Y and G_X of the separate device-side calls; G_W is the sum of
@@ -210,6 +211,7 @@ def test_layer_from_host_buffers_matches_the_device_calls(fmts, slabs, knobs):
             if name != "dW" or slabs == 1:
                 assert torch.equal(got, exp), f"{name} from host buffers differs from the device call"
     if slabs != 1:
+        fmts = tuple({mq.E3M2_P6: E3M2, mq.E2M3_P6: E2M3}.get(f, f) for f in fmts)   # (packed storage: the same codes)
         oq = [oracle.quantize(d, r, f, t) for r, f, t in zip((oracle.ROLE_X, oracle.ROLE_W, oracle.ROLE_DY), fmts, (x, w, g))]
         xh, gh = oracle.dequant(d, oracle.ROLE_X, fmts[0], *oq[0]), oracle.dequant(d, oracle.ROLE_DY, fmts[2], *oq[2])
         ref, ab = oracle.conv_bwd_weight(d, gh, xh)
