@@ -542,7 +542,11 @@ WgradPlan wgrad_plan(const Geom& g, int fmt_x, int fmt_g, bool ts16 = false) {
   w.P_b = (w.P_a + (g.Kh - 1) * p.Wp + g.Kw - 1 + 7) / 8 * 8;
   size_t o = up256((size_t)splits * g.Cout * g.Kh * g.Kw * g.Cp * sizeof(float));
   w.off_sfa = o; o += up256((size_t)p.m_tiles128 * p.stages_total * 512 * spa);
-  w.off_sfb = o; o += up256(fp8 ? (size_t)p.cb_tiles * p.Hp * p.Wp * p.nchunks * p.NB * 512 : (size_t)p.cb_tiles * (g.Kh * g.Kw / p.TG) * p.stages_total * p.NB * 512 * spa);
+  // flat mode with whole 128-channel tap panels: the X-side scale chunks once per padded start pixel (Kh Kw / KPX times fewer)
+  p.sfb_S = (flat && p.b_rows == 128 && !env_int("MQ_WGRAD_NO_SFB_DEDUP", 0)) ? w.P_b : 0;
+  w.off_sfb = o; o += up256(fp8 ? (size_t)p.cb_tiles * p.Hp * p.Wp * p.nchunks * p.NB * 512
+                                : p.sfb_S > 0 ? ((size_t)p.cb_tiles * p.sfb_S + p.NB) * 512 * spa
+                                              : (size_t)p.cb_tiles * (g.Kh * g.Kw / p.TG) * p.stages_total * p.NB * 512 * spa);
   w.off_xt = o;
   if (flat) { p.xt_block_bytes = (long long)w.P_b * p.b_rows * p.KBn; o += up256((size_t)p.cb_tiles * p.xt_block_bytes); }
   else if (fp4) o += up256((size_t)g.Cp * g.H * g.W * w.Npad / 2);

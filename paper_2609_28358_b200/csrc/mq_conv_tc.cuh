@@ -137,6 +137,9 @@ struct WgradTcParams {
   int mma_cp;           // E2M1: 1 = the MMA lane issues the scale copies itself (no copier warp)
   int cta2;             // 1: pairs of blocks (clusters of 2) compute 256 x 256 tiles with cta_group::2 MMAs
   int TG;               // taps per block: 1, or Kw (flat mode: the taps of a kernel row share the stage's pixels)
+  int sfb_S;            // flat E2M1 mode, 128 input channels per tap panel: > 0 = the X-side scale chunks are stored once per padded
+                        // START pixel (sfb_S of them per channel block; tap (kh, kw) of stage st reads chunk st KPX + kh Wp + kw), not
+                        // once per (tap group, stage, tap)
   int grp8;             // 8-bit operands, 32 or 64 bytes of input channels, unit strides: the Kw taps of a kernel row are one wide B operand
                         // (TG = Kw, b_rows = Cp) whose panels are views of one loaded strip of KPX + Kw - 1 pixels, one pixel apart
   int NB;               // 128-row chunks of the group's B rows = ceil(TG * b_rows / 128)

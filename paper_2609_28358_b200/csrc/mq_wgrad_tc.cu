@@ -51,7 +51,7 @@ __device__ __forceinline__ void expand_wgrad_scales_nv_body(const WgradTcParams&
   const int taps = p.Kh * p.Kw;
   const long long nA = (long long)p.m_tiles128 * p.stages_total;
   const int groups = taps / p.TG;
-  const long long nB = (long long)p.cb_tiles * groups * p.stages_total * p.NB;
+  const long long nB = p.sfb_S > 0 ? (long long)p.cb_tiles * p.sfb_S : (long long)p.cb_tiles * groups * p.stages_total * p.NB;
   if (wid >= nA + nB) return;
   const int Nt16 = (p.N + 15) >> 4, Cot16 = p.Cot * 2, Ct16 = p.Ct * 2;
   // A chunk holds 16 K-blocks x 8 row blocks (16 rows each) = 128 distinct scale bytes: lane (b16, jh) = (lane >> 1, lane & 1)
@@ -59,13 +59,30 @@ __device__ __forceinline__ void expand_wgrad_scales_nv_body(const WgradTcParams&
   // (a lane loading its own 64 bytes, two distinct addresses per warp-wide load, took 2.5 times as long).
   const int b16 = lane >> 1, jh = lane & 1;
   uint32_t mine = 0;
-  uint8_t* dst;
+  uint8_t* dst = nullptr;
   const int st = wid < nA ? (int)(wid % p.stages_total) : (int)(((wid - nA) / p.NB) % p.stages_total);
   int ho, wo, nb;
   stage_block(p, st, b16 >> 1, ho, wo, nb);
   const int nb16 = 2 * nb + (b16 & 1);
   const bool kok = ho < p.Ho && wo < p.Wo && nb16 < Nt16;
-  if (wid < nA) {
+  if (wid >= nA && p.sfb_S > 0) {
+    // chunk of (channel block, padded start pixel s): K-block b is padded pixel s + b / BPP (row-major over the padded image,
+    // running on into the next row: there the G_Y side is zero), sample block b % BPP; 128 channels of one tap panel
+    const long long idx = wid - nA;
+    const int s = (int)(idx % p.sfb_S), cb = (int)(idx / p.sfb_S);
+    const int b = b16 >> 1, px = b / p.BPP;
+    const int lin = s + px, hp = lin / p.Wp, wp = lin - hp * p.Wp;
+    const int h = hp - p.ph, w = wp - p.pw;
+    const int n16 = 2 * (b - px * p.BPP) + (b16 & 1);
+    if (h >= 0 && h < p.H && w >= 0 && w < p.W && n16 < Nt16) {
+#pragma unroll
+      for (int k = 0; k < 4; ++k) {
+        const int cib16 = (cb * p.b_rows + 16 * (4 * jh + k)) >> 4;
+        if (cib16 < Ct16) mine |= (uint32_t)__ldg(p.x_scales + (((long long)h * p.W + w) * Nt16 + n16) * Ct16 + cib16) << (8 * k);
+      }
+    }
+    dst = p.sfb_img + idx * 2048;
+  } else if (wid < nA) {
     const int mt = (int)(wid / p.stages_total);
     if (kok) {
       const uint8_t* line = p.g_scales + (((long long)ho * p.Wo + wo) * Nt16 + nb16) * Cot16;
@@ -128,7 +145,8 @@ __device__ __forceinline__ void expand_wgrad_scales_body(const WgradTcParams& p,
   const int groups = taps / p.TG;
   // B-side chunks: E2M1 modes one per (channel block, tap group, stage); 8-bit mode one per (channel block, padded X
   // pixel, sample chunk) - a stage's chunk depends only on where its taps' pixels start, so the taps share them
-  const long long nB = FP4 ? (long long)p.cb_tiles * groups * p.stages_total * p.NB : (long long)p.cb_tiles * p.Hp * p.Wp * p.nchunks * p.NB;
+  const long long nB = (FP4 && p.sfb_S > 0) ? (long long)p.cb_tiles * p.sfb_S
+                     : FP4 ? (long long)p.cb_tiles * groups * p.stages_total * p.NB : (long long)p.cb_tiles * p.Hp * p.Wp * p.nchunks * p.NB;
   if (wid >= nA + nB) return;
   // this lane's byte: 32-row group j of the 128-row chunk, K-block b of the stage
   const int j = lane >> 3, b = lane & 7;
@@ -159,6 +177,18 @@ __device__ __forceinline__ void expand_wgrad_scales_body(const WgradTcParams& p,
       if (b < NBS && cib < p.Ct && tj < p.TG) {
         const int px = b / p.BPP, nb = nc * p.BPP + (b - px * p.BPP);
         const int h = hp - p.ph, w = wp - p.pw + px * p.sw + tj;
+        if (nb < p.Nt && h >= 0 && h < p.H && w >= 0 && w < p.W) v = __ldg(p.x_scales + (((long long)h * p.W + w) * p.Nt + nb) * p.Ct + cib);
+      }
+    } else if (p.sfb_S > 0) {
+      // chunk of (channel block, padded start pixel s): K-block b is padded pixel s + b / BPP (row-major over the padded
+      // image, running on into the next row: there the G_Y side is zero), sample block b % BPP; 128 channels of one tap panel
+      idx = wid - nA;
+      const int s = (int)(idx % p.sfb_S), cb = (int)(idx / p.sfb_S);
+      const int cib = (cb * p.b_rows + 32 * j) / 32;
+      if (b < NBS && cib < p.Ct) {
+        const int px = b / p.BPP, nb = b - px * p.BPP;
+        const int lin = s + px, hp = lin / p.Wp, wp = lin - hp * p.Wp;
+        const int h = hp - p.ph, w = wp - p.pw;
         if (nb < p.Nt && h >= 0 && h < p.H && w >= 0 && w < p.W) v = __ldg(p.x_scales + (((long long)h * p.W + w) * p.Nt + nb) * p.Ct + cib);
       }
     } else {
@@ -293,7 +323,11 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
     const int taps = p.Kh * p.Kw;
     const uint8_t* sfa_src = p.sfa_img + ((size_t)mt * p.stages_total + st_begin) * (512 * SPA);
     const uint32_t sfb_bytes = (uint32_t)p.NB * 512 * SPA;
-    const uint8_t* sfb_src = p.sfb_img + (((size_t)cb * (taps / TG) + tgi) * p.stages_total + st_begin) * sfb_bytes;
+    // X-side scale chunks: per (tap group, stage), NB chunks each; or (sfb_S) per padded start pixel - the NB taps of the
+    // stage are NB consecutive start pixels, the next stage starts KPX pixels on
+    const uint32_t sfb_step = p.sfb_S > 0 ? (uint32_t)p.KPX * 512 * SPA : sfb_bytes;
+    const uint8_t* sfb_src = p.sfb_S > 0 ? p.sfb_img + ((size_t)cb * p.sfb_S + (size_t)st_begin * p.KPX + (size_t)kh * p.Wp + kw) * (512 * SPA)
+                                         : p.sfb_img + (((size_t)cb * (taps / TG) + tgi) * p.stages_total + st_begin) * sfb_bytes;
     const uint32_t a_bytes = 128 * 128, b_step = (uint32_t)p.b_rows * 128;
     const uint32_t b_bytes = (p.mode == MQ_WG_FP8 && !p.grp8) ? 128u * 128u : (uint32_t)p.b_tile_bytes;   // per loader
     const uint8_t* ga = nullptr; const uint8_t* gb = nullptr;
@@ -336,7 +370,7 @@ wgrad_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant
           }
         } else if (kind == 3) {
           bulk_load(ssf, sfa_src + (size_t)i * (512 * SPA), 512 * SPA, bar);
-          bulk_load(ssf + SFC_BYTES, FP4 ? sfb_src + (size_t)i * sfb_bytes : p.sfb_img + (size_t)xchunk * sfb_bytes, sfb_bytes, bar);
+          bulk_load(ssf + SFC_BYTES, FP4 ? sfb_src + (size_t)i * sfb_step : p.sfb_img + (size_t)xchunk * sfb_bytes, sfb_bytes, bar);
         } else if (p.mode == MQ_WG_FP4_FLAT) {
           if (kind == 0) bulk_load(sa, ga + (size_t)i * a_bytes, a_bytes, bar);
           else bulk_load(sb, gb + (size_t)i * b_step, b_bytes, bar);          // KPX + TG - 1 consecutive pixels
@@ -827,7 +861,8 @@ cudaError_t launch_wgrad_flat_prep(const WgradTcParams& p, const uint8_t* x_code
   FlatArgs fx, fg;
   if (!make_flat_args(&fx, x_codes, xt, p.H, p.W, p.N, p.Cp, P_b, p.Wp, p.ph, p.pw, p.b_rows, p.cb_tiles, p.KBn)) return cudaErrorInvalidValue;
   if (!make_flat_args(&fg, g_codes, gt, p.Ho, p.Wo, p.N, p.Cot * 32, P_a, p.Wp, 0, 0, 128, p.m_tiles, p.KBn)) return cudaErrorInvalidValue;
-  const long long warps = (long long)p.m_tiles128 * p.stages_total + (long long)p.cb_tiles * (p.Kh * p.Kw / p.TG) * p.stages_total * p.NB;
+  const long long warps = (long long)p.m_tiles128 * p.stages_total +
+                          (p.sfb_S > 0 ? (long long)p.cb_tiles * p.sfb_S : (long long)p.cb_tiles * (p.Kh * p.Kw / p.TG) * p.stages_total * p.NB);
   const unsigned sc_blocks = (unsigned)((warps + 7) / 8);
   count_launches(1);
   const size_t smem = (fx.wide || fg.wide) ? (size_t)FLAT_WIDE_SMEM : 0;
