@@ -226,6 +226,76 @@ __device__ __forceinline__ void epilogue_role(const ConvTcParams& p, uint32_t tm
     }
 }
 
+// Epilogue role for 256-column tiles (ONE accumulator: the MMA lane cannot start the next tile before this one has left
+// tensor memory).  Each of the eight warps copies its 32 rows x 128 columns into REGISTERS, hands the accumulator back at
+// once and only then stores - so the stores of a tile (request-bound: 128 KB through 4-byte rows) overlap the next tile's
+// MMAs instead of holding them up.  The registers come from the loader / MMA warpgroups (warpgroup_regs_inc / _dec).
+template <int MODE>
+__device__ __forceinline__ void epilogue_snap_role(const ConvTcParams& p, uint32_t tmem, uint64_t* tfull, uint64_t* tempty, volatile int* abort_flag,
+                                                   int warp, int lane, unsigned total) {
+    const int quad = warp & 3;
+    const int half = (warp - 4) >> 2;
+    const int r = 32 * quad + lane;
+    const int tw_ = r & (p.TW - 1), tn = r >> p.lgTW;
+    const int cbeg = 128 * half;
+    const long long cs = (long long)p.Hd * p.Wd;
+    const float os = out_scale_of(p);
+    uint32_t tcount = 0;
+    for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
+      const Tile tile = decode_tile(p, t);
+      TapWalk<MODE> tw;
+      tw.init(p, tile);
+      const int Q = tw.chunks(p);
+      const int acc = acc_index(p, tcount);
+      bool ok = true;
+      if (lane == 0) ok = mbar_wait(&tfull[acc], acc_phase(p, tcount), p.status, MQ_ERR_TIMEOUT);
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) { *abort_flag = 1; break; }
+      tc_fence_after_sync();
+      uint32_t v[128];
+      if (Q > 0) {
+        const uint32_t taddr = tmem + acc * p.BN + ((uint32_t)(32 * quad) << 16) + cbeg;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) tmem_ld_32x32b_x16(taddr + 16 * k, v + 16 * k);
+        tmem_ld_wait();
+      } else {
+#pragma unroll
+        for (int j = 0; j < 128; ++j) v[j] = 0u;
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty[acc]);      // the accumulator is free: the next tile's MMAs may start
+      int yo, xo;
+      if (MODE == MQ_OP_FWD) { yo = tile.h; xo = tile.w0 + tw_; }
+      else {
+        const int ch = (int)fdiv((unsigned)tile.cls, p.sw, p.m_sw);
+        yo = ch + p.sh * tile.h; xo = tile.cls - ch * p.sw + p.sw * (tile.w0 + tw_);
+      }
+      const int n = tile.n0 + tn;
+      if (!(yo < p.Hd && xo < p.Wd && n < p.N)) continue;
+      const int ncols = min(128, p.Cd - tile.c0 - cbeg);     // columns of this half inside the tensor (may be <= 0)
+      if (p.kind_fp4 == 2) {
+#pragma unroll
+        for (int j = 0; j < 128; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * os);
+      }
+      if (p.out_layout == MQ_NCHW) {
+        float* o = p.out + (((long long)n * p.Cd + tile.c0 + cbeg) * p.Hd + yo) * p.Wd + xo;
+#pragma unroll
+        for (int j = 0; j < 128; ++j) { if (j < ncols) *o = __uint_as_float(v[j]); o += cs; }
+      } else {
+        float* o = p.out + (((long long)yo * p.Wd + xo) * p.N + n) * p.Cd + tile.c0 + cbeg;
+        if (ncols == 128 && (p.Cd & 3) == 0) {
+#pragma unroll
+          for (int j = 0; j < 128; j += 4)
+            *reinterpret_cast<float4*>(o + j) = make_float4(__uint_as_float(v[j]), __uint_as_float(v[j + 1]), __uint_as_float(v[j + 2]), __uint_as_float(v[j + 3]));
+        } else {
+#pragma unroll
+          for (int j = 0; j < 128; ++j) if (j < ncols) o[j] = __uint_as_float(v[j]);
+        }
+      }
+    }
+}
+
 // Epilogue role of the pair mode (see tile_of_iter): both accumulators hold the same output rows and channels for the
 // even and the odd output columns; a thread writes them as float2 (x = 2 (w0 + tw), x + 1), so a warp's store covers
 // 64-byte runs per sample instead of every other float.
@@ -674,6 +744,10 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
 
 // EPI: -1 = fp32 output (the three fp32 epilogue roles, chosen at run time: an instance per role was measured, no
 // change); 0..4 = quantizing epilogue emitting element format EPI
+// registers per thread of the epilogue warpgroups / of the others in the fp32-output kernels (16 warps, 128 per thread at launch)
+constexpr uint32_t EPI_REGS = 168, OTHER_REGS = 88;
+static_assert(2 * (EPI_REGS + OTHER_REGS) * 128 == 512 * 128, "the warpgroups' register budgets must add up to the launch's");
+
 template <int MODE, int KB, int KIND, int EPI = -1>
 __global__ void __launch_bounds__(tc_threads_of(EPI), 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_out,
@@ -728,6 +802,18 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   // loader warps: (kind, parity of the stages it serves)
   const int lkind = (warp == 0 || warp == 12) ? 0 : ((warp == 3 || warp == 13) ? 1 : ((warp == 14 || warp == 15) ? 2 : -1));
   const int lhalf = (warp == 12 || warp == 13 || warp == 15) ? 1 : 0;
+  // The epilogue warps are whole warpgroups (4-7, 8-11; with 24 warps also 16-23), the other roles share groups 0-3 and 12-15.
+  // fp32 output: the epilogue groups take registers from the other two for their copy of a 256-column accumulator
+  // (epilogue_snap_role): (2 x OTHER_REGS + 2 x EPI_REGS) x 128 threads = the 512 x 128 registers of the launch bound.
+  if ((warp >= 4 && warp < 12) || warp >= 16) {
+    if (EPI < 0) warpgroup_regs_inc<EPI_REGS>();
+    if (EPI >= 0) epilogue_mx_role<MODE, EPI < 0 ? 0 : EPI>(p, mx_red, tmem, tfull, tempty, abort_flag, warp, lane, total);
+    else if (p.pair) epilogue_pair_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
+    else if (p.tma_store) epilogue_tma_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total);
+    else if (p.BN == 256 && p.snap) epilogue_snap_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
+    else epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
+  } else {
+  if (EPI < 0) warpgroup_regs_dec<OTHER_REGS>();
   if (lkind >= 0) {
     // ------------------------------------------------------------------ TMA loaders
     // A warp gets one bulk copy accepted per ~170 cycles whatever its size, and the loop around it is a chain of
@@ -902,11 +988,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
         }
       }
     }
-  } else if ((warp >= 4 && warp < 12) || warp >= 16) {
-    if (EPI >= 0) epilogue_mx_role<MODE, EPI < 0 ? 0 : EPI>(p, mx_red, tmem, tfull, tempty, abort_flag, warp, lane, total);
-    else if (p.pair) epilogue_pair_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
-    else if (p.tma_store) epilogue_tma_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total);
-    else epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
+  }
   }
   // teardown: everyone meets here (all loops are bounded), then the allocating warp frees TMEM
   tc_fence_before_sync();

@@ -52,6 +52,7 @@ struct ConvTcParams {
   // whole-tile-per-stage variant (small channel counts, stride 1): see conv_tc_halo_kernel
   int halo;                 // 1: use it
   int WH;                   // columns of the activation halo box = TW + Kw - 1
+  int snap;                 // 1: 256-column tiles, direct fp32 stores: the epilogue copies the accumulator into registers and frees it before storing
   int a_tx34;               // 1: the activation boxes come from packed 6-bit storage - a box counts 3/4 of its shared-memory bytes on the barrier
   int halo_box_bytes;       // bytes of one activation box = Kh * TN * WH * KB
   int halo_a_bytes;         // bytes of a tile's activation boxes (rounded up to 1024)

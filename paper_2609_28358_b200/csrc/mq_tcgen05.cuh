@@ -246,6 +246,11 @@ __device__ __forceinline__ void tmem_ld_32x32b_x16(uint32_t taddr, uint32_t* r) 
       : "r"(taddr)
       : "memory");
 }
+// Register budget of the calling warpgroup (four consecutive warps, all of whose threads must execute it): a group that
+// needs few registers hands some back, another takes them.  The sum over the block's groups must not exceed what the
+// launch allotted (threads x registers per thread of the launch bound), or the increase would wait for ever.
+template <uint32_t R> __device__ __forceinline__ void warpgroup_regs_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(R)); }
+template <uint32_t R> __device__ __forceinline__ void warpgroup_regs_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(R)); }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
 }  // namespace tc
