@@ -742,10 +742,93 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
     if (lane == 0) bulk_wait_group_all();
 }
 
+// The same for 256-column tiles with ONE accumulator: the warp first copies its 32 rows x 128 columns into registers and hands
+// the accumulator back (see epilogue_snap_role), then stages and stores its two 64-channel slices from the registers.
+template <int MODE>
+__device__ __forceinline__ void epilogue_tma_snap_role(const ConvTcParams& p, const CUtensorMap* map_out, float* staging, uint32_t tmem,
+                                                       uint64_t* tfull, uint64_t* tempty, volatile int* abort_flag, int warp, int lane, unsigned total) {
+    const int quad = warp & 3;
+    const int half = (warp - 4) >> 2;
+    const int cbeg = 128 * half;
+    float* buf = staging + (warp - 4) * (64 * 32);
+    const int n_off = quad * (32 >> p.lgTW);
+    const bool hwnc = p.out_layout == MQ_HWNC;
+    const int hrow = lane;
+    const float os = out_scale_of(p);
+    uint32_t tcount = 0;
+    for (unsigned t = blockIdx.x; t < total && !*abort_flag; t += gridDim.x, ++tcount) {
+      const Tile tile = decode_tile(p, t);
+      TapWalk<MODE> tw;
+      tw.init(p, tile);
+      const int Q = tw.chunks(p);
+      const int acc = acc_index(p, tcount);
+      bool ok = true;
+      if (lane == 0) ok = mbar_wait(&tfull[acc], acc_phase(p, tcount), p.status, MQ_ERR_TIMEOUT);
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) { *abort_flag = 1; break; }
+      tc_fence_after_sync();
+      uint32_t v[128];
+      if (Q > 0) {
+        const uint32_t taddr = tmem + acc * p.BN + ((uint32_t)(32 * quad) << 16) + cbeg;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) tmem_ld_32x32b_x16(taddr + 16 * k, v + 16 * k);
+        tmem_ld_wait();
+      } else {
+#pragma unroll
+        for (int j = 0; j < 128; ++j) v[j] = 0u;
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tempty[acc]);      // the accumulator is free: the next tile's MMAs may start
+      if (p.kind_fp4 == 2) {
+#pragma unroll
+        for (int j = 0; j < 128; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * os);
+      }
+      const int cls_h = MODE == MQ_OP_FWD ? 0 : (int)fdiv((unsigned)tile.cls, p.sw, p.m_sw);
+      const int yo = MODE == MQ_OP_FWD ? tile.h : cls_h + p.sh * tile.h;
+      const int xo0 = MODE == MQ_OP_FWD ? tile.w0 : (tile.cls - cls_h * p.sw) + p.sw * tile.w0;
+#pragma unroll
+      for (int rd = 0; rd < 2; ++rd) {
+        const int c0 = cbeg + 64 * rd;
+        if (tile.c0 + c0 >= p.Cd) break;              // (a ragged last channel tile: nothing of this slice is inside the tensor)
+        if (lane == 0) bulk_wait_group_read<0>();      // the previous store has read the slice
+        __syncwarp();
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t* vv = v + 64 * rd + 16 * i;
+          if (!hwnc) {
+            float* bi = buf + (16 * i) * 32 + lane;
+#pragma unroll
+            for (int j = 0; j < 16; ++j) bi[j * 32] = __uint_as_float(vv[j]);
+          } else {
+            uint8_t* bg = reinterpret_cast<uint8_t*>(buf) + (i >> 1) * 4096 + hrow * 128;
+#pragma unroll
+            for (int u = 0; u < 4; ++u)
+              *reinterpret_cast<uint4*>(bg + ((((i & 1) * 4 + u) ^ (hrow & 7)) << 4)) = make_uint4(vv[4 * u], vv[4 * u + 1], vv[4 * u + 2], vv[4 * u + 3]);
+          }
+        }
+        fence_proxy_async_smem();
+        __syncwarp();
+        if (lane == 0) {
+          if (!hwnc) tma_store_4d(map_out, buf, xo0, tile.n0 + n_off, tile.c0 + c0, yo);
+          else {
+            tma_store_4d(map_out, buf, tile.c0 + c0, xo0, tile.n0 + n_off, yo);
+            tma_store_4d(map_out, buf + 1024, tile.c0 + c0 + 32, xo0, tile.n0 + n_off, yo);
+          }
+          bulk_commit_group();
+        }
+      }
+    }
+    if (lane == 0) bulk_wait_group_all();
+}
+
 // EPI: -1 = fp32 output (the three fp32 epilogue roles, chosen at run time: an instance per role was measured, no
 // change); 0..4 = quantizing epilogue emitting element format EPI
 // registers per thread of the epilogue warpgroups / of the others in the fp32-output kernels (16 warps, 128 per thread at launch)
-constexpr uint32_t EPI_REGS = 168, OTHER_REGS = 88;
+#ifndef MQ_EPI_REGS
+#define MQ_EPI_REGS 192
+#endif
+constexpr uint32_t EPI_REGS = MQ_EPI_REGS, OTHER_REGS = 256 - MQ_EPI_REGS;
 static_assert(2 * (EPI_REGS + OTHER_REGS) * 128 == 512 * 128, "the warpgroups' register budgets must add up to the launch's");
 
 template <int MODE, int KB, int KIND, int EPI = -1>
@@ -809,6 +892,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (EPI < 0) warpgroup_regs_inc<EPI_REGS>();
     if (EPI >= 0) epilogue_mx_role<MODE, EPI < 0 ? 0 : EPI>(p, mx_red, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else if (p.pair) epilogue_pair_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
+    else if (p.tma_store && p.BN == 256 && p.snap) epilogue_tma_snap_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else if (p.tma_store) epilogue_tma_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else if (p.BN == 256 && p.snap) epilogue_snap_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
