@@ -273,8 +273,18 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
             (!p.tma_store || p.max_stages >= env_int("MQ_TC_SNAP_MIN_STAGES", 4))) ? 1 : 0;
   const uint32_t fa = fp4 ? 1u : fmt_mma_code(fmt_x_like);   // kind::mxf4: 1 = E2M1; kind::mxf8f6f4: E4M3 0, E5M2 1, E2M3 3, E3M2 4
   const uint32_t fb = fp4 ? 1u : fmt_mma_code(fmt_w);
+  // pairs of blocks on 256 x 256 tiles (see conv_tc_kernel's DUO): tiles 2k and 2k + 1 must exist and share the channel tile
+  // (and have at least eight pipeline stages of MMAs per tile: 1x1 layers, four stages, measured 538-548 us without, 609 us with it)
+  p.duo = (p.snap && !p.halo && p.KB == 128 && p.classes == 1 && p.mma_cp && p.total_tiles % 2 == 0 &&
+           (p.tiles_w * p.tiles_h) % 2 == 0 && !fmt_is_6bit(fmt_x_like) && !fmt_is_6bit(fmt_w) && p.max_stages >= 8 && !env_int("MQ_TC_NO_DUO", 0)) ? 1 : 0;
+  if (p.duo) {   // half of the weight tile per block: a stage is 16 KB smaller, the ring two stages deeper
+    int st = (int)((227 * 1024 - 2048 - (p.tma_store ? 65536 : 0)) / (stage_bytes - (size_t)p.BN * 64));
+    if (st > 8) st = 8;
+    while (st > 2 && p.BN + sf_cols * st > 512) --st;
+    p.stages = st;
+  }
   // bit 23: scale type, 1 = E8M0, 0 = E4M3 (kind::mxf4nvf4)
-  p.idesc = (fa << 7) | (fb << 10) | ((uint32_t)(p.BN >> 3) << 17) | (ts16 ? 0u : (1u << 23)) | ((128u >> 4) << 24);
+  p.idesc = (fa << 7) | (fb << 10) | ((uint32_t)(p.BN >> 3) << 17) | (ts16 ? 0u : (1u << 23)) | (((p.duo ? 256u : 128u) >> 4) << 24);
   // whole-tile-per-stage variant: stride 1, one chunk per tap (<= 64 bytes of channels).  One box with the column
   // halo needs 8-column tiles; one box per column shift takes 8, 16 or 32 columns (longer NCHW store runs).
   p.halo = 0;
@@ -403,8 +413,16 @@ mq_status run_conv_tc(int op, const Geom& g, ConvTcPlan& pl, const mq_qtensor* q
     const uint64_t rb = (uint64_t)pl.rowbytes;
     const uint64_t dims[3] = {rb, (uint64_t)taps, (uint64_t)pl.rows_b};
     const uint64_t strides[2] = {rb, (uint64_t)taps * rb};
-    const uint32_t box[3] = {(uint32_t)p.KB, 1u, (uint32_t)p.BN};
+    const uint32_t box[3] = {(uint32_t)p.KB, 1u, (uint32_t)(p.duo ? p.BN / 2 : p.BN)};   // (a pair of blocks: each loads half of the tile's rows)
     if (!encode_tensor_map_u8(&map_w, b_codes, 3, dims, strides, box, nullptr, p.KB)) return MQ_ERR_CUDA;
+  }
+  CUtensorMap map_sfa = map_a, map_sfb = map_a;
+  if (p.duo) {   // the scale images as rows of 256 bytes: one box = the chunks of one stage
+    const uint32_t spa = p.kind_fp4 == 2 ? 4u : (p.kind_fp4 == 1 ? 2u : 1u), atoms_b = (uint32_t)(p.BN + 127) / 128;
+    const uint64_t da[2] = {256, (uint64_t)(conv_tc_sfa_bytes(p) / 256)}, db[2] = {256, (uint64_t)(conv_tc_sfb_bytes(p) / 256)}, st[1] = {256};
+    const uint32_t ba[2] = {256u, 2u * spa}, bb[2] = {256u, 2u * spa * atoms_b};
+    if (!encode_tensor_map_u8(&map_sfa, p.sfa_img, 2, da, st, ba, nullptr, 0)) return MQ_ERR_CUDA;
+    if (!encode_tensor_map_u8(&map_sfb, p.sfb_img, 2, db, st, bb, nullptr, 0)) return MQ_ERR_CUDA;
   }
   CUtensorMap map_out = map_a;
   if (p.tma_store) {
@@ -441,7 +459,7 @@ mq_status run_conv_tc(int op, const Geom& g, ConvTcPlan& pl, const mq_qtensor* q
     if ((pk_w ? launch_unpack6(b_unpacked, base + pl.off_pack_b, n, 0, fw, stream) : launch_pack6(b_unpacked, base + pl.off_pack_b, n, stream)) != cudaSuccess) return MQ_ERR_CUDA;
   }
   if (!(p.halo && p.fused) && launch_expand_conv_scales(p, stream) != cudaSuccess) return MQ_ERR_CUDA;
-  return launch_conv_tc(p, map_a, map_w, map_out, stream) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
+  return launch_conv_tc(p, map_a, map_w, map_out, stream, &map_sfa, &map_sfb) == cudaSuccess ? MQ_OK : MQ_ERR_CUDA;
 }
 
 // ---- weight gradient on tensor cores ---------------------------------------------------------------

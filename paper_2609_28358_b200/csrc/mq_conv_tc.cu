@@ -232,7 +232,7 @@ __device__ __forceinline__ void epilogue_role(const ConvTcParams& p, uint32_t tm
 // MMAs instead of holding them up.  The registers come from the loader / MMA warpgroups (warpgroup_regs_inc / _dec).
 template <int MODE>
 __device__ __forceinline__ void epilogue_snap_role(const ConvTcParams& p, uint32_t tmem, uint64_t* tfull, uint64_t* tempty, volatile int* abort_flag,
-                                                   int warp, int lane, unsigned total) {
+                                                   int warp, int lane, unsigned total, int leader_remote = 0) {
     const int quad = warp & 3;
     const int half = (warp - 4) >> 2;
     const int r = 32 * quad + lane;
@@ -264,7 +264,7 @@ __device__ __forceinline__ void epilogue_snap_role(const ConvTcParams& p, uint32
       }
       tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&tempty[acc]);      // the accumulator is free: the next tile's MMAs may start
+      if (lane == 0) release_acc(&tempty[acc], leader_remote);      // the accumulator is free: the next tile's MMAs may start
       int yo, xo;
       if (MODE == MQ_OP_FWD) { yo = tile.h; xo = tile.w0 + tw_; }
       else {
@@ -746,7 +746,8 @@ __device__ __forceinline__ void epilogue_tma_role(const ConvTcParams& p, const C
 // the accumulator back (see epilogue_snap_role), then stages and stores its two 64-channel slices from the registers.
 template <int MODE>
 __device__ __forceinline__ void epilogue_tma_snap_role(const ConvTcParams& p, const CUtensorMap* map_out, float* staging, uint32_t tmem,
-                                                       uint64_t* tfull, uint64_t* tempty, volatile int* abort_flag, int warp, int lane, unsigned total) {
+                                                       uint64_t* tfull, uint64_t* tempty, volatile int* abort_flag, int warp, int lane, unsigned total,
+                                                       int leader_remote = 0) {
     const int quad = warp & 3;
     const int half = (warp - 4) >> 2;
     const int cbeg = 128 * half;
@@ -779,7 +780,7 @@ __device__ __forceinline__ void epilogue_tma_snap_role(const ConvTcParams& p, co
       }
       tc_fence_before_sync();
       __syncwarp();
-      if (lane == 0) mbar_arrive(&tempty[acc]);      // the accumulator is free: the next tile's MMAs may start
+      if (lane == 0) release_acc(&tempty[acc], leader_remote);      // the accumulator is free: the next tile's MMAs may start
       if (p.kind_fp4 == 2) {
 #pragma unroll
         for (int j = 0; j < 128; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) * os);
@@ -831,10 +832,18 @@ __device__ __forceinline__ void epilogue_tma_snap_role(const ConvTcParams& p, co
 constexpr uint32_t EPI_REGS = MQ_EPI_REGS, OTHER_REGS = 256 - MQ_EPI_REGS;
 static_assert(2 * (EPI_REGS + OTHER_REGS) * 128 == 512 * 128, "the warpgroups' register budgets must add up to the launch's");
 
-template <int MODE, int KB, int KIND, int EPI = -1>
+// DUO: the two blocks of a cluster work on ONE 256 x 256 tile (cta_group::2): each loads the activation rows of its own
+// 128-row tile (tiles 2k and 2k + 1 of the round robin: same channel tile, neighbouring positions) and HALF of the weight
+// tile's 256 rows, so a stage brings 32 KB instead of 48 KB of operands into a block's shared memory - these GEMMs wait for
+// operands (E2M1) or run at the power cap (E4M3).  The leader's lane issues the scale copies, MMAs and commits for both
+// blocks; every copy of either block counts on the LEADER's stage barrier (its loaders announce both blocks' bytes); the
+// commits free the stage and publish the accumulator in both blocks; the peer's epilogue warps hand the accumulator back
+// on the leader's barrier.  map_sfa / map_sfb: the scale images as rows of 256 bytes (tiled copies can count on a barrier
+// of the other block, plain bulk copies cannot).
+template <int MODE, int KB, int KIND, int EPI = -1, bool DUO = false>
 __global__ void __launch_bounds__(tc_threads_of(EPI), 1)
 conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b, const __grid_constant__ CUtensorMap map_out,
-               const ConvTcParams p) {
+               const __grid_constant__ CUtensorMap map_sfa, const __grid_constant__ CUtensorMap map_sfb, const ConvTcParams p) {
   constexpr int G = 128 / KB;          // chunks per stage
   constexpr int APC = KB / 32;         // MMA K-atoms (32 bytes) per chunk
   constexpr bool FP4 = KIND != 0;
@@ -846,7 +855,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
 
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-  const int b_stage_bytes = p.BN * 128;
+  const int b_stage_bytes = (DUO ? p.BN / 2 : p.BN) * 128;    // (a pair of blocks: each holds half of the weight tile's rows)
   const int stage_bytes = A_STAGE_BYTES + b_stage_bytes + SFA_B + SFB_B;
   float* staging = reinterpret_cast<float*>(smem + (size_t)p.stages * stage_bytes);   // TMA-store epilogue only
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + (size_t)p.stages * stage_bytes + (p.tma_store ? EPI_STAGING_BYTES : 0));
@@ -863,21 +872,26 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   // are issued by one elected lane (around `if (lane == 0)` every operand of those instructions would first be moved
   // out of a per-thread register, which more than doubles the issuing thread's cycles per instruction).
   const int warp = __shfl_sync(0xffffffffu, (int)(threadIdx.x >> 5), 0), lane = threadIdx.x & 31;
+  const uint32_t rank = DUO ? __shfl_sync(0xffffffffu, cluster_ctarank(), 0) : 0u;   // 0: the pair's leader
   const int atoms_b = (p.BN + 127) / 128;
   const unsigned total = (unsigned)p.total_tiles;
 
   if (threadIdx.x == 0) {
     for (int s = 0; s < p.stages; ++s) { mbar_init(&full[s], 3); mbar_init(&empty[s], 1); mbar_init(&sffull[s], 1); }
-    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], EPI == 5 ? 16 : 8); }
+    for (int a = 0; a < 2; ++a) { mbar_init(&tfull[a], 1); mbar_init(&tempty[a], (EPI == 5 || DUO) ? 16 : 8); }
     *abort_flag = 0;
     mbar_fence_init();
     prefetch_tensormap(&map_a);
     prefetch_tensormap(&map_b);
     if (p.tma_store) prefetch_tensormap(&map_out);
   }
-  if (warp == 1) { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  if (warp == 1) {
+    if (DUO) { tmem_alloc_2(tmem_slot, 512); tmem_relinquish_2(); }
+    else { tmem_alloc(tmem_slot, 512); tmem_relinquish(); }
+  }
   tc_fence_before_sync();
   __syncthreads();
+  if (DUO) cluster_sync_all();   // both blocks' barriers and tensor memory exist before anything crosses over
   tc_fence_after_sync();
   const uint32_t tmem = *tmem_slot;
   pdl_wait();   // set-up above touched only shared memory, tensor memory and the kernel parameters
@@ -892,9 +906,9 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     if (EPI < 0) warpgroup_regs_inc<EPI_REGS>();
     if (EPI >= 0) epilogue_mx_role<MODE, EPI < 0 ? 0 : EPI>(p, mx_red, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else if (p.pair) epilogue_pair_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
-    else if (p.tma_store && p.BN == 256 && p.snap) epilogue_tma_snap_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total);
+    else if (p.tma_store && p.BN == 256 && p.snap) epilogue_tma_snap_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total, DUO && rank != 0);
     else if (p.tma_store) epilogue_tma_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total);
-    else if (p.BN == 256 && p.snap) epilogue_snap_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
+    else if (p.BN == 256 && p.snap) epilogue_snap_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total, DUO && rank != 0);
     else epilogue_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
   } else {
   if (EPI < 0) warpgroup_regs_dec<OTHER_REGS>();
@@ -907,7 +921,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     // stage's barrier with its own byte count.
     {
       uint32_t s = 0, phase = 0, gi = 0;
-      const uint32_t row_bytes = lkind == 1 ? (uint32_t)p.BN * KB : (p.a_tx34 ? 96u * KB : 128u * KB);
+      const uint32_t row_bytes = lkind == 1 ? (uint32_t)(DUO ? p.BN / 2 : p.BN) * KB : (p.a_tx34 ? 96u * KB : 128u * KB);
       for (unsigned i = 0, t; (t = tile_of_iter(p, i)) < total && !*abort_flag; ++i) {
         const Tile tile = decode_tile(p, t);
         TapWalk<MODE> tw;
@@ -941,6 +955,21 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             uint8_t* sa = smem + (size_t)s * stage_bytes;
             uint8_t* sb = sa + A_STAGE_BYTES;
             if (!mbar_wait(&empty[s], phase ^ 1, p.status, MQ_ERR_TIMEOUT)) { *abort_flag = 1; break; }
+            if (DUO) {
+              // both blocks' copies count on the leader's barrier; its loaders announce the bytes of both
+              if (elect_one()) {
+                const uint32_t lbar = cluster_addr_of(&full[s], 0);
+                if (lkind == 2) {
+                  if (rank == 0) mbar_arrive_expect_tx(&full[s], 2u * 512u * SPA * (1 + atoms_b));
+                  tma_load_2d_pair(sb + b_stage_bytes, &map_sfa, lbar, 0, (int)((sfa_src - p.sfa_img) >> 8));
+                  tma_load_2d_pair(sb + b_stage_bytes + SFA_B, &map_sfb, lbar, 0, (int)((sfb_src - p.sfb_img) >> 8));
+                } else {
+                  if (rank == 0) mbar_arrive_expect_tx(&full[s], 2u * row_bytes);
+                  if (lkind == 1) tma_load_3d_pair(sb, &map_b, lbar, c0[0], c1[0], tile.c0 + (int)rank * (p.BN / 2));
+                  else tma_load_4d_pair(sa, &map_a, lbar, c0[0], c1[0], tile.n0, c2[0]);
+                }
+              }
+            } else
             if (elect_one()) {
               if (lkind == 2) {
                 mbar_arrive_expect_tx(&full[s], 512u * SPA * (1 + atoms_b));
@@ -966,8 +995,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
       }
     }
   } else if (warp == 1) {
-    // ------------------------------------------------------------------ MMA issuer
-    {
+    // ------------------------------------------------------------------ MMA issuer (a pair of blocks: the leader's)
+    if (!DUO || rank == 0) {
       const uint64_t op_desc = smem_desc_base(16, 8 * KB, LAYOUT);
       const uint32_t sf_base = tmem + p.n_acc * p.BN;
       const uint32_t stage16 = (uint32_t)stage_bytes >> 4;
@@ -1003,7 +1032,14 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
           const uint32_t sfa_t = sf_base + s * SFC, sfb_t = sfa_t + SFB_OFF;
           const int natoms = min(G, Q - q0) * APC;
           if (elect_one()) {
-            if (self_cp) {
+            if (DUO) {
+#pragma unroll
+              for (int g = 0; g < SPA; ++g) {
+                tmem_cp_32x128b_warpx4_2(sfa_t + 4 * g, sfa_desc0 + so + g * 32);
+                tmem_cp_32x128b_warpx4_2(sfb_t + 4 * g * atoms_b, sfb_desc0 + so + g * atoms_b * 32);
+                tmem_cp_32x128b_warpx4_2(sfb_t + 4 * (g * atoms_b + 1), sfb_desc0 + so + (g * atoms_b + 1) * 32);
+              }
+            } else if (self_cp) {
 #pragma unroll
               for (int g = 0; g < SPA; ++g) {
                 tmem_cp_32x128b_warpx4(sfa_t + 4 * g, sfa_desc0 + so + g * 32);
@@ -1019,19 +1055,25 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                 const uint64_t ad = a_desc0 + so + c * ((128 * KB) >> 4) + ja * 2;
                 const uint64_t bd = b_desc0 + so + c * b_chunk16 + ja * 2;
                 const int g = (a * SPA) >> 2, id = (a * SPA) & 3;
-                if (KIND == 2) mma_nvf4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accu);
+                if (DUO && KIND == 2) mma_nvf4_2(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accu);
+                else if (DUO && KIND == 1) mma_mxf4_2(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accu);
+                else if (DUO) mma_mxf8f6f4_2(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accu);
+                else if (KIND == 2) mma_nvf4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accu);
                 else if (KIND == 1) mma_mxf4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accu);
                 else mma_mxf8f6f4(d_tmem, ad, bd, idesc_id[id], sfa_t + 4 * g, sfb_t + 4 * g * atoms_b, accu);
                 accu = 1;
               }
             }
-            tc_commit(&empty[s]);
+            if (DUO) tc_commit_2_multicast(&empty[s], 3); else tc_commit(&empty[s]);   // (a pair: frees the stage in both blocks)
           }
           __syncwarp();
           accumulate = 1;
           if (++s == (uint32_t)p.stages) { s = 0; phase ^= 1; }
         }
-        if (elect_one()) { if (Q > 0) tc_commit(&tfull[acc]); else mbar_arrive(&tfull[acc]); }
+        if (elect_one()) {
+          if (DUO) { if (Q > 0) tc_commit_2_multicast(&tfull[acc], 3); else { mbar_arrive(&tfull[acc]); mbar_arrive_remote(&tfull[acc], 1); } }
+          else if (Q > 0) tc_commit(&tfull[acc]); else mbar_arrive(&tfull[acc]);
+        }
         __syncwarp();
       }
     }
@@ -1077,7 +1119,8 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   // teardown: everyone meets here (all loops are bounded), then the allocating warp frees TMEM
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 1) tmem_dealloc(tmem, 512);
+  if (DUO) cluster_sync_all();   // nothing of the peer block is touched after this point
+  if (warp == 1) { if (DUO) tmem_dealloc_2(tmem, 512); else tmem_dealloc(tmem, 512); }
 }
 
 template <int BPC>
@@ -1863,24 +1906,30 @@ bool encode_tensor_map_p6(CUtensorMap* map, const void* base, int rank, const ui
 }
 
 size_t conv_tc_smem_bytes(const ConvTcParams& p) {
-  const size_t stage = A_STAGE_BYTES + (size_t)p.BN * 128 + (p.kind_fp4 == 2 ? SFA_BYTES_NV + SFB_BYTES_NV : SFA_BYTES + SFB_BYTES);
+  const size_t stage = A_STAGE_BYTES + (size_t)(p.duo ? p.BN / 2 : p.BN) * 128 + (p.kind_fp4 == 2 ? SFA_BYTES_NV + SFB_BYTES_NV : SFA_BYTES + SFB_BYTES);
   return 1024 + (size_t)p.stages * stage + (p.tma_store ? EPI_STAGING_BYTES : 0) + (3 * (size_t)p.stages + 4) * 8 + 64 + (p.mx_out ? 544 : 0);
 }
 
-template <int MODE, int KB, int FP4, int EPI = -1>
-cudaError_t launch_conv_tc_inst(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_out, cudaStream_t s) {
+template <int MODE, int KB, int FP4, int EPI = -1, bool DUO = false>
+cudaError_t launch_conv_tc_inst(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_b, const CUtensorMap& map_out, cudaStream_t s,
+                                const CUtensorMap* map_sfa = nullptr, const CUtensorMap* map_sfb = nullptr) {
   static bool attr_set = false;
   const size_t smem = conv_tc_smem_bytes(p);
   if (!attr_set) {
-    cudaError_t e = cudaFuncSetAttribute(conv_tc_kernel<MODE, KB, FP4, EPI>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
+    cudaError_t e = cudaFuncSetAttribute(conv_tc_kernel<MODE, KB, FP4, EPI, DUO>, cudaFuncAttributeMaxDynamicSharedMemorySize, 227 * 1024);
     if (e != cudaSuccess) return e;
     attr_set = true;
   }
   const int sms = sm_count();
   const long long units = p.pair ? p.total_tiles / 2 : p.total_tiles;
-  const unsigned grid = (unsigned)(units < sms ? units : sms);
+  unsigned grid = (unsigned)(units < sms ? units : sms);
   count_launches(1);
-  return launch_pdl(conv_tc_kernel<MODE, KB, FP4, EPI>, dim3(grid), dim3(tc_threads_of(EPI)), smem, s, map_a, map_b, map_out, p);
+  if (DUO) {   // clusters of two blocks; the tile count is even (the plan's condition), so is the grid
+    if (!map_sfa || !map_sfb) return cudaErrorInvalidValue;
+    grid &= ~1u;
+    return launch_pdl_cluster(conv_tc_kernel<MODE, KB, FP4, EPI, DUO>, dim3(grid), dim3(tc_threads_of(EPI)), smem, s, 2u, map_a, map_b, map_out, *map_sfa, *map_sfb, p);
+  }
+  return launch_pdl(conv_tc_kernel<MODE, KB, FP4, EPI, DUO>, dim3(grid), dim3(tc_threads_of(EPI)), smem, s, map_a, map_b, map_out, map_a, map_a, p);
 }
 
 size_t conv_tc_sfa_bytes(const ConvTcParams& p) {
@@ -2064,8 +2113,17 @@ cudaError_t launch_recode4_e4m3(const uint8_t* in, uint8_t* out, size_t n_out, c
   return launch_pdl(recode4_kernel, dim3((unsigned)blocks), dim3(256), 0, s, reinterpret_cast<const uint2*>(in), reinterpret_cast<uint4*>(out), nchunks);
 }
 
-cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_out, cudaStream_t s) {
+cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_out, cudaStream_t s,
+                           const CUtensorMap* map_sfa, const CUtensorMap* map_sfb) {
   if (p.total_tiles <= 0 || p.total_tiles > 0x7fffffffLL) return cudaErrorInvalidValue;
+  if (p.duo) {   // pairs of blocks on 256 x 256 tiles: fp32 output, 128-byte K chunks, 8-bit or MX E2M1 operands
+    if (p.halo || p.mx_out || p.KB != 128) return cudaErrorInvalidValue;
+#define MQ_TC_DUO_CASE(M, F) if (p.mode == M && p.kind_fp4 == F) return launch_conv_tc_inst<M, 128, F, -1, true>(p, map_a, map_w, map_out, s, map_sfa, map_sfb)
+    MQ_TC_DUO_CASE(MQ_OP_FWD, 0); MQ_TC_DUO_CASE(MQ_OP_FWD, 1); MQ_TC_DUO_CASE(MQ_OP_FWD, 2);
+    MQ_TC_DUO_CASE(MQ_OP_BWD_DATA, 0); MQ_TC_DUO_CASE(MQ_OP_BWD_DATA, 1); MQ_TC_DUO_CASE(MQ_OP_BWD_DATA, 2);
+#undef MQ_TC_DUO_CASE
+    return cudaErrorInvalidValue;
+  }
   if (p.halo) {
 #define MQ_TC_HCASE(M, K, F) if (p.mode == M && p.KB == K && p.kind_fp4 == (F ? 1 : 0)) return launch_conv_tc_halo_inst<M, K, F>(p, map_a, map_out, map_w, s)
     MQ_TC_HCASE(MQ_OP_FWD, 64, false); MQ_TC_HCASE(MQ_OP_FWD, 32, false); MQ_TC_HCASE(MQ_OP_FWD, 64, true); MQ_TC_HCASE(MQ_OP_FWD, 32, true);

@@ -52,6 +52,7 @@ struct ConvTcParams {
   // whole-tile-per-stage variant (small channel counts, stride 1): see conv_tc_halo_kernel
   int halo;                 // 1: use it
   int WH;                   // columns of the activation halo box = TW + Kw - 1
+  int duo;                  // 1: clusters of two blocks on 256 x 256 tiles (cta_group::2), each loading half of the weight tile
   int snap;                 // 1: 256-column tiles, direct fp32 stores: the epilogue copies the accumulator into registers and frees it before storing
   int a_tx34;               // 1: the activation boxes come from packed 6-bit storage - a box counts 3/4 of its shared-memory bytes on the barrier
   int halo_box_bytes;       // bytes of one activation box = Kh * TN * WH * KB
@@ -101,7 +102,9 @@ cudaError_t launch_unpack6(const uint8_t* in, uint8_t* out, size_t n_codes, int 
 cudaError_t launch_recode6_e4m3(const uint8_t* in, uint8_t* out, size_t nbytes, int fmt6, cudaStream_t s);
 // packed E2M1 codes (two per byte) -> the E4M3 codes of the same values, one per byte; n_out = elements = output bytes
 cudaError_t launch_recode4_e4m3(const uint8_t* in, uint8_t* out, size_t n_out, cudaStream_t s);
-cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_out, cudaStream_t s);
+// map_sfa, map_sfb: p.duo only - the two scale images as rows of 256 bytes (boxes of one stage's chunks)
+cudaError_t launch_conv_tc(const ConvTcParams& p, const CUtensorMap& map_a, const CUtensorMap& map_w, const CUtensorMap& map_out, cudaStream_t s,
+                           const CUtensorMap* map_sfa = nullptr, const CUtensorMap* map_sfb = nullptr);
 // Expands the compact tile scales into the per-stage scale-vector chunks the MMA reads (p.sfa_img, p.sfb_img).
 cudaError_t launch_expand_conv_scales(const ConvTcParams& p, cudaStream_t s);
 size_t conv_tc_sfa_bytes(const ConvTcParams& p);

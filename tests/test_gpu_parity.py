@@ -233,13 +233,25 @@ def test_6bit_gemms_on_cuda_cores(knobs):
 ALT_PATHS = [("MQ_TC_NO_HALO", "1"), ("MQ_TC_NO_FUSED", "1"), ("MQ_TC_NO_TMA_STORE", "1"), ("MQ_TC_TMA_STORE", "1"), ("MQ_TC_NO_PAIR", "1"),
              ("MQ_TC_BN", "256"), ("MQ_TC_TW", "4"), ("MQ_TC_TW", "16"), ("MQ_TC_TW", "32"), ("MQ_WGRAD_NO_FLAT", "1"),
              ("MQ_WGRAD_NO_GROUP", "1"), ("MQ_WGRAD_NO_GROUP8", "1"), ("MQ_WGRAD_N128", "1"), ("MQ_WGRAD_NO_CTA2", "1"), ("MQ_TC_NO_MMA_CP", "1"), ("MQ_WGRAD_MMA_CP", "1"), ("MQ_TC_FP4_BN128", "1"), ("MQ_TC_NO_SFA_DEDUP", "1"), ("MQ_TC_NO_WT_FUSED", "1"), ("MQ_WGRAD_FP4_PIXEL", "1"), ("MQ_WGRAD_SPLITS", "3"), ("MQ_DISABLE_TC_WGRAD", "1"), ("MQ_DISABLE_TC", "1"),
-             ("MQ_NO_PDL", "1"), ("MQ_QUANT_NO_R16", "1"), ("MQ_QUANT_TMA", "0"), ("MQ_WGRAD_NO_WIDE_PREP", "1"), ("MQ_WGRAD_NO_SFB_DEDUP", "1"), ("MQ_TC_NO_SNAP", "1")]
+             ("MQ_NO_PDL", "1"), ("MQ_QUANT_NO_R16", "1"), ("MQ_QUANT_TMA", "0"), ("MQ_WGRAD_NO_WIDE_PREP", "1"), ("MQ_WGRAD_NO_SFB_DEDUP", "1"), ("MQ_TC_NO_SNAP", "1"), ("MQ_TC_NO_DUO", "1")]
 ALT_SHAPES = [("thin", (32, 64, 8, 16, 96, 3, 1, 1)), ("wide_s2", (32, 256, 8, 12, 288, 3, 2, 1)), ("wide_s1", (32, 256, 4, 8, 288, 3, 1, 1)),
               ("thin32_s2", (40, 20, 9, 10, 48, 3, 2, 1))]
 # knobs that act on other shapes: at most 16 samples (quantizer items of 16 positions), 256 samples x 256 channels (the wide E2M1
 # weight-gradient preparation)
 ALT_EXTRA = {"MQ_QUANT_NO_R16": [("batch16", (16, 40, 10, 12, 72, 3, 1, 1))], "MQ_WGRAD_NO_WIDE_PREP": [("n256_c256", (256, 256, 4, 4, 256, 3, 1, 1))],
-             "MQ_TC_NO_SNAP": [("c512_bn256", (40, 512, 6, 7, 500, 3, 1, 1))]}
+             "MQ_TC_NO_SNAP": [("c512_bn256", (40, 512, 6, 7, 500, 3, 1, 1))],
+             "MQ_TC_NO_DUO": [("c512_pairs", (32, 512, 8, 8, 512, 3, 1, 1))]}
+
+
+@pytest.mark.parametrize("fmts", [(E4M3, E4M3, E5M2), (E2M1, E2M1, E2M1)], ids=["fp8", "fp4"])
+@pytest.mark.parametrize("name,shape", [("c512", (32, 512, 8, 8, 512, 3, 1, 1)), ("c256_ragged", (48, 256, 6, 12, 300, 3, 1, 1))], ids=["c512", "c256_ragged"])
+def test_block_pairs_on_256_column_tiles(name, shape, fmts):
+    """Forward and input gradient of layers with 256-column tiles, unit strides and an even tile count run as pairs of blocks
+    on 256 x 256 tiles (each block loads half of the weight tile): same parity bar, both output layouts."""
+    d = inputs.conv_desc(*shape)
+    ol = OracleLayer(make_layer(name, d, fmts, seed=29, kinds=("relu", "kaiming", "gauss")))
+    qs = check_quantize(ol)
+    check_convs(ol, qs, samples=30000, layouts=(mq.NCHW, mq.HWNC), ops=("fwd", "dx"))
 
 
 @pytest.mark.parametrize("knob", ALT_PATHS, ids=[f"{k}={v}" for k, v in ALT_PATHS])

@@ -27,6 +27,7 @@ SHAPES = [
     ("tc_c512_k1", (32, 512, 3, 4, 512, 1, 1, 0)),    # two 128-byte chunks per tap
     ("tc_n96", (96, 64, 6, 5, 128, 3, 1, 1)),         # three 32-sample tiles: the weight gradient's per-pixel mode (four K-blocks per pixel)
     ("tc_n24", (24, 128, 5, 5, 64, 3, 1, 1)),         # fewer than 32 samples: a half-empty sample tile
+    ("tc_c512_pairs", (32, 512, 4, 8, 512, 3, 1, 1)), # 256-column tiles in pairs of blocks (each loads half of the weight tile)
 ]
 
 
