@@ -269,7 +269,7 @@ bool conv_tc_plan(int op, const Geom& g, int fmt_x_like, int fmt_w, int layout, 
   // one 256-column accumulator: the epilogue copies it into registers and frees it before storing (with the staged TMA
   // stores only when a tile has at least MQ_TC_SNAP_MIN_STAGES pipeline stages of MMAs to overlap: E2M1 1x1 512 channels, two
   // stages per tile, measured 384-407 us without and 517-601 us with it; E4M3, four stages, 562-567 against 521 us)
-  p.snap = (!mx && p.BN == 256 && p.n_acc == 1 && !p.pair && !env_int("MQ_TC_NO_SNAP", 0) &&
+  p.snap = (!mx && ((p.BN == 256 && p.n_acc == 1 && !p.pair) || (p.pair && p.BN == 128)) && !env_int("MQ_TC_NO_SNAP", 0) &&
             (!p.tma_store || p.max_stages >= env_int("MQ_TC_SNAP_MIN_STAGES", 4))) ? 1 : 0;
   const uint32_t fa = fp4 ? 1u : fmt_mma_code(fmt_x_like);   // kind::mxf4: 1 = E2M1; kind::mxf8f6f4: E4M3 0, E5M2 1, E2M3 3, E3M2 4
   const uint32_t fb = fp4 ? 1u : fmt_mma_code(fmt_w);

@@ -358,6 +358,62 @@ __device__ __forceinline__ void epilogue_pair_role(const ConvTcParams& p, uint32
     }
 }
 
+// The same with the accumulators copied into registers first (128-column tiles: 2 x 64 columns per warp = 128 registers, see
+// epilogue_snap_role): both accumulators are handed back before the stores, which then run under the next pair's MMAs.
+template <int MODE>
+__device__ __forceinline__ void epilogue_pair_snap_role(const ConvTcParams& p, uint32_t tmem, uint64_t* tfull, uint64_t* tempty, volatile int* abort_flag,
+                                                        int warp, int lane, unsigned total) {
+    const int quad = warp & 3;
+    const int half = (warp - 4) >> 2;
+    const int r = 32 * quad + lane;
+    const int tw_ = r & (p.TW - 1), tn = r >> p.lgTW;
+    const int cbeg = 64 * half;
+    const long long cs = (long long)p.Hd * p.Wd;
+    const float os = out_scale_of(p);
+#pragma unroll 1
+    for (unsigned j = 0, t; (t = tile_of_iter(p, 2 * j)) < total && !*abort_flag; ++j) {
+      const Tile t0 = decode_tile(p, t), t1 = decode_tile(p, t + 1);
+      TapWalk<MODE> w0, w1;
+      w0.init(p, t0); w1.init(p, t1);
+      const int Q0 = w0.chunks(p), Q1 = w1.chunks(p);
+      bool ok = true;
+      if (lane == 0) ok = mbar_wait(&tfull[0], j & 1, p.status, MQ_ERR_TIMEOUT) && mbar_wait(&tfull[1], j & 1, p.status, MQ_ERR_TIMEOUT);
+      ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+      if (!ok) { *abort_flag = 1; break; }
+      tc_fence_after_sync();
+      uint32_t v0[64], v1[64];
+      const uint32_t taddr = tmem + ((uint32_t)(32 * quad) << 16) + cbeg;
+      if (Q0 > 0) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) tmem_ld_32x32b_x16(taddr + 16 * k, v0 + 16 * k);
+      }
+      if (Q1 > 0) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) tmem_ld_32x32b_x16(taddr + 128 + 16 * k, v1 + 16 * k);
+      }
+      tmem_ld_wait();
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) { mbar_arrive(&tempty[0]); mbar_arrive(&tempty[1]); }
+      const float s0 = Q0 > 0 ? os : 0.f, s1 = Q1 > 0 ? os : 0.f;     // (an accumulator without taps holds nothing of this tile)
+      const int ch = (int)fdiv((unsigned)t0.cls, p.sw, p.m_sw);
+      const int yo = ch + p.sh * t0.h, xo = p.sw * (t0.w0 + tw_);     // even column; the odd class writes xo + 1
+      const int n = t0.n0 + tn;
+      if (!(yo < p.Hd && xo < p.Wd && n < p.N)) continue;            // Wd is even in this mode: xo + 1 < Wd as well
+      const int ncols = min(64, p.Cd - t0.c0 - cbeg);
+      float* o = p.out + (((long long)n * p.Cd + t0.c0 + cbeg) * p.Hd + yo) * p.Wd + xo;
+      const bool plain = p.kind_fp4 != 2 && Q0 > 0 && Q1 > 0;
+#pragma unroll
+      for (int q = 0; q < 64; ++q) {
+        if (q < ncols) {
+          if (plain) *reinterpret_cast<float2*>(o) = make_float2(__uint_as_float(v0[q]), __uint_as_float(v1[q]));
+          else *reinterpret_cast<float2*>(o) = make_float2(Q0 > 0 ? __uint_as_float(v0[q]) * s0 : 0.f, Q1 > 0 ? __uint_as_float(v1[q]) * s1 : 0.f);
+        }
+        o += cs;
+      }
+    }
+}
+
 // Quantizing epilogue (warps 4-11): the producer applies the activation and emits the NEXT tensor's stored MX form -
 // codes [Hd][Wd][N][Cp] and one E8M0 byte per 32-sample x 32-channel tile at a pixel - instead of fp32, i.e. the
 // tensor is quantized on chip before it is stored and the fp32 round trip through HBM disappears.  Tiles are TW <= 4
@@ -905,6 +961,7 @@ conv_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
   if ((warp >= 4 && warp < 12) || warp >= 16) {
     if (EPI < 0) warpgroup_regs_inc<EPI_REGS>();
     if (EPI >= 0) epilogue_mx_role<MODE, EPI < 0 ? 0 : EPI>(p, mx_red, tmem, tfull, tempty, abort_flag, warp, lane, total);
+    else if (p.pair && p.BN == 128 && p.snap) epilogue_pair_snap_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else if (p.pair) epilogue_pair_role<MODE>(p, tmem, tfull, tempty, abort_flag, warp, lane, total);
     else if (p.tma_store && p.BN == 256 && p.snap) epilogue_tma_snap_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total, DUO && rank != 0);
     else if (p.tma_store) epilogue_tma_role<MODE>(p, &map_out, staging, tmem, tfull, tempty, abort_flag, warp, lane, total);
