@@ -421,10 +421,12 @@ def run_ours(args):
     ms_step = ms_total / K
     value = flops / (ms_step * 1e-3) / 1e12
 
-    # ---- roofline of the dominant kernel: the call with the largest time per launched kernel
+    # ---- roofline of the dominant kernel
     pk, pk_src = peaks()
     kern, qi = roofline_table(wl, per_ms, n_launch, pk)
-    dom = max(CALLS, key=lambda n: kern[n]["ms"] / n_launch[n])
+    # the dominant kernel = the main kernel of the call that takes longest (a GEMM call's other launch, the expansion of its
+    # scale chunks, is a few microseconds; the call's whole time is charged to the main kernel)
+    dom = max(CALLS, key=lambda n: kern[n]["ms"])
     roof = {k: kern[dom][k] for k in ("bound", "achieved", "peak", "unit", "frac", "frac_of_published")}
     traffic = NCU_TRAFFIC.get((args.workload, dom))
     roof.update({"kernel": dom,
