@@ -50,11 +50,11 @@ CALLS = ("quantize_x", "quantize_w", "quantize_dy", "cbf_im2col", "conv_fwd", "c
 # of the captured one, traffic being proportional to the units processed).
 NCU_TRAFFIC = {
     # (bench workload, call): (captured workload, bytes per launch there, scale)
-    ("cfg5_e4m3_k3s1_c512_hw56", "conv_fwd"): ("cfg5_e4m3_k3s1_c512_hw28", 120224512 + 358202112, 4.0),       # conv_tc_kernel<fwd>
-    ("cfg5_e4m3_k3s1_c512_hw56", "conv_bwd_data"): ("cfg5_e4m3_k3s1_c512_hw28", 119526656 + 357814528, 4.0),  # conv_tc_kernel<bwd_data>
+    ("cfg5_e4m3_k3s1_c512_hw56", "conv_fwd"): ("cfg5_e4m3_k3s1_c512_hw28", 117502208 + 356616960, 4.0),       # conv_tc_kernel<fwd>
+    ("cfg5_e4m3_k3s1_c512_hw56", "conv_bwd_data"): ("cfg5_e4m3_k3s1_c512_hw28", 117229568 + 356492544, 4.0),  # conv_tc_kernel<bwd_data>
     ("cfg5_e4m3_k3s1_c512_hw56", "quantize_x"): ("cfg5_e4m3_k3s1_c512_hw28", 420059648 + 81590016, 4.0),      # quantize_tma_kernel
     ("cfg5_e4m3_k3s1_c512_hw56", "quantize_dy"): ("cfg5_e4m3_k3s1_c512_hw28", 423871488 + 81877248, 4.0),
-    ("cfg5_e4m3_k3s1_c512_hw28", "conv_fwd"): ("cfg5_e4m3_k3s1_c512_hw28", 120224512 + 358202112, 1.0),
+    ("cfg5_e4m3_k3s1_c512_hw28", "conv_fwd"): ("cfg5_e4m3_k3s1_c512_hw28", 117502208 + 356616960, 1.0),
 }
 
 
