@@ -15,7 +15,10 @@
 //   warp 1        MMA issuer: the stage's scale copies smem -> TMEM (tcgen05.cp), then its MMAs
 //   warp 2        scale copier (E2M1 with the separate-copier option only)
 //   warps 4-11    epilogue: TMEM -> registers -> global (fp32) or a staged TMA store, overlapped with the next tile's
-//                 main loop when a second accumulator fits; two warps per TMEM lane quadrant, half of the columns each
+//                 main loop: a second accumulator where it fits; 256-column tiles (one accumulator) are copied whole into
+//                 registers and handed back before the stores (fp32 output: these two warpgroups take registers from the
+//                 other two with setmaxnreg); two warps per TMEM lane quadrant, half of the columns each
+// Wide layers run the DUO instance: clusters of two blocks on 256 x 256 tiles (cta_group::2), see conv_tc_kernel.
 // A pipeline stage holds 128 bytes of K per row (four MMAs): one 128-byte box, or 128/KB boxes of KB
 // bytes when a tap has fewer than 128 bytes of channels (then several taps share a stage).
 // Every wait is bounded; on expiry the kernel records MQ_ERR_TIMEOUT in the status word and drains.
